@@ -1,0 +1,296 @@
+/*
+ * CPU oracle for Attention Pruning's compute path.  TEST INFRASTRUCTURE ONLY.
+ *
+ * Plain, slow, fp64 restatement of what the CUDA library computes, written from
+ * the paper's equations.  It shares no code with the CUDA path and must never be
+ * called from it: only the test-suite, the smoke check and the CPU-baseline leg
+ * of the benchmark may load this file.
+ *
+ *   oracle_accumulate      Eq. 1 (the element-wise sum of softmax attention
+ *                          matrices over samples; the 1/n factor is left to the
+ *                          caller, see below) with the attention matrix of
+ *                          Section 3.1, softmax(Q K^T / sqrt(d_k)).
+ *   oracle_build_mask      Eq. 2 read as an exact top-k selection per head.
+ *   oracle_mask_to_tiles   the 128x128 tile list + bitmaps (an encoding of the
+ *                          mask of Eq. 2; no counterpart in the paper).
+ *   oracle_attention_fwd   the masked attention equation of Section 3.2,
+ *                          softmax((Q K^T + M_p)/sqrt(d_k)) V with M_p = -inf
+ *                          on pruned entries.
+ *
+ * Parity status: every function here is pinned by tests that do not go through
+ * this file's own formulas (library SDPA, closed forms, brute force, invariants,
+ * a hand-computed 4x4 example).  The one thing that cannot be pinned is whether
+ * the synthetic masks look like masks of the paper's trained models: parity
+ * unpinned for mask realism (no weights, no datasets).
+ *
+ * Inputs are float arrays holding the exact values the GPU receives (bf16 or
+ * fp32 values widened to float); all arithmetic below is double.
+ * OpenMP is used over independent (batch, head) units only.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define AP_TILE 128
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+/* Row domain: all keys, or keys j <= i under the causal constraint. */
+static int row_domain_end(int i, int Lk, int causal) {
+  if (!causal) return Lk;
+  return (i + 1 < Lk) ? i + 1 : Lk;
+}
+
+/*
+ * Eq. 1 without the 1/n factor, one row (h, i) of the accumulator.  For every
+ * sample b:
+ *   s_j = (q_i . k_j) * scale + bias[h,i,j]       for j in the row's domain
+ *   p_j = exp(s_j - max_j s) / sum_j exp(s_j - max_j s)
+ *   arow[j] += p_j
+ * Entries outside the domain are never touched.  `bias` may be NULL.
+ * Samples are added in ascending b.  The raw sum is kept: dividing by n would
+ * not change which entries are largest.
+ */
+static void accumulate_row(double *arow, const float *Q, const float *K, const float *bias, int h,
+                           int i, int B, int H, int Lq, int Lk, int d, int causal, double scale) {
+  int jend = row_domain_end(i, Lk, causal);
+  double *s = (double *)malloc(sizeof(double) * (size_t)(jend > 0 ? jend : 1));
+  for (int b = 0; b < B; ++b) {
+    const float *q = Q + (((size_t)b * H + h) * Lq + i) * d;
+    const float *Kh = K + ((size_t)b * H + h) * (size_t)Lk * d;
+    double m = -INFINITY;
+    for (int j = 0; j < jend; ++j) {
+      double dot = 0.0;
+      for (int t = 0; t < d; ++t) dot += (double)q[t] * (double)Kh[(size_t)j * d + t];
+      double v = dot * scale;
+      if (bias) v += (double)bias[((size_t)h * Lq + i) * Lk + j];
+      s[j] = v;
+      if (v > m) m = v;
+    }
+    double z = 0.0;
+    for (int j = 0; j < jend; ++j) {
+      s[j] = exp(s[j] - m);
+      z += s[j];
+    }
+    for (int j = 0; j < jend; ++j) arow[j] += s[j] / z;
+  }
+  free(s);
+}
+
+/* Eq. 1 (sum form) for every head and row: acc[H,Lq,Lk] += sum_b softmax rows. */
+void oracle_accumulate(double *acc, const float *Q, const float *K, const float *bias, int B,
+                       int H, int Lq, int Lk, int d, int causal, double scale) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int hi = 0; hi < H * Lq; ++hi) {
+    int h = hi / Lq, i = hi % Lq;
+    accumulate_row(acc + ((size_t)h * Lq + i) * Lk, Q, K, bias, h, i, B, H, Lq, Lk, d, causal,
+                   scale);
+  }
+}
+
+/*
+ * The same for a sample of rows, for sizes where all rows take too long:
+ * rows[r] = (h, i) pairs, out[r, 0..Lk) += the row's sum (out is not cleared).
+ */
+void oracle_accumulate_rows(double *out, const int32_t *rows, int n_rows, const float *Q,
+                            const float *K, const float *bias, int B, int H, int Lq, int Lk, int d,
+                            int causal, double scale) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int r = 0; r < n_rows; ++r)
+    accumulate_row(out + (size_t)r * Lk, Q, K, bias, rows[2 * r], rows[2 * r + 1], B, H, Lq, Lk, d,
+                   causal, scale);
+}
+
+/* One candidate of the selection in Eq. 2. */
+typedef struct {
+  float value;
+  int32_t forced;
+  int64_t index; /* i * Lk + j */
+} ap_entry;
+
+/* forced first, then larger value first (compared as fp32), then lower index. */
+static int entry_before(const void *pa, const void *pb) {
+  const ap_entry *a = (const ap_entry *)pa, *b = (const ap_entry *)pb;
+  if (a->forced != b->forced) return b->forced - a->forced;
+  if (a->value > b->value) return -1;
+  if (a->value < b->value) return 1;
+  if (a->index < b->index) return -1;
+  if (a->index > b->index) return 1;
+  return 0;
+}
+
+/* Number of entries to keep out of n_valid, rounded half up in double. */
+int64_t oracle_keep_count(int64_t n_valid, int64_t n_forced, double keep_frac) {
+  int64_t k = (int64_t)floor(keep_frac * (double)n_valid + 0.5);
+  if (k > n_valid) k = n_valid;
+  if (k < n_forced) k = n_forced;
+  return k;
+}
+
+/*
+ * Eq. 2 as an exact per-head top-k: an entry is pruned (M_p = -inf) iff it does
+ * not belong to the k largest entries of the head's average attention matrix.
+ *   domain   all (i,j), or j <= i when causal
+ *   forced   the diagonal, when keep_diag and Lq == Lk
+ *   k        max(|forced|, min(n_valid, floor(keep_frac * n_valid + 0.5)))
+ *   order    forced first, value descending (as fp32), index i*Lk+j ascending
+ * mask[h,i,j] = 1 for the first k entries in that order, 0 elsewhere;
+ * nnz[h] = k.  Returns 0, or -1 when an allocation fails.
+ */
+int oracle_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal,
+                      int keep_diag, uint8_t *mask, int64_t *nnz) {
+  int failed = 0;
+  memset(mask, 0, (size_t)H * Lq * Lk);
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int h = 0; h < H; ++h) {
+    int64_t n_valid = 0;
+    for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lk, causal);
+    ap_entry *e = (ap_entry *)malloc(sizeof(ap_entry) * (size_t)(n_valid > 0 ? n_valid : 1));
+    if (!e) {
+      failed = 1;
+      continue;
+    }
+    int64_t n = 0, n_forced = 0;
+    for (int i = 0; i < Lq; ++i) {
+      int jend = row_domain_end(i, Lk, causal);
+      for (int j = 0; j < jend; ++j) {
+        e[n].value = acc[((size_t)h * Lq + i) * Lk + j];
+        e[n].forced = (keep_diag && Lq == Lk && i == j) ? 1 : 0;
+        e[n].index = (int64_t)i * Lk + j;
+        n_forced += e[n].forced;
+        ++n;
+      }
+    }
+    int64_t k = oracle_keep_count(n_valid, n_forced, keep_frac);
+    qsort(e, (size_t)n, sizeof(ap_entry), entry_before);
+    for (int64_t r = 0; r < k; ++r) mask[(size_t)h * Lq * Lk + (size_t)e[r].index] = 1;
+    nnz[h] = k;
+    free(e);
+  }
+  return failed ? -1 : 0;
+}
+
+/*
+ * Tile encoding of a mask.  Rows of the list are (h, qt) in ascending order;
+ * inside a row the key tiles kt are ascending and only tiles with at least one
+ * kept entry appear.  bitmap[t][r][w] bit c (LSB first) is entry
+ * (128*qt + r, 128*kt + 32*w + c); flags[t] bit 0 says all 128*128 bits are set.
+ * Returns the number of tiles, or -1 if it exceeds `cap`.
+ */
+int64_t oracle_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, int32_t *row_ptr,
+                             int32_t *col_idx, uint8_t *flags, uint32_t *bitmap, int64_t cap) {
+  int n_qt = (Lq + AP_TILE - 1) / AP_TILE, n_kt = (Lk + AP_TILE - 1) / AP_TILE;
+  int64_t t = 0;
+  row_ptr[0] = 0;
+  for (int h = 0; h < H; ++h) {
+    for (int qt = 0; qt < n_qt; ++qt) {
+      for (int kt = 0; kt < n_kt; ++kt) {
+        uint32_t words[AP_TILE][4];
+        int64_t count = 0;
+        memset(words, 0, sizeof(words));
+        for (int r = 0; r < AP_TILE; ++r) {
+          int i = qt * AP_TILE + r;
+          if (i >= Lq) break;
+          for (int c = 0; c < AP_TILE; ++c) {
+            int j = kt * AP_TILE + c;
+            if (j >= Lk) break;
+            if (mask[((size_t)h * Lq + i) * Lk + j]) {
+              words[r][c >> 5] |= 1u << (c & 31);
+              ++count;
+            }
+          }
+        }
+        if (count == 0) continue;
+        if (t >= cap) return -1;
+        col_idx[t] = kt;
+        flags[t] = (count == (int64_t)AP_TILE * AP_TILE) ? 1 : 0;
+        memcpy(bitmap + (size_t)t * AP_TILE * 4, words, sizeof(words));
+        ++t;
+      }
+      row_ptr[h * n_qt + qt + 1] = (int32_t)t;
+    }
+  }
+  return t;
+}
+
+/*
+ * Masked attention (Section 3.2), one output row.  With M_p = -inf on pruned
+ * entries, row i of the output is the softmax-weighted mean of v_j over the
+ * kept keys j only:
+ *   J = { j : mrow[j] = 1 },  s_j = (q . k_j) * scale,  w_j = exp(s_j - max_J s)
+ *   o = sum_J w_j v_j / sum_J w_j,   and exactly 0 when J is empty.
+ */
+static void attention_row(double *o, const float *q, const float *Kh, const float *Vh,
+                          const uint8_t *mrow, int Lk, int d, double scale) {
+  double *s = (double *)malloc(sizeof(double) * (size_t)Lk);
+  double m = -INFINITY, z = 0.0;
+  int any = 0;
+  for (int t = 0; t < d; ++t) o[t] = 0.0;
+  for (int j = 0; j < Lk; ++j) {
+    if (!mrow[j]) continue;
+    double dot = 0.0;
+    for (int t = 0; t < d; ++t) dot += (double)q[t] * (double)Kh[(size_t)j * d + t];
+    s[j] = dot * scale;
+    if (s[j] > m) m = s[j];
+    any = 1;
+  }
+  if (any) {
+    for (int j = 0; j < Lk; ++j) {
+      if (!mrow[j]) continue;
+      double w = exp(s[j] - m);
+      z += w;
+      for (int t = 0; t < d; ++t) o[t] += w * (double)Vh[(size_t)j * d + t];
+    }
+    for (int t = 0; t < d; ++t) o[t] /= z;
+  }
+  free(s);
+}
+
+/* Masked attention for all rows: Q[B,H,Lq,d], K,V[B,H,Lk,d], mask[H,Lq,Lk] -> O[B,H,Lq,d]. */
+void oracle_attention_fwd(const float *Q, const float *K, const float *V, const uint8_t *mask,
+                          double *O, int B, int H, int Lq, int Lk, int d, double scale) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int bh = 0; bh < B * H; ++bh) {
+    int h = bh % H;
+    for (int i = 0; i < Lq; ++i)
+      attention_row(O + ((size_t)bh * Lq + i) * d, Q + ((size_t)bh * Lq + i) * d,
+                    K + (size_t)bh * Lk * d, V + (size_t)bh * Lk * d,
+                    mask + ((size_t)h * Lq + i) * Lk, Lk, d, scale);
+  }
+}
+
+/*
+ * The same for a sample of output rows, for sizes where all rows take too long:
+ * rows[r] = (b, h, i) triples, out[r, 0..d).
+ */
+void oracle_attention_rows(const float *Q, const float *K, const float *V, const uint8_t *mask,
+                           double *out, const int32_t *rows, int n_rows, int B, int H, int Lq,
+                           int Lk, int d, double scale) {
+  (void)B;
+#pragma omp parallel for schedule(dynamic, 8)
+  for (int r = 0; r < n_rows; ++r) {
+    int b = rows[3 * r], h = rows[3 * r + 1], i = rows[3 * r + 2];
+    size_t bh = (size_t)b * H + h;
+    attention_row(out + (size_t)r * d, Q + (bh * Lq + i) * d, K + bh * (size_t)Lk * d,
+                  V + bh * (size_t)Lk * d, mask + ((size_t)h * Lq + i) * Lk, Lk, d, scale);
+  }
+}

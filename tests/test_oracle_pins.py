@@ -1,0 +1,435 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+Library routines (torch SDPA / softmax in fp64), closed forms, invariants, brute
+force on tiny sizes and a hand-computed 4x4 example.  Chosen so that a dropped
+term, a wrong sign or index, or a transposed operand in the oracle fails at
+least one test.  No GPU needed.
+"""
+import itertools
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ap_oracle as orc
+from paper_2012_02030_b200 import inputs, metrics
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "hand_4x4.txt")
+
+
+def _golden():
+    out = {}
+    for line in open(GOLDEN):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, *vals = line.split()
+        out[key] = np.array([float(v) for v in vals], dtype=np.float64).reshape(4, 4)
+    return out
+
+
+def _rand(shape, seed, dtype=torch.bfloat16):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn(shape, generator=g).to(dtype).to(torch.float32)
+
+
+# --------------------------------------------------------------------------- forward
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("shape", [(2, 3, 37, 37, 16), (1, 2, 130, 130, 64), (1, 1, 20, 45, 8)])
+def test_fwd_all_kept_equals_library_sdpa(shape, causal):
+    """Zero mask matrix (nothing pruned) gives the original attention (Section 3.2)."""
+    B, H, Lq, Lk, d = shape
+    if causal and Lq != Lk:
+        pytest.skip("causal needs Lq == Lk")
+    q, k, v = _rand((B, H, Lq, d), 1), _rand((B, H, Lk, d), 2), _rand((B, H, Lk, d), 3)
+    mask = torch.ones((H, Lq, Lk), dtype=torch.uint8)
+    if causal:
+        mask = torch.tril(mask)
+    got = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy())
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q.double(), k.double(), v.double(), is_causal=causal)
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-12, atol=1e-13)
+
+
+def test_fwd_random_mask_equals_library_masked_softmax():
+    """Additive -inf mask inside a library softmax (the paper's own implementation
+    route: a large negative value added before the softmax)."""
+    B, H, Lq, Lk, d = 2, 2, 50, 70, 16
+    q, k, v = _rand((B, H, Lq, d), 4), _rand((B, H, Lk, d), 5), _rand((B, H, Lk, d), 6)
+    mask = inputs.random_mask(H, Lq, Lk, 0.3, seed=7)
+    mask[:, :, 0] = 1  # no empty rows here
+    s = torch.einsum("bhid,bhjd->bhij", q.double(), k.double()) / math.sqrt(d)
+    s = s.masked_fill(mask.bool().unsqueeze(0) == 0, float("-inf"))
+    ref = torch.softmax(s, dim=-1) @ v.double()
+    got = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy())
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-12, atol=1e-13)
+
+
+def test_fwd_custom_scale_and_rows_sampler():
+    B, H, L, d = 2, 2, 33, 8
+    q, k, v = _rand((B, H, L, d), 8), _rand((B, H, L, d), 9), _rand((B, H, L, d), 10)
+    mask = inputs.random_mask(H, L, L, 0.5, seed=11)
+    full = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy(), scale=0.37)
+    s = torch.einsum("bhid,bhjd->bhij", q.double(), k.double()) * 0.37
+    s = s.masked_fill(mask.bool().unsqueeze(0) == 0, float("-inf"))
+    ref = torch.nan_to_num(torch.softmax(s, dim=-1), nan=0.0) @ v.double()
+    np.testing.assert_allclose(full, ref.numpy(), rtol=1e-12, atol=1e-13)
+    rows = [(b, h, i) for b in range(B) for h in range(H) for i in (0, 5, 32)]
+    some = orc.attention_rows(q.numpy(), k.numpy(), v.numpy(), mask.numpy(), rows, scale=0.37)
+    for r, (b, h, i) in enumerate(rows):
+        np.testing.assert_array_equal(some[r], full[b, h, i])
+
+
+def test_fwd_one_kept_entry_copies_value_row():
+    B, H, L, d = 2, 2, 19, 8
+    q, k, v = _rand((B, H, L, d), 12), _rand((B, H, L, d), 13), _rand((B, H, L, d), 14)
+    g = torch.Generator().manual_seed(15)
+    cols = torch.randint(0, L, (H, L), generator=g)
+    mask = torch.zeros((H, L, L), dtype=torch.uint8)
+    mask.scatter_(2, cols.unsqueeze(-1), 1)
+    got = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy())
+    for h in range(H):
+        for i in range(L):
+            np.testing.assert_array_equal(got[:, h, i], v[:, h, cols[h, i]].double().numpy())
+    eye = torch.eye(L, dtype=torch.uint8).expand(H, L, L)
+    got = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), eye.numpy())
+    np.testing.assert_array_equal(got, v.double().numpy())
+
+
+def test_fwd_zero_queries_give_plain_mean_and_empty_rows_zero():
+    B, H, L, d = 1, 2, 23, 8
+    k, v = _rand((B, H, L, d), 16), _rand((B, H, L, d), 17)
+    q = torch.zeros((B, H, L, d))
+    mask = inputs.random_mask(H, L, L, 0.4, seed=18, empty_rows=(3, 22))
+    got = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy())
+    m = mask.double()
+    cnt = m.sum(-1, keepdim=True)
+    ref = (m.unsqueeze(0) @ v.double()) / cnt.clamp(min=1)
+    np.testing.assert_allclose(got, ref.numpy(), rtol=1e-13, atol=1e-14)
+    assert np.all(got[:, :, 3] == 0.0) and np.all(got[:, :, 22] == 0.0)
+
+
+def test_fwd_key_shift_and_permutation_invariance():
+    B, H, L, d = 1, 2, 29, 8
+    q, k, v = _rand((B, H, L, d), 19), _rand((B, H, L, d), 20), _rand((B, H, L, d), 21)
+    mask = inputs.random_mask(H, L, L, 0.5, seed=22)
+    base = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy())
+    shift = torch.tensor([1.0, -2.0, 0.5, 0.25, -1.0, 2.0, 4.0, -0.5])  # exact in fp32
+    got = orc.attention_fwd(q.numpy(), (k + shift).numpy(), v.numpy(), mask.numpy())
+    np.testing.assert_allclose(got, base, rtol=1e-10, atol=1e-12)
+    perm = torch.randperm(L, generator=torch.Generator().manual_seed(23))
+    got = orc.attention_fwd(q.numpy(), k[:, :, perm].numpy(), v[:, :, perm].numpy(),
+                            mask[:, :, perm].numpy())
+    np.testing.assert_allclose(got, base, rtol=1e-12, atol=1e-13)
+
+
+def test_fwd_weights_sum_to_one_over_kept_entries():
+    """With V = identity the output is the weight matrix itself."""
+    H, L = 2, 24
+    q, k = _rand((1, H, L, L), 24), _rand((1, H, L, L), 25)
+    v = torch.eye(L).expand(1, H, L, L).contiguous()
+    mask = inputs.random_mask(H, L, L, 0.3, seed=26, empty_rows=(7,))
+    w = orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy())[0]
+    assert np.all(w[mask.numpy() == 0] == 0.0)
+    sums = w.sum(-1)
+    has = mask.numpy().sum(-1) > 0
+    np.testing.assert_allclose(sums[has], 1.0, rtol=0, atol=1e-14)
+    assert np.all(sums[~has] == 0.0)
+    assert np.all(w >= 0)
+
+
+# ------------------------------------------------------------------------ accumulate
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("with_bias", [False, True])
+def test_acc_equals_library_softmax_sum(causal, with_bias):
+    B, H, L, d = 3, 2, 41, 16
+    q, k = _rand((B, H, L, d), 30), _rand((B, H, L, d), 31)
+    bias = _rand((H, L, L), 32, torch.float32) if with_bias else None
+    acc = np.zeros((H, L, L))
+    orc.accumulate(acc, q.numpy(), k.numpy(), None if bias is None else bias.numpy(), causal=causal)
+    s = torch.einsum("bhid,bhjd->bhij", q.double(), k.double()) / math.sqrt(d)
+    if with_bias:
+        s = s + bias.double()
+    if causal:
+        s = s.masked_fill(~torch.tril(torch.ones(L, L, dtype=torch.bool)), float("-inf"))
+    ref = torch.softmax(s, dim=-1).sum(0)
+    np.testing.assert_allclose(acc, ref.numpy(), rtol=1e-12, atol=1e-14)
+    if causal:
+        assert np.all(acc[:, ~np.tril(np.ones((L, L), dtype=bool))] == 0.0)
+    # calling again continues the running sum (Eq. 1 is a plain sum over samples)
+    orc.accumulate(acc, q.numpy(), k.numpy(), None if bias is None else bias.numpy(), causal=causal)
+    np.testing.assert_allclose(acc, 2 * ref.numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_acc_rows_sum_to_sample_count_and_rect_shapes():
+    B, H, Lq, Lk, d = 5, 2, 17, 33, 8
+    q, k = _rand((B, H, Lq, d), 33), _rand((B, H, Lk, d), 34)
+    acc = np.zeros((H, Lq, Lk))
+    orc.accumulate(acc, q.numpy(), k.numpy())
+    np.testing.assert_allclose(acc.sum(-1), B, rtol=1e-13)
+    s = torch.einsum("bhid,bhjd->bhij", q.double(), k.double()) / math.sqrt(d)
+    np.testing.assert_allclose(acc, torch.softmax(s, -1).sum(0).numpy(), rtol=1e-12, atol=1e-14)
+    rows = [(0, 0), (1, 16), (1, 3)]
+    got = orc.accumulate_rows(rows, q.numpy(), k.numpy())
+    for r, (h, i) in enumerate(rows):
+        np.testing.assert_array_equal(got[r], acc[h, i])
+
+
+def test_acc_zero_queries_closed_form():
+    B, H, L, d = 4, 1, 12, 8
+    k = _rand((B, H, L, d), 35)
+    q = torch.zeros((B, H, L, d))
+    acc = np.zeros((H, L, L))
+    orc.accumulate(acc, q.numpy(), k.numpy())
+    np.testing.assert_allclose(acc, B / L, rtol=1e-15)
+    acc = np.zeros((H, L, L))
+    orc.accumulate(acc, q.numpy(), k.numpy(), causal=True)
+    for i in range(L):
+        np.testing.assert_allclose(acc[0, i, : i + 1], B / (i + 1), rtol=1e-15)
+        assert np.all(acc[0, i, i + 1:] == 0.0)
+
+
+# ------------------------------------------------------------------------- build mask
+
+
+def _domain(Lq, Lk, causal):
+    return [(i, j) for i in range(Lq) for j in range(Lk) if (not causal or j <= i)]
+
+
+def _brute_force_mask(acc, keep_frac, causal, keep_diag):
+    """Among all k-subsets of the domain that contain the forced entries, the one
+    with the largest exact sum; among those, the first in index order."""
+    Lq, Lk = acc.shape
+    dom = _domain(Lq, Lk, causal)
+    forced = [(i, j) for (i, j) in dom if keep_diag and Lq == Lk and i == j]
+    n_valid = len(dom)
+    k = max(len(forced), min(n_valid, int(math.floor(keep_frac * n_valid + 0.5))))
+    free = [e for e in dom if e not in forced]
+    best, best_key = None, None
+    for combo in itertools.combinations(free, k - len(forced)):
+        chosen = sorted(forced + list(combo), key=lambda e: e[0] * Lk + e[1])
+        total = sum(Fraction(float(acc[i, j])) for (i, j) in chosen)
+        key = (-total, tuple(i * Lk + j for (i, j) in chosen))
+        if best_key is None or key < best_key:
+            best, best_key = chosen, key
+    mask = np.zeros((Lq, Lk), dtype=np.uint8)
+    for (i, j) in best:
+        mask[i, j] = 1
+    return mask, k
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("keep_diag", [False, True])
+def test_mask_brute_force_tiny(causal, keep_diag):
+    rng = np.random.default_rng(40)
+    for L in (2, 3, 4):
+        for keep in (0.2, 0.5, 0.75):
+            for trial in range(6):
+                # few distinct values => many exact ties, which exercise the index rule
+                acc = rng.integers(0, 4, size=(1, L, L)).astype(np.float32) / 4.0
+                want, k = _brute_force_mask(acc[0], keep, causal, keep_diag)
+                got, nnz = orc.build_mask(acc, keep, causal=causal, keep_diag=keep_diag)
+                assert nnz[0] == k
+                np.testing.assert_array_equal(got[0], want)
+
+
+def test_mask_brute_force_rectangular():
+    rng = np.random.default_rng(41)
+    for (Lq, Lk) in ((2, 4), (3, 2), (4, 3)):
+        acc = rng.integers(0, 3, size=(1, Lq, Lk)).astype(np.float32)
+        want, k = _brute_force_mask(acc[0], 0.5, False, True)  # keep_diag ignored: Lq != Lk
+        got, nnz = orc.build_mask(acc, 0.5, causal=False, keep_diag=True)
+        assert nnz[0] == k
+        np.testing.assert_array_equal(got[0], want)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_mask_invariants(causal):
+    rng = np.random.default_rng(42)
+    H, L = 3, 67
+    acc = rng.random((H, L, L), dtype=np.float32)
+    acc[0].flat[::3] = 0.5  # plant ties
+    dom = np.tril(np.ones((L, L), dtype=bool)) if causal else np.ones((L, L), dtype=bool)
+    n_valid = int(dom.sum())
+    prev = None
+    for keep in (0.05, 0.1, 0.33, 0.5, 0.9, 1.0):
+        mask, nnz = orc.build_mask(acc, keep, causal=causal, keep_diag=True)
+        k = max(L, min(n_valid, int(math.floor(keep * n_valid + 0.5))))
+        assert metrics.keep_count(n_valid, L, keep) == k == orc.keep_count(n_valid, L, keep)
+        for h in range(H):
+            m = mask[h].astype(bool)
+            assert nnz[h] == k and m.sum() == k          # kept fraction exact
+            assert not m[~dom].any()                     # never outside the domain
+            assert m[np.arange(L), np.arange(L)].all()   # diagonal forced
+            off = ~np.eye(L, dtype=bool)
+            kept_free, pruned = acc[h][m & off], acc[h][~m & dom]
+            if kept_free.size and pruned.size:
+                assert kept_free.min() >= pruned.max()
+        if prev is not None:
+            assert np.all(prev <= mask)                  # nesting
+        prev = mask
+    np.testing.assert_array_equal(prev, np.broadcast_to(dom, (H, L, L)).astype(np.uint8))
+
+
+def test_mask_constant_acc_keeps_forced_then_first_indices():
+    L = 6
+    acc = np.full((1, L, L), 0.125, dtype=np.float32)
+    mask, nnz = orc.build_mask(acc, 0.5, causal=False, keep_diag=True)
+    want = np.eye(L, dtype=np.uint8)
+    need = 18 - L
+    for idx in range(L * L):
+        i, j = divmod(idx, L)
+        if need and i != j:
+            want[i, j] = 1
+            need -= 1
+    np.testing.assert_array_equal(mask[0], want)
+    assert nnz[0] == 18
+
+
+def test_mask_k_smaller_than_forced_keeps_diagonal_only():
+    rng = np.random.default_rng(43)
+    acc = rng.random((2, 9, 9), dtype=np.float32)
+    mask, nnz = orc.build_mask(acc, 0.01, causal=False, keep_diag=True)
+    np.testing.assert_array_equal(mask, np.broadcast_to(np.eye(9, dtype=np.uint8), (2, 9, 9)))
+    assert list(nnz) == [9, 9]
+
+
+def test_mask_in_domain_zero_beats_nothing_outside_domain():
+    """Causal domain is by index, not by value: in-domain zeros can be kept, out-of-domain never."""
+    L = 4
+    acc = np.zeros((1, L, L), dtype=np.float32)
+    acc[0, 0, 3] = 9.0  # outside the causal domain
+    mask, nnz = orc.build_mask(acc, 1.0, causal=True, keep_diag=True)
+    np.testing.assert_array_equal(mask[0], np.tril(np.ones((L, L), dtype=np.uint8)))
+
+
+def test_rounding_of_k_matches_the_workloads():
+    want = {"tiny": 1638, "bert": 8192, "lm": 13133, "s2s_self": 16448, "s2s_cross": 32768,
+            "long": 419533}
+    for name, w in inputs.WORKLOADS.items():
+        assert orc.keep_count(w.n_valid, w.n_forced, w.keep_frac) == want[name]
+        assert metrics.keep_count(w.n_valid, w.n_forced, w.keep_frac) == want[name]
+
+
+# ------------------------------------------------------------------------------ tiles
+
+
+def _numpy_tiles(mask):
+    """Independent re-statement with numpy.packbits (LSB-first)."""
+    H, Lq, Lk = mask.shape
+    n_qt, n_kt = -(-Lq // 128), -(-Lk // 128)
+    pad = np.zeros((H, n_qt * 128, n_kt * 128), dtype=np.uint8)
+    pad[:, :Lq, :Lk] = mask
+    row_ptr, col_idx, flags, bitmaps = [0], [], [], []
+    for h in range(H):
+        for qt in range(n_qt):
+            for kt in range(n_kt):
+                t = pad[h, qt * 128:(qt + 1) * 128, kt * 128:(kt + 1) * 128]
+                if t.any():
+                    col_idx.append(kt)
+                    flags.append(1 if t.all() else 0)
+                    bitmaps.append(np.packbits(t, axis=1, bitorder="little").view("<u4"))
+            row_ptr.append(len(col_idx))
+    return np.array(row_ptr), np.array(col_idx), np.array(flags), np.array(bitmaps).reshape(-1, 128, 4)
+
+
+@pytest.mark.parametrize("shape", [(2, 128, 128), (2, 300, 200), (1, 130, 515), (3, 5, 7)])
+def test_tiles_roundtrip_and_structure(shape):
+    H, Lq, Lk = shape
+    mask = inputs.random_mask(H, Lq, Lk, 0.02, seed=50).numpy()
+    mask[0, : min(128, Lq), : min(128, Lk)] = 1         # a full (or edge-full) tile
+    if Lk > 256:
+        mask[:, :, 128:256] = 0                          # an empty tile column
+    t = orc.mask_to_tiles(mask)
+    rp, ci, fl, bm = _numpy_tiles(mask)
+    np.testing.assert_array_equal(t["row_ptr"], rp)
+    np.testing.assert_array_equal(t["col_idx"], ci)
+    np.testing.assert_array_equal(t["flags"], fl)
+    np.testing.assert_array_equal(t["bitmap"], bm)
+    # structure
+    assert t["row_ptr"][0] == 0 and np.all(np.diff(t["row_ptr"]) >= 0)
+    n_qt = t["n_qt"]
+    back = np.zeros_like(mask)
+    pop = 0
+    for row in range(H * n_qt):
+        cols = t["col_idx"][t["row_ptr"][row]:t["row_ptr"][row + 1]]
+        assert np.all(np.diff(cols) > 0)
+        h, qt = divmod(row, n_qt)
+        for s in range(t["row_ptr"][row], t["row_ptr"][row + 1]):
+            bits = np.unpackbits(t["bitmap"][s].view(np.uint8), axis=1, bitorder="little")
+            c = int(bits.sum())
+            assert c > 0 and (t["flags"][s] == 1) == (c == 128 * 128)
+            pop += c
+            kt = t["col_idx"][s]
+            r1, c1 = min(128, Lq - qt * 128), min(128, Lk - kt * 128)
+            assert bits[r1:].sum() == 0 and bits[:, c1:].sum() == 0
+            back[h, qt * 128:qt * 128 + r1, kt * 128:kt * 128 + c1] = bits[:r1, :c1]
+    np.testing.assert_array_equal(back, mask)
+    assert pop == int(mask.sum())
+
+
+# ------------------------------------------------------------------------ hand example
+
+
+def test_hand_example_4x4():
+    g = _golden()
+    e = math.e
+    a, b, D2 = e / (2 * e + 2), 1 / (2 * e + 2), 2 * e + e * e + 1
+    dense = np.array([[a, b, a, b], [b, a, a, b], [e / D2, e / D2, e * e / D2, 1 / D2], [.25] * 4])
+    c2 = 2 * e + e * e
+    causal = np.array([[1, 0, 0, 0], [1 / (1 + e), e / (1 + e), 0, 0],
+                       [e / c2, e / c2, e * e / c2, 0], [.25] * 4])
+    np.testing.assert_allclose(g["dense_attention"], dense, atol=5e-7)
+    np.testing.assert_allclose(g["causal_attention"], causal, atol=5e-7)
+    Q, K, V = (g[x].astype(np.float32).reshape(1, 1, 4, 4) for x in "QKV")
+    np.testing.assert_array_equal((Q[0, 0] @ K[0, 0].T) / 2, g["logits"])
+
+    for is_causal, want in ((False, dense), (True, causal)):
+        acc = np.zeros((1, 4, 4))
+        orc.accumulate(acc, Q, K, causal=is_causal)
+        np.testing.assert_allclose(acc[0], want, rtol=1e-14, atol=1e-16)
+        dom = np.tril(np.ones((4, 4), np.uint8)) if is_causal else np.ones((4, 4), np.uint8)
+        O = orc.attention_fwd(Q, K, V, dom.reshape(1, 4, 4))
+        np.testing.assert_allclose(O[0, 0], want, rtol=1e-14, atol=1e-16)
+
+        key = "causal" if is_causal else "noncausal"
+        mask, nnz = orc.build_mask(acc.astype(np.float32), 0.5, causal=is_causal, keep_diag=True)
+        np.testing.assert_array_equal(mask[0], g[f"mask_{key}_keep50"].astype(np.uint8))
+        assert nnz[0] == (5 if is_causal else 8)
+        O = orc.attention_fwd(Q, K, V, mask)
+        np.testing.assert_allclose(O[0, 0], g[f"out_{key}_keep50"], atol=5e-7)
+
+    third = 1.0 / 3.0
+    mask = g["mask_noncausal_keep50"].astype(np.uint8).reshape(1, 4, 4)
+    O = orc.attention_fwd(Q, K, V, mask)
+    exact = np.array([[.5, 0, .5, 0], [0, .5, .5, 0], [0, 0, 1, 0], [third, third, 0, third]])
+    np.testing.assert_allclose(O[0, 0], exact, rtol=1e-15, atol=0)
+    mask[0, 2, :] = 0
+    O = orc.attention_fwd(Q, K, V, mask)
+    assert np.all(O[0, 0, 2] == 0.0)
+    np.testing.assert_allclose(O[0, 0, [0, 1, 3]], exact[[0, 1, 3]], rtol=1e-15, atol=0)
+
+
+# ------------------------------------------------------------------- MAC model (Eq. 3)
+
+
+def test_mac_fraction_closed_form():
+    """Eq. 3 and its derivation: per token 3d + d projection MACs (per unit of d)
+    and N + N attention MACs, of which a fraction p of the P.V product is saved."""
+    for d, N, p in ((768, 384, 0.9), (512, 128, 0.5), (4096, 4096, 0.6)):
+        B = 3
+        proj, qk, pv, outp = 3 * B * N * d * d, B * N * N * d, B * N * N * d, B * N * d * d
+        frac = (proj + qk + (1 - p) * pv + outp) / (proj + qk + pv + outp)
+        assert metrics.attention_macs_fraction(d, N, p) == pytest.approx(frac, rel=1e-14)
+        frac2 = (proj + (1 - p) * (qk + pv) + outp) / (proj + qk + pv + outp)
+        assert metrics.attention_macs_fraction(d, N, p, credit_qk=True) == pytest.approx(frac2, rel=1e-14)
+    assert metrics.attention_macs_fraction(768, 384, 0.9) == pytest.approx(3494.4 / 3840)
+    assert metrics.effective_flops(10, 2, 64) == 4 * 64 * 10 * 2
+    assert metrics.tile_flops(3, 2, 64) == 4 * 64 * 128 * 128 * 3 * 2
