@@ -1,0 +1,394 @@
+#!/usr/bin/env python
+"""Benchmark of the Attention Pruning path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input, all
+through the C ABI: ap_accumulate_attention (one calibration batch) ->
+ap_build_mask (mask + tile list) -> ap_sparse_attention_fwd under that mask ->
+the library's dense path at the same shape (ap_dense_tiles + the same forward
+kernel).  Prints ONE JSON line (rank 0).
+
+  metric / value   effective TFLOP/s of the sparse forward, 4*d*nnz FLOPs per
+                   (b, h), over the forward's device time inside the steps
+  ms_per_step      the whole step (all four stages)
+  e2e              the same metric through ap_sparse_attention_fwd_host: pinned
+                   host Q, K, V in, O back, copies inside the timed region
+  roofline         the forward kernel: executed tile FLOPs / time vs the
+                   measured bf16 peak; `by_stage` gives the other stages
+  cpu_baseline     the oracle (plain fp64 C) timed on a bounded sample
+
+The path does not shard (single-GPU method): --gpus N runs N independent
+replicas, one per GPU, and adds their throughput ("replicas only").
+
+--impl reference times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2012_02030_b200 import inputs, metrics  # noqa: E402
+
+METRIC = "sparse-attention fwd effective TFLOP/s (4*d*nnz)"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the ncu
+# captures summarised under profiles/ (None until a capture exists).
+NCU_FWD_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p["bf16_tflops_sustained"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+
+
+def oracle_sample_step(w, units, calib_seqs=1):
+    """One pass of the path on the CPU oracle for a bounded sample: `units` heads of
+    batch element 0.  Returns per-stage seconds and the FLOPs (4*d*nnz) of the forward."""
+    from oracle import ap_oracle as orc
+
+    heads = list(range(units))
+    q, k = inputs.calib_qk(w, 0)
+    bias = inputs.calib_bias(w)[heads].numpy()
+    qs, ks = inputs.widen(q[:calib_seqs, heads]), inputs.widen(k[:calib_seqs, heads])
+    acc64 = np.zeros((units, w.Lq, w.Lk))
+    t0 = time.perf_counter()
+    orc.accumulate(acc64, qs, ks, bias, causal=w.causal)
+    t1 = time.perf_counter()
+    mask, nnz = orc.build_mask(acc64.astype(np.float32), w.keep_frac, w.causal, w.keep_diag)
+    t2 = time.perf_counter()
+    eq, ek, ev = inputs.eval_qkv(w)
+    eq, ek, ev = (inputs.widen(t[:1, heads]) for t in (eq, ek, ev))
+    t3 = time.perf_counter()
+    orc.attention_fwd(eq, ek, ev, mask)
+    t4 = time.perf_counter()
+    flops = 4.0 * w.d * float(nnz.sum())
+    return dict(acc_s=t1 - t0, mask_s=t2 - t1, fwd_s=t4 - t3, flops=flops, cores=min(orc.num_threads(), units))
+
+
+def run_reference(args, w):
+    """The oracle as it stands, on the host cores, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    units = min(w.H, 8)
+    for _ in range(args.warmup):
+        oracle_sample_step(w, units)
+    fwd_s, step_s, flops, cores = 0.0, 0.0, 0.0, 1
+    for _ in range(args.steps):
+        r = oracle_sample_step(w, units)
+        fwd_s += r["fwd_s"]
+        step_s += r["acc_s"] + r["mask_s"] + r["fwd_s"]
+        flops += r["flops"]
+        cores = r["cores"]
+    value = flops / fwd_s / 1e12
+    sample = "heads 0..%d of batch element 0 (%d of %d (b,h) units); one calibration sequence" % (
+        units - 1, units, w.B * w.H)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * step_s / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w):
+    return {"workload": w.name, "B": w.B, "H": w.H, "Lq": w.Lq, "Lk": w.Lk, "d": w.d, "causal": w.causal,
+            "keep_frac": w.keep_frac, "keep_diag": w.keep_diag, "calib_batches": w.calib_batches,
+            "replicas": "one per GPU, no exchange"}
+
+
+# ------------------------------------------------------------------------------- GPU arm
+
+
+def run_gpu(args, w):
+    from paper_2012_02030_b200 import binding as ap
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    elem = 4 if w.dtype == "f32" else 2
+
+    # ---- resident inputs (host-generated, seeded) --------------------------------------
+    bias = inputs.calib_bias(w).to(dev)
+    n_rot = 2  # calibration batches kept resident and cycled through by the timed steps
+    calib = [tuple(t.to(dev) for t in inputs.calib_qk(w, w.calib_batches + r)) for r in range(n_rot)]
+    q, k, v = (t.to(dev) for t in inputs.eval_qkv(w))
+    out = torch.empty_like(q)
+    out_dense = torch.empty_like(q)
+    acc = torch.zeros((w.H, w.Lq, w.Lk), dtype=torch.float32, device=dev)
+    mask = torch.empty((w.H, w.Lq, w.Lk), dtype=torch.uint8, device=dev)
+    nnz = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    dense = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    ws = torch.empty(ap.ap_build_mask_workspace_bytes(w.H, w.Lq, w.Lk), dtype=torch.uint8, device=dev)
+    # small shapes: an L2 flush between steps; large ones exceed L2 by themselves
+    resident = acc.numel() * 4 + bias.numel() * 4 + 4 * q.numel() * elem
+    flush = None if resident > 400e6 else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    # the calibration set proper (untimed): the mask the steps work with is the real one
+    for t in range(w.calib_batches):
+        cq, ck = inputs.calib_qk(w, t)
+        ap.ap_accumulate_attention(acc, cq.to(dev), ck.to(dev), bias, causal=w.causal)
+    torch.cuda.synchronize()
+
+    t_log = torch.zeros((max(args.steps, 1),), dtype=torch.int32, device=dev)
+    stages = ("accumulate", "build_mask", "sparse_fwd", "dense_tiles", "dense_fwd")
+
+    def step(i, ev=None):
+        cq, ck = calib[i % n_rot]
+        if flush is not None:
+            flush.zero_()
+        if ev:
+            ev[0].record()
+        ap.ap_accumulate_attention(acc, cq, ck, bias, causal=w.causal)
+        if ev:
+            ev[1].record()
+        ap.ap_build_mask(acc, w.keep_frac, w.causal, w.keep_diag, mask, tiles, nnz, ws)
+        if ev:
+            ev[2].record()
+        ap.ap_sparse_attention_fwd(q, k, v, tiles, out)
+        if ev:
+            ev[3].record()
+        ap.ap_dense_tiles(dense, causal=w.causal)
+        if ev:
+            ev[4].record()
+        ap.ap_sparse_attention_fwd(q, k, v, dense, out_dense)
+        if ev:
+            ev[5].record()
+            t_log[i].copy_(tiles.row_ptr[-1])
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if ap.ap_device_status() != ap.AP_OK:
+        raise RuntimeError("device status not OK after warm-up")
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    launches0 = ap.ap_launch_count()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    barrier()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(args.steps):
+        step(i, events[i])
+    end.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = ap.ap_launch_count() - launches0
+    status = ap.ap_device_status()
+    if status != ap.AP_OK:
+        raise RuntimeError("device status %d after the timed steps" % status)
+    total_ms = start.elapsed_time(end)
+    stage_ms = {s: float(np.mean([events[i][j].elapsed_time(events[i][j + 1]) for i in range(args.steps)]))
+                for j, s in enumerate(stages)}
+    if world > 1:
+        import torch.distributed as dist
+
+        tt = torch.tensor([total_ms, stage_ms["sparse_fwd"]], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms, fwd_ms_max = float(tt[0]), float(tt[1])
+    else:
+        fwd_ms_max = stage_ms["sparse_fwd"]
+
+    # ---- counts -----------------------------------------------------------------------------
+    nnz_total = int(nnz.sum().item())
+    k_expected = metrics.keep_count(w.n_valid, w.n_forced, w.keep_frac)
+    assert nnz_total == k_expected * w.H, (nnz_total, k_expected)
+    T_sparse = float(t_log[: args.steps].float().mean().item())
+    T_dense = dense.n_tiles()
+    eff_flops = metrics.effective_flops(nnz_total, w.B, w.d)
+    value = world * eff_flops / (fwd_ms_max * 1e-3) / 1e12
+
+    # ---- end to end through host buffers ---------------------------------------------------------
+    hq, hk, hv = (t.pin_memory() for t in inputs.eval_qkv(w))
+    ho = torch.empty_like(hq).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        ap.ap_sparse_attention_fwd_host(hq, hk, hv, tiles, ho, q, k, v, out)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        ap.ap_sparse_attention_fwd_host(hq, hk, hv, tiles, ho, q, k, v, out)
+        torch.cuda.current_stream().synchronize()  # the caller reads O on the host every step
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        import torch.distributed as dist
+
+        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt[0])
+    h2d = 3 * 0 + (hq.numel() + hk.numel() + hv.numel()) * elem
+    d2h = ho.numel() * elem
+
+    if rank != 0:
+        return
+    # ---- rooflines ---------------------------------------------------------------------------------
+    tile_fl = metrics.tile_flops(T_sparse, w.B, w.d)
+    fwd_s = stage_ms["sparse_fwd"] * 1e-3
+    comp_bytes = metrics.compulsory_bytes(w.B, w.H, w.Lq, w.Lk, w.d, elem)
+    tensor_bound = w.dtype == "bf16" and tile_fl / comp_bytes > peaks["bf16_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if tensor_bound:
+        roof = {"bound": "tensor", "achieved": tile_fl / fwd_s / 1e12, "peak": peaks["bf16_sustained"],
+                "unit": "TFLOP/s", "peak_kind": "bf16 sustained, of " + peaks["source"]}
+    else:
+        roof = {"bound": "hbm", "achieved": comp_bytes / fwd_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "peak_kind": "copy bandwidth, of " + peaks["source"]}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_FWD_TRAFFIC_BYTES.get(w.name)
+    roof["kernel"] = "sparse_fwd"
+    roof["algorithmic"] = {"tile_flops": tile_fl, "compulsory_bytes": comp_bytes, "tiles_per_step": T_sparse}
+    # other stages, HBM view: accumulate = acc read+write over the domain + bias + Q,K;
+    # build_mask = 2 reads of acc + mask bytes + bitmap bits over H*Lq*Lk
+    dom = w.n_valid * w.H
+    acc_bytes = 8.0 * dom + 4.0 * dom + elem * w.B * w.H * (w.Lq + w.Lk) * w.d
+    mask_bytes = 8.0 * dom + 1.125 * w.H * w.Lq * w.Lk
+    by_stage = {
+        "accumulate": {"bound": "hbm", "achieved": acc_bytes / (stage_ms["accumulate"] * 1e-3) / 1e9,
+                       "peak": peaks["hbm_gbs"], "unit": "GB/s"},
+        "build_mask": {"bound": "hbm", "achieved": mask_bytes / (stage_ms["build_mask"] * 1e-3) / 1e9,
+                       "peak": peaks["hbm_gbs"], "unit": "GB/s"},
+        "dense_fwd": {"bound": "tensor", "unit": "TFLOP/s", "peak": peaks["bf16_sustained"],
+                      "achieved": metrics.tile_flops(T_dense, w.B, w.d) / (stage_ms["dense_fwd"] * 1e-3) / 1e12},
+    }
+    for r in by_stage.values():
+        r["frac"] = r["achieved"] / r["peak"]
+
+    # ---- CPU baseline (bounded sample) -----------------------------------------------------
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        units = min(w.H, 8)
+        r = oracle_sample_step(w, units)
+        cpu = {"value": r["flops"] / r["fwd_s"] / 1e12, "unit": UNIT, "cores": r["cores"], "kind": "oracle",
+               "sample": "forward of heads 0..%d of batch element 0 (%d of %d (b,h) units), mask from one "
+                         "calibration sequence" % (units - 1, units, w.B * w.H),
+               "stage_seconds": {"accumulate": r["acc_s"], "build_mask": r["mask_s"], "sparse_fwd": r["fwd_s"]}}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": dict(workload_config(w),
+                       l2="inputs exceed L2" if flush is None else "256 MiB flush write between steps",
+                       value_scope="sparse forward's device time inside the step; ms_per_step is the whole step"),
+        "stage_ms": stage_ms,
+        "tokens_per_s": world * w.B * w.Lq / (fwd_ms_max * 1e-3),
+        "speedup_vs_dense_path": stage_ms["dense_fwd"] / stage_ms["sparse_fwd"],
+        "density": {"kept_fraction": nnz_total / float(dom), "tiles_kept": T_sparse, "tiles_domain": T_dense,
+                    "tile_fill": nnz_total / (T_sparse * 128.0 * 128.0) if T_sparse else None},
+        "pct_of_bf16_roofline": {"effective_flops_burst": 100 * eff_flops / fwd_s / 1e12 / peaks["bf16"],
+                                 "tile_flops_burst": 100 * tile_fl / fwd_s / 1e12 / peaks["bf16"],
+                                 "tile_flops_sustained": 100 * tile_fl / fwd_s / 1e12 / peaks["bf16_sustained"]},
+        "pct_of_hbm_roofline": 100 * comp_bytes / fwd_s / 1e9 / peaks["hbm_gbs"],
+        "roofline": roof, "roofline_by_stage": by_stage, "cpu_baseline": cpu,
+        "e2e": {"value": world * eff_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=10)
+    p.add_argument("--warmup", type=int, default=3)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--workload", default="long", choices=sorted(inputs.WORKLOADS))
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    args = p.parse_args()
+    w = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    run_gpu(args, w)
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,184 @@
+/*
+ * ap.h - C ABI of the Attention Pruning library for NVIDIA B200 (sm_100a).
+ *
+ * Attention Pruning (AP) observes, for every attention head, the average
+ * softmax attention matrix over a calibration set (Eq. 1), prunes the entries
+ * whose average falls below a percentile threshold (Eq. 2) and then runs every
+ * later forward pass with the pruned entries forced to -infinity before the
+ * softmax (the masked attention equation of Section 3.2).  This library holds
+ * the three device-side steps of that procedure and nothing else:
+ *
+ *   ap_accumulate_attention   Eq. 1: running element-wise sum of softmax(QK^T/sqrt(d))
+ *   ap_build_mask             Eq. 2: per-head top-fraction selection -> mask + tile list
+ *   ap_sparse_attention_fwd   Section 3.2: masked attention that visits only kept tiles
+ *
+ * Conventions that hold for every entry point
+ *   - Tensors are contiguous, innermost dimension last: Q[B,H,Lq,d],
+ *     K,V[B,H,Lk,d], O[B,H,Lq,d], acc/bias/mask[H,Lq,Lk].
+ *   - Unless a parameter says "host", every pointer is DEVICE memory owned by
+ *     the caller and 16-byte aligned.  The library allocates no memory; scratch
+ *     space is passed in as a workspace whose size the *_workspace_bytes
+ *     functions report.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Work is enqueued on it and the call returns without synchronising.
+ *   - Argument errors are detected on the host and returned BEFORE anything is
+ *     enqueued.  Nothing throws, aborts or traps.  Conditions only the device
+ *     can see (a tile list that outgrew its capacity, a bounded wait that
+ *     expired) set a sticky device word that ap_device_status() returns.
+ *   - d is 64 or 128.  Any Lq, Lk >= 1 is accepted; `causal` needs Lq == Lk.
+ *   - There is no CPU fallback: without a CUDA device the compute calls return
+ *     AP_ERR_CUDA.
+ */
+#ifndef AP_H_
+#define AP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AP_TILE 128 /* edge of the square tiles of the tile list */
+
+typedef enum {
+  AP_OK = 0,
+  AP_ERR_INVALID_ARG = 1, /* null/misaligned pointer, size or fraction out of range */
+  AP_ERR_UNSUPPORTED = 2, /* d or dtype the kernels are not built for              */
+  AP_ERR_WORKSPACE = 3,   /* workspace or tile capacity too small                   */
+  AP_ERR_CUDA = 4,        /* a CUDA runtime call failed (no device, launch error)   */
+  AP_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up                     */
+} ap_status;
+
+typedef enum { AP_F32 = 0, AP_BF16 = 1 } ap_dtype;
+
+/*
+ * Tile list: the mask of Eq. 2 for H heads, cut into 128x128 tiles, with only
+ * the tiles that contain at least one kept entry stored (CSR over tile rows).
+ * The struct itself lives in host memory; its pointers are device memory.
+ *
+ *   row_ptr[H*n_qt + 1]  offsets into col_idx; list row r = h*n_qt + qt
+ *   col_idx[cap]         key-tile index kt of each stored tile, strictly
+ *                        ascending inside a list row
+ *   flags[cap]           bit 0: every one of the 128*128 entries is kept
+ *   bitmap[cap][128][4]  entry (r, c) of a tile is bit (c & 31) of word
+ *                        [r][c >> 5], least significant bit first; bits of
+ *                        rows >= Lq or columns >= Lk are 0
+ *
+ * cap is the capacity in tiles; ap_tiles_capacity() always suffices.
+ */
+typedef struct ap_tiles {
+  int32_t H, Lq, Lk;
+  int32_t n_qt, n_kt; /* ceil(Lq/128), ceil(Lk/128) */
+  int32_t cap;
+  int32_t *row_ptr;
+  int32_t *col_idx;
+  uint8_t *flags;
+  uint32_t *bitmap;
+} ap_tiles;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int ap_version(void);
+
+/* Kernels this library has launched so far in this process (a diagnostic counter). */
+uint64_t ap_launch_count(void);
+
+/* Static, human-readable name of a status code. */
+const char *ap_status_string(ap_status s);
+
+/* Upper bound on the tiles of any mask of this shape: H * ceil(Lq/128) * ceil(Lk/128). */
+int64_t ap_tiles_capacity(int H, int Lq, int Lk);
+
+/* Workspace sizes in bytes (0 if the shape is invalid). */
+size_t ap_build_mask_workspace_bytes(int H, int Lq, int Lk);
+size_t ap_mask_to_tiles_workspace_bytes(int H, int Lq, int Lk);
+
+/*
+ * Eq. 1 (with the attention matrix of Section 3.1), as a running sum:
+ *   acc[h,i,j] += sum_{b<B} softmax_j( Q[b,h,i,:].K[b,h,j,:] * scale + bias[h,i,j] )
+ * over the row's domain (all j, or j <= i when causal); entries outside the
+ * domain are not touched.  The 1/n of Eq. 1 is left to the caller, who counts
+ * the samples: the selection of Eq. 2 does not depend on it.
+ *   acc    [H,Lq,Lk] fp32, in/out.  The sum over b is taken in ascending b with no
+ *          floating-point atomics, so results are reproducible bit for bit.
+ *   Q, K   [B,H,Lq,d], [B,H,Lk,d] of type dt
+ *   bias   [H,Lq,Lk] fp32 added after scaling, or NULL
+ *   scale  multiplier of Q.K^T; 0 selects 1/sqrt(d)
+ */
+ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, const float *bias,
+                                  int B, int H, int Lq, int Lk, int d, ap_dtype dt, int causal,
+                                  float scale, void *stream);
+
+/*
+ * Eq. 2 with one threshold per head, as an exact top-k: an entry is pruned
+ * unless it is among the k largest of its head.
+ *   domain  all (i,j), or j <= i when causal; n_valid = its size
+ *   forced  the diagonal when keep_diag != 0 and Lq == Lk (counted inside k)
+ *   k       max(#forced, min(n_valid, floor(keep_frac*n_valid + 0.5))), in double
+ *   order   forced first, then larger fp32 value, then lower index i*Lk + j
+ * Outputs (any of mask / tiles / nnz_per_head may be NULL):
+ *   mask          [H,Lq,Lk] uint8, 1 = kept
+ *   tiles         tile list of the same mask; tiles->H/Lq/Lk/n_qt/n_kt are
+ *                 written by this call, pointers and cap are read
+ *   nnz_per_head  [H] int64, entries kept per head (= k)
+ * acc must not contain NaN; -0 is treated as +0.  keep_frac must be in (0, 1].
+ * More stored tiles than tiles->cap sets AP_ERR_WORKSPACE in the device status
+ * and leaves a truncated list.
+ */
+ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal,
+                        int keep_diag, uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Tile list of an arbitrary element mask (uint8 [H,Lq,Lk], non-zero = kept):
+ * the same encoding ap_build_mask emits, for masks made elsewhere (random
+ * masks as in the paper's control experiment, all-ones, hand-made).
+ */
+ap_status ap_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles *tiles,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Tile list of the unpruned attention (the zero mask matrix of Section 3.2):
+ * every tile of the domain, written without reading any mask.  This is the
+ * library's dense path and the baseline the sparse path is compared with.
+ * Needs tiles->cap >= the number of domain tiles (ap_tiles_capacity suffices).
+ */
+ap_status ap_dense_tiles(int H, int Lq, int Lk, int causal, ap_tiles *tiles, void *stream);
+
+/*
+ * Masked attention of Section 3.2.  For every b, h and query row i, with
+ * J = { j : entry (i,j) of head h is kept }:
+ *   O[b,h,i,:] = sum_{j in J} w_j V[b,h,j,:] / sum_{j in J} w_j,
+ *   w_j = exp( (Q[b,h,i,:].K[b,h,j,:]) * scale - max_J(...) ),
+ * and exactly 0 when J is empty.  Pruned entries get weight exactly 0.  Only the
+ * tiles stored in `tiles` are visited; causality is whatever the mask says.
+ *   Q, K, V, O  of type dt (O is rounded once, from fp32)
+ *   tiles       list for H heads and this Lq, Lk, shared by all b
+ *   scale       0 selects 1/sqrt(d)
+ */
+ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V,
+                                  const ap_tiles *tiles, void *O, int B, int H, int Lq, int Lk,
+                                  int d, ap_dtype dt, float scale, void *stream);
+
+/*
+ * The same call for HOST tensors (pinned memory recommended): copies Q, K, V to
+ * the caller's device staging buffers, runs ap_sparse_attention_fwd and copies
+ * O back, all on `stream`.  dQ..dO are device buffers of the tensors' sizes.
+ */
+ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const void *hV,
+                                       const ap_tiles *tiles, void *hO, void *dQ, void *dK,
+                                       void *dV, void *dO, int B, int H, int Lq, int Lk, int d,
+                                       ap_dtype dt, float scale, void *stream);
+
+/*
+ * Synchronises `stream`, then returns and clears the sticky device status of
+ * the current device: AP_OK, AP_ERR_WORKSPACE (tile capacity exceeded),
+ * AP_ERR_TIMEOUT (a bounded wait expired; outputs of that call are invalid) or
+ * AP_ERR_CUDA (the stream reported an error).
+ */
+ap_status ap_device_status(void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AP_H_ */

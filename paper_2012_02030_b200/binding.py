@@ -1,0 +1,229 @@
+"""Thin ctypes binding of libap_b200.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/ap.h)
+and takes torch tensors that live on the CUDA device (PyTorch is used for
+device memory and streams only).  All arithmetic happens inside the library's
+kernels.  If the shared library has not been built the import of this module
+fails: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+TILE = 128
+AP_OK, AP_ERR_INVALID_ARG, AP_ERR_UNSUPPORTED, AP_ERR_WORKSPACE, AP_ERR_CUDA, AP_ERR_TIMEOUT = range(6)
+AP_F32, AP_BF16 = 0, 1
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libap_b200.so")
+
+
+class ApError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+class ap_tiles(ctypes.Structure):
+    _fields_ = [
+        ("H", ctypes.c_int32), ("Lq", ctypes.c_int32), ("Lk", ctypes.c_int32),
+        ("n_qt", ctypes.c_int32), ("n_kt", ctypes.c_int32), ("cap", ctypes.c_int32),
+        ("row_ptr", ctypes.c_void_p), ("col_idx", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p), ("bitmap", ctypes.c_void_p),
+    ]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            "libap_b200.so is missing: build it with `python -m paper_2012_02030_b200.build` "
+            "(there is no fallback implementation)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i, f, d, sz, i64 = (ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_double,
+                            ctypes.c_size_t, ctypes.c_int64)
+    tp = ctypes.POINTER(ap_tiles)
+    sig = {
+        "ap_version": (i, []),
+        "ap_launch_count": (ctypes.c_uint64, []),
+        "ap_status_string": (ctypes.c_char_p, [i]),
+        "ap_tiles_capacity": (i64, [i, i, i]),
+        "ap_build_mask_workspace_bytes": (sz, [i, i, i]),
+        "ap_mask_to_tiles_workspace_bytes": (sz, [i, i, i]),
+        "ap_accumulate_attention": (i, [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp]),
+        "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
+        "ap_mask_to_tiles": (i, [vp, i, i, i, tp, vp, sz, vp]),
+        "ap_dense_tiles": (i, [i, i, i, i, tp, vp]),
+        "ap_sparse_attention_fwd": (i, [vp, vp, vp, tp, vp, i, i, i, i, i, i, f, vp]),
+        "ap_sparse_attention_fwd_host": (i, [vp, vp, vp, tp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, vp]),
+        "ap_device_status": (i, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+lib = _load()
+EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
+           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask",
+           "ap_mask_to_tiles", "ap_dense_tiles", "ap_sparse_attention_fwd",
+           "ap_sparse_attention_fwd_host", "ap_device_status")
+
+
+def status_string(status: int) -> str:
+    return lib.ap_status_string(int(status)).decode()
+
+
+ap_status_string = status_string
+
+
+def ap_version() -> int:
+    return int(lib.ap_version())
+
+
+def ap_launch_count() -> int:
+    return int(lib.ap_launch_count())
+
+
+def ap_tiles_capacity(H: int, Lq: int, Lk: int) -> int:
+    return int(lib.ap_tiles_capacity(H, Lq, Lk))
+
+
+def ap_build_mask_workspace_bytes(H: int, Lq: int, Lk: int) -> int:
+    return int(lib.ap_build_mask_workspace_bytes(H, Lq, Lk))
+
+
+def ap_mask_to_tiles_workspace_bytes(H: int, Lq: int, Lk: int) -> int:
+    return int(lib.ap_mask_to_tiles_workspace_bytes(H, Lq, Lk))
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return AP_F32
+    if t.dtype == torch.bfloat16:
+        return AP_BF16
+    raise TypeError("dtype must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _check(status: int, where: str) -> None:
+    if status != AP_OK:
+        raise ApError(status, where)
+
+
+def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA tensor" % name)
+    return t
+
+
+class Tiles:
+    """Device buffers of a tile list plus the ap_tiles descriptor that points at them."""
+
+    def __init__(self, H: int, Lq: int, Lk: int, device="cuda", cap: int | None = None):
+        self.H, self.Lq, self.Lk = H, Lq, Lk
+        self.n_qt, self.n_kt = -(-Lq // TILE), -(-Lk // TILE)
+        self.cap = ap_tiles_capacity(H, Lq, Lk) if cap is None else cap
+        self.row_ptr = torch.zeros(H * self.n_qt + 1, dtype=torch.int32, device=device)
+        self.col_idx = torch.zeros(max(self.cap, 1), dtype=torch.int32, device=device)
+        self.flags = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
+        self.bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
+        self.c = ap_tiles(H, Lq, Lk, self.n_qt, self.n_kt, self.cap, self.row_ptr.data_ptr(),
+                          self.col_idx.data_ptr(), self.flags.data_ptr(), self.bitmap.data_ptr())
+
+    def n_tiles(self) -> int:
+        """Number of stored tiles (synchronises)."""
+        return int(self.row_ptr[-1].item())
+
+    def to_host(self):
+        """dict of numpy arrays trimmed to the stored tiles (synchronises)."""
+        T = self.n_tiles()
+        return dict(row_ptr=self.row_ptr.cpu().numpy(), col_idx=self.col_idx[:T].cpu().numpy(),
+                    flags=self.flags[:T].cpu().numpy(),
+                    bitmap=self.bitmap[:T].cpu().numpy().view("uint32"), n_qt=self.n_qt, n_kt=self.n_kt)
+
+
+def ap_accumulate_attention(acc, Q, K, bias=None, causal=False, scale=0.0, stream=None) -> None:
+    _dev(acc, "acc"), _dev(Q, "Q"), _dev(K, "K")
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    if K.shape != (B, H, Lk, d) or acc.shape != (H, Lq, Lk) or acc.dtype != torch.float32 or K.dtype != Q.dtype:
+        raise ValueError("shape/dtype mismatch")
+    if bias is not None and (_dev(bias, "bias").shape != (H, Lq, Lk) or bias.dtype != torch.float32):
+        raise ValueError("bias must be float32 [H,Lq,Lk]")
+    _check(lib.ap_accumulate_attention(_ptr(acc), _ptr(Q), _ptr(K), _ptr(bias), B, H, Lq, Lk, d,
+                                       _dtype_code(Q), int(bool(causal)), float(scale), _stream(stream)),
+           "ap_accumulate_attention")
+
+
+def ap_build_mask(acc, keep_frac, causal=False, keep_diag=True, mask=None, tiles: Tiles | None = None,
+                  nnz_per_head=None, workspace=None, stream=None) -> None:
+    _dev(acc, "acc")
+    H, Lq, Lk = acc.shape
+    if acc.dtype != torch.float32:
+        raise ValueError("acc must be float32")
+    if workspace is None:
+        workspace = torch.empty(ap_build_mask_workspace_bytes(H, Lq, Lk), dtype=torch.uint8, device=acc.device)
+    _check(lib.ap_build_mask(_ptr(acc), H, Lq, Lk, float(keep_frac), int(bool(causal)), int(bool(keep_diag)),
+                             _ptr(mask), ctypes.byref(tiles.c) if tiles is not None else None,
+                             _ptr(nnz_per_head), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "ap_build_mask")
+
+
+def ap_mask_to_tiles(mask, tiles: Tiles, workspace=None, stream=None) -> None:
+    _dev(mask, "mask")
+    H, Lq, Lk = mask.shape
+    if mask.dtype != torch.uint8:
+        raise ValueError("mask must be uint8")
+    if workspace is None:
+        workspace = torch.empty(ap_mask_to_tiles_workspace_bytes(H, Lq, Lk), dtype=torch.uint8, device=mask.device)
+    _check(lib.ap_mask_to_tiles(_ptr(mask), H, Lq, Lk, ctypes.byref(tiles.c), _ptr(workspace),
+                                workspace.numel(), _stream(stream)), "ap_mask_to_tiles")
+
+
+def ap_dense_tiles(tiles: Tiles, causal=False, stream=None) -> None:
+    _check(lib.ap_dense_tiles(tiles.H, tiles.Lq, tiles.Lk, int(bool(causal)), ctypes.byref(tiles.c),
+                              _stream(stream)), "ap_dense_tiles")
+
+
+def ap_sparse_attention_fwd(Q, K, V, tiles: Tiles, O=None, scale=0.0, stream=None):
+    _dev(Q, "Q"), _dev(K, "K"), _dev(V, "V")
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    if K.shape != (B, H, Lk, d) or V.shape != K.shape or K.dtype != Q.dtype or V.dtype != Q.dtype:
+        raise ValueError("shape/dtype mismatch")
+    if O is None:
+        O = torch.empty_like(Q)
+    _check(lib.ap_sparse_attention_fwd(_ptr(Q), _ptr(K), _ptr(V), ctypes.byref(tiles.c), _ptr(_dev(O, "O")),
+                                       B, H, Lq, Lk, d, _dtype_code(Q), float(scale), _stream(stream)),
+           "ap_sparse_attention_fwd")
+    return O
+
+
+def ap_sparse_attention_fwd_host(hQ, hK, hV, tiles: Tiles, hO, dQ, dK, dV, dO, scale=0.0, stream=None):
+    """Host tensors in, host tensor out; d* are device staging buffers of the same shapes."""
+    B, H, Lq, d = hQ.shape
+    Lk = hK.shape[2]
+    for t in (hQ, hK, hV, hO):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("h* must be contiguous host tensors")
+    _check(lib.ap_sparse_attention_fwd_host(_ptr(hQ), _ptr(hK), _ptr(hV), ctypes.byref(tiles.c), _ptr(hO),
+                                            _ptr(_dev(dQ, "dQ")), _ptr(_dev(dK, "dK")), _ptr(_dev(dV, "dV")),
+                                            _ptr(_dev(dO, "dO")), B, H, Lq, Lk, d, _dtype_code(hQ),
+                                            float(scale), _stream(stream)), "ap_sparse_attention_fwd_host")
+    return hO
+
+
+def ap_device_status(stream=None) -> int:
+    return int(lib.ap_device_status(_stream(stream)))

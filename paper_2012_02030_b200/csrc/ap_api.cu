@@ -1,0 +1,265 @@
+// The C ABI declared in ap.h: argument validation, workspace carving, dispatch.
+// Nothing is enqueued before every argument has been checked.
+#include <math.h>
+
+#include <atomic>
+
+#include "ap_common.cuh"
+
+namespace ap {
+
+namespace {
+
+__device__ unsigned g_error_word = 0u;  // sticky device status, one per device
+
+std::atomic<unsigned long long> g_launches{0};
+
+constexpr int kMaxDevices = 64;
+unsigned *g_error_ptr[kMaxDevices] = {nullptr};
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool shape_ok(int H, int Lq, int Lk) {
+  if (H < 1 || Lq < 1 || Lk < 1) return false;
+  if ((int64_t)Lq * Lk > (int64_t)1 << 31) return false;                  // 32-bit tie ranks / indices
+  if ((int64_t)H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile) > (1 << 24)) return false;
+  if ((int64_t)H * Lq * ceil_div(Lk, kTile) > (int64_t)1 << 31) return false;
+  return true;
+}
+
+ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shape_must_match) {
+  if (!t) return AP_ERR_INVALID_ARG;
+  if (!t->row_ptr || !t->col_idx || !t->flags || !t->bitmap) return AP_ERR_INVALID_ARG;
+  if (!aligned16(t->bitmap) || (reinterpret_cast<uintptr_t>(t->row_ptr) & 3u) ||
+      (reinterpret_cast<uintptr_t>(t->col_idx) & 3u))
+    return AP_ERR_INVALID_ARG;
+  if (t->cap < 1) return AP_ERR_WORKSPACE;
+  if (shape_must_match) {
+    if (t->H != H || t->Lq != Lq || t->Lk != Lk || t->n_qt != ceil_div(Lq, kTile) ||
+        t->n_kt != ceil_div(Lk, kTile))
+      return AP_ERR_INVALID_ARG;
+  }
+  return AP_OK;
+}
+
+void fill_tiles_shape(ap_tiles *t, int H, int Lq, int Lk) {
+  t->H = H;
+  t->Lq = Lq;
+  t->Lk = Lk;
+  t->n_qt = ceil_div(Lq, kTile);
+  t->n_kt = ceil_div(Lk, kTile);
+}
+
+bool have_device() {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev >= 0;
+}
+
+}  // namespace
+
+void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+unsigned *device_error_word() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  if (!g_error_ptr[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_error_word) != cudaSuccess) return nullptr;
+    g_error_ptr[dev] = static_cast<unsigned *>(p);
+  }
+  return g_error_ptr[dev];
+}
+
+int64_t domain_size(int Lq, int Lk, int causal) {
+  if (!causal) return (int64_t)Lq * Lk;
+  int64_t n = 0;
+  for (int i = 0; i < Lq; ++i) n += (i + 1 < Lk) ? i + 1 : Lk;
+  return n;
+}
+
+int64_t keep_count(int64_t n_valid, int64_t n_forced, double keep_frac) {
+  int64_t k = (int64_t)floor(keep_frac * (double)n_valid + 0.5);
+  if (k > n_valid) k = n_valid;
+  if (k < n_forced) k = n_forced;
+  return k;
+}
+
+}  // namespace ap
+
+using namespace ap;
+
+extern "C" {
+
+int ap_version(void) { return 100; }
+
+uint64_t ap_launch_count(void) { return (uint64_t)g_launches.load(std::memory_order_relaxed); }
+
+const char *ap_status_string(ap_status s) {
+  switch (s) {
+    case AP_OK: return "ok";
+    case AP_ERR_INVALID_ARG: return "invalid argument";
+    case AP_ERR_UNSUPPORTED: return "unsupported head dimension or dtype";
+    case AP_ERR_WORKSPACE: return "workspace or tile capacity too small";
+    case AP_ERR_CUDA: return "CUDA runtime error";
+    case AP_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int64_t ap_tiles_capacity(int H, int Lq, int Lk) {
+  if (H < 1 || Lq < 1 || Lk < 1) return 0;
+  return (int64_t)H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile);
+}
+
+size_t ap_mask_to_tiles_workspace_bytes(int H, int Lq, int Lk) {
+  if (!shape_ok(H, Lq, Lk)) return 0;
+  return stage_bytes(H, Lq, Lk);
+}
+
+size_t ap_build_mask_workspace_bytes(int H, int Lq, int Lk) {
+  if (!shape_ok(H, Lq, Lk)) return 0;
+  return stage_bytes(H, Lq, Lk) + select_scratch_bytes(H, Lq, Lk);
+}
+
+ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
+                                  int Lq, int Lk, int d, ap_dtype dt, int causal, float scale, void *stream) {
+  if (!acc || !Q || !K || !aligned16(acc) || !aligned16(Q) || !aligned16(K) || (bias && !aligned16(bias)))
+    return AP_ERR_INVALID_ARG;
+  if (B < 1 || !shape_ok(H, Lq, Lk) || (causal && Lq != Lk) || !(scale >= 0.f) || isinf(scale))
+    return AP_ERR_INVALID_ARG;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
+  if (!have_device()) return AP_ERR_CUDA;
+  const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
+  cudaError_t e = launch_accumulate_simt(acc, Q, K, bias, B, H, Lq, Lk, d, dt, causal ? 1 : 0, sc,
+                                         static_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return AP_ERR_UNSUPPORTED;  // key length beyond the shared-memory budget
+  return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
+}
+
+ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
+                        uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
+                        size_t workspace_bytes, void *stream) {
+  if (!acc || !aligned16(acc) || !shape_ok(H, Lq, Lk) || (causal && Lq != Lk)) return AP_ERR_INVALID_ARG;
+  if (!(keep_frac > 0.0) || !(keep_frac <= 1.0)) return AP_ERR_INVALID_ARG;
+  if (mask && !aligned16(mask)) return AP_ERR_INVALID_ARG;
+  if (nnz_per_head && (reinterpret_cast<uintptr_t>(nnz_per_head) & 7u)) return AP_ERR_INVALID_ARG;
+  if (tiles) {
+    ap_status st = check_tiles(tiles, H, Lq, Lk, false);
+    if (st != AP_OK) return st;
+  }
+  if (!workspace || !aligned16(workspace)) return AP_ERR_INVALID_ARG;
+  if (workspace_bytes < ap_build_mask_workspace_bytes(H, Lq, Lk)) return AP_ERR_WORKSPACE;
+  if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int n_tiles = H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile);
+  char *ws = static_cast<char *>(workspace);
+  const size_t stage = stage_bytes(H, Lq, Lk);
+  BuildMaskArgs a;
+  a.acc = acc;
+  a.H = H; a.Lq = Lq; a.Lk = Lk;
+  a.causal = causal ? 1 : 0;
+  a.keep_diag = keep_diag ? 1 : 0;
+  const int64_t n_valid = domain_size(Lq, Lk, a.causal);
+  const int64_t n_forced = (a.keep_diag && Lq == Lk) ? Lq : 0;
+  a.k = keep_count(n_valid, n_forced, keep_frac);
+  a.k_rest = a.k - n_forced;
+  a.mask = mask;
+  a.nnz = nnz_per_head;
+  a.stage_bitmap = tiles ? reinterpret_cast<uint32_t *>(ws) : nullptr;
+  a.stage_count = tiles ? reinterpret_cast<int32_t *>(ws + (size_t)n_tiles * kBitmapWords * sizeof(uint32_t)) : nullptr;
+  a.scratch = ws + stage;
+  if (launch_build_mask(a, s) != cudaSuccess) return AP_ERR_CUDA;
+  if (tiles) {
+    fill_tiles_shape(tiles, H, Lq, Lk);
+    if (launch_compact_tiles(a.stage_bitmap, a.stage_count, *tiles, s) != cudaSuccess) return AP_ERR_CUDA;
+  }
+  return AP_OK;
+}
+
+ap_status ap_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles *tiles, void *workspace,
+                           size_t workspace_bytes, void *stream) {
+  if (!mask || !shape_ok(H, Lq, Lk)) return AP_ERR_INVALID_ARG;
+  ap_status st = check_tiles(tiles, H, Lq, Lk, false);
+  if (st != AP_OK) return st;
+  if (!workspace || !aligned16(workspace)) return AP_ERR_INVALID_ARG;
+  if (workspace_bytes < ap_mask_to_tiles_workspace_bytes(H, Lq, Lk)) return AP_ERR_WORKSPACE;
+  if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int n_tiles = H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile);
+  char *ws = static_cast<char *>(workspace);
+  uint32_t *stage_bitmap = reinterpret_cast<uint32_t *>(ws);
+  int32_t *stage_count = reinterpret_cast<int32_t *>(ws + (size_t)n_tiles * kBitmapWords * sizeof(uint32_t));
+  if (launch_stage_from_mask(mask, H, Lq, Lk, stage_bitmap, stage_count, s) != cudaSuccess) return AP_ERR_CUDA;
+  fill_tiles_shape(tiles, H, Lq, Lk);
+  if (launch_compact_tiles(stage_bitmap, stage_count, *tiles, s) != cudaSuccess) return AP_ERR_CUDA;
+  return AP_OK;
+}
+
+ap_status ap_dense_tiles(int H, int Lq, int Lk, int causal, ap_tiles *tiles, void *stream) {
+  if (!shape_ok(H, Lq, Lk) || (causal && Lq != Lk)) return AP_ERR_INVALID_ARG;
+  ap_status st = check_tiles(tiles, H, Lq, Lk, false);
+  if (st != AP_OK) return st;
+  const int n_qt = ceil_div(Lq, kTile), n_kt = ceil_div(Lk, kTile);
+  const int64_t need = (int64_t)H * (causal ? (int64_t)n_qt * (n_qt + 1) / 2 : (int64_t)n_qt * n_kt);
+  if (tiles->cap < need) return AP_ERR_WORKSPACE;
+  if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
+  fill_tiles_shape(tiles, H, Lq, Lk);
+  return launch_dense_tiles(*tiles, causal ? 1 : 0, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? AP_OK
+             : AP_ERR_CUDA;
+}
+
+ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V, const ap_tiles *tiles, void *O,
+                                  int B, int H, int Lq, int Lk, int d, ap_dtype dt, float scale, void *stream) {
+  if (!Q || !K || !V || !O || !aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O))
+    return AP_ERR_INVALID_ARG;
+  if (B < 1 || !shape_ok(H, Lq, Lk) || !(scale >= 0.f) || isinf(scale)) return AP_ERR_INVALID_ARG;
+  if ((int64_t)B * H * ceil_div(Lq, kTile) > (int64_t)0x7fffffff) return AP_ERR_INVALID_ARG;
+  ap_status st = check_tiles(tiles, H, Lq, Lk, true);
+  if (st != AP_OK) return st;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
+  if (!have_device()) return AP_ERR_CUDA;
+  const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
+  cudaError_t e = launch_fwd_simt(Q, K, V, *tiles, O, B, H, Lq, Lk, d, dt, sc, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
+}
+
+ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const void *hV, const ap_tiles *tiles,
+                                       void *hO, void *dQ, void *dK, void *dV, void *dO, int B, int H, int Lq,
+                                       int Lk, int d, ap_dtype dt, float scale, void *stream) {
+  if (!hQ || !hK || !hV || !hO) return AP_ERR_INVALID_ARG;
+  if (!dQ || !dK || !dV || !dO || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(dO))
+    return AP_ERR_INVALID_ARG;
+  if (B < 1 || !shape_ok(H, Lq, Lk) || !(scale >= 0.f) || isinf(scale)) return AP_ERR_INVALID_ARG;
+  ap_status st = check_tiles(tiles, H, Lq, Lk, true);
+  if (st != AP_OK) return st;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
+  if (!have_device()) return AP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t elem = dt == AP_F32 ? 4 : 2;
+  const size_t q_bytes = elem * B * H * (size_t)Lq * d, k_bytes = elem * B * H * (size_t)Lk * d;
+  if (cudaMemcpyAsync(dQ, hQ, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AP_ERR_CUDA;
+  if (cudaMemcpyAsync(dK, hK, k_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AP_ERR_CUDA;
+  if (cudaMemcpyAsync(dV, hV, k_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AP_ERR_CUDA;
+  st = ap_sparse_attention_fwd(dQ, dK, dV, tiles, dO, B, H, Lq, Lk, d, dt, scale, stream);
+  if (st != AP_OK) return st;
+  if (cudaMemcpyAsync(hO, dO, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return AP_ERR_CUDA;
+  return AP_OK;
+}
+
+ap_status ap_device_status(void *stream) {
+  if (!have_device()) return AP_ERR_CUDA;
+  unsigned *word = device_error_word();
+  if (!word) return AP_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned host = 0u;
+  if (cudaMemcpyAsync(&host, word, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess) return AP_ERR_CUDA;
+  if (cudaMemsetAsync(word, 0, sizeof(host), s) != cudaSuccess) return AP_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return AP_ERR_CUDA;
+  if (host & kDevErrTimeout) return AP_ERR_TIMEOUT;
+  if (host & kDevErrCapacity) return AP_ERR_WORKSPACE;
+  return AP_OK;
+}
+
+}  // extern "C"

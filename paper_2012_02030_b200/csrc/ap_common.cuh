@@ -1,0 +1,66 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ap.h"
+
+namespace ap {
+
+constexpr int kTile = AP_TILE;
+constexpr int kBitmapWords = kTile * 4;  // 32-bit words of one tile bitmap
+
+// Bits of the sticky device status word.
+constexpr unsigned kDevErrCapacity = 1u;
+constexpr unsigned kDevErrTimeout = 2u;
+
+// Address of the device status word of the current device (NULL on failure).
+unsigned *device_error_word();
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Kernels launched by this library in this process (see ap_launch_count in ap.h).
+void count_launches(int n);
+
+// Host: entries kept per head (see ap_build_mask in ap.h).
+int64_t keep_count(int64_t n_valid, int64_t n_forced, double keep_frac);
+int64_t domain_size(int Lq, int Lk, int causal);
+
+// ---- launchers (each returns the cudaError_t of its launches) -------------------------------
+
+// Per-tile bitmaps + popcounts of an element mask into a dense staging area
+// stage_bitmap[H*n_qt*n_kt][128][4], stage_count[H*n_qt*n_kt].
+cudaError_t launch_stage_from_mask(const uint8_t *mask, int H, int Lq, int Lk, uint32_t *stage_bitmap,
+                                   int32_t *stage_count, cudaStream_t s);
+// Staging area -> compacted tile list.
+cudaError_t launch_compact_tiles(const uint32_t *stage_bitmap, const int32_t *stage_count,
+                                 const ap_tiles &t, cudaStream_t s);
+cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s);
+
+size_t stage_bytes(int H, int Lq, int Lk);
+
+struct BuildMaskArgs {
+  const float *acc;
+  int H, Lq, Lk, causal, keep_diag;
+  int64_t k_rest;  // entries to select among the non-forced domain entries
+  int64_t k;       // entries kept per head
+  uint8_t *mask;   // may be NULL
+  int64_t *nnz;    // may be NULL
+  uint32_t *stage_bitmap;  // may be NULL (no tile list wanted)
+  int32_t *stage_count;
+  void *scratch;  // select scratch
+};
+size_t select_scratch_bytes(int H, int Lq, int Lk);
+cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s);
+
+cudaError_t launch_accumulate_simt(float *acc, const void *Q, const void *K, const float *bias, int B,
+                                   int H, int Lq, int Lk, int d, ap_dtype dt, int causal, float scale,
+                                   cudaStream_t s);
+
+cudaError_t launch_fwd_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
+                            int B, int H, int Lq, int Lk, int d, ap_dtype dt, float scale,
+                            cudaStream_t s);
+
+}  // namespace ap

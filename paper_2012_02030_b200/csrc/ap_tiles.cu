@@ -1,0 +1,203 @@
+// Tile lists: element mask -> per-tile bitmaps -> compacted CSR of non-empty tiles.
+//
+// The tile list is an encoding of the pruning mask of Eq. 2 (the paper itself
+// only states the element mask).  Bitmaps are first written for every tile of
+// the grid into a staging area ordered (h, qt, kt); a single-CTA scan then
+// assigns list positions to the non-empty ones in that order, and a copy
+// kernel moves their bitmaps to the compacted list.
+#include "ap_common.cuh"
+
+namespace ap {
+
+size_t stage_bytes(int H, int Lq, int Lk) {
+  size_t n = (size_t)H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile);
+  // bitmaps, popcounts, list positions
+  return n * (kBitmapWords * sizeof(uint32_t)) + 2 * ((n * sizeof(int32_t) + 255) / 256 * 256);
+}
+
+namespace {
+
+// One CTA per tile; warp w takes rows w, w+4, ...; a ballot over 32 consecutive
+// mask bytes yields one bitmap word.
+__global__ void __launch_bounds__(128) stage_from_mask_kernel(const uint8_t *__restrict__ mask, int Lq,
+                                                              int Lk, int n_qt, int n_kt,
+                                                              uint32_t *__restrict__ stage_bitmap,
+                                                              int32_t *__restrict__ stage_count) {
+  const int tile = blockIdx.x;
+  const int kt = tile % n_kt;
+  const int qt = (tile / n_kt) % n_qt;
+  const int h = tile / (n_kt * n_qt);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ int warp_count[4];
+  int count = 0;
+  uint4 *out = reinterpret_cast<uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords);
+  for (int r = warp; r < kTile; r += 4) {
+    const int i = qt * kTile + r;
+    uint32_t w[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int j = kt * kTile + 32 * c + lane;
+      bool keep = false;
+      if (i < Lq && j < Lk) keep = mask[((size_t)h * Lq + i) * Lk + j] != 0;
+      w[c] = __ballot_sync(0xffffffffu, keep);
+      count += __popc(w[c]);
+    }
+    if (lane == 0) out[r] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  // every lane of a warp holds the same count
+  if (lane == 0) warp_count[warp] = count;
+  __syncthreads();
+  if (threadIdx.x == 0)
+    stage_count[tile] = warp_count[0] + warp_count[1] + warp_count[2] + warp_count[3];
+}
+
+// Single CTA: exclusive scan of "tile is non-empty" over the (h, qt, kt) order.
+__global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restrict__ stage_count,
+                                                          int32_t *__restrict__ stage_pos, int n_tiles,
+                                                          int n_kt, int cap, int32_t *__restrict__ row_ptr,
+                                                          unsigned *err) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) {
+    carry_s = 0;
+    row_ptr[0] = 0;
+  }
+  __syncthreads();
+  for (int base = 0; base < n_tiles; base += 1024) {
+    const int idx = base + threadIdx.x;
+    const int flag = (idx < n_tiles && stage_count[idx] > 0) ? 1 : 0;
+    int incl = flag;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int v = warp_sums[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += u;
+      }
+      warp_sums[lane] = v;  // inclusive over warps
+    }
+    __syncthreads();
+    const int carry = carry_s;
+    const int before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - flag;
+    if (idx < n_tiles) {
+      stage_pos[idx] = flag ? before : -1;
+      if (idx % n_kt == n_kt - 1) row_ptr[idx / n_kt + 1] = min(before + flag, cap);
+    }
+    __syncthreads();
+    if (threadIdx.x == 1023) carry_s = carry + warp_sums[31];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0 && carry_s > cap) atomicOr(err, kDevErrCapacity);
+}
+
+// One CTA per grid tile: non-empty tiles copy their bitmap to their list slot.
+__global__ void __launch_bounds__(128) gather_tiles_kernel(const uint32_t *__restrict__ stage_bitmap,
+                                                           const int32_t *__restrict__ stage_count,
+                                                           const int32_t *__restrict__ stage_pos, int n_kt,
+                                                           int cap, int32_t *__restrict__ col_idx,
+                                                           uint8_t *__restrict__ flags,
+                                                           uint32_t *__restrict__ bitmap) {
+  const int tile = blockIdx.x;
+  const int pos = stage_pos[tile];
+  if (pos < 0 || pos >= cap) return;
+  const uint4 *src = reinterpret_cast<const uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords);
+  uint4 *dst = reinterpret_cast<uint4 *>(bitmap + (size_t)pos * kBitmapWords);
+  dst[threadIdx.x] = src[threadIdx.x];
+  if (threadIdx.x == 0) {
+    col_idx[pos] = tile % n_kt;
+    flags[pos] = stage_count[tile] == kTile * kTile ? 1 : 0;
+  }
+}
+
+// One CTA per grid tile, thread r = tile row r: writes the list of the full
+// (optionally causal) domain in closed form.
+__global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk, int n_qt, int n_kt, int causal,
+                                                          int cap, int32_t *__restrict__ row_ptr,
+                                                          int32_t *__restrict__ col_idx,
+                                                          uint8_t *__restrict__ flags,
+                                                          uint32_t *__restrict__ bitmap, unsigned *err) {
+  const int tile = blockIdx.x;
+  const int kt = tile % n_kt;
+  const int qt = (tile / n_kt) % n_qt;
+  const int h = tile / (n_kt * n_qt);
+  // causal needs Lq == Lk, so n_qt == n_kt and the row of qt holds tiles 0..qt
+  const int per_head = causal ? n_qt * (n_qt + 1) / 2 : n_qt * n_kt;
+  const int row_start = h * per_head + (causal ? qt * (qt + 1) / 2 : qt * n_kt);
+  if (threadIdx.x == 0 && kt == 0) {
+    row_ptr[h * n_qt + qt] = min(row_start, cap);
+    if (h == H - 1 && qt == n_qt - 1) {
+      row_ptr[H * n_qt] = min(H * per_head, cap);
+      if (H * per_head > cap) atomicOr(err, kDevErrCapacity);
+    }
+  }
+  if (causal && kt > qt) return;
+  const int pos = row_start + kt;
+  if (pos >= cap) return;
+  const int r = threadIdx.x;
+  const int i = qt * kTile + r;
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  if (i < Lq) {
+    int jend = causal ? min(Lk, i + 1) : Lk;  // first column not kept
+    int n = jend - kt * kTile;                // kept columns of this tile row
+    n = max(0, min(kTile, n));
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      int m = n - 32 * c;
+      w[c] = m >= 32 ? 0xffffffffu : (m > 0 ? ((1u << m) - 1u) : 0u);
+    }
+  }
+  reinterpret_cast<uint4 *>(bitmap + (size_t)pos * kBitmapWords)[r] = make_uint4(w[0], w[1], w[2], w[3]);
+  const int full = __syncthreads_and(w[0] == 0xffffffffu && w[1] == 0xffffffffu &&
+                                     w[2] == 0xffffffffu && w[3] == 0xffffffffu);
+  if (r == 0) {
+    col_idx[pos] = kt;
+    flags[pos] = full ? 1 : 0;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_stage_from_mask(const uint8_t *mask, int H, int Lq, int Lk, uint32_t *stage_bitmap,
+                                   int32_t *stage_count, cudaStream_t s) {
+  const int n_qt = ceil_div(Lq, kTile), n_kt = ceil_div(Lk, kTile);
+  stage_from_mask_kernel<<<H * n_qt * n_kt, 128, 0, s>>>(mask, Lq, Lk, n_qt, n_kt, stage_bitmap,
+                                                       stage_count);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compact_tiles(const uint32_t *stage_bitmap, const int32_t *stage_count,
+                                 const ap_tiles &t, cudaStream_t s) {
+  const int n_tiles = t.H * t.n_qt * t.n_kt;
+  unsigned *err = device_error_word();
+  if (!err) return cudaErrorUnknown;
+  // list positions live right behind the popcounts in the staging area
+  int32_t *stage_pos = const_cast<int32_t *>(stage_count) + ((size_t)n_tiles * 4 + 255) / 256 * 64;
+  scan_tiles_kernel<<<1, 1024, 0, s>>>(stage_count, stage_pos, n_tiles, t.n_kt, t.cap, t.row_ptr, err);
+  count_launches(1);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  gather_tiles_kernel<<<n_tiles, 128, 0, s>>>(stage_bitmap, stage_count, stage_pos, t.n_kt, t.cap,
+                                              t.col_idx, t.flags, t.bitmap);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
+  unsigned *err = device_error_word();
+  if (!err) return cudaErrorUnknown;
+  dense_tiles_kernel<<<t.H * t.n_qt * t.n_kt, 128, 0, s>>>(t.H, t.Lq, t.Lk, t.n_qt, t.n_kt, causal, t.cap,
+                                                         t.row_ptr, t.col_idx, t.flags, t.bitmap, err);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace ap

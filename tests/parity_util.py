@@ -1,0 +1,57 @@
+"""Helpers shared by the GPU parity tests: run a stage on the CUDA library and
+on the oracle with the same host-generated inputs, and compare."""
+import numpy as np
+import torch
+
+from oracle import ap_oracle as orc
+from paper_2012_02030_b200 import inputs
+
+# tolerances of the attention output against the fp64 oracle
+TOL = {"bf16": dict(max_abs=1e-2, rel_l2=5e-3), "f32": dict(max_abs=1e-5, rel_l2=1e-6)}
+
+
+def errors(got: np.ndarray, ref: np.ndarray):
+    got = got.astype(np.float64)
+    diff = got - ref
+    return float(np.abs(diff).max()), float(np.linalg.norm(diff.ravel()) / max(np.linalg.norm(ref.ravel()), 1e-300))
+
+
+def assert_close_attention(got_t: torch.Tensor, ref: np.ndarray, dtype: str, what=""):
+    max_abs, rel_l2 = errors(got_t.float().cpu().numpy(), ref)
+    tol = TOL[dtype]
+    assert max_abs <= tol["max_abs"] and rel_l2 <= tol["rel_l2"], (what, dtype, max_abs, rel_l2)
+    return max_abs, rel_l2
+
+
+def assert_tiles_equal(got: dict, want: dict):
+    np.testing.assert_array_equal(got["row_ptr"], want["row_ptr"])
+    np.testing.assert_array_equal(got["col_idx"], want["col_idx"])
+    np.testing.assert_array_equal(got["flags"], want["flags"])
+    np.testing.assert_array_equal(got["bitmap"], want["bitmap"])
+
+
+def gpu_accumulate(ap, w, n_batches, bias_dev):
+    acc = torch.zeros((w.H, w.Lq, w.Lk), dtype=torch.float32, device="cuda")
+    for t in range(n_batches):
+        q, k = inputs.calib_qk(w, t)
+        ap.ap_accumulate_attention(acc, q.cuda(), k.cuda(), bias_dev, causal=w.causal)
+    return acc
+
+
+def oracle_accumulate(w, n_batches, bias):
+    acc64 = np.zeros((w.H, w.Lq, w.Lk))
+    for t in range(n_batches):
+        q, k = inputs.calib_qk(w, t)
+        orc.accumulate(acc64, inputs.widen(q), inputs.widen(k), None if bias is None else bias.numpy(),
+                       causal=w.causal)
+    return acc64
+
+
+def gpu_build_mask(ap, acc_dev, w, want_tiles=True):
+    H, Lq, Lk = acc_dev.shape
+    mask = torch.full((H, Lq, Lk), 7, dtype=torch.uint8, device="cuda")  # poison: every byte must be written
+    nnz = torch.full((H,), -1, dtype=torch.int64, device="cuda")
+    tiles = ap.Tiles(H, Lq, Lk) if want_tiles else None
+    ap.ap_build_mask(acc_dev, w.keep_frac, w.causal, w.keep_diag, mask, tiles, nnz)
+    assert ap.ap_device_status() == ap.AP_OK
+    return mask, tiles, nnz

@@ -1,0 +1,334 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+the same seeded inputs.  Integer outputs (masks, tile lists, counts) must be
+bit-exact; attention outputs within max-abs 1e-2 / rel-L2 5e-3 (bf16) and
+1e-5 / 1e-6 (fp32)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ap_oracle as orc
+from paper_2012_02030_b200 import inputs
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ap():
+    from paper_2012_02030_b200 import binding
+
+    assert torch.cuda.is_available()
+    return binding
+
+
+W = inputs.WORKLOADS
+
+# ------------------------------------------------------------------------------ tile lists
+
+
+@pytest.mark.parametrize("shape", [(2, 128, 128), (2, 300, 200), (1, 130, 515), (3, 5, 7), (1, 1024, 1024)])
+def test_mask_to_tiles_bit_exact(ap, shape):
+    H, Lq, Lk = shape
+    mask = inputs.random_mask(H, Lq, Lk, 0.01, seed=60)
+    mask[0, : min(128, Lq), : min(128, Lk)] = 1
+    if Lk > 256:
+        mask[:, :, 128:256] = 0
+    tiles = ap.Tiles(H, Lq, Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(mask.numpy()))
+
+
+def test_mask_to_tiles_all_zero_and_capacity_overflow(ap):
+    H, Lq, Lk = 2, 256, 384
+    tiles = ap.Tiles(H, Lq, Lk)
+    ap.ap_mask_to_tiles(torch.zeros((H, Lq, Lk), dtype=torch.uint8, device="cuda"), tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    assert tiles.n_tiles() == 0 and int(tiles.row_ptr.abs().sum()) == 0
+    small = ap.Tiles(H, Lq, Lk, cap=3)
+    ap.ap_mask_to_tiles(torch.ones((H, Lq, Lk), dtype=torch.uint8, device="cuda"), small)
+    assert ap.ap_device_status() == ap.AP_ERR_WORKSPACE   # reported ...
+    assert ap.ap_device_status() == ap.AP_OK              # ... and cleared
+    assert int(small.row_ptr.max()) == 3                  # truncated, never past the capacity
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("L", [(128, 128), (200, 200), (512, 512), (130, 300)])
+def test_dense_tiles_equal_tiles_of_the_full_domain(ap, L, causal):
+    Lq, Lk = L
+    if causal and Lq != Lk:
+        pytest.skip("causal needs Lq == Lk")
+    H = 2
+    dom = torch.ones((H, Lq, Lk), dtype=torch.uint8)
+    if causal:
+        dom = torch.tril(dom)
+    tiles = ap.Tiles(H, Lq, Lk)
+    ap.ap_dense_tiles(tiles, causal=causal)
+    assert ap.ap_device_status() == ap.AP_OK
+    pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(dom.numpy()))
+
+
+# ------------------------------------------------------------------------------ build mask
+
+
+def _check_build_mask(ap, acc32: np.ndarray, w):
+    acc_dev = torch.from_numpy(acc32).cuda()
+    mask, tiles, nnz = pu.gpu_build_mask(ap, acc_dev, w)
+    want_mask, want_nnz = orc.build_mask(acc32, w.keep_frac, w.causal, w.keep_diag)
+    np.testing.assert_array_equal(nnz.cpu().numpy(), want_nnz)
+    np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
+    pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
+    return want_mask
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("keep_diag", [False, True])
+@pytest.mark.parametrize("shape", [(3, 67, 67), (2, 128, 128), (2, 300, 300), (1, 5, 5)])
+def test_build_mask_random_values_with_ties(ap, shape, causal, keep_diag):
+    H, Lq, Lk = shape
+    rng = np.random.default_rng(70)
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc[0].flat[::3] = 0.5                      # a third of head 0 ties at one value
+    acc[-1] = np.round(acc[-1] * 8) / 8         # 9 distinct values: the threshold is always tied
+    acc[0, 0, :3] = [-1.0, -0.0, 0.0]           # negatives and signed zeros
+    for keep in (0.1, 0.5, 1.0):
+        _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=causal, keep_diag=keep_diag,
+                                                     keep_frac=keep))
+
+
+@pytest.mark.parametrize("shape", [(2, 100, 260), (1, 257, 31)])
+def test_build_mask_rectangular(ap, shape):
+    H, Lq, Lk = shape
+    acc = np.random.default_rng(71).random((H, Lq, Lk), dtype=np.float32)
+    acc[0] = np.round(acc[0] * 4) / 4
+    _check_build_mask(ap, acc, W["s2s_cross"].scaled(H=H, Lq=Lq, Lk=Lk, keep_frac=0.3))
+
+
+def test_build_mask_constant_and_tiny_fraction(ap):
+    acc = np.full((2, 130, 130), 0.25, dtype=np.float32)
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=0.37))
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=1e-6))       # forced entries only
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=1e-6, keep_diag=False))
+
+
+def test_build_mask_optional_outputs(ap):
+    acc = np.random.default_rng(72).random((2, 140, 140), dtype=np.float32)
+    acc_dev = torch.from_numpy(acc).cuda()
+    want_mask, _ = orc.build_mask(acc, 0.2, True, True)
+    mask = torch.empty((2, 140, 140), dtype=torch.uint8, device="cuda")
+    ap.ap_build_mask(acc_dev, 0.2, True, True, mask=mask)
+    np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
+    tiles = ap.Tiles(2, 140, 140)
+    ap.ap_build_mask(acc_dev, 0.2, True, True, tiles=tiles)
+    pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
+    assert ap.ap_device_status() == ap.AP_OK
+
+
+# ------------------------------------------------------------------------------ accumulate
+
+
+def _acc_tolerance(dtype):
+    # fp32 FMA dot products + fp32 exp against fp64: relative error of an entry
+    return dict(rtol=2e-5, atol=1e-7)
+
+
+@pytest.mark.parametrize("name,over,n_batches", [
+    ("tiny", {}, 3),
+    ("tiny", dict(Lq=77, Lk=77, B=3), 2),
+    ("tiny", dict(Lq=50, Lk=300, d=128), 2),
+    ("bert", dict(B=4, H=3), 2),
+    ("lm", dict(B=2, H=2, Lq=300, Lk=300), 2),
+    ("long", dict(B=1, H=2, Lq=640, Lk=640), 2),
+])
+def test_accumulate_matches_oracle(ap, name, over, n_batches):
+    w = W[name].scaled(**over)
+    bias = inputs.calib_bias(w)
+    acc = pu.gpu_accumulate(ap, w, n_batches, bias.cuda())
+    again = pu.gpu_accumulate(ap, w, n_batches, bias.cuda())
+    assert torch.equal(acc, again)  # fixed summation order: bit-reproducible
+    want = pu.oracle_accumulate(w, n_batches, bias)
+    got = acc.cpu().numpy()
+    tol = _acc_tolerance(w.dtype)
+    np.testing.assert_allclose(got, want, rtol=tol["rtol"], atol=tol["atol"] * n_batches * w.B)
+    if w.causal:
+        assert np.all(got[:, ~np.tril(np.ones((w.Lq, w.Lk), dtype=bool))] == 0.0)
+    np.testing.assert_allclose(got.sum(-1), n_batches * w.B, rtol=1e-5)
+
+
+def test_accumulate_without_bias_and_custom_scale(ap):
+    w = W["tiny"].scaled(Lq=40, Lk=90)
+    q, k = inputs.calib_qk(w, 0)
+    acc = torch.zeros((w.H, w.Lq, w.Lk), device="cuda")
+    ap.ap_accumulate_attention(acc, q.cuda(), k.cuda(), None, causal=False, scale=0.2)
+    want = np.zeros((w.H, w.Lq, w.Lk))
+    orc.accumulate(want, inputs.widen(q), inputs.widen(k), None, causal=False, scale=0.2)
+    np.testing.assert_allclose(acc.cpu().numpy(), want, rtol=2e-5, atol=1e-7)
+
+
+# ------------------------------------------------------------------------------ forward
+
+
+def _fwd_case(ap, w, mask: torch.Tensor, scale=0.0):
+    q, k, v = inputs.eval_qkv(w)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles, scale=scale)
+    assert ap.ap_device_status() == ap.AP_OK
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy(),
+                            scale=None if scale == 0.0 else scale)
+    pu.assert_close_attention(out, ref, w.dtype, w.name)
+    return out, ref
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("shape", [(2, 2, 128, 128), (1, 2, 200, 333), (2, 1, 513, 130), (1, 1, 5, 7)])
+def test_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
+    B, H, Lq, Lk = shape
+    w = W["tiny"].scaled(B=B, H=H, Lq=Lq, Lk=Lk, d=d, dtype=dtype)
+    mask = inputs.random_mask(H, Lq, Lk, 0.15, seed=80, empty_rows=(0, Lq - 1) if Lq > 2 else ())
+    mask[0, : min(128, Lq), : min(128, Lk)] = 1   # a FULL (or edge-full) tile next to partial ones
+    out, _ = _fwd_case(ap, w, mask)
+    o = out.float().cpu().numpy()
+    if Lq > 2:
+        assert np.all(o[:, 1:, 0] == 0.0) and np.all(o[:, :, Lq - 1] == 0.0)   # rows with no kept entry
+
+
+def test_forward_custom_scale(ap):
+    w = W["tiny"].scaled(B=1, H=2, Lq=150, Lk=150, dtype="bf16")
+    _fwd_case(ap, w, inputs.random_mask(2, 150, 150, 0.3, seed=81), scale=0.31)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_dense_tiles_equal_unpruned_attention(ap, dtype, causal):
+    w = W["tiny"].scaled(B=2, H=2, Lq=300, Lk=300, dtype=dtype)
+    q, k, v = inputs.eval_qkv(w)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_dense_tiles(tiles, causal=causal)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles)
+    dom = torch.ones((w.H, w.Lq, w.Lk), dtype=torch.uint8)
+    if causal:
+        dom = torch.tril(dom)
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), dom.numpy())
+    pu.assert_close_attention(out, ref, dtype)
+
+
+def test_forward_single_kept_entry_copies_value_rows_exactly(ap):
+    w = W["bert"].scaled(B=2, H=2, Lq=260, Lk=260)
+    q, k, v = inputs.eval_qkv(w)
+    eye = torch.eye(260, dtype=torch.uint8).expand(2, 260, 260).contiguous()
+    tiles = ap.Tiles(2, 260, 260)
+    ap.ap_mask_to_tiles(eye.cuda(), tiles)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles)
+    assert torch.equal(out.cpu(), v)
+
+
+# ------------------------------------------------------------------- the five workloads
+
+
+def _pipeline(ap, w, n_batches, oracle_acc=True):
+    """accumulate -> build mask -> forward on the GPU; stage-exact mask check on the
+    GPU's own accumulator bits; forward against the oracle under the GPU-built mask."""
+    bias = inputs.calib_bias(w)
+    acc = pu.gpu_accumulate(ap, w, n_batches, bias.cuda())
+    acc_host = acc.cpu().numpy()
+    if oracle_acc:
+        want_acc = pu.oracle_accumulate(w, n_batches, bias)
+        np.testing.assert_allclose(acc_host, want_acc, rtol=2e-5, atol=1e-7 * n_batches * w.B)
+    mask, tiles, nnz = pu.gpu_build_mask(ap, acc, w)
+    want_mask, want_nnz = orc.build_mask(acc_host, w.keep_frac, w.causal, w.keep_diag)
+    np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
+    np.testing.assert_array_equal(nnz.cpu().numpy(), want_nnz)
+    pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
+    k = orc.keep_count(w.n_valid, w.n_forced, w.keep_frac)
+    assert np.all(want_nnz == k)                       # kept fraction exact per head
+    if oracle_acc:
+        # pure-oracle pipeline: masks may differ only where the average sits at the threshold
+        pure_mask, _ = orc.build_mask(want_acc.astype(np.float32), w.keep_frac, w.causal, w.keep_diag)
+        differ = pure_mask != want_mask
+        if differ.any():
+            for h in range(w.H):
+                forced = np.eye(w.Lq, w.Lk, dtype=bool) if w.n_forced else np.zeros((w.Lq, w.Lk), dtype=bool)
+                kept = want_acc[h][pure_mask[h].astype(bool) & ~forced]
+                tau = kept.min()
+                assert np.all(np.abs(want_acc[h][differ[h]] - tau) <= 4e-5 * tau), h
+    q, kk, v = inputs.eval_qkv(w)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), kk.cuda(), v.cuda(), tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(kk), inputs.widen(v), want_mask)
+    return pu.assert_close_attention(out, ref, w.dtype, w.name)
+
+
+def test_workload_tiny_full(ap):
+    _pipeline(ap, W["tiny"], W["tiny"].calib_batches)
+
+
+@pytest.mark.parametrize("name", ["bert", "lm", "s2s_self", "s2s_cross"])
+def test_workload_full_shape_short_calibration(ap, name):
+    """Full evaluation shape; two calibration batches (the oracle's accumulate is the slow part)."""
+    _pipeline(ap, W[name], 2)
+
+
+def test_workload_long_reduced(ap):
+    """The long-context recipe at L = 1024 (8x8 tiles, causal, d = 128), end to end."""
+    _pipeline(ap, W["long"].scaled(B=2, H=4, Lq=1024, Lk=1024), 2)
+
+
+def test_workload_long_full_size_sampled(ap):
+    """Full size (B4 H16 L4096 d128): accumulator rows, two heads' masks and sampled
+    output rows against the oracle; counts and bitmap popcounts for every head."""
+    w = W["long"]
+    n_batches = 2
+    bias = inputs.calib_bias(w)
+    bias_dev = bias.cuda()
+    acc = pu.gpu_accumulate(ap, w, n_batches, bias_dev)
+    rng = np.random.default_rng(90)
+    rows = [(int(h), int(i)) for h, i in zip(rng.integers(0, w.H, 48), rng.integers(0, w.Lq, 48))]
+    rows += [(0, 0), (w.H - 1, w.Lq - 1), (3, 127), (3, 128)]
+    want_rows = np.zeros((len(rows), w.Lk))
+    for t in range(n_batches):
+        q, k = inputs.calib_qk(w, t)
+        want_rows += orc.accumulate_rows(rows, inputs.widen(q), inputs.widen(k), bias.numpy(), causal=True)
+    got_rows = np.stack([acc[h, i].cpu().numpy() for h, i in rows])
+    np.testing.assert_allclose(got_rows, want_rows, rtol=2e-5, atol=1e-7 * n_batches * w.B)
+    del bias_dev
+
+    mask, tiles, nnz = pu.gpu_build_mask(ap, acc, w)
+    k = orc.keep_count(w.n_valid, w.n_forced, w.keep_frac)
+    assert k == 419533 and torch.all(nnz == k)
+    assert torch.all(mask.view(w.H, -1).sum(-1, dtype=torch.int64) == k)
+    host_tiles = tiles.to_host()
+    pop = np.unpackbits(host_tiles["bitmap"].view(np.uint8)).sum()
+    assert pop == k * w.H
+    heads = [0, 11]
+    sub = acc[heads].cpu().numpy()
+    want_mask, _ = orc.build_mask(sub, w.keep_frac, True, True)
+    np.testing.assert_array_equal(mask[heads].cpu().numpy(), want_mask)
+    mask_host = mask.cpu().numpy()
+    pu.assert_tiles_equal(host_tiles, orc.mask_to_tiles(mask_host))
+
+    q, kk, v = inputs.eval_qkv(w)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), kk.cuda(), v.cuda(), tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    srows = [(int(b), int(h), int(i)) for b, h, i in zip(rng.integers(0, w.B, 2048), rng.integers(0, w.H, 2048),
+                                                        rng.integers(0, w.Lq, 2048))]
+    srows += [(0, 0, 0), (0, 0, 1), (w.B - 1, w.H - 1, w.Lq - 1)]
+    ref = orc.attention_rows(inputs.widen(q), inputs.widen(kk), inputs.widen(v), mask_host, srows)
+    idx = np.array(srows)
+    got = out[idx[:, 0], idx[:, 1], idx[:, 2]]
+    pu.assert_close_attention(got, ref, "bf16", "long/sampled")
+
+
+def test_host_buffer_entry_point(ap):
+    w = W["bert"].scaled(B=2, H=2)
+    q, k, v = (t.pin_memory() for t in inputs.eval_qkv(w))
+    mask = inputs.random_mask(w.H, w.Lq, w.Lk, 0.5, seed=91)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    ho = torch.empty_like(q).pin_memory()
+    dq, dk, dv, do = (torch.empty_like(t, device="cuda") for t in (q, k, v, q))
+    ap.ap_sparse_attention_fwd_host(q, k, v, tiles, ho, dq, dk, dv, do)
+    assert ap.ap_device_status() == ap.AP_OK
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy())
+    pu.assert_close_attention(ho, ref, "bf16")
