@@ -190,8 +190,10 @@ def test_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
     mask[0, : min(128, Lq), : min(128, Lk)] = 1   # a FULL (or edge-full) tile next to partial ones
     out, _ = _fwd_case(ap, w, mask)
     o = out.float().cpu().numpy()
-    if Lq > 2:
-        assert np.all(o[:, 1:, 0] == 0.0) and np.all(o[:, :, Lq - 1] == 0.0)   # rows with no kept entry
+    empty = mask.numpy().sum(-1) == 0                  # rows with no kept entry output exact zeros
+    if H > 1 or Lq > 128:
+        assert empty.any()
+    assert np.all(o[:, empty] == 0.0)
 
 
 def test_forward_custom_scale(ap):
