@@ -138,6 +138,33 @@ ap_status ap_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles 
                            void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * ap_mask_to_tiles for callers that cannot allocate device memory (the paper has
+ * no counterpart for this entry point; it exists for the library's users only).
+ * Who needs it: code that runs where cudaMalloc is off limits - a plugin living
+ * inside another framework's memory pool, a latency-critical loop that must not
+ * enter the allocator, a process whose memory budget is fixed at start-up.
+ * Instead of a caller-provided workspace the staging area is a fixed array in
+ * device global memory that is part of the library image: every GPU that loads
+ * the library holds AP_STATIC_SCRATCH_BYTES (about 2.1 MB) of it until exit.
+ *   - Inputs and outputs are the caller's, exactly as for ap_mask_to_tiles, and
+ *     the resulting tile list is identical bit for bit.
+ *   - Limit: H * ceil(Lq/128) * ceil(Lk/128) <= AP_STATIC_MAX_TILES; larger shapes
+ *     return AP_ERR_WORKSPACE before anything is enqueued.
+ *   - The call itself allocates nothing (no cudaMalloc/cudaFree, no allocating
+ *     library routine).  The first call on each device looks up the array's
+ *     device address (cudaGetSymbolAddress, with that device current); make that
+ *     first call before starting any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents.
+ *     Each call overwrites everything it later reads, so a stale array is
+ *     harmless, but two calls that overlap on the GPU (different streams, no
+ *     ordering between them) race on it: serialise them.
+ */
+#define AP_STATIC_MAX_TILES 1024
+#define AP_STATIC_SCRATCH_BYTES (AP_STATIC_MAX_TILES * (128 * 4 * 4 + 8))
+ap_status ap_mask_to_tiles_static(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles *tiles,
+                                  void *stream);
+
+/*
  * Tile list of the unpruned attention (the zero mask matrix of Section 3.2):
  * every tile of the domain, written without reading any mask.  This is the
  * library's dense path and the baseline the sparse path is compared with.

@@ -16,6 +16,7 @@ import torch
 TILE = 128
 AP_OK, AP_ERR_INVALID_ARG, AP_ERR_UNSUPPORTED, AP_ERR_WORKSPACE, AP_ERR_CUDA, AP_ERR_TIMEOUT = range(6)
 AP_F32, AP_BF16 = 0, 1
+AP_STATIC_MAX_TILES = 1024
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libap_b200.so")
 
@@ -55,6 +56,7 @@ def _load() -> ctypes.CDLL:
         "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_mask_to_tiles": (i, [vp, i, i, i, tp, vp, sz, vp]),
         "ap_dense_tiles": (i, [i, i, i, i, tp, vp]),
+        "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
         "ap_sparse_attention_fwd": (i, [vp, vp, vp, tp, vp, i, i, i, i, i, i, f, vp]),
         "ap_sparse_attention_fwd_host": (i, [vp, vp, vp, tp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, vp]),
         "ap_device_status": (i, [vp]),
@@ -68,7 +70,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
            "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask",
-           "ap_mask_to_tiles", "ap_dense_tiles", "ap_sparse_attention_fwd",
+           "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
            "ap_sparse_attention_fwd_host", "ap_device_status")
 
 
@@ -190,6 +192,18 @@ def ap_mask_to_tiles(mask, tiles: Tiles, workspace=None, stream=None) -> None:
         workspace = torch.empty(ap_mask_to_tiles_workspace_bytes(H, Lq, Lk), dtype=torch.uint8, device=mask.device)
     _check(lib.ap_mask_to_tiles(_ptr(mask), H, Lq, Lk, ctypes.byref(tiles.c), _ptr(workspace),
                                 workspace.numel(), _stream(stream)), "ap_mask_to_tiles")
+
+
+def ap_mask_to_tiles_static(mask, tiles: Tiles, stream=None) -> None:
+    """ap_mask_to_tiles without a workspace: the staging area is the library's built-in
+    device array (shapes of at most AP_STATIC_MAX_TILES grid tiles).  The binding passes
+    the caller's mask and tile buffers straight through and allocates nothing."""
+    _dev(mask, "mask")
+    H, Lq, Lk = mask.shape
+    if mask.dtype != torch.uint8:
+        raise ValueError("mask must be uint8")
+    _check(lib.ap_mask_to_tiles_static(_ptr(mask), H, Lq, Lk, ctypes.byref(tiles.c), _stream(stream)),
+           "ap_mask_to_tiles_static")
 
 
 def ap_dense_tiles(tiles: Tiles, causal=False, stream=None) -> None:
