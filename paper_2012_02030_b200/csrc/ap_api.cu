@@ -221,7 +221,9 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V, c
   if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
-  cudaError_t e = launch_fwd_simt(Q, K, V, *tiles, O, B, H, Lq, Lk, d, dt, sc, static_cast<cudaStream_t>(stream));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = dt == AP_F32 ? launch_fwd_simt(Q, K, V, *tiles, O, B, H, Lq, Lk, d, sc, s)
+                               : launch_fwd_tc(Q, K, V, *tiles, O, B, H, Lq, Lk, d, sc, s);
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 

@@ -59,8 +59,11 @@ cudaError_t launch_accumulate_simt(float *acc, const void *Q, const void *K, con
                                    int H, int Lq, int Lk, int d, ap_dtype dt, int causal, float scale,
                                    cudaStream_t s);
 
+// fp32 tensors: CUDA-core kernel
 cudaError_t launch_fwd_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
-                            int B, int H, int Lq, int Lk, int d, ap_dtype dt, float scale,
-                            cudaStream_t s);
+                            int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
+// bf16 tensors: tcgen05 tensor-core kernel
+cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
+                          int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
 
 }  // namespace ap

@@ -160,13 +160,9 @@ cudaError_t launch(const void *Q, const void *K, const void *V, const ap_tiles &
 }  // namespace
 
 cudaError_t launch_fwd_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O, int B, int H,
-                            int Lq, int Lk, int d, ap_dtype dt, float scale, cudaStream_t s) {
-  if (dt == AP_F32) {
-    return d == 64 ? launch<float, 64>(Q, K, V, t, O, B, H, Lq, Lk, scale, s)
-                   : launch<float, 128>(Q, K, V, t, O, B, H, Lq, Lk, scale, s);
-  }
-  return d == 64 ? launch<__nv_bfloat16, 64>(Q, K, V, t, O, B, H, Lq, Lk, scale, s)
-                 : launch<__nv_bfloat16, 128>(Q, K, V, t, O, B, H, Lq, Lk, scale, s);
+                            int Lq, int Lk, int d, float scale, cudaStream_t s) {
+  return d == 64 ? launch<float, 64>(Q, K, V, t, O, B, H, Lq, Lk, scale, s)
+                 : launch<float, 128>(Q, K, V, t, O, B, H, Lq, Lk, scale, s);
 }
 
 }  // namespace ap
