@@ -197,7 +197,7 @@ def run_gpu(args, w):
     flush = None if resident > 400e6 else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     # the calibration set proper (untimed): the mask the steps work with is the real one
-    for t in range(w.calib_batches):
+    for t in range(args.calib_batches if args.calib_batches > 0 else w.calib_batches):
         cq, ck = inputs.calib_qk(w, t)
         ap.ap_accumulate_attention(acc, cq.to(dev), ck.to(dev), bias, causal=w.causal)
     torch.cuda.synchronize()
@@ -376,6 +376,9 @@ def main():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--workload", default="long", choices=sorted(inputs.WORKLOADS))
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--calib-batches", type=int, default=0,
+                   help="calibration batches accumulated before the timed steps (0 = the workload's own count); "
+                        "profiling runs use a small number to keep the launch list short")
     args = p.parse_args()
     w = inputs.WORKLOADS[args.workload]
     if args.impl == "reference":

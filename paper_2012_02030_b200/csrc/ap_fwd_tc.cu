@@ -218,7 +218,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const int r = warp * 32 + lane;          // row of the query tile == TMEM lane
     const int i = qt * kTile + r;
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-    float m = -CUDART_INF_F, l = 0.f;
+    float m = -CUDART_INF_F, l = 0.f;       // exponent reference and running sum of weights
+    const float ref_slack = 8.f / scale_log2;
     bool ok = true;
     uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)t_begin * kBitmapWords + r * 4);
     bool full = flags[t_begin] & 1;
@@ -232,26 +233,38 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       ok = wait_or_abort(&bars->s_full, (uint32_t)it & 1u, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
+      // 32-column chunks in which none of this warp's 32 rows keeps anything are skipped
+      // (their P is written as zeros without reading S)
+      const uint32_t w0 = tile_full ? 0xffffffffu : cur.x, w1 = tile_full ? 0xffffffffu : cur.y,
+                     w2 = tile_full ? 0xffffffffu : cur.z, w3 = tile_full ? 0xffffffffu : cur.w;
+      const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u) |
+                              (__any_sync(0xffffffffu, w2 != 0u) ? 4u : 0u) | (__any_sync(0xffffffffu, w3 != 0u) ? 8u : 0u);
       // pass 1: row maximum over kept entries
       float tile_max = -CUDART_INF_F;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
+        if (!((active >> c) & 1u)) continue;
         uint32_t x[32];
         tmem_ld32(tmem_s + lane_addr + 32 * c, x);
         tmem_wait_ld();
-        const uint32_t w = tile_full ? 0xffffffffu : (c == 0 ? cur.x : c == 1 ? cur.y : c == 2 ? cur.z : cur.w);
+        const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const float v = (w >> e) & 1u ? __uint_as_float(x[e]) : -CUDART_INF_F;
           tile_max = fmaxf(tile_max, v);
         }
       }
-      const float m_new = fmaxf(m, tile_max);
+      // The exponent's reference m follows the running maximum lazily: it moves only when
+      // the maximum outgrows it by more than 2^8 in the exp2 domain (weights stay <= 256,
+      // well inside bf16 and fp32 range), which saves most rescales of O.  O / l does not
+      // depend on the reference.
+      const bool move = tile_max > m + ref_slack;   // also true for the first kept entry (m = -inf)
+      const float m_new = move ? tile_max : m;
       const float m_safe = m_new == -CUDART_INF_F ? 0.f : m_new;
-      const float alpha = ex2_approx((m - m_safe) * scale_log2);  // 0 when m = -inf, 1 when unchanged
+      const float alpha = move ? ex2_approx((m - m_safe) * scale_log2) : 1.f;  // 0 when m was -inf
       const float neg_mc = -m_safe * scale_log2;
       m = m_new;
-      // rescale the running output when some row's maximum moved (O of step it-1 is complete:
+      // rescale the running output where the reference moved (O of step it-1 is complete:
       // the MMA thread committed s_full after it)
       if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
@@ -268,11 +281,17 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       float sum = 0.f;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+        if (!((active >> c) & 1u)) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) pk[e] = 0u;
+          tmem_st16(tmem_s + lane_addr + 16 * c, pk);
+          continue;
+        }
         uint32_t x[32];
         tmem_ld32(tmem_s + lane_addr + 32 * c, x);
         tmem_wait_ld();
-        const uint32_t w = tile_full ? 0xffffffffu : (c == 0 ? cur.x : c == 1 ? cur.y : c == 2 ? cur.z : cur.w);
-        uint32_t pk[16];
+        const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
