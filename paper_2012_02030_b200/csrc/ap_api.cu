@@ -130,8 +130,10 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
   if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
-  cudaError_t e = launch_accumulate_simt(acc, Q, K, bias, B, H, Lq, Lk, d, dt, causal ? 1 : 0, sc,
-                                         static_cast<cudaStream_t>(stream));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == AP_BF16 && !device_error_word()) return AP_ERR_CUDA;
+  cudaError_t e = dt == AP_F32 ? launch_accumulate_simt(acc, Q, K, bias, B, H, Lq, Lk, d, dt, causal ? 1 : 0, sc, s)
+                               : launch_accumulate_tc(acc, Q, K, bias, B, H, Lq, Lk, d, causal ? 1 : 0, sc, s);
   if (e == cudaErrorInvalidValue) return AP_ERR_UNSUPPORTED;  // key length beyond the shared-memory budget
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }

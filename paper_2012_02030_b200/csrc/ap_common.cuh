@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -62,6 +63,14 @@ cudaError_t launch_accumulate_simt(float *acc, const void *Q, const void *K, con
 // fp32 tensors: CUDA-core kernel
 cudaError_t launch_fwd_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
                             int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
+cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
+                                 int Lq, int Lk, int d, int causal, float scale, cudaStream_t s);
+
+// Tensor map of a [B*H, L, d] bf16 tensor for 128-row x 64-element swizzled boxes.
+bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d);
+// Tensor map of an [H, Lq, Lk] fp32 tensor for 128-row x 32-column swizzled boxes (Lk % 4 == 0).
+bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk);
+
 // bf16 tensors: tcgen05 tensor-core kernel
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
                           int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);

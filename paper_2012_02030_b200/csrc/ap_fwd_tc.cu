@@ -345,36 +345,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (warp == 5) tmem_dealloc(tmem, kTmemCols);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void *p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// [B*H, L, d] bf16 tensor, boxes of 128 rows x 64 elements, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap *m, const void *base, int BH, int L, int d) {
-  EncodeTiledFn enc = encode_fn();
-  if (!enc) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)L, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)L * d * 2};
-  cuuint32_t box[3] = {64, 128, 1};
-  cuuint32_t elem_strides[3] = {1, 1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, elem_strides,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int D>
 cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, void *O, const ap_tiles &t,
                    int B, int H, int Lq, float scale, unsigned *err, cudaStream_t s) {
@@ -396,7 +366,8 @@ cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, Q, B * H, Lq, d) || !make_map(&mk, K, B * H, Lk, d) || !make_map(&mv, V, B * H, Lk, d))
+  if (!make_tile_map_bf16(&mq, Q, B * H, Lq, d) || !make_tile_map_bf16(&mk, K, B * H, Lk, d) ||
+      !make_tile_map_bf16(&mv, V, B * H, Lk, d))
     return cudaErrorUnknown;
   return d == 64 ? launch<64>(mq, mk, mv, O, t, B, H, Lq, scale, err, s)
                  : launch<128>(mq, mk, mv, O, t, B, H, Lq, scale, err, s);
