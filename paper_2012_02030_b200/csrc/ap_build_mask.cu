@@ -3,11 +3,13 @@
 // Order of the entries of one head: forced (diagonal) first, then larger fp32
 // value, then lower linear index i*Lk + j.  The k-th entry of that order is
 // found with a most-significant-digit-first radix select over order-preserving
-// 32-bit keys (four 8-bit digits, one histogram pass over the accumulator
-// each); ties with the threshold key are ranked by linear index with per-row-
-// segment tie counts and a prefix sum, so exactly k entries are kept.  The
-// emit pass writes the element mask and per-tile bitmaps; ap_tiles.cu compacts
-// them.  Integer work throughout: no floating-point arithmetic decides a bit.
+// 32-bit keys: three digits of 11, 11 and 10 bits, one histogram pass over the
+// accumulator each.  Entries equal to the threshold key are all kept when the
+// count allows it (the usual case); otherwise they are ranked by linear index
+// with per-row-segment tie counts and a prefix sum, so that exactly k entries
+// are kept.  The emit pass writes the element mask and per-tile bitmaps;
+// ap_tiles.cu compacts them.  Integer work throughout: no floating-point
+// arithmetic decides a bit.
 #include "ap_common.cuh"
 
 namespace ap {
@@ -16,6 +18,11 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
+constexpr int kBins = 2048;
+constexpr int kPasses = 3;
+
+__host__ __device__ constexpr int digit_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
+__host__ __device__ constexpr uint32_t digit_mask(int pass) { return pass == 2 ? 0x3ffu : 0x7ffu; }
 
 // Larger float <=> larger key; -0 is mapped onto +0 first.
 __device__ __forceinline__ uint32_t key_of(float f) {
@@ -29,10 +36,12 @@ struct SelectState {  // per head
   uint32_t thr;       // threshold key (valid after the last digit)
   unsigned long long remaining;  // rank still to resolve inside the current prefix
   unsigned long long ties_kept;  // entries equal to thr that are kept (lowest indices first)
+  uint32_t all_ties_kept;        // every entry equal to thr is kept: no ranking needed
+  uint32_t pad;
 };
 
 struct Scratch {
-  uint32_t *hist;       // [H][256]
+  uint32_t *hist;       // [H][kBins]
   SelectState *state;   // [H]
   uint32_t *tie_count;  // [H][Lq][n_kt] -> exclusive prefix after the scan
 };
@@ -54,95 +63,131 @@ __device__ __forceinline__ void load4(const float *__restrict__ row, int j0, int
 __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int H, unsigned long long k_rest,
                                   long long k, int64_t *nnz) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx < H * 256) hist[idx] = 0u;
+  if (idx < H * kBins) hist[idx] = 0u;
   if (idx < H) {
     state[idx].prefix = 0u;
     state[idx].thr = 0xffffffffu;
     state[idx].remaining = k_rest;
     state[idx].ties_kept = 0ull;
+    state[idx].all_ties_kept = 0u;
+    state[idx].pad = 0u;
     if (nnz) nnz[idx] = k;
   }
 }
 
-// Histogram of one 8-bit digit over the non-forced domain entries whose higher
-// digits equal the prefix found so far.  grid = (row blocks, H); a warp takes a
-// row at a time, lanes stride over the row in float4 steps.
+// Histogram of one digit over the non-forced domain entries whose higher digits
+// equal the prefix found so far.  grid = (row blocks, H); a warp takes a row at
+// a time and its lanes stride over the row, two float4 loads in flight each.
 __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *__restrict__ acc, int Lq, int Lk,
                                                                    int causal, int diag, int pass,
                                                                    const SelectState *__restrict__ state,
                                                                    uint32_t *__restrict__ hist) {
-  __shared__ uint32_t sh[kWarps][256];
+  __shared__ uint32_t sh[kBins];
   const int h = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int b = threadIdx.x; b < kWarps * 256; b += kThreads) (&sh[0][0])[b] = 0u;
+  for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0u;
   __syncthreads();
-  const int shift = 24 - 8 * pass;
+  const int shift = digit_shift(pass);
+  const uint32_t dmask = digit_mask(pass);
   const uint32_t prefix = state[h].prefix;
-  const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+  const uint32_t hi_mask = pass == 0 ? 0u : ~((1u << (shift + (pass == 1 ? 11 : 10))) - 1u);
+  const uint32_t want_hi = prefix & hi_mask;
   const bool vec = (Lk & 3) == 0;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
     const int jend = causal ? min(Lk, i + 1) : Lk;
-    for (int base = 0; base < jend; base += 128) {  // warp-uniform trip count
-      const int j0 = base + 4 * lane;
-      float v[4] = {0.f, 0.f, 0.f, 0.f};
-      if (j0 < jend) load4(row, j0, jend, vec, v);
+    for (int base = 0; base < jend; base += 256) {  // warp-uniform trip count
+      float v[2][4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int j = j0 + c;
-        const uint32_t key = key_of(v[c]);
-        const bool take = j < jend && !(diag && j == i) && ((key & hi_mask) == (prefix & hi_mask));
-        const uint32_t bin = (key >> shift) & 255u;
-        // lanes that hit the same bin elect one to add their count
-        const unsigned voters = __ballot_sync(0xffffffffu, take);
-        if (take) {
-          const unsigned peers = __match_any_sync(voters, bin);
-          if (lane == __ffs(peers) - 1) atomicAdd(&sh[warp][bin], (uint32_t)__popc(peers));
+      for (int u = 0; u < 2; ++u) {
+        const int j0 = base + 128 * u + 4 * lane;
+        v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+        if (j0 < jend) load4(row, j0, jend, vec, v[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int j0 = base + 128 * u + 4 * lane;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int j = j0 + c;
+          const uint32_t key = key_of(v[u][c]);
+          const bool take = j < jend && !(diag && j == i) && ((key & hi_mask) == want_hi);
+          const uint32_t bin = (key >> shift) & dmask;
+          // lanes that hit the same bin elect one to add their count
+          const unsigned voters = __ballot_sync(0xffffffffu, take);
+          if (take) {
+            const unsigned peers = __match_any_sync(voters, bin);
+            if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], (uint32_t)__popc(peers));
+          }
         }
       }
     }
   }
   __syncthreads();
-  for (int b = threadIdx.x; b < 256; b += kThreads) {
-    uint32_t s = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) s += sh[w][b];
-    if (s) atomicAdd(&hist[h * 256 + b], s);
+  for (int b = threadIdx.x; b < kBins; b += kThreads) {
+    const uint32_t s = sh[b];
+    if (s) atomicAdd(&hist[h * kBins + b], s);
   }
 }
 
-// One CTA per head: picks the digit whose bin contains the wanted rank.
+// One CTA per head: picks the digit whose bin contains the wanted rank.  Thread t
+// owns bins [kBins-1-8t, kBins-8-8t] (descending); a block-wide prefix over the
+// threads' sums locates the owner, which then walks its eight bins.
 __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass) {
-  __shared__ uint32_t cnt[256];
+  __shared__ uint32_t warp_sums[8];
   const int h = blockIdx.x;
-  cnt[threadIdx.x] = hist[h * 256 + threadIdx.x];
-  hist[h * 256 + threadIdx.x] = 0u;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t cnt[8];
+  uint32_t mine = 0u;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int bin = kBins - 1 - (8 * (int)threadIdx.x + e);
+    cnt[e] = hist[h * kBins + bin];
+    hist[h * kBins + bin] = 0u;
+    mine += cnt[e];
+  }
+  uint32_t incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  const SelectState st = state[h];  // read by everyone before the barrier, written by the owner after it
   __syncthreads();
-  if (threadIdx.x == 0) {
-    SelectState st = state[h];
-    unsigned long long above = 0ull;
-    int bin = 255;
-    for (; bin > 0; --bin) {
-      if (above + cnt[bin] >= st.remaining) break;
-      above += cnt[bin];
+  unsigned long long before = incl - mine;  // entries in bins above this thread's
+  for (int w = 0; w < warp; ++w) before += warp_sums[w];
+  // the owner: fewer than `remaining` entries above its bins, at least that many including them;
+  // the last thread also takes the case of an over-long rank (cannot happen for valid k)
+  const bool owner = before < st.remaining && (before + mine >= st.remaining || threadIdx.x == 255);
+  if (owner) {
+    unsigned long long above = before;
+    int e = 0;
+    for (; e < 7; ++e) {
+      if (above + cnt[e] >= st.remaining) break;
+      above += cnt[e];
     }
-    st.remaining -= above;
-    st.prefix |= (uint32_t)bin << (24 - 8 * pass);
-    if (pass == 3) {
-      st.thr = st.prefix;
-      st.ties_kept = st.remaining;
+    const int bin = kBins - 1 - (8 * (int)threadIdx.x + e);
+    SelectState out = st;
+    out.remaining = st.remaining - above;
+    out.prefix = st.prefix | ((uint32_t)bin << digit_shift(pass));
+    if (pass == kPasses - 1) {
+      out.thr = out.prefix;
+      out.ties_kept = out.remaining;
+      out.all_ties_kept = out.remaining == cnt[e] ? 1u : 0u;
     }
-    state[h] = st;
+    state[h] = out;
   }
 }
 
-// Entries equal to the threshold key per (row, 128-column segment).
-// grid = (row blocks, H); a warp takes a row, then its segments in turn.
+// Entries equal to the threshold key per (row, 128-column segment); only for heads
+// where the ties must be ranked.  grid = (row blocks, H); a warp takes a row.
 __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_kt,
                                                              int causal, int diag,
                                                              const SelectState *__restrict__ state,
                                                              uint32_t *__restrict__ tie_count) {
   const int h = blockIdx.y;
+  if (state[h].all_ties_kept) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t thr = state[h].thr;
   const bool vec = (Lk & 3) == 0;
@@ -169,7 +214,9 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
 }
 
 // One CTA per head: in-place exclusive prefix sum over the head's (row, segment) tie counts.
-__global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ tie_count, int n_per_head) {
+__global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ tie_count, int n_per_head,
+                                                        const SelectState *__restrict__ state) {
+  if (state[blockIdx.x].all_ties_kept) return;
   __shared__ uint32_t warp_sums[32];
   __shared__ uint32_t carry_s;
   uint32_t *a = tie_count + (size_t)blockIdx.x * n_per_head;
@@ -206,8 +253,8 @@ __global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ t
 }
 
 // One CTA per tile of the (h, qt, kt) grid; warp w takes tile rows w, w+4, ...
-// and each lane four consecutive columns.  Writes the element mask, the tile's
-// bitmap and popcount into the staging area.
+// (four rows loaded ahead) and each lane four consecutive columns.  Writes the
+// element mask, the tile's bitmap and popcount into the staging area.
 __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_qt, int n_kt,
                                                    int causal, int diag, const SelectState *__restrict__ state,
                                                    const uint32_t *__restrict__ tie_prefix,
@@ -220,74 +267,88 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t thr = state[h].thr;
   const unsigned long long ties_kept = state[h].ties_kept;
+  const bool all_ties = state[h].all_ties_kept != 0u;
   const bool vec = (Lk & 3) == 0;
+  const int j0 = kt * kTile + 4 * lane;
   __shared__ int warp_count[4];
   int count = 0;
-  for (int r = warp; r < kTile; r += 4) {
-    const int i = qt * kTile + r;
-    const int j0 = kt * kTile + 4 * lane;
-    uint32_t nib = 0u;
-    if (i < Lq) {  // warp-uniform
-      const float *row = acc + ((size_t)h * Lq + i) * Lk;
-      const int jend = causal ? min(Lk, i + 1) : Lk;
-      float v[4] = {0.f, 0.f, 0.f, 0.f};
-      if (j0 < jend) load4(row, j0, jend, vec, v);
-      uint32_t tie_bits = 0u, gt_bits = 0u;
+  for (int r0 = warp; r0 < kTile; r0 += 16) {
+    float v[4][4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int j = j0 + c;
-        if (j < jend) {
-          if (diag && j == i) {
-            gt_bits |= 1u << c;
-          } else {
-            const uint32_t key = key_of(v[c]);
-            if (key > thr) gt_bits |= 1u << c;
-            if (key == thr) tie_bits |= 1u << c;
-          }
-        }
-      }
-      nib = gt_bits;
-      if (__any_sync(0xffffffffu, tie_bits != 0u)) {
-        // rank of each tie in linear-index order = ties before this row segment
-        // + ties in lower lanes + ties in lower columns of this lane
-        int before = __popc(tie_bits);
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          int u = __shfl_up_sync(0xffffffffu, before, o);
-          if (lane >= o) before += u;
-        }
-        before -= __popc(tie_bits);
-        unsigned long long rank = (unsigned long long)tie_prefix[((size_t)h * Lq + i) * n_kt + kt] + before;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (tie_bits & (1u << c)) {
-            if (rank < ties_kept) nib |= 1u << c;
-            ++rank;
-          }
-        }
-      }
-      if (mask) {
-        uint8_t *mrow = mask + ((size_t)h * Lq + i) * Lk;
-        if (vec && j0 + 4 <= Lk) {
-          *reinterpret_cast<uchar4 *>(mrow + j0) =
-              make_uchar4(nib & 1u, (nib >> 1) & 1u, (nib >> 2) & 1u, (nib >> 3) & 1u);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            if (j0 + c < Lk) mrow[j0 + c] = (nib >> c) & 1u;
-        }
+    for (int u = 0; u < 4; ++u) {  // rows r0, r0+4, r0+8, r0+12: four loads in flight
+      const int i = qt * kTile + r0 + 4 * u;
+      v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+      if (i < Lq) {
+        const int jend = causal ? min(Lk, i + 1) : Lk;
+        if (j0 < jend) load4(acc + ((size_t)h * Lq + i) * Lk, j0, jend, vec, v[u]);
       }
     }
-    // 8 lanes x 4 bits -> one bitmap word
-    uint32_t w = nib << (4 * (lane & 7));
-    w |= __shfl_xor_sync(0xffffffffu, w, 1);
-    w |= __shfl_xor_sync(0xffffffffu, w, 2);
-    w |= __shfl_xor_sync(0xffffffffu, w, 4);
-    const uint32_t w0 = __shfl_sync(0xffffffffu, w, 0), w1 = __shfl_sync(0xffffffffu, w, 8),
-                   w2 = __shfl_sync(0xffffffffu, w, 16), w3 = __shfl_sync(0xffffffffu, w, 24);
-    count += __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
-    if (stage_bitmap && lane == 0)
-      reinterpret_cast<uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords)[r] = make_uint4(w0, w1, w2, w3);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + 4 * u;
+      const int i = qt * kTile + r;
+      uint32_t nib = 0u;
+      if (i < Lq) {  // warp-uniform
+        const int jend = causal ? min(Lk, i + 1) : Lk;
+        uint32_t tie_bits = 0u, gt_bits = 0u;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int j = j0 + c;
+          if (j < jend) {
+            if (diag && j == i) {
+              gt_bits |= 1u << c;
+            } else {
+              const uint32_t key = key_of(v[u][c]);
+              if (key > thr) gt_bits |= 1u << c;
+              if (key == thr) tie_bits |= 1u << c;
+            }
+          }
+        }
+        nib = gt_bits;
+        if (all_ties) {
+          nib |= tie_bits;
+        } else if (__any_sync(0xffffffffu, tie_bits != 0u)) {
+          // rank of each tie in linear-index order = ties before this row segment
+          // + ties in lower lanes + ties in lower columns of this lane
+          int before = __popc(tie_bits);
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, before, o);
+            if (lane >= o) before += t;
+          }
+          before -= __popc(tie_bits);
+          unsigned long long rank = (unsigned long long)tie_prefix[((size_t)h * Lq + i) * n_kt + kt] + before;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (tie_bits & (1u << c)) {
+              if (rank < ties_kept) nib |= 1u << c;
+              ++rank;
+            }
+          }
+        }
+        if (mask) {
+          uint8_t *mrow = mask + ((size_t)h * Lq + i) * Lk;
+          if (vec && j0 + 4 <= Lk) {
+            *reinterpret_cast<uchar4 *>(mrow + j0) =
+                make_uchar4(nib & 1u, (nib >> 1) & 1u, (nib >> 2) & 1u, (nib >> 3) & 1u);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if (j0 + c < Lk) mrow[j0 + c] = (nib >> c) & 1u;
+          }
+        }
+      }
+      // 8 lanes x 4 bits -> one bitmap word
+      uint32_t w = nib << (4 * (lane & 7));
+      w |= __shfl_xor_sync(0xffffffffu, w, 1);
+      w |= __shfl_xor_sync(0xffffffffu, w, 2);
+      w |= __shfl_xor_sync(0xffffffffu, w, 4);
+      const uint32_t w0 = __shfl_sync(0xffffffffu, w, 0), w1 = __shfl_sync(0xffffffffu, w, 8),
+                     w2 = __shfl_sync(0xffffffffu, w, 16), w3 = __shfl_sync(0xffffffffu, w, 24);
+      count += __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
+      if (stage_bitmap && lane == 0)
+        reinterpret_cast<uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords)[r] = make_uint4(w0, w1, w2, w3);
+    }
   }
   if (lane == 0) warp_count[warp] = count;
   __syncthreads();
@@ -299,7 +360,7 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
   char *p = static_cast<char *>(scratch);
   Scratch s;
   s.hist = reinterpret_cast<uint32_t *>(p);
-  p += align256((size_t)H * 256 * sizeof(uint32_t));
+  p += align256((size_t)H * kBins * sizeof(uint32_t));
   s.state = reinterpret_cast<SelectState *>(p);
   p += align256((size_t)H * sizeof(SelectState));
   s.tie_count = reinterpret_cast<uint32_t *>(p);
@@ -309,7 +370,7 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
 }  // namespace
 
 size_t select_scratch_bytes(int H, int Lq, int Lk) {
-  return align256((size_t)H * 256 * sizeof(uint32_t)) + align256((size_t)H * sizeof(SelectState)) +
+  return align256((size_t)H * kBins * sizeof(uint32_t)) + align256((size_t)H * sizeof(SelectState)) +
          align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t));
 }
 
@@ -318,8 +379,8 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   const int diag = (a.keep_diag && a.Lq == a.Lk) ? 1 : 0;
   Scratch sc = carve(a.scratch, a.H, a.Lq, a.Lk);
   cudaError_t e;
-  init_state_kernel<<<ceil_div(a.H * 256, 256), 256, 0, s>>>(sc.state, sc.hist, a.H,
-                                                            (unsigned long long)a.k_rest, (long long)a.k, a.nnz);
+  init_state_kernel<<<ceil_div(a.H * kBins, 256), 256, 0, s>>>(sc.state, sc.hist, a.H,
+                                                              (unsigned long long)a.k_rest, (long long)a.k, a.nnz);
   count_launches(1);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // enough CTAs per head to fill the GPU, at most one warp-row each
@@ -328,19 +389,20 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   if (row_blocks > want) row_blocks = want;
   dim3 grid(row_blocks, a.H);
   if (a.k_rest > 0) {
-    for (int pass = 0; pass < 4; ++pass) {
+    for (int pass = 0; pass < kPasses; ++pass) {
       digit_histogram_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, pass, sc.state, sc.hist);
-  count_launches(1);
+      count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
       pick_digit_kernel<<<a.H, 256, 0, s>>>(sc.state, sc.hist, pass);
-  count_launches(1);
+      count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
+    // both return at once for heads whose ties with the threshold are all kept
     tie_count_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, n_kt, a.causal, diag, sc.state, sc.tie_count);
-  count_launches(1);
+    count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    tie_scan_kernel<<<a.H, 1024, 0, s>>>(sc.tie_count, a.Lq * n_kt);
-  count_launches(1);
+    tie_scan_kernel<<<a.H, 1024, 0, s>>>(sc.tie_count, a.Lq * n_kt, sc.state);
+    count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, sc.state,
