@@ -44,7 +44,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the ncu
 # captures summarised under profiles/ (None until a capture exists).
-NCU_FWD_TRAFFIC_BYTES = {}
+NCU_FWD_TRAFFIC_BYTES = {"long": 422.9e6}  # profiles/long_workload_ncu.md
 
 
 def load_peaks():
