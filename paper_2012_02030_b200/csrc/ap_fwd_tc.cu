@@ -239,21 +239,33 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                      w2 = tile_full ? 0xffffffffu : cur.z, w3 = tile_full ? 0xffffffffu : cur.w;
       const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u) |
                               (__any_sync(0xffffffffu, w2 != 0u) ? 4u : 0u) | (__any_sync(0xffffffffu, w3 != 0u) ? 8u : 0u);
-      // pass 1: row maximum over kept entries
-      float tile_max = -CUDART_INF_F;
+      // pass 1: row maximum over kept entries (four independent chains).  In a partially filled
+      // tile the pruned entries are replaced by -inf and the chunk is written back to TMEM, so
+      // that pass 2 needs no bitmap: exp2 of -inf is exactly 0.
+      float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         if (!((active >> c) & 1u)) continue;
         uint32_t x[32];
         tmem_ld32(tmem_s + lane_addr + 32 * c, x);
         tmem_wait_ld();
-        const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
+        if (!tile_full) {
+          const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float v = (w >> e) & 1u ? __uint_as_float(x[e]) : -CUDART_INF_F;
-          tile_max = fmaxf(tile_max, v);
+          for (int e = 0; e < 32; ++e)
+            if (!((w >> e) & 1u)) x[e] = 0xff800000u;  // -inf
+          tmem_st32(tmem_s + lane_addr + 32 * c, x);
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(x[e]));
+          mx1 = fmaxf(mx1, __uint_as_float(x[e + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(x[e + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(x[e + 3]));
         }
       }
+      const float tile_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      if (!tile_full) tmem_wait_st();  // the masked chunks are re-read below
       // The exponent's reference m follows the running maximum lazily: it moves only when
       // the maximum outgrows it by more than 2^8 in the exp2 domain (weights stay <= 256,
       // well inside bf16 and fp32 range), which saves most rescales of O.  O / l does not
@@ -277,8 +289,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           tmem_st32(tmem_o + lane_addr + 32 * c, o);
         }
       }
-      // pass 2: P = exp2(c*S - c*m) on kept entries, exactly 0 elsewhere; bf16 P over S
-      float sum = 0.f;
+      // pass 2: P = exp2(c*S - c*m); pruned entries are -inf by now and give exactly 0; bf16 P over S
+      float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
@@ -291,22 +303,20 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         uint32_t x[32];
         tmem_ld32(tmem_s + lane_addr + 32 * c, x);
         tmem_wait_ld();
-        const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
-          float p1 = ex2_approx(fmaf(__uint_as_float(x[2 * e + 1]), scale_log2, neg_mc));
-          p0 = (w >> (2 * e)) & 1u ? p0 : 0.f;
-          p1 = (w >> (2 * e + 1)) & 1u ? p1 : 0.f;
+          const float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(x[2 * e + 1]), scale_log2, neg_mc));
           __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
           pk[e] = *reinterpret_cast<uint32_t *>(&hh);
           // the row sum is taken over the bf16-rounded weights the MMA will use, so that
           // O / l is an exact convex combination of V rows whatever the rounding of P
-          sum += __uint_as_float(pk[e] << 16) + __uint_as_float(pk[e] & 0xffff0000u);
+          sum0 += __uint_as_float(pk[e] << 16);
+          sum1 += __uint_as_float(pk[e] & 0xffff0000u);
         }
         tmem_st16(tmem_s + lane_addr + 16 * c, pk);
       }
-      l = l * alpha + sum;
+      l = l * alpha + (sum0 + sum1);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(&bars->p_full);
