@@ -1,23 +1,30 @@
 // Masked attention of Section 3.2 for bf16 tensors on the tcgen05 tensor cores.
 //
-// One CTA per (b, h, query tile of 128 rows).  It walks the tile list of its
-// (h, qt) row and, for every stored key tile:
-//   S  = Q_tile K_tile^T            tcgen05.mma, both operands in shared memory
-//                                   (TMA, 128-byte swizzle), fp32 accumulator in TMEM
-//   P  = exp2(c*S - c*m) on kept    one thread per query row reads its S row from
-//        entries, 0 on pruned ones  TMEM, applies the tile's bitmap row exactly,
-//                                   keeps the running row maximum m and sum l
-//                                   (online softmax), rescales O when m moved,
-//                                   and writes P as bf16 over S in TMEM
-//   O += P V_tile                   tcgen05.mma with A = P from TMEM and
-//                                   B = V (MN-major) from shared memory
-// and finally writes O / l (zeros for rows that never saw a kept entry).
+// One CTA per (b, h, query tile of 128 rows).  The CTA walks the tile list of its
+// (h, qt) row.  Each stored tile's bitmap is cut into eight groups of 16 key
+// columns, and only the groups in which some row keeps an entry are looked at:
+// the producer packs up to eight such groups, taken in list order from one or
+// several key tiles, into one PACKED tile of 16..128 key columns.  It stages
+// their K and V rows in shared memory with TMA boxes of 16 rows (128-byte
+// swizzle) and assembles the matching bitmap rows.  Everything downstream is a
+// dense tile of reduced width:
+//   S  = Q K_packed^T        tcgen05.mma, N = 16 * groups, fp32 accumulator in TMEM
+//   P  = exp2(c*S - c*m)     one thread per query row reads its S row from TMEM,
+//                            replaces pruned entries by -inf (the packed bitmap row
+//                            decides, exactly), keeps the running reference m and
+//                            sum l of an online softmax, rescales O when m moved,
+//                            and writes P as bf16 over S in TMEM
+//   O += P V_packed          tcgen05.mma, A = P from TMEM, B = V (MN-major), one K
+//                            step of 16 keys per group
+// and finally O / l is written (zeros for rows that never saw a kept entry).  A
+// skipped group holds no kept entry, so leaving it out is exact.
 //
 // Warp roles (192 threads): warps 0-3 softmax + epilogue (thread = query row),
-// warp 4 TMA producer, warp 5 MMA issuer and TMEM owner.  TMEM: columns
-// [0,128) S / P, [128,128+D) O; 256 columns per CTA so two CTAs share an SM and
-// one CTA's softmax overlaps the other's MMAs.  Every mbarrier wait is bounded;
-// a wait that expires raises the device status word and the CTA winds down.
+// warp 4 producer (all lanes scan and pack bitmaps, lane 0 issues TMA), warp 5
+// MMA issuer and TMEM owner.  TMEM: columns [0,128) S / P, [128,128+D) O; 256
+// columns per CTA so two CTAs share an SM and one CTA's softmax overlaps the
+// other's MMAs.  Every mbarrier wait is bounded; a wait that expires raises the
+// device status word and the CTA winds down.
 #include <math_constants.h>
 
 #include "ap_common.cuh"
@@ -31,8 +38,11 @@ using namespace sm100;
 
 constexpr int kThreads = 192;
 constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-tile
+constexpr int kGroupBytes = 16 * 128; // 16 rows of one sub-tile
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kMaxPolls = 1u << 22;
+constexpr int kPlanRing = 4;          // packed bitmaps / tile infos in flight (>= K stages + 2)
+constexpr int kMinTilesToPack = 6;    // shorter lists are processed tile by tile
 
 template <int D>
 struct Cfg {
@@ -40,14 +50,22 @@ struct Cfg {
   static constexpr int kTileBytes = kSub * kSubBytes;
   static constexpr int kStages = D == 64 ? 2 : 1;     // K and V ring depth
   static constexpr int kBarOffset = (1 + 2 * kStages) * kTileBytes;
-  static constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // + barriers + alignment slack
+  static constexpr int kSmemBytes = kBarOffset + 9 * 1024 + 1024;  // + barriers/plans + alignment slack
 };
 
-struct Barriers {
+struct Shared {
   uint64_t q_full, s_full, p_full, o_done;
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t plan_full[kPlanRing];     // producer -> MMA thread and softmax: info + packed bitmap written
+  uint64_t mode_ready;               // producer -> everyone: `packing` is valid
   uint32_t tmem_base;
   int abort_flag;
+  // per packed tile: bits 0..3 number of groups (1..8), bit 8 last packed tile of the item,
+  // bit 9 every entry of the packed tile is kept
+  uint32_t info[kPlanRing];
+  uint32_t packing;                  // 1: the item's groups are packed, 0: tile by tile
+  uint32_t pad[3];
+  uint32_t bitmap[kPlanRing][128][4];  // packed bitmap rows: slot s of row r = bits [16s, 16s+16)
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -69,10 +87,27 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
   return false;
 }
 
-template <int D>
+// Whole-warp vote on how an item is processed: packing pays when the list is long and most of
+// its tiles are partially filled; lists of mostly fully kept tiles go tile by tile.  The
+// producer warp decides and publishes the mode to the other warps.
+__device__ __forceinline__ bool decide_packing(const uint8_t *__restrict__ flags, int t_begin, int n_tiles,
+                                               int lane) {
+  if (n_tiles < kMinTilesToPack) return false;
+  int n_full = 0;
+  for (int base = 0; base < n_tiles; base += 32) {
+    const int t = base + lane;
+    const bool f = t < n_tiles && (flags[t_begin + t] & 1);
+    n_full += __popc(__ballot_sync(0xffffffffu, f));
+  }
+  return 2 * n_full < n_tiles;
+}
+
+// kCanPack = false compiles the tile-by-tile path only (no list of the launch is long enough to pack).
+template <int D, bool kCanPack>
 __global__ void __launch_bounds__(kThreads, 2)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, __nv_bfloat16 *__restrict__ O,
+              const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_k16,
+              const __grid_constant__ CUtensorMap map_v16, __nv_bfloat16 *__restrict__ O,
               const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
               const uint8_t *__restrict__ flags, const uint32_t *__restrict__ bitmap, int B, int H, int Lq,
               int n_qt, float scale_log2, unsigned *err) {
@@ -83,7 +118,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   unsigned char *q_s = smem;
   unsigned char *k_s = smem + C::kTileBytes;
   unsigned char *v_s = smem + (1 + C::kStages) * C::kTileBytes;
-  Barriers *bars = reinterpret_cast<Barriers *>(smem + C::kBarOffset);
+  Shared *sh = reinterpret_cast<Shared *>(smem + C::kBarOffset);
 
   // work item: heavy (late, under a causal mask) query tiles first; b fastest so
   // that neighbouring CTAs share one tile list and its bitmaps in L2
@@ -109,86 +144,256 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   }
 
   if (threadIdx.x == 0) {
-    mbar_init(&bars->q_full, 1);
-    mbar_init(&bars->s_full, 1);
-    mbar_init(&bars->p_full, 128);
-    mbar_init(&bars->o_done, 1);
+    mbar_init(&sh->q_full, 1);
+    mbar_init(&sh->s_full, 1);
+    mbar_init(&sh->p_full, 128);
+    mbar_init(&sh->o_done, 1);
     for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(&bars->k_full[s], 1);
-      mbar_init(&bars->k_empty[s], 1);
-      mbar_init(&bars->v_full[s], 1);
-      mbar_init(&bars->v_empty[s], 1);
+      mbar_init(&sh->k_full[s], 1);
+      mbar_init(&sh->k_empty[s], 1);
+      mbar_init(&sh->v_full[s], 1);
+      mbar_init(&sh->v_empty[s], 1);
     }
-    bars->abort_flag = 0;
+    for (int s = 0; s < kPlanRing; ++s) mbar_init(&sh->plan_full[s], 1);
+    mbar_init(&sh->mode_ready, 1);
+    sh->abort_flag = 0;
     fence_mbar_init();
   }
   if (warp == 5) {
-    tmem_alloc(&bars->tmem_base, kTmemCols);
+    tmem_alloc(&sh->tmem_base, kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem = bars->tmem_base;
+  const uint32_t tmem = sh->tmem_base;
   const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
-  volatile int *abort_flag = &bars->abort_flag;
+  volatile int *abort_flag = &sh->abort_flag;
 
   if (warp == 4) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ producer
     if (lane == 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      mbar_arrive_expect_tx(&bars->q_full, C::kTileBytes);
+      prefetch_tensormap(&map_k16);
+      prefetch_tensormap(&map_v16);
+      mbar_arrive_expect_tx(&sh->q_full, C::kTileBytes);
 #pragma unroll
-      for (int s = 0; s < C::kSub; ++s) tma_load_3d(q_s + s * kSubBytes, &map_q, &bars->q_full, 64 * s, qt * kTile, bh);
-      int it = 0;
-      bool ok = true;
-      for (; it < n_tiles && ok; ++it) {
-        const int st = it % C::kStages;
-        const uint32_t ph = (uint32_t)(it / C::kStages) & 1u;
-        const int kt = col_idx[t_begin + it];
-        ok = wait_or_abort(&bars->k_empty[st], ph ^ 1u, abort_flag, err);
-        if (!ok) break;
-        mbar_arrive_expect_tx(&bars->k_full[st], C::kTileBytes);
+      for (int s = 0; s < C::kSub; ++s) tma_load_3d(q_s + s * kSubBytes, &map_q, &sh->q_full, 64 * s, qt * kTile, bh);
+    }
+    // Scan state.  Lane L holds bitmap rows 4L..4L+3 of the tile being scanned (a0..a3) and
+    // of the next one (r0..r3, loaded one tile ahead and first touched an iteration later).
+    uint4 r0, r1, r2, r3;
+    int next_kt = 0, next2_kt = 0;          // key tile of the next / next-but-one list tile
+    bool next_full = false, next2_full = false;  // ... and whether it is flagged fully kept
+    auto prefetch_rows = [&](int t) {       // bitmap rows of a tile that is not fully kept
+      const uint4 *src = reinterpret_cast<const uint4 *>(bitmap + (size_t)t * kBitmapWords) + 4 * lane;
+      r0 = src[0]; r1 = src[1]; r2 = src[2]; r3 = src[3];
+    };
+    // packed tile under construction
+    uint32_t v = 0;                 // packed tiles emitted so far
+    int ns = 0;                     // slots filled
+    int slot_row[8];                // first key row of each slot
+    uint32_t pr[4][4];              // packed bitmap rows 4L..4L+3
 #pragma unroll
-        for (int s = 0; s < C::kSub; ++s)
-          tma_load_3d(k_s + st * C::kTileBytes + s * kSubBytes, &map_k, &bars->k_full[st], 64 * s, kt * kTile, bh);
-        ok = wait_or_abort(&bars->v_empty[st], ph ^ 1u, abort_flag, err);
-        if (!ok) {
-          // the K copy just armed is still in flight: let it land before leaving
-          mbar_wait(&bars->k_full[st], ph, kMaxPolls);
-          break;
+    for (int i = 0; i < 4; ++i) pr[i][0] = pr[i][1] = pr[i][2] = pr[i][3] = 0u;
+    bool all_full = true;           // every contributing tile is flagged FULL
+    bool whole = true;              // slots 0..7 are groups 0..7 of one tile
+    int first_kt = 0;
+    bool ok = true;
+    uint32_t armed_k = 0, armed_v = 0;
+
+    // Publishes the packed tile's bitmap rows and info (their ring slot is free by construction,
+    // see kPlanRing) for the MMA thread and the softmax warps.
+    auto publish = [&](bool last) {
+      const uint32_t slot = v % kPlanRing;
+      uint4 *dst = reinterpret_cast<uint4 *>(&sh->bitmap[slot][4 * lane][0]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pr[i][0], pr[i][1], pr[i][2], pr[i][3]);
+      const bool one_tile = whole && ns == 8;
+      if (lane == 0)
+        sh->info[slot] = (uint32_t)ns | (last ? 0x100u : 0u) | ((all_full && one_tile) ? 0x200u : 0u);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->plan_full[slot]);
+    };
+    // Issues the K and V copies of the packed tile as soon as their stage is free (lane 0).
+    auto issue_loads = [&]() {
+      const int st = v % C::kStages;
+      const uint32_t ph = (v / C::kStages) & 1u;
+      const bool one_tile = whole && ns == 8;
+      if (lane == 0) {
+        const uint32_t bytes = (uint32_t)ns * 16u * D * 2u;
+        ok = wait_or_abort(&sh->k_empty[st], ph ^ 1u, abort_flag, err);
+        if (ok) {
+          mbar_arrive_expect_tx(&sh->k_full[st], bytes);
+          unsigned char *kd = k_s + st * C::kTileBytes;
+          if (one_tile) {
+#pragma unroll
+            for (int s = 0; s < C::kSub; ++s) tma_load_3d(kd + s * kSubBytes, &map_k, &sh->k_full[st], 64 * s, first_kt * kTile, bh);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              if (q >= ns) continue;
+#pragma unroll
+              for (int s = 0; s < C::kSub; ++s)
+                tma_load_3d(kd + s * kSubBytes + q * kGroupBytes, &map_k16, &sh->k_full[st], 64 * s, slot_row[q], bh);
+            }
+          }
+          armed_k = v + 1;
+          ok = wait_or_abort(&sh->v_empty[st], ph ^ 1u, abort_flag, err);
         }
-        mbar_arrive_expect_tx(&bars->v_full[st], C::kTileBytes);
+        if (ok) {
+          mbar_arrive_expect_tx(&sh->v_full[st], bytes);
+          unsigned char *vd = v_s + st * C::kTileBytes;
+          if (one_tile) {
 #pragma unroll
-        for (int s = 0; s < C::kSub; ++s)
-          tma_load_3d(v_s + st * C::kTileBytes + s * kSubBytes, &map_v, &bars->v_full[st], 64 * s, kt * kTile, bh);
-      }
-      if (*abort_flag) {
-        // winding down: wait (bounded) for every copy this thread armed and nobody consumed
-        mbar_wait(&bars->q_full, 0, kMaxPolls);
-        for (int j = max(0, it - C::kStages); j < it; ++j) {
-          const int st = j % C::kStages;
-          const uint32_t ph = (uint32_t)(j / C::kStages) & 1u;
-          mbar_wait(&bars->k_full[st], ph, kMaxPolls);
-          mbar_wait(&bars->v_full[st], ph, kMaxPolls);
+            for (int s = 0; s < C::kSub; ++s) tma_load_3d(vd + s * kSubBytes, &map_v, &sh->v_full[st], 64 * s, first_kt * kTile, bh);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              if (q >= ns) continue;
+#pragma unroll
+              for (int s = 0; s < C::kSub; ++s)
+                tma_load_3d(vd + s * kSubBytes + q * kGroupBytes, &map_v16, &sh->v_full[st], 64 * s, slot_row[q], bh);
+            }
+          }
+          armed_v = v + 1;
         }
       }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    };
+    auto next_packed_tile = [&]() {
+      ++v;
+      ns = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pr[i][0] = pr[i][1] = pr[i][2] = pr[i][3] = 0u;
+      all_full = true;
+      whole = true;
+    };
+    auto emit = [&](bool last) {  // packed mode: the plan is known before the loads can start
+      publish(last);
+      issue_loads();
+      next_packed_tile();
+    };
+
+    // Short lists are not worth packing: the scan would delay the first loads by a bitmap
+    // round trip.  Their tiles go out whole and the softmax threads read the bitmap rows
+    // themselves.
+    const bool packing = kCanPack && decide_packing(flags, t_begin, n_tiles, lane);
+    if (kCanPack && lane == 0) {
+      sh->packing = packing ? 1u : 0u;
+      mbar_arrive(&sh->mode_ready);
+    }
+    if (!packing) {
+      int kt_next = col_idx[t_begin];
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        first_kt = kt_next;
+        if (j + 1 < n_tiles) kt_next = col_idx[t_begin + j + 1];
+        whole = true;
+        ns = 8;
+        issue_loads();
+        ++v;
+      }
+    } else {
+      // key tile and flag are known two tiles ahead, so that the bitmap rows of a tile are
+      // requested one tile ahead and only when the tile is not flagged fully kept
+      next_kt = col_idx[t_begin];
+      next_full = flags[t_begin] & 1;
+      if (n_tiles > 1) {
+        next2_kt = col_idx[t_begin + 1];
+        next2_full = flags[t_begin + 1] & 1;
+      }
+      if (!next_full) prefetch_rows(t_begin);
+    }
+    for (int j = 0; j < n_tiles && ok && packing; ++j) {
+      // this tile's key tile, flag, rows and group mask; then request the next tile's
+      const int kt = next_kt;
+      const bool tile_full = next_full;
+      const uint4 ones = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+      const uint4 a0 = tile_full ? ones : r0, a1 = tile_full ? ones : r1, a2 = tile_full ? ones : r2,
+                  a3 = tile_full ? ones : r3;
+      uint32_t gm = 0xffu;
+      if (!tile_full) {
+        const uint32_t w0 = __reduce_or_sync(0xffffffffu, a0.x | a1.x | a2.x | a3.x),
+                       w1 = __reduce_or_sync(0xffffffffu, a0.y | a1.y | a2.y | a3.y),
+                       w2 = __reduce_or_sync(0xffffffffu, a0.z | a1.z | a2.z | a3.z),
+                       w3 = __reduce_or_sync(0xffffffffu, a0.w | a1.w | a2.w | a3.w);
+        gm = ((w0 & 0xffffu) ? 1u : 0u) | ((w0 >> 16) ? 2u : 0u) | ((w1 & 0xffffu) ? 4u : 0u) |
+             ((w1 >> 16) ? 8u : 0u) | ((w2 & 0xffffu) ? 16u : 0u) | ((w2 >> 16) ? 32u : 0u) |
+             ((w3 & 0xffffu) ? 64u : 0u) | ((w3 >> 16) ? 128u : 0u);
+      }
+      next_kt = next2_kt;
+      next_full = next2_full;
+      if (j + 1 < n_tiles && !next_full) prefetch_rows(t_begin + j + 1);
+      if (j + 2 < n_tiles) {
+        next2_kt = col_idx[t_begin + j + 2];
+        next2_full = flags[t_begin + j + 2] & 1;
+      }
+      while (gm && ok) {
+        const int g = __ffs((int)gm) - 1;
+        gm &= gm - 1u;
+        // 16-bit fields of group g for this lane's four rows
+        const int wi = g >> 1, sft = 16 * (g & 1);
+        const uint32_t f0 = ((wi == 0 ? a0.x : wi == 1 ? a0.y : wi == 2 ? a0.z : a0.w) >> sft) & 0xffffu;
+        const uint32_t f1 = ((wi == 0 ? a1.x : wi == 1 ? a1.y : wi == 2 ? a1.z : a1.w) >> sft) & 0xffffu;
+        const uint32_t f2 = ((wi == 0 ? a2.x : wi == 1 ? a2.y : wi == 2 ? a2.z : a2.w) >> sft) & 0xffffu;
+        const uint32_t f3 = ((wi == 0 ? a3.x : wi == 1 ? a3.y : wi == 2 ? a3.z : a3.w) >> sft) & 0xffffu;
+        if (ns == 0) first_kt = kt;
+        whole = whole && g == ns && kt == first_kt;
+        all_full = all_full && tile_full;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (q != ns) continue;
+          slot_row[q] = kt * kTile + 16 * g;
+          pr[0][q >> 1] |= f0 << (16 * (q & 1));
+          pr[1][q >> 1] |= f1 << (16 * (q & 1));
+          pr[2][q >> 1] |= f2 << (16 * (q & 1));
+          pr[3][q >> 1] |= f3 << (16 * (q & 1));
+        }
+        ++ns;
+        if (ns == 8) emit(j == n_tiles - 1 && gm == 0u);
+      }
+    }
+    if (ok && ns > 0) emit(true);
+    if (lane == 0 && *abort_flag) {
+      // winding down: wait (bounded) for the copies this thread armed most recently
+      mbar_wait(&sh->q_full, 0, kMaxPolls);
+      for (uint32_t a = armed_k > (uint32_t)C::kStages ? armed_k - C::kStages : 0; a < armed_k; ++a)
+        mbar_wait(&sh->k_full[a % C::kStages], (a / C::kStages) & 1u, kMaxPolls);
+      for (uint32_t a = armed_v > (uint32_t)C::kStages ? armed_v - C::kStages : 0; a < armed_v; ++a)
+        mbar_wait(&sh->v_full[a % C::kStages], (a / C::kStages) & 1u, kMaxPolls);
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
-      bool ok = wait_or_abort(&bars->q_full, 0, abort_flag, err);
-      for (int it = 0; it < n_tiles && ok; ++it) {
-        const int st = it % C::kStages;
-        const uint32_t ph = (uint32_t)(it / C::kStages) & 1u;
-        ok = wait_or_abort(&bars->k_full[st], ph, abort_flag, err);
+      bool ok = wait_or_abort(&sh->q_full, 0, abort_flag, err);
+      bool packing = false;
+      if (kCanPack && ok) {
+        ok = wait_or_abort(&sh->mode_ready, 0, abort_flag, err);
+        packing = sh->packing != 0u;
+      }
+      for (uint32_t v = 0; ok; ++v) {
+        const int st = v % C::kStages;
+        const uint32_t ph = (v / C::kStages) & 1u;
+        const uint32_t slot = v % kPlanRing;
+        // short lists go tile by tile: whole tiles, as many packed tiles as list tiles
+        int ng = 8;
+        bool last = (int)v == n_tiles - 1;
+        if (packing) {
+          ok = wait_or_abort(&sh->plan_full[slot], (v / kPlanRing) & 1u, abort_flag, err);
+          if (!ok) break;
+          const uint32_t info = sh->info[slot];
+          ng = (int)(info & 15u);
+          last = (info & 0x100u) != 0u;
+        }
+        ok = wait_or_abort(&sh->k_full[st], ph, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
-        // S = Q K^T: D/16 steps of K = 16 (32 bytes inside the 128-byte swizzled rows)
+        // S = Q K_packed^T over the ng packed groups: N = 16 ng, D/16 steps of K = 16
+        // (32 bytes inside the 128-byte swizzled rows)
+        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const int sub = ks / 4, off = (ks % 4) * 32;
@@ -196,21 +401,26 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           const uint64_t db = smem_desc_sw128(smem_u32(k_s + st * C::kTileBytes + sub * kSubBytes + off), 16, 1024);
           mma_ss(tmem_s, da, db, idesc_qk, ks > 0);
         }
-        mma_commit(&bars->k_empty[st]);
-        mma_commit(&bars->s_full);
-        ok = wait_or_abort(&bars->p_full, (uint32_t)it & 1u, abort_flag, err);
+        mma_commit(&sh->k_empty[st]);
+        mma_commit(&sh->s_full);
+        ok = wait_or_abort(&sh->p_full, v & 1u, abort_flag, err);
         if (!ok) break;
-        ok = wait_or_abort(&bars->v_full[st], ph, abort_flag, err);
+        ok = wait_or_abort(&sh->v_full[st], ph, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
-        // O += P V: 8 steps of 16 keys; P (bf16) sits in the first 64 columns of S
+        // O += P V_packed: one K step of 16 keys per group; P (bf16) of group g sits in columns
+        // [8g, 8g+8) of S.  The first step of the item overwrites O.
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t db = smem_desc_sw128(smem_u32(v_s + st * C::kTileBytes + ks * 2048), kSubBytes, 1024);
-          mma_ts(tmem_o, tmem_s + 8 * ks, db, idesc_pv, (it > 0 || ks > 0) ? 1u : 0u);
+          if (ks >= ng) continue;
+          const uint64_t db = smem_desc_sw128(smem_u32(v_s + st * C::kTileBytes + ks * kGroupBytes), kSubBytes, 1024);
+          mma_ts(tmem_o, tmem_s + 8 * ks, db, idesc_pv, (v > 0 || ks > 0) ? 1u : 0u);
         }
-        mma_commit(&bars->v_empty[st]);
-        if (it == n_tiles - 1) mma_commit(&bars->o_done);
+        mma_commit(&sh->v_empty[st]);
+        if (last) {
+          mma_commit(&sh->o_done);
+          break;
+        }
       }
     }
   } else {
@@ -221,30 +431,52 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     float m = -CUDART_INF_F, l = 0.f;       // exponent reference and running sum of weights
     const float ref_slack = 8.f / scale_log2;
     bool ok = true;
-    uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)t_begin * kBitmapWords + r * 4);
-    bool full = flags[t_begin] & 1;
-    for (int it = 0; it < n_tiles; ++it) {
-      const uint4 cur = bw;
-      const bool tile_full = full;
-      if (it + 1 < n_tiles) {  // next tile's bitmap row while this one computes
-        bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)(t_begin + it + 1) * kBitmapWords + r * 4);
-        full = flags[t_begin + it + 1] & 1;
+    bool packing = false;
+    if (kCanPack) {
+      ok = wait_or_abort(&sh->mode_ready, 0, abort_flag, err);
+      packing = ok && sh->packing != 0u;
+    }
+    // tile-by-tile mode: this thread's bitmap row and the flag of the next tile, one tile ahead
+    uint4 bw = make_uint4(0u, 0u, 0u, 0u);
+    bool full = false;
+    if (!packing) {
+      bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)t_begin * kBitmapWords + r * 4);
+      full = flags[t_begin] & 1;
+    }
+    for (uint32_t v = 0;; ++v) {
+      int n_chunks = 4;            // 32-column chunks the (packed) tile spans
+      bool last = (int)v == n_tiles - 1;
+      bool tile_full = full;
+      uint4 cur = bw;
+      if (packing) {
+        const uint32_t slot = v % kPlanRing;
+        ok = wait_or_abort(&sh->plan_full[slot], (v / kPlanRing) & 1u, abort_flag, err);
+        if (!ok) break;
+        const uint32_t info = sh->info[slot];
+        n_chunks = ((int)(info & 15u) + 1) >> 1;
+        last = (info & 0x100u) != 0u;
+        tile_full = (info & 0x200u) != 0u;
+        cur = *reinterpret_cast<const uint4 *>(&sh->bitmap[slot][r][0]);
+      } else if (!last) {  // next tile's bitmap row while this one computes
+        bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)(t_begin + v + 1) * kBitmapWords + r * 4);
+        full = flags[t_begin + v + 1] & 1;
       }
-      ok = wait_or_abort(&bars->s_full, (uint32_t)it & 1u, abort_flag, err);
-      if (!ok) break;
-      tc_fence_after_sync();
       // 32-column chunks in which none of this warp's 32 rows keeps anything are skipped
       // (their P is written as zeros without reading S)
+      // (the bitmap rows of a tile flagged as fully kept are not published: all ones)
       const uint32_t w0 = tile_full ? 0xffffffffu : cur.x, w1 = tile_full ? 0xffffffffu : cur.y,
                      w2 = tile_full ? 0xffffffffu : cur.z, w3 = tile_full ? 0xffffffffu : cur.w;
       const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u) |
                               (__any_sync(0xffffffffu, w2 != 0u) ? 4u : 0u) | (__any_sync(0xffffffffu, w3 != 0u) ? 8u : 0u);
+      ok = wait_or_abort(&sh->s_full, v & 1u, abort_flag, err);
+      if (!ok) break;
+      tc_fence_after_sync();
       // pass 1: row maximum over kept entries (four independent chains).  In a partially filled
       // tile the pruned entries are replaced by -inf and the chunk is written back to TMEM, so
       // that pass 2 needs no bitmap: exp2 of -inf is exactly 0.
       float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < n_chunks; ++c) {
         if (!((active >> c) & 1u)) continue;
         uint32_t x[32];
         tmem_ld32(tmem_s + lane_addr + 32 * c, x);
@@ -276,9 +508,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       const float alpha = move ? ex2_approx((m - m_safe) * scale_log2) : 1.f;  // 0 when m was -inf
       const float neg_mc = -m_safe * scale_log2;
       m = m_new;
-      // rescale the running output where the reference moved (O of step it-1 is complete:
-      // the MMA thread committed s_full after it)
-      if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+      // rescale the running output where the reference moved (O of the previous packed tile is
+      // complete: the MMA thread committed s_full after it)
+      if (v > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
@@ -292,7 +524,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       // pass 2: P = exp2(c*S - c*m); pruned entries are -inf by now and give exactly 0; bf16 P over S
       float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < n_chunks; ++c) {
         uint32_t pk[16];
         if (!((active >> c) & 1u)) {
 #pragma unroll
@@ -319,10 +551,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       l = l * alpha + (sum0 + sum1);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(&bars->p_full);
+      mbar_arrive(&sh->p_full);
+      if (last) break;
     }
     // epilogue: O / l, rounded once to bf16
-    if (ok) ok = wait_or_abort(&bars->o_done, 0, abort_flag, err);
+    if (ok) ok = wait_or_abort(&sh->o_done, 0, abort_flag, err);
     if (ok) {
       tc_fence_after_sync();
       const float inv = l > 0.f ? 1.f / l : 0.f;
@@ -355,16 +588,16 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (warp == 5) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int D>
-cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv, void *O, const ap_tiles &t,
-                   int B, int H, int Lq, float scale, unsigned *err, cudaStream_t s) {
-  auto kern = fwd_tc_kernel<D>;
+template <int D, bool kCanPack>
+cudaError_t launch(const CUtensorMap *maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
+                   unsigned *err, cudaStream_t s) {
+  auto kern = fwd_tc_kernel<D, kCanPack>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
   const float scale_log2 = scale * 1.4426950408889634f;
-  kern<<<B * H * t.n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(mq, mk, mv, static_cast<__nv_bfloat16 *>(O), t.row_ptr,
-                                                          t.col_idx, t.flags, t.bitmap, B, H, Lq, t.n_qt,
-                                                          scale_log2, err);
+  kern<<<B * H * t.n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4],
+                                                          static_cast<__nv_bfloat16 *>(O), t.row_ptr, t.col_idx,
+                                                          t.flags, t.bitmap, B, H, Lq, t.n_qt, scale_log2, err);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -373,14 +606,21 @@ cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorM
 
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O, int B, int H,
                           int Lq, int Lk, int d, float scale, cudaStream_t s) {
+  static_assert(sizeof(Shared) <= 9 * 1024, "shared bookkeeping outgrew its reservation");
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
-  CUtensorMap mq, mk, mv;
-  if (!make_tile_map_bf16(&mq, Q, B * H, Lq, d) || !make_tile_map_bf16(&mk, K, B * H, Lk, d) ||
-      !make_tile_map_bf16(&mv, V, B * H, Lk, d))
+  // whole-tile boxes for Q, K, V and 16-row boxes (one group of key columns) for K and V
+  CUtensorMap maps[5];
+  if (!make_tile_map_bf16(&maps[0], Q, B * H, Lq, d) || !make_tile_map_bf16(&maps[1], K, B * H, Lk, d) ||
+      !make_tile_map_bf16(&maps[2], V, B * H, Lk, d) || !make_tile_map_bf16(&maps[3], K, B * H, Lk, d, 16) ||
+      !make_tile_map_bf16(&maps[4], V, B * H, Lk, d, 16))
     return cudaErrorUnknown;
-  return d == 64 ? launch<64>(mq, mk, mv, O, t, B, H, Lq, scale, err, s)
-                 : launch<128>(mq, mk, mv, O, t, B, H, Lq, scale, err, s);
+  // lists are at most n_kt tiles long: below the packing threshold the smaller kernel does
+  if (t.n_kt < kMinTilesToPack)
+    return d == 64 ? launch<64, false>(maps, O, t, B, H, Lq, scale, err, s)
+                   : launch<128, false>(maps, O, t, B, H, Lq, scale, err, s);
+  return d == 64 ? launch<64, true>(maps, O, t, B, H, Lq, scale, err, s)
+                 : launch<128, true>(maps, O, t, B, H, Lq, scale, err, s);
 }
 
 }  // namespace ap

@@ -26,13 +26,13 @@ EncodeTiledFn encode_fn() {
 
 }  // namespace
 
-// [B*H, L, d] bf16 tensor, boxes of 128 rows x 64 elements, 128-byte swizzle, zero fill outside.
-bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d) {
+// [B*H, L, d] bf16 tensor, boxes of box_rows rows x 64 elements, 128-byte swizzle, zero fill outside.
+bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d, int box_rows) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)L, (cuuint64_t)BH};
   cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)L * d * 2};
-  cuuint32_t box[3] = {64, 128, 1};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
   cuuint32_t elem_strides[3] = {1, 1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, elem_strides,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
