@@ -37,7 +37,7 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-from paper_2012_02030_b200 import inputs, metrics  # noqa: E402
+from paper_2012_02030_b200 import inputs, metrics, replicas  # noqa: E402
 
 METRIC = "sparse-attention fwd effective TFLOP/s (4*d*nnz)"
 UNIT = "TFLOP/s"
@@ -127,8 +127,7 @@ def oracle_sample_step(w, units, calib_seqs=1):
 
 def run_reference(args, w):
     """The oracle as it stands, on the host cores, on a bounded sample per step."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if replicas.rank_info().rank != 0:  # rank 0 alone runs the CPU arm
         return
     units = min(w.H, 8)
     for _ in range(args.warmup):
@@ -167,15 +166,11 @@ def workload_config(w):
 def run_gpu(args, w):
     from paper_2012_02030_b200 import binding as ap
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    info = replicas.rank_info()
+    rank, local_rank, world = info.rank, info.local_rank, info.world
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init(info, "nccl", dev)
     peaks = load_peaks()
     elem = 4 if w.dtype == "f32" else 2
 
@@ -235,11 +230,7 @@ def run_gpu(args, w):
         raise RuntimeError("device status not OK after warm-up")
 
     def barrier():
-        if world > 1:
-            import torch.distributed as dist
-
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(info, dev)
 
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     launches0 = ap.ap_launch_count()
@@ -259,14 +250,7 @@ def run_gpu(args, w):
     total_ms = start.elapsed_time(end)
     stage_ms = {s: float(np.mean([events[i][j].elapsed_time(events[i][j + 1]) for i in range(args.steps)]))
                 for j, s in enumerate(stages)}
-    if world > 1:
-        import torch.distributed as dist
-
-        tt = torch.tensor([total_ms, stage_ms["sparse_fwd"]], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, fwd_ms_max = float(tt[0]), float(tt[1])
-    else:
-        fwd_ms_max = stage_ms["sparse_fwd"]
+    total_ms, fwd_ms_max = replicas.max_over_ranks(info, [total_ms, stage_ms["sparse_fwd"]], dev)
 
     # ---- counts -----------------------------------------------------------------------------
     nnz_total = int(nnz.sum().item())
@@ -275,7 +259,7 @@ def run_gpu(args, w):
     T_sparse = float(t_log[: args.steps].float().mean().item())
     T_dense = dense.n_tiles()
     eff_flops = metrics.effective_flops(nnz_total, w.B, w.d)
-    value = world * eff_flops / (fwd_ms_max * 1e-3) / 1e12
+    value = replicas.job_throughput(info, eff_flops, fwd_ms_max * 1e-3) / 1e12
 
     # ---- end to end through host buffers ---------------------------------------------------------
     hq, hk, hv = (t.pin_memory() for t in inputs.eval_qkv(w))
@@ -292,12 +276,7 @@ def run_gpu(args, w):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        import torch.distributed as dist
-
-        tt = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt[0])
+    (e2e_ms,) = replicas.max_over_ranks(info, [e2e_ms], dev)
     h2d = 3 * 0 + (hq.numel() + hk.numel() + hv.numel()) * elem
     d2h = ho.numel() * elem
 
@@ -352,7 +331,7 @@ def run_gpu(args, w):
                        l2="inputs exceed L2" if flush is None else "256 MiB flush write between steps",
                        value_scope="sparse forward's device time inside the step; ms_per_step is the whole step"),
         "stage_ms": stage_ms,
-        "tokens_per_s": world * w.B * w.Lq / (fwd_ms_max * 1e-3),
+        "tokens_per_s": replicas.job_throughput(info, w.B * w.Lq, fwd_ms_max * 1e-3),
         "speedup_vs_dense_path": stage_ms["dense_fwd"] / stage_ms["sparse_fwd"],
         "density": {"kept_fraction": nnz_total / float(dom), "tiles_kept": T_sparse, "tiles_domain": T_dense,
                     "tile_fill": nnz_total / (T_sparse * 128.0 * 128.0) if T_sparse else None},
@@ -361,7 +340,7 @@ def run_gpu(args, w):
                                  "tile_flops_sustained": 100 * tile_fl / fwd_s / 1e12 / peaks["bf16_sustained"]},
         "pct_of_hbm_roofline": 100 * comp_bytes / fwd_s / 1e9 / peaks["hbm_gbs"],
         "roofline": roof, "roofline_by_stage": by_stage, "cpu_baseline": cpu,
-        "e2e": {"value": world * eff_flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches), "clocks": clocks,
     }
@@ -387,10 +366,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     run_gpu(args, w)
-    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
-        import torch.distributed as dist
-
-        dist.destroy_process_group()
+    replicas.shutdown(replicas.rank_info())
 
 
 if __name__ == "__main__":
