@@ -63,7 +63,13 @@ typedef enum { AP_F32 = 0, AP_BF16 = 1 } ap_dtype;
  *   flags[cap]           bit 0: every one of the 128*128 entries is kept
  *   bitmap[cap][128][4]  entry (r, c) of a tile is bit (c & 31) of word
  *                        [r][c >> 5], least significant bit first; bits of
- *                        rows >= Lq or columns >= Lk are 0
+ *                        rows >= Lq or columns >= Lk are 0 (also written, all
+ *                        ones, for tiles flagged as fully kept)
+ *   groups[cap]          summary of the bitmap: bit g is set iff some row keeps
+ *                        an entry among key columns [16g, 16g+16) of the tile.
+ *                        The forward pass plans from it which 16-column groups
+ *                        to visit, so it must agree with the bitmap; every
+ *                        builder of this library writes it.
  *
  * cap is the capacity in tiles; ap_tiles_capacity() always suffices.
  */
@@ -75,6 +81,7 @@ typedef struct ap_tiles {
   int32_t *col_idx;
   uint8_t *flags;
   uint32_t *bitmap;
+  uint8_t *groups;
 } ap_tiles;
 
 /* Library version (major*10000 + minor*100 + patch). */

@@ -32,7 +32,7 @@ class ap_tiles(ctypes.Structure):
         ("H", ctypes.c_int32), ("Lq", ctypes.c_int32), ("Lk", ctypes.c_int32),
         ("n_qt", ctypes.c_int32), ("n_kt", ctypes.c_int32), ("cap", ctypes.c_int32),
         ("row_ptr", ctypes.c_void_p), ("col_idx", ctypes.c_void_p),
-        ("flags", ctypes.c_void_p), ("bitmap", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p), ("bitmap", ctypes.c_void_p), ("groups", ctypes.c_void_p),
     ]
 
 
@@ -141,8 +141,10 @@ class Tiles:
         self.col_idx = torch.zeros(max(self.cap, 1), dtype=torch.int32, device=device)
         self.flags = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
         self.bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
+        self.groups = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
         self.c = ap_tiles(H, Lq, Lk, self.n_qt, self.n_kt, self.cap, self.row_ptr.data_ptr(),
-                          self.col_idx.data_ptr(), self.flags.data_ptr(), self.bitmap.data_ptr())
+                          self.col_idx.data_ptr(), self.flags.data_ptr(), self.bitmap.data_ptr(),
+                          self.groups.data_ptr())
 
     def n_tiles(self) -> int:
         """Number of stored tiles (synchronises)."""
@@ -152,7 +154,7 @@ class Tiles:
         """dict of numpy arrays trimmed to the stored tiles (synchronises)."""
         T = self.n_tiles()
         return dict(row_ptr=self.row_ptr.cpu().numpy(), col_idx=self.col_idx[:T].cpu().numpy(),
-                    flags=self.flags[:T].cpu().numpy(),
+                    flags=self.flags[:T].cpu().numpy(), groups=self.groups[:T].cpu().numpy(),
                     bitmap=self.bitmap[:T].cpu().numpy().view("uint32"), n_qt=self.n_qt, n_kt=self.n_kt)
 
 

@@ -29,7 +29,7 @@ bool shape_ok(int H, int Lq, int Lk) {
 
 ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shape_must_match) {
   if (!t) return AP_ERR_INVALID_ARG;
-  if (!t->row_ptr || !t->col_idx || !t->flags || !t->bitmap) return AP_ERR_INVALID_ARG;
+  if (!t->row_ptr || !t->col_idx || !t->flags || !t->bitmap || !t->groups) return AP_ERR_INVALID_ARG;
   if (!aligned16(t->bitmap) || (reinterpret_cast<uintptr_t>(t->row_ptr) & 3u) ||
       (reinterpret_cast<uintptr_t>(t->col_idx) & 3u))
     return AP_ERR_INVALID_ARG;

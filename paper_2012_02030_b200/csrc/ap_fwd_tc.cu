@@ -41,8 +41,9 @@ constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-ti
 constexpr int kGroupBytes = 16 * 128; // 16 rows of one sub-tile
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kMaxPolls = 1u << 22;
-constexpr int kPlanRing = 4;          // packed bitmaps / tile infos in flight (>= K stages + 2)
-constexpr int kMinTilesToPack = 6;    // shorter lists are processed tile by tile
+constexpr int kMaxPlanTiles = 128;    // longest list whose groups are packed (longer ones go tile by tile)
+constexpr int kMaxSlots = 8 * kMaxPlanTiles;
+constexpr int kMinTilesToPack = 3;    // shorter lists are processed tile by tile
 
 template <int D>
 struct Cfg {
@@ -50,22 +51,23 @@ struct Cfg {
   static constexpr int kTileBytes = kSub * kSubBytes;
   static constexpr int kStages = D == 64 ? 2 : 1;     // K and V ring depth
   static constexpr int kBarOffset = (1 + 2 * kStages) * kTileBytes;
-  static constexpr int kSmemBytes = kBarOffset + 9 * 1024 + 1024;  // + barriers/plans + alignment slack
+  static constexpr int kSmemBytes = kBarOffset + 7 * 1024 + 1024;  // + barriers/plan + alignment slack
 };
 
+// The plan of a packed item: slot s (s = 0, 1, ... in list order) is one non-empty group of 16 key
+// columns; packed tile v consists of slots [8v, 8v + 8).
 struct Shared {
   uint64_t q_full, s_full, p_full, o_done;
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-  uint64_t plan_full[kPlanRing];     // producer -> MMA thread and softmax: info + packed bitmap written
-  uint64_t mode_ready;               // producer -> everyone: `packing` is valid
+  uint64_t mode_ready;               // producer -> everyone: `packing`, `n_slots` and the plan are valid
   uint32_t tmem_base;
   int abort_flag;
-  // per packed tile: bits 0..3 number of groups (1..8), bit 8 last packed tile of the item,
-  // bit 9 every entry of the packed tile is kept
-  uint32_t info[kPlanRing];
   uint32_t packing;                  // 1: the item's groups are packed, 0: tile by tile
-  uint32_t pad[3];
-  uint32_t bitmap[kPlanRing][128][4];  // packed bitmap rows: slot s of row r = bits [16s, 16s+16)
+  uint32_t n_slots;
+  uint8_t partial[kMaxPlanTiles];    // packed tile v holds a slot of a tile that is not fully kept
+  alignas(16) uint16_t plan_tg[kMaxSlots];  // bit 15: tile flagged fully kept; bits 3..14: list index
+                                            // relative to the item's first tile; bits 0..2: group
+  alignas(16) int32_t plan_row[kMaxSlots];  // first key row of the slot
 };
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -87,21 +89,6 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
   return false;
 }
 
-// Whole-warp vote on how an item is processed: packing pays when the list is long and most of
-// its tiles are partially filled; lists of mostly fully kept tiles go tile by tile.  The
-// producer warp decides and publishes the mode to the other warps.
-__device__ __forceinline__ bool decide_packing(const uint8_t *__restrict__ flags, int t_begin, int n_tiles,
-                                               int lane) {
-  if (n_tiles < kMinTilesToPack) return false;
-  int n_full = 0;
-  for (int base = 0; base < n_tiles; base += 32) {
-    const int t = base + lane;
-    const bool f = t < n_tiles && (flags[t_begin + t] & 1);
-    n_full += __popc(__ballot_sync(0xffffffffu, f));
-  }
-  return 2 * n_full < n_tiles;
-}
-
 // kCanPack = false compiles the tile-by-tile path only (no list of the launch is long enough to pack).
 template <int D, bool kCanPack>
 __global__ void __launch_bounds__(kThreads, 2)
@@ -109,8 +96,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
               const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_k16,
               const __grid_constant__ CUtensorMap map_v16, __nv_bfloat16 *__restrict__ O,
               const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
-              const uint8_t *__restrict__ flags, const uint32_t *__restrict__ bitmap, int B, int H, int Lq,
-              int n_qt, float scale_log2, unsigned *err) {
+              const uint8_t *__restrict__ flags, const uint32_t *__restrict__ bitmap,
+              const uint8_t *__restrict__ groups, int B, int H, int Lq, int n_qt, float scale_log2,
+              unsigned *err) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -154,7 +142,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       mbar_init(&sh->v_full[s], 1);
       mbar_init(&sh->v_empty[s], 1);
     }
-    for (int s = 0; s < kPlanRing; ++s) mbar_init(&sh->plan_full[s], 1);
     mbar_init(&sh->mode_ready, 1);
     sh->abort_flag = 0;
     fence_mbar_init();
@@ -176,188 +163,140 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      prefetch_tensormap(&map_k16);
-      prefetch_tensormap(&map_v16);
       mbar_arrive_expect_tx(&sh->q_full, C::kTileBytes);
 #pragma unroll
       for (int s = 0; s < C::kSub; ++s) tma_load_3d(q_s + s * kSubBytes, &map_q, &sh->q_full, 64 * s, qt * kTile, bh);
     }
-    // Scan state.  Lane L holds bitmap rows 4L..4L+3 of the tile being scanned (a0..a3) and
-    // of the next one (r0..r3, loaded one tile ahead and first touched an iteration later).
-    uint4 r0, r1, r2, r3;
-    int next_kt = 0, next2_kt = 0;          // key tile of the next / next-but-one list tile
-    bool next_full = false, next2_full = false;  // ... and whether it is flagged fully kept
-    auto prefetch_rows = [&](int t) {       // bitmap rows of a tile that is not fully kept
-      const uint4 *src = reinterpret_cast<const uint4 *>(bitmap + (size_t)t * kBitmapWords) + 4 * lane;
-      r0 = src[0]; r1 = src[1]; r2 = src[2]; r3 = src[3];
-    };
-    // packed tile under construction
-    uint32_t v = 0;                 // packed tiles emitted so far
-    int ns = 0;                     // slots filled
-    int slot_row[8];                // first key row of each slot
-    uint32_t pr[4][4];              // packed bitmap rows 4L..4L+3
-#pragma unroll
-    for (int i = 0; i < 4; ++i) pr[i][0] = pr[i][1] = pr[i][2] = pr[i][3] = 0u;
-    bool all_full = true;           // every contributing tile is flagged FULL
-    bool whole = true;              // slots 0..7 are groups 0..7 of one tile
-    int first_kt = 0;
     bool ok = true;
     uint32_t armed_k = 0, armed_v = 0;
 
-    // Publishes the packed tile's bitmap rows and info (their ring slot is free by construction,
-    // see kPlanRing) for the MMA thread and the softmax warps.
-    auto publish = [&](bool last) {
-      const uint32_t slot = v % kPlanRing;
-      uint4 *dst = reinterpret_cast<uint4 *>(&sh->bitmap[slot][4 * lane][0]);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pr[i][0], pr[i][1], pr[i][2], pr[i][3]);
-      const bool one_tile = whole && ns == 8;
-      if (lane == 0)
-        sh->info[slot] = (uint32_t)ns | (last ? 0x100u : 0u) | ((all_full && one_tile) ? 0x200u : 0u);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->plan_full[slot]);
-    };
-    // Issues the K and V copies of the packed tile as soon as their stage is free (lane 0).
-    auto issue_loads = [&]() {
-      const int st = v % C::kStages;
-      const uint32_t ph = (v / C::kStages) & 1u;
-      const bool one_tile = whole && ns == 8;
+    // The plan: every lane takes one list tile per round, reads its group summary, and a prefix
+    // sum over the lanes gives each tile's first slot.  Packing pays when it saves enough
+    // MMA / softmax round trips over going tile by tile.
+    bool packing = false;
+    uint32_t n_slots = 0;
+    if (kCanPack && n_tiles >= kMinTilesToPack && n_tiles <= kMaxPlanTiles) {
       if (lane == 0) {
-        const uint32_t bytes = (uint32_t)ns * 16u * D * 2u;
-        ok = wait_or_abort(&sh->k_empty[st], ph ^ 1u, abort_flag, err);
-        if (ok) {
-          mbar_arrive_expect_tx(&sh->k_full[st], bytes);
-          unsigned char *kd = k_s + st * C::kTileBytes;
-          if (one_tile) {
-#pragma unroll
-            for (int s = 0; s < C::kSub; ++s) tma_load_3d(kd + s * kSubBytes, &map_k, &sh->k_full[st], 64 * s, first_kt * kTile, bh);
-          } else {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              if (q >= ns) continue;
-#pragma unroll
-              for (int s = 0; s < C::kSub; ++s)
-                tma_load_3d(kd + s * kSubBytes + q * kGroupBytes, &map_k16, &sh->k_full[st], 64 * s, slot_row[q], bh);
-            }
-          }
-          armed_k = v + 1;
-          ok = wait_or_abort(&sh->v_empty[st], ph ^ 1u, abort_flag, err);
-        }
-        if (ok) {
-          mbar_arrive_expect_tx(&sh->v_full[st], bytes);
-          unsigned char *vd = v_s + st * C::kTileBytes;
-          if (one_tile) {
-#pragma unroll
-            for (int s = 0; s < C::kSub; ++s) tma_load_3d(vd + s * kSubBytes, &map_v, &sh->v_full[st], 64 * s, first_kt * kTile, bh);
-          } else {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              if (q >= ns) continue;
-#pragma unroll
-              for (int s = 0; s < C::kSub; ++s)
-                tma_load_3d(vd + s * kSubBytes + q * kGroupBytes, &map_v16, &sh->v_full[st], 64 * s, slot_row[q], bh);
-            }
-          }
-          armed_v = v + 1;
-        }
+        prefetch_tensormap(&map_k16);
+        prefetch_tensormap(&map_v16);
       }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-    };
-    auto next_packed_tile = [&]() {
-      ++v;
-      ns = 0;
+      reinterpret_cast<uint32_t *>(sh->partial)[lane] = 0u;
+      static_assert(kMaxPlanTiles == 128, "one 32-bit word of `partial` per lane");
+      __syncwarp();
+      int carry = 0;
+      for (int base = 0; base < n_tiles; base += 32) {
+        const int t = base + lane;
+        uint32_t gm = 0u;
+        int kt = 0;
+        bool full = false;
+        if (t < n_tiles) {
+          full = flags[t_begin + t] & 1;
+          gm = groups[t_begin + t];
+          kt = col_idx[t_begin + t];
+          if (full) gm = 0xffu;
+        }
+        const int cnt = __popc(gm);
+        int incl = cnt;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) pr[i][0] = pr[i][1] = pr[i][2] = pr[i][3] = 0u;
-      all_full = true;
-      whole = true;
-    };
-    auto emit = [&](bool last) {  // packed mode: the plan is known before the loads can start
-      publish(last);
-      issue_loads();
-      next_packed_tile();
-    };
-
-    // Short lists are not worth packing: the scan would delay the first loads by a bitmap
-    // round trip.  Their tiles go out whole and the softmax threads read the bitmap rows
-    // themselves.
-    const bool packing = kCanPack && decide_packing(flags, t_begin, n_tiles, lane);
-    if (kCanPack && lane == 0) {
-      sh->packing = packing ? 1u : 0u;
-      mbar_arrive(&sh->mode_ready);
+        for (int o = 1; o < 32; o <<= 1) {
+          const int up = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += up;
+        }
+        int s = carry + incl - cnt;
+        while (gm) {
+          const int g = __ffs((int)gm) - 1;
+          gm &= gm - 1u;
+          sh->plan_tg[s] = (uint16_t)((full ? 0x8000u : 0u) | ((uint32_t)t << 3) | (uint32_t)g);
+          sh->plan_row[s] = kt * kTile + 16 * g;
+          if (!full) sh->partial[s >> 3] = 1;
+          ++s;
+        }
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      n_slots = (uint32_t)carry;
+      const uint32_t n_packed = (n_slots + 7u) / 8u;
+      packing = n_slots > 0u && 4u * n_packed <= 3u * (uint32_t)n_tiles;
+    }
+    if (kCanPack) {
+      __syncwarp();
+      if (lane == 0) {
+        sh->packing = packing ? 1u : 0u;
+        sh->n_slots = n_slots;
+        mbar_arrive(&sh->mode_ready);
+      }
     }
     if (!packing) {
-      int kt_next = col_idx[t_begin];
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        first_kt = kt_next;
-        if (j + 1 < n_tiles) kt_next = col_idx[t_begin + j + 1];
-        whole = true;
-        ns = 8;
-        issue_loads();
-        ++v;
+      // tile by tile: whole-tile boxes, one lane
+      if (lane == 0) {
+        int kt_next = col_idx[t_begin];
+        for (int j = 0; j < n_tiles && ok; ++j) {
+          const int kt = kt_next;
+          if (j + 1 < n_tiles) kt_next = col_idx[t_begin + j + 1];
+          const int st = j % C::kStages;
+          const uint32_t ph = ((uint32_t)j / C::kStages) & 1u;
+          ok = wait_or_abort(&sh->k_empty[st], ph ^ 1u, abort_flag, err);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&sh->k_full[st], C::kTileBytes);
+#pragma unroll
+          for (int s = 0; s < C::kSub; ++s)
+            tma_load_3d(k_s + st * C::kTileBytes + s * kSubBytes, &map_k, &sh->k_full[st], 64 * s, kt * kTile, bh);
+          armed_k = (uint32_t)j + 1u;
+          ok = wait_or_abort(&sh->v_empty[st], ph ^ 1u, abort_flag, err);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&sh->v_full[st], C::kTileBytes);
+#pragma unroll
+          for (int s = 0; s < C::kSub; ++s)
+            tma_load_3d(v_s + st * C::kTileBytes + s * kSubBytes, &map_v, &sh->v_full[st], 64 * s, kt * kTile, bh);
+          armed_v = (uint32_t)j + 1u;
+        }
       }
     } else {
-      // key tile and flag are known two tiles ahead, so that the bitmap rows of a tile are
-      // requested one tile ahead and only when the tile is not flagged fully kept
-      next_kt = col_idx[t_begin];
-      next_full = flags[t_begin] & 1;
-      if (n_tiles > 1) {
-        next2_kt = col_idx[t_begin + 1];
-        next2_full = flags[t_begin + 1] & 1;
-      }
-      if (!next_full) prefetch_rows(t_begin);
-    }
-    for (int j = 0; j < n_tiles && ok && packing; ++j) {
-      // this tile's key tile, flag, rows and group mask; then request the next tile's
-      const int kt = next_kt;
-      const bool tile_full = next_full;
-      const uint4 ones = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
-      const uint4 a0 = tile_full ? ones : r0, a1 = tile_full ? ones : r1, a2 = tile_full ? ones : r2,
-                  a3 = tile_full ? ones : r3;
-      uint32_t gm = 0xffu;
-      if (!tile_full) {
-        const uint32_t w0 = __reduce_or_sync(0xffffffffu, a0.x | a1.x | a2.x | a3.x),
-                       w1 = __reduce_or_sync(0xffffffffu, a0.y | a1.y | a2.y | a3.y),
-                       w2 = __reduce_or_sync(0xffffffffu, a0.z | a1.z | a2.z | a3.z),
-                       w3 = __reduce_or_sync(0xffffffffu, a0.w | a1.w | a2.w | a3.w);
-        gm = ((w0 & 0xffffu) ? 1u : 0u) | ((w0 >> 16) ? 2u : 0u) | ((w1 & 0xffffu) ? 4u : 0u) |
-             ((w1 >> 16) ? 8u : 0u) | ((w2 & 0xffffu) ? 16u : 0u) | ((w2 >> 16) ? 32u : 0u) |
-             ((w3 & 0xffffu) ? 64u : 0u) | ((w3 >> 16) ? 128u : 0u);
-      }
-      next_kt = next2_kt;
-      next_full = next2_full;
-      if (j + 1 < n_tiles && !next_full) prefetch_rows(t_begin + j + 1);
-      if (j + 2 < n_tiles) {
-        next2_kt = col_idx[t_begin + j + 2];
-        next2_full = flags[t_begin + j + 2] & 1;
-      }
-      while (gm && ok) {
-        const int g = __ffs((int)gm) - 1;
-        gm &= gm - 1u;
-        // 16-bit fields of group g for this lane's four rows
-        const int wi = g >> 1, sft = 16 * (g & 1);
-        const uint32_t f0 = ((wi == 0 ? a0.x : wi == 1 ? a0.y : wi == 2 ? a0.z : a0.w) >> sft) & 0xffffu;
-        const uint32_t f1 = ((wi == 0 ? a1.x : wi == 1 ? a1.y : wi == 2 ? a1.z : a1.w) >> sft) & 0xffffu;
-        const uint32_t f2 = ((wi == 0 ? a2.x : wi == 1 ? a2.y : wi == 2 ? a2.z : a2.w) >> sft) & 0xffffu;
-        const uint32_t f3 = ((wi == 0 ? a3.x : wi == 1 ? a3.y : wi == 2 ? a3.z : a3.w) >> sft) & 0xffffu;
-        if (ns == 0) first_kt = kt;
-        whole = whole && g == ns && kt == first_kt;
-        all_full = all_full && tile_full;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          if (q != ns) continue;
-          slot_row[q] = kt * kTile + 16 * g;
-          pr[0][q >> 1] |= f0 << (16 * (q & 1));
-          pr[1][q >> 1] |= f1 << (16 * (q & 1));
-          pr[2][q >> 1] |= f2 << (16 * (q & 1));
-          pr[3][q >> 1] |= f3 << (16 * (q & 1));
+      // packed: lane q copies the 16 key rows of slot q (K, then V) into the stage
+      const uint32_t n_packed = (n_slots + 7u) / 8u;
+      for (uint32_t v = 0; v < n_packed && ok; ++v) {
+        const int st = v % C::kStages;
+        const uint32_t ph = (v / C::kStages) & 1u;
+        const int ng = min(8, (int)(n_slots - 8u * v));
+        const int row = lane < ng ? sh->plan_row[8u * v + lane] : 0;
+        const int row0 = __shfl_sync(0xffffffffu, row, 0), row_last = __shfl_sync(0xffffffffu, row, ng - 1);
+        // rows ascend by at least 16 from slot to slot: eight slots spanning 112 rows from a tile
+        // boundary are the eight groups of one tile, which goes out as whole-tile boxes
+        const bool one_tile = ng == 8 && (row0 & (kTile - 1)) == 0 && row_last - row0 == kTile - 16;
+        const uint32_t bytes = (uint32_t)ng * 16u * D * 2u;
+        if (lane == 0) {
+          ok = wait_or_abort(&sh->k_empty[st], ph ^ 1u, abort_flag, err);
+          if (ok) mbar_arrive_expect_tx(&sh->k_full[st], bytes);
         }
-        ++ns;
-        if (ns == 8) emit(j == n_tiles - 1 && gm == 0u);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        unsigned char *kd = k_s + st * C::kTileBytes;
+        if (one_tile) {
+          if (lane < C::kSub) tma_load_3d(kd + lane * kSubBytes, &map_k, &sh->k_full[st], 64 * lane, row0, bh);
+        } else if (lane < ng) {
+#pragma unroll
+          for (int s = 0; s < C::kSub; ++s)
+            tma_load_3d(kd + s * kSubBytes + lane * kGroupBytes, &map_k16, &sh->k_full[st], 64 * s, row, bh);
+        }
+        armed_k = v + 1u;
+        if (lane == 0) {
+          ok = wait_or_abort(&sh->v_empty[st], ph ^ 1u, abort_flag, err);
+          if (ok) mbar_arrive_expect_tx(&sh->v_full[st], bytes);
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        unsigned char *vd = v_s + st * C::kTileBytes;
+        if (one_tile) {
+          if (lane < C::kSub) tma_load_3d(vd + lane * kSubBytes, &map_v, &sh->v_full[st], 64 * lane, row0, bh);
+        } else if (lane < ng) {
+#pragma unroll
+          for (int s = 0; s < C::kSub; ++s)
+            tma_load_3d(vd + s * kSubBytes + lane * kGroupBytes, &map_v16, &sh->v_full[st], 64 * s, row, bh);
+        }
+        armed_v = v + 1u;
       }
     }
-    if (ok && ns > 0) emit(true);
     if (lane == 0 && *abort_flag) {
-      // winding down: wait (bounded) for the copies this thread armed most recently
+      // winding down: wait (bounded) for the copies armed most recently
       mbar_wait(&sh->q_full, 0, kMaxPolls);
       for (uint32_t a = armed_k > (uint32_t)C::kStages ? armed_k - C::kStages : 0; a < armed_k; ++a)
         mbar_wait(&sh->k_full[a % C::kStages], (a / C::kStages) & 1u, kMaxPolls);
@@ -370,23 +309,21 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
       bool ok = wait_or_abort(&sh->q_full, 0, abort_flag, err);
       bool packing = false;
+      uint32_t n_slots = 0;
       if (kCanPack && ok) {
         ok = wait_or_abort(&sh->mode_ready, 0, abort_flag, err);
-        packing = sh->packing != 0u;
+        packing = ok && sh->packing != 0u;
+        n_slots = sh->n_slots;
       }
       for (uint32_t v = 0; ok; ++v) {
         const int st = v % C::kStages;
         const uint32_t ph = (v / C::kStages) & 1u;
-        const uint32_t slot = v % kPlanRing;
-        // short lists go tile by tile: whole tiles, as many packed tiles as list tiles
+        // tile by tile: whole tiles, as many rounds as list tiles; packed: eight slots per round
         int ng = 8;
         bool last = (int)v == n_tiles - 1;
         if (packing) {
-          ok = wait_or_abort(&sh->plan_full[slot], (v / kPlanRing) & 1u, abort_flag, err);
-          if (!ok) break;
-          const uint32_t info = sh->info[slot];
-          ng = (int)(info & 15u);
-          last = (info & 0x100u) != 0u;
+          ng = min(8, (int)(n_slots - 8u * v));
+          last = 8u * v + 8u >= n_slots;
         }
         ok = wait_or_abort(&sh->k_full[st], ph, abort_flag, err);
         if (!ok) break;
@@ -432,31 +369,59 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const float ref_slack = 8.f / scale_log2;
     bool ok = true;
     bool packing = false;
+    uint32_t n_slots = 0;
     if (kCanPack) {
       ok = wait_or_abort(&sh->mode_ready, 0, abort_flag, err);
       packing = ok && sh->packing != 0u;
+      n_slots = sh->n_slots;
     }
-    // tile-by-tile mode: this thread's bitmap row and the flag of the next tile, one tile ahead
+    // Bitmap words of the round after the current one, requested one round ahead.
+    // Tile by tile: this thread's row of the next tile (bw) and that tile's flag.
+    // Packed: for each of the eight slots the word of this thread's row that holds the slot's
+    // 16 columns (raw[q]), and the slots' plan entries (tg).
     uint4 bw = make_uint4(0u, 0u, 0u, 0u);
     bool full = false;
+    uint32_t raw[8];
+    uint4 tg = make_uint4(0u, 0u, 0u, 0u);
+    auto fetch_packed = [&](uint32_t v) {
+      tg = *reinterpret_cast<const uint4 *>(&sh->plan_tg[8u * v]);
+      const int ng = min(8, (int)(n_slots - 8u * v));
+      const bool partial = sh->partial[v] != 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const uint32_t pair = q < 2 ? tg.x : q < 4 ? tg.y : q < 6 ? tg.z : tg.w;
+        const uint32_t e = (q & 1) ? pair >> 16 : pair & 0xffffu;
+        raw[q] = q < ng ? 0xffffffffu : 0u;
+        if (partial && q < ng && !(e & 0x8000u))
+          raw[q] = bitmap[(size_t)(t_begin + (int)((e >> 3) & 0xfffu)) * kBitmapWords + r * 4 + ((e & 7u) >> 1)];
+      }
+    };
     if (!packing) {
       bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)t_begin * kBitmapWords + r * 4);
       full = flags[t_begin] & 1;
+    } else if (ok) {
+      fetch_packed(0);
     }
-    for (uint32_t v = 0;; ++v) {
+    for (uint32_t v = 0; ok; ++v) {
       int n_chunks = 4;            // 32-column chunks the (packed) tile spans
       bool last = (int)v == n_tiles - 1;
       bool tile_full = full;
       uint4 cur = bw;
       if (packing) {
-        const uint32_t slot = v % kPlanRing;
-        ok = wait_or_abort(&sh->plan_full[slot], (v / kPlanRing) & 1u, abort_flag, err);
-        if (!ok) break;
-        const uint32_t info = sh->info[slot];
-        n_chunks = ((int)(info & 15u) + 1) >> 1;
-        last = (info & 0x100u) != 0u;
-        tile_full = (info & 0x200u) != 0u;
-        cur = *reinterpret_cast<const uint4 *>(&sh->bitmap[slot][r][0]);
+        const int ng = min(8, (int)(n_slots - 8u * v));
+        n_chunks = (ng + 1) >> 1;
+        last = 8u * v + 8u >= n_slots;
+        tile_full = ng == 8 && sh->partial[v] == 0;
+        // this thread's packed bitmap row: slot q's 16 bits at [16q, 16q + 16)
+        uint32_t f[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const uint32_t pair = q < 2 ? tg.x : q < 4 ? tg.y : q < 6 ? tg.z : tg.w;
+          const uint32_t e = (q & 1) ? pair >> 16 : pair & 0xffffu;
+          f[q] = (raw[q] >> (16u * (e & 1u))) & 0xffffu;
+        }
+        cur = make_uint4(f[0] | (f[1] << 16), f[2] | (f[3] << 16), f[4] | (f[5] << 16), f[6] | (f[7] << 16));
+        if (!last) fetch_packed(v + 1);
       } else if (!last) {  // next tile's bitmap row while this one computes
         bw = *reinterpret_cast<const uint4 *>(bitmap + (size_t)(t_begin + v + 1) * kBitmapWords + r * 4);
         full = flags[t_begin + v + 1] & 1;
@@ -597,7 +562,8 @@ cudaError_t launch(const CUtensorMap *maps, void *O, const ap_tiles &t, int B, i
   const float scale_log2 = scale * 1.4426950408889634f;
   kern<<<B * H * t.n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4],
                                                           static_cast<__nv_bfloat16 *>(O), t.row_ptr, t.col_idx,
-                                                          t.flags, t.bitmap, B, H, Lq, t.n_qt, scale_log2, err);
+                                                          t.flags, t.bitmap, t.groups, B, H, Lq, t.n_qt, scale_log2,
+                                                          err);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -606,7 +572,7 @@ cudaError_t launch(const CUtensorMap *maps, void *O, const ap_tiles &t, int B, i
 
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O, int B, int H,
                           int Lq, int Lk, int d, float scale, cudaStream_t s) {
-  static_assert(sizeof(Shared) <= 9 * 1024, "shared bookkeeping outgrew its reservation");
+  static_assert(sizeof(Shared) <= 7 * 1024, "shared bookkeeping outgrew its reservation");
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   // whole-tile boxes for Q, K, V and 16-row boxes (one group of key columns) for K and V

@@ -98,22 +98,50 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
   if (threadIdx.x == 0 && carry_s > cap) atomicOr(err, kDevErrCapacity);
 }
 
+// Called by all 128 threads of a CTA, thread r holding bitmap row r of one tile: bit g of the
+// result says whether any row keeps an entry among columns [16g, 16g+16).
+__device__ __forceinline__ uint32_t group_mask_of_tile(uint4 row) {
+  __shared__ uint32_t warp_or[4][4];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t w0 = __reduce_or_sync(0xffffffffu, row.x), w1 = __reduce_or_sync(0xffffffffu, row.y),
+                 w2 = __reduce_or_sync(0xffffffffu, row.z), w3 = __reduce_or_sync(0xffffffffu, row.w);
+  if (lane == 0) {
+    warp_or[warp][0] = w0;
+    warp_or[warp][1] = w1;
+    warp_or[warp][2] = w2;
+    warp_or[warp][3] = w3;
+  }
+  __syncthreads();
+  uint32_t gm = 0u;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const uint32_t w = warp_or[0][c] | warp_or[1][c] | warp_or[2][c] | warp_or[3][c];
+    gm |= ((w & 0xffffu) ? 1u : 0u) << (2 * c);
+    gm |= ((w >> 16) ? 1u : 0u) << (2 * c + 1);
+  }
+  return gm;
+}
+
 // One CTA per grid tile: non-empty tiles copy their bitmap to their list slot.
 __global__ void __launch_bounds__(128) gather_tiles_kernel(const uint32_t *__restrict__ stage_bitmap,
                                                            const int32_t *__restrict__ stage_count,
                                                            const int32_t *__restrict__ stage_pos, int n_kt,
                                                            int cap, int32_t *__restrict__ col_idx,
                                                            uint8_t *__restrict__ flags,
-                                                           uint32_t *__restrict__ bitmap) {
+                                                           uint32_t *__restrict__ bitmap,
+                                                           uint8_t *__restrict__ groups) {
   const int tile = blockIdx.x;
   const int pos = stage_pos[tile];
   if (pos < 0 || pos >= cap) return;
   const uint4 *src = reinterpret_cast<const uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords);
   uint4 *dst = reinterpret_cast<uint4 *>(bitmap + (size_t)pos * kBitmapWords);
-  dst[threadIdx.x] = src[threadIdx.x];
+  const uint4 row = src[threadIdx.x];
+  dst[threadIdx.x] = row;
+  const uint32_t gm = group_mask_of_tile(row);
   if (threadIdx.x == 0) {
     col_idx[pos] = tile % n_kt;
     flags[pos] = stage_count[tile] == kTile * kTile ? 1 : 0;
+    groups[pos] = (uint8_t)gm;
   }
 }
 
@@ -123,7 +151,8 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
                                                           int cap, int32_t *__restrict__ row_ptr,
                                                           int32_t *__restrict__ col_idx,
                                                           uint8_t *__restrict__ flags,
-                                                          uint32_t *__restrict__ bitmap, unsigned *err) {
+                                                          uint32_t *__restrict__ bitmap,
+                                                          uint8_t *__restrict__ groups, unsigned *err) {
   const int tile = blockIdx.x;
   const int kt = tile % n_kt;
   const int qt = (tile / n_kt) % n_qt;
@@ -157,9 +186,11 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
   reinterpret_cast<uint4 *>(bitmap + (size_t)pos * kBitmapWords)[r] = make_uint4(w[0], w[1], w[2], w[3]);
   const int full = __syncthreads_and(w[0] == 0xffffffffu && w[1] == 0xffffffffu &&
                                      w[2] == 0xffffffffu && w[3] == 0xffffffffu);
+  const uint32_t gm = group_mask_of_tile(make_uint4(w[0], w[1], w[2], w[3]));
   if (r == 0) {
     col_idx[pos] = kt;
     flags[pos] = full ? 1 : 0;
+    groups[pos] = (uint8_t)gm;
   }
 }
 
@@ -186,7 +217,7 @@ cudaError_t launch_compact_tiles(const uint32_t *stage_bitmap, const int32_t *st
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   gather_tiles_kernel<<<n_tiles, 128, 0, s>>>(stage_bitmap, stage_count, stage_pos, t.n_kt, t.cap,
-                                              t.col_idx, t.flags, t.bitmap);
+                                              t.col_idx, t.flags, t.bitmap, t.groups);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -195,7 +226,7 @@ cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   dense_tiles_kernel<<<t.H * t.n_qt * t.n_kt, 128, 0, s>>>(t.H, t.Lq, t.Lk, t.n_qt, t.n_kt, causal, t.cap,
-                                                         t.row_ptr, t.col_idx, t.flags, t.bitmap, err);
+                                                         t.row_ptr, t.col_idx, t.flags, t.bitmap, t.groups, err);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -23,11 +23,28 @@ def assert_close_attention(got_t: torch.Tensor, ref: np.ndarray, dtype: str, wha
     return max_abs, rel_l2
 
 
+def groups_from_bitmap(bitmap: np.ndarray) -> np.ndarray:
+    """The tile list's group summary restated from its definition: bit g of a tile's byte is set
+    iff some row keeps an entry among the tile's columns [16g, 16g+16).  bitmap: [T,128,4] uint32."""
+    T = bitmap.shape[0]
+    out = np.zeros(T, dtype=np.uint8)
+    if T == 0:
+        return out
+    bits = np.unpackbits(np.ascontiguousarray(bitmap).view(np.uint8).reshape(T, 128, 16), axis=2, bitorder="little")
+    any_col = bits.reshape(T, 128, 128).any(axis=1)          # [T,128]: column holds a kept entry
+    any_group = any_col.reshape(T, 8, 16).any(axis=2)        # [T,8]
+    for g in range(8):
+        out |= (any_group[:, g].astype(np.uint8) << g).astype(np.uint8)
+    return out
+
+
 def assert_tiles_equal(got: dict, want: dict):
     np.testing.assert_array_equal(got["row_ptr"], want["row_ptr"])
     np.testing.assert_array_equal(got["col_idx"], want["col_idx"])
     np.testing.assert_array_equal(got["flags"], want["flags"])
     np.testing.assert_array_equal(got["bitmap"], want["bitmap"])
+    if "groups" in got:  # derived data: checked against its definition applied to the oracle's bitmaps
+        np.testing.assert_array_equal(got["groups"], groups_from_bitmap(want["bitmap"]))
 
 
 def gpu_accumulate(ap, w, n_batches, bias_dev):
