@@ -68,6 +68,7 @@ cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const
 
 // Tensor map of a [B*H, L, d] bf16 tensor for box_rows-row x 64-element swizzled boxes.
 bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d, int box_rows = 128);
+bool make_split_map_bf16_d128(CUtensorMap *m, const void *base, int BH, int L, int box_rows);
 // Tensor map of an [H, Lq, Lk] fp32 tensor for 128-row x 32-column swizzled boxes (Lk % 4 == 0).
 bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk);
 

@@ -45,13 +45,29 @@ constexpr int kMaxPlanTiles = 128;    // longest list whose groups are packed (l
 constexpr int kMaxSlots = 8 * kMaxPlanTiles;
 constexpr int kMinTilesToPack = 3;    // shorter lists are processed tile by tile
 
-template <int D>
+// Shared-memory layout of a K or V stage.  Rows are the (packed) tile's keys, a row's d elements are
+// cut into halves of 64 (128 bytes, the swizzle span).
+//   kSplit = false: [half][row / 8][8 rows][128 B]   one TMA box per half (3-D tensor map)
+//   kSplit = true:  [row / 8][half][8 rows][128 B]   d = 128 only: one box brings both halves (5-D map)
+template <int D, bool kSplit>
 struct Cfg {
-  static constexpr int kSub = D / 64;                 // sub-tiles per operand tile
+  static_assert(!kSplit || D == 128, "the split layout is for d = 128");
+  static constexpr int kSub = D / 64;                 // halves per row
   static constexpr int kTileBytes = kSub * kSubBytes;
   static constexpr int kStages = D == 64 ? 2 : 1;     // K and V ring depth
   static constexpr int kBarOffset = (1 + 2 * kStages) * kTileBytes;
   static constexpr int kSmemBytes = kBarOffset + 7 * 1024 + 1024;  // + barriers/plan + alignment slack
+  static constexpr int kHalfStride = kSplit ? 1024 : kSubBytes;          // half 0 -> half 1 of the same rows
+  static constexpr int kSbo = kSplit ? 2048 : 1024;                      // one group of 8 rows -> the next
+  static constexpr int kSlotStride = 2 * kSbo;                           // 16 rows (one slot) -> the next
+  static constexpr int kBoxesPerPiece = kSplit ? 1 : kSub;
+};
+
+// Tensor maps of one launch: Q in whole-tile boxes; K and V in boxes of 16, 32, 64 and 128 rows.
+struct FwdMaps {
+  CUtensorMap q;
+  CUtensorMap k[4];
+  CUtensorMap v[4];
 };
 
 // The plan of a packed item: slot s (s = 0, 1, ... in list order) is one non-empty group of 16 key
@@ -90,16 +106,14 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
 }
 
 // kCanPack = false compiles the tile-by-tile path only (no list of the launch is long enough to pack).
-template <int D, bool kCanPack>
+template <int D, bool kCanPack, bool kSplit>
 __global__ void __launch_bounds__(kThreads, 2)
-fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_k16,
-              const __grid_constant__ CUtensorMap map_v16, __nv_bfloat16 *__restrict__ O,
+fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ O,
               const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
               const uint8_t *__restrict__ flags, const uint32_t *__restrict__ bitmap,
               const uint8_t *__restrict__ groups, int B, int H, int Lq, int n_qt, float scale_log2,
               unsigned *err) {
-  using C = Cfg<D>;
+  using C = Cfg<D, kSplit>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
       reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -160,15 +174,25 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (warp == 4) {
     // ------------------------------------------------------------ producer
     if (lane == 0) {
-      prefetch_tensormap(&map_q);
-      prefetch_tensormap(&map_k);
-      prefetch_tensormap(&map_v);
+      prefetch_tensormap(&maps.q);
+      prefetch_tensormap(&maps.k[3]);
+      prefetch_tensormap(&maps.v[3]);
       mbar_arrive_expect_tx(&sh->q_full, C::kTileBytes);
 #pragma unroll
-      for (int s = 0; s < C::kSub; ++s) tma_load_3d(q_s + s * kSubBytes, &map_q, &sh->q_full, 64 * s, qt * kTile, bh);
+      for (int s = 0; s < C::kSub; ++s) tma_load_3d(q_s + s * kSubBytes, &maps.q, &sh->q_full, 64 * s, qt * kTile, bh);
     }
     bool ok = true;
     uint32_t armed_k = 0, armed_v = 0;
+    // One piece of a stage: (16 << lg) consecutive key rows from `row` on, to slot `q` of the stage.
+    auto load_piece = [&](unsigned char *stage, const CUtensorMap *m, uint64_t *bar, int q, int row) {
+      if (kSplit) {
+        tma_load_5d(stage + q * C::kSlotStride, m, bar, 0, 0, 0, row >> 3, bh);
+      } else {
+#pragma unroll
+        for (int s = 0; s < C::kSub; ++s)
+          tma_load_3d(stage + s * kSubBytes + q * C::kSlotStride, m, bar, 64 * s, row, bh);
+      }
+    };
 
     // The plan: every lane takes one list tile per round, reads its group summary, and a prefix
     // sum over the lanes gives each tile's first slot.  Packing pays when it saves enough
@@ -176,9 +200,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     bool packing = false;
     uint32_t n_slots = 0;
     if (kCanPack && n_tiles >= kMinTilesToPack && n_tiles <= kMaxPlanTiles) {
-      if (lane == 0) {
-        prefetch_tensormap(&map_k16);
-        prefetch_tensormap(&map_v16);
+      if (lane < 3) {
+        prefetch_tensormap(&maps.k[lane]);
+        prefetch_tensormap(&maps.v[lane]);
       }
       reinterpret_cast<uint32_t *>(sh->partial)[lane] = 0u;
       static_assert(kMaxPlanTiles == 128, "one 32-bit word of `partial` per lane");
@@ -237,31 +261,39 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           ok = wait_or_abort(&sh->k_empty[st], ph ^ 1u, abort_flag, err);
           if (!ok) break;
           mbar_arrive_expect_tx(&sh->k_full[st], C::kTileBytes);
-#pragma unroll
-          for (int s = 0; s < C::kSub; ++s)
-            tma_load_3d(k_s + st * C::kTileBytes + s * kSubBytes, &map_k, &sh->k_full[st], 64 * s, kt * kTile, bh);
+          load_piece(k_s + st * C::kTileBytes, &maps.k[3], &sh->k_full[st], 0, kt * kTile);
           armed_k = (uint32_t)j + 1u;
           ok = wait_or_abort(&sh->v_empty[st], ph ^ 1u, abort_flag, err);
           if (!ok) break;
           mbar_arrive_expect_tx(&sh->v_full[st], C::kTileBytes);
-#pragma unroll
-          for (int s = 0; s < C::kSub; ++s)
-            tma_load_3d(v_s + st * C::kTileBytes + s * kSubBytes, &map_v, &sh->v_full[st], 64 * s, kt * kTile, bh);
+          load_piece(v_s + st * C::kTileBytes, &maps.v[3], &sh->v_full[st], 0, kt * kTile);
           armed_v = (uint32_t)j + 1u;
         }
       }
     } else {
-      // packed: lane q copies the 16 key rows of slot q (K, then V) into the stage
+      // packed: slots whose key rows follow one another form a run; the lane of a run's first slot
+      // copies it (K, then V) in pieces of 8, 4, 2 or 1 slots
       const uint32_t n_packed = (n_slots + 7u) / 8u;
       for (uint32_t v = 0; v < n_packed && ok; ++v) {
         const int st = v % C::kStages;
         const uint32_t ph = (v / C::kStages) & 1u;
         const int ng = min(8, (int)(n_slots - 8u * v));
         const int row = lane < ng ? sh->plan_row[8u * v + lane] : 0;
-        const int row0 = __shfl_sync(0xffffffffu, row, 0), row_last = __shfl_sync(0xffffffffu, row, ng - 1);
-        // rows ascend by at least 16 from slot to slot: eight slots spanning 112 rows from a tile
-        // boundary are the eight groups of one tile, which goes out as whole-tile boxes
-        const bool one_tile = ng == 8 && (row0 & (kTile - 1)) == 0 && row_last - row0 == kTile - 16;
+        const int row_before = __shfl_up_sync(0xffffffffu, row, 1);
+        const bool head = lane < ng && (lane == 0 || row != row_before + 16);
+        const uint32_t heads = __ballot_sync(0xffffffffu, head);
+        const uint32_t later = heads >> (lane + 1);
+        const int run = head ? (later ? __ffs((int)later) : ng - lane) : 0;  // slots in this lane's run
+        auto load_run = [&](unsigned char *stage, const CUtensorMap *m4, uint64_t *bar) {
+          int q = lane, r = row, left = run;
+          while (left > 0) {
+            const int lg = left >= 8 ? 3 : left >= 4 ? 2 : left >= 2 ? 1 : 0;
+            load_piece(stage, m4 + lg, bar, q, r);
+            q += 1 << lg;
+            r += 16 << lg;
+            left -= 1 << lg;
+          }
+        };
         const uint32_t bytes = (uint32_t)ng * 16u * D * 2u;
         if (lane == 0) {
           ok = wait_or_abort(&sh->k_empty[st], ph ^ 1u, abort_flag, err);
@@ -269,14 +301,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
-        unsigned char *kd = k_s + st * C::kTileBytes;
-        if (one_tile) {
-          if (lane < C::kSub) tma_load_3d(kd + lane * kSubBytes, &map_k, &sh->k_full[st], 64 * lane, row0, bh);
-        } else if (lane < ng) {
-#pragma unroll
-          for (int s = 0; s < C::kSub; ++s)
-            tma_load_3d(kd + s * kSubBytes + lane * kGroupBytes, &map_k16, &sh->k_full[st], 64 * s, row, bh);
-        }
+        load_run(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st]);
         armed_k = v + 1u;
         if (lane == 0) {
           ok = wait_or_abort(&sh->v_empty[st], ph ^ 1u, abort_flag, err);
@@ -284,14 +309,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
-        unsigned char *vd = v_s + st * C::kTileBytes;
-        if (one_tile) {
-          if (lane < C::kSub) tma_load_3d(vd + lane * kSubBytes, &map_v, &sh->v_full[st], 64 * lane, row0, bh);
-        } else if (lane < ng) {
-#pragma unroll
-          for (int s = 0; s < C::kSub; ++s)
-            tma_load_3d(vd + s * kSubBytes + lane * kGroupBytes, &map_v16, &sh->v_full[st], 64 * s, row, bh);
-        }
+        load_run(v_s + st * C::kTileBytes, maps.v, &sh->v_full[st]);
         armed_v = v + 1u;
       }
     }
@@ -335,7 +353,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         for (int ks = 0; ks < D / 16; ++ks) {
           const int sub = ks / 4, off = (ks % 4) * 32;
           const uint64_t da = smem_desc_sw128(smem_u32(q_s + sub * kSubBytes + off), 16, 1024);
-          const uint64_t db = smem_desc_sw128(smem_u32(k_s + st * C::kTileBytes + sub * kSubBytes + off), 16, 1024);
+          const uint64_t db =
+              smem_desc_sw128(smem_u32(k_s + st * C::kTileBytes + sub * C::kHalfStride + off), 16, C::kSbo);
           mma_ss(tmem_s, da, db, idesc_qk, ks > 0);
         }
         mma_commit(&sh->k_empty[st]);
@@ -350,7 +369,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           if (ks >= ng) continue;
-          const uint64_t db = smem_desc_sw128(smem_u32(v_s + st * C::kTileBytes + ks * kGroupBytes), kSubBytes, 1024);
+          const uint64_t db =
+              smem_desc_sw128(smem_u32(v_s + st * C::kTileBytes + ks * C::kSlotStride), C::kHalfStride, C::kSbo);
           mma_ts(tmem_o, tmem_s + 8 * ks, db, idesc_pv, (v > 0 || ks > 0) ? 1u : 0u);
         }
         mma_commit(&sh->v_empty[st]);
@@ -553,17 +573,17 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (warp == 5) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int D, bool kCanPack>
-cudaError_t launch(const CUtensorMap *maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
+template <int D, bool kCanPack, bool kSplit>
+cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
                    unsigned *err, cudaStream_t s) {
-  auto kern = fwd_tc_kernel<D, kCanPack>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
+  using C = Cfg<D, kSplit>;
+  auto kern = fwd_tc_kernel<D, kCanPack, kSplit>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
   const float scale_log2 = scale * 1.4426950408889634f;
-  kern<<<B * H * t.n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4],
-                                                          static_cast<__nv_bfloat16 *>(O), t.row_ptr, t.col_idx,
-                                                          t.flags, t.bitmap, t.groups, B, H, Lq, t.n_qt, scale_log2,
-                                                          err);
+  kern<<<B * H * t.n_qt, kThreads, C::kSmemBytes, s>>>(maps, static_cast<__nv_bfloat16 *>(O), t.row_ptr, t.col_idx,
+                                                     t.flags, t.bitmap, t.groups, B, H, Lq, t.n_qt, scale_log2,
+                                                     err);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -575,18 +595,28 @@ cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_
   static_assert(sizeof(Shared) <= 7 * 1024, "shared bookkeeping outgrew its reservation");
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
-  // whole-tile boxes for Q, K, V and 16-row boxes (one group of key columns) for K and V
-  CUtensorMap maps[5];
-  if (!make_tile_map_bf16(&maps[0], Q, B * H, Lq, d) || !make_tile_map_bf16(&maps[1], K, B * H, Lk, d) ||
-      !make_tile_map_bf16(&maps[2], V, B * H, Lk, d) || !make_tile_map_bf16(&maps[3], K, B * H, Lk, d, 16) ||
-      !make_tile_map_bf16(&maps[4], V, B * H, Lk, d, 16))
-    return cudaErrorUnknown;
+  // d = 128 with whole groups of eight key rows: both halves of a row come with one box
+  const bool split = d == 128 && Lk % 8 == 0;
+  FwdMaps maps;
+  bool ok = make_tile_map_bf16(&maps.q, Q, B * H, Lq, d);
+  for (int i = 0; i < 4 && ok; ++i) {
+    const int rows = 16 << i;
+    ok = split ? make_split_map_bf16_d128(&maps.k[i], K, B * H, Lk, rows) &&
+                     make_split_map_bf16_d128(&maps.v[i], V, B * H, Lk, rows)
+               : make_tile_map_bf16(&maps.k[i], K, B * H, Lk, d, rows) &&
+                     make_tile_map_bf16(&maps.v[i], V, B * H, Lk, d, rows);
+  }
+  if (!ok) return cudaErrorUnknown;
   // lists are at most n_kt tiles long: below the packing threshold the smaller kernel does
-  if (t.n_kt < kMinTilesToPack)
-    return d == 64 ? launch<64, false>(maps, O, t, B, H, Lq, scale, err, s)
-                   : launch<128, false>(maps, O, t, B, H, Lq, scale, err, s);
-  return d == 64 ? launch<64, true>(maps, O, t, B, H, Lq, scale, err, s)
-                 : launch<128, true>(maps, O, t, B, H, Lq, scale, err, s);
+  const bool can_pack = t.n_kt >= kMinTilesToPack;
+  if (d == 64)
+    return can_pack ? launch<64, true, false>(maps, O, t, B, H, Lq, scale, err, s)
+                    : launch<64, false, false>(maps, O, t, B, H, Lq, scale, err, s);
+  if (split)
+    return can_pack ? launch<128, true, true>(maps, O, t, B, H, Lq, scale, err, s)
+                    : launch<128, false, true>(maps, O, t, B, H, Lq, scale, err, s);
+  return can_pack ? launch<128, true, false>(maps, O, t, B, H, Lq, scale, err, s)
+                  : launch<128, false, false>(maps, O, t, B, H, Lq, scale, err, s);
 }
 
 }  // namespace ap

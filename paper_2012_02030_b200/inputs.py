@@ -146,6 +146,28 @@ def random_mask(H: int, Lq: int, Lk: int, density: float, seed: int, causal: boo
     return m.to(torch.uint8).contiguous()
 
 
+def group_sparse_mask(H: int, Lq: int, Lk: int, group_frac: float, fill: float, seed: int,
+                      full_tile_frac: float = 0.0, causal: bool = False) -> torch.Tensor:
+    """Structured random mask (uint8 [H,Lq,Lk]) for tests of the forward pass: per (head, block of
+    128 query rows) each group of 16 key columns is active with probability group_frac, and only
+    inside active groups entries are kept (each with probability fill), so that most 16-column
+    groups of a tile stay empty, as in masks made of bands and a few heavy columns.  A fraction
+    full_tile_frac of the 128 x 128 tiles is kept entirely."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    n_qt, n_g, n_kt = -(-Lq // 128), -(-Lk // 16), -(-Lk // 128)
+    active = torch.rand((H, n_qt, n_g), generator=g) < group_frac
+    m = torch.rand((H, Lq, Lk), generator=g) < fill
+    act = active.repeat_interleave(128, dim=1)[:, :Lq].repeat_interleave(16, dim=2)[:, :, :Lk]
+    m &= act
+    if full_tile_frac > 0.0:
+        full = torch.rand((H, n_qt, n_kt), generator=g) < full_tile_frac
+        m |= full.repeat_interleave(128, dim=1)[:, :Lq].repeat_interleave(128, dim=2)[:, :, :Lk]
+    if causal:
+        m &= torch.tril(torch.ones((Lq, Lk), dtype=torch.bool))
+    return m.to(torch.uint8).contiguous()
+
+
 def widen(t: torch.Tensor):
     """Host tensor -> float32 numpy array with exactly the same values."""
     return t.to(torch.float32).numpy()

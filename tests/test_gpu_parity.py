@@ -196,6 +196,39 @@ def test_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
     assert np.all(o[:, empty] == 0.0)
 
 
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("case", [
+    # (B, H, Lq, Lk, group_frac, fill, full_tile_frac, causal)
+    (2, 2, 256, 1024, 0.10, 0.30, 0.00, False),   # few active groups per tile: lists pack 8 tiles into ~1
+    (1, 2, 300, 1000, 0.25, 0.05, 0.10, False),   # partial tiles mixed with fully kept ones; Lk % 128 != 0
+    (1, 2, 640, 640, 0.30, 0.50, 0.00, True),     # causal: lists of 1..5 tiles, packed and tile by tile
+    (1, 1, 128, 2052, 0.05, 0.90, 0.00, False),   # 17 key tiles, a last tile of 4 columns; Lk % 8 != 0
+    (2, 1, 200, 777, 0.50, 0.02, 0.20, False),    # odd sizes; rows >= Lq in the last query tile
+    (1, 1, 128, 1536, 1.00, 0.02, 0.00, False),   # every group active (nothing to pack away)
+])
+def test_forward_group_sparse_masks(ap, case, d):
+    """Masks whose tiles hold few non-empty 16-column groups: the forward packs the groups of
+    several key tiles into one tile; runs of neighbouring groups, lone groups, fully kept tiles
+    and ragged edges all occur."""
+    B, H, Lq, Lk, group_frac, fill, full_frac, causal = case
+    w = W["tiny"].scaled(B=B, H=H, Lq=Lq, Lk=Lk, d=d, dtype="bf16")
+    mask = inputs.group_sparse_mask(H, Lq, Lk, group_frac, fill, seed=90 + Lk, full_tile_frac=full_frac,
+                                    causal=causal)
+    assert mask.any()
+    out, _ = _fwd_case(ap, w, mask)
+    empty = mask.numpy().sum(-1) == 0
+    assert np.all(out.float().cpu().numpy()[:, empty] == 0.0)
+
+
+def test_forward_long_list_beyond_the_packing_plan(ap):
+    """A list of more key tiles than the packing plan holds (128) is processed tile by tile."""
+    H, Lq, Lk = 1, 128, 129 * 128 + 40
+    w = W["tiny"].scaled(B=1, H=H, Lq=Lq, Lk=Lk, d=64, dtype="bf16")
+    mask = inputs.group_sparse_mask(H, Lq, Lk, 0.2, 0.2, seed=93)
+    mask[:, :, ::128] = 1  # every key tile is in the list
+    _fwd_case(ap, w, mask)
+
+
 def test_forward_custom_scale(ap):
     w = W["tiny"].scaled(B=1, H=2, Lq=150, Lk=150, dtype="bf16")
     _fwd_case(ap, w, inputs.random_mask(2, 150, 150, 0.3, seed=81), scale=0.31)
