@@ -71,6 +71,24 @@ typedef enum { AP_F32 = 0, AP_BF16 = 1 } ap_dtype;
  *                        to visit, so it must agree with the bitmap; every
  *                        builder of this library writes it.
  *
+ * Rounds: the schedule the forward pass follows, derived from the fields above.
+ * The non-empty groups of a list row (eight per tile flagged as fully kept),
+ * taken in list order, are numbered as SLOTS 0, 1, ...; round k of the list row
+ * consists of its slots [8k, 8k+8), so a round covers 16..128 key columns that
+ * may come from several key tiles.  A list row with s slots has ceil(s/8) rounds;
+ * there are never more rounds than stored tiles.
+ *   round_ptr[H*n_qt + 1]      offsets into the round arrays, per list row
+ *   round_rows[cap][8]         first key row (kt*128 + 16*group) of each slot of a
+ *                              round; -1 for the unused slots of a row's last round
+ *   round_info[cap]            bits 0..3: slots of the round (1..8); bit 7: all
+ *                              128*128 entries of the round are kept
+ *   round_bitmap[cap][128][4]  the round's bitmap: the 16 columns of slot q are
+ *                              bits [16q, 16q+16) of row r (bit 16q + c of the
+ *                              128-bit row, words LSB first); 0 for unused slots
+ * Every builder of this library (ap_build_mask, ap_mask_to_tiles[_static],
+ * ap_dense_tiles) writes groups and the round arrays along with the tile list; a
+ * list assembled by hand must provide them too for ap_sparse_attention_fwd.
+ *
  * cap is the capacity in tiles; ap_tiles_capacity() always suffices.
  */
 typedef struct ap_tiles {
@@ -82,6 +100,10 @@ typedef struct ap_tiles {
   uint8_t *flags;
   uint32_t *bitmap;
   uint8_t *groups;
+  int32_t *round_ptr;
+  int32_t *round_rows;
+  uint8_t *round_info;
+  uint32_t *round_bitmap;
 } ap_tiles;
 
 /* Library version (major*10000 + minor*100 + patch). */

@@ -33,6 +33,8 @@ class ap_tiles(ctypes.Structure):
         ("n_qt", ctypes.c_int32), ("n_kt", ctypes.c_int32), ("cap", ctypes.c_int32),
         ("row_ptr", ctypes.c_void_p), ("col_idx", ctypes.c_void_p),
         ("flags", ctypes.c_void_p), ("bitmap", ctypes.c_void_p), ("groups", ctypes.c_void_p),
+        ("round_ptr", ctypes.c_void_p), ("round_rows", ctypes.c_void_p), ("round_info", ctypes.c_void_p),
+        ("round_bitmap", ctypes.c_void_p),
     ]
 
 
@@ -142,9 +144,15 @@ class Tiles:
         self.flags = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
         self.bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
         self.groups = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
+        # the forward pass's schedule (rounds of up to eight non-empty 16-column groups)
+        self.round_ptr = torch.zeros(H * self.n_qt + 1, dtype=torch.int32, device=device)
+        self.round_rows = torch.zeros((max(self.cap, 1), 8), dtype=torch.int32, device=device)
+        self.round_info = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
+        self.round_bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
         self.c = ap_tiles(H, Lq, Lk, self.n_qt, self.n_kt, self.cap, self.row_ptr.data_ptr(),
                           self.col_idx.data_ptr(), self.flags.data_ptr(), self.bitmap.data_ptr(),
-                          self.groups.data_ptr())
+                          self.groups.data_ptr(), self.round_ptr.data_ptr(), self.round_rows.data_ptr(),
+                          self.round_info.data_ptr(), self.round_bitmap.data_ptr())
 
     def n_tiles(self) -> int:
         """Number of stored tiles (synchronises)."""
@@ -155,7 +163,15 @@ class Tiles:
         T = self.n_tiles()
         return dict(row_ptr=self.row_ptr.cpu().numpy(), col_idx=self.col_idx[:T].cpu().numpy(),
                     flags=self.flags[:T].cpu().numpy(), groups=self.groups[:T].cpu().numpy(),
-                    bitmap=self.bitmap[:T].cpu().numpy().view("uint32"), n_qt=self.n_qt, n_kt=self.n_kt)
+                    bitmap=self.bitmap[:T].cpu().numpy().view("uint32"), n_qt=self.n_qt, n_kt=self.n_kt,
+                    **self.rounds_to_host())
+
+    def rounds_to_host(self):
+        """The round arrays trimmed to the stored rounds (synchronises)."""
+        R = int(self.round_ptr[-1].item())
+        return dict(round_ptr=self.round_ptr.cpu().numpy(), round_rows=self.round_rows[:R].cpu().numpy(),
+                    round_info=self.round_info[:R].cpu().numpy(),
+                    round_bitmap=self.round_bitmap[:R].cpu().numpy().view("uint32"))
 
 
 def ap_accumulate_attention(acc, Q, K, bias=None, causal=False, scale=0.0, stream=None) -> None:

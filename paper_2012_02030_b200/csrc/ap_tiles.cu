@@ -194,7 +194,172 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
   }
 }
 
+// ---- rounds: the forward pass's schedule (slots = non-empty 16-column groups in list order, eight per round)
+
+__device__ __forceinline__ uint32_t group_mask_of(const uint8_t *flags, const uint8_t *groups, int t) {
+  return (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
+}
+
+// One warp per list row: round_ptr[row + 1] = number of rounds of the row (scanned afterwards).
+__global__ void __launch_bounds__(128) count_rounds_kernel(const int32_t *__restrict__ row_ptr,
+                                                           const uint8_t *__restrict__ flags,
+                                                           const uint8_t *__restrict__ groups, int n_rows,
+                                                           int32_t *__restrict__ round_ptr) {
+  const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= n_rows) return;
+  int slots = 0;
+  for (int t = row_ptr[row] + lane; t < row_ptr[row + 1]; t += 32) slots += __popc(group_mask_of(flags, groups, t));
+  slots = __reduce_add_sync(0xffffffffu, slots);
+  if (lane == 0) {
+    round_ptr[row + 1] = (slots + 7) / 8;
+    if (row == 0) round_ptr[0] = 0;
+  }
+}
+
+// Single CTA: inclusive scan in place over round_ptr[1 .. n_rows].
+__global__ void __launch_bounds__(1024) scan_rounds_kernel(int32_t *__restrict__ round_ptr, int n_rows) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry_s;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < n_rows; base += 1024) {
+    const int idx = base + threadIdx.x;
+    const int x = idx < n_rows ? round_ptr[idx + 1] : 0;
+    int incl = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int v = warp_sums[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += u;
+      }
+      warp_sums[lane] = v;
+    }
+    __syncthreads();
+    const int carry = carry_s;
+    if (idx < n_rows) round_ptr[idx + 1] = carry + (warp ? warp_sums[warp - 1] : 0) + incl;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry_s = carry + warp_sums[31];
+    __syncthreads();
+  }
+}
+
+// One CTA per list row, thread r = bitmap row r.  The row's tiles are taken 128 at a time: their
+// slots are listed in shared memory, and every complete group of eight slots (plus the remainder
+// at the end of the list row) is written out as a round.
+__global__ void __launch_bounds__(128) fill_rounds_kernel(const int32_t *__restrict__ row_ptr,
+                                                          const int32_t *__restrict__ col_idx,
+                                                          const uint8_t *__restrict__ flags,
+                                                          const uint8_t *__restrict__ groups,
+                                                          const uint32_t *__restrict__ bitmap,
+                                                          const int32_t *__restrict__ round_ptr, int cap,
+                                                          int32_t *__restrict__ round_rows,
+                                                          uint8_t *__restrict__ round_info,
+                                                          uint32_t *__restrict__ round_bitmap) {
+  constexpr int kSeg = 128;                      // tiles per pass
+  __shared__ uint32_t slot_src[kSeg * 8 + 8];    // tile index << 4 | group << 1 | tile fully kept
+  __shared__ int32_t slot_row[kSeg * 8 + 8];     // first key row of the slot
+  __shared__ int warp_sums[4];
+  const int row = blockIdx.x, r = threadIdx.x, lane = r & 31, warp = r >> 5;
+  const int t_begin = row_ptr[row], t_end = row_ptr[row + 1];
+  int rho = round_ptr[row];
+  int pending = 0;  // slots carried over from the previous pass (fewer than eight)
+  for (int base = t_begin; base < t_end; base += kSeg) {
+    const int t = base + r;
+    uint32_t gm = 0u;
+    int kt = 0;
+    bool full = false;
+    if (t < t_end) {
+      full = flags[t] & 1;
+      gm = full ? 0xffu : (uint32_t)groups[t];
+      kt = col_idx[t];
+    }
+    const int cnt = __popc(gm);
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      if (w < warp) before += warp_sums[w];
+      total += warp_sums[w];
+    }
+    int s = pending + before + incl - cnt;
+    while (gm) {
+      const int g = __ffs((int)gm) - 1;
+      gm &= gm - 1u;
+      slot_src[s] = ((uint32_t)t << 4) | ((uint32_t)g << 1) | (full ? 1u : 0u);
+      slot_row[s] = kt * kTile + 16 * g;
+      ++s;
+    }
+    __syncthreads();
+    const int avail = pending + total;
+    const bool last_pass = base + kSeg >= t_end;
+    const int n_emit = last_pass ? (avail + 7) / 8 : avail / 8;
+    for (int k = 0; k < n_emit; ++k) {
+      const int ng = min(8, avail - 8 * k);
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      bool all_full = true;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (q >= ng) continue;
+        const uint32_t src = slot_src[8 * k + q];
+        uint32_t field = 0xffffu;
+        if (!(src & 1u)) {
+          const uint32_t g = (src >> 1) & 7u;
+          field = (bitmap[(size_t)(src >> 4) * kBitmapWords + r * 4 + (g >> 1)] >> (16u * (g & 1u))) & 0xffffu;
+          all_full = false;
+        }
+        w[q >> 1] |= field << (16 * (q & 1));
+      }
+      const int out = rho + k;
+      if (out < cap) {
+        reinterpret_cast<uint4 *>(round_bitmap + (size_t)out * kBitmapWords)[r] = make_uint4(w[0], w[1], w[2], w[3]);
+        if (r < 8) round_rows[(size_t)out * 8 + r] = r < ng ? slot_row[8 * k + r] : -1;
+        if (r == 0) round_info[out] = (uint8_t)(ng | ((all_full && ng == 8) ? 0x80 : 0));
+      }
+    }
+    rho += n_emit;
+    __syncthreads();
+    // fewer than eight slots are left over; they move to the front (no overlap: they start at or
+    // beyond index 8 unless nothing was written out, in which case they are in place already)
+    const int left = avail - 8 * n_emit;
+    if (!last_pass && n_emit > 0 && r < left) {
+      const uint32_t a = slot_src[8 * n_emit + r];
+      const int32_t b = slot_row[8 * n_emit + r];
+      slot_src[r] = a;
+      slot_row[r] = b;
+    }
+    pending = last_pass ? 0 : left;
+    __syncthreads();
+  }
+}
+
 }  // namespace
+
+// Writes the round arrays of a finished tile list (row_ptr, col_idx, flags, groups, bitmap).
+cudaError_t launch_build_rounds(const ap_tiles &t, cudaStream_t s) {
+  const int n_rows = t.H * t.n_qt;
+  count_rounds_kernel<<<ceil_div(n_rows, 4), 128, 0, s>>>(t.row_ptr, t.flags, t.groups, n_rows, t.round_ptr);
+  scan_rounds_kernel<<<1, 1024, 0, s>>>(t.round_ptr, n_rows);
+  fill_rounds_kernel<<<n_rows, 128, 0, s>>>(t.row_ptr, t.col_idx, t.flags, t.groups, t.bitmap, t.round_ptr, t.cap,
+                                            t.round_rows, t.round_info, t.round_bitmap);
+  count_launches(3);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_stage_from_mask(const uint8_t *mask, int H, int Lq, int Lk, uint32_t *stage_bitmap,
                                    int32_t *stage_count, cudaStream_t s) {
@@ -219,7 +384,9 @@ cudaError_t launch_compact_tiles(const uint32_t *stage_bitmap, const int32_t *st
   gather_tiles_kernel<<<n_tiles, 128, 0, s>>>(stage_bitmap, stage_count, stage_pos, t.n_kt, t.cap,
                                               t.col_idx, t.flags, t.bitmap, t.groups);
   count_launches(1);
-  return cudaGetLastError();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return launch_build_rounds(t, s);
 }
 
 cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
@@ -228,7 +395,9 @@ cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
   dense_tiles_kernel<<<t.H * t.n_qt * t.n_kt, 128, 0, s>>>(t.H, t.Lq, t.Lk, t.n_qt, t.n_kt, causal, t.cap,
                                                          t.row_ptr, t.col_idx, t.flags, t.bitmap, t.groups, err);
   count_launches(1);
-  return cudaGetLastError();
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  return launch_build_rounds(t, s);
 }
 
 }  // namespace ap

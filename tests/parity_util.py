@@ -38,6 +38,37 @@ def groups_from_bitmap(bitmap: np.ndarray) -> np.ndarray:
     return out
 
 
+def rounds_from_tiles(t: dict) -> dict:
+    """The forward pass's schedule restated from its definition, slot by slot, from a tile list
+    (row_ptr, col_idx, flags, bitmap): the non-empty 16-column groups of a list row in list order
+    are its slots, eight slots make a round."""
+    row_ptr, col_idx, flags, bitmap = t["row_ptr"], t["col_idx"], t["flags"], t["bitmap"]
+    T = len(col_idx)
+    bits = np.unpackbits(np.ascontiguousarray(bitmap).view(np.uint8).reshape(T, 128, 16), axis=2,
+                         bitorder="little").reshape(T, 128, 8, 16) if T else np.zeros((0, 128, 8, 16), np.uint8)
+    round_ptr, rows, info, rbits = [0], [], [], []
+    for lr in range(len(row_ptr) - 1):
+        slots = []  # (first key row, [128,16] bits, tile fully kept)
+        for tt in range(row_ptr[lr], row_ptr[lr + 1]):
+            for g in range(8):
+                if bits[tt, :, g, :].any():
+                    slots.append((int(col_idx[tt]) * 128 + 16 * g, bits[tt, :, g, :], bool(flags[tt] & 1)))
+        for k in range(0, len(slots), 8):
+            chunk = slots[k:k + 8]
+            rows.append([s[0] for s in chunk] + [-1] * (8 - len(chunk)))
+            info.append(len(chunk) | (0x80 if len(chunk) == 8 and all(s[2] for s in chunk) else 0))
+            b = np.zeros((128, 8, 16), np.uint8)
+            for q, s in enumerate(chunk):
+                b[:, q, :] = s[1]
+            rbits.append(b.reshape(128, 128))
+        round_ptr.append(len(rows))
+    R = len(rows)
+    packed = (np.packbits(np.array(rbits, dtype=np.uint8).reshape(R, 128, 128), axis=2, bitorder="little")
+              .view(np.uint32).reshape(R, 128, 4) if R else np.zeros((0, 128, 4), np.uint32))
+    return dict(round_ptr=np.array(round_ptr, dtype=np.int32), round_rows=np.array(rows, dtype=np.int32).reshape(R, 8),
+                round_info=np.array(info, dtype=np.uint8), round_bitmap=packed)
+
+
 def assert_tiles_equal(got: dict, want: dict):
     np.testing.assert_array_equal(got["row_ptr"], want["row_ptr"])
     np.testing.assert_array_equal(got["col_idx"], want["col_idx"])
@@ -45,6 +76,10 @@ def assert_tiles_equal(got: dict, want: dict):
     np.testing.assert_array_equal(got["bitmap"], want["bitmap"])
     if "groups" in got:  # derived data: checked against its definition applied to the oracle's bitmaps
         np.testing.assert_array_equal(got["groups"], groups_from_bitmap(want["bitmap"]))
+    if "round_ptr" in got:  # the schedule, likewise, against its definition applied to the oracle's list
+        rounds = rounds_from_tiles(want)
+        for key in ("round_ptr", "round_rows", "round_info", "round_bitmap"):
+            np.testing.assert_array_equal(got[key], rounds[key], err_msg=key)
 
 
 def gpu_accumulate(ap, w, n_batches, bias_dev):

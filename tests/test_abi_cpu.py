@@ -45,7 +45,7 @@ def test_version_strings_sizes():
 
 
 def _tiles(H=2, Lq=128, Lk=128, cap=2, ptr=FAKE):
-    return ap.ap_tiles(H, Lq, Lk, -(-Lq // 128), -(-Lk // 128), cap, ptr, ptr, ptr, ptr, ptr)
+    return ap.ap_tiles(H, Lq, Lk, -(-Lq // 128), -(-Lk // 128), cap, *([ptr] * 9))
 
 
 def test_forward_rejects_bad_arguments_before_any_device_work():

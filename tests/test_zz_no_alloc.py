@@ -21,7 +21,7 @@ FAKE = 0x10000
 def test_static_variant_rejects_shapes_beyond_its_scratch_before_touching_a_device():
     from paper_2012_02030_b200 import binding as ap
 
-    t = ap.ap_tiles(16, 4096, 4096, 32, 32, 16384, FAKE, FAKE, FAKE, FAKE, FAKE)
+    t = ap.ap_tiles(16, 4096, 4096, 32, 32, 16384, *([FAKE] * 9))
     assert 16 * 32 * 32 > ap.AP_STATIC_MAX_TILES
     st = ap.lib.ap_mask_to_tiles_static(FAKE, 16, 4096, 4096, ctypes.byref(t), None)
     assert st == ap.AP_ERR_WORKSPACE
@@ -44,10 +44,11 @@ def test_static_variant_matches_workspace_variant_on_two_calls_in_a_row():
         got = ap.Tiles(H, Lq, Lk)
         before = ap.ap_launch_count()
         ap.ap_mask_to_tiles_static(mask, got)
-        assert ap.ap_launch_count() - before == 3
+        assert ap.ap_launch_count() - before == 6  # bitmaps, scan, gather; rounds: count, scan, fill
         assert ap.ap_device_status() == ap.AP_OK
         a, b = got.to_host(), want.to_host()
-        for key in ("row_ptr", "col_idx", "flags", "bitmap", "groups"):
+        for key in ("row_ptr", "col_idx", "flags", "bitmap", "groups", "round_ptr", "round_rows", "round_info",
+                    "round_bitmap"):
             np.testing.assert_array_equal(a[key], b[key], err_msg=key)
         assert got.n_tiles() > 0
     # exactly at the limit is accepted, one tile more is refused
