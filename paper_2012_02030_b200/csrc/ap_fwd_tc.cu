@@ -23,10 +23,18 @@
 // item's last rounds.  S is double-buffered in TMEM and the MMA thread issues S(g+1) = Q K^T
 // before O += P(g) V, so the softmax threads find the next S ready when they finish a round.
 //
-// Warp roles (192 threads): warps 0-3 softmax + epilogue (thread = query row = TMEM lane),
-// warp 4 producer, warp 5 MMA issuer and TMEM owner.  TMEM (512 columns): S[0] at column 0, S[1]
-// at 128, O at 256.  Every wait is bounded; a wait that expires raises the device status word
-// and the CTA winds down.
+//
+// The softmax is shared by two groups of four warps.  The 32-column chunks of a round alternate
+// between them (chunk c belongs to group c & 1), and each group is an online softmax of its own:
+// its own reference m and sum l per query row and its own output accumulator in TMEM (O += P V
+// of a slot goes to the accumulator of the slot's group), so the groups never exchange anything
+// inside a round.  The item's epilogue merges the two partial results
+//   O = (a_0 O_0 + a_1 O_1) / (a_0 l_0 + a_1 l_1),   a_i = exp2(c (m_i - max(m_0, m_1))).
+//
+// Warp roles (320 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
+// TMEM lane), warp 8 producer, warp 9 MMA issuer and TMEM owner.  TMEM (512 columns): S[0] at
+// column 0, S[1] at 128, O_0 at 256, O_1 at 384.  Every wait is bounded; a wait that expires
+// raises the device status word and the CTA winds down.
 #include <math_constants.h>
 
 #include "ap_common.cuh"
@@ -38,7 +46,8 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
+constexpr int kSoftmaxThreads = 256;   // two groups of 128
 constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-tile
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kMaxPolls = 1u << 22;
@@ -64,7 +73,7 @@ struct Cfg {
   static constexpr int kKOffset = 2 * kTileBytes;     // after the two Q buffers
   static constexpr int kVOffset = kKOffset + kStages * kTileBytes;
   static constexpr int kBarOffset = kVOffset + kStages * kTileBytes;
-  static constexpr int kSmemBytes = kBarOffset + 9 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
+  static constexpr int kSmemBytes = kBarOffset + 13 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
   static constexpr int kHalfStride = kSplit ? 1024 : kSubBytes;          // half 0 -> half 1 of the same rows
   static constexpr int kSbo = kSplit ? 2048 : 1024;                      // one group of 8 rows -> the next
   static constexpr int kSlotStride = 2 * kSbo;                           // 16 rows (one slot) -> the next
@@ -86,6 +95,8 @@ struct Shared {
   uint64_t s_full[2], p_full[2];                      // per S buffer
   uint64_t pv_done;                                   // O += P V of a round has completed
   uint64_t o_done, o_free;                            // per item: O complete / O read out by the epilogue
+  uint64_t ml_ready;                                  // per item: both groups have published (m, l)
+  float2 ml[2][2][kTile];                             // [item parity][group][row] = (m, l)
   uint32_t info[kMaxStages];
   int32_t item[kMaxStages];                           // the item a stage's round belongs to
   uint32_t tmem_base;
@@ -131,7 +142,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       mbar_init(&sh->q_full[i], 1);
       mbar_init(&sh->q_empty[i], 1);
       mbar_init(&sh->s_full[i], 1);
-      mbar_init(&sh->p_full[i], 128);
+      mbar_init(&sh->p_full[i], kSoftmaxThreads);
     }
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&sh->k_full[s], 1);
@@ -142,11 +153,12 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     for (int s = 0; s < kMaxStages; ++s) mbar_init(&sh->b_full[s], 1);
     mbar_init(&sh->pv_done, 1);
     mbar_init(&sh->o_done, 1);
-    mbar_init(&sh->o_free, 128);
+    mbar_init(&sh->o_free, kSoftmaxThreads);
+    mbar_init(&sh->ml_ready, kSoftmaxThreads);
     sh->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 5) {
+  if (warp == 9) {
     tmem_alloc(&sh->tmem_base, kTmemCols);
     tmem_relinquish();
   }
@@ -158,7 +170,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
   volatile int *abort_flag = &sh->abort_flag;
   const int item_step = (int)gridDim.x;
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ------------------------------------------------------------ producer
     if (lane < 4) {
       prefetch_tensormap(&maps.k[lane]);
@@ -309,7 +321,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         mbar_wait(&sh->b_full[a % kMaxStages], (a / kMaxStages) & 1u, 1u << 16);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
@@ -320,6 +332,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       uint32_t pend_g = 0, pend_n = 0;
       int pend_ng = 0;
       bool pend_first = false, pend_last = false;
+      uint32_t started0 = 0u, started1 = 0u;  // the item's O_0 / O_1 holds a partial result already
       auto issue_pv = [&]() {
         const uint32_t sb = pend_g & 1u;
         const int st = (int)(pend_g % C::kStages);
@@ -329,12 +342,20 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         if (ok && pend_first && pend_n > 0) ok = wait_or_abort(&sh->o_free, (pend_n - 1u) & 1u, abort_flag, err);
         if (!ok) return;
         tc_fence_after_sync();
-        // one K step of 16 keys per slot; P (bf16) of slot q sits in columns [8q, 8q + 8) of S
+        // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
+        // 16 columns of that chunk of S (each group stays inside its own chunks), so slot q's
+        // eight columns of P start at column 32 (q / 2) + 8 (q % 2).
+        // Slots 0, 1, 4, 5 (chunks 0 and 2) belong to softmax group 0 and add to O_0, the others to
+        // O_1; a group's first step of an item overwrites its accumulator.
+        if (pend_first) started0 = started1 = 0u;
 #pragma unroll 1
         for (int ks = 0; ks < pend_ng; ++ks) {
+          const int grp = (ks >> 1) & 1;
           const uint64_t db =
               smem_desc_sw128(smem_u32(v_s + st * C::kTileBytes + ks * C::kSlotStride), C::kHalfStride, C::kSbo);
-          mma_ts(tmem_o, tmem + 128u * sb + 8 * ks, db, idesc_pv, (!pend_first || ks > 0) ? 1u : 0u);
+          mma_ts(tmem_o + 128u * grp, tmem + 128u * sb + 32 * (ks >> 1) + 8 * (ks & 1), db, idesc_pv,
+                 grp ? started1 : started0);
+          if (grp) started1 = 1u; else started0 = 1u;
         }
         mma_commit(&sh->v_empty[st]);
         mma_commit(&sh->pv_done);
@@ -388,12 +409,15 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue
-    const int r = warp * 32 + lane;          // row of the query tile == TMEM lane
-    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const int grp = warp >> 2;               // softmax group: chunks grp and grp + 2 of every round
+    const int r = (warp & 3) * 32 + lane;    // row of the query tile == TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tmem_og = tmem_o + 128u * grp;  // this group's output accumulator
     const float ref_slack = 8.f / scale_log2;
     bool ok = true;
     uint32_t n = 0;
-    float m = -CUDART_INF_F, l = 0.f;       // exponent reference and running sum of weights
+    float m = -CUDART_INF_F, l = 0.f;       // this group's exponent reference and running sum of weights
+    bool o_started = false;                  // an earlier round of the item added to this group's accumulator
     int i = 0;                               // this thread's query row in the tensor
     __nv_bfloat16 *orow = O;
     for (uint32_t g = 0; ok; ++g) {
@@ -414,30 +438,39 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         orow = O + ((size_t)bh * Lq + i) * D;
         m = -CUDART_INF_F;
         l = 0.f;
+        o_started = false;
       }
-      const int n_chunks = (ng + 1) >> 1;  // 32-column chunks the round spans
-      uint4 cur = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
-      if (!tile_full) cur = *reinterpret_cast<const uint4 *>(&sh->bitmap[st][r][0]);
-      // 32-column chunks in which none of this warp's 32 rows keeps anything are skipped
-      // (their P is written as zeros without reading S)
-      const uint32_t w0 = cur.x, w1 = cur.y, w2 = cur.z, w3 = cur.w;
-      const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u) |
-                              (__any_sync(0xffffffffu, w2 != 0u) ? 4u : 0u) | (__any_sync(0xffffffffu, w3 != 0u) ? 8u : 0u);
-      ok = wait_or_abort(&sh->s_full[sb], (g >> 1) & 1u, abort_flag, err);
-      if (!ok) break;
+      // this group's 32-column chunks of the round: grp and grp + 2, as far as the round reaches
+      const int n_mine = ((ng + 1) >> 1) > grp + 2 ? 2 : ((ng + 1) >> 1) > grp ? 1 : 0;
+      float alpha = 1.f;
+      if (n_mine > 0) {
+      uint32_t w0 = 0xffffffffu, w1 = 0xffffffffu;   // bitmap words of chunks grp and grp + 2
+      if (!tile_full) {
+        const uint32_t *brow = &sh->bitmap[st][r][0];
+        w0 = brow[grp];
+        w1 = brow[grp + 2];
+      }
+      // chunks in which none of this warp's 32 rows keeps anything are skipped (their P is
+      // written as zeros without reading S)
+      const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u);
+      if (!mbar_try_wait(&sh->s_full[sb], (g >> 1) & 1u)) {
+        ok = wait_or_abort(&sh->s_full[sb], (g >> 1) & 1u, abort_flag, err);
+        if (!ok) break;
+      }
       tc_fence_after_sync();
       // pass 1: row maximum over kept entries (four independent chains).  In a partially filled
       // round the pruned entries are replaced by -inf and the chunk is written back to TMEM, so
       // that pass 2 needs no bitmap: exp2 of -inf is exactly 0.
       float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
 #pragma unroll 1
-      for (int c = 0; c < n_chunks; ++c) {
-        if (!((active >> c) & 1u)) continue;
+      for (int cc = 0; cc < n_mine; ++cc) {
+        if (!((active >> cc) & 1u)) continue;
+        const int c = grp + 2 * cc;
         uint32_t x[32];
         tmem_ld32(tmem_s + lane_addr + 32 * c, x);
         tmem_wait_ld();
         if (!tile_full) {
-          const uint32_t w = c == 0 ? w0 : c == 1 ? w1 : c == 2 ? w2 : w3;
+          const uint32_t w = cc == 0 ? w0 : w1;
 #pragma unroll
           for (int e = 0; e < 32; ++e)
             if (!((w >> e) & 1u)) x[e] = 0xff800000u;  // -inf
@@ -460,34 +493,35 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       const bool move = tile_max > m + ref_slack;   // also true for the first kept entry (m = -inf)
       const float m_new = move ? tile_max : m;
       const float m_safe = m_new == -CUDART_INF_F ? 0.f : m_new;
-      const float alpha = move ? ex2_approx((m - m_safe) * scale_log2) : 1.f;  // 0 when m was -inf
+      alpha = move ? ex2_approx((m - m_safe) * scale_log2) : 1.f;  // 0 when m was -inf
       const float neg_mc = -m_safe * scale_log2;
       m = m_new;
-      // Rescale the running output where the reference moved.  O += P V of the previous round may
-      // still be running (this round's S was computed ahead of it): wait for it first.
-      if (!first && __any_sync(0xffffffffu, alpha != 1.f)) {
+      // Rescale the group's running output where the reference moved.  O += P V of the previous
+      // round may still be running (this round's S was computed ahead of it): wait for it first.
+      if (o_started && __any_sync(0xffffffffu, alpha != 1.f)) {
         ok = wait_or_abort(&sh->pv_done, (g - 1u) & 1u, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll 1
         for (int c = 0; c < D / 32; ++c) {
           uint32_t o[32];
-          tmem_ld32(tmem_o + lane_addr + 32 * c, o);
+          tmem_ld32(tmem_og + lane_addr + 32 * c, o);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(tmem_o + lane_addr + 32 * c, o);
+          tmem_st32(tmem_og + lane_addr + 32 * c, o);
         }
       }
       // pass 2: P = exp2(c*S - c*m); pruned entries are -inf by now and give exactly 0; bf16 P over S
       float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll 1
-      for (int c = 0; c < n_chunks; ++c) {
+      for (int cc = 0; cc < n_mine; ++cc) {
+        const int c = grp + 2 * cc;
         uint32_t pk[16];
-        if (!((active >> c) & 1u)) {
+        if (!((active >> cc) & 1u)) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) pk[e] = 0u;
-          tmem_st16(tmem_s + lane_addr + 16 * c, pk);
+          tmem_st16(tmem_s + lane_addr + 32 * c, pk);
           continue;
         }
         uint32_t x[32];
@@ -504,24 +538,41 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
           sum0 += __uint_as_float(pk[e] << 16);
           sum1 += __uint_as_float(pk[e] & 0xffff0000u);
         }
-        tmem_st16(tmem_s + lane_addr + 16 * c, pk);
+        tmem_st16(tmem_s + lane_addr + 32 * c, pk);
       }
       l = l * alpha + (sum0 + sum1);
+      o_started = true;
       tmem_wait_st();
+      }  // n_mine > 0
       tc_fence_before_sync();
       mbar_arrive(&sh->p_full[sb]);
       if (!last) continue;
-      // epilogue: O / l, rounded once to bf16
-      ok = wait_or_abort(&sh->o_done, n & 1u, abort_flag, err);
+      // Epilogue.  The groups exchange (m, l), then each takes half of the output columns, merges
+      // the two accumulators and writes O / l, rounded once to bf16.
+      sh->ml[n & 1u][grp][r] = make_float2(m, l);
+      mbar_arrive(&sh->ml_ready);
+      ok = wait_or_abort(&sh->ml_ready, n & 1u, abort_flag, err);
+      if (ok) ok = wait_or_abort(&sh->o_done, n & 1u, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const float2 other = sh->ml[n & 1u][grp ^ 1][r];
+      const float m_tot = fmaxf(m, other.x);
+      // weight of a partial result; 0 for a group that saw no kept entry of this row (m = -inf),
+      // whose accumulator is then never read into the sum (it may hold a previous item's data)
+      const float a_mine = m == -CUDART_INF_F ? 0.f : ex2_approx((m - m_tot) * scale_log2);
+      const float a_other = other.x == -CUDART_INF_F ? 0.f : ex2_approx((other.x - m_tot) * scale_log2);
+      const float l_tot = l * a_mine + other.y * a_other;
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      const float f0 = (grp == 0 ? a_mine : a_other) * inv, f1 = (grp == 0 ? a_other : a_mine) * inv;
+      constexpr int kHalf = D / 2;  // output columns per group
 #pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem_o + lane_addr + 32 * c, o);
+      for (int c = 0; c < kHalf / 32; ++c) {
+        const int col = grp * kHalf + 32 * c;
+        uint32_t o0[32], o1[32];
+        tmem_ld32(tmem_o + lane_addr + col, o0);
+        tmem_ld32(tmem_o + 128u + lane_addr + col, o1);
         tmem_wait_ld();
-        if (c == D / 32 - 1) {  // O is in registers: the next item may overwrite it
+        if (c == kHalf / 32 - 1) {  // this thread's share of O is in registers: the next item may overwrite it
           tc_fence_before_sync();
           mbar_arrive(&sh->o_free);
         }
@@ -532,12 +583,14 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               // a row without kept entries has l = 0 and P = 0 throughout: write exact zeros
-              const float a = l > 0.f ? __uint_as_float(o[8 * q + 2 * e]) * inv : 0.f;
-              const float bb = l > 0.f ? __uint_as_float(o[8 * q + 2 * e + 1]) * inv : 0.f;
-              __nv_bfloat162 hh = __floats2bfloat162_rn(a, bb);
+              const int j = 8 * q + 2 * e;
+              const float x0 = (f0 > 0.f ? __uint_as_float(o0[j]) * f0 : 0.f) + (f1 > 0.f ? __uint_as_float(o1[j]) * f1 : 0.f);
+              const float x1 = (f0 > 0.f ? __uint_as_float(o0[j + 1]) * f0 : 0.f) +
+                               (f1 > 0.f ? __uint_as_float(o1[j + 1]) * f1 : 0.f);
+              __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
               pk[e] = *reinterpret_cast<uint32_t *>(&hh);
             }
-            *reinterpret_cast<uint4 *>(orow + 32 * c + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4 *>(orow + col + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
       }
@@ -546,7 +599,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
 int sm_count() {
@@ -565,7 +618,7 @@ template <int D, bool kSplit>
 cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
                    unsigned *err, cudaStream_t s) {
   using C = Cfg<D, kSplit>;
-  static_assert(sizeof(Shared) <= 9 * 1024, "shared bookkeeping outgrew its reservation");
+  static_assert(sizeof(Shared) <= 13 * 1024, "shared bookkeeping outgrew its reservation");
   static_assert(C::kStages <= kMaxStages, "ring deeper than its barriers");
   static_assert(C::kSmemBytes > 114 * 1024 && C::kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
   auto kern = fwd_tc_kernel<D, kSplit>;
