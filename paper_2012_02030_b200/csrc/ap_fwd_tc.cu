@@ -1,7 +1,8 @@
 // Masked attention of Section 3.2 for bf16 tensors on the tcgen05 tensor cores.
 //
-// Persistent kernel, one CTA per SM.  A work item is one (b, h, query tile of 128 rows); CTA c
-// takes items c, c + gridDim.x, ... (heavy items first).  The CTA follows the schedule stored
+// Persistent kernel, one CTA per SM.  A work item is one (b, h, query tile of 128 rows); items
+// are handed out in pairs (a late and an early query tile of the same head), CTA c taking pairs
+// c, c + gridDim.x, ...  The CTA follows the schedule stored
 // with the tile list: the ROUNDS of the item's (h, qt) list row.  A round holds up to eight
 // non-empty groups of 16 key columns (slots), taken in list order from one or several key tiles,
 // together with the bitmap of exactly those columns; groups without a kept entry never appear, so
@@ -121,12 +122,21 @@ __device__ __noinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volat
   return false;
 }
 
+// The same wait for a whole (converged) warp: one lane polls - 32 lanes polling one barrier would
+// serialise - and the outcome is shared.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag,
+                                          unsigned *err) {
+  bool ok = true;
+  if (lane == 0 && !mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, abort_flag, err);
+  return __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+}
+
 template <int D, bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ O,
               const int32_t *__restrict__ round_ptr, const int32_t *__restrict__ round_rows,
               const uint8_t *__restrict__ round_info, const uint32_t *__restrict__ round_bitmap, int B, int H,
-              int Lq, int n_qt, int n_items, float scale_log2, unsigned *err) {
+              int Lq, int n_qt, float scale_log2, unsigned *err) {
   using C = Cfg<D, kSplit>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -180,9 +190,33 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     bool ok = true;
     uint32_t g = 0, n = 0;   // rounds / non-empty items so far
     int armed_q = -1;        // non-empty item whose Q copy was armed last
-    // Items are numbered so that heavy (late, under a causal mask) query tiles come first and b
-    // runs fastest, so that CTAs working at the same time share rounds and bitmaps in L2.
-    auto list_row_of = [&](int item) { return ((item / B) % H) * n_qt + (n_qt - 1 - item / (B * H)); };
+    // Work is handed out in units of two items of one (b, h): query tile n_qt - 1 - j and query
+    // tile j.  Under a causal mask a late tile has a long list and an early one a short list, so
+    // units weigh about the same; and because consecutive units belong to the same (b, h), the
+    // CTAs running at any time share a few heads' K and V, which then stay in L2.  The t-th item
+    // of this CTA is half t & 1 of unit blockIdx.x + (t >> 1) * gridDim.x.
+    const int n_half = (n_qt + 1) / 2, n_units = B * H * n_half;
+    struct ItemRef {
+      int bh, qt, rho0, n_rounds;  // n_rounds < 0: no such item (the unit's halves coincide)
+      bool in_range;
+    };
+    auto item_ref = [&](int t) {
+      ItemRef it;
+      const int u = (int)blockIdx.x + (t >> 1) * item_step;
+      it.in_range = u < n_units;
+      it.bh = 0, it.qt = 0, it.rho0 = 0, it.n_rounds = -1;
+      if (it.in_range) {
+        const int j = u % n_half;
+        it.bh = u / n_half;
+        it.qt = (t & 1) ? j : n_qt - 1 - j;
+        if (!(t & 1) || j != n_qt - 1 - j) {
+          const int lr = (it.bh % H) * n_qt + it.qt;
+          it.rho0 = round_ptr[lr];
+          it.n_rounds = round_ptr[lr + 1] - it.rho0;
+        }
+      }
+      return it;
+    };
     // One piece of a stage: (16 << lg) consecutive key rows from `row` on, to slot `q` of the stage.
     auto load_piece = [&](unsigned char *stage, const CUtensorMap *m, uint64_t *bar, int q, int row, int bh) {
       if (kSplit) {
@@ -204,23 +238,40 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       if (lane == 0) ok = wait_or_abort(bar, ph ^ 1u, abort_flag, err);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     };
-    // the rounds of an item are looked up one item ahead
-    int nb = 0, ne = 0;
-    if ((int)blockIdx.x < n_items) {
-      const int lr = list_row_of((int)blockIdx.x);
-      nb = round_ptr[lr];
-      ne = round_ptr[lr + 1];
-    }
-    for (int item = (int)blockIdx.x; item < n_items && ok; item += item_step) {
-      const int bh = (item % B) * H + (item / B) % H;
-      const int qt = n_qt - 1 - item / (B * H);
-      const int rho0 = nb, n_rounds = ne - nb;
-      if (item + item_step < n_items) {
-        const int lr = list_row_of(item + item_step);
-        nb = round_ptr[lr];
-        ne = round_ptr[lr + 1];
+    // A run of slots (key rows following one another) is copied by the lane of its first slot, in
+    // pieces of 8, 4, 2 or 1 slots.
+    auto load_run = [&](unsigned char *stage, const CUtensorMap *m4, uint64_t *bar, int row, int run, int bh) {
+      int q = lane, r = row, left = run;
+      while (left > 0) {
+        const int lg = left >= 8 ? 3 : left >= 4 ? 2 : left >= 2 ? 1 : 0;
+        load_piece(stage, m4 + lg, bar, q, r, bh);
+        q += 1 << lg;
+        r += 16 << lg;
+        left -= 1 << lg;
       }
-      if (n_rounds <= 0) {
+    };
+    // V of a round is copied one round later than its K: K only needs S = Q K^T of the round that
+    // used the stage before to be over, V needs that round's O += P V, which comes much later;
+    // issued in round order, the V copy would hold back the next round's K.
+    bool pv_valid = false;
+    int pv_st = 0, pv_ng = 0, pv_row = 0, pv_run = 0, pv_bh = 0;
+    uint32_t pv_ph = 0;
+    auto issue_v = [&]() {
+      if (C::kStages != kMaxStages) wait_free(&sh->v_empty[pv_st], pv_ph);
+      if (!ok) return;
+      if (lane == 0) mbar_arrive_expect_tx(&sh->v_full[pv_st], (uint32_t)pv_ng * 16u * D * 2u);
+      __syncwarp();
+      load_run(v_s + pv_st * C::kTileBytes, maps.v, &sh->v_full[pv_st], pv_row, pv_run, pv_bh);
+      pv_valid = false;
+    };
+    // the rounds of an item are looked up one item ahead
+    ItemRef next = item_ref(0);
+    for (int t = 0; next.in_range && ok; ++t) {
+      const ItemRef cur = next;
+      next = item_ref(t + 1);
+      const int bh = cur.bh, qt = cur.qt, rho0 = cur.rho0, n_rounds = cur.n_rounds;
+      if (n_rounds < 0) continue;
+      if (n_rounds == 0) {
         // nothing kept in this query tile: its output rows are zero (nobody else sees the item)
         const int rows = min(kTile, Lq - qt * kTile);
         uint4 *dst = reinterpret_cast<uint4 *>(O + ((size_t)bh * Lq + (size_t)qt * kTile) * D);
@@ -255,23 +306,12 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         const uint32_t ph = (g / C::kStages) & 1u;
         const int ng = (int)(rinfo & 15u);
         const bool full = (rinfo & 0x80u) != 0u;
-        // slots whose key rows follow one another form a run; the lane of a run's first slot
-        // copies it (K, then V) in pieces of 8, 4, 2 or 1 slots
+        // slots whose key rows follow one another form a run
         const int row_before = __shfl_up_sync(0xffffffffu, row, 1);
         const bool head = lane < ng && (lane == 0 || row != row_before + 16);
         const uint32_t heads = __ballot_sync(0xffffffffu, head);
         const uint32_t later = lane < 31 ? heads >> (lane + 1) : 0u;
         const int run = head ? (later ? __ffs((int)later) : ng - lane) : 0;  // slots in this lane's run
-        auto load_run = [&](unsigned char *stage, const CUtensorMap *m4, uint64_t *bar) {
-          int q = lane, r = row, left = run;
-          while (left > 0) {
-            const int lg = left >= 8 ? 3 : left >= 4 ? 2 : left >= 2 ? 1 : 0;
-            load_piece(stage, m4 + lg, bar, q, r, bh);
-            q += 1 << lg;
-            r += 16 << lg;
-            left -= 1 << lg;
-          }
-        };
         const int si = (int)(g % kMaxStages);
         wait_free(&sh->k_empty[st], ph);
         if (ok && C::kStages == kMaxStages) wait_free(&sh->v_empty[st], ph);
@@ -280,7 +320,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         if (lane == 0) {
           sh->info[si] = (uint32_t)ng | (v == 0 ? kInfoFirst : 0u) | (v + 1 == n_rounds ? kInfoLast : 0u) |
                          (full ? kInfoFull : 0u);
-          sh->item[si] = item;
+          sh->item[si] = bh * n_qt + qt;
           mbar_arrive_expect_tx(&sh->k_full[st], bytes);
           if (full) {
             mbar_arrive(&sh->b_full[si]);
@@ -291,15 +331,15 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
           }
         }
         __syncwarp();
-        load_run(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st]);
-        if (C::kStages != kMaxStages) wait_free(&sh->v_empty[st], ph);
+        load_run(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st], row, run, bh);
+        if (pv_valid) issue_v();
         if (!ok) break;
-        if (lane == 0) mbar_arrive_expect_tx(&sh->v_full[st], bytes);
-        __syncwarp();
-        load_run(v_s + st * C::kTileBytes, maps.v, &sh->v_full[st]);
+        pv_valid = true;
+        pv_st = st, pv_ph = ph, pv_ng = ng, pv_row = row, pv_run = run, pv_bh = bh;
       }
       ++n;
     }
+    if (ok && pv_valid) issue_v();
     // no more work: one more stage carries the stop word
     if (ok) {
       const int st = (int)(g % C::kStages);
@@ -323,8 +363,11 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the rounds in lockstep (every lane waits on the barriers and keeps the
+    // same, warp-uniform state); one elected lane issues the tcgen05 instructions.
+    {
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
+      const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s), v_addr = smem_u32(v_s);
       bool ok = true;
       uint32_t n = 0;  // non-empty items started so far
       // O += P V of the round before the current one is issued after the current S = Q K^T
@@ -333,13 +376,14 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       int pend_ng = 0;
       bool pend_first = false, pend_last = false;
       uint32_t started0 = 0u, started1 = 0u;  // the item's O_0 / O_1 holds a partial result already
+      auto wait = [&](uint64_t *bar, uint32_t parity) { ok = warp_wait(bar, parity, lane, abort_flag, err); };
       auto issue_pv = [&]() {
         const uint32_t sb = pend_g & 1u;
         const int st = (int)(pend_g % C::kStages);
-        ok = wait_or_abort(&sh->p_full[sb], (pend_g >> 1) & 1u, abort_flag, err);
-        if (ok) ok = wait_or_abort(&sh->v_full[st], (pend_g / C::kStages) & 1u, abort_flag, err);
+        wait(&sh->p_full[sb], (pend_g >> 1) & 1u);
+        if (ok) wait(&sh->v_full[st], (pend_g / C::kStages) & 1u);
         // the first round of an item overwrites O: the epilogue of the previous item must have read it
-        if (ok && pend_first && pend_n > 0) ok = wait_or_abort(&sh->o_free, (pend_n - 1u) & 1u, abort_flag, err);
+        if (ok && pend_first && pend_n > 0) wait(&sh->o_free, (pend_n - 1u) & 1u);
         if (!ok) return;
         tc_fence_after_sync();
         // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
@@ -348,24 +392,31 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         // Slots 0, 1, 4, 5 (chunks 0 and 2) belong to softmax group 0 and add to O_0, the others to
         // O_1; a group's first step of an item overwrites its accumulator.
         if (pend_first) started0 = started1 = 0u;
-#pragma unroll 1
-        for (int ks = 0; ks < pend_ng; ++ks) {
-          const int grp = (ks >> 1) & 1;
-          const uint64_t db =
-              smem_desc_sw128(smem_u32(v_s + st * C::kTileBytes + ks * C::kSlotStride), C::kHalfStride, C::kSbo);
-          mma_ts(tmem_o + 128u * grp, tmem + 128u * sb + 32 * (ks >> 1) + 8 * (ks & 1), db, idesc_pv,
-                 grp ? started1 : started0);
-          if (grp) started1 = 1u; else started0 = 1u;
+        if (elect_one()) {
+          const uint32_t v_stage = v_addr + st * C::kTileBytes;
+          const uint32_t p_base = tmem + 128u * sb;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            if (ks < pend_ng) {
+              const int grp = (ks >> 1) & 1;
+              const uint32_t acc = ks == 0 ? started0 : ks == 2 ? started1 : 1u;  // slots 0 / 2 open their group
+              mma_ts(tmem_o + 128u * grp, p_base + 32 * (ks >> 1) + 8 * (ks & 1),
+                     smem_desc_sw128(v_stage + ks * C::kSlotStride, C::kHalfStride, C::kSbo), idesc_pv, acc);
+            }
+          }
+          mma_commit(&sh->v_empty[st]);
+          mma_commit(&sh->pv_done);
+          if (pend_last) mma_commit(&sh->o_done);
         }
-        mma_commit(&sh->v_empty[st]);
-        mma_commit(&sh->pv_done);
-        if (pend_last) mma_commit(&sh->o_done);
+        __syncwarp();
+        started0 = 1u;
+        if (pend_ng > 2) started1 = 1u;
         pending = false;
       };
       for (uint32_t g = 0; ok; ++g) {
         const int st = (int)(g % C::kStages);
         const uint32_t sb = g & 1u;
-        ok = wait_or_abort(&sh->k_full[st], (g / C::kStages) & 1u, abort_flag, err);
+        wait(&sh->k_full[st], (g / C::kStages) & 1u);
         if (!ok) break;
         const uint32_t info = sh->info[g % kMaxStages];
         if (info & kInfoStop) break;
@@ -377,24 +428,26 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
           // item's Q
           if (pending) issue_pv();
           if (!ok) break;
-          ok = wait_or_abort(&sh->q_full[qb], (n >> 1) & 1u, abort_flag, err);
+          wait(&sh->q_full[qb], (n >> 1) & 1u);
           if (!ok) break;
         }
         tc_fence_after_sync();
         // S[sb] = Q K_round^T: N = 16 ng, D/16 steps of K = 16 (32 bytes inside the swizzled rows).
         // S[sb] last held P of round g - 2, whose O += P V was issued before this.
-        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false);
-#pragma unroll 1
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const int sub = ks / 4, off = (ks % 4) * 32;
-          const uint64_t da = smem_desc_sw128(smem_u32(q_s + qb * C::kTileBytes + sub * kSubBytes + off), 16, 1024);
-          const uint64_t db =
-              smem_desc_sw128(smem_u32(k_s + st * C::kTileBytes + sub * C::kHalfStride + off), 16, C::kSbo);
-          mma_ss(tmem + 128u * sb, da, db, idesc_qk, ks > 0);
+        if (elect_one()) {
+          const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false);
+          const uint32_t q_buf = q_addr + qb * C::kTileBytes, k_stage = k_addr + st * C::kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const int sub = ks / 4, off = (ks % 4) * 32;
+            mma_ss(tmem + 128u * sb, smem_desc_sw128(q_buf + sub * kSubBytes + off, 16, 1024),
+                   smem_desc_sw128(k_stage + sub * C::kHalfStride + off, 16, C::kSbo), idesc_qk, ks > 0);
+          }
+          mma_commit(&sh->k_empty[st]);
+          if (last) mma_commit(&sh->q_empty[qb]);
+          mma_commit(&sh->s_full[sb]);
         }
-        mma_commit(&sh->k_empty[st]);
-        if (last) mma_commit(&sh->q_empty[qb]);
-        mma_commit(&sh->s_full[sb]);
+        __syncwarp();
         if (pending) issue_pv();
         if (!ok) break;
         pending = true;
@@ -424,7 +477,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       const int st = (int)(g % kMaxStages);  // info / bitmap slot of the round
       const uint32_t sb = g & 1u;
       const uint32_t tmem_s = tmem + 128u * sb;
-      ok = wait_or_abort(&sh->b_full[st], (g / kMaxStages) & 1u, abort_flag, err);
+      ok = warp_wait(&sh->b_full[st], (g / kMaxStages) & 1u, lane, abort_flag, err);
       if (!ok) break;
       const uint32_t info = sh->info[st];
       if (info & kInfoStop) break;
@@ -432,9 +485,9 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
       const bool tile_full = (info & kInfoFull) != 0u;
       if (first) {
-        const int item = sh->item[st];
-        const int bh = (item % B) * H + (item / B) % H;
-        i = (n_qt - 1 - item / (B * H)) * kTile + r;
+        const int item = sh->item[st];  // (b * H + h) * n_qt + qt
+        const int bh = item / n_qt;
+        i = (item % n_qt) * kTile + r;
         orow = O + ((size_t)bh * Lq + i) * D;
         m = -CUDART_INF_F;
         l = 0.f;
@@ -453,10 +506,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       // chunks in which none of this warp's 32 rows keeps anything are skipped (their P is
       // written as zeros without reading S)
       const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u);
-      if (!mbar_try_wait(&sh->s_full[sb], (g >> 1) & 1u)) {
-        ok = wait_or_abort(&sh->s_full[sb], (g >> 1) & 1u, abort_flag, err);
-        if (!ok) break;
-      }
+      ok = warp_wait(&sh->s_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
+      if (!ok) break;
       tc_fence_after_sync();
       // pass 1: row maximum over kept entries (four independent chains).  In a partially filled
       // round the pruned entries are replaced by -inf and the chunk is written back to TMEM, so
@@ -499,7 +550,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       // Rescale the group's running output where the reference moved.  O += P V of the previous
       // round may still be running (this round's S was computed ahead of it): wait for it first.
       if (o_started && __any_sync(0xffffffffu, alpha != 1.f)) {
-        ok = wait_or_abort(&sh->pv_done, (g - 1u) & 1u, abort_flag, err);
+        ok = warp_wait(&sh->pv_done, (g - 1u) & 1u, lane, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll 1
@@ -551,8 +602,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       // the two accumulators and writes O / l, rounded once to bf16.
       sh->ml[n & 1u][grp][r] = make_float2(m, l);
       mbar_arrive(&sh->ml_ready);
-      ok = wait_or_abort(&sh->ml_ready, n & 1u, abort_flag, err);
-      if (ok) ok = wait_or_abort(&sh->o_done, n & 1u, abort_flag, err);
+      ok = warp_wait(&sh->ml_ready, n & 1u, lane, abort_flag, err);
+      if (ok) ok = warp_wait(&sh->o_done, n & 1u, lane, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
       const float2 other = sh->ml[n & 1u][grp ^ 1][r];
@@ -626,11 +677,11 @@ cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
-  const int n_items = B * H * t.n_qt;
+  const int n_units = B * H * ((t.n_qt + 1) / 2);  // pairs of query tiles, see the producer
   const float scale_log2 = scale * 1.4426950408889634f;
-  kern<<<n_items < sms ? n_items : sms, kThreads, C::kSmemBytes, s>>>(
+  kern<<<n_units < sms ? n_units : sms, kThreads, C::kSmemBytes, s>>>(
       maps, static_cast<__nv_bfloat16 *>(O), t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, B, H, Lq,
-      t.n_qt, n_items, scale_log2, err);
+      t.n_qt, scale_log2, err);
   count_launches(1);
   return cudaGetLastError();
 }
