@@ -124,11 +124,12 @@ __device__ __noinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volat
 
 // The same wait for a whole (converged) warp: one lane polls - 32 lanes polling one barrier would
 // serialise - and the outcome is shared.
+template <int kPollLane = 0>
 __device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag,
                                           unsigned *err) {
   bool ok = true;
-  if (lane == 0 && !mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, abort_flag, err);
-  return __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+  if (lane == kPollLane && !mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, abort_flag, err);
+  return __shfl_sync(0xffffffffu, ok ? 1 : 0, kPollLane) != 0;
 }
 
 template <int D, bool kSplit>
@@ -376,7 +377,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       int pend_ng = 0;
       bool pend_first = false, pend_last = false;
       uint32_t started0 = 0u, started1 = 0u;  // the item's O_0 / O_1 holds a partial result already
-      auto wait = [&](uint64_t *bar, uint32_t parity) { ok = warp_wait(bar, parity, lane, abort_flag, err); };
+      // (the polling lane is not the lane that issues the MMAs and commits)
+      auto wait = [&](uint64_t *bar, uint32_t parity) { ok = warp_wait<31>(bar, parity, lane, abort_flag, err); };
       auto issue_pv = [&]() {
         const uint32_t sb = pend_g & 1u;
         const int st = (int)(pend_g % C::kStages);
