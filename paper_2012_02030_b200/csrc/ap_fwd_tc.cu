@@ -21,8 +21,10 @@
 // rows follow one another are copied as one box), the round's bitmap (one bulk copy) and a word
 // that says how many slots there are and whether the round starts or ends an item.  The producer
 // runs ahead across item boundaries, so an item's first loads are hidden behind the previous
-// item's last rounds.  S is double-buffered in TMEM and the MMA thread issues S(g+1) = Q K^T
-// before O += P(g) V, so the softmax threads find the next S ready when they finish a round.
+// item's last rounds.  S is double-buffered in TMEM and the two kinds of MMA are issued by two
+// warps, each held back only by what it really depends on: S(g) = Q K^T waits for K(g) and for
+// O += P V of round g - 2 (the previous user of that S buffer), O += P(g) V for P(g) and V(g).
+// So the softmax threads find the next S ready when they finish a round.
 //
 //
 // The softmax is shared by two groups of four warps.  The 32-column chunks of a round alternate
@@ -32,9 +34,9 @@
 // inside a round.  The item's epilogue merges the two partial results
 //   O = (a_0 O_0 + a_1 O_1) / (a_0 l_0 + a_1 l_1),   a_i = exp2(c (m_i - max(m_0, m_1))).
 //
-// Warp roles (320 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
-// TMEM lane), warp 8 producer, warp 9 MMA issuer and TMEM owner.  TMEM (512 columns): S[0] at
-// column 0, S[1] at 128, O_0 at 256, O_1 at 384.  Every wait is bounded; a wait that expires
+// Warp roles (352 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
+// TMEM lane), warp 8 producer, warp 9 issuer of S = Q K^T and TMEM owner, warp 10 issuer of
+// O += P V.  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384.  Every wait is bounded; a wait that expires
 // raises the device status word and the CTA winds down.
 #include <math_constants.h>
 
@@ -47,7 +49,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;
 constexpr int kSoftmaxThreads = 256;   // two groups of 128
 constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-tile
 constexpr uint32_t kTmemCols = 512;
@@ -94,7 +96,7 @@ struct Shared {
   uint64_t b_full[kMaxStages];                        // info word and bitmap of the stage are valid
   uint64_t k_empty[kMaxStages], v_empty[kMaxStages];  // S = Q K^T / O += P V of the stage has completed
   uint64_t s_full[2], p_full[2];                      // per S buffer
-  uint64_t pv_done;                                   // O += P V of a round has completed
+  uint64_t pv_done[2];                                // O += P V of a round has completed, per S buffer
   uint64_t o_done, o_free;                            // per item: O complete / O read out by the epilogue
   uint64_t ml_ready;                                  // per item: both groups have published (m, l)
   float2 ml[2][2][kTile];                             // [item parity][group][row] = (m, l)
@@ -162,7 +164,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       mbar_init(&sh->v_empty[s], 1);
     }
     for (int s = 0; s < kMaxStages; ++s) mbar_init(&sh->b_full[s], 1);
-    mbar_init(&sh->pv_done, 1);
+    mbar_init(&sh->pv_done[0], 1);
+    mbar_init(&sh->pv_done[1], 1);
     mbar_init(&sh->o_done, 1);
     mbar_init(&sh->o_free, kSoftmaxThreads);
     mbar_init(&sh->ml_ready, kSoftmaxThreads);
@@ -363,104 +366,93 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       }
     }
   } else if (warp == 9) {
-    // ------------------------------------------------------------ MMA issuer
-    // The whole warp walks the rounds in lockstep (every lane waits on the barriers and keeps the
-    // same, warp-uniform state); one elected lane issues the tcgen05 instructions.
-    {
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
-      const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s), v_addr = smem_u32(v_s);
-      bool ok = true;
-      uint32_t n = 0;  // non-empty items started so far
-      // O += P V of the round before the current one is issued after the current S = Q K^T
-      bool pending = false;
-      uint32_t pend_g = 0, pend_n = 0;
-      int pend_ng = 0;
-      bool pend_first = false, pend_last = false;
-      uint32_t started0 = 0u, started1 = 0u;  // the item's O_0 / O_1 holds a partial result already
-      // (the polling lane is not the lane that issues the MMAs and commits)
-      auto wait = [&](uint64_t *bar, uint32_t parity) { ok = warp_wait<31>(bar, parity, lane, abort_flag, err); };
-      auto issue_pv = [&]() {
-        const uint32_t sb = pend_g & 1u;
-        const int st = (int)(pend_g % C::kStages);
-        wait(&sh->p_full[sb], (pend_g >> 1) & 1u);
-        if (ok) wait(&sh->v_full[st], (pend_g / C::kStages) & 1u);
-        // the first round of an item overwrites O: the epilogue of the previous item must have read it
-        if (ok && pend_first && pend_n > 0) wait(&sh->o_free, (pend_n - 1u) & 1u);
-        if (!ok) return;
-        tc_fence_after_sync();
-        // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
-        // 16 columns of that chunk of S (each group stays inside its own chunks), so slot q's
-        // eight columns of P start at column 32 (q / 2) + 8 (q % 2).
-        // Slots 0, 1, 4, 5 (chunks 0 and 2) belong to softmax group 0 and add to O_0, the others to
-        // O_1; a group's first step of an item overwrites its accumulator.
-        if (pend_first) started0 = started1 = 0u;
-        if (elect_one()) {
-          const uint32_t v_stage = v_addr + st * C::kTileBytes;
-          const uint32_t p_base = tmem + 128u * sb;
+    // ------------------------------------------------------------ issuer of S = Q K^T
+    // The whole warp walks the rounds in lockstep (one lane polls the barriers, another, elected
+    // one issues the tcgen05 instructions; the state is warp-uniform).
+    const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s);
+    bool ok = true;
+    uint32_t n = 0;  // non-empty items started so far
+    for (uint32_t g = 0; ok; ++g) {
+      const int st = (int)(g % C::kStages);
+      const uint32_t sb = g & 1u;
+      ok = warp_wait<31>(&sh->k_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
+      if (!ok) break;
+      const uint32_t info = sh->info[g % kMaxStages];
+      if (info & kInfoStop) break;
+      const int ng = (int)(info & kInfoSlots);
+      const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
+      const int qb = (int)(n & 1u);
+      if (first) ok = warp_wait<31>(&sh->q_full[qb], (n >> 1) & 1u, lane, abort_flag, err);
+      // S[sb] still holds P of round g - 2 until that round's O += P V (issued by another warp) has
+      // completed
+      if (ok && g >= 2) ok = warp_wait<31>(&sh->pv_done[sb], ((g >> 1) - 1u) & 1u, lane, abort_flag, err);
+      if (!ok) break;
+      tc_fence_after_sync();
+      // N = 16 ng, D/16 steps of K = 16 (32 bytes inside the swizzled rows)
+      if (elect_one()) {
+        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false);
+        const uint32_t q_buf = q_addr + qb * C::kTileBytes, k_stage = k_addr + st * C::kTileBytes;
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            if (ks < pend_ng) {
-              const int grp = (ks >> 1) & 1;
-              const uint32_t acc = ks == 0 ? started0 : ks == 2 ? started1 : 1u;  // slots 0 / 2 open their group
-              mma_ts(tmem_o + 128u * grp, p_base + 32 * (ks >> 1) + 8 * (ks & 1),
-                     smem_desc_sw128(v_stage + ks * C::kSlotStride, C::kHalfStride, C::kSbo), idesc_pv, acc);
-            }
-          }
-          mma_commit(&sh->v_empty[st]);
-          mma_commit(&sh->pv_done);
-          if (pend_last) mma_commit(&sh->o_done);
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const int sub = ks / 4, off = (ks % 4) * 32;
+          mma_ss(tmem + 128u * sb, smem_desc_sw128(q_buf + sub * kSubBytes + off, 16, 1024),
+                 smem_desc_sw128(k_stage + sub * C::kHalfStride + off, 16, C::kSbo), idesc_qk, ks > 0);
         }
-        __syncwarp();
-        started0 = 1u;
-        if (pend_ng > 2) started1 = 1u;
-        pending = false;
-      };
-      for (uint32_t g = 0; ok; ++g) {
-        const int st = (int)(g % C::kStages);
-        const uint32_t sb = g & 1u;
-        wait(&sh->k_full[st], (g / C::kStages) & 1u);
-        if (!ok) break;
-        const uint32_t info = sh->info[g % kMaxStages];
-        if (info & kInfoStop) break;
-        const int ng = (int)(info & kInfoSlots);
-        const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
-        const int qb = (int)(n & 1u);
-        if (first) {
-          // the previous item's last O += P V goes first: its epilogue should not wait for this
-          // item's Q
-          if (pending) issue_pv();
-          if (!ok) break;
-          wait(&sh->q_full[qb], (n >> 1) & 1u);
-          if (!ok) break;
-        }
-        tc_fence_after_sync();
-        // S[sb] = Q K_round^T: N = 16 ng, D/16 steps of K = 16 (32 bytes inside the swizzled rows).
-        // S[sb] last held P of round g - 2, whose O += P V was issued before this.
-        if (elect_one()) {
-          const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false);
-          const uint32_t q_buf = q_addr + qb * C::kTileBytes, k_stage = k_addr + st * C::kTileBytes;
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const int sub = ks / 4, off = (ks % 4) * 32;
-            mma_ss(tmem + 128u * sb, smem_desc_sw128(q_buf + sub * kSubBytes + off, 16, 1024),
-                   smem_desc_sw128(k_stage + sub * C::kHalfStride + off, 16, C::kSbo), idesc_qk, ks > 0);
-          }
-          mma_commit(&sh->k_empty[st]);
-          if (last) mma_commit(&sh->q_empty[qb]);
-          mma_commit(&sh->s_full[sb]);
-        }
-        __syncwarp();
-        if (pending) issue_pv();
-        if (!ok) break;
-        pending = true;
-        pend_g = g;
-        pend_n = n;
-        pend_ng = ng;
-        pend_first = first;
-        pend_last = last;
-        if (last) ++n;
+        mma_commit(&sh->k_empty[st]);
+        if (last) mma_commit(&sh->q_empty[qb]);
+        mma_commit(&sh->s_full[sb]);
       }
-      if (ok && pending) issue_pv();
+      __syncwarp();
+      if (last) ++n;
+    }
+  } else if (warp == 10) {
+    // ------------------------------------------------------------ issuer of O += P V
+    constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
+    const uint32_t v_addr = smem_u32(v_s);
+    bool ok = true;
+    uint32_t n = 0;                          // non-empty items started so far
+    uint32_t started0 = 0u, started1 = 0u;  // the item's O_0 / O_1 holds a partial result already
+    for (uint32_t g = 0; ok; ++g) {
+      const int st = (int)(g % C::kStages);
+      const uint32_t sb = g & 1u;
+      ok = warp_wait<31>(&sh->b_full[g % kMaxStages], (g / kMaxStages) & 1u, lane, abort_flag, err);
+      if (!ok) break;
+      const uint32_t info = sh->info[g % kMaxStages];
+      if (info & kInfoStop) break;
+      const int ng = (int)(info & kInfoSlots);
+      const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
+      ok = warp_wait<31>(&sh->p_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
+      if (ok) ok = warp_wait<31>(&sh->v_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
+      // the first round of an item overwrites O: the epilogue of the previous item must have read it
+      if (ok && first && n > 0) ok = warp_wait<31>(&sh->o_free, (n - 1u) & 1u, lane, abort_flag, err);
+      if (!ok) break;
+      tc_fence_after_sync();
+      // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
+      // 16 columns of that chunk of S (each group stays inside its own chunks), so slot q's
+      // eight columns of P start at column 32 (q / 2) + 8 (q % 2).
+      // Slots 0, 1, 4, 5 (chunks 0 and 2) belong to softmax group 0 and add to O_0, the others to
+      // O_1; a group's first step of an item overwrites its accumulator.
+      if (first) started0 = started1 = 0u;
+      if (elect_one()) {
+        const uint32_t v_stage = v_addr + st * C::kTileBytes;
+        const uint32_t p_base = tmem + 128u * sb;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          if (ks < ng) {
+            const int grp = (ks >> 1) & 1;
+            const uint32_t acc = ks == 0 ? started0 : ks == 2 ? started1 : 1u;  // slots 0 / 2 open their group
+            mma_ts(tmem_o + 128u * grp, p_base + 32 * (ks >> 1) + 8 * (ks & 1),
+                   smem_desc_sw128(v_stage + ks * C::kSlotStride, C::kHalfStride, C::kSbo), idesc_pv, acc);
+          }
+        }
+        mma_commit(&sh->v_empty[st]);
+        mma_commit(&sh->pv_done[sb]);
+        if (last) mma_commit(&sh->o_done);
+      }
+      __syncwarp();
+      started0 = 1u;
+      if (ng > 2) started1 = 1u;
+      if (last) ++n;
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue
@@ -552,7 +544,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       // Rescale the group's running output where the reference moved.  O += P V of the previous
       // round may still be running (this round's S was computed ahead of it): wait for it first.
       if (o_started && __any_sync(0xffffffffu, alpha != 1.f)) {
-        ok = warp_wait(&sh->pv_done, (g - 1u) & 1u, lane, abort_flag, err);
+        ok = warp_wait(&sh->pv_done[(g - 1u) & 1u], ((g - 1u) >> 1) & 1u, lane, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll 1
