@@ -34,9 +34,10 @@
 // inside a round.  The item's epilogue merges the two partial results
 //   O = (a_0 O_0 + a_1 O_1) / (a_0 l_0 + a_1 l_1),   a_i = exp2(c (m_i - max(m_0, m_1))).
 //
-// Warp roles (352 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
+// Warp roles (480 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
 // TMEM lane), warp 8 producer, warp 9 issuer of S = Q K^T and TMEM owner, warp 10 issuer of
-// O += P V.  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384.  Every wait is bounded; a wait that expires
+// O += P V, warps 11-14 epilogue (the softmax groups hand (m, l) over and go on with the next
+// item while the epilogue warps wait for the item's last O += P V, merge and write).  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384.  Every wait is bounded; a wait that expires
 // raises the device status word and the CTA winds down.
 #include <math_constants.h>
 
@@ -49,7 +50,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 352;
+constexpr int kThreads = 480;
 constexpr int kSoftmaxThreads = 256;   // two groups of 128
 constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-tile
 constexpr uint32_t kTmemCols = 512;
@@ -76,7 +77,7 @@ struct Cfg {
   static constexpr int kKOffset = 2 * kTileBytes;     // after the two Q buffers
   static constexpr int kVOffset = kKOffset + kStages * kTileBytes;
   static constexpr int kBarOffset = kVOffset + kStages * kTileBytes;
-  static constexpr int kSmemBytes = kBarOffset + 13 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
+  static constexpr int kSmemBytes = kBarOffset + 17 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
   static constexpr int kHalfStride = kSplit ? 1024 : kSubBytes;          // half 0 -> half 1 of the same rows
   static constexpr int kSbo = kSplit ? 2048 : 1024;                      // one group of 8 rows -> the next
   static constexpr int kSlotStride = 2 * kSbo;                           // 16 rows (one slot) -> the next
@@ -98,8 +99,9 @@ struct Shared {
   uint64_t s_full[2], p_full[2];                      // per S buffer
   uint64_t pv_done[2];                                // O += P V of a round has completed, per S buffer
   uint64_t o_done, o_free;                            // per item: O complete / O read out by the epilogue
-  uint64_t ml_ready;                                  // per item: both groups have published (m, l)
-  float2 ml[2][2][kTile];                             // [item parity][group][row] = (m, l)
+  uint64_t ml_ready[4];                               // per item: both groups have handed over (m, l)
+  float2 ml[4][2][kTile];                             // [item % 4][group][row] = (m, l)
+  int32_t ml_item[4];                                 // the item handed over, -1: no more items
   uint32_t info[kMaxStages];
   int32_t item[kMaxStages];                           // the item a stage's round belongs to
   uint32_t tmem_base;
@@ -167,8 +169,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     mbar_init(&sh->pv_done[0], 1);
     mbar_init(&sh->pv_done[1], 1);
     mbar_init(&sh->o_done, 1);
-    mbar_init(&sh->o_free, kSoftmaxThreads);
-    mbar_init(&sh->ml_ready, kSoftmaxThreads);
+    mbar_init(&sh->o_free, 128);
+    for (int i = 0; i < 4; ++i) mbar_init(&sh->ml_ready[i], kSoftmaxThreads);
     sh->abort_flag = 0;
     fence_mbar_init();
   }
@@ -270,6 +272,9 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     };
     // the rounds of an item are looked up one item ahead
     ItemRef next = item_ref(0);
+    // ... and the slot rows and info byte of its first round while the current item is under way
+    int pf_t = -1, pf_row = -1;
+    uint32_t pf_info = 0u;
     for (int t = 0; next.in_range && ok; ++t) {
       const ItemRef cur = next;
       next = item_ref(t + 1);
@@ -297,14 +302,22 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       // slot rows (lanes 0..7) and info byte of a round are fetched one round ahead
-      int next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)rho0 * 8 + lane) : -1;
-      uint32_t next_info = ldg_now_u8(round_info + rho0);
+      int next_row = pf_row;
+      uint32_t next_info = pf_info;
+      if (pf_t != t) {
+        next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)rho0 * 8 + lane) : -1;
+        next_info = ldg_now_u8(round_info + rho0);
+      }
       for (int v = 0; v < n_rounds && ok; ++v, ++g) {
         const int row = next_row;
         const uint32_t rinfo = next_info;
         if (v + 1 < n_rounds) {
           next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)(rho0 + v + 1) * 8 + lane) : -1;
           next_info = ldg_now_u8(round_info + rho0 + v + 1);
+        } else if (next.n_rounds > 0) {
+          pf_t = t + 1;
+          pf_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)next.rho0 * 8 + lane) : -1;
+          pf_info = ldg_now_u8(round_info + next.rho0);
         }
         const int st = (int)(g % C::kStages);
         const uint32_t ph = (g / C::kStages) & 1u;
@@ -454,8 +467,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       if (ng > 2) started1 = 1u;
       if (last) ++n;
     }
-  } else {
-    // ------------------------------------------------------------ softmax + epilogue
+  } else if (warp < 8) {
+    // ------------------------------------------------------------ softmax
     const int grp = warp >> 2;               // softmax group: chunks grp and grp + 2 of every round
     const int r = (warp & 3) * 32 + lane;    // row of the query tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -465,8 +478,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     uint32_t n = 0;
     float m = -CUDART_INF_F, l = 0.f;       // this group's exponent reference and running sum of weights
     bool o_started = false;                  // an earlier round of the item added to this group's accumulator
-    int i = 0;                               // this thread's query row in the tensor
-    __nv_bfloat16 *orow = O;
+    int cur_item = 0;
     for (uint32_t g = 0; ok; ++g) {
       const int st = (int)(g % kMaxStages);  // info / bitmap slot of the round
       const uint32_t sb = g & 1u;
@@ -479,10 +491,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
       const bool tile_full = (info & kInfoFull) != 0u;
       if (first) {
-        const int item = sh->item[st];  // (b * H + h) * n_qt + qt
-        const int bh = item / n_qt;
-        i = (item % n_qt) * kTile + r;
-        orow = O + ((size_t)bh * Lq + i) * D;
+        cur_item = sh->item[st];  // (b * H + h) * n_qt + qt
         m = -CUDART_INF_F;
         l = 0.f;
         o_started = false;
@@ -592,32 +601,51 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       tc_fence_before_sync();
       mbar_arrive(&sh->p_full[sb]);
       if (!last) continue;
-      // Epilogue.  The groups exchange (m, l), then each takes half of the output columns, merges
-      // the two accumulators and writes O / l, rounded once to bf16.
-      sh->ml[n & 1u][grp][r] = make_float2(m, l);
-      mbar_arrive(&sh->ml_ready);
-      ok = warp_wait(&sh->ml_ready, n & 1u, lane, abort_flag, err);
-      if (ok) ok = warp_wait(&sh->o_done, n & 1u, lane, abort_flag, err);
+      // The item's rounds are over for this group: it hands (m, l) to the epilogue warps and goes on
+      // with the next item; the slot of the hand-over ring was read by the epilogue of item n - 4,
+      // which is over (this item's S needed O += P V of item n - 2, that the epilogue of item n - 3).
+      sh->ml[n & 3u][grp][r] = make_float2(m, l);
+      if (threadIdx.x == 0) sh->ml_item[n & 3u] = cur_item;
+      mbar_arrive(&sh->ml_ready[n & 3u]);
+      ++n;
+    }
+    // no more items: tell the epilogue warps
+    if (ok) {
+      if (threadIdx.x == 0) sh->ml_item[n & 3u] = -1;
+      mbar_arrive(&sh->ml_ready[n & 3u]);
+    }
+  } else if (warp >= 11) {
+    // ------------------------------------------------------------ epilogue
+    // Per item: merge the two groups' accumulators and write O / l, rounded once to bf16.
+    const int r = (warp & 3) * 32 + lane;    // row of the query tile == TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    bool ok = true;
+    for (uint32_t n = 0; ok; ++n) {
+      ok = warp_wait(&sh->ml_ready[n & 3u], (n >> 2) & 1u, lane, abort_flag, err);
       if (!ok) break;
-      tc_fence_after_sync();
-      const float2 other = sh->ml[n & 1u][grp ^ 1][r];
-      const float m_tot = fmaxf(m, other.x);
+      const int item = sh->ml_item[n & 3u];  // (b * H + h) * n_qt + qt
+      if (item < 0) break;
+      const float2 g0 = sh->ml[n & 3u][0][r], g1 = sh->ml[n & 3u][1][r];
+      const int i = (item % n_qt) * kTile + r;
+      __nv_bfloat16 *orow = O + ((size_t)(item / n_qt) * Lq + i) * D;
+      const float m_tot = fmaxf(g0.x, g1.x);
       // weight of a partial result; 0 for a group that saw no kept entry of this row (m = -inf),
       // whose accumulator is then never read into the sum (it may hold a previous item's data)
-      const float a_mine = m == -CUDART_INF_F ? 0.f : ex2_approx((m - m_tot) * scale_log2);
-      const float a_other = other.x == -CUDART_INF_F ? 0.f : ex2_approx((other.x - m_tot) * scale_log2);
-      const float l_tot = l * a_mine + other.y * a_other;
+      const float a0 = g0.x == -CUDART_INF_F ? 0.f : ex2_approx((g0.x - m_tot) * scale_log2);
+      const float a1 = g1.x == -CUDART_INF_F ? 0.f : ex2_approx((g1.x - m_tot) * scale_log2);
+      const float l_tot = g0.y * a0 + g1.y * a1;
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      const float f0 = (grp == 0 ? a_mine : a_other) * inv, f1 = (grp == 0 ? a_other : a_mine) * inv;
-      constexpr int kHalf = D / 2;  // output columns per group
+      const float f0 = a0 * inv, f1 = a1 * inv;
+      ok = warp_wait(&sh->o_done, n & 1u, lane, abort_flag, err);
+      if (!ok) break;
+      tc_fence_after_sync();
 #pragma unroll 1
-      for (int c = 0; c < kHalf / 32; ++c) {
-        const int col = grp * kHalf + 32 * c;
+      for (int c = 0; c < D / 32; ++c) {
         uint32_t o0[32], o1[32];
-        tmem_ld32(tmem_o + lane_addr + col, o0);
-        tmem_ld32(tmem_o + 128u + lane_addr + col, o1);
+        tmem_ld32(tmem_o + lane_addr + 32 * c, o0);
+        tmem_ld32(tmem_o + 128u + lane_addr + 32 * c, o1);
         tmem_wait_ld();
-        if (c == kHalf / 32 - 1) {  // this thread's share of O is in registers: the next item may overwrite it
+        if (c == D / 32 - 1) {  // this thread's rows of O are in registers: the next item may overwrite them
           tc_fence_before_sync();
           mbar_arrive(&sh->o_free);
         }
@@ -635,11 +663,10 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
               __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
               pk[e] = *reinterpret_cast<uint32_t *>(&hh);
             }
-            *reinterpret_cast<uint4 *>(orow + col + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4 *>(orow + 32 * c + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
       }
-      ++n;
     }
   }
   tc_fence_before_sync();
@@ -663,7 +690,7 @@ template <int D, bool kSplit>
 cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
                    unsigned *err, cudaStream_t s) {
   using C = Cfg<D, kSplit>;
-  static_assert(sizeof(Shared) <= 13 * 1024, "shared bookkeeping outgrew its reservation");
+  static_assert(sizeof(Shared) <= 17 * 1024, "shared bookkeeping outgrew its reservation");
   static_assert(C::kStages <= kMaxStages, "ring deeper than its barriers");
   static_assert(C::kSmemBytes > 114 * 1024 && C::kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
   auto kern = fwd_tc_kernel<D, kSplit>;
