@@ -51,7 +51,7 @@ namespace {
 using namespace sm100;
 
 constexpr int kThreads = 480;
-constexpr int kSoftmaxThreads = 256;   // two groups of 128
+constexpr int kSoftmaxWarps = 8;       // two groups of four; barriers the softmax warps arrive on count warps
 constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-tile
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kMaxPolls = 1u << 22;
@@ -157,7 +157,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       mbar_init(&sh->q_full[i], 1);
       mbar_init(&sh->q_empty[i], 1);
       mbar_init(&sh->s_full[i], 1);
-      mbar_init(&sh->p_full[i], kSoftmaxThreads);
+      mbar_init(&sh->p_full[i], kSoftmaxWarps);
     }
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&sh->k_full[s], 1);
@@ -169,8 +169,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     mbar_init(&sh->pv_done[0], 1);
     mbar_init(&sh->pv_done[1], 1);
     mbar_init(&sh->o_done, 1);
-    mbar_init(&sh->o_free, 128);
-    for (int i = 0; i < 4; ++i) mbar_init(&sh->ml_ready[i], kSoftmaxThreads);
+    mbar_init(&sh->o_free, 4);  // epilogue warps
+    for (int i = 0; i < 4; ++i) mbar_init(&sh->ml_ready[i], kSoftmaxWarps);
     sh->abort_flag = 0;
     fence_mbar_init();
   }
@@ -434,10 +434,11 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       if (info & kInfoStop) break;
       const int ng = (int)(info & kInfoSlots);
       const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
-      ok = warp_wait<31>(&sh->p_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
-      if (ok) ok = warp_wait<31>(&sh->v_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
+      // (what is ready early first; P, which the softmax has just finished, last)
+      ok = warp_wait<31>(&sh->v_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
       // the first round of an item overwrites O: the epilogue of the previous item must have read it
       if (ok && first && n > 0) ok = warp_wait<31>(&sh->o_free, (n - 1u) & 1u, lane, abort_flag, err);
+      if (ok) ok = warp_wait<31>(&sh->p_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
       // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
@@ -598,21 +599,25 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       o_started = true;
       tmem_wait_st();
       }  // n_mine > 0
+      // one arrival per warp (32 lanes arriving one by one would take hundreds of cycles)
       tc_fence_before_sync();
-      mbar_arrive(&sh->p_full[sb]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->p_full[sb]);
       if (!last) continue;
       // The item's rounds are over for this group: it hands (m, l) to the epilogue warps and goes on
       // with the next item; the slot of the hand-over ring was read by the epilogue of item n - 4,
       // which is over (this item's S needed O += P V of item n - 2, that the epilogue of item n - 3).
       sh->ml[n & 3u][grp][r] = make_float2(m, l);
       if (threadIdx.x == 0) sh->ml_item[n & 3u] = cur_item;
-      mbar_arrive(&sh->ml_ready[n & 3u]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->ml_ready[n & 3u]);
       ++n;
     }
     // no more items: tell the epilogue warps
     if (ok) {
       if (threadIdx.x == 0) sh->ml_item[n & 3u] = -1;
-      mbar_arrive(&sh->ml_ready[n & 3u]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->ml_ready[n & 3u]);
     }
   } else if (warp >= 11) {
     // ------------------------------------------------------------ epilogue
@@ -647,7 +652,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
         tmem_wait_ld();
         if (c == D / 32 - 1) {  // this thread's rows of O are in registers: the next item may overwrite them
           tc_fence_before_sync();
-          mbar_arrive(&sh->o_free);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh->o_free);
         }
         if (i < Lq) {
 #pragma unroll
