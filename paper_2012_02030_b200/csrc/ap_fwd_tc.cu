@@ -513,34 +513,44 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       ok = warp_wait(&sh->s_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
-      // pass 1: row maximum over kept entries (four independent chains).  In a partially filled
-      // round the pruned entries are replaced by -inf and the chunk is written back to TMEM, so
-      // that pass 2 needs no bitmap: exp2 of -inf is exactly 0.
+      // pass 1: the group's (up to) two chunks of S come into registers and stay there; pruned
+      // entries are replaced by -inf (exp2 of -inf is exactly 0); row maximum over kept entries
+      // (four independent chains)
+      uint32_t xa[32], xb[32];
+      const bool act0 = (active & 1u) != 0u, act1 = n_mine > 1 && (active & 2u) != 0u;
+      if (act0) tmem_ld32(tmem_s + lane_addr + 32 * grp, xa);
+      if (act1) tmem_ld32(tmem_s + lane_addr + 32 * (grp + 2), xb);
+      tmem_wait_ld();
       float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
-#pragma unroll 1
-      for (int cc = 0; cc < n_mine; ++cc) {
-        if (!((active >> cc) & 1u)) continue;
-        const int c = grp + 2 * cc;
-        uint32_t x[32];
-        tmem_ld32(tmem_s + lane_addr + 32 * c, x);
-        tmem_wait_ld();
+      if (act0) {
         if (!tile_full) {
-          const uint32_t w = cc == 0 ? w0 : w1;
 #pragma unroll
           for (int e = 0; e < 32; ++e)
-            if (!((w >> e) & 1u)) x[e] = 0xff800000u;  // -inf
-          tmem_st32(tmem_s + lane_addr + 32 * c, x);
+            if (!((w0 >> e) & 1u)) xa[e] = 0xff800000u;  // -inf
         }
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(x[e]));
-          mx1 = fmaxf(mx1, __uint_as_float(x[e + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(x[e + 2]));
-          mx3 = fmaxf(mx3, __uint_as_float(x[e + 3]));
+          mx0 = fmaxf(mx0, __uint_as_float(xa[e]));
+          mx1 = fmaxf(mx1, __uint_as_float(xa[e + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(xa[e + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(xa[e + 3]));
+        }
+      }
+      if (act1) {
+        if (!tile_full) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (!((w1 >> e) & 1u)) xb[e] = 0xff800000u;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(xb[e]));
+          mx1 = fmaxf(mx1, __uint_as_float(xb[e + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(xb[e + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(xb[e + 3]));
         }
       }
       const float tile_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      if (!tile_full) tmem_wait_st();  // the masked chunks are re-read below
       // The exponent's reference m follows the running maximum lazily: it moves only when
       // the maximum outgrows it by more than 2^8 in the exp2 domain (weights stay <= 256,
       // well inside bf16 and fp32 range), which saves most rescales of O.  O / l does not
@@ -567,34 +577,31 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
           tmem_st32(tmem_og + lane_addr + 32 * c, o);
         }
       }
-      // pass 2: P = exp2(c*S - c*m); pruned entries are -inf by now and give exactly 0; bf16 P over S
+      // pass 2: P = exp2(c*S - c*m); pruned entries are -inf by now and give exactly 0; bf16 P over
+      // the first half of the chunk's columns of S
       float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll 1
-      for (int cc = 0; cc < n_mine; ++cc) {
-        const int c = grp + 2 * cc;
+      auto emit = [&](const uint32_t (&x)[32], bool act, int c) {
         uint32_t pk[16];
-        if (!((active >> cc) & 1u)) {
+        if (!act) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) pk[e] = 0u;
-          tmem_st16(tmem_s + lane_addr + 32 * c, pk);
-          continue;
-        }
-        uint32_t x[32];
-        tmem_ld32(tmem_s + lane_addr + 32 * c, x);
-        tmem_wait_ld();
+        } else {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
-          const float p1 = ex2_approx(fmaf(__uint_as_float(x[2 * e + 1]), scale_log2, neg_mc));
-          __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-          pk[e] = *reinterpret_cast<uint32_t *>(&hh);
-          // the row sum is taken over the bf16-rounded weights the MMA will use, so that
-          // O / l is an exact convex combination of V rows whatever the rounding of P
-          sum0 += __uint_as_float(pk[e] << 16);
-          sum1 += __uint_as_float(pk[e] & 0xffff0000u);
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(x[2 * e + 1]), scale_log2, neg_mc));
+            __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+            pk[e] = *reinterpret_cast<uint32_t *>(&hh);
+            // the row sum is taken over the bf16-rounded weights the MMA will use, so that
+            // O / l is an exact convex combination of V rows whatever the rounding of P
+            sum0 += __uint_as_float(pk[e] << 16);
+            sum1 += __uint_as_float(pk[e] & 0xffff0000u);
+          }
         }
         tmem_st16(tmem_s + lane_addr + 32 * c, pk);
-      }
+      };
+      emit(xa, act0, grp);
+      if (n_mine > 1) emit(xb, act1, grp + 2);
       l = l * alpha + (sum0 + sum1);
       o_started = true;
       tmem_wait_st();
