@@ -57,23 +57,70 @@ def load_peaks():
 
 
 class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU while the timed steps run.
+
+    Read-only NVML queries from a background thread every few milliseconds (the timed region of
+    the default run lasts tens of milliseconds, too short for `nvidia-smi -lms`); falls back to
+    an `nvidia-smi` child process where NVML cannot be loaded.  The device index is resolved
+    through CUDA_VISIBLE_DEVICES when that holds plain indices.
+    """
+
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.proc = None
+    def __init__(self, gpu_index: int, period_s: float = 0.004):
+        import threading
+
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        ids = [x.strip() for x in vis.split(",") if x.strip()]
+        if ids and all(x.isdigit() for x in ids) and gpu_index < len(ids):
+            gpu_index = int(ids[gpu_index])
+        self.sm, self.reasons, self.max_mhz = [], set(), None
+        self.proc = self.thread = None
+        self._stop = threading.Event()
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+            import pynvml
+
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            bits = {"hw_slowdown": pynvml.nvmlClocksEventReasonHwSlowdown,
+                    "hw_thermal_slowdown": pynvml.nvmlClocksEventReasonHwThermalSlowdown,
+                    "sw_thermal_slowdown": pynvml.nvmlClocksEventReasonSwThermalSlowdown,
+                    "sw_power_cap": pynvml.nvmlClocksEventReasonSwPowerCap}
+
+            def loop():
+                while not self._stop.is_set():
+                    try:
+                        self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                        r = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                        for name, bit in bits.items():
+                            if r & bit:
+                                self.reasons.add(name)
+                    except Exception:
+                        pass
+                    time.sleep(period_s)
+
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+        except Exception:
+            try:
+                self.proc = subprocess.Popen(
+                    ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.FIELDS,
+                     "--format=csv,noheader,nounits", "-lms", "20"],
+                    stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            except OSError:
+                self.proc = None
 
     def stop(self):
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+            return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz,
+                    "samples": len(self.sm), "reasons": sorted(self.reasons), "source": "nvml"}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["clock sampling unavailable"]}
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
@@ -95,7 +142,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi"}
 
 
 # --------------------------------------------------------------------------- CPU oracle legs
@@ -176,7 +223,11 @@ def run_gpu(args, w):
 
     # ---- resident inputs (host-generated, seeded) --------------------------------------
     bias = inputs.calib_bias(w).to(dev)
-    n_rot = 2  # calibration batches kept resident and cycled through by the timed steps
+    # Calibration batches the steps add, one per step: distinct from the calibration set proper and
+    # from one another (a few batches repeated over and over would come to dominate the running
+    # sum and with it the mask the forward is timed on); they stay resident and are reused in turn
+    # only when there are more steps than batches.
+    n_rot = max(1, min(16, args.warmup + args.steps))
     calib = [tuple(t.to(dev) for t in inputs.calib_qk(w, w.calib_batches + r)) for r in range(n_rot)]
     q, k, v = (t.to(dev) for t in inputs.eval_qkv(w))
     out = torch.empty_like(q)
