@@ -44,7 +44,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the ncu
 # captures summarised under profiles/ (None until a capture exists).
-NCU_FWD_TRAFFIC_BYTES = {"long": 422.9e6}  # profiles/long_workload_ncu.md
+NCU_FWD_TRAFFIC_BYTES = {"long": 255.8e6}  # profiles/long_workload_ncu.md (209.3 MB read + 46.5 MB written)
 
 
 def load_peaks():
@@ -309,6 +309,9 @@ def run_gpu(args, w):
     assert nnz_total == k_expected * w.H, (nnz_total, k_expected)
     T_sparse = float(t_log[: args.steps].float().mean().item())
     T_dense = dense.n_tiles()
+    # what the forward kernel executes: rounds of slots (non-empty groups of 16 key columns)
+    n_rounds = int(tiles.round_ptr[-1].item())
+    n_slots = int((tiles.round_info[:n_rounds] & 15).sum().item())
     eff_flops = metrics.effective_flops(nnz_total, w.B, w.d)
     value = replicas.job_throughput(info, eff_flops, fwd_ms_max * 1e-3) / 1e12
 
@@ -334,20 +337,28 @@ def run_gpu(args, w):
     if rank != 0:
         return
     # ---- rooflines ---------------------------------------------------------------------------------
+    # The forward's algorithmic unit is the slot (128 query rows x 16 key columns): the kernel
+    # executes exactly the slots of the schedule, 4*d*128*16 FLOPs each per batch element.  The
+    # kept-tile figure (every stored 128x128 tile computed in full) is given beside it; it exceeds
+    # what is executed because empty groups inside stored tiles are skipped.
     tile_fl = metrics.tile_flops(T_sparse, w.B, w.d)
+    slot_fl = metrics.slot_flops(n_slots, w.B, w.d)
     fwd_s = stage_ms["sparse_fwd"] * 1e-3
     comp_bytes = metrics.compulsory_bytes(w.B, w.H, w.Lq, w.Lk, w.d, elem)
-    tensor_bound = w.dtype == "bf16" and tile_fl / comp_bytes > peaks["bf16_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    tensor_bound = w.dtype == "bf16" and slot_fl / comp_bytes > peaks["bf16_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
     if tensor_bound:
-        roof = {"bound": "tensor", "achieved": tile_fl / fwd_s / 1e12, "peak": peaks["bf16_sustained"],
+        roof = {"bound": "tensor", "achieved": slot_fl / fwd_s / 1e12, "peak": peaks["bf16_sustained"],
                 "unit": "TFLOP/s", "peak_kind": "bf16 sustained, of " + peaks["source"]}
     else:
         roof = {"bound": "hbm", "achieved": comp_bytes / fwd_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "peak_kind": "copy bandwidth, of " + peaks["source"]}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_FWD_TRAFFIC_BYTES.get(w.name)
-    roof["kernel"] = "sparse_fwd"
-    roof["algorithmic"] = {"tile_flops": tile_fl, "compulsory_bytes": comp_bytes, "tiles_per_step": T_sparse}
+    roof["kernel"] = "sparse_fwd (fwd_tc_kernel)" if w.dtype == "bf16" else "sparse_fwd (fwd_simt_kernel)"
+    roof["algorithmic"] = {"slot_flops": slot_fl, "slots_per_launch": n_slots * w.B, "rounds_per_launch": n_rounds * w.B,
+                           "kept_tile_flops": tile_fl, "compulsory_bytes": comp_bytes, "tiles_per_step": T_sparse}
+    roof["other_views"] = {"kept_tile_flops_frac_of_bf16_sustained": tile_fl / fwd_s / 1e12 / peaks["bf16_sustained"],
+                           "compulsory_bytes_frac_of_hbm": comp_bytes / fwd_s / 1e9 / peaks["hbm_gbs"]}
     # other stages, HBM view: accumulate = acc read+write over the domain + bias + Q,K;
     # build_mask = 2 reads of acc + mask bytes + bitmap bits over H*Lq*Lk
     dom = w.n_valid * w.H

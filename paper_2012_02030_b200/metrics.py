@@ -36,6 +36,12 @@ def tile_flops(n_tiles: int, B: int, d: int) -> float:
     return 4.0 * d * TILE * TILE * float(n_tiles) * B
 
 
+def slot_flops(n_slots: int, B: int, d: int) -> float:
+    """FLOPs the tensor cores execute for n_slots slots (one slot = 128 query rows x 16 key columns:
+    2*d*128*16 for S = Q K^T and as many for O += P V), per batch element."""
+    return 4.0 * d * TILE * 16.0 * float(n_slots) * B
+
+
 def compulsory_bytes(B: int, H: int, Lq: int, Lk: int, d: int, elem: int) -> float:
     """One read of Q, K, V and one write of O."""
     return float(elem) * B * H * d * (2 * Lq + 2 * Lk)
