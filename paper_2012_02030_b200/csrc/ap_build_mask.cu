@@ -4,7 +4,12 @@
 // value, then lower linear index i*Lk + j.  The k-th entry of that order is
 // found with a most-significant-digit-first radix select over order-preserving
 // 32-bit keys: three digits of 11, 11 and 10 bits, one histogram pass over the
-// accumulator each.  Entries equal to the threshold key are all kept when the
+// accumulator each.  Large heads first try a shortcut that needs one pass: a
+// random sample of the head brackets the threshold between two pivot keys, one
+// pass counts the keys above the upper pivot and collects those between the
+// pivots, and the threshold is selected among the collected keys; it is exact
+// whenever the bracket holds the threshold and the collected keys fit their
+// buffer (checked with the exact counts), else the head takes the three passes.  Entries equal to the threshold key are all kept when the
 // count allows it (the usual case); otherwise they are ranked by linear index
 // with per-row-segment tie counts and a prefix sum, so that exactly k entries
 // are kept.  The emit pass writes the element mask and per-tile bitmaps;
@@ -37,14 +42,27 @@ struct SelectState {  // per head
   unsigned long long remaining;  // rank still to resolve inside the current prefix
   unsigned long long ties_kept;  // entries equal to thr that are kept (lowest indices first)
   uint32_t all_ties_kept;        // every entry equal to thr is kept: no ranking needed
-  uint32_t pad;
+  uint32_t done;                 // thr, ties_kept, all_ties_kept are final (set by the one-pass shortcut)
+  // the shortcut's bracket and what the collecting pass found
+  uint32_t lo, hi;               // pivot keys, lo <= hi; hi == 0xffffffff: no upper pivot
+  unsigned long long above_hi;   // keys > hi
+  uint32_t n_cand;               // keys in [lo, hi] (may exceed the buffer: then the shortcut fails)
+  uint32_t use_shortcut;
 };
 
 struct Scratch {
   uint32_t *hist;       // [H][kBins]
   SelectState *state;   // [H]
   uint32_t *tie_count;  // [H][Lq][n_kt] -> exclusive prefix after the scan
+  uint32_t *cand;       // [H][cand_cap] keys collected by the shortcut
 };
+
+// The shortcut is tried for heads of at least this many selectable entries.
+constexpr long long kShortcutMinEntries = 1ll << 20;
+constexpr int kSamples = 16384;  // draws per head (over the Lq x Lk rectangle; draws outside the domain are dropped)
+__host__ __device__ inline long long cand_capacity(long long n_rest) {
+  return n_rest >= kShortcutMinEntries ? n_rest / 16 : 0;
+}
 
 __host__ __device__ inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
@@ -70,7 +88,12 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int H, uns
     state[idx].remaining = k_rest;
     state[idx].ties_kept = 0ull;
     state[idx].all_ties_kept = 0u;
-    state[idx].pad = 0u;
+    state[idx].done = 0u;
+    state[idx].lo = 0u;
+    state[idx].hi = 0xffffffffu;
+    state[idx].above_hi = 0ull;
+    state[idx].n_cand = 0u;
+    state[idx].use_shortcut = 0u;
     if (nnz) nnz[idx] = k;
   }
 }
@@ -84,6 +107,7 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
                                                                    uint32_t *__restrict__ hist) {
   __shared__ uint32_t sh[kBins];
   const int h = blockIdx.y;
+  if (state[h].done) return;  // resolved by the shortcut
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0u;
   __syncthreads();
@@ -136,6 +160,7 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
 __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass) {
   __shared__ uint32_t warp_sums[8];
   const int h = blockIdx.x;
+  if (state[h].done) return;  // resolved by the shortcut
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t cnt[8];
   uint32_t mine = 0u;
@@ -177,6 +202,207 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
       out.all_ties_kept = out.remaining == cnt[e] ? 1u : 0u;
     }
     state[h] = out;
+  }
+}
+
+// ---- the one-pass shortcut ------------------------------------------------------------------
+
+// CTA-wide (1024 threads) radix select: the key of rank `rank` (1 = largest) among keys[0..n),
+// 1 <= rank <= n.  Returns the key, how many keys equal it, and the rank inside that group of
+// equals.  hist: 2048 words of shared memory; xch: 4 words.
+struct Picked {
+  uint32_t key, count, rank_in_ties;
+};
+__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch) {
+  __shared__ uint32_t warp_sums[32];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  uint32_t prefix = 0u, hi_mask = 0u, count = 0u;
+  for (int pass = 0; pass < kPasses; ++pass) {
+    const int shift = digit_shift(pass);
+    const uint32_t dmask = digit_mask(pass);
+    hist[t] = 0u;
+    hist[t + 1024] = 0u;
+    __syncthreads();
+    for (uint32_t idx = t; idx < n; idx += 1024) {
+      const uint32_t key = keys[idx];
+      if ((key & hi_mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+    }
+    __syncthreads();
+    // thread t owns bins 2047 - 2t and 2046 - 2t (descending order of keys)
+    const uint32_t c0 = hist[kBins - 1 - 2 * t], c1 = hist[kBins - 2 - 2 * t];
+    const uint32_t mine = c0 + c1;
+    uint32_t incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    uint32_t before = incl - mine;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    if (before < rank && before + mine >= rank) {  // exactly one thread
+      const bool first = before + c0 >= rank;
+      xch[0] = (uint32_t)(kBins - 1 - 2 * t - (first ? 0 : 1));
+      xch[1] = rank - before - (first ? 0u : c0);
+      xch[2] = first ? c0 : c1;
+    }
+    __syncthreads();
+    prefix |= xch[0] << shift;
+    rank = xch[1];
+    count = xch[2];
+    hi_mask |= dmask << shift;
+    __syncthreads();
+  }
+  Picked p;
+  p.key = prefix;
+  p.count = count;
+  p.rank_in_ties = rank;
+  return p;
+}
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
+  x += 0x9e3779b97f4a7c15ull;
+  x = (x ^ (x >> 30)) * 0xbf58476d1ce4e5b9ull;
+  x = (x ^ (x >> 27)) * 0x94d049bb133111ebull;
+  return x ^ (x >> 31);
+}
+
+// One CTA per head: samples the head and sets the bracket [lo, hi] around the expected threshold.
+__global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__restrict__ acc, int Lq, int Lk, int causal,
+                                                             int diag, unsigned long long k_rest,
+                                                             unsigned long long n_rest, SelectState *state) {
+  extern __shared__ uint32_t sm_dyn[];
+  uint32_t *keys = sm_dyn;               // kSamples
+  uint32_t *hist = sm_dyn + kSamples;    // kBins
+  __shared__ uint32_t xch[4];
+  __shared__ uint32_t n_valid_s;
+  const int h = blockIdx.x, t = threadIdx.x;
+  if (t == 0) n_valid_s = 0u;
+  __syncthreads();
+  const unsigned long long cells = (unsigned long long)Lq * Lk;
+  for (int s = t; s < kSamples; s += 1024) {
+    const unsigned long long idx = mix64(((unsigned long long)h << 32) | (unsigned)s) % cells;
+    const int i = (int)(idx / Lk), j = (int)(idx % Lk);
+    if ((causal && j > i) || (diag && j == i)) continue;
+    const uint32_t pos = atomicAdd(&n_valid_s, 1u);
+    keys[pos] = key_of(acc[((size_t)h * Lq + i) * Lk + j]);
+  }
+  __syncthreads();
+  const uint32_t nv = n_valid_s;
+  if (nv < 1024u) return;  // too few draws landed in the domain: no shortcut for this head
+  // expected rank of the threshold inside the sample and a bracket of six standard deviations
+  const double frac = (double)k_rest / (double)n_rest;
+  const double r = frac * nv;
+  const double dev = 6.0 * sqrt(fmax(r * (1.0 - frac), 1.0)) + 16.0;
+  const long long r_hi = (long long)floor(r - dev), r_lo = (long long)ceil(r + dev);
+  uint32_t hi = 0xffffffffu, lo = 0u;
+  if (r_hi >= 1) hi = block_select(keys, nv, (uint32_t)r_hi, hist, xch).key;
+  if (r_lo <= (long long)nv) lo = block_select(keys, nv, (uint32_t)r_lo, hist, xch).key;
+  if (t == 0) {
+    state[h].hi = hi;
+    state[h].lo = lo;
+    state[h].use_shortcut = 1u;
+  }
+}
+
+// One pass over the head: counts the keys above the upper pivot and collects those inside the
+// bracket.  grid = (row blocks, H); a warp takes a row at a time.  Collected keys are staged in
+// shared memory and appended to the head's buffer with one reservation per CTA (keys that do not
+// fit the stage any more are appended one warp at a time).
+constexpr int kStageKeys = 8192;
+__global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restrict__ acc, int Lq, int Lk, int causal,
+                                                           int diag, SelectState *state, uint32_t *__restrict__ cand,
+                                                           uint32_t cand_cap) {
+  __shared__ uint32_t stage[kStageKeys];
+  // stage_n only grows; a reservation that does not fit fails, and so do all later ones, so the
+  // staged keys are the contiguous range below the first failed reservation (stage_end)
+  __shared__ uint32_t stage_n, stage_end, stage_base;
+  const int h = blockIdx.y;
+  if (!state[h].use_shortcut) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    stage_n = 0u;
+    stage_end = 0xffffffffu;
+  }
+  __syncthreads();
+  const uint32_t lo = state[h].lo, hi = state[h].hi;
+  uint32_t *out = cand + (size_t)h * cand_cap;
+  const bool vec = (Lk & 3) == 0;
+  unsigned long long above = 0ull;
+  for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
+    const float *row = acc + ((size_t)h * Lq + i) * Lk;
+    const int jend = causal ? min(Lk, i + 1) : Lk;
+    for (int base = 0; base < jend; base += 512) {  // warp-uniform trip count
+      float v[4][4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j0 = base + 128 * u + 4 * lane;
+        v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+        if (j0 < jend) load4(row, j0, jend, vec, v[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j0 = base + 128 * u + 4 * lane;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int j = j0 + c;
+          const uint32_t key = key_of(v[u][c]);
+          const bool in = j < jend && !(diag && j == i);
+          above += (in && key > hi) ? 1u : 0u;
+          const bool take = in && key >= lo && key <= hi;
+          const unsigned takers = __ballot_sync(0xffffffffu, take);
+          if (takers) {  // warp-uniform
+            uint32_t start = 0u;
+            if (lane == 0) start = atomicAdd(&stage_n, (uint32_t)__popc(takers));
+            start = __shfl_sync(0xffffffffu, start, 0);
+            if (start + 32u <= (uint32_t)kStageKeys) {
+              if (take) stage[start + __popc(takers & ((1u << lane) - 1u))] = key;
+            } else {
+              // the stage is full: this warp's keys go straight to the head's buffer
+              if (lane == 0) {
+                atomicMin(&stage_end, start);
+                start = atomicAdd(&state[h].n_cand, (uint32_t)__popc(takers));
+              }
+              start = __shfl_sync(0xffffffffu, start, 0);
+              const uint32_t pos = start + __popc(takers & ((1u << lane) - 1u));
+              if (take && pos < cand_cap) out[pos] = key;
+            }
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
+  if (lane == 0 && above) atomicAdd(&state[h].above_hi, above);
+  __syncthreads();
+  const uint32_t n = min(stage_n, stage_end);
+  if (threadIdx.x == 0) stage_base = atomicAdd(&state[h].n_cand, n);
+  __syncthreads();
+  const uint32_t dst = stage_base;
+  for (uint32_t e = threadIdx.x; e < n; e += kThreads)
+    if (dst + e < cand_cap) out[dst + e] = stage[e];
+}
+
+// One CTA per head: if the bracket holds the threshold, selects it among the collected keys.
+__global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *state, const uint32_t *__restrict__ cand,
+                                                                 uint32_t cand_cap, unsigned long long k_rest) {
+  __shared__ uint32_t hist[kBins];
+  __shared__ uint32_t xch[4];
+  const int h = blockIdx.x;
+  const SelectState st = state[h];
+  if (!st.use_shortcut) return;
+  // the threshold is the (k_rest - above_hi)-th largest collected key, if there is one
+  if (st.n_cand > cand_cap || st.above_hi >= k_rest || k_rest - st.above_hi > st.n_cand) return;
+  const Picked p = block_select(cand + (size_t)h * cand_cap, st.n_cand, (uint32_t)(k_rest - st.above_hi), hist, xch);
+  if (threadIdx.x == 0) {
+    state[h].thr = p.key;
+    state[h].prefix = p.key;
+    state[h].ties_kept = p.rank_in_ties;
+    state[h].remaining = p.rank_in_ties;
+    state[h].all_ties_kept = p.rank_in_ties == p.count ? 1u : 0u;
+    state[h].done = 1u;
   }
 }
 
@@ -364,14 +590,18 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
   s.state = reinterpret_cast<SelectState *>(p);
   p += align256((size_t)H * sizeof(SelectState));
   s.tie_count = reinterpret_cast<uint32_t *>(p);
+  p += align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t));
+  s.cand = reinterpret_cast<uint32_t *>(p);
   return s;
 }
 
 }  // namespace
 
 size_t select_scratch_bytes(int H, int Lq, int Lk) {
+  // the candidate buffer is sized for the larger of the causal and the full domain
   return align256((size_t)H * kBins * sizeof(uint32_t)) + align256((size_t)H * sizeof(SelectState)) +
-         align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t));
+         align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t)) +
+         align256((size_t)H * (size_t)cand_capacity((long long)Lq * Lk) * sizeof(uint32_t));
 }
 
 cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
@@ -389,6 +619,21 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   if (row_blocks > want) row_blocks = want;
   dim3 grid(row_blocks, a.H);
   if (a.k_rest > 0) {
+    // large heads: the one-pass shortcut first (heads it resolves skip the three passes below)
+    const long long n_valid = a.causal ? (long long)a.Lq * (a.Lq + 1) / 2 : (long long)a.Lq * a.Lk;
+    const long long n_rest = n_valid - (diag ? a.Lq : 0);
+    const long long cap = cand_capacity(n_rest);
+    if (cap > 0) {
+      const size_t smem = (kSamples + kBins) * sizeof(uint32_t);
+      e = cudaFuncSetAttribute(sample_pivots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      sample_pivots_kernel<<<a.H, 1024, smem, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, (unsigned long long)a.k_rest,
+                                                   (unsigned long long)n_rest, sc.state);
+      collect_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, sc.state, sc.cand, (uint32_t)cap);
+      select_candidates_kernel<<<a.H, 1024, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, (unsigned long long)a.k_rest);
+      count_launches(3);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
     for (int pass = 0; pass < kPasses; ++pass) {
       digit_histogram_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, pass, sc.state, sc.hist);
       count_launches(1);

@@ -111,6 +111,24 @@ def test_build_mask_constant_and_tiny_fraction(ap):
     _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=1e-6, keep_diag=False))
 
 
+@pytest.mark.parametrize("causal,L", [(False, 1100), (True, 1536)])
+def test_build_mask_large_heads_take_the_one_pass_shortcut(ap, causal, L):
+    """Heads of more than 2^20 selectable entries first try to bracket the threshold with a sample
+    and select among the keys collected in one pass.  Head 0: distinct values (the shortcut holds);
+    head 1: heavily quantised values, so the threshold key is tied thousands of times; head 2:
+    skewed values (most mass near zero); head 3: constant, every key falls into the bracket and
+    the collected keys overflow their buffer, so the head falls back to the three-pass select."""
+    H = 4
+    rng = np.random.default_rng(73 + L)
+    acc = rng.random((H, L, L), dtype=np.float32)
+    acc[1] = np.round(acc[1] * 32) / 32
+    acc[2] = acc[2] ** 8
+    acc[3] = 0.75
+    for keep, keep_diag in ((0.05, True), (0.5, False), (0.999, True)):
+        _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=L, Lk=L, causal=causal, keep_diag=keep_diag,
+                                                     keep_frac=keep))
+
+
 def test_build_mask_optional_outputs(ap):
     acc = np.random.default_rng(72).random((2, 140, 140), dtype=np.float32)
     acc_dev = torch.from_numpy(acc).cuda()
