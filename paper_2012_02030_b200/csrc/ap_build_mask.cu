@@ -213,19 +213,33 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
 struct Picked {
   uint32_t key, count, rank_in_ties;
 };
-__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch) {
+// All keys lie in [base, base + span]: the select runs on key - base, and leading digits in which
+// span is zero are known to be zero (no pass, and no pile-up of every key in one bin).
+__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch,
+                               uint32_t base = 0u, uint32_t span = 0xffffffffu) {
   __shared__ uint32_t warp_sums[32];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-  uint32_t prefix = 0u, hi_mask = 0u, count = 0u;
+  uint32_t prefix = 0u, hi_mask = 0u, count = n;
   for (int pass = 0; pass < kPasses; ++pass) {
     const int shift = digit_shift(pass);
     const uint32_t dmask = digit_mask(pass);
+    if (((span >> shift) & ~0u) == 0u && pass < kPasses - 1) {  // the digit is 0 for every key
+      hi_mask |= dmask << shift;
+      continue;
+    }
     hist[t] = 0u;
     hist[t + 1024] = 0u;
     __syncthreads();
-    for (uint32_t idx = t; idx < n; idx += 1024) {
-      const uint32_t key = keys[idx];
-      if ((key & hi_mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+    for (uint32_t idx0 = t; idx0 < n; idx0 += 8 * 1024) {  // eight loads in flight per thread
+      uint32_t kk[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t idx = idx0 + u * 1024;
+        kk[u] = idx < n ? keys[idx] - base : 0xffffffffu;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (idx0 + u * 1024 < n && (kk[u] & hi_mask) == prefix) atomicAdd(&hist[(kk[u] >> shift) & dmask], 1u);
     }
     __syncthreads();
     // thread t owns bins 2047 - 2t and 2046 - 2t (descending order of keys)
@@ -255,7 +269,7 @@ __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, 
     __syncthreads();
   }
   Picked p;
-  p.key = prefix;
+  p.key = prefix + base;
   p.count = count;
   p.rank_in_ties = rank;
   return p;
@@ -315,16 +329,11 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
                                                            int diag, SelectState *state, uint32_t *__restrict__ cand,
                                                            uint32_t cand_cap) {
   __shared__ uint32_t stage[kStageKeys];
-  // stage_n only grows; a reservation that does not fit fails, and so do all later ones, so the
-  // staged keys are the contiguous range below the first failed reservation (stage_end)
-  __shared__ uint32_t stage_n, stage_end, stage_base;
+  __shared__ uint32_t stage_n, stage_base;  // stage_n only grows; positions beyond the stage were not staged
   const int h = blockIdx.y;
   if (!state[h].use_shortcut) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    stage_n = 0u;
-    stage_end = 0xffffffffu;
-  }
+  if (threadIdx.x == 0) stage_n = 0u;
   __syncthreads();
   const uint32_t lo = state[h].lo, hi = state[h].hi;
   uint32_t *out = cand + (size_t)h * cand_cap;
@@ -350,23 +359,14 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
           const uint32_t key = key_of(v[u][c]);
           const bool in = j < jend && !(diag && j == i);
           above += (in && key > hi) ? 1u : 0u;
-          const bool take = in && key >= lo && key <= hi;
-          const unsigned takers = __ballot_sync(0xffffffffu, take);
-          if (takers) {  // warp-uniform
-            uint32_t start = 0u;
-            if (lane == 0) start = atomicAdd(&stage_n, (uint32_t)__popc(takers));
-            start = __shfl_sync(0xffffffffu, start, 0);
-            if (start + 32u <= (uint32_t)kStageKeys) {
-              if (take) stage[start + __popc(takers & ((1u << lane) - 1u))] = key;
+          if (in && key >= lo && key <= hi) {  // a few per cent of the entries
+            const uint32_t pos = atomicAdd(&stage_n, 1u);
+            if (pos < (uint32_t)kStageKeys) {
+              stage[pos] = key;
             } else {
-              // the stage is full: this warp's keys go straight to the head's buffer
-              if (lane == 0) {
-                atomicMin(&stage_end, start);
-                start = atomicAdd(&state[h].n_cand, (uint32_t)__popc(takers));
-              }
-              start = __shfl_sync(0xffffffffu, start, 0);
-              const uint32_t pos = start + __popc(takers & ((1u << lane) - 1u));
-              if (take && pos < cand_cap) out[pos] = key;
+              // the stage is full: the key goes straight to the head's buffer
+              const uint32_t g = atomicAdd(&state[h].n_cand, 1u);
+              if (g < cand_cap) out[g] = key;
             }
           }
         }
@@ -377,7 +377,7 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
   for (int o = 16; o > 0; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
   if (lane == 0 && above) atomicAdd(&state[h].above_hi, above);
   __syncthreads();
-  const uint32_t n = min(stage_n, stage_end);
+  const uint32_t n = min(stage_n, (uint32_t)kStageKeys);
   if (threadIdx.x == 0) stage_base = atomicAdd(&state[h].n_cand, n);
   __syncthreads();
   const uint32_t dst = stage_base;
@@ -395,7 +395,8 @@ __global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *st
   if (!st.use_shortcut) return;
   // the threshold is the (k_rest - above_hi)-th largest collected key, if there is one
   if (st.n_cand > cand_cap || st.above_hi >= k_rest || k_rest - st.above_hi > st.n_cand) return;
-  const Picked p = block_select(cand + (size_t)h * cand_cap, st.n_cand, (uint32_t)(k_rest - st.above_hi), hist, xch);
+  const Picked p = block_select(cand + (size_t)h * cand_cap, st.n_cand, (uint32_t)(k_rest - st.above_hi), hist, xch,
+                                st.lo, st.hi - st.lo);
   if (threadIdx.x == 0) {
     state[h].thr = p.key;
     state[h].prefix = p.key;
@@ -498,6 +499,25 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   const int j0 = kt * kTile + 4 * lane;
   __shared__ int warp_count[4];
   int count = 0;
+  if (causal && kt > qt) {
+    // the whole tile lies above the diagonal: nothing is kept, nothing needs to be read
+    for (int r = warp; r < kTile; r += 4) {
+      const int i = qt * kTile + r;
+      if (i < Lq && mask) {
+        uint8_t *mrow = mask + ((size_t)h * Lq + i) * Lk;
+        if (vec && j0 + 4 <= Lk) {
+          *reinterpret_cast<uchar4 *>(mrow + j0) = make_uchar4(0, 0, 0, 0);
+        } else {
+          for (int c = 0; c < 4; ++c)
+            if (j0 + c < Lk) mrow[j0 + c] = 0;
+        }
+      }
+      if (stage_bitmap && lane == 0)
+        reinterpret_cast<uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords)[r] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (stage_count && threadIdx.x == 0) stage_count[tile] = 0;
+    return;
+  }
   for (int r0 = warp; r0 < kTile; r0 += 16) {
     float v[4][4];
 #pragma unroll
