@@ -48,14 +48,18 @@ struct SelectState {  // per head
   unsigned long long above_hi;   // keys > hi
   uint32_t n_cand;               // keys in [lo, hi] (may exceed the buffer: then the shortcut fails)
   uint32_t use_shortcut;
+  // when not all entries equal to thr are kept: those with linear index i*Lk + j <= tie_cut are
+  // (valid if have_cut; otherwise the ties are ranked with tie counts and a prefix sum)
+  uint32_t tie_cut, have_cut;
 };
 
 struct Scratch {
   uint32_t *hist;       // [H][kBins]
   SelectState *state;   // [H]
   uint32_t *tie_count;  // [H][Lq][n_kt] -> exclusive prefix after the scan
-  uint32_t *cand;       // [H][cand_cap] keys collected by the shortcut
+  uint2 *cand;          // [H][cand_cap] (key, linear index) of the entries collected by the shortcut
 };
+constexpr int kMaxCutTies = 4096;  // ties with the threshold ranked inside the shortcut (more: tie counts + scan)
 
 // The shortcut is tried for heads of at least this many selectable entries.
 constexpr long long kShortcutMinEntries = 1ll << 20;
@@ -94,6 +98,8 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int H, uns
     state[idx].above_hi = 0ull;
     state[idx].n_cand = 0u;
     state[idx].use_shortcut = 0u;
+    state[idx].tie_cut = 0u;
+    state[idx].have_cut = 0u;
     if (nnz) nnz[idx] = k;
   }
 }
@@ -216,7 +222,7 @@ struct Picked {
 // All keys lie in [base, base + span]: the select runs on key - base, and leading digits in which
 // span is zero are known to be zero (no pass, and no pile-up of every key in one bin).
 __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch,
-                               uint32_t base = 0u, uint32_t span = 0xffffffffu) {
+                               uint32_t base = 0u, uint32_t span = 0xffffffffu, int stride = 1) {
   __shared__ uint32_t warp_sums[32];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   uint32_t prefix = 0u, hi_mask = 0u, count = n;
@@ -235,7 +241,7 @@ __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, 
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const uint32_t idx = idx0 + u * 1024;
-        kk[u] = idx < n ? keys[idx] - base : 0xffffffffu;
+        kk[u] = idx < n ? keys[(size_t)idx * stride] - base : 0xffffffffu;
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u)
@@ -324,11 +330,11 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
 // bracket.  grid = (row blocks, H); a warp takes a row at a time.  Collected keys are staged in
 // shared memory and appended to the head's buffer with one reservation per CTA (keys that do not
 // fit the stage any more are appended one warp at a time).
-constexpr int kStageKeys = 8192;
+constexpr int kStageKeys = 4096;
 __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restrict__ acc, int Lq, int Lk, int causal,
-                                                           int diag, SelectState *state, uint32_t *__restrict__ cand,
+                                                           int diag, SelectState *state, uint2 *__restrict__ cand,
                                                            uint32_t cand_cap) {
-  __shared__ uint32_t stage[kStageKeys];
+  __shared__ uint2 stage[kStageKeys];
   __shared__ uint32_t stage_n, stage_base;  // stage_n only grows; positions beyond the stage were not staged
   const int h = blockIdx.y;
   if (!state[h].use_shortcut) return;
@@ -336,7 +342,7 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
   if (threadIdx.x == 0) stage_n = 0u;
   __syncthreads();
   const uint32_t lo = state[h].lo, hi = state[h].hi;
-  uint32_t *out = cand + (size_t)h * cand_cap;
+  uint2 *out = cand + (size_t)h * cand_cap;
   const bool vec = (Lk & 3) == 0;
   unsigned long long above = 0ull;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
@@ -360,13 +366,14 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
           const bool in = j < jend && !(diag && j == i);
           above += (in && key > hi) ? 1u : 0u;
           if (in && key >= lo && key <= hi) {  // a few per cent of the entries
+            const uint2 entry = make_uint2(key, (uint32_t)i * (uint32_t)Lk + (uint32_t)j);
             const uint32_t pos = atomicAdd(&stage_n, 1u);
             if (pos < (uint32_t)kStageKeys) {
-              stage[pos] = key;
+              stage[pos] = entry;
             } else {
-              // the stage is full: the key goes straight to the head's buffer
+              // the stage is full: the entry goes straight to the head's buffer
               const uint32_t g = atomicAdd(&state[h].n_cand, 1u);
-              if (g < cand_cap) out[g] = key;
+              if (g < cand_cap) out[g] = entry;
             }
           }
         }
@@ -386,18 +393,44 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
 }
 
 // One CTA per head: if the bracket holds the threshold, selects it among the collected keys.
-__global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *state, const uint32_t *__restrict__ cand,
+__global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *state, const uint2 *__restrict__ cand,
                                                                  uint32_t cand_cap, unsigned long long k_rest) {
   __shared__ uint32_t hist[kBins];
   __shared__ uint32_t xch[4];
+  __shared__ uint32_t tie_idx[kMaxCutTies];
+  __shared__ uint32_t tie_n, cut_s;
   const int h = blockIdx.x;
   const SelectState st = state[h];
   if (!st.use_shortcut) return;
   // the threshold is the (k_rest - above_hi)-th largest collected key, if there is one
   if (st.n_cand > cand_cap || st.above_hi >= k_rest || k_rest - st.above_hi > st.n_cand) return;
-  const Picked p = block_select(cand + (size_t)h * cand_cap, st.n_cand, (uint32_t)(k_rest - st.above_hi), hist, xch,
-                                st.lo, st.hi - st.lo);
+  const uint2 *mine = cand + (size_t)h * cand_cap;
+  const Picked p = block_select(reinterpret_cast<const uint32_t *>(mine), st.n_cand, (uint32_t)(k_rest - st.above_hi),
+                                hist, xch, st.lo, st.hi - st.lo, 2);
+  // Not all entries equal to the threshold are kept: the ones with the lowest linear indices are.
+  // With few enough of them, the index of the last kept one is found here.
+  bool have_cut = false;
+  if (p.rank_in_ties < p.count && p.count <= (uint32_t)kMaxCutTies) {
+    if (threadIdx.x == 0) tie_n = 0u;
+    __syncthreads();
+    for (uint32_t e = threadIdx.x; e < st.n_cand; e += 1024) {
+      const uint2 c = mine[e];
+      if (c.x == p.key) tie_idx[atomicAdd(&tie_n, 1u)] = c.y;
+    }
+    __syncthreads();
+    // the index with exactly rank_in_ties - 1 smaller ones (indices are distinct)
+    for (uint32_t e = threadIdx.x; e < p.count; e += 1024) {
+      const uint32_t me = tie_idx[e];
+      uint32_t smaller = 0u;
+      for (uint32_t f = 0; f < p.count; ++f) smaller += tie_idx[f] < me ? 1u : 0u;
+      if (smaller == p.rank_in_ties - 1u) cut_s = me;
+    }
+    __syncthreads();
+    have_cut = true;
+  }
   if (threadIdx.x == 0) {
+    state[h].tie_cut = have_cut ? cut_s : 0u;
+    state[h].have_cut = have_cut ? 1u : 0u;
     state[h].thr = p.key;
     state[h].prefix = p.key;
     state[h].ties_kept = p.rank_in_ties;
@@ -414,7 +447,7 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
                                                              const SelectState *__restrict__ state,
                                                              uint32_t *__restrict__ tie_count) {
   const int h = blockIdx.y;
-  if (state[h].all_ties_kept) return;
+  if (state[h].all_ties_kept || state[h].have_cut) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t thr = state[h].thr;
   const bool vec = (Lk & 3) == 0;
@@ -443,7 +476,7 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
 // One CTA per head: in-place exclusive prefix sum over the head's (row, segment) tie counts.
 __global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ tie_count, int n_per_head,
                                                         const SelectState *__restrict__ state) {
-  if (state[blockIdx.x].all_ties_kept) return;
+  if (state[blockIdx.x].all_ties_kept || state[blockIdx.x].have_cut) return;
   __shared__ uint32_t warp_sums[32];
   __shared__ uint32_t carry_s;
   uint32_t *a = tie_count + (size_t)blockIdx.x * n_per_head;
@@ -495,6 +528,8 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   const uint32_t thr = state[h].thr;
   const unsigned long long ties_kept = state[h].ties_kept;
   const bool all_ties = state[h].all_ties_kept != 0u;
+  const bool have_cut = state[h].have_cut != 0u;
+  const uint32_t tie_cut = state[h].tie_cut;
   const bool vec = (Lk & 3) == 0;
   const int j0 = kt * kTile + 4 * lane;
   __shared__ int warp_count[4];
@@ -553,6 +588,10 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
         nib = gt_bits;
         if (all_ties) {
           nib |= tie_bits;
+        } else if (have_cut) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            if ((tie_bits & (1u << c)) && (uint32_t)i * (uint32_t)Lk + (uint32_t)(j0 + c) <= tie_cut) nib |= 1u << c;
         } else if (__any_sync(0xffffffffu, tie_bits != 0u)) {
           // rank of each tie in linear-index order = ties before this row segment
           // + ties in lower lanes + ties in lower columns of this lane
@@ -611,7 +650,7 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
   p += align256((size_t)H * sizeof(SelectState));
   s.tie_count = reinterpret_cast<uint32_t *>(p);
   p += align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t));
-  s.cand = reinterpret_cast<uint32_t *>(p);
+  s.cand = reinterpret_cast<uint2 *>(p);
   return s;
 }
 
@@ -621,7 +660,7 @@ size_t select_scratch_bytes(int H, int Lq, int Lk) {
   // the candidate buffer is sized for the larger of the causal and the full domain
   return align256((size_t)H * kBins * sizeof(uint32_t)) + align256((size_t)H * sizeof(SelectState)) +
          align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t)) +
-         align256((size_t)H * (size_t)cand_capacity((long long)Lq * Lk) * sizeof(uint32_t));
+         align256((size_t)H * (size_t)cand_capacity((long long)Lq * Lk) * sizeof(uint2));
 }
 
 cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {

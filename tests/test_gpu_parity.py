@@ -124,7 +124,16 @@ def test_build_mask_large_heads_take_the_one_pass_shortcut(ap, causal, L):
     acc[1] = np.round(acc[1] * 32) / 32
     acc[2] = acc[2] ** 8
     acc[3] = 0.75
-    for keep, keep_diag in ((0.05, True), (0.5, False), (0.999, True)):
+    # head 0: a handful of exact copies of the value at the 5 % threshold, scattered over the head, so
+    # that the threshold key is tied a few times and only the copies with the lowest indices are kept
+    dom = np.tril(np.ones((L, L), dtype=bool)) if causal else np.ones((L, L), dtype=bool)
+    vals = acc[0][dom]
+    k = int(0.05 * vals.size)
+    v_thr = np.partition(vals, vals.size - k)[vals.size - k]
+    rows = rng.integers(L // 2, L, size=9)
+    cols = rng.integers(0, L // 2, size=9)
+    acc[0, rows, cols] = v_thr
+    for keep, keep_diag in ((0.05, True), (0.05, False), (0.5, False), (0.999, True)):
         _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=L, Lk=L, causal=causal, keep_diag=keep_diag,
                                                      keep_frac=keep))
 
