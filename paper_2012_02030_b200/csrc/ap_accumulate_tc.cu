@@ -281,14 +281,26 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           if (!interior && 32 * c + e >= n_valid) t[e] = -CUDART_INF_F;
         }
         if (sweep == 0) {
-          float cm = st.x;
+          // four independent chains each for the maximum and for the sum
+          float m0 = st.x, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) cm = fmaxf(cm, t[e]);
+          for (int e = 0; e < 32; e += 4) {
+            m0 = fmaxf(m0, t[e]);
+            m1 = fmaxf(m1, t[e + 1]);
+            m2 = fmaxf(m2, t[e + 2]);
+            m3 = fmaxf(m3, t[e + 3]);
+          }
+          const float cm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
           const float cm_safe = cm == -CUDART_INF_F ? 0.f : cm;
-          float z = st.y * ex2_approx(st.x - cm_safe);
+          float z0 = st.y * ex2_approx(st.x - cm_safe), z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) z += ex2_approx(t[e] - cm_safe);
-          st = make_float2(cm, z);
+          for (int e = 0; e < 32; e += 4) {
+            z0 += ex2_approx(t[e] - cm_safe);
+            z1 += ex2_approx(t[e + 1] - cm_safe);
+            z2 += ex2_approx(t[e + 2] - cm_safe);
+            z3 += ex2_approx(t[e + 3] - cm_safe);
+          }
+          st = make_float2(cm, (z0 + z1) + (z2 + z3));
         } else {
           // running sum over b of the normalised weights, kept in TMEM next to S
           const uint32_t ps_addr = tmem + 256 + 64 * wg + 32 * c + lane_addr;
