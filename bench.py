@@ -409,6 +409,89 @@ def run_gpu(args, w):
     print(json.dumps(line))
 
 
+def run_density_sweep(args, w):
+    """Speedup of the sparse forward over the library's dense path as a function of the kept
+    fraction, on the workload's shape and calibration statistics (one GPU).  Two mask families:
+    'topk' = the method's per-head top-fraction masks; 'blocks' = masks whose kept entries fill
+    whole 128x128 tiles (the tiles with the largest accumulated mass), where tile occupancy tracks
+    density.  Prints one JSON line with the table."""
+    from paper_2012_02030_b200 import binding as ap
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    bias = inputs.calib_bias(w).to(dev)
+    acc = torch.zeros((w.H, w.Lq, w.Lk), dtype=torch.float32, device=dev)
+    for t in range(args.calib_batches if args.calib_batches > 0 else w.calib_batches):
+        cq, ck = inputs.calib_qk(w, t)
+        ap.ap_accumulate_attention(acc, cq.to(dev), ck.to(dev), bias, causal=w.causal)
+    q, k, v = (t.to(dev) for t in inputs.eval_qkv(w))
+    out = torch.empty_like(q)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    dense = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    nnz = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+    ws = torch.empty(ap.ap_build_mask_workspace_bytes(w.H, w.Lq, w.Lk), dtype=torch.uint8, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def time_fwd(tl):
+        for _ in range(3):
+            ap.ap_sparse_attention_fwd(q, k, v, tl, out)
+        ms = []
+        for _ in range(max(args.steps, 5)):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ap.ap_sparse_attention_fwd(q, k, v, tl, out)
+            e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        return float(np.median(ms))
+
+    ap.ap_dense_tiles(dense, causal=w.causal)
+    dense_ms = time_fwd(dense)
+    n_qt, n_kt = dense.n_qt, dense.n_kt
+    # accumulated mass per 128x128 tile, for the block-structured family
+    pad_q, pad_k = n_qt * 128 - w.Lq, n_kt * 128 - w.Lk
+    mass = torch.nn.functional.pad(acc, (0, pad_k, 0, pad_q)).view(w.H, n_qt, 128, n_kt, 128).sum((2, 4))
+    dom_tiles = torch.ones((n_qt, n_kt), dtype=torch.bool, device=dev)
+    if w.causal:
+        dom_tiles = torch.tril(dom_tiles)
+    rows = []
+    for keep in (1.0, 0.5, 0.25, 0.1, 0.05, 0.02):
+        ap.ap_build_mask(acc, keep, w.causal, w.keep_diag, None, tiles, nnz, ws)
+        ms = time_fwd(tiles)
+        n_rounds = int(tiles.round_ptr[-1].item())
+        slots = int((tiles.round_info[:n_rounds] & 15).sum().item())
+        rows.append({"family": "topk", "keep": keep, "kept_fraction": float(nnz.sum().item()) / (w.n_valid * w.H),
+                     "tiles": tiles.n_tiles(), "slots": slots, "fwd_ms": ms, "speedup_vs_dense_path": dense_ms / ms,
+                     "effective_tflops": metrics.effective_flops(int(nnz.sum().item()), w.B, w.d) / (ms * 1e-3) / 1e12})
+    for keep in (1.0, 0.5, 0.25, 0.1, 0.05, 0.02):
+        # keep the heaviest tiles of every head (the diagonal tiles always), entries inside the domain
+        score = mass.masked_fill(~dom_tiles, float("-inf")).clone()
+        idx = torch.arange(min(n_qt, n_kt), device=dev)
+        score[:, idx, idx] = float("inf")
+        n_keep = max(min(n_qt, n_kt), int(round(keep * int(dom_tiles.sum().item()))))
+        thr = score.flatten(1).topk(n_keep, dim=1).values[:, -1]
+        tile_keep = score >= thr[:, None, None]
+        m = tile_keep[:, :, None, :, None].expand(w.H, n_qt, 128, n_kt, 128).reshape(w.H, n_qt * 128, n_kt * 128)
+        m = m[:, :w.Lq, :w.Lk]
+        if w.causal:
+            m = m & torch.tril(torch.ones((w.Lq, w.Lk), dtype=torch.bool, device=dev))
+        mask = m.to(torch.uint8).contiguous()
+        ap.ap_mask_to_tiles(mask, tiles)
+        kept = int(mask.sum().item())
+        ms = time_fwd(tiles)
+        n_rounds = int(tiles.round_ptr[-1].item())
+        slots = int((tiles.round_info[:n_rounds] & 15).sum().item())
+        rows.append({"family": "blocks", "keep": keep, "kept_fraction": kept / float(w.n_valid * w.H),
+                     "tiles": tiles.n_tiles(), "slots": slots, "fwd_ms": ms, "speedup_vs_dense_path": dense_ms / ms,
+                     "effective_tflops": metrics.effective_flops(kept, w.B, w.d) / (ms * 1e-3) / 1e12})
+    if ap.ap_device_status() != ap.AP_OK:
+        raise RuntimeError("device status not OK after the sweep")
+    print(json.dumps({"density_sweep": {"workload": w.name, "dense_path_ms": dense_ms, "dense_tiles": dense.n_tiles(),
+                                        "timing": "median of single launches, 256 MiB L2 flush before each",
+                                        "rows": rows}}))
+
+
 def main():
     p = argparse.ArgumentParser()
     p.add_argument("--gpus", type=int, default=1)
@@ -420,8 +503,15 @@ def main():
     p.add_argument("--calib-batches", type=int, default=0,
                    help="calibration batches accumulated before the timed steps (0 = the workload's own count); "
                         "profiling runs use a small number to keep the launch list short")
+    p.add_argument("--density-sweep", action="store_true",
+                   help="instead of the bench line: forward time vs kept fraction on the workload's shape")
     args = p.parse_args()
     w = inputs.WORKLOADS[args.workload]
+    if args.density_sweep:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+        run_density_sweep(args, w)
+        return
     if args.impl == "reference":
         run_reference(args, w)
         return
