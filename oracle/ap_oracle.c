@@ -11,6 +11,7 @@
  *                          caller, see below) with the attention matrix of
  *                          Section 3.1, softmax(Q K^T / sqrt(d_k)).
  *   oracle_build_mask      Eq. 2 read as an exact top-k selection per head.
+ *   oracle_build_mask_layer  Eq. 2 with one threshold for all heads of the layer.
  *   oracle_mask_to_tiles   the 128x128 tile list + bitmaps (an encoding of the
  *                          mask of Eq. 2; no counterpart in the paper).
  *   oracle_attention_fwd   the masked attention equation of Section 3.2,
@@ -187,6 +188,50 @@ int oracle_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac,
     free(e);
   }
   return failed ? -1 : 0;
+}
+
+/*
+ * Eq. 2 with one threshold for the whole layer, as the paper states it: the
+ * percentile is taken over the averaged attention matrices of ALL heads of the
+ * layer together, so heads keep unequal numbers of entries.  Read, like the
+ * per-head variant, as an exact top-k: the population is the union of the
+ * heads' domains (N = H * n_valid entries), the diagonals of all heads are
+ * forced (when keep_diag and Lq == Lk) and counted inside
+ *   k = max(#forced, min(N, floor(keep_frac * N + 0.5))),
+ * and the order is: forced first, then larger value, then lower global index
+ * (h * Lq + i) * Lk + j.  mask[h,i,j] = 1 for the first k entries; nnz[h] =
+ * entries kept in head h.  Returns 0, or -1 when an allocation fails.
+ */
+int oracle_build_mask_layer(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal,
+                            int keep_diag, uint8_t *mask, int64_t *nnz) {
+  memset(mask, 0, (size_t)H * Lq * Lk);
+  int64_t n_valid = 0;
+  for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lk, causal);
+  int64_t N = n_valid * H;
+  ap_entry *e = (ap_entry *)malloc(sizeof(ap_entry) * (size_t)(N > 0 ? N : 1));
+  if (!e) return -1;
+  int64_t n = 0, n_forced = 0;
+  for (int h = 0; h < H; ++h) {
+    nnz[h] = 0;
+    for (int i = 0; i < Lq; ++i) {
+      int jend = row_domain_end(i, Lk, causal);
+      for (int j = 0; j < jend; ++j) {
+        e[n].value = acc[((size_t)h * Lq + i) * Lk + j];
+        e[n].forced = (keep_diag && Lq == Lk && i == j) ? 1 : 0;
+        e[n].index = ((int64_t)h * Lq + i) * Lk + j;
+        n_forced += e[n].forced;
+        ++n;
+      }
+    }
+  }
+  int64_t k = oracle_keep_count(N, n_forced, keep_frac);
+  qsort(e, (size_t)n, sizeof(ap_entry), entry_before);
+  for (int64_t r = 0; r < k; ++r) {
+    mask[(size_t)e[r].index] = 1;
+    nnz[e[r].index / ((int64_t)Lq * Lk)] += 1;
+  }
+  free(e);
+  return 0;
 }
 
 /*

@@ -119,6 +119,24 @@ def build_mask(acc32, keep_frac: float, causal: bool = False, keep_diag: bool = 
     return mask, nnz
 
 
+def build_mask_layer(acc32, keep_frac: float, causal: bool = False, keep_diag: bool = True):
+    """Eq. 2 with one threshold for all heads of the layer (the paper's own statement), as an exact
+    top-k over the union of the heads' domains; returns (mask uint8 [H,Lq,Lk], nnz int64 [H])."""
+    acc32 = _f32(acc32)
+    H, Lq, Lk = acc32.shape
+    mask = np.zeros((H, Lq, Lk), dtype=np.uint8)
+    nnz = np.zeros((H,), dtype=np.int64)
+    lib = _load()
+    lib.oracle_build_mask_layer.restype = ctypes.c_int
+    rc = lib.oracle_build_mask_layer(
+        _p(acc32), H, Lq, Lk, ctypes.c_double(keep_frac), int(bool(causal)), int(bool(keep_diag)),
+        _p(mask), _p(nnz),
+    )
+    if rc != 0:
+        raise MemoryError("oracle_build_mask_layer")
+    return mask, nnz
+
+
 def mask_to_tiles(mask):
     """Tile list of a mask: dict(row_ptr, col_idx, flags, bitmap) trimmed to the T non-empty tiles."""
     mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))

@@ -278,6 +278,94 @@ def test_mask_invariants(causal):
     np.testing.assert_array_equal(prev, np.broadcast_to(dom, (H, L, L)).astype(np.uint8))
 
 
+# --- the per-layer threshold (one selection over all heads, as Eq. 2 is stated in the paper)
+
+
+def _brute_force_layer(acc, keep_frac, causal, keep_diag):
+    """Among all k-subsets of the union of the heads' domains that contain every head's forced
+    entries, the one with the largest exact sum; among those, the first in global index order."""
+    H, Lq, Lk = acc.shape
+    dom = [(h, i, j) for h in range(H) for (i, j) in _domain(Lq, Lk, causal)]
+    forced = [e for e in dom if keep_diag and Lq == Lk and e[1] == e[2]]
+    N = len(dom)
+    k = max(len(forced), min(N, int(math.floor(keep_frac * N + 0.5))))
+    free = [e for e in dom if e not in forced]
+    gidx = lambda e: (e[0] * Lq + e[1]) * Lk + e[2]
+    best, best_key = None, None
+    for combo in itertools.combinations(free, k - len(forced)):
+        chosen = sorted(forced + list(combo), key=gidx)
+        total = sum(Fraction(float(acc[e])) for e in chosen)
+        key = (-total, tuple(gidx(e) for e in chosen))
+        if best_key is None or key < best_key:
+            best, best_key = chosen, key
+    mask = np.zeros((H, Lq, Lk), dtype=np.uint8)
+    for e in best:
+        mask[e] = 1
+    return mask, k
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("keep_diag", [False, True])
+def test_layer_mask_brute_force_tiny(causal, keep_diag):
+    rng = np.random.default_rng(44)
+    for (H, L) in ((2, 2), (3, 2), (2, 3)):
+        for keep in (0.25, 0.5, 0.7):
+            for trial in range(4):
+                acc = rng.integers(0, 4, size=(H, L, L)).astype(np.float32) / 4.0  # many exact ties
+                want, k = _brute_force_layer(acc, keep, causal, keep_diag)
+                got, nnz = orc.build_mask_layer(acc, keep, causal=causal, keep_diag=keep_diag)
+                np.testing.assert_array_equal(got, want)
+                assert nnz.sum() == k and list(nnz) == [int(want[h].sum()) for h in range(H)]
+
+
+def test_layer_mask_is_the_per_head_selection_of_the_stacked_heads():
+    """Without causal or diagonal structure, one threshold over H heads of [Lq, Lk] is the per-head
+    rule applied to a single head of [H*Lq, Lk] (same population, same index order); with one
+    head the two rules coincide whatever the structure."""
+    rng = np.random.default_rng(45)
+    H, Lq, Lk = 3, 17, 23
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc.flat[::5] = 0.25  # ties
+    for keep in (0.1, 0.5, 0.93):
+        got, nnz = orc.build_mask_layer(acc, keep, causal=False, keep_diag=False)
+        want, k = orc.build_mask(acc.reshape(1, H * Lq, Lk), keep, causal=False, keep_diag=False)
+        np.testing.assert_array_equal(got.reshape(1, H * Lq, Lk), want)
+        assert nnz.sum() == k[0]
+    one = rng.random((1, 19, 19), dtype=np.float32)
+    for causal in (False, True):
+        a, na = orc.build_mask_layer(one, 0.3, causal=causal, keep_diag=True)
+        b, nb = orc.build_mask(one, 0.3, causal=causal, keep_diag=True)
+        np.testing.assert_array_equal(a, b)
+        assert list(na) == list(nb)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_layer_mask_invariants(causal):
+    rng = np.random.default_rng(46)
+    H, L = 4, 41
+    acc = rng.random((H, L, L), dtype=np.float32) * np.array([1.0, 2.0, 0.5, 1.5], dtype=np.float32)[:, None, None]
+    dom = np.tril(np.ones((L, L), dtype=bool)) if causal else np.ones((L, L), dtype=bool)
+    N = int(dom.sum()) * H
+    off = ~np.eye(L, dtype=bool)
+    prev = None
+    for keep in (0.05, 0.2, 0.5, 0.9, 1.0):
+        mask, nnz = orc.build_mask_layer(acc, keep, causal=causal, keep_diag=True)
+        k = max(H * L, min(N, int(math.floor(keep * N + 0.5))))
+        m = mask.astype(bool)
+        assert m.sum() == k == nnz.sum()                      # the kept fraction of the LAYER is exact
+        assert [int(m[h].sum()) for h in range(H)] == list(nnz)
+        assert not m[:, ~dom].any()                           # never outside the domain
+        assert m[:, np.arange(L), np.arange(L)].all()         # every head's diagonal forced
+        kept_free, pruned = acc[m & off[None]], acc[~m & dom[None]]
+        if kept_free.size and pruned.size:
+            assert kept_free.min() >= pruned.max()            # one threshold across all heads
+        if keep < 1.0:
+            assert nnz[1] > nnz[2]                            # the head with larger values keeps more
+        if prev is not None:
+            assert np.all(prev <= mask)
+        prev = mask
+
+
 def test_mask_constant_acc_keeps_forced_then_first_indices():
     L = 6
     acc = np.full((1, L, L), 0.125, dtype=np.float32)
