@@ -159,6 +159,21 @@ ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_fra
                         void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Eq. 2 as the paper states it: ONE threshold for all H heads passed in (the heads of one
+ * layer), i.e. an exact top-k over the union of the heads' domains, so that heads keep unequal
+ * numbers of entries.  Same arguments, outputs and conventions as ap_build_mask with
+ *   domain  the union over h of head h's domain; N = H * n_valid entries
+ *   forced  every head's diagonal when keep_diag != 0 and Lq == Lk (counted inside k)
+ *   k       max(#forced, min(N, floor(keep_frac*N + 0.5))), in double
+ *   order   forced first, then larger fp32 value, then lower index (h*Lq + i)*Lk + j
+ *   nnz_per_head[h]  entries kept in head h (they sum to k)
+ * Needs H*Lq*Lk < 2^32 (AP_ERR_UNSUPPORTED otherwise).
+ */
+ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal,
+                              int keep_diag, uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Tile list of an arbitrary element mask (uint8 [H,Lq,Lk], non-zero = kept):
  * the same encoding ap_build_mask emits, for masks made elsewhere (random
  * masks as in the paper's control experiment, all-ones, hand-made).

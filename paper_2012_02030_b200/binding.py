@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
         "ap_mask_to_tiles_workspace_bytes": (sz, [i, i, i]),
         "ap_accumulate_attention": (i, [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp]),
         "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
+        "ap_build_mask_layer": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_mask_to_tiles": (i, [vp, i, i, i, tp, vp, sz, vp]),
         "ap_dense_tiles": (i, [i, i, i, i, tp, vp]),
         "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
@@ -71,7 +72,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
-           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask",
+           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
            "ap_sparse_attention_fwd_host", "ap_device_status")
 
@@ -187,18 +188,28 @@ def ap_accumulate_attention(acc, Q, K, bias=None, causal=False, scale=0.0, strea
            "ap_accumulate_attention")
 
 
-def ap_build_mask(acc, keep_frac, causal=False, keep_diag=True, mask=None, tiles: Tiles | None = None,
-                  nnz_per_head=None, workspace=None, stream=None) -> None:
+def _build_mask(fn, name, acc, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head, workspace, stream) -> None:
     _dev(acc, "acc")
     H, Lq, Lk = acc.shape
     if acc.dtype != torch.float32:
         raise ValueError("acc must be float32")
     if workspace is None:
         workspace = torch.empty(ap_build_mask_workspace_bytes(H, Lq, Lk), dtype=torch.uint8, device=acc.device)
-    _check(lib.ap_build_mask(_ptr(acc), H, Lq, Lk, float(keep_frac), int(bool(causal)), int(bool(keep_diag)),
-                             _ptr(mask), ctypes.byref(tiles.c) if tiles is not None else None,
-                             _ptr(nnz_per_head), _ptr(workspace), workspace.numel(), _stream(stream)),
-           "ap_build_mask")
+    _check(fn(_ptr(acc), H, Lq, Lk, float(keep_frac), int(bool(causal)), int(bool(keep_diag)),
+              _ptr(mask), ctypes.byref(tiles.c) if tiles is not None else None,
+              _ptr(nnz_per_head), _ptr(workspace), workspace.numel(), _stream(stream)), name)
+
+
+def ap_build_mask(acc, keep_frac, causal=False, keep_diag=True, mask=None, tiles: Tiles | None = None,
+                  nnz_per_head=None, workspace=None, stream=None) -> None:
+    _build_mask(lib.ap_build_mask, "ap_build_mask", acc, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head,
+                workspace, stream)
+
+
+def ap_build_mask_layer(acc, keep_frac, causal=False, keep_diag=True, mask=None, tiles: Tiles | None = None,
+                        nnz_per_head=None, workspace=None, stream=None) -> None:
+    _build_mask(lib.ap_build_mask_layer, "ap_build_mask_layer", acc, keep_frac, causal, keep_diag, mask, tiles,
+                nnz_per_head, workspace, stream)
 
 
 def ap_mask_to_tiles(mask, tiles: Tiles, workspace=None, stream=None) -> None:

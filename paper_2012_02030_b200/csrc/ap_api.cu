@@ -141,9 +141,10 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
-ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
-                        uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
-                        size_t workspace_bytes, void *stream) {
+namespace {
+ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
+                          uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
+                          size_t workspace_bytes, void *stream, int per_layer) {
   if (!acc || !aligned16(acc) || !shape_ok(H, Lq, Lk) || (causal && Lq != Lk)) return AP_ERR_INVALID_ARG;
   if (!(keep_frac > 0.0) || !(keep_frac <= 1.0)) return AP_ERR_INVALID_ARG;
   if (mask && !aligned16(mask)) return AP_ERR_INVALID_ARG;
@@ -154,6 +155,8 @@ ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_fra
   }
   if (!workspace || !aligned16(workspace)) return AP_ERR_INVALID_ARG;
   if (workspace_bytes < ap_build_mask_workspace_bytes(H, Lq, Lk)) return AP_ERR_WORKSPACE;
+  // the selection over a whole layer ranks ties by a 32-bit global index (h*Lq + i)*Lk + j
+  if (per_layer && (int64_t)H * Lq * Lk > (int64_t)0xffffffffLL) return AP_ERR_UNSUPPORTED;
   if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -165,8 +168,11 @@ ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_fra
   a.H = H; a.Lq = Lq; a.Lk = Lk;
   a.causal = causal ? 1 : 0;
   a.keep_diag = keep_diag ? 1 : 0;
-  const int64_t n_valid = domain_size(Lq, Lk, a.causal);
-  const int64_t n_forced = (a.keep_diag && Lq == Lk) ? Lq : 0;
+  a.per_layer = per_layer;
+  // population of one selection: a head's domain, or the union of the heads' domains
+  const int64_t heads = per_layer ? H : 1;
+  const int64_t n_valid = domain_size(Lq, Lk, a.causal) * heads;
+  const int64_t n_forced = ((a.keep_diag && Lq == Lk) ? Lq : 0) * heads;
   a.k = keep_count(n_valid, n_forced, keep_frac);
   a.k_rest = a.k - n_forced;
   a.mask = mask;
@@ -180,6 +186,21 @@ ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_fra
     if (launch_compact_tiles(a.stage_bitmap, a.stage_count, *tiles, s) != cudaSuccess) return AP_ERR_CUDA;
   }
   return AP_OK;
+}
+}  // namespace
+
+ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
+                        uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
+                        size_t workspace_bytes, void *stream) {
+  return build_mask_impl(acc, H, Lq, Lk, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head, workspace,
+                         workspace_bytes, stream, 0);
+}
+
+ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
+                              uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
+                              size_t workspace_bytes, void *stream) {
+  return build_mask_impl(acc, H, Lq, Lk, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head, workspace,
+                         workspace_bytes, stream, 1);
 }
 
 ap_status ap_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles *tiles, void *workspace,

@@ -15,6 +15,12 @@
 // are kept.  The emit pass writes the element mask and per-tile bitmaps;
 // ap_tiles.cu compacts them.  Integer work throughout: no floating-point
 // arithmetic decides a bit.
+//
+// One threshold for the whole layer (Eq. 2 as stated) is the same selection run
+// once over a virtual head of H*Lq rows: row i' = h*Lq + i has the domain of row
+// i, and the linear index i'*Lk + j is the layer-wide tie order.  Its collected
+// keys are too many for one CTA, so the threshold is selected among them with
+// grid-wide histogram passes instead.
 #include "ap_common.cuh"
 
 namespace ap {
@@ -51,15 +57,21 @@ struct SelectState {  // per head
   // when not all entries equal to thr are kept: those with linear index i*Lk + j <= tie_cut are
   // (valid if have_cut; otherwise the ties are ranked with tie counts and a prefix sum)
   uint32_t tie_cut, have_cut;
+  // selection among the collected keys with grid-wide passes (one threshold for the layer)
+  uint32_t cand_select;          // the bracket holds the threshold: the passes over the collected keys run
+  uint32_t thr_count;            // entries equal to the threshold key
+  uint32_t tie_n;                // entries gathered in the tie list
 };
+
+constexpr int kMaxCutTies = 4096;  // ties with the threshold ranked inside the shortcut (more: tie counts + scan)
 
 struct Scratch {
   uint32_t *hist;       // [H][kBins]
   SelectState *state;   // [H]
   uint32_t *tie_count;  // [H][Lq][n_kt] -> exclusive prefix after the scan
+  uint32_t *tie_list;   // [kMaxCutTies] linear indices of the entries equal to the threshold (layer selection)
   uint2 *cand;          // [H][cand_cap] (key, linear index) of the entries collected by the shortcut
 };
-constexpr int kMaxCutTies = 4096;  // ties with the threshold ranked inside the shortcut (more: tie counts + scan)
 
 // The shortcut is tried for heads of at least this many selectable entries.
 constexpr long long kShortcutMinEntries = 1ll << 20;
@@ -82,11 +94,13 @@ __device__ __forceinline__ void load4(const float *__restrict__ row, int j0, int
   }
 }
 
-__global__ void init_state_kernel(SelectState *state, uint32_t *hist, int H, unsigned long long k_rest,
-                                  long long k, int64_t *nnz) {
+// n_sel selections (one per head, or one for the layer); nnz[H] starts at nnz_init.
+__global__ void init_state_kernel(SelectState *state, uint32_t *hist, int n_sel, unsigned long long k_rest, int H,
+                                  long long nnz_init, int64_t *nnz) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx < H * kBins) hist[idx] = 0u;
-  if (idx < H) {
+  if (idx < n_sel * kBins) hist[idx] = 0u;
+  if (nnz && idx < H) nnz[idx] = nnz_init;
+  if (idx < n_sel) {
     state[idx].prefix = 0u;
     state[idx].thr = 0xffffffffu;
     state[idx].remaining = k_rest;
@@ -100,15 +114,19 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int H, uns
     state[idx].use_shortcut = 0u;
     state[idx].tie_cut = 0u;
     state[idx].have_cut = 0u;
-    if (nnz) nnz[idx] = k;
+    state[idx].cand_select = 0u;
+    state[idx].thr_count = 0u;
+    state[idx].tie_n = 0u;
   }
 }
 
 // Histogram of one digit over the non-forced domain entries whose higher digits
-// equal the prefix found so far.  grid = (row blocks, H); a warp takes a row at
+// equal the prefix found so far.  grid = (row blocks, selections); a warp takes a row at
 // a time and its lanes stride over the row, two float4 loads in flight each.
+// Here and in the kernels below Lq counts the rows of the selection and row i has
+// the domain of row i % period of a head (period == Lq unless heads are stacked).
 __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *__restrict__ acc, int Lq, int Lk,
-                                                                   int causal, int diag, int pass,
+                                                                   int period, int causal, int diag, int pass,
                                                                    const SelectState *__restrict__ state,
                                                                    uint32_t *__restrict__ hist) {
   __shared__ uint32_t sh[kBins];
@@ -125,7 +143,8 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
   const bool vec = (Lk & 3) == 0;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
-    const int jend = causal ? min(Lk, i + 1) : Lk;
+    const int ii = i % period;
+    const int jend = causal ? min(Lk, ii + 1) : Lk;
     for (int base = 0; base < jend; base += 256) {  // warp-uniform trip count
       float v[2][4];
 #pragma unroll
@@ -141,7 +160,7 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
         for (int c = 0; c < 4; ++c) {
           const int j = j0 + c;
           const uint32_t key = key_of(v[u][c]);
-          const bool take = j < jend && !(diag && j == i) && ((key & hi_mask) == want_hi);
+          const bool take = j < jend && !(diag && j == ii) && ((key & hi_mask) == want_hi);
           const uint32_t bin = (key >> shift) & dmask;
           // lanes that hit the same bin elect one to add their count
           const unsigned voters = __ballot_sync(0xffffffffu, take);
@@ -163,10 +182,11 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
 // One CTA per head: picks the digit whose bin contains the wanted rank.  Thread t
 // owns bins [kBins-1-8t, kBins-8-8t] (descending); a block-wide prefix over the
 // threads' sums locates the owner, which then walks its eight bins.
-__global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass) {
+// from_cand: the histogram came from the collected keys (offsets from the lower pivot).
+__global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass, int from_cand) {
   __shared__ uint32_t warp_sums[8];
   const int h = blockIdx.x;
-  if (state[h].done) return;  // resolved by the shortcut
+  if (from_cand ? !state[h].cand_select : state[h].done) return;  // no such passes / resolved by the shortcut
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t cnt[8];
   uint32_t mine = 0u;
@@ -206,6 +226,7 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
       out.thr = out.prefix;
       out.ties_kept = out.remaining;
       out.all_ties_kept = out.remaining == cnt[e] ? 1u : 0u;
+      out.thr_count = cnt[e];
     }
     state[h] = out;
   }
@@ -289,8 +310,8 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
 }
 
 // One CTA per head: samples the head and sets the bracket [lo, hi] around the expected threshold.
-__global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__restrict__ acc, int Lq, int Lk, int causal,
-                                                             int diag, unsigned long long k_rest,
+__global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
+                                                             int causal, int diag, unsigned long long k_rest,
                                                              unsigned long long n_rest, SelectState *state) {
   extern __shared__ uint32_t sm_dyn[];
   uint32_t *keys = sm_dyn;               // kSamples
@@ -304,7 +325,8 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
   for (int s = t; s < kSamples; s += 1024) {
     const unsigned long long idx = mix64(((unsigned long long)h << 32) | (unsigned)s) % cells;
     const int i = (int)(idx / Lk), j = (int)(idx % Lk);
-    if ((causal && j > i) || (diag && j == i)) continue;
+    const int ii = i % period;
+    if ((causal && j > ii) || (diag && j == ii)) continue;
     const uint32_t pos = atomicAdd(&n_valid_s, 1u);
     keys[pos] = key_of(acc[((size_t)h * Lq + i) * Lk + j]);
   }
@@ -331,9 +353,9 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
 // shared memory and appended to the head's buffer with one reservation per CTA (keys that do not
 // fit the stage any more are appended one warp at a time).
 constexpr int kStageKeys = 4096;
-__global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restrict__ acc, int Lq, int Lk, int causal,
-                                                           int diag, SelectState *state, uint2 *__restrict__ cand,
-                                                           uint32_t cand_cap) {
+__global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
+                                                           int causal, int diag, SelectState *state,
+                                                           uint2 *__restrict__ cand, uint32_t cand_cap) {
   __shared__ uint2 stage[kStageKeys];
   __shared__ uint32_t stage_n, stage_base;  // stage_n only grows; positions beyond the stage were not staged
   const int h = blockIdx.y;
@@ -347,7 +369,8 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
   unsigned long long above = 0ull;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
-    const int jend = causal ? min(Lk, i + 1) : Lk;
+    const int ii = i % period;
+    const int jend = causal ? min(Lk, ii + 1) : Lk;
     for (int base = 0; base < jend; base += 512) {  // warp-uniform trip count
       float v[4][4];
 #pragma unroll
@@ -363,7 +386,7 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
         for (int c = 0; c < 4; ++c) {
           const int j = j0 + c;
           const uint32_t key = key_of(v[u][c]);
-          const bool in = j < jend && !(diag && j == i);
+          const bool in = j < jend && !(diag && j == ii);
           above += (in && key > hi) ? 1u : 0u;
           if (in && key >= lo && key <= hi) {  // a few per cent of the entries
             const uint2 entry = make_uint2(key, (uint32_t)i * (uint32_t)Lk + (uint32_t)j);
@@ -392,6 +415,18 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
     if (dst + e < cand_cap) out[dst + e] = stage[e];
 }
 
+// Ranks `count` <= kMaxCutTies distinct linear indices: returns (in *cut_s, after a barrier) the one
+// with exactly rank - 1 smaller ones.  CTA of 1024 threads.
+__device__ void rank_ties(const uint32_t *tie_idx, uint32_t count, uint32_t rank, uint32_t *cut_s) {
+  for (uint32_t e = threadIdx.x; e < count; e += 1024) {
+    const uint32_t me = tie_idx[e];
+    uint32_t smaller = 0u;
+    for (uint32_t f = 0; f < count; ++f) smaller += tie_idx[f] < me ? 1u : 0u;
+    if (smaller == rank - 1u) *cut_s = me;
+  }
+  __syncthreads();
+}
+
 // One CTA per head: if the bracket holds the threshold, selects it among the collected keys.
 __global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *state, const uint2 *__restrict__ cand,
                                                                  uint32_t cand_cap, unsigned long long k_rest) {
@@ -418,14 +453,7 @@ __global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *st
       if (c.x == p.key) tie_idx[atomicAdd(&tie_n, 1u)] = c.y;
     }
     __syncthreads();
-    // the index with exactly rank_in_ties - 1 smaller ones (indices are distinct)
-    for (uint32_t e = threadIdx.x; e < p.count; e += 1024) {
-      const uint32_t me = tie_idx[e];
-      uint32_t smaller = 0u;
-      for (uint32_t f = 0; f < p.count; ++f) smaller += tie_idx[f] < me ? 1u : 0u;
-      if (smaller == p.rank_in_ties - 1u) cut_s = me;
-    }
-    __syncthreads();
+    rank_ties(tie_idx, p.count, p.rank_in_ties, &cut_s);
     have_cut = true;
   }
   if (threadIdx.x == 0) {
@@ -440,10 +468,92 @@ __global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *st
   }
 }
 
+// ---- the same selection among the collected keys with grid-wide passes (selection 0 only) -----
+
+// Decides whether the bracket holds the threshold; if so the digit passes below run on the
+// collected keys' offsets from the lower pivot, else the selection takes the three full passes.
+__global__ void cand_begin_kernel(SelectState *state, uint32_t cand_cap, unsigned long long k_rest) {
+  const SelectState st = state[0];
+  if (!st.use_shortcut) return;
+  if (st.n_cand > cand_cap || st.above_hi >= k_rest || k_rest - st.above_hi > st.n_cand) return;
+  state[0].remaining = k_rest - st.above_hi;
+  state[0].prefix = 0u;
+  state[0].cand_select = 1u;
+}
+
+__global__ void __launch_bounds__(kThreads) cand_histogram_kernel(const SelectState *__restrict__ state,
+                                                                  const uint2 *__restrict__ cand, int pass,
+                                                                  uint32_t *__restrict__ hist) {
+  __shared__ uint32_t sh[kBins];
+  if (!state[0].cand_select) return;
+  const int lane = threadIdx.x & 31;
+  for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0u;
+  __syncthreads();
+  const int shift = digit_shift(pass);
+  const uint32_t dmask = digit_mask(pass);
+  const uint32_t hi_mask = pass == 0 ? 0u : ~((1u << (shift + (pass == 1 ? 11 : 10))) - 1u);
+  const uint32_t want_hi = state[0].prefix & hi_mask;
+  const uint32_t n = state[0].n_cand, lo = state[0].lo;
+  for (uint32_t base = blockIdx.x * kThreads; base < n; base += gridDim.x * kThreads) {  // warp-uniform
+    const uint32_t idx = base + threadIdx.x;
+    const uint32_t key = idx < n ? cand[idx].x - lo : 0u;
+    const bool take = idx < n && (key & hi_mask) == want_hi;
+    const uint32_t bin = (key >> shift) & dmask;
+    const unsigned voters = __ballot_sync(0xffffffffu, take);
+    if (take) {
+      const unsigned peers = __match_any_sync(voters, bin);
+      if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], (uint32_t)__popc(peers));
+    }
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < kBins; b += kThreads) {
+    const uint32_t s = sh[b];
+    if (s) atomicAdd(&hist[b], s);
+  }
+}
+
+// Gathers the linear indices of the collected entries equal to the threshold, when they must be
+// ranked and are few enough.
+__global__ void __launch_bounds__(kThreads) cand_ties_kernel(SelectState *state, const uint2 *__restrict__ cand,
+                                                             uint32_t *__restrict__ tie_list) {
+  const SelectState st = state[0];
+  if (!st.cand_select || st.all_ties_kept || st.thr_count > (uint32_t)kMaxCutTies) return;
+  const uint32_t want = st.prefix + st.lo;
+  for (uint32_t idx = blockIdx.x * kThreads + threadIdx.x; idx < st.n_cand; idx += gridDim.x * kThreads) {
+    const uint2 c = cand[idx];
+    if (c.x == want) {
+      const uint32_t pos = atomicAdd(&state[0].tie_n, 1u);
+      if (pos < (uint32_t)kMaxCutTies) tie_list[pos] = c.y;
+    }
+  }
+}
+
+// One CTA: turns the digits found among the collected keys into the threshold and closes the selection.
+__global__ void __launch_bounds__(1024) cand_finish_kernel(SelectState *state, const uint32_t *__restrict__ tie_list) {
+  __shared__ uint32_t tie_idx[kMaxCutTies];
+  __shared__ uint32_t cut_s;
+  const SelectState st = state[0];
+  if (!st.cand_select) return;
+  bool have_cut = false;
+  if (!st.all_ties_kept && st.thr_count <= (uint32_t)kMaxCutTies) {
+    for (uint32_t e = threadIdx.x; e < st.thr_count; e += 1024) tie_idx[e] = tie_list[e];
+    __syncthreads();
+    rank_ties(tie_idx, st.thr_count, (uint32_t)st.ties_kept, &cut_s);
+    have_cut = true;
+  }
+  if (threadIdx.x == 0) {
+    state[0].tie_cut = have_cut ? cut_s : 0u;
+    state[0].have_cut = have_cut ? 1u : 0u;
+    state[0].thr = st.prefix + st.lo;
+    state[0].prefix = st.prefix + st.lo;
+    state[0].done = 1u;
+  }
+}
+
 // Entries equal to the threshold key per (row, 128-column segment); only for heads
 // where the ties must be ranked.  grid = (row blocks, H); a warp takes a row.
-__global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_kt,
-                                                             int causal, int diag,
+__global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
+                                                             int n_kt, int causal, int diag,
                                                              const SelectState *__restrict__ state,
                                                              uint32_t *__restrict__ tie_count) {
   const int h = blockIdx.y;
@@ -453,7 +563,8 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
   const bool vec = (Lk & 3) == 0;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
-    const int jend = causal ? min(Lk, i + 1) : Lk;
+    const int ii = i % period;
+    const int jend = causal ? min(Lk, ii + 1) : Lk;
     for (int kt = 0; kt < n_kt; ++kt) {
       const int j0 = kt * kTile + 4 * lane;
       int ties = 0;
@@ -463,7 +574,7 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           const int j = j0 + c;
-          ties += (j < jend && !(diag && j == i) && key_of(v[c]) == thr) ? 1 : 0;
+          ties += (j < jend && !(diag && j == ii) && key_of(v[c]) == thr) ? 1 : 0;
         }
       }
 #pragma unroll
@@ -514,22 +625,27 @@ __global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ t
 
 // One CTA per tile of the (h, qt, kt) grid; warp w takes tile rows w, w+4, ...
 // (four rows loaded ahead) and each lane four consecutive columns.  Writes the
-// element mask, the tile's bitmap and popcount into the staging area.
+// element mask, the tile's bitmap and popcount into the staging area.  per_layer:
+// all heads share selection 0, ties are ordered by (h*Lq + i)*Lk + j, and the
+// tiles' popcounts are added up into nnz[h].
 __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_qt, int n_kt,
-                                                   int causal, int diag, const SelectState *__restrict__ state,
+                                                   int causal, int diag, int per_layer,
+                                                   const SelectState *__restrict__ state,
                                                    const uint32_t *__restrict__ tie_prefix,
                                                    uint8_t *__restrict__ mask, uint32_t *__restrict__ stage_bitmap,
-                                                   int32_t *__restrict__ stage_count) {
+                                                   int32_t *__restrict__ stage_count, int64_t *__restrict__ nnz) {
   const int tile = blockIdx.x;
   const int kt = tile % n_kt;
   const int qt = (tile / n_kt) % n_qt;
   const int h = tile / (n_kt * n_qt);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t thr = state[h].thr;
-  const unsigned long long ties_kept = state[h].ties_kept;
-  const bool all_ties = state[h].all_ties_kept != 0u;
-  const bool have_cut = state[h].have_cut != 0u;
-  const uint32_t tie_cut = state[h].tie_cut;
+  const int sel = per_layer ? 0 : h;
+  const uint32_t thr = state[sel].thr;
+  const unsigned long long ties_kept = state[sel].ties_kept;
+  const bool all_ties = state[sel].all_ties_kept != 0u;
+  const bool have_cut = state[sel].have_cut != 0u;
+  const uint32_t tie_cut = state[sel].tie_cut;
+  const uint32_t first_row = per_layer ? (uint32_t)h * (uint32_t)Lq : 0u;  // of this head in the tie order
   const bool vec = (Lk & 3) == 0;
   const int j0 = kt * kTile + 4 * lane;
   __shared__ int warp_count[4];
@@ -591,7 +707,8 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
         } else if (have_cut) {
 #pragma unroll
           for (int c = 0; c < 4; ++c)
-            if ((tie_bits & (1u << c)) && (uint32_t)i * (uint32_t)Lk + (uint32_t)(j0 + c) <= tie_cut) nib |= 1u << c;
+            if ((tie_bits & (1u << c)) && (first_row + (uint32_t)i) * (uint32_t)Lk + (uint32_t)(j0 + c) <= tie_cut)
+              nib |= 1u << c;
         } else if (__any_sync(0xffffffffu, tie_bits != 0u)) {
           // rank of each tie in linear-index order = ties before this row segment
           // + ties in lower lanes + ties in lower columns of this lane
@@ -637,8 +754,12 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   }
   if (lane == 0) warp_count[warp] = count;
   __syncthreads();
-  if (stage_count && threadIdx.x == 0)
-    stage_count[tile] = warp_count[0] + warp_count[1] + warp_count[2] + warp_count[3];
+  if (threadIdx.x == 0) {
+    const int total = warp_count[0] + warp_count[1] + warp_count[2] + warp_count[3];
+    if (stage_count) stage_count[tile] = total;
+    if (per_layer && nnz && total)
+      atomicAdd(reinterpret_cast<unsigned long long *>(nnz + h), (unsigned long long)total);
+  }
 }
 
 Scratch carve(void *scratch, int H, int Lq, int Lk) {
@@ -650,6 +771,8 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
   p += align256((size_t)H * sizeof(SelectState));
   s.tie_count = reinterpret_cast<uint32_t *>(p);
   p += align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t));
+  s.tie_list = reinterpret_cast<uint32_t *>(p);
+  p += align256((size_t)kMaxCutTies * sizeof(uint32_t));
   s.cand = reinterpret_cast<uint2 *>(p);
   return s;
 }
@@ -657,60 +780,84 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
 }  // namespace
 
 size_t select_scratch_bytes(int H, int Lq, int Lk) {
-  // the candidate buffer is sized for the larger of the causal and the full domain
+  // the candidate buffer is sized for the larger of the causal and the full domain, and for one
+  // selection over all heads (never smaller than H selections of one head each)
   return align256((size_t)H * kBins * sizeof(uint32_t)) + align256((size_t)H * sizeof(SelectState)) +
          align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t)) +
-         align256((size_t)H * (size_t)cand_capacity((long long)Lq * Lk) * sizeof(uint2));
+         align256((size_t)kMaxCutTies * sizeof(uint32_t)) +
+         align256((size_t)cand_capacity((long long)H * Lq * Lk) * sizeof(uint2));
 }
 
 cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   const int n_qt = ceil_div(a.Lq, kTile), n_kt = ceil_div(a.Lk, kTile);
   const int diag = (a.keep_diag && a.Lq == a.Lk) ? 1 : 0;
   Scratch sc = carve(a.scratch, a.H, a.Lq, a.Lk);
+  // the selections: one per head over Lq rows, or one over the H*Lq rows of the layer
+  const int n_sel = a.per_layer ? 1 : a.H;
+  const int rows = a.per_layer ? a.H * a.Lq : a.Lq;
+  const int period = a.Lq;
   cudaError_t e;
-  init_state_kernel<<<ceil_div(a.H * kBins, 256), 256, 0, s>>>(sc.state, sc.hist, a.H,
-                                                              (unsigned long long)a.k_rest, (long long)a.k, a.nnz);
+  // per head nnz = k; per layer the emit pass counts it
+  init_state_kernel<<<ceil_div(max(n_sel * kBins, a.H), 256), 256, 0, s>>>(
+      sc.state, sc.hist, n_sel, (unsigned long long)a.k_rest, a.H, a.per_layer ? 0ll : (long long)a.k, a.nnz);
   count_launches(1);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  // enough CTAs per head to fill the GPU, at most one warp-row each
-  int row_blocks = ceil_div(a.Lq, kWarps);
-  const int want = ceil_div(148 * 8, a.H);
+  // enough CTAs per selection to fill the GPU, at most one warp-row each
+  int row_blocks = ceil_div(rows, kWarps);
+  const int want = ceil_div(148 * 8, n_sel);
   if (row_blocks > want) row_blocks = want;
-  dim3 grid(row_blocks, a.H);
+  dim3 grid(row_blocks, n_sel);
   if (a.k_rest > 0) {
-    // large heads: the one-pass shortcut first (heads it resolves skip the three passes below)
+    // large selections: the one-pass shortcut first (those it resolves skip the three passes below)
     const long long n_valid = a.causal ? (long long)a.Lq * (a.Lq + 1) / 2 : (long long)a.Lq * a.Lk;
-    const long long n_rest = n_valid - (diag ? a.Lq : 0);
+    const long long n_rest = (n_valid - (diag ? a.Lq : 0)) * (a.per_layer ? a.H : 1);
     const long long cap = cand_capacity(n_rest);
     if (cap > 0) {
       const size_t smem = (kSamples + kBins) * sizeof(uint32_t);
       e = cudaFuncSetAttribute(sample_pivots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      sample_pivots_kernel<<<a.H, 1024, smem, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, (unsigned long long)a.k_rest,
-                                                   (unsigned long long)n_rest, sc.state);
-      collect_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, sc.state, sc.cand, (uint32_t)cap);
-      select_candidates_kernel<<<a.H, 1024, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, (unsigned long long)a.k_rest);
-      count_launches(3);
+      sample_pivots_kernel<<<n_sel, 1024, smem, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
+                                                     (unsigned long long)a.k_rest, (unsigned long long)n_rest, sc.state);
+      collect_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag, sc.state, sc.cand,
+                                               (uint32_t)cap);
+      count_launches(2);
+      if (!a.per_layer) {
+        select_candidates_kernel<<<n_sel, 1024, 0, s>>>(sc.state, sc.cand, (uint32_t)cap,
+                                                        (unsigned long long)a.k_rest);
+        count_launches(1);
+      } else {
+        const int cand_grid = 148 * 4;
+        cand_begin_kernel<<<1, 1, 0, s>>>(sc.state, (uint32_t)cap, (unsigned long long)a.k_rest);
+        for (int pass = 0; pass < kPasses; ++pass) {
+          cand_histogram_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, pass, sc.hist);
+          pick_digit_kernel<<<1, 256, 0, s>>>(sc.state, sc.hist, pass, 1);
+        }
+        cand_ties_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, sc.tie_list);
+        cand_finish_kernel<<<1, 1024, 0, s>>>(sc.state, sc.tie_list);
+        count_launches(3 + 2 * kPasses);
+      }
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     for (int pass = 0; pass < kPasses; ++pass) {
-      digit_histogram_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, a.causal, diag, pass, sc.state, sc.hist);
+      digit_histogram_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag, pass, sc.state,
+                                                       sc.hist);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
-      pick_digit_kernel<<<a.H, 256, 0, s>>>(sc.state, sc.hist, pass);
+      pick_digit_kernel<<<n_sel, 256, 0, s>>>(sc.state, sc.hist, pass, 0);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    // both return at once for heads whose ties with the threshold are all kept
-    tie_count_kernel<<<grid, kThreads, 0, s>>>(a.acc, a.Lq, a.Lk, n_kt, a.causal, diag, sc.state, sc.tie_count);
+    // both return at once for selections whose ties with the threshold are all kept
+    tie_count_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, n_kt, a.causal, diag, sc.state,
+                                               sc.tie_count);
     count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    tie_scan_kernel<<<a.H, 1024, 0, s>>>(sc.tie_count, a.Lq * n_kt, sc.state);
+    tie_scan_kernel<<<n_sel, 1024, 0, s>>>(sc.tie_count, rows * n_kt, sc.state);
     count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, sc.state,
-                                                sc.tie_count, a.mask, a.stage_bitmap, a.stage_count);
+  emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer, sc.state,
+                                                sc.tie_count, a.mask, a.stage_bitmap, a.stage_count, a.nnz);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -45,8 +45,9 @@ size_t stage_bytes(int H, int Lq, int Lk);
 struct BuildMaskArgs {
   const float *acc;
   int H, Lq, Lk, causal, keep_diag;
-  int64_t k_rest;  // entries to select among the non-forced domain entries
-  int64_t k;       // entries kept per head
+  int per_layer;   // one selection over all heads instead of one per head
+  int64_t k_rest;  // entries to select among the non-forced entries of the selection's population
+  int64_t k;       // entries kept per selection (per head, or in the whole layer)
   uint8_t *mask;   // may be NULL
   int64_t *nnz;    // may be NULL
   uint32_t *stage_bitmap;  // may be NULL (no tile list wanted)

@@ -99,11 +99,12 @@ def oracle_accumulate(w, n_batches, bias):
     return acc64
 
 
-def gpu_build_mask(ap, acc_dev, w, want_tiles=True):
+def gpu_build_mask(ap, acc_dev, w, want_tiles=True, layer=False):
     H, Lq, Lk = acc_dev.shape
     mask = torch.full((H, Lq, Lk), 7, dtype=torch.uint8, device="cuda")  # poison: every byte must be written
     nnz = torch.full((H,), -1, dtype=torch.int64, device="cuda")
     tiles = ap.Tiles(H, Lq, Lk) if want_tiles else None
-    ap.ap_build_mask(acc_dev, w.keep_frac, w.causal, w.keep_diag, mask, tiles, nnz)
+    build = ap.ap_build_mask_layer if layer else ap.ap_build_mask
+    build(acc_dev, w.keep_frac, w.causal, w.keep_diag, mask, tiles, nnz)
     assert ap.ap_device_status() == ap.AP_OK
     return mask, tiles, nnz

@@ -81,20 +81,24 @@ def test_accumulate_and_mask_reject_bad_arguments():
     assert f(FAKE, FAKE, FAKE, FAKE + 4, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 9, 64, 1, 1, 0.0, None) == ap.AP_ERR_INVALID_ARG  # causal, Lq != Lk
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 32, 1, 0, 0.0, None) == ap.AP_ERR_UNSUPPORTED
-    g = ap.lib.ap_build_mask
     t = _tiles(H=1, Lq=8, Lk=8, cap=1)
     ws = ap.ap_build_mask_workspace_bytes(1, 8, 8)
-    base = [FAKE, 1, 8, 8, 0.5, 0, 1, FAKE, ctypes.byref(t), FAKE, FAKE, ws, None]
-    for idx, val in ((0, None), (4, 0.0), (4, 1.5), (4, float("nan")), (10, None), (7, FAKE + 1)):
+    for g in (ap.lib.ap_build_mask, ap.lib.ap_build_mask_layer):
+        base = [FAKE, 1, 8, 8, 0.5, 0, 1, FAKE, ctypes.byref(t), FAKE, FAKE, ws, None]
+        for idx, val in ((0, None), (4, 0.0), (4, 1.5), (4, float("nan")), (10, None), (7, FAKE + 1)):
+            a = list(base)
+            a[idx] = val
+            assert g(*a) == ap.AP_ERR_INVALID_ARG, (idx, val)
         a = list(base)
-        a[idx] = val
-        assert g(*a) == ap.AP_ERR_INVALID_ARG, (idx, val)
-    a = list(base)
-    a[11] = ws - 1
-    assert g(*a) == ap.AP_ERR_WORKSPACE
-    a = list(base)
-    a[2], a[5] = 9, 1  # causal with Lq != Lk
-    assert g(*a) == ap.AP_ERR_INVALID_ARG
+        a[11] = ws - 1
+        assert g(*a) == ap.AP_ERR_WORKSPACE
+        a = list(base)
+        a[2], a[5] = 9, 1  # causal with Lq != Lk
+        assert g(*a) == ap.AP_ERR_INVALID_ARG
+    # one selection over the layer ranks ties by a 32-bit index over all heads
+    big = [FAKE, 64, 8192, 8192, 0.5, 0, 1, FAKE, None, FAKE, FAKE, ap.ap_build_mask_workspace_bytes(64, 8192, 8192),
+           None]
+    assert ap.lib.ap_build_mask_layer(*big) == ap.AP_ERR_UNSUPPORTED
     m = ap.lib.ap_mask_to_tiles
     assert m(None, 1, 8, 8, ctypes.byref(t), FAKE, 1 << 20, None) == ap.AP_ERR_INVALID_ARG
     assert m(FAKE, 1, 8, 8, ctypes.byref(t), FAKE, 16, None) == ap.AP_ERR_WORKSPACE

@@ -71,10 +71,11 @@ def test_dense_tiles_equal_tiles_of_the_full_domain(ap, L, causal):
 # ------------------------------------------------------------------------------ build mask
 
 
-def _check_build_mask(ap, acc32: np.ndarray, w):
+def _check_build_mask(ap, acc32: np.ndarray, w, layer=False):
     acc_dev = torch.from_numpy(acc32).cuda()
-    mask, tiles, nnz = pu.gpu_build_mask(ap, acc_dev, w)
-    want_mask, want_nnz = orc.build_mask(acc32, w.keep_frac, w.causal, w.keep_diag)
+    mask, tiles, nnz = pu.gpu_build_mask(ap, acc_dev, w, layer=layer)
+    want = orc.build_mask_layer if layer else orc.build_mask
+    want_mask, want_nnz = want(acc32, w.keep_frac, w.causal, w.keep_diag)
     np.testing.assert_array_equal(nnz.cpu().numpy(), want_nnz)
     np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
     pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
@@ -149,6 +150,114 @@ def test_build_mask_optional_outputs(ap):
     ap.ap_build_mask(acc_dev, 0.2, True, True, tiles=tiles)
     pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
     assert ap.ap_device_status() == ap.AP_OK
+
+
+# ------------------------------------------------------------- build mask, one threshold per layer
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("keep_diag", [False, True])
+@pytest.mark.parametrize("shape", [(3, 67, 67), (2, 128, 128), (4, 300, 300), (1, 5, 5)])
+def test_build_mask_layer_random_values_with_ties(ap, shape, causal, keep_diag):
+    H, Lq, Lk = shape
+    rng = np.random.default_rng(80)
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc[0].flat[::3] = 0.5                      # ties inside head 0 and with the last head's values
+    acc[-1] = np.round(acc[-1] * 8) / 8
+    acc[0, 0, :3] = [-1.0, -0.0, 0.0]
+    if H > 2:
+        acc[1] *= 0.25                          # a head that loses almost everything at small fractions
+    for keep in (0.1, 0.5, 1.0):
+        _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=causal, keep_diag=keep_diag,
+                                                     keep_frac=keep), layer=True)
+
+
+def test_build_mask_layer_rectangular_constant_and_tiny_fraction(ap):
+    acc = np.random.default_rng(81).random((3, 100, 260), dtype=np.float32)
+    acc[0] = np.round(acc[0] * 4) / 4
+    _check_build_mask(ap, acc, W["s2s_cross"].scaled(H=3, Lq=100, Lk=260, keep_frac=0.3), layer=True)
+    acc = np.full((2, 130, 130), 0.25, dtype=np.float32)    # every entry ties: the lowest global indices win
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=0.37), layer=True)
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=0.37, causal=True), layer=True)
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=1e-6), layer=True)
+    _check_build_mask(ap, acc, W["tiny"].scaled(H=2, Lq=130, Lk=130, keep_frac=1e-6, keep_diag=False), layer=True)
+
+
+def _domain(H, L, causal):
+    dom = np.tril(np.ones((L, L), dtype=bool)) if causal else np.ones((L, L), dtype=bool)
+    return np.broadcast_to(dom, (H, L, L))
+
+
+@pytest.mark.parametrize("causal,L", [(False, 1100), (True, 1536)])
+def test_build_mask_layer_large_takes_the_one_pass_shortcut(ap, causal, L):
+    """More than 2^20 selectable entries in the layer: the threshold is bracketed with a sample and
+    selected among the collected keys with grid-wide passes.  Head 1 is quantised to 32 levels, head
+    2 skewed towards zero, head 3 constant.  Covered: a threshold tied a few times across heads (the
+    copies with the lowest global indices are kept), a threshold on one of head 1's levels (tens of
+    thousands of ties: tie counts and a prefix sum), a threshold on head 3's constant (the bracket
+    overflows its buffer: three full passes), and thresholds in between."""
+    H = 4
+    rng = np.random.default_rng(83 + L)
+    acc = rng.random((H, L, L), dtype=np.float32)
+    acc[1] = np.round(acc[1] * 32) / 32
+    acc[2] = acc[2] ** 8
+    acc[3] = 0.75
+    dom = _domain(H, L, causal)
+    vals = acc[dom]
+    n = vals.size
+    k = int(0.05 * n)
+    v_thr = np.partition(vals, n - k)[n - k]
+    for h in (0, 2, 0, 2, 0, 2, 0, 2, 0):       # copies of the 5 % threshold in the lower left of two heads
+        acc[h, rng.integers(L // 2, L), rng.integers(0, L // 2)] = v_thr
+    vals = acc[dom]
+    level = np.float32(0.5)                      # one of head 1's levels, cut in the middle of its ties
+    k_level = int((vals > level).sum() + (vals == level).sum() // 2)
+    for keep, keep_diag in ((0.05, True), (0.05, False), (k_level / n, False), (0.25, False), (0.5, True),
+                            (0.999, True)):
+        _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=L, Lk=L, causal=causal, keep_diag=keep_diag,
+                                                     keep_frac=keep), layer=True)
+
+
+def test_build_mask_layer_many_small_heads(ap):
+    """Each head is far below the size at which the shortcut is tried, the layer is above it."""
+    H, L = 16, 300
+    acc = np.random.default_rng(84).random((H, L, L), dtype=np.float32)
+    acc *= np.linspace(0.2, 1.0, H, dtype=np.float32)[:, None, None]
+    for keep in (0.1, 0.6):
+        want = _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=L, Lk=L, causal=True, keep_frac=keep), layer=True)
+        per_head = want.reshape(H, -1).sum(1)
+        assert per_head[0] < per_head[-1]        # unlike the per-head rule, heads keep unequal shares
+
+
+def test_build_mask_layer_full_size_long(ap):
+    """The long workload's layer at full size, on the accumulator the calibration kernel wrote.
+    The first four heads as a layer of their own are compared with the oracle entry by entry; for
+    all sixteen, the properties that define the result: k entries kept in all, every forced entry
+    kept, no pruned entry larger than a kept one, and among the entries equal to the smallest kept
+    value the kept ones come first in global index order."""
+    w = W["long"]
+    acc = pu.gpu_accumulate(ap, w, 1, None)
+    _check_build_mask(ap, acc[:4].cpu().numpy(), w.scaled(H=4), layer=True)
+
+    mask, tiles, nnz = pu.gpu_build_mask(ap, acc, w, layer=True)
+    k = orc.keep_count(w.H * w.n_valid, w.H * w.n_forced, w.keep_frac)
+    assert int(nnz.sum()) == k
+    assert torch.equal(mask.view(w.H, -1).sum(-1, dtype=torch.int64), nnz)
+    assert int(nnz.min()) < int(nnz.max())
+    pop = np.unpackbits(tiles.to_host()["bitmap"].view(np.uint8)).sum()
+    assert pop == k
+    eye = torch.eye(w.Lq, dtype=torch.bool, device="cuda")
+    dom = torch.tril(torch.ones((w.Lq, w.Lk), dtype=torch.bool, device="cuda"))
+    assert bool(mask[:, eye].all()) and not bool(mask[:, ~dom].any())
+    free = (dom & ~eye).expand(w.H, -1, -1)
+    kept, pruned = free & (mask != 0), free & (mask == 0)
+    v_kept, v_pruned = acc[kept].min(), acc[pruned].max()
+    assert v_kept >= v_pruned
+    if v_kept == v_pruned:
+        tie = (acc == v_kept).view(-1)
+        first_pruned = torch.nonzero(tie & pruned.reshape(-1))[0]
+        last_kept = torch.nonzero(tie & kept.reshape(-1))[-1]
+        assert int(last_kept) < int(first_pruned)
 
 
 # ------------------------------------------------------------------------------ accumulate
