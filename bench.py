@@ -334,6 +334,32 @@ def run_gpu(args, w):
     h2d = 3 * 0 + (hq.numel() + hk.numel() + hv.numel()) * elem
     d2h = ho.numel() * elem
 
+    # ---- Eq. 2 with one threshold for the layer (outside the step: the workloads prescribe per head) ----
+    tiles_layer = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    nnz_layer = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+    layer_ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    layer_ms = [0.0, 0.0]
+    n_layer = 5
+    for it in range(2 + n_layer):
+        layer_ev[0].record()
+        ap.ap_build_mask_layer(acc, w.keep_frac, w.causal, w.keep_diag, mask, tiles_layer, nnz_layer, ws)
+        layer_ev[1].record()
+        ap.ap_sparse_attention_fwd(q, k, v, tiles_layer, out)
+        layer_ev[2].record()
+        torch.cuda.synchronize()
+        if it >= 2:
+            layer_ms[0] += layer_ev[0].elapsed_time(layer_ev[1]) / n_layer
+            layer_ms[1] += layer_ev[1].elapsed_time(layer_ev[2]) / n_layer
+    if ap.ap_device_status() != ap.AP_OK:
+        raise RuntimeError("device status not OK after the layer-threshold runs")
+    k_layer = metrics.keep_count(w.n_valid * w.H, w.n_forced * w.H, w.keep_frac)
+    assert int(nnz_layer.sum().item()) == k_layer
+    layer = {"build_mask_layer_ms": layer_ms[0], "sparse_fwd_ms": layer_ms[1], "tiles_kept": tiles_layer.n_tiles(),
+             "nnz_per_head_min": int(nnz_layer.min().item()), "nnz_per_head_max": int(nnz_layer.max().item()),
+             "effective_tflops": metrics.effective_flops(k_layer, w.B, w.d) / (layer_ms[1] * 1e-3) / 1e12,
+             "note": "one threshold over all heads of the layer; %d runs after 2 warm-up runs, outside the step"
+                     % n_layer}
+
     if rank != 0:
         return
     # ---- rooflines ---------------------------------------------------------------------------------
@@ -404,7 +430,7 @@ def run_gpu(args, w):
         "roofline": roof, "roofline_by_stage": by_stage, "cpu_baseline": cpu,
         "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": int(launches), "clocks": clocks,
+        "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer,
     }
     print(json.dumps(line))
 

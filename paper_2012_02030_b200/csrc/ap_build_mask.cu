@@ -7,7 +7,8 @@
 // accumulator each.  Large heads first try a shortcut that needs one pass: a
 // random sample of the head brackets the threshold between two pivot keys, one
 // pass counts the keys above the upper pivot and collects those between the
-// pivots, and the threshold is selected among the collected keys; it is exact
+// pivots, and the threshold is selected among the collected keys (the same radix
+// select on their offsets from the lower pivot, grid-wide); it is exact
 // whenever the bracket holds the threshold and the collected keys fit their
 // buffer (checked with the exact counts), else the head takes the three passes.  Entries equal to the threshold key are all kept when the
 // count allows it (the usual case); otherwise they are ranked by linear index
@@ -18,9 +19,7 @@
 //
 // One threshold for the whole layer (Eq. 2 as stated) is the same selection run
 // once over a virtual head of H*Lq rows: row i' = h*Lq + i has the domain of row
-// i, and the linear index i'*Lk + j is the layer-wide tie order.  Its collected
-// keys are too many for one CTA, so the threshold is selected among them with
-// grid-wide histogram passes instead.
+// i, and the linear index i'*Lk + j is the layer-wide tie order.
 #include "ap_common.cuh"
 
 namespace ap {
@@ -42,7 +41,14 @@ __device__ __forceinline__ uint32_t key_of(float f) {
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
-struct SelectState {  // per head
+// The float whose key is `key`.  Keys 0 and 0xffffffff (no pivot / no threshold) give NaNs, for
+// which every ordered comparison is false.  For values and pivots that are not NaN,
+// key_of(f) > key <=> f > float_of_key(key), and likewise for == and <.
+__device__ __forceinline__ float float_of_key(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
+}
+
+struct SelectState {  // per selection
   uint32_t prefix;    // digits of the threshold key found so far
   uint32_t thr;       // threshold key (valid after the last digit)
   unsigned long long remaining;  // rank still to resolve inside the current prefix
@@ -57,11 +63,23 @@ struct SelectState {  // per head
   // when not all entries equal to thr are kept: those with linear index i*Lk + j <= tie_cut are
   // (valid if have_cut; otherwise the ties are ranked with tie counts and a prefix sum)
   uint32_t tie_cut, have_cut;
-  // selection among the collected keys with grid-wide passes (one threshold for the layer)
+  // selection among the collected keys
   uint32_t cand_select;          // the bracket holds the threshold: the passes over the collected keys run
   uint32_t thr_count;            // entries equal to the threshold key
   uint32_t tie_n;                // entries gathered in the tie list
 };
+
+// Selection among the keys the one-pass shortcut collected (see below).
+// The bracket holds the threshold (the (k_rest - above_hi)-th largest collected key) and every key
+// of the bracket was collected.  All fields are final once the collecting pass has ended.
+__device__ __forceinline__ bool bracket_holds(const SelectState &st, uint32_t cand_cap, unsigned long long k_rest) {
+  return st.use_shortcut && st.n_cand <= cand_cap && st.above_hi < k_rest && k_rest - st.above_hi <= st.n_cand;
+}
+// All offsets are at most hi - lo: a leading digit in which that span is zero is zero for every
+// key and needs no pass (the pick leaves the digit at zero).
+__device__ __forceinline__ bool digit_is_zero(const SelectState &st, int pass) {
+  return pass < kPasses - 1 && ((st.hi - st.lo) >> digit_shift(pass)) == 0u;
+}
 
 constexpr int kMaxCutTies = 4096;  // ties with the threshold ranked inside the shortcut (more: tie counts + scan)
 
@@ -69,7 +87,7 @@ struct Scratch {
   uint32_t *hist;       // [H][kBins]
   SelectState *state;   // [H]
   uint32_t *tie_count;  // [H][Lq][n_kt] -> exclusive prefix after the scan
-  uint32_t *tie_list;   // [kMaxCutTies] linear indices of the entries equal to the threshold (layer selection)
+  uint32_t *tie_list;   // [H][kMaxCutTies] linear indices of the collected entries equal to the threshold
   uint2 *cand;          // [H][cand_cap] (key, linear index) of the entries collected by the shortcut
 };
 
@@ -182,11 +200,25 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
 // One CTA per head: picks the digit whose bin contains the wanted rank.  Thread t
 // owns bins [kBins-1-8t, kBins-8-8t] (descending); a block-wide prefix over the
 // threads' sums locates the owner, which then walks its eight bins.
-// from_cand: the histogram came from the collected keys (offsets from the lower pivot).
-__global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass, int from_cand) {
+// from_cand: the histogram came from the collected keys (offsets from the lower pivot); the first
+// such pass opens the selection among them if the bracket holds the threshold.
+__global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass, int from_cand,
+                                                         uint32_t cand_cap, unsigned long long k_rest) {
   __shared__ uint32_t warp_sums[8];
   const int h = blockIdx.x;
-  if (from_cand ? !state[h].cand_select : state[h].done) return;  // no such passes / resolved by the shortcut
+  if (!from_cand && state[h].done) return;  // resolved by the shortcut
+  if (from_cand) {
+    const SelectState cur = state[h];
+    if (!(pass == 0 ? bracket_holds(cur, cand_cap, k_rest) : cur.cand_select != 0u)) return;
+    if (digit_is_zero(cur, pass)) {
+      if (pass == 0 && threadIdx.x == 0) {
+        state[h].remaining = k_rest - cur.above_hi;
+        state[h].prefix = 0u;
+        state[h].cand_select = 1u;
+      }
+      return;
+    }
+  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t cnt[8];
   uint32_t mine = 0u;
@@ -204,7 +236,12 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
     if (lane >= o) incl += v;
   }
   if (lane == 31) warp_sums[warp] = incl;
-  const SelectState st = state[h];  // read by everyone before the barrier, written by the owner after it
+  SelectState st = state[h];  // read by everyone before the barrier, written by the owner after it
+  if (from_cand && pass == 0) {
+    st.remaining = k_rest - st.above_hi;
+    st.prefix = 0u;
+    st.cand_select = 1u;
+  }
   __syncthreads();
   unsigned long long before = incl - mine;  // entries in bins above this thread's
   for (int w = 0; w < warp; ++w) before += warp_sums[w];
@@ -240,20 +277,13 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
 struct Picked {
   uint32_t key, count, rank_in_ties;
 };
-// All keys lie in [base, base + span]: the select runs on key - base, and leading digits in which
-// span is zero are known to be zero (no pass, and no pile-up of every key in one bin).
-__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch,
-                               uint32_t base = 0u, uint32_t span = 0xffffffffu, int stride = 1) {
+__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch) {
   __shared__ uint32_t warp_sums[32];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   uint32_t prefix = 0u, hi_mask = 0u, count = n;
   for (int pass = 0; pass < kPasses; ++pass) {
     const int shift = digit_shift(pass);
     const uint32_t dmask = digit_mask(pass);
-    if (((span >> shift) & ~0u) == 0u && pass < kPasses - 1) {  // the digit is 0 for every key
-      hi_mask |= dmask << shift;
-      continue;
-    }
     hist[t] = 0u;
     hist[t + 1024] = 0u;
     __syncthreads();
@@ -262,7 +292,7 @@ __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, 
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const uint32_t idx = idx0 + u * 1024;
-        kk[u] = idx < n ? keys[(size_t)idx * stride] - base : 0xffffffffu;
+        kk[u] = idx < n ? keys[idx] : 0xffffffffu;
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u)
@@ -296,7 +326,7 @@ __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, 
     __syncthreads();
   }
   Picked p;
-  p.key = prefix + base;
+  p.key = prefix;
   p.count = count;
   p.rank_in_ties = rank;
   return p;
@@ -348,10 +378,12 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
   }
 }
 
-// One pass over the head: counts the keys above the upper pivot and collects those inside the
-// bracket.  grid = (row blocks, H); a warp takes a row at a time.  Collected keys are staged in
-// shared memory and appended to the head's buffer with one reservation per CTA (keys that do not
-// fit the stage any more are appended one warp at a time).
+// One pass over the selection's rows: counts the keys above the upper pivot and collects those
+// inside the bracket.  grid = (row blocks, selections); a warp takes a row at a time.  Values are
+// compared with the pivots as floats (the same order as their keys); the key is computed for the
+// collected entries only.  Collected entries are staged in shared memory and appended to the
+// selection's buffer with one reservation per CTA (entries that do not fit the stage any more
+// go straight to the buffer).
 constexpr int kStageKeys = 4096;
 __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
                                                            int causal, int diag, SelectState *state,
@@ -363,14 +395,26 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) stage_n = 0u;
   __syncthreads();
-  const uint32_t lo = state[h].lo, hi = state[h].hi;
+  const float lo_f = float_of_key(state[h].lo), hi_f = float_of_key(state[h].hi);
   uint2 *out = cand + (size_t)h * cand_cap;
+  uint32_t *n_cand = &state[h].n_cand;
+  auto push = [&](float f, uint32_t index) {  // a few per cent of the entries
+    const uint2 entry = make_uint2(key_of(f), index);
+    const uint32_t pos = atomicAdd(&stage_n, 1u);
+    if (pos < (uint32_t)kStageKeys) {
+      stage[pos] = entry;
+    } else {
+      const uint32_t g = atomicAdd(n_cand, 1u);
+      if (g < cand_cap) out[g] = entry;
+    }
+  };
   const bool vec = (Lk & 3) == 0;
-  unsigned long long above = 0ull;
+  uint32_t above = 0u;  // per thread: fewer than 2^32 entries
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
     const int ii = i % period;
     const int jend = causal ? min(Lk, ii + 1) : Lk;
+    const uint32_t row_index = (uint32_t)i * (uint32_t)Lk;
     for (int base = 0; base < jend; base += 512) {  // warp-uniform trip count
       float v[4][4];
 #pragma unroll
@@ -382,37 +426,97 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int j0 = base + 128 * u + 4 * lane;
+        if (j0 + 4 <= jend && !(diag && ii >= j0 && ii < j0 + 4)) {
+          // four entries of the domain: nothing to check per entry
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int j = j0 + c;
-          const uint32_t key = key_of(v[u][c]);
-          const bool in = j < jend && !(diag && j == ii);
-          above += (in && key > hi) ? 1u : 0u;
-          if (in && key >= lo && key <= hi) {  // a few per cent of the entries
-            const uint2 entry = make_uint2(key, (uint32_t)i * (uint32_t)Lk + (uint32_t)j);
-            const uint32_t pos = atomicAdd(&stage_n, 1u);
-            if (pos < (uint32_t)kStageKeys) {
-              stage[pos] = entry;
-            } else {
-              // the stage is full: the entry goes straight to the head's buffer
-              const uint32_t g = atomicAdd(&state[h].n_cand, 1u);
-              if (g < cand_cap) out[g] = entry;
-            }
+          for (int c = 0; c < 4; ++c) {
+            const float f = v[u][c];
+            const bool gt = f > hi_f;
+            above += gt ? 1u : 0u;
+            if (!(f < lo_f) && !gt) push(f, row_index + (uint32_t)(j0 + c));
+          }
+        } else if (j0 < jend) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int j = j0 + c;
+            const float f = v[u][c];
+            const bool in = j < jend && !(diag && j == ii);
+            const bool gt = in && f > hi_f;
+            above += gt ? 1u : 0u;
+            if (in && !(f < lo_f) && !gt) push(f, row_index + (uint32_t)j);
           }
         }
       }
     }
   }
+  unsigned long long above_warp = above;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) above += __shfl_xor_sync(0xffffffffu, above, o);
-  if (lane == 0 && above) atomicAdd(&state[h].above_hi, above);
+  for (int o = 16; o > 0; o >>= 1) above_warp += __shfl_xor_sync(0xffffffffu, above_warp, o);
+  if (lane == 0 && above_warp) atomicAdd(&state[h].above_hi, above_warp);
   __syncthreads();
   const uint32_t n = min(stage_n, (uint32_t)kStageKeys);
-  if (threadIdx.x == 0) stage_base = atomicAdd(&state[h].n_cand, n);
+  if (threadIdx.x == 0) stage_base = atomicAdd(n_cand, n);
   __syncthreads();
   const uint32_t dst = stage_base;
   for (uint32_t e = threadIdx.x; e < n; e += kThreads)
     if (dst + e < cand_cap) out[dst + e] = stage[e];
+}
+
+// ---- selection among the collected keys: the radix select on their offsets from the lower pivot ----
+
+
+// grid = (CTAs, selections)
+__global__ void __launch_bounds__(kThreads) cand_histogram_kernel(const SelectState *__restrict__ state,
+                                                                  const uint2 *__restrict__ cand, uint32_t cand_cap,
+                                                                  unsigned long long k_rest, int pass,
+                                                                  uint32_t *__restrict__ hist) {
+  __shared__ uint32_t sh[kBins];
+  const int h = blockIdx.y;
+  const SelectState st = state[h];
+  if (!(pass == 0 ? bracket_holds(st, cand_cap, k_rest) : st.cand_select != 0u) || digit_is_zero(st, pass)) return;
+  const int lane = threadIdx.x & 31;
+  for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0u;
+  __syncthreads();
+  const int shift = digit_shift(pass);
+  const uint32_t dmask = digit_mask(pass);
+  const uint32_t hi_mask = pass == 0 ? 0u : ~((1u << (shift + (pass == 1 ? 11 : 10))) - 1u);
+  const uint32_t want_hi = (pass == 0 ? 0u : st.prefix) & hi_mask;
+  const uint32_t n = st.n_cand, lo = st.lo;
+  const uint2 *mine = cand + (size_t)h * cand_cap;
+  for (uint32_t base = blockIdx.x * kThreads; base < n; base += gridDim.x * kThreads) {  // warp-uniform
+    const uint32_t idx = base + threadIdx.x;
+    const uint32_t key = idx < n ? mine[idx].x - lo : 0u;
+    const bool take = idx < n && (key & hi_mask) == want_hi;
+    const uint32_t bin = (key >> shift) & dmask;
+    const unsigned voters = __ballot_sync(0xffffffffu, take);
+    if (take) {
+      const unsigned peers = __match_any_sync(voters, bin);
+      if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], (uint32_t)__popc(peers));
+    }
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < kBins; b += kThreads) {
+    const uint32_t s = sh[b];
+    if (s) atomicAdd(&hist[h * kBins + b], s);
+  }
+}
+
+// Gathers the linear indices of the collected entries equal to the threshold, when they must be
+// ranked and are few enough.  grid = (CTAs, selections)
+__global__ void __launch_bounds__(kThreads) cand_ties_kernel(SelectState *state, const uint2 *__restrict__ cand,
+                                                             uint32_t cand_cap, uint32_t *__restrict__ tie_list) {
+  const int h = blockIdx.y;
+  const SelectState st = state[h];
+  if (!st.cand_select || st.all_ties_kept || st.thr_count > (uint32_t)kMaxCutTies) return;
+  const uint32_t want = st.prefix + st.lo;
+  const uint2 *mine = cand + (size_t)h * cand_cap;
+  for (uint32_t idx = blockIdx.x * kThreads + threadIdx.x; idx < st.n_cand; idx += gridDim.x * kThreads) {
+    const uint2 c = mine[idx];
+    if (c.x == want) {
+      const uint32_t pos = atomicAdd(&state[h].tie_n, 1u);
+      if (pos < (uint32_t)kMaxCutTies) tie_list[(size_t)h * kMaxCutTies + pos] = c.y;
+    }
+  }
 }
 
 // Ranks `count` <= kMaxCutTies distinct linear indices: returns (in *cut_s, after a barrier) the one
@@ -427,126 +531,28 @@ __device__ void rank_ties(const uint32_t *tie_idx, uint32_t count, uint32_t rank
   __syncthreads();
 }
 
-// One CTA per head: if the bracket holds the threshold, selects it among the collected keys.
-__global__ void __launch_bounds__(1024) select_candidates_kernel(SelectState *state, const uint2 *__restrict__ cand,
-                                                                 uint32_t cand_cap, unsigned long long k_rest) {
-  __shared__ uint32_t hist[kBins];
-  __shared__ uint32_t xch[4];
-  __shared__ uint32_t tie_idx[kMaxCutTies];
-  __shared__ uint32_t tie_n, cut_s;
-  const int h = blockIdx.x;
-  const SelectState st = state[h];
-  if (!st.use_shortcut) return;
-  // the threshold is the (k_rest - above_hi)-th largest collected key, if there is one
-  if (st.n_cand > cand_cap || st.above_hi >= k_rest || k_rest - st.above_hi > st.n_cand) return;
-  const uint2 *mine = cand + (size_t)h * cand_cap;
-  const Picked p = block_select(reinterpret_cast<const uint32_t *>(mine), st.n_cand, (uint32_t)(k_rest - st.above_hi),
-                                hist, xch, st.lo, st.hi - st.lo, 2);
-  // Not all entries equal to the threshold are kept: the ones with the lowest linear indices are.
-  // With few enough of them, the index of the last kept one is found here.
-  bool have_cut = false;
-  if (p.rank_in_ties < p.count && p.count <= (uint32_t)kMaxCutTies) {
-    if (threadIdx.x == 0) tie_n = 0u;
-    __syncthreads();
-    for (uint32_t e = threadIdx.x; e < st.n_cand; e += 1024) {
-      const uint2 c = mine[e];
-      if (c.x == p.key) tie_idx[atomicAdd(&tie_n, 1u)] = c.y;
-    }
-    __syncthreads();
-    rank_ties(tie_idx, p.count, p.rank_in_ties, &cut_s);
-    have_cut = true;
-  }
-  if (threadIdx.x == 0) {
-    state[h].tie_cut = have_cut ? cut_s : 0u;
-    state[h].have_cut = have_cut ? 1u : 0u;
-    state[h].thr = p.key;
-    state[h].prefix = p.key;
-    state[h].ties_kept = p.rank_in_ties;
-    state[h].remaining = p.rank_in_ties;
-    state[h].all_ties_kept = p.rank_in_ties == p.count ? 1u : 0u;
-    state[h].done = 1u;
-  }
-}
-
-// ---- the same selection among the collected keys with grid-wide passes (selection 0 only) -----
-
-// Decides whether the bracket holds the threshold; if so the digit passes below run on the
-// collected keys' offsets from the lower pivot, else the selection takes the three full passes.
-__global__ void cand_begin_kernel(SelectState *state, uint32_t cand_cap, unsigned long long k_rest) {
-  const SelectState st = state[0];
-  if (!st.use_shortcut) return;
-  if (st.n_cand > cand_cap || st.above_hi >= k_rest || k_rest - st.above_hi > st.n_cand) return;
-  state[0].remaining = k_rest - st.above_hi;
-  state[0].prefix = 0u;
-  state[0].cand_select = 1u;
-}
-
-__global__ void __launch_bounds__(kThreads) cand_histogram_kernel(const SelectState *__restrict__ state,
-                                                                  const uint2 *__restrict__ cand, int pass,
-                                                                  uint32_t *__restrict__ hist) {
-  __shared__ uint32_t sh[kBins];
-  if (!state[0].cand_select) return;
-  const int lane = threadIdx.x & 31;
-  for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0u;
-  __syncthreads();
-  const int shift = digit_shift(pass);
-  const uint32_t dmask = digit_mask(pass);
-  const uint32_t hi_mask = pass == 0 ? 0u : ~((1u << (shift + (pass == 1 ? 11 : 10))) - 1u);
-  const uint32_t want_hi = state[0].prefix & hi_mask;
-  const uint32_t n = state[0].n_cand, lo = state[0].lo;
-  for (uint32_t base = blockIdx.x * kThreads; base < n; base += gridDim.x * kThreads) {  // warp-uniform
-    const uint32_t idx = base + threadIdx.x;
-    const uint32_t key = idx < n ? cand[idx].x - lo : 0u;
-    const bool take = idx < n && (key & hi_mask) == want_hi;
-    const uint32_t bin = (key >> shift) & dmask;
-    const unsigned voters = __ballot_sync(0xffffffffu, take);
-    if (take) {
-      const unsigned peers = __match_any_sync(voters, bin);
-      if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], (uint32_t)__popc(peers));
-    }
-  }
-  __syncthreads();
-  for (int b = threadIdx.x; b < kBins; b += kThreads) {
-    const uint32_t s = sh[b];
-    if (s) atomicAdd(&hist[b], s);
-  }
-}
-
-// Gathers the linear indices of the collected entries equal to the threshold, when they must be
-// ranked and are few enough.
-__global__ void __launch_bounds__(kThreads) cand_ties_kernel(SelectState *state, const uint2 *__restrict__ cand,
-                                                             uint32_t *__restrict__ tie_list) {
-  const SelectState st = state[0];
-  if (!st.cand_select || st.all_ties_kept || st.thr_count > (uint32_t)kMaxCutTies) return;
-  const uint32_t want = st.prefix + st.lo;
-  for (uint32_t idx = blockIdx.x * kThreads + threadIdx.x; idx < st.n_cand; idx += gridDim.x * kThreads) {
-    const uint2 c = cand[idx];
-    if (c.x == want) {
-      const uint32_t pos = atomicAdd(&state[0].tie_n, 1u);
-      if (pos < (uint32_t)kMaxCutTies) tie_list[pos] = c.y;
-    }
-  }
-}
-
-// One CTA: turns the digits found among the collected keys into the threshold and closes the selection.
+// One CTA per selection: turns the digits found among the collected keys into the threshold,
+// ranks its ties when not all of them are kept (the lowest linear indices are), and closes the
+// selection.
 __global__ void __launch_bounds__(1024) cand_finish_kernel(SelectState *state, const uint32_t *__restrict__ tie_list) {
   __shared__ uint32_t tie_idx[kMaxCutTies];
   __shared__ uint32_t cut_s;
-  const SelectState st = state[0];
+  const int h = blockIdx.x;
+  const SelectState st = state[h];
   if (!st.cand_select) return;
   bool have_cut = false;
   if (!st.all_ties_kept && st.thr_count <= (uint32_t)kMaxCutTies) {
-    for (uint32_t e = threadIdx.x; e < st.thr_count; e += 1024) tie_idx[e] = tie_list[e];
+    for (uint32_t e = threadIdx.x; e < st.thr_count; e += 1024) tie_idx[e] = tie_list[(size_t)h * kMaxCutTies + e];
     __syncthreads();
     rank_ties(tie_idx, st.thr_count, (uint32_t)st.ties_kept, &cut_s);
     have_cut = true;
   }
   if (threadIdx.x == 0) {
-    state[0].tie_cut = have_cut ? cut_s : 0u;
-    state[0].have_cut = have_cut ? 1u : 0u;
-    state[0].thr = st.prefix + st.lo;
-    state[0].prefix = st.prefix + st.lo;
-    state[0].done = 1u;
+    state[h].tie_cut = have_cut ? cut_s : 0u;
+    state[h].have_cut = have_cut ? 1u : 0u;
+    state[h].thr = st.prefix + st.lo;
+    state[h].prefix = st.prefix + st.lo;
+    state[h].done = 1u;
   }
 }
 
@@ -623,9 +629,132 @@ __global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ t
   }
 }
 
+// What the emit pass needs of a selection.
+struct EmitSel {
+  float thr_f;  // the threshold as a float (NaN when nothing but the forced entries is kept)
+  unsigned long long ties_kept;
+  bool all_ties, have_cut;
+  uint32_t tie_cut;
+  uint32_t first_row;  // of this head in the tie order
+};
+
+// The rows of one tile; returns this lane's share of the tile's popcount (lanes 0, 8, 16, 24).
+// kInterior: every row and column of the tile exists and lies in the domain and none is forced,
+// so nothing is checked per entry.
+template <bool kInterior>
+__device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int Lq, int Lk, int n_kt, int h, int qt,
+                                              int kt, int tile, int causal, int diag, const EmitSel &sel,
+                                              const uint32_t *__restrict__ tie_prefix, uint8_t *__restrict__ mask,
+                                              uint32_t *__restrict__ stage_bitmap) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool vec = (Lk & 3) == 0;
+  const int j0 = kt * kTile + 4 * lane;
+  const float thr_f = sel.thr_f;
+  int count = 0;
+  for (int r0 = warp; r0 < kTile; r0 += 16) {
+    float v[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {  // rows r0, r0+4, r0+8, r0+12: four loads in flight
+      const int i = qt * kTile + r0 + 4 * u;
+      if (kInterior) {
+        const float4 t = *reinterpret_cast<const float4 *>(acc + ((size_t)h * Lq + i) * Lk + j0);
+        v[u][0] = t.x; v[u][1] = t.y; v[u][2] = t.z; v[u][3] = t.w;
+      } else {
+        v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+        if (i < Lq) {
+          const int jend = causal ? min(Lk, i + 1) : Lk;
+          if (j0 < jend) load4(acc + ((size_t)h * Lq + i) * Lk, j0, jend, vec, v[u]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + 4 * u;
+      const int i = qt * kTile + r;
+      uint32_t nib = 0u;
+      if (kInterior || i < Lq) {  // warp-uniform
+        uint32_t tie_bits = 0u, gt_bits = 0u;
+        if (kInterior) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
+            tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
+          }
+        } else {
+          const int jend = causal ? min(Lk, i + 1) : Lk;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int j = j0 + c;
+            if (j < jend) {
+              if (diag && j == i) {
+                gt_bits |= 1u << c;
+              } else {
+                gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
+                tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
+              }
+            }
+          }
+        }
+        nib = gt_bits;
+        if (sel.all_ties) {
+          nib |= tie_bits;
+        } else if (sel.have_cut) {
+          if (tie_bits) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if ((tie_bits & (1u << c)) &&
+                  (sel.first_row + (uint32_t)i) * (uint32_t)Lk + (uint32_t)(j0 + c) <= sel.tie_cut)
+                nib |= 1u << c;
+          }
+        } else if (__any_sync(0xffffffffu, tie_bits != 0u)) {
+          // rank of each tie in linear-index order = ties before this row segment
+          // + ties in lower lanes + ties in lower columns of this lane
+          int before = __popc(tie_bits);
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, before, o);
+            if (lane >= o) before += t;
+          }
+          before -= __popc(tie_bits);
+          unsigned long long rank = (unsigned long long)tie_prefix[((size_t)h * Lq + i) * n_kt + kt] + before;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (tie_bits & (1u << c)) {
+              if (rank < sel.ties_kept) nib |= 1u << c;
+              ++rank;
+            }
+          }
+        }
+        if (mask) {
+          uint8_t *mrow = mask + ((size_t)h * Lq + i) * Lk;
+          if (kInterior || (vec && j0 + 4 <= Lk)) {
+            *reinterpret_cast<uchar4 *>(mrow + j0) =
+                make_uchar4(nib & 1u, (nib >> 1) & 1u, (nib >> 2) & 1u, (nib >> 3) & 1u);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if (j0 + c < Lk) mrow[j0 + c] = (nib >> c) & 1u;
+          }
+        }
+      }
+      // 8 lanes x 4 bits -> one bitmap word, complete in the first lane of each group of eight
+      uint32_t w = nib << (4 * (lane & 7));
+      w |= __shfl_xor_sync(0xffffffffu, w, 1);
+      w |= __shfl_xor_sync(0xffffffffu, w, 2);
+      w |= __shfl_xor_sync(0xffffffffu, w, 4);
+      if ((lane & 7) == 0) {
+        count += __popc(w);
+        if (stage_bitmap) stage_bitmap[(size_t)tile * kBitmapWords + 4 * r + (lane >> 3)] = w;
+      }
+    }
+  }
+  return count;
+}
+
 // One CTA per tile of the (h, qt, kt) grid; warp w takes tile rows w, w+4, ...
 // (four rows loaded ahead) and each lane four consecutive columns.  Writes the
-// element mask, the tile's bitmap and popcount into the staging area.  per_layer:
+// element mask, the tile's bitmap and popcount into the staging area.  Values are
+// compared with the threshold as floats (the same order as their keys).  per_layer:
 // all heads share selection 0, ties are ordered by (h*Lq + i)*Lk + j, and the
 // tiles' popcounts are added up into nnz[h].
 __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_qt, int n_kt,
@@ -639,19 +768,11 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   const int qt = (tile / n_kt) % n_qt;
   const int h = tile / (n_kt * n_qt);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int sel = per_layer ? 0 : h;
-  const uint32_t thr = state[sel].thr;
-  const unsigned long long ties_kept = state[sel].ties_kept;
-  const bool all_ties = state[sel].all_ties_kept != 0u;
-  const bool have_cut = state[sel].have_cut != 0u;
-  const uint32_t tie_cut = state[sel].tie_cut;
-  const uint32_t first_row = per_layer ? (uint32_t)h * (uint32_t)Lq : 0u;  // of this head in the tie order
-  const bool vec = (Lk & 3) == 0;
-  const int j0 = kt * kTile + 4 * lane;
   __shared__ int warp_count[4];
-  int count = 0;
   if (causal && kt > qt) {
     // the whole tile lies above the diagonal: nothing is kept, nothing needs to be read
+    const bool vec = (Lk & 3) == 0;
+    const int j0 = kt * kTile + 4 * lane;
     for (int r = warp; r < kTile; r += 4) {
       const int i = qt * kTile + r;
       if (i < Lq && mask) {
@@ -669,89 +790,22 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
     if (stage_count && threadIdx.x == 0) stage_count[tile] = 0;
     return;
   }
-  for (int r0 = warp; r0 < kTile; r0 += 16) {
-    float v[4][4];
+  const SelectState &st = state[per_layer ? 0 : h];
+  EmitSel sel;
+  sel.thr_f = float_of_key(st.thr);
+  sel.ties_kept = st.ties_kept;
+  sel.all_ties = st.all_ties_kept != 0u;
+  sel.have_cut = st.have_cut != 0u;
+  sel.tie_cut = st.tie_cut;
+  sel.first_row = per_layer ? (uint32_t)h * (uint32_t)Lq : 0u;
+  const bool interior = (qt + 1) * kTile <= Lq && (kt + 1) * kTile <= Lk && (Lk & 3) == 0 && !(causal && kt >= qt) &&
+                        !(diag && kt == qt);
+  int count = interior ? emit_tile_rows<true>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel, tie_prefix, mask,
+                                              stage_bitmap)
+                       : emit_tile_rows<false>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel, tie_prefix, mask,
+                                               stage_bitmap);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {  // rows r0, r0+4, r0+8, r0+12: four loads in flight
-      const int i = qt * kTile + r0 + 4 * u;
-      v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
-      if (i < Lq) {
-        const int jend = causal ? min(Lk, i + 1) : Lk;
-        if (j0 < jend) load4(acc + ((size_t)h * Lq + i) * Lk, j0, jend, vec, v[u]);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int r = r0 + 4 * u;
-      const int i = qt * kTile + r;
-      uint32_t nib = 0u;
-      if (i < Lq) {  // warp-uniform
-        const int jend = causal ? min(Lk, i + 1) : Lk;
-        uint32_t tie_bits = 0u, gt_bits = 0u;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int j = j0 + c;
-          if (j < jend) {
-            if (diag && j == i) {
-              gt_bits |= 1u << c;
-            } else {
-              const uint32_t key = key_of(v[u][c]);
-              if (key > thr) gt_bits |= 1u << c;
-              if (key == thr) tie_bits |= 1u << c;
-            }
-          }
-        }
-        nib = gt_bits;
-        if (all_ties) {
-          nib |= tie_bits;
-        } else if (have_cut) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            if ((tie_bits & (1u << c)) && (first_row + (uint32_t)i) * (uint32_t)Lk + (uint32_t)(j0 + c) <= tie_cut)
-              nib |= 1u << c;
-        } else if (__any_sync(0xffffffffu, tie_bits != 0u)) {
-          // rank of each tie in linear-index order = ties before this row segment
-          // + ties in lower lanes + ties in lower columns of this lane
-          int before = __popc(tie_bits);
-#pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, before, o);
-            if (lane >= o) before += t;
-          }
-          before -= __popc(tie_bits);
-          unsigned long long rank = (unsigned long long)tie_prefix[((size_t)h * Lq + i) * n_kt + kt] + before;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            if (tie_bits & (1u << c)) {
-              if (rank < ties_kept) nib |= 1u << c;
-              ++rank;
-            }
-          }
-        }
-        if (mask) {
-          uint8_t *mrow = mask + ((size_t)h * Lq + i) * Lk;
-          if (vec && j0 + 4 <= Lk) {
-            *reinterpret_cast<uchar4 *>(mrow + j0) =
-                make_uchar4(nib & 1u, (nib >> 1) & 1u, (nib >> 2) & 1u, (nib >> 3) & 1u);
-          } else {
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-              if (j0 + c < Lk) mrow[j0 + c] = (nib >> c) & 1u;
-          }
-        }
-      }
-      // 8 lanes x 4 bits -> one bitmap word
-      uint32_t w = nib << (4 * (lane & 7));
-      w |= __shfl_xor_sync(0xffffffffu, w, 1);
-      w |= __shfl_xor_sync(0xffffffffu, w, 2);
-      w |= __shfl_xor_sync(0xffffffffu, w, 4);
-      const uint32_t w0 = __shfl_sync(0xffffffffu, w, 0), w1 = __shfl_sync(0xffffffffu, w, 8),
-                     w2 = __shfl_sync(0xffffffffu, w, 16), w3 = __shfl_sync(0xffffffffu, w, 24);
-      count += __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
-      if (stage_bitmap && lane == 0)
-        reinterpret_cast<uint4 *>(stage_bitmap + (size_t)tile * kBitmapWords)[r] = make_uint4(w0, w1, w2, w3);
-    }
-  }
+  for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xffffffffu, count, o);
   if (lane == 0) warp_count[warp] = count;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -772,7 +826,7 @@ Scratch carve(void *scratch, int H, int Lq, int Lk) {
   s.tie_count = reinterpret_cast<uint32_t *>(p);
   p += align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t));
   s.tie_list = reinterpret_cast<uint32_t *>(p);
-  p += align256((size_t)kMaxCutTies * sizeof(uint32_t));
+  p += align256((size_t)H * kMaxCutTies * sizeof(uint32_t));
   s.cand = reinterpret_cast<uint2 *>(p);
   return s;
 }
@@ -784,7 +838,7 @@ size_t select_scratch_bytes(int H, int Lq, int Lk) {
   // selection over all heads (never smaller than H selections of one head each)
   return align256((size_t)H * kBins * sizeof(uint32_t)) + align256((size_t)H * sizeof(SelectState)) +
          align256((size_t)H * Lq * ceil_div(Lk, kTile) * sizeof(uint32_t)) +
-         align256((size_t)kMaxCutTies * sizeof(uint32_t)) +
+         align256((size_t)H * kMaxCutTies * sizeof(uint32_t)) +
          align256((size_t)cand_capacity((long long)H * Lq * Lk) * sizeof(uint2));
 }
 
@@ -820,22 +874,17 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
                                                      (unsigned long long)a.k_rest, (unsigned long long)n_rest, sc.state);
       collect_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag, sc.state, sc.cand,
                                                (uint32_t)cap);
-      count_launches(2);
-      if (!a.per_layer) {
-        select_candidates_kernel<<<n_sel, 1024, 0, s>>>(sc.state, sc.cand, (uint32_t)cap,
-                                                        (unsigned long long)a.k_rest);
-        count_launches(1);
-      } else {
-        const int cand_grid = 148 * 4;
-        cand_begin_kernel<<<1, 1, 0, s>>>(sc.state, (uint32_t)cap, (unsigned long long)a.k_rest);
-        for (int pass = 0; pass < kPasses; ++pass) {
-          cand_histogram_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, pass, sc.hist);
-          pick_digit_kernel<<<1, 256, 0, s>>>(sc.state, sc.hist, pass, 1);
-        }
-        cand_ties_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, sc.tie_list);
-        cand_finish_kernel<<<1, 1024, 0, s>>>(sc.state, sc.tie_list);
-        count_launches(3 + 2 * kPasses);
+      // the threshold among the collected keys: the same three digits, on offsets from the lower pivot
+      const dim3 cand_grid(ceil_div(148 * 4, n_sel), n_sel);
+      for (int pass = 0; pass < kPasses; ++pass) {
+        cand_histogram_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap,
+                                                             (unsigned long long)a.k_rest, pass, sc.hist);
+        pick_digit_kernel<<<n_sel, 256, 0, s>>>(sc.state, sc.hist, pass, 1, (uint32_t)cap,
+                                                (unsigned long long)a.k_rest);
       }
+      cand_ties_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, sc.tie_list);
+      cand_finish_kernel<<<n_sel, 1024, 0, s>>>(sc.state, sc.tie_list);
+      count_launches(4 + 2 * kPasses);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     for (int pass = 0; pass < kPasses; ++pass) {
@@ -843,7 +892,7 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
                                                        sc.hist);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
-      pick_digit_kernel<<<n_sel, 256, 0, s>>>(sc.state, sc.hist, pass, 0);
+      pick_digit_kernel<<<n_sel, 256, 0, s>>>(sc.state, sc.hist, pass, 0, 0u, 0ull);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
