@@ -339,7 +339,9 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
   return x ^ (x >> 31);
 }
 
-// One CTA per head: samples the head and sets the bracket [lo, hi] around the expected threshold.
+// Two CTAs per selection (blockIdx.y = 0: upper pivot, 1: lower pivot), each of which samples the
+// selection's entries (the same draws) and sets its end of the bracket [lo, hi] around the
+// expected threshold.
 __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
                                                              int causal, int diag, unsigned long long k_rest,
                                                              unsigned long long n_rest, SelectState *state) {
@@ -352,14 +354,21 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
   if (t == 0) n_valid_s = 0u;
   __syncthreads();
   const unsigned long long cells = (unsigned long long)Lq * Lk;
-  for (int s = t; s < kSamples; s += 1024) {
+  constexpr int kDraws = kSamples / 1024;  // per thread, all loads in flight at once
+  float drawn[kDraws];
+  bool valid[kDraws];
+#pragma unroll
+  for (int u = 0; u < kDraws; ++u) {
+    const int s = t + 1024 * u;
     const unsigned long long idx = mix64(((unsigned long long)h << 32) | (unsigned)s) % cells;
     const int i = (int)(idx / Lk), j = (int)(idx % Lk);
     const int ii = i % period;
-    if ((causal && j > ii) || (diag && j == ii)) continue;
-    const uint32_t pos = atomicAdd(&n_valid_s, 1u);
-    keys[pos] = key_of(acc[((size_t)h * Lq + i) * Lk + j]);
+    valid[u] = !((causal && j > ii) || (diag && j == ii));
+    drawn[u] = valid[u] ? acc[((size_t)h * Lq + i) * Lk + j] : 0.f;
   }
+#pragma unroll
+  for (int u = 0; u < kDraws; ++u)
+    if (valid[u]) keys[atomicAdd(&n_valid_s, 1u)] = key_of(drawn[u]);
   __syncthreads();
   const uint32_t nv = n_valid_s;
   if (nv < 1024u) return;  // too few draws landed in the domain: no shortcut for this head
@@ -368,44 +377,62 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
   const double r = frac * nv;
   const double dev = 6.0 * sqrt(fmax(r * (1.0 - frac), 1.0)) + 16.0;
   const long long r_hi = (long long)floor(r - dev), r_lo = (long long)ceil(r + dev);
-  uint32_t hi = 0xffffffffu, lo = 0u;
-  if (r_hi >= 1) hi = block_select(keys, nv, (uint32_t)r_hi, hist, xch).key;
-  if (r_lo <= (long long)nv) lo = block_select(keys, nv, (uint32_t)r_lo, hist, xch).key;
-  if (t == 0) {
-    state[h].hi = hi;
-    state[h].lo = lo;
-    state[h].use_shortcut = 1u;
+  if (blockIdx.y == 0) {
+    uint32_t hi = 0xffffffffu;
+    if (r_hi >= 1) hi = block_select(keys, nv, (uint32_t)r_hi, hist, xch).key;
+    if (t == 0) state[h].hi = hi;
+  } else {
+    uint32_t lo = 0u;
+    if (r_lo <= (long long)nv) lo = block_select(keys, nv, (uint32_t)r_lo, hist, xch).key;
+    if (t == 0) state[h].lo = lo;
   }
+  if (t == 0) state[h].use_shortcut = 1u;  // both CTAs take the same decision
 }
 
 // One pass over the selection's rows: counts the keys above the upper pivot and collects those
 // inside the bracket.  grid = (row blocks, selections); a warp takes a row at a time.  Values are
 // compared with the pivots as floats (the same order as their keys); the key is computed for the
-// collected entries only.  Collected entries are staged in shared memory and appended to the
-// selection's buffer with one reservation per CTA (entries that do not fit the stage any more
-// go straight to the buffer).
-constexpr int kStageKeys = 4096;
+// collected entries only.  Each warp stages its collected entries in shared memory and appends
+// them to the selection's buffer, one reservation per flush, whenever the stage is half full at
+// the end of a chunk of the row (an entry that finds the stage full goes straight to the buffer).
+constexpr int kWarpStage = 512;
 __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
                                                            int causal, int diag, SelectState *state,
                                                            uint2 *__restrict__ cand, uint32_t cand_cap) {
-  __shared__ uint2 stage[kStageKeys];
-  __shared__ uint32_t stage_n, stage_base;  // stage_n only grows; positions beyond the stage were not staged
+  __shared__ uint2 stage_all[kWarps][kWarpStage];
+  __shared__ uint32_t stage_n_all[kWarps];  // may run past the stage: those entries were not staged
   const int h = blockIdx.y;
   if (!state[h].use_shortcut) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) stage_n = 0u;
-  __syncthreads();
+  uint2 *stage = stage_all[warp];
+  uint32_t *stage_n = &stage_n_all[warp];
+  if (lane == 0) *stage_n = 0u;
+  __syncwarp();
   const float lo_f = float_of_key(state[h].lo), hi_f = float_of_key(state[h].hi);
   uint2 *out = cand + (size_t)h * cand_cap;
   uint32_t *n_cand = &state[h].n_cand;
   auto push = [&](float f, uint32_t index) {  // a few per cent of the entries
     const uint2 entry = make_uint2(key_of(f), index);
-    const uint32_t pos = atomicAdd(&stage_n, 1u);
-    if (pos < (uint32_t)kStageKeys) {
+    const uint32_t pos = atomicAdd(stage_n, 1u);
+    if (pos < (uint32_t)kWarpStage) {
       stage[pos] = entry;
     } else {
       const uint32_t g = atomicAdd(n_cand, 1u);
       if (g < cand_cap) out[g] = entry;
+    }
+  };
+  auto flush = [&](uint32_t at_least) {  // by the whole warp
+    __syncwarp();
+    const uint32_t n = min(*stage_n, (uint32_t)kWarpStage);
+    if (n >= at_least && n > 0u) {
+      uint32_t dst = 0u;
+      if (lane == 0) dst = atomicAdd(n_cand, n);
+      dst = __shfl_sync(0xffffffffu, dst, 0);
+      for (uint32_t e = lane; e < n; e += 32)
+        if (dst + e < cand_cap) out[dst + e] = stage[e];
+      __syncwarp();
+      if (lane == 0) *stage_n = 0u;
+      __syncwarp();
     }
   };
   const bool vec = (Lk & 3) == 0;
@@ -447,19 +474,14 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
           }
         }
       }
+      flush(kWarpStage / 2);
     }
   }
+  flush(1u);
   unsigned long long above_warp = above;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) above_warp += __shfl_xor_sync(0xffffffffu, above_warp, o);
   if (lane == 0 && above_warp) atomicAdd(&state[h].above_hi, above_warp);
-  __syncthreads();
-  const uint32_t n = min(stage_n, (uint32_t)kStageKeys);
-  if (threadIdx.x == 0) stage_base = atomicAdd(n_cand, n);
-  __syncthreads();
-  const uint32_t dst = stage_base;
-  for (uint32_t e = threadIdx.x; e < n; e += kThreads)
-    if (dst + e < cand_cap) out[dst + e] = stage[e];
 }
 
 // ---- selection among the collected keys: the radix select on their offsets from the lower pivot ----
@@ -483,15 +505,23 @@ __global__ void __launch_bounds__(kThreads) cand_histogram_kernel(const SelectSt
   const uint32_t want_hi = (pass == 0 ? 0u : st.prefix) & hi_mask;
   const uint32_t n = st.n_cand, lo = st.lo;
   const uint2 *mine = cand + (size_t)h * cand_cap;
-  for (uint32_t base = blockIdx.x * kThreads; base < n; base += gridDim.x * kThreads) {  // warp-uniform
-    const uint32_t idx = base + threadIdx.x;
-    const uint32_t key = idx < n ? mine[idx].x - lo : 0u;
-    const bool take = idx < n && (key & hi_mask) == want_hi;
-    const uint32_t bin = (key >> shift) & dmask;
-    const unsigned voters = __ballot_sync(0xffffffffu, take);
-    if (take) {
-      const unsigned peers = __match_any_sync(voters, bin);
-      if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], (uint32_t)__popc(peers));
+  for (uint32_t base = blockIdx.x * (4 * kThreads); base < n; base += gridDim.x * (4 * kThreads)) {  // warp-uniform
+    uint32_t key[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {  // four loads in flight
+      const uint32_t idx = base + u * kThreads + threadIdx.x;
+      key[u] = idx < n ? mine[idx].x - lo : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t idx = base + u * kThreads + threadIdx.x;
+      const bool take = idx < n && (key[u] & hi_mask) == want_hi;
+      const uint32_t bin = (key[u] >> shift) & dmask;
+      const unsigned voters = __ballot_sync(0xffffffffu, take);
+      if (take) {
+        const unsigned peers = __match_any_sync(voters, bin);
+        if (lane == __ffs(peers) - 1) atomicAdd(&sh[bin], (uint32_t)__popc(peers));
+      }
     }
   }
   __syncthreads();
@@ -870,12 +900,15 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
       const size_t smem = (kSamples + kBins) * sizeof(uint32_t);
       e = cudaFuncSetAttribute(sample_pivots_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
-      sample_pivots_kernel<<<n_sel, 1024, smem, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
+      sample_pivots_kernel<<<dim3(n_sel, 2), 1024, smem, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
                                                      (unsigned long long)a.k_rest, (unsigned long long)n_rest, sc.state);
-      collect_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag, sc.state, sc.cand,
-                                               (uint32_t)cap);
+      // one wave of CTAs (five fit an SM), so that no SM idles while a second, partial wave runs
+      int collect_blocks = ceil_div(rows, kWarps);
+      if (collect_blocks > 148 * 5 / n_sel) collect_blocks = max(148 * 5 / n_sel, 1);
+      collect_kernel<<<dim3(collect_blocks, n_sel), kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
+                                                                     sc.state, sc.cand, (uint32_t)cap);
       // the threshold among the collected keys: the same three digits, on offsets from the lower pivot
-      const dim3 cand_grid(ceil_div(148 * 4, n_sel), n_sel);
+      const dim3 cand_grid(ceil_div(148 * 8, n_sel), n_sel);
       for (int pass = 0; pass < kPasses; ++pass) {
         cand_histogram_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap,
                                                              (unsigned long long)a.k_rest, pass, sc.hist);

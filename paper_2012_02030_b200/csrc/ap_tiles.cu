@@ -51,11 +51,13 @@ __global__ void __launch_bounds__(128) stage_from_mask_kernel(const uint8_t *__r
     stage_count[tile] = warp_count[0] + warp_count[1] + warp_count[2] + warp_count[3];
 }
 
-// Single CTA: exclusive scan of "tile is non-empty" over the (h, qt, kt) order.
+// Single CTA: exclusive scan of "tile is non-empty" over the (h, qt, kt) order.  A thread takes
+// sixteen consecutive tiles at a time (all loads in flight), the CTA scans the threads' sums.
 __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restrict__ stage_count,
                                                           int32_t *__restrict__ stage_pos, int n_tiles,
                                                           int n_kt, int cap, int32_t *__restrict__ row_ptr,
                                                           unsigned *err) {
+  constexpr int kPer = 16;
   __shared__ int warp_sums[32];
   __shared__ int carry_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -64,10 +66,15 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
     row_ptr[0] = 0;
   }
   __syncthreads();
-  for (int base = 0; base < n_tiles; base += 1024) {
-    const int idx = base + threadIdx.x;
-    const int flag = (idx < n_tiles && stage_count[idx] > 0) ? 1 : 0;
-    int incl = flag;
+  for (int base = 0; base < n_tiles; base += 1024 * kPer) {
+    const int idx0 = base + (int)threadIdx.x * kPer;
+    int cnt[kPer];
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) cnt[e] = idx0 + e < n_tiles ? stage_count[idx0 + e] : 0;
+    int mine = 0;
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) mine += cnt[e] > 0 ? 1 : 0;
+    int incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       int v = __shfl_up_sync(0xffffffffu, incl, o);
@@ -86,10 +93,16 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
     }
     __syncthreads();
     const int carry = carry_s;
-    const int before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - flag;
-    if (idx < n_tiles) {
-      stage_pos[idx] = flag ? before : -1;
-      if (idx % n_kt == n_kt - 1) row_ptr[idx / n_kt + 1] = min(before + flag, cap);
+    int before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - mine;
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) {
+      const int idx = idx0 + e;
+      const int flag = cnt[e] > 0 ? 1 : 0;
+      if (idx < n_tiles) {
+        stage_pos[idx] = flag ? before : -1;
+        if (idx % n_kt == n_kt - 1) row_ptr[idx / n_kt + 1] = min(before + flag, cap);
+      }
+      before += flag;
     }
     __syncthreads();
     if (threadIdx.x == 1023) carry_s = carry + warp_sums[31];
