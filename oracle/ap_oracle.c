@@ -55,10 +55,24 @@ void oracle_set_num_threads(int n) {
 #endif
 }
 
-/* Row domain: all keys, or keys j <= i under the causal constraint. */
-static int row_domain_end(int i, int Lk, int causal) {
+/*
+ * Row domain: all keys, or, under the causal constraint, keys j <= i + (Lk - Lq).
+ * With Lq == Lk that is j <= i.  With Lk = mem + Lq it is the mask of a model that
+ * attends to `mem` cached positions of earlier segments, all visible, followed by
+ * the current segment under its autoregressive mask (the Transformer-XL masks of
+ * the language-modelling section: memory in the left half, causal right half).
+ * Query i's own position is key i + (Lk - Lq).  Needs Lk >= Lq.
+ */
+static int row_domain_end(int i, int Lq, int Lk, int causal) {
   if (!causal) return Lk;
-  return (i + 1 < Lk) ? i + 1 : Lk;
+  int end = i + 1 + (Lk - Lq);
+  if (end < 0) end = 0;
+  return end < Lk ? end : Lk;
+}
+
+/* Forced entries of Eq. 2's selection: each query's own position, when asked for. */
+static int is_forced(int i, int j, int Lq, int Lk, int causal, int keep_diag) {
+  return keep_diag && (Lq == Lk || causal) && j == i + (Lk - Lq);
 }
 
 /*
@@ -73,7 +87,7 @@ static int row_domain_end(int i, int Lk, int causal) {
  */
 static void accumulate_row(double *arow, const float *Q, const float *K, const float *bias, int h,
                            int i, int B, int H, int Lq, int Lk, int d, int causal, double scale) {
-  int jend = row_domain_end(i, Lk, causal);
+  int jend = row_domain_end(i, Lq, Lk, causal);
   double *s = (double *)malloc(sizeof(double) * (size_t)(jend > 0 ? jend : 1));
   for (int b = 0; b < B; ++b) {
     const float *q = Q + (((size_t)b * H + h) * Lq + i) * d;
@@ -150,8 +164,9 @@ int64_t oracle_keep_count(int64_t n_valid, int64_t n_forced, double keep_frac) {
 /*
  * Eq. 2 as an exact per-head top-k: an entry is pruned (M_p = -inf) iff it does
  * not belong to the k largest entries of the head's average attention matrix.
- *   domain   all (i,j), or j <= i when causal
- *   forced   the diagonal, when keep_diag and Lq == Lk
+ *   domain   all (i,j), or j <= i + (Lk - Lq) when causal
+ *   forced   each query's own position j = i + (Lk - Lq), when keep_diag and
+ *            (Lq == Lk or causal)
  *   k        max(|forced|, min(n_valid, floor(keep_frac * n_valid + 0.5)))
  *   order    forced first, value descending (as fp32), index i*Lk+j ascending
  * mask[h,i,j] = 1 for the first k entries in that order, 0 elsewhere;
@@ -164,7 +179,7 @@ int oracle_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac,
 #pragma omp parallel for schedule(dynamic, 1)
   for (int h = 0; h < H; ++h) {
     int64_t n_valid = 0;
-    for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lk, causal);
+    for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lq, Lk, causal);
     ap_entry *e = (ap_entry *)malloc(sizeof(ap_entry) * (size_t)(n_valid > 0 ? n_valid : 1));
     if (!e) {
       failed = 1;
@@ -172,10 +187,10 @@ int oracle_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac,
     }
     int64_t n = 0, n_forced = 0;
     for (int i = 0; i < Lq; ++i) {
-      int jend = row_domain_end(i, Lk, causal);
+      int jend = row_domain_end(i, Lq, Lk, causal);
       for (int j = 0; j < jend; ++j) {
         e[n].value = acc[((size_t)h * Lq + i) * Lk + j];
-        e[n].forced = (keep_diag && Lq == Lk && i == j) ? 1 : 0;
+        e[n].forced = is_forced(i, j, Lq, Lk, causal, keep_diag);
         e[n].index = (int64_t)i * Lk + j;
         n_forced += e[n].forced;
         ++n;
@@ -196,7 +211,7 @@ int oracle_build_mask(const float *acc, int H, int Lq, int Lk, double keep_frac,
  * layer together, so heads keep unequal numbers of entries.  Read, like the
  * per-head variant, as an exact top-k: the population is the union of the
  * heads' domains (N = H * n_valid entries), the diagonals of all heads are
- * forced (when keep_diag and Lq == Lk) and counted inside
+ * forced (under the per-head rule's condition) and counted inside
  *   k = max(#forced, min(N, floor(keep_frac * N + 0.5))),
  * and the order is: forced first, then larger value, then lower global index
  * (h * Lq + i) * Lk + j.  mask[h,i,j] = 1 for the first k entries; nnz[h] =
@@ -206,7 +221,7 @@ int oracle_build_mask_layer(const float *acc, int H, int Lq, int Lk, double keep
                             int keep_diag, uint8_t *mask, int64_t *nnz) {
   memset(mask, 0, (size_t)H * Lq * Lk);
   int64_t n_valid = 0;
-  for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lk, causal);
+  for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lq, Lk, causal);
   int64_t N = n_valid * H;
   ap_entry *e = (ap_entry *)malloc(sizeof(ap_entry) * (size_t)(N > 0 ? N : 1));
   if (!e) return -1;
@@ -214,10 +229,10 @@ int oracle_build_mask_layer(const float *acc, int H, int Lq, int Lk, double keep
   for (int h = 0; h < H; ++h) {
     nnz[h] = 0;
     for (int i = 0; i < Lq; ++i) {
-      int jend = row_domain_end(i, Lk, causal);
+      int jend = row_domain_end(i, Lq, Lk, causal);
       for (int j = 0; j < jend; ++j) {
         e[n].value = acc[((size_t)h * Lq + i) * Lk + j];
-        e[n].forced = (keep_diag && Lq == Lk && i == j) ? 1 : 0;
+        e[n].forced = is_forced(i, j, Lq, Lk, causal, keep_diag);
         e[n].index = ((int64_t)h * Lq + i) * Lk + j;
         n_forced += e[n].forced;
         ++n;

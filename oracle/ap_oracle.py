@@ -69,6 +69,12 @@ def keep_count(n_valid: int, n_forced: int, keep_frac: float) -> int:
     return int(_load().oracle_keep_count(n_valid, n_forced, float(keep_frac)))
 
 
+def _check_domain(Lq: int, Lk: int, causal: bool) -> None:
+    """Causal: keys j <= i + (Lk - Lq), i.e. Lk - Lq memory keys before the current segment."""
+    if causal and Lk < Lq:
+        raise ValueError("the causal domain needs Lk >= Lq")
+
+
 def accumulate(acc: np.ndarray, Q, K, bias=None, causal: bool = False, scale: float | None = None):
     """Eq. 1 as a running sum: acc[H,Lq,Lk] (float64, in place) += sum_b softmax(Q_b K_b^T*scale + bias)."""
     Q, K = _f32(Q), _f32(K)
@@ -76,6 +82,7 @@ def accumulate(acc: np.ndarray, Q, K, bias=None, causal: bool = False, scale: fl
     Lk = K.shape[2]
     assert K.shape == (B, H, Lk, d) and acc.shape == (H, Lq, Lk)
     assert acc.dtype == np.float64 and acc.flags.c_contiguous
+    _check_domain(Lq, Lk, causal)
     if bias is not None:
         bias = _f32(bias)
         assert bias.shape == (H, Lq, Lk)
@@ -92,6 +99,7 @@ def accumulate_rows(rows, Q, K, bias=None, causal: bool = False, scale: float | 
     Q, K = _f32(Q), _f32(K)
     B, H, Lq, d = Q.shape
     Lk = K.shape[2]
+    _check_domain(Lq, Lk, causal)
     rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int32).reshape(-1, 2))
     out = np.zeros((rows.shape[0], Lk), dtype=np.float64)
     if bias is not None:
@@ -108,6 +116,7 @@ def build_mask(acc32, keep_frac: float, causal: bool = False, keep_diag: bool = 
     """Eq. 2 as exact per-head top-k on fp32 values; returns (mask uint8 [H,Lq,Lk], nnz int64 [H])."""
     acc32 = _f32(acc32)
     H, Lq, Lk = acc32.shape
+    _check_domain(Lq, Lk, causal)
     mask = np.zeros((H, Lq, Lk), dtype=np.uint8)
     nnz = np.zeros((H,), dtype=np.int64)
     rc = _load().oracle_build_mask(
@@ -124,6 +133,7 @@ def build_mask_layer(acc32, keep_frac: float, causal: bool = False, keep_diag: b
     top-k over the union of the heads' domains; returns (mask uint8 [H,Lq,Lk], nnz int64 [H])."""
     acc32 = _f32(acc32)
     H, Lq, Lk = acc32.shape
+    _check_domain(Lq, Lk, causal)
     mask = np.zeros((H, Lq, Lk), dtype=np.uint8)
     nnz = np.zeros((H,), dtype=np.int64)
     lib = _load()

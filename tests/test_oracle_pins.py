@@ -182,6 +182,32 @@ def test_acc_rows_sum_to_sample_count_and_rect_shapes():
         np.testing.assert_array_equal(got[r], acc[h, i])
 
 
+@pytest.mark.parametrize("with_bias", [False, True])
+def test_acc_causal_with_memory_keys_equals_library_softmax_sum(with_bias):
+    """Lk = mem + Lq: query i attends to keys 0 .. mem + i (a library softmax over an additive
+    -inf mask with the diagonal shifted by mem); entries outside stay untouched."""
+    B, H, Lq, mem, d = 3, 2, 23, 18, 16
+    Lk = mem + Lq
+    q, k = _rand((B, H, Lq, d), 36), _rand((B, H, Lk, d), 37)
+    bias = _rand((H, Lq, Lk), 38, torch.float32) if with_bias else None
+    acc = np.zeros((H, Lq, Lk))
+    orc.accumulate(acc, q.numpy(), k.numpy(), None if bias is None else bias.numpy(), causal=True)
+    s = torch.einsum("bhid,bhjd->bhij", q.double(), k.double()) / math.sqrt(d)
+    if with_bias:
+        s = s + bias.double()
+    dom = torch.tril(torch.ones(Lq, Lk, dtype=torch.bool), diagonal=mem)
+    ref = torch.softmax(s.masked_fill(~dom, float("-inf")), dim=-1).sum(0)
+    np.testing.assert_allclose(acc, ref.numpy(), rtol=1e-12, atol=1e-14)
+    assert np.all(acc[:, ~dom.numpy()] == 0.0)
+    np.testing.assert_allclose(acc.sum(-1), B, rtol=1e-13)
+    rows = [(0, 0), (1, Lq - 1), (1, 7)]
+    got = orc.accumulate_rows(rows, q.numpy(), k.numpy(), None if bias is None else bias.numpy(), causal=True)
+    for r, (h, i) in enumerate(rows):
+        np.testing.assert_array_equal(got[r], acc[h, i])
+    with pytest.raises(ValueError):
+        orc.accumulate(np.zeros((H, Lk, Lq)), k.numpy(), q.numpy(), causal=True)
+
+
 def test_acc_zero_queries_closed_form():
     B, H, L, d = 4, 1, 12, 8
     k = _rand((B, H, L, d), 35)
@@ -200,7 +226,14 @@ def test_acc_zero_queries_closed_form():
 
 
 def _domain(Lq, Lk, causal):
-    return [(i, j) for i in range(Lq) for j in range(Lk) if (not causal or j <= i)]
+    """All (i, j), or under the causal constraint those with j <= i + (Lk - Lq): Lk - Lq memory
+    keys that every query sees, then the current segment under its autoregressive mask."""
+    return [(i, j) for i in range(Lq) for j in range(Lk) if (not causal or j <= i + (Lk - Lq))]
+
+
+def _forced(dom, Lq, Lk, causal, keep_diag):
+    """Each query's own position, when asked for and defined (square, or causal with memory)."""
+    return [(i, j) for (i, j) in dom if keep_diag and (Lq == Lk or causal) and j == i + (Lk - Lq)]
 
 
 def _brute_force_mask(acc, keep_frac, causal, keep_diag):
@@ -208,7 +241,7 @@ def _brute_force_mask(acc, keep_frac, causal, keep_diag):
     with the largest exact sum; among those, the first in index order."""
     Lq, Lk = acc.shape
     dom = _domain(Lq, Lk, causal)
-    forced = [(i, j) for (i, j) in dom if keep_diag and Lq == Lk and i == j]
+    forced = _forced(dom, Lq, Lk, causal, keep_diag)
     n_valid = len(dom)
     k = max(len(forced), min(n_valid, int(math.floor(keep_frac * n_valid + 0.5))))
     free = [e for e in dom if e not in forced]
@@ -250,6 +283,49 @@ def test_mask_brute_force_rectangular():
         np.testing.assert_array_equal(got[0], want)
 
 
+@pytest.mark.parametrize("keep_diag", [False, True])
+def test_mask_brute_force_causal_with_memory_keys(keep_diag):
+    """Lk = mem + Lq: the memory keys are visible to every query, the current segment is causal
+    (the Transformer-XL masks of the language-modelling section); the forced entry of query i is
+    its own position mem + i."""
+    rng = np.random.default_rng(47)
+    for (Lq, Lk) in ((2, 3), (2, 5), (3, 4), (3, 5)):
+        for keep in (0.3, 0.6):
+            for trial in range(4):
+                acc = rng.integers(0, 4, size=(1, Lq, Lk)).astype(np.float32) / 4.0
+                want, k = _brute_force_mask(acc[0], keep, True, keep_diag)
+                got, nnz = orc.build_mask(acc, keep, causal=True, keep_diag=keep_diag)
+                assert nnz[0] == k
+                np.testing.assert_array_equal(got[0], want)
+                if keep_diag:
+                    assert all(got[0, i, Lk - Lq + i] == 1 for i in range(Lq))
+                assert not got[0][~np.tril(np.ones((Lq, Lk), dtype=bool), Lk - Lq)].any()
+    with pytest.raises(ValueError):
+        orc.build_mask(np.zeros((1, 3, 2), dtype=np.float32), 0.5, causal=True)
+
+
+def test_mask_causal_with_memory_equals_last_rows_of_the_square_problem():
+    """The domain of (Lq, mem + Lq) is the last Lq rows of the square causal domain of size
+    mem + Lq.  With the upper rows of the square problem far below every other value they are the
+    last to be kept, so with a count chosen accordingly the square problem's mask restricted to
+    the last rows is the rectangular problem's mask."""
+    rng = np.random.default_rng(48)
+    Lq, mem = 29, 35
+    Lk = mem + Lq
+    rect = rng.random((2, Lq, Lk), dtype=np.float32)
+    rect[1] = np.round(rect[1] * 6) / 6                    # ties
+    square = np.full((2, Lk, Lk), -1.0, dtype=np.float32)
+    square[:, mem:, :] = rect
+    n_rect = Lq * (Lq + 1) // 2 + Lq * mem
+    n_square = Lk * (Lk + 1) // 2
+    k = 300
+    got, nnz = orc.build_mask(rect, k / n_rect, causal=True, keep_diag=False)
+    want, _ = orc.build_mask(square, k / n_square, causal=True, keep_diag=False)
+    assert nnz.tolist() == [k, k]
+    np.testing.assert_array_equal(got, want[:, mem:, :])
+    assert not want[:, :mem, :].any()
+
+
 @pytest.mark.parametrize("causal", [False, True])
 def test_mask_invariants(causal):
     rng = np.random.default_rng(42)
@@ -286,7 +362,7 @@ def _brute_force_layer(acc, keep_frac, causal, keep_diag):
     entries, the one with the largest exact sum; among those, the first in global index order."""
     H, Lq, Lk = acc.shape
     dom = [(h, i, j) for h in range(H) for (i, j) in _domain(Lq, Lk, causal)]
-    forced = [e for e in dom if keep_diag and Lq == Lk and e[1] == e[2]]
+    forced = [e for e in dom if keep_diag and (Lq == Lk or causal) and e[2] == e[1] + (Lk - Lq)]
     N = len(dom)
     k = max(len(forced), min(N, int(math.floor(keep_frac * N + 0.5))))
     free = [e for e in dom if e not in forced]
