@@ -25,7 +25,13 @@
  *     enqueued.  Nothing throws, aborts or traps.  Conditions only the device
  *     can see (a tile list that outgrew its capacity, a bounded wait that
  *     expired) set a sticky device word that ap_device_status() returns.
- *   - d is 64 or 128.  Any Lq, Lk >= 1 is accepted; `causal` needs Lq == Lk.
+ *   - d is 64 or 128.  Any Lq, Lk >= 1 is accepted.
+ *   - `causal` != 0 restricts query i to the keys j <= i + (Lk - Lq) and needs
+ *     Lk >= Lq.  With Lq == Lk that is the usual autoregressive mask; with
+ *     Lk = mem + Lq the first `mem` keys are cached positions of earlier segments,
+ *     visible to every query, followed by the current segment under its
+ *     autoregressive mask (the Transformer-XL masks of the paper's language-
+ *     modelling section).  Query i's own position is key i + (Lk - Lq).
  *   - There is no CPU fallback: without a CUDA device the compute calls return
  *     AP_ERR_CUDA.
  */
@@ -125,7 +131,7 @@ size_t ap_mask_to_tiles_workspace_bytes(int H, int Lq, int Lk);
 /*
  * Eq. 1 (with the attention matrix of Section 3.1), as a running sum:
  *   acc[h,i,j] += sum_{b<B} softmax_j( Q[b,h,i,:].K[b,h,j,:] * scale + bias[h,i,j] )
- * over the row's domain (all j, or j <= i when causal); entries outside the
+ * over the row's domain (all j, or the causal domain above); entries outside the
  * domain are not touched.  The 1/n of Eq. 1 is left to the caller, who counts
  * the samples: the selection of Eq. 2 does not depend on it.
  *   acc    [H,Lq,Lk] fp32, in/out.  The sum over b is taken in ascending b with no
@@ -141,8 +147,9 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
 /*
  * Eq. 2 with one threshold per head, as an exact top-k: an entry is pruned
  * unless it is among the k largest of its head.
- *   domain  all (i,j), or j <= i when causal; n_valid = its size
- *   forced  the diagonal when keep_diag != 0 and Lq == Lk (counted inside k)
+ *   domain  all (i,j), or the causal domain; n_valid = its size
+ *   forced  when keep_diag != 0 and (Lq == Lk or causal): every query's own
+ *           position j = i + (Lk - Lq) (counted inside k)
  *   k       max(#forced, min(n_valid, floor(keep_frac*n_valid + 0.5))), in double
  *   order   forced first, then larger fp32 value, then lower index i*Lk + j
  * Outputs (any of mask / tiles / nnz_per_head may be NULL):
@@ -163,7 +170,7 @@ ap_status ap_build_mask(const float *acc, int H, int Lq, int Lk, double keep_fra
  * layer), i.e. an exact top-k over the union of the heads' domains, so that heads keep unequal
  * numbers of entries.  Same arguments, outputs and conventions as ap_build_mask with
  *   domain  the union over h of head h's domain; N = H * n_valid entries
- *   forced  every head's diagonal when keep_diag != 0 and Lq == Lk (counted inside k)
+ *   forced  every head's forced entries under the per-head rule (counted inside k)
  *   k       max(#forced, min(N, floor(keep_frac*N + 0.5))), in double
  *   order   forced first, then larger fp32 value, then lower index (h*Lq + i)*Lk + j
  *   nnz_per_head[h]  entries kept in head h (they sum to k)

@@ -53,7 +53,8 @@ __global__ void __launch_bounds__(kThreads) accumulate_simt_kernel(float *__rest
   const int n_rows = min(rows, Lq - i0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // keys any row of this block may look at
-  const int jmax = causal ? min(Lk, i0 + n_rows) : Lk;
+  const int off = causal ? Lk - Lq : 0;  // causal: row i looks at keys j <= i + (Lk - Lq)
+  const int jmax = causal ? min(Lk, i0 + n_rows + off) : Lk;
 
   for (int b = 0; b < B; ++b) {
     const T *Qb = Q + (((size_t)b * H + h) * Lq + i0) * D;
@@ -95,7 +96,7 @@ __global__ void __launch_bounds__(kThreads) accumulate_simt_kernel(float *__rest
     // warp r normalises row r and adds it to the accumulator
     for (int r = warp; r < n_rows; r += kThreads / 32) {
       const int i = i0 + r;
-      const int jend = causal ? min(Lk, i + 1) : Lk;
+      const int jend = causal ? min(Lk, i + 1 + off) : Lk;
       const float *srow = s_s + (size_t)r * Lk;
       float m = -CUDART_INF_F;
       for (int j = lane; j < jend; j += 32) m = fmaxf(m, srow[j]);

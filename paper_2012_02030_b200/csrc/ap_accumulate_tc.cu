@@ -105,7 +105,9 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const int qt = n_qt - 1 - (int)(blockIdx.x / H);
   const int h = blockIdx.x % H;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_k = causal ? min(n_kt, qt + 1) : n_kt;  // key tiles this query tile looks at
+  // causal: row i looks at keys j <= i + (Lk - Lq), i.e. Lk - Lq memory keys, then its own segment
+  const int off = causal ? Lk - Lq : 0;
+  const int n_k = causal ? min(n_kt, (qt * kTile + kTile - 1 + off) / kTile + 1) : n_kt;  // key tiles of this query tile
   const int visits_per_sweep = n_k * Bc;
   const int n_visits = 2 * visits_per_sweep;
 
@@ -202,7 +204,7 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int i = qt * kTile + r;
     const bool row_ok = i < Lq;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const int jend = causal ? min(Lk, i + 1) : Lk;  // first key outside this row's domain
+    const int jend = causal ? min(Lk, i + 1 + off) : Lk;  // first key outside this row's domain
     const bool vec = (Lk & 3) == 0;
     float2 *my_stats = stats + (size_t)wg * kMaxB * 128 + r;  // + b * 128
     for (int b = 0; b < Bc; ++b) my_stats[b * 128] = make_float2(-CUDART_INF_F, 0.f);

@@ -75,9 +75,8 @@ unsigned *device_error_word() {
 
 int64_t domain_size(int Lq, int Lk, int causal) {
   if (!causal) return (int64_t)Lq * Lk;
-  int64_t n = 0;
-  for (int i = 0; i < Lq; ++i) n += (i + 1 < Lk) ? i + 1 : Lk;
-  return n;
+  // row i sees the keys j <= i + (Lk - Lq), Lk >= Lq
+  return (int64_t)Lq * (Lq + 1) / 2 + (int64_t)Lq * (Lk - Lq);
 }
 
 int64_t keep_count(int64_t n_valid, int64_t n_forced, double keep_frac) {
@@ -128,7 +127,7 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
                                   int Lq, int Lk, int d, ap_dtype dt, int causal, float scale, void *stream) {
   if (!acc || !Q || !K || !aligned16(acc) || !aligned16(Q) || !aligned16(K) || (bias && !aligned16(bias)))
     return AP_ERR_INVALID_ARG;
-  if (B < 1 || !shape_ok(H, Lq, Lk) || (causal && Lq != Lk) || !(scale >= 0.f) || isinf(scale))
+  if (B < 1 || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq) || !(scale >= 0.f) || isinf(scale))
     return AP_ERR_INVALID_ARG;
   if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
@@ -145,7 +144,7 @@ namespace {
 ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
                           uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
                           size_t workspace_bytes, void *stream, int per_layer) {
-  if (!acc || !aligned16(acc) || !shape_ok(H, Lq, Lk) || (causal && Lq != Lk)) return AP_ERR_INVALID_ARG;
+  if (!acc || !aligned16(acc) || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq)) return AP_ERR_INVALID_ARG;
   if (!(keep_frac > 0.0) || !(keep_frac <= 1.0)) return AP_ERR_INVALID_ARG;
   if (mask && !aligned16(mask)) return AP_ERR_INVALID_ARG;
   if (nnz_per_head && (reinterpret_cast<uintptr_t>(nnz_per_head) & 7u)) return AP_ERR_INVALID_ARG;
@@ -172,7 +171,7 @@ ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_f
   // population of one selection: a head's domain, or the union of the heads' domains
   const int64_t heads = per_layer ? H : 1;
   const int64_t n_valid = domain_size(Lq, Lk, a.causal) * heads;
-  const int64_t n_forced = ((a.keep_diag && Lq == Lk) ? Lq : 0) * heads;
+  const int64_t n_forced = ((a.keep_diag && (Lq == Lk || a.causal)) ? Lq : 0) * heads;
   a.k = keep_count(n_valid, n_forced, keep_frac);
   a.k_rest = a.k - n_forced;
   a.mask = mask;
@@ -223,11 +222,11 @@ ap_status ap_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles 
 }
 
 ap_status ap_dense_tiles(int H, int Lq, int Lk, int causal, ap_tiles *tiles, void *stream) {
-  if (!shape_ok(H, Lq, Lk) || (causal && Lq != Lk)) return AP_ERR_INVALID_ARG;
+  if (!shape_ok(H, Lq, Lk) || (causal && Lk < Lq)) return AP_ERR_INVALID_ARG;
   ap_status st = check_tiles(tiles, H, Lq, Lk, false);
   if (st != AP_OK) return st;
   const int n_qt = ceil_div(Lq, kTile), n_kt = ceil_div(Lk, kTile);
-  const int64_t need = (int64_t)H * (causal ? (int64_t)n_qt * (n_qt + 1) / 2 : (int64_t)n_qt * n_kt);
+  const int64_t need = (int64_t)H * dense_row_start(n_qt, n_kt, Lq, Lk, causal ? 1 : 0);
   if (tiles->cap < need) return AP_ERR_WORKSPACE;
   if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
   fill_tiles_shape(tiles, H, Lq, Lk);

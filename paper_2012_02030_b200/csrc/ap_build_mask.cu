@@ -143,6 +143,9 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int n_sel,
 // a time and its lanes stride over the row, two float4 loads in flight each.
 // Here and in the kernels below Lq counts the rows of the selection and row i has
 // the domain of row i % period of a head (period == Lq unless heads are stacked).
+// Under the causal constraint row r of a head sees the keys j <= r + (Lk - period):
+// Lk - period memory keys, then its own segment; its own position r + (Lk - period)
+// is the forced entry when the diagonal is kept.
 __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *__restrict__ acc, int Lq, int Lk,
                                                                    int period, int causal, int diag, int pass,
                                                                    const SelectState *__restrict__ state,
@@ -159,10 +162,11 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
   const uint32_t hi_mask = pass == 0 ? 0u : ~((1u << (shift + (pass == 1 ? 11 : 10))) - 1u);
   const uint32_t want_hi = prefix & hi_mask;
   const bool vec = (Lk & 3) == 0;
+  const int off = (causal || diag) ? Lk - period : 0;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
-    const int ii = i % period;
-    const int jend = causal ? min(Lk, ii + 1) : Lk;
+    const int own = i % period + off;  // the row's own position among the keys
+    const int jend = causal ? min(Lk, own + 1) : Lk;
     for (int base = 0; base < jend; base += 256) {  // warp-uniform trip count
       float v[2][4];
 #pragma unroll
@@ -178,7 +182,7 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
         for (int c = 0; c < 4; ++c) {
           const int j = j0 + c;
           const uint32_t key = key_of(v[u][c]);
-          const bool take = j < jend && !(diag && j == ii) && ((key & hi_mask) == want_hi);
+          const bool take = j < jend && !(diag && j == own) && ((key & hi_mask) == want_hi);
           const uint32_t bin = (key >> shift) & dmask;
           // lanes that hit the same bin elect one to add their count
           const unsigned voters = __ballot_sync(0xffffffffu, take);
@@ -354,6 +358,7 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
   if (t == 0) n_valid_s = 0u;
   __syncthreads();
   const unsigned long long cells = (unsigned long long)Lq * Lk;
+  const int off = (causal || diag) ? Lk - period : 0;
   constexpr int kDraws = kSamples / 1024;  // per thread, all loads in flight at once
   float drawn[kDraws];
   bool valid[kDraws];
@@ -362,8 +367,8 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
     const int s = t + 1024 * u;
     const unsigned long long idx = mix64(((unsigned long long)h << 32) | (unsigned)s) % cells;
     const int i = (int)(idx / Lk), j = (int)(idx % Lk);
-    const int ii = i % period;
-    valid[u] = !((causal && j > ii) || (diag && j == ii));
+    const int own = i % period + off;
+    valid[u] = !((causal && j > own) || (diag && j == own));
     drawn[u] = valid[u] ? acc[((size_t)h * Lq + i) * Lk + j] : 0.f;
   }
 #pragma unroll
@@ -437,10 +442,11 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
   };
   const bool vec = (Lk & 3) == 0;
   uint32_t above = 0u;  // per thread: fewer than 2^32 entries
+  const int off = (causal || diag) ? Lk - period : 0;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
-    const int ii = i % period;
-    const int jend = causal ? min(Lk, ii + 1) : Lk;
+    const int own = i % period + off;  // the row's own position among the keys
+    const int jend = causal ? min(Lk, own + 1) : Lk;
     const uint32_t row_index = (uint32_t)i * (uint32_t)Lk;
     for (int base = 0; base < jend; base += 512) {  // warp-uniform trip count
       float v[4][4];
@@ -453,7 +459,7 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int j0 = base + 128 * u + 4 * lane;
-        if (j0 + 4 <= jend && !(diag && ii >= j0 && ii < j0 + 4)) {
+        if (j0 + 4 <= jend && !(diag && own >= j0 && own < j0 + 4)) {
           // four entries of the domain: nothing to check per entry
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -467,7 +473,7 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
           for (int c = 0; c < 4; ++c) {
             const int j = j0 + c;
             const float f = v[u][c];
-            const bool in = j < jend && !(diag && j == ii);
+            const bool in = j < jend && !(diag && j == own);
             const bool gt = in && f > hi_f;
             above += gt ? 1u : 0u;
             if (in && !(f < lo_f) && !gt) push(f, row_index + (uint32_t)j);
@@ -597,10 +603,11 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t thr = state[h].thr;
   const bool vec = (Lk & 3) == 0;
+  const int off = (causal || diag) ? Lk - period : 0;
   for (int i = blockIdx.x * kWarps + warp; i < Lq; i += gridDim.x * kWarps) {
     const float *row = acc + ((size_t)h * Lq + i) * Lk;
-    const int ii = i % period;
-    const int jend = causal ? min(Lk, ii + 1) : Lk;
+    const int own = i % period + off;  // the row's own position among the keys
+    const int jend = causal ? min(Lk, own + 1) : Lk;
     for (int kt = 0; kt < n_kt; ++kt) {
       const int j0 = kt * kTile + 4 * lane;
       int ties = 0;
@@ -610,7 +617,7 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           const int j = j0 + c;
-          ties += (j < jend && !(diag && j == ii) && key_of(v[c]) == thr) ? 1 : 0;
+          ties += (j < jend && !(diag && j == own) && key_of(v[c]) == thr) ? 1 : 0;
         }
       }
 #pragma unroll
@@ -680,6 +687,7 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
   const bool vec = (Lk & 3) == 0;
   const int j0 = kt * kTile + 4 * lane;
   const float thr_f = sel.thr_f;
+  const int off = (causal || diag) ? Lk - Lq : 0;  // row i's own position is key i + off
   int count = 0;
   for (int r0 = warp; r0 < kTile; r0 += 16) {
     float v[4][4];
@@ -692,7 +700,7 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
       } else {
         v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
         if (i < Lq) {
-          const int jend = causal ? min(Lk, i + 1) : Lk;
+          const int jend = causal ? min(Lk, i + 1 + off) : Lk;
           if (j0 < jend) load4(acc + ((size_t)h * Lq + i) * Lk, j0, jend, vec, v[u]);
         }
       }
@@ -711,12 +719,12 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
             tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
           }
         } else {
-          const int jend = causal ? min(Lk, i + 1) : Lk;
+          const int jend = causal ? min(Lk, i + 1 + off) : Lk;
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const int j = j0 + c;
             if (j < jend) {
-              if (diag && j == i) {
+              if (diag && j == i + off) {
                 gt_bits |= 1u << c;
               } else {
                 gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
@@ -799,7 +807,9 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   const int h = tile / (n_kt * n_qt);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ int warp_count[4];
-  if (causal && kt > qt) {
+  // own positions of the tile's rows among the keys: columns own_lo .. own_hi
+  const int own_lo = qt * kTile + ((causal || diag) ? Lk - Lq : 0), own_hi = own_lo + kTile - 1;
+  if (causal && kt * kTile > own_hi) {
     // the whole tile lies above the diagonal: nothing is kept, nothing needs to be read
     const bool vec = (Lk & 3) == 0;
     const int j0 = kt * kTile + 4 * lane;
@@ -828,8 +838,9 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   sel.have_cut = st.have_cut != 0u;
   sel.tie_cut = st.tie_cut;
   sel.first_row = per_layer ? (uint32_t)h * (uint32_t)Lq : 0u;
-  const bool interior = (qt + 1) * kTile <= Lq && (kt + 1) * kTile <= Lk && (Lk & 3) == 0 && !(causal && kt >= qt) &&
-                        !(diag && kt == qt);
+  const bool below = !causal || kt * kTile + kTile - 1 <= own_lo;  // every column in every row's domain
+  const bool has_diag = diag && own_lo <= kt * kTile + kTile - 1 && own_hi >= kt * kTile;
+  const bool interior = (qt + 1) * kTile <= Lq && (kt + 1) * kTile <= Lk && (Lk & 3) == 0 && below && !has_diag;
   int count = interior ? emit_tile_rows<true>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel, tie_prefix, mask,
                                               stage_bitmap)
                        : emit_tile_rows<false>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel, tie_prefix, mask,
@@ -874,7 +885,7 @@ size_t select_scratch_bytes(int H, int Lq, int Lk) {
 
 cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   const int n_qt = ceil_div(a.Lq, kTile), n_kt = ceil_div(a.Lk, kTile);
-  const int diag = (a.keep_diag && a.Lq == a.Lk) ? 1 : 0;
+  const int diag = (a.keep_diag && (a.Lq == a.Lk || a.causal)) ? 1 : 0;
   Scratch sc = carve(a.scratch, a.H, a.Lq, a.Lk);
   // the selections: one per head over Lq rows, or one over the H*Lq rows of the layer
   const int n_sel = a.per_layer ? 1 : a.H;
@@ -893,7 +904,7 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   dim3 grid(row_blocks, n_sel);
   if (a.k_rest > 0) {
     // large selections: the one-pass shortcut first (those it resolves skip the three passes below)
-    const long long n_valid = a.causal ? (long long)a.Lq * (a.Lq + 1) / 2 : (long long)a.Lq * a.Lk;
+    const long long n_valid = domain_size(a.Lq, a.Lk, a.causal);
     const long long n_rest = (n_valid - (diag ? a.Lq : 0)) * (a.per_layer ? a.H : 1);
     const long long cap = cand_capacity(n_rest);
     if (cap > 0) {

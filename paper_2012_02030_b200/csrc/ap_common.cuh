@@ -29,6 +29,23 @@ void count_launches(int n);
 int64_t keep_count(int64_t n_valid, int64_t n_forced, double keep_frac);
 int64_t domain_size(int Lq, int Lk, int causal);
 
+// Tiles of the full domain in the list rows 0..qt-1 of a head.  Causal: row i sees the keys
+// j <= i + (Lk - Lq), so query tile q holds the key tiles 0 .. min(n_kt, q + 1 + c) - 1 with
+// c = ceil((Lk - Lq) / 128).
+__host__ __device__ inline int dense_row_tiles(int qt, int n_kt, int Lq, int Lk, int causal) {
+  if (!causal) return n_kt;
+  const int c = (Lk - Lq + kTile - 1) / kTile;
+  return qt + 1 + c < n_kt ? qt + 1 + c : n_kt;
+}
+__host__ __device__ inline int64_t dense_row_start(int qt, int n_kt, int Lq, int Lk, int causal) {
+  if (!causal) return (int64_t)qt * n_kt;
+  const int c = (Lk - Lq + kTile - 1) / kTile;
+  int a = n_kt - 1 - c;  // query tiles below this one hold fewer than n_kt key tiles
+  if (a < 0) a = 0;
+  if (a > qt) a = qt;
+  return (int64_t)a * (a + 1) / 2 + (int64_t)a * c + (int64_t)(qt - a) * n_kt;
+}
+
 // ---- launchers (each returns the cudaError_t of its launches) -------------------------------
 
 // Per-tile bitmaps + popcounts of an element mask into a dense staging area

@@ -170,9 +170,8 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
   const int kt = tile % n_kt;
   const int qt = (tile / n_kt) % n_qt;
   const int h = tile / (n_kt * n_qt);
-  // causal needs Lq == Lk, so n_qt == n_kt and the row of qt holds tiles 0..qt
-  const int per_head = causal ? n_qt * (n_qt + 1) / 2 : n_qt * n_kt;
-  const int row_start = h * per_head + (causal ? qt * (qt + 1) / 2 : qt * n_kt);
+  const int per_head = (int)dense_row_start(n_qt, n_kt, Lq, Lk, causal);
+  const int row_start = h * per_head + (int)dense_row_start(qt, n_kt, Lq, Lk, causal);
   if (threadIdx.x == 0 && kt == 0) {
     row_ptr[h * n_qt + qt] = min(row_start, cap);
     if (h == H - 1 && qt == n_qt - 1) {
@@ -180,14 +179,14 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
       if (H * per_head > cap) atomicOr(err, kDevErrCapacity);
     }
   }
-  if (causal && kt > qt) return;
+  if (kt >= dense_row_tiles(qt, n_kt, Lq, Lk, causal)) return;
   const int pos = row_start + kt;
   if (pos >= cap) return;
   const int r = threadIdx.x;
   const int i = qt * kTile + r;
   uint32_t w[4] = {0u, 0u, 0u, 0u};
   if (i < Lq) {
-    int jend = causal ? min(Lk, i + 1) : Lk;  // first column not kept
+    int jend = causal ? min(Lk, i + 1 + (Lk - Lq)) : Lk;  // first column not kept
     int n = jend - kt * kTile;                // kept columns of this tile row
     n = max(0, min(kTile, n));
 #pragma unroll

@@ -48,13 +48,13 @@ class Workload:
     @property
     def n_valid(self) -> int:
         """Entries of one head's domain."""
-        if self.causal:
-            return sum(min(i + 1, self.Lk) for i in range(self.Lq))
+        if self.causal:  # row i sees keys j <= i + (Lk - Lq): memory keys, then its own segment
+            return self.Lq * (self.Lq + 1) // 2 + self.Lq * (self.Lk - self.Lq)
         return self.Lq * self.Lk
 
     @property
     def n_forced(self) -> int:
-        return min(self.Lq, self.Lk) if (self.keep_diag and self.Lq == self.Lk) else 0
+        return self.Lq if (self.keep_diag and (self.Lq == self.Lk or self.causal)) else 0
 
     def scaled(self, **kw) -> "Workload":
         return dataclasses.replace(self, **kw)
@@ -71,6 +71,12 @@ WORKLOADS = {
     "s2s_self": Workload("s2s_self", 64, 8, 256, 256, 64, "bf16", True, 0.50, True, 64, "causal12", _seed(3)),
     "s2s_cross": Workload("s2s_cross", 64, 8, 256, 256, 64, "bf16", False, 0.50, False, 64, "cross12", _seed(3) + 500),
     "long": Workload("long", 4, 16, 4096, 4096, 128, "bf16", True, 0.05, True, 16, "causal64_sink16_stride256", _seed(4)),
+    # beyond the five prescribed configurations: a segment of 384 tokens attending to 384 cached
+    # positions of earlier segments plus itself (Transformer-XL's recurrence), and the long causal
+    # shape with the head count of the paper's Llama-2 experiment
+    "txl": Workload("txl", 16, 16, 384, 768, 64, "bf16", True, 0.10, True, 16, "mem32_sink8", _seed(5)),
+    "llama": Workload("llama", 1, 32, 4096, 4096, 128, "bf16", True, 0.05, True, 16, "causal64_sink16_stride256",
+                      _seed(6)),
 }
 
 
@@ -99,7 +105,7 @@ def calib_bias(w: Workload) -> torch.Tensor:
     """Additive bias on the scaled calibration logits, fp32 [H,Lq,Lk].
 
     Evaluated in fp64 and rounded once.  Under the causal constraint the
-    formulas are evaluated for j <= i only; the rest is 0 and never read.
+    formulas are evaluated inside the domain only; the rest is 0 and never read.
     """
     i = torch.arange(w.Lq, dtype=torch.float64).view(1, -1, 1)
     j = torch.arange(w.Lk, dtype=torch.float64).view(1, 1, -1)
@@ -125,10 +131,13 @@ def calib_bias(w: Workload) -> torch.Tensor:
     elif kind == "causal64_sink16_stride256":
         dist = (i - j).clamp(min=0.0)
         b = (3.0 * torch.exp(-dist / 64.0) + 2.0 * (j < 16) + 1.5 * (torch.remainder(j, 256) == 0))
+    elif kind == "mem32_sink8":
+        dist = (i + (w.Lk - w.Lq) - j).clamp(min=0.0)  # distance from the query's own position
+        b = (3.0 * torch.exp(-dist / 32.0) + 2.0 * (j < 8))
     else:
         raise ValueError(kind)
     if w.causal:
-        b = b * (j <= i)
+        b = b * (j <= i + (w.Lk - w.Lq))
     return b.to(torch.float32).expand(w.H, w.Lq, w.Lk).contiguous()
 
 
@@ -140,7 +149,7 @@ def random_mask(H: int, Lq: int, Lk: int, density: float, seed: int, causal: boo
     g.manual_seed(seed)
     m = (torch.rand((H, Lq, Lk), generator=g) < density)
     if causal:
-        m &= torch.tril(torch.ones((Lq, Lk), dtype=torch.bool))
+        m &= torch.tril(torch.ones((Lq, Lk), dtype=torch.bool), diagonal=Lk - Lq)
     for r in empty_rows:
         m[:, r, :] = False
     return m.to(torch.uint8).contiguous()

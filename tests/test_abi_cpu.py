@@ -79,7 +79,7 @@ def test_accumulate_and_mask_reject_bad_arguments():
     f = ap.lib.ap_accumulate_attention
     assert f(None, FAKE, FAKE, None, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, FAKE + 4, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG
-    assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 9, 64, 1, 1, 0.0, None) == ap.AP_ERR_INVALID_ARG  # causal, Lq != Lk
+    assert f(FAKE, FAKE, FAKE, None, 1, 1, 9, 8, 64, 1, 1, 0.0, None) == ap.AP_ERR_INVALID_ARG  # causal, Lk < Lq
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 32, 1, 0, 0.0, None) == ap.AP_ERR_UNSUPPORTED
     t = _tiles(H=1, Lq=8, Lk=8, cap=1)
     ws = ap.ap_build_mask_workspace_bytes(1, 8, 8)
@@ -93,7 +93,7 @@ def test_accumulate_and_mask_reject_bad_arguments():
         a[11] = ws - 1
         assert g(*a) == ap.AP_ERR_WORKSPACE
         a = list(base)
-        a[2], a[5] = 9, 1  # causal with Lq != Lk
+        a[2], a[5] = 9, 1  # causal with Lk < Lq
         assert g(*a) == ap.AP_ERR_INVALID_ARG
     # one selection over the layer ranks ties by a 32-bit index over all heads
     big = [FAKE, 64, 8192, 8192, 0.5, 0, 1, FAKE, None, FAKE, FAKE, ap.ap_build_mask_workspace_bytes(64, 8192, 8192),
@@ -105,7 +105,9 @@ def test_accumulate_and_mask_reject_bad_arguments():
     dt = ap.lib.ap_dense_tiles
     t4 = _tiles(H=1, Lq=256, Lk=256, cap=2)
     assert dt(1, 256, 256, 1, ctypes.byref(t4), None) == ap.AP_ERR_WORKSPACE  # needs 3 tiles
-    assert dt(1, 256, 128, 1, ctypes.byref(t4), None) == ap.AP_ERR_INVALID_ARG
+    assert dt(1, 256, 128, 1, ctypes.byref(t4), None) == ap.AP_ERR_INVALID_ARG  # causal with Lk < Lq
+    t5 = _tiles(H=1, Lq=256, Lk=300, cap=4)
+    assert dt(1, 256, 300, 1, ctypes.byref(t5), None) == ap.AP_ERR_WORKSPACE  # 44 memory keys: 2 + 3 tiles
 
 
 def test_no_cpu_fallback_without_a_device():

@@ -53,15 +53,13 @@ def test_mask_to_tiles_all_zero_and_capacity_overflow(ap):
 
 
 @pytest.mark.parametrize("causal", [False, True])
-@pytest.mark.parametrize("L", [(128, 128), (200, 200), (512, 512), (130, 300)])
+@pytest.mark.parametrize("L", [(128, 128), (200, 200), (512, 512), (130, 300), (384, 768), (256, 257), (300, 1000)])
 def test_dense_tiles_equal_tiles_of_the_full_domain(ap, L, causal):
     Lq, Lk = L
-    if causal and Lq != Lk:
-        pytest.skip("causal needs Lq == Lk")
     H = 2
     dom = torch.ones((H, Lq, Lk), dtype=torch.uint8)
-    if causal:
-        dom = torch.tril(dom)
+    if causal:  # with Lk > Lq: Lk - Lq memory keys before the causal segment
+        dom = torch.tril(dom, diagonal=Lk - Lq)
     tiles = ap.Tiles(H, Lq, Lk)
     ap.ap_dense_tiles(tiles, causal=causal)
     assert ap.ap_device_status() == ap.AP_OK
@@ -150,6 +148,36 @@ def test_build_mask_optional_outputs(ap):
     ap.ap_build_mask(acc_dev, 0.2, True, True, tiles=tiles)
     pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
     assert ap.ap_device_status() == ap.AP_OK
+
+
+@pytest.mark.parametrize("layer", [False, True])
+@pytest.mark.parametrize("keep_diag", [False, True])
+@pytest.mark.parametrize("shape", [(2, 100, 260), (3, 67, 200), (2, 384, 768), (2, 128, 129), (1, 5, 9)])
+def test_build_mask_causal_with_memory_keys(ap, shape, keep_diag, layer):
+    """Lk = mem + Lq: query i sees the keys j <= i + mem; its own position mem + i is the forced entry."""
+    H, Lq, Lk = shape
+    rng = np.random.default_rng(75)
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc[0].flat[::3] = 0.5
+    acc[-1] = np.round(acc[-1] * 8) / 8
+    for keep in (0.1, 0.5, 1.0):
+        want = _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=True, keep_diag=keep_diag,
+                                                            keep_frac=keep), layer=layer)
+        assert not want[:, ~np.tril(np.ones((Lq, Lk), dtype=bool), Lk - Lq)].any()
+        if keep_diag:
+            assert all(want[:, i, Lk - Lq + i].all() for i in range(Lq))
+
+
+@pytest.mark.parametrize("layer", [False, True])
+def test_build_mask_causal_with_memory_keys_large(ap, layer):
+    """Large enough for the sampled shortcut (more than 2^20 selectable entries per head)."""
+    H, Lq, Lk = 2, 1100, 1500
+    rng = np.random.default_rng(76)
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc[1] = np.round(acc[1] * 64) / 64
+    for keep, keep_diag in ((0.05, True), (0.4, False)):
+        _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=True, keep_diag=keep_diag,
+                                                     keep_frac=keep), layer=layer)
 
 
 # ------------------------------------------------------------- build mask, one threshold per layer
@@ -275,6 +303,11 @@ def _acc_tolerance(dtype):
     ("bert", dict(B=4, H=3), 2),
     ("lm", dict(B=2, H=2, Lq=300, Lk=300), 2),
     ("long", dict(B=1, H=2, Lq=640, Lk=640), 2),
+    # causal with memory keys (Lk = mem + Lq): tile-aligned, ragged, and on the CUDA-core path
+    ("txl", dict(B=2, H=2), 2),
+    ("txl", dict(B=2, H=2, Lq=200, Lk=333), 2),
+    ("long", dict(B=1, H=2, Lq=256, Lk=700), 1),
+    ("tiny", dict(Lq=77, Lk=130, causal=True), 2),
 ])
 def test_accumulate_matches_oracle(ap, name, over, n_batches):
     w = W[name].scaled(**over)
@@ -287,7 +320,7 @@ def test_accumulate_matches_oracle(ap, name, over, n_batches):
     tol = _acc_tolerance(w.dtype)
     np.testing.assert_allclose(got, want, rtol=tol["rtol"], atol=tol["atol"] * n_batches * w.B)
     if w.causal:
-        assert np.all(got[:, ~np.tril(np.ones((w.Lq, w.Lk), dtype=bool))] == 0.0)
+        assert np.all(got[:, ~np.tril(np.ones((w.Lq, w.Lk), dtype=bool), w.Lk - w.Lq)] == 0.0)
     np.testing.assert_allclose(got.sum(-1), n_batches * w.B, rtol=1e-5)
 
 
@@ -372,15 +405,16 @@ def test_forward_custom_scale(ap):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("causal", [False, True])
-def test_forward_dense_tiles_equal_unpruned_attention(ap, dtype, causal):
-    w = W["tiny"].scaled(B=2, H=2, Lq=300, Lk=300, dtype=dtype)
+@pytest.mark.parametrize("L", [(300, 300), (200, 456)])
+def test_forward_dense_tiles_equal_unpruned_attention(ap, dtype, causal, L):
+    w = W["tiny"].scaled(B=2, H=2, Lq=L[0], Lk=L[1], dtype=dtype)
     q, k, v = inputs.eval_qkv(w)
     tiles = ap.Tiles(w.H, w.Lq, w.Lk)
     ap.ap_dense_tiles(tiles, causal=causal)
     out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles)
     dom = torch.ones((w.H, w.Lq, w.Lk), dtype=torch.uint8)
     if causal:
-        dom = torch.tril(dom)
+        dom = torch.tril(dom, diagonal=w.Lk - w.Lq)
     ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), dom.numpy())
     pu.assert_close_attention(out, ref, dtype)
 
@@ -435,7 +469,7 @@ def test_workload_tiny_full(ap):
     _pipeline(ap, W["tiny"], W["tiny"].calib_batches)
 
 
-@pytest.mark.parametrize("name", ["bert", "lm", "s2s_self", "s2s_cross"])
+@pytest.mark.parametrize("name", ["bert", "lm", "s2s_self", "s2s_cross", "txl"])
 def test_workload_full_shape_short_calibration(ap, name):
     """Full evaluation shape; two calibration batches (the oracle's accumulate is the slow part)."""
     _pipeline(ap, W[name], 2)
@@ -446,10 +480,12 @@ def test_workload_long_reduced(ap):
     _pipeline(ap, W["long"].scaled(B=2, H=4, Lq=1024, Lk=1024), 2)
 
 
-def test_workload_long_full_size_sampled(ap):
-    """Full size (B4 H16 L4096 d128): accumulator rows, two heads' masks and sampled
-    output rows against the oracle; counts and bitmap popcounts for every head."""
-    w = W["long"]
+@pytest.mark.parametrize("name", ["long", "llama"])
+def test_workload_long_full_size_sampled(ap, name):
+    """Full size (long: B4 H16 L4096 d128; llama: the same context with B1 H32): accumulator rows,
+    two heads' masks and sampled output rows against the oracle; counts and bitmap popcounts for
+    every head."""
+    w = W[name]
     n_batches = 2
     bias = inputs.calib_bias(w)
     bias_dev = bias.cuda()

@@ -476,7 +476,7 @@ def test_mask_in_domain_zero_beats_nothing_outside_domain():
 
 def test_rounding_of_k_matches_the_workloads():
     want = {"tiny": 1638, "bert": 8192, "lm": 13133, "s2s_self": 16448, "s2s_cross": 32768,
-            "long": 419533}
+            "long": 419533, "txl": 22138, "llama": 419533}  # txl: 0.1 * (384*385/2 + 384*384) = 22137.6
     for name, w in inputs.WORKLOADS.items():
         assert orc.keep_count(w.n_valid, w.n_forced, w.keep_frac) == want[name]
         assert metrics.keep_count(w.n_valid, w.n_forced, w.keep_frac) == want[name]
