@@ -277,10 +277,13 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         tmem_ld32(tmem + 128 * buf + 64 * wg + 32 * c + lane_addr, x);
         tmem_wait_ld();
         float t[32];
+        if (interior) {  // the usual case: nothing to mask, no per-entry comparison
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          t[e] = fmaf(__uint_as_float(x[e]), scale_log2, bias2[32 * c + e]);
-          if (!interior && 32 * c + e >= n_valid) t[e] = -CUDART_INF_F;
+          for (int e = 0; e < 32; ++e) t[e] = fmaf(__uint_as_float(x[e]), scale_log2, bias2[32 * c + e]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            t[e] = 32 * c + e < n_valid ? fmaf(__uint_as_float(x[e]), scale_log2, bias2[32 * c + e]) : -CUDART_INF_F;
         }
         if (sweep == 0) {
           // four independent chains each for the maximum and for the sum
