@@ -334,6 +334,35 @@ def run_gpu(args, w):
     h2d = 3 * 0 + (hq.numel() + hk.numel() + hv.numel()) * elem
     d2h = ho.numel() * elem
 
+    # ---- the same step replayed from a CUDA graph (launch gaps of the ~25 kernels of a step removed) ----
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step(0)  # same stream as the capture: library state (function attributes) is set up
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(0)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        g0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        g1.record()
+        barrier()
+        graph_ms = g0.elapsed_time(g1) / args.steps
+        (graph_ms,) = replicas.max_over_ranks(info, [graph_ms], dev)
+        if ap.ap_device_status() != ap.AP_OK:
+            raise RuntimeError("device status not OK after the graph replays")
+    except RuntimeError as exc:  # capture refused: reported, not fatal
+        graph_ms = "unavailable: %s" % str(exc).splitlines()[0][:120]
+
     # ---- Eq. 2 with one threshold for the layer (outside the step: the workloads prescribe per head) ----
     tiles_layer = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
     nnz_layer = torch.zeros((w.H,), dtype=torch.int64, device=dev)
@@ -431,6 +460,8 @@ def run_gpu(args, w):
         "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer,
+        "graph_replay": {"ms_per_step": graph_ms, "note": "the same step (same calibration batch every replay) "
+                         "captured once in a CUDA graph; steps replays timed with one pair of events"},
     }
     print(json.dumps(line))
 
