@@ -56,7 +56,7 @@ typedef enum {
   AP_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up                     */
 } ap_status;
 
-typedef enum { AP_F32 = 0, AP_BF16 = 1 } ap_dtype;
+typedef enum { AP_F32 = 0, AP_BF16 = 1, AP_F16 = 2 } ap_dtype; /* AP_F16: IEEE half precision */
 
 /*
  * Tile list: the mask of Eq. 2 for H heads, cut into 128x128 tiles, with only
@@ -136,7 +136,7 @@ size_t ap_mask_to_tiles_workspace_bytes(int H, int Lq, int Lk);
  * the samples: the selection of Eq. 2 does not depend on it.
  *   acc    [H,Lq,Lk] fp32, in/out.  The sum over b is taken in ascending b with no
  *          floating-point atomics, so results are reproducible bit for bit.
- *   Q, K   [B,H,Lq,d], [B,H,Lk,d] of type dt
+ *   Q, K   [B,H,Lq,d], [B,H,Lk,d] of type dt (AP_BF16 and AP_F16 run on the tensor cores)
  *   bias   [H,Lq,Lk] fp32 added after scaling, or NULL
  *   scale  multiplier of Q.K^T; 0 selects 1/sqrt(d)
  */

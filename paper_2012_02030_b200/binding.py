@@ -15,7 +15,7 @@ import torch
 
 TILE = 128
 AP_OK, AP_ERR_INVALID_ARG, AP_ERR_UNSUPPORTED, AP_ERR_WORKSPACE, AP_ERR_CUDA, AP_ERR_TIMEOUT = range(6)
-AP_F32, AP_BF16 = 0, 1
+AP_F32, AP_BF16, AP_F16 = 0, 1, 2
 AP_STATIC_MAX_TILES = 1024
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libap_b200.so")
@@ -119,7 +119,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return AP_F32
     if t.dtype == torch.bfloat16:
         return AP_BF16
-    raise TypeError("dtype must be float32 or bfloat16, got %s" % t.dtype)
+    if t.dtype == torch.float16:
+        return AP_F16
+    raise TypeError("dtype must be float32, bfloat16 or float16, got %s" % t.dtype)
 
 
 def _check(status: int, where: str) -> None:

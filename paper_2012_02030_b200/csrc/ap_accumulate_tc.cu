@@ -1,4 +1,4 @@
-// Eq. 1 as a running sum for bf16 tensors, on the tcgen05 tensor cores.
+// Eq. 1 as a running sum for bf16 and fp16 tensors, on the tcgen05 tensor cores.
 //
 // One CTA owns one (head, 128-row query tile) and adds, for up to 32 samples b,
 // the normalised softmax rows to the accumulator.  A softmax row needs its
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_bias, int bias_by_tma, float *__restrict__ acc,
                      const float *__restrict__ bias, int b0, int Bc, int H, int Lq, int Lk,
-                     int n_qt, int n_kt, int causal, float scale_log2, unsigned *err) {
+                     int n_qt, int n_kt, int causal, int f16, float scale_log2, unsigned *err) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -177,7 +177,7 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_f32(128, 128, false, false);
+      const uint32_t idesc = idesc_bf16_f32(128, 128, false, false, f16 != 0);
       for (int v = 0; v < n_visits; ++v) {
         const int st = v % C::kStages;
         const uint32_t ph = (uint32_t)(v / C::kStages) & 1u;
@@ -360,7 +360,7 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
 template <int D>
 cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mb, int bias_by_tma, float *acc,
-                   const float *bias, int B, int H, int Lq, int Lk, int causal, float scale, unsigned *err,
+                   const float *bias, int B, int H, int Lq, int Lk, int causal, int f16, float scale, unsigned *err,
                    cudaStream_t s) {
   auto kern = accumulate_tc_kernel<D>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
@@ -370,7 +370,7 @@ cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorM
   for (int b0 = 0; b0 < B; b0 += kMaxB) {
     const int Bc = B - b0 < kMaxB ? B - b0 : kMaxB;
     kern<<<H * n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(mq, mk, mb, bias_by_tma, acc, bias, b0, Bc, H, Lq, Lk, n_qt,
-                                                       n_kt, causal, scale * kLog2e, err);
+                                                       n_kt, causal, f16, scale * kLog2e, err);
     count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -380,7 +380,7 @@ cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorM
 }  // namespace
 
 cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const float *bias, int B, int H, int Lq,
-                                 int Lk, int d, int causal, float scale, cudaStream_t s) {
+                                 int Lk, int d, int causal, int f16, float scale, cudaStream_t s) {
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   CUtensorMap mq, mk;
@@ -389,8 +389,8 @@ cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const
   CUtensorMap mb = mq;
   const int bias_by_tma = (bias && (Lk & 3) == 0) ? 1 : 0;
   if (bias_by_tma && !make_tile_map_f32(&mb, bias, H, Lq, Lk)) return cudaErrorUnknown;
-  return d == 64 ? launch<64>(mq, mk, mb, bias_by_tma, acc, bias, B, H, Lq, Lk, causal, scale, err, s)
-                 : launch<128>(mq, mk, mb, bias_by_tma, acc, bias, B, H, Lq, Lk, causal, scale, err, s);
+  return d == 64 ? launch<64>(mq, mk, mb, bias_by_tma, acc, bias, B, H, Lq, Lk, causal, f16, scale, err, s)
+                 : launch<128>(mq, mk, mb, bias_by_tma, acc, bias, B, H, Lq, Lk, causal, f16, scale, err, s);
 }
 
 }  // namespace ap

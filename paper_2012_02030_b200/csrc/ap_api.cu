@@ -129,13 +129,14 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
     return AP_ERR_INVALID_ARG;
   if (B < 1 || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq) || !(scale >= 0.f) || isinf(scale))
     return AP_ERR_INVALID_ARG;
-  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (dt == AP_BF16 && !device_error_word()) return AP_ERR_CUDA;
+  if (dt != AP_F32 && !device_error_word()) return AP_ERR_CUDA;
   cudaError_t e = dt == AP_F32 ? launch_accumulate_simt(acc, Q, K, bias, B, H, Lq, Lk, d, dt, causal ? 1 : 0, sc, s)
-                               : launch_accumulate_tc(acc, Q, K, bias, B, H, Lq, Lk, d, causal ? 1 : 0, sc, s);
+                               : launch_accumulate_tc(acc, Q, K, bias, B, H, Lq, Lk, d, causal ? 1 : 0,
+                                                      dt == AP_F16 ? 1 : 0, sc, s);
   if (e == cudaErrorInvalidValue) return AP_ERR_UNSUPPORTED;  // key length beyond the shared-memory budget
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
@@ -243,12 +244,12 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V, c
   if ((int64_t)B * H * ceil_div(Lq, kTile) > (int64_t)0x7fffffff) return AP_ERR_INVALID_ARG;
   ap_status st = check_tiles(tiles, H, Lq, Lk, true);
   if (st != AP_OK) return st;
-  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = dt == AP_F32 ? launch_fwd_simt(Q, K, V, *tiles, O, B, H, Lq, Lk, d, sc, s)
-                               : launch_fwd_tc(Q, K, V, *tiles, O, B, H, Lq, Lk, d, sc, s);
+                               : launch_fwd_tc(Q, K, V, *tiles, O, B, H, Lq, Lk, d, dt == AP_F16 ? 1 : 0, sc, s);
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
@@ -261,7 +262,7 @@ ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const voi
   if (B < 1 || !shape_ok(H, Lq, Lk) || !(scale >= 0.f) || isinf(scale)) return AP_ERR_INVALID_ARG;
   ap_status st = check_tiles(tiles, H, Lq, Lk, true);
   if (st != AP_OK) return st;
-  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16)) return AP_ERR_UNSUPPORTED;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t elem = dt == AP_F32 ? 4 : 2;

@@ -3,6 +3,7 @@
 
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -82,9 +83,10 @@ cudaError_t launch_accumulate_simt(float *acc, const void *Q, const void *K, con
 cudaError_t launch_fwd_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
                             int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
 cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
-                                 int Lq, int Lk, int d, int causal, float scale, cudaStream_t s);
+                                 int Lq, int Lk, int d, int causal, int f16, float scale, cudaStream_t s);
 
-// Tensor map of a [B*H, L, d] bf16 tensor for box_rows-row x 64-element swizzled boxes.
+// Tensor map of a [B*H, L, d] tensor of 16-bit elements (bf16 or fp16: the copy engine moves them
+// unchanged and fills out-of-range elements with zero bits) for box_rows-row x 64-element swizzled boxes.
 bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d, int box_rows = 128);
 bool make_split_map_bf16_d128(CUtensorMap *m, const void *base, int BH, int L, int box_rows);
 // Tensor map of an [H, Lq, Lk] fp32 tensor for 128-row x 32-column swizzled boxes (Lk % 4 == 0).
@@ -92,6 +94,6 @@ bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk);
 
 // bf16 tensors: tcgen05 tensor-core kernel
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
-                          int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
+                          int B, int H, int Lq, int Lk, int d, int f16, float scale, cudaStream_t s);
 
 }  // namespace ap

@@ -136,9 +136,30 @@ __device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int la
   return __shfl_sync(0xffffffffu, ok ? 1 : 0, kPollLane) != 0;
 }
 
-template <int D, bool kSplit>
+// Two fp32 values rounded to the tensors' 16-bit type and packed (first value in the low half),
+// and back: exactly the values the tensor cores will see.
+template <bool kF16>
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi) {
+  if constexpr (kF16) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+  } else {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+  }
+}
+template <bool kF16>
+__device__ __forceinline__ float2 unpack16x2(uint32_t pk) {
+  if constexpr (kF16) {
+    return __half22float2(*reinterpret_cast<const __half2 *>(&pk));
+  } else {
+    return make_float2(__uint_as_float(pk << 16), __uint_as_float(pk & 0xffff0000u));
+  }
+}
+
+template <int D, bool kSplit, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
-fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ O,
+fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
               const int32_t *__restrict__ round_ptr, const int32_t *__restrict__ round_rows,
               const uint8_t *__restrict__ round_info, const uint32_t *__restrict__ round_bitmap, int B, int H,
               int Lq, int n_qt, float scale_log2, unsigned *err) {
@@ -403,7 +424,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       tc_fence_after_sync();
       // N = 16 ng, D/16 steps of K = 16 (32 bytes inside the swizzled rows)
       if (elect_one()) {
-        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false);
+        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false, kF16);
         const uint32_t q_buf = q_addr + qb * C::kTileBytes, k_stage = k_addr + st * C::kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
@@ -420,7 +441,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
     }
   } else if (warp == 10) {
     // ------------------------------------------------------------ issuer of O += P V
-    constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
+    constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true, kF16);
     const uint32_t v_addr = smem_u32(v_s);
     bool ok = true;
     uint32_t n = 0;                          // non-empty items started so far
@@ -590,12 +611,12 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
           for (int e = 0; e < 16; ++e) {
             const float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
             const float p1 = ex2_approx(fmaf(__uint_as_float(x[2 * e + 1]), scale_log2, neg_mc));
-            __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<uint32_t *>(&hh);
-            // the row sum is taken over the bf16-rounded weights the MMA will use, so that
+            pk[e] = pack16x2<kF16>(p0, p1);
+            // the row sum is taken over the rounded weights the MMA will use, so that
             // O / l is an exact convex combination of V rows whatever the rounding of P
-            sum0 += __uint_as_float(pk[e] << 16);
-            sum1 += __uint_as_float(pk[e] & 0xffff0000u);
+            const float2 pr = unpack16x2<kF16>(pk[e]);
+            sum0 += pr.x;
+            sum1 += pr.y;
           }
         }
         tmem_st16(tmem_s + lane_addr + 32 * c, pk);
@@ -639,7 +660,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
       if (item < 0) break;
       const float2 g0 = sh->ml[n & 3u][0][r], g1 = sh->ml[n & 3u][1][r];
       const int i = (item % n_qt) * kTile + r;
-      __nv_bfloat16 *orow = O + ((size_t)(item / n_qt) * Lq + i) * D;
+      uint16_t *orow = O + ((size_t)(item / n_qt) * Lq + i) * D;
       const float m_tot = fmaxf(g0.x, g1.x);
       // weight of a partial result; 0 for a group that saw no kept entry of this row (m = -inf),
       // whose accumulator is then never read into the sum (it may hold a previous item's data)
@@ -673,8 +694,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, __nv_bfloat16 *__restrict__ 
               const float x0 = (f0 > 0.f ? __uint_as_float(o0[j]) * f0 : 0.f) + (f1 > 0.f ? __uint_as_float(o1[j]) * f1 : 0.f);
               const float x1 = (f0 > 0.f ? __uint_as_float(o0[j + 1]) * f0 : 0.f) +
                                (f1 > 0.f ? __uint_as_float(o1[j + 1]) * f1 : 0.f);
-              __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-              pk[e] = *reinterpret_cast<uint32_t *>(&hh);
+              pk[e] = pack16x2<kF16>(x0, x1);
             }
             *reinterpret_cast<uint4 *>(orow + 32 * c + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
@@ -699,14 +719,14 @@ int sm_count() {
   return cached[dev];
 }
 
-template <int D, bool kSplit>
+template <int D, bool kSplit, bool kF16>
 cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
                    unsigned *err, cudaStream_t s) {
   using C = Cfg<D, kSplit>;
   static_assert(sizeof(Shared) <= 17 * 1024, "shared bookkeeping outgrew its reservation");
   static_assert(C::kStages <= kMaxStages, "ring deeper than its barriers");
   static_assert(C::kSmemBytes > 114 * 1024 && C::kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
-  auto kern = fwd_tc_kernel<D, kSplit>;
+  auto kern = fwd_tc_kernel<D, kSplit, kF16>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
@@ -714,7 +734,7 @@ cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H
   const int n_units = B * H * ((t.n_qt + 1) / 2);  // pairs of query tiles, see the producer
   const float scale_log2 = scale * 1.4426950408889634f;
   kern<<<n_units < sms ? n_units : sms, kThreads, C::kSmemBytes, s>>>(
-      maps, static_cast<__nv_bfloat16 *>(O), t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, B, H, Lq,
+      maps, static_cast<uint16_t *>(O), t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, B, H, Lq,
       t.n_qt, scale_log2, err);
   count_launches(1);
   return cudaGetLastError();
@@ -723,7 +743,7 @@ cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H
 }  // namespace
 
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O, int B, int H,
-                          int Lq, int Lk, int d, float scale, cudaStream_t s) {
+                          int Lq, int Lk, int d, int f16, float scale, cudaStream_t s) {
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   // d = 128 with whole groups of eight key rows: both halves of a row come with one box
@@ -738,9 +758,14 @@ cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_
                      make_tile_map_bf16(&maps.v[i], V, B * H, Lk, d, rows);
   }
   if (!ok) return cudaErrorUnknown;
-  if (d == 64) return launch<64, false>(maps, O, t, B, H, Lq, scale, err, s);
-  return split ? launch<128, true>(maps, O, t, B, H, Lq, scale, err, s)
-               : launch<128, false>(maps, O, t, B, H, Lq, scale, err, s);
+  if (f16) {
+    if (d == 64) return launch<64, false, true>(maps, O, t, B, H, Lq, scale, err, s);
+    return split ? launch<128, true, true>(maps, O, t, B, H, Lq, scale, err, s)
+                 : launch<128, false, true>(maps, O, t, B, H, Lq, scale, err, s);
+  }
+  if (d == 64) return launch<64, false, false>(maps, O, t, B, H, Lq, scale, err, s);
+  return split ? launch<128, true, false>(maps, O, t, B, H, Lq, scale, err, s)
+               : launch<128, false, false>(maps, O, t, B, H, Lq, scale, err, s);
 }
 
 }  // namespace ap

@@ -228,11 +228,12 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t
   return d;
 }
 
-// Instruction descriptor of kind::f16 with bf16 operands and fp32 accumulation.
-__host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, bool a_mn_major, bool b_mn_major) {
+// Instruction descriptor of kind::f16 with bf16 (or, f16 = true, fp16) operands and fp32 accumulation.
+__host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, bool a_mn_major, bool b_mn_major,
+                                                      bool f16 = false) {
   return (1u << 4)                          // D format: F32
-         | (1u << 7)                        // A format: BF16
-         | (1u << 10)                       // B format: BF16
+         | ((f16 ? 0u : 1u) << 7)           // A format: F16 = 0, BF16 = 1
+         | ((f16 ? 0u : 1u) << 10)          // B format
          | ((a_mn_major ? 1u : 0u) << 15)   // A major-ness
          | ((b_mn_major ? 1u : 0u) << 16)   // B major-ness
          | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);

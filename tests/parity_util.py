@@ -7,7 +7,10 @@ from oracle import ap_oracle as orc
 from paper_2012_02030_b200 import inputs
 
 # tolerances of the attention output against the fp64 oracle
-TOL = {"bf16": dict(max_abs=1e-2, rel_l2=5e-3), "f32": dict(max_abs=1e-5, rel_l2=1e-6)}
+# bf16 and f32: the stated bounds.  f16 (11 significant bits against bf16's 8): the output's rounding
+# to half precision dominates, half an ulp is 2^-11 relative and 2^-10 absolute for |O| in [2, 4).
+TOL = {"bf16": dict(max_abs=1e-2, rel_l2=5e-3), "f32": dict(max_abs=1e-5, rel_l2=1e-6),
+       "f16": dict(max_abs=2e-3, rel_l2=1e-3)}
 
 
 def errors(got: np.ndarray, ref: np.ndarray):

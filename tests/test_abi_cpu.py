@@ -67,6 +67,8 @@ def test_forward_rejects_bad_arguments_before_any_device_work():
     assert call(a7=129) == ap.AP_ERR_INVALID_ARG             # tiles built for another Lq
     assert call(a9=96) == ap.AP_ERR_UNSUPPORTED              # d
     assert call(a10=7) == ap.AP_ERR_UNSUPPORTED              # dtype
+    assert call(a10=3) == ap.AP_ERR_UNSUPPORTED              # the code after AP_F16
+    assert (ap.AP_F32, ap.AP_BF16, ap.AP_F16) == (0, 1, 2)
     assert call(a11=-1.0) == ap.AP_ERR_INVALID_ARG           # scale
     assert call(a11=float("nan")) == ap.AP_ERR_INVALID_ARG
     t0 = _tiles(cap=0)

@@ -308,6 +308,9 @@ def _acc_tolerance(dtype):
     ("txl", dict(B=2, H=2, Lq=200, Lk=333), 2),
     ("long", dict(B=1, H=2, Lq=256, Lk=700), 1),
     ("tiny", dict(Lq=77, Lk=130, causal=True), 2),
+    # half precision (the precision of the paper's translation experiments)
+    ("s2s_cross", dict(B=3, H=2, dtype="f16"), 2),
+    ("long", dict(B=1, H=2, Lq=384, Lk=384, dtype="f16"), 1),
 ])
 def test_accumulate_matches_oracle(ap, name, over, n_batches):
     w = W[name].scaled(**over)
@@ -349,7 +352,7 @@ def _fwd_case(ap, w, mask: torch.Tensor, scale=0.0):
     return out, ref
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("d", [64, 128])
 @pytest.mark.parametrize("shape", [(2, 2, 128, 128), (1, 2, 200, 333), (2, 1, 513, 130), (1, 1, 5, 7)])
 def test_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
@@ -403,7 +406,7 @@ def test_forward_custom_scale(ap):
     _fwd_case(ap, w, inputs.random_mask(2, 150, 150, 0.3, seed=81), scale=0.31)
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("L", [(300, 300), (200, 456)])
 def test_forward_dense_tiles_equal_unpruned_attention(ap, dtype, causal, L):
@@ -473,6 +476,12 @@ def test_workload_tiny_full(ap):
 def test_workload_full_shape_short_calibration(ap, name):
     """Full evaluation shape; two calibration batches (the oracle's accumulate is the slow part)."""
     _pipeline(ap, W[name], 2)
+
+
+@pytest.mark.parametrize("name", ["s2s_self", "s2s_cross"])
+def test_workload_seq2seq_in_half_precision(ap, name):
+    """The translation experiments run in fp16: the same recipe with fp16 tensors, end to end."""
+    _pipeline(ap, W[name].scaled(B=8, dtype="f16"), 2)
 
 
 def test_workload_long_reduced(ap):
