@@ -162,6 +162,28 @@ int64_t oracle_keep_count(int64_t n_valid, int64_t n_forced, double keep_frac) {
 }
 
 /*
+ * Scores for the random-pruning control (the section that compares tailored masks
+ * with pruning random entries): score n, n = (h*Lq + i)*Lk + j, is the top 24 bits
+ * of the (n+1)-th output of the SplitMix64 generator seeded with `seed`, scaled to
+ * [0, 1).  Passed through Eq. 2's selection they give a random mask with exactly
+ * the count of a tailored one, inside the same domain and with the same forced
+ * entries.  The generator (Steele, Lea, Flood: "Fast splittable pseudorandom number
+ * generators", 2014) advances a 64-bit state by the odd constant below and scrambles
+ * it with two multiply-xorshift steps; output n+1 depends only on seed and n.
+ */
+void oracle_random_scores(float *out, int64_t count, uint64_t seed) {
+  uint64_t state = seed;
+  for (int64_t n = 0; n < count; ++n) {
+    state += 0x9E3779B97F4A7C15ull;
+    uint64_t z = state;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z = z ^ (z >> 31);
+    out[n] = (float)(z >> 40) * (1.0f / 16777216.0f);
+  }
+}
+
+/*
  * Eq. 2 as an exact per-head top-k: an entry is pruned (M_p = -inf) iff it does
  * not belong to the k largest entries of the head's average attention matrix.
  *   domain   all (i,j), or j <= i + (Lk - Lq) when causal

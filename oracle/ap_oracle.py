@@ -75,6 +75,16 @@ def _check_domain(Lq: int, Lk: int, causal: bool) -> None:
         raise ValueError("the causal domain needs Lk >= Lq")
 
 
+def random_scores(H: int, Lq: int, Lk: int, seed: int) -> np.ndarray:
+    """Scores of the random-pruning control: float32 [H,Lq,Lk] in [0,1), entry n = (h*Lq+i)*Lk+j from
+    the (n+1)-th SplitMix64 output for `seed` (top 24 bits)."""
+    out = np.zeros((H, Lq, Lk), dtype=np.float32)
+    lib = _load()
+    lib.oracle_random_scores.restype = None
+    lib.oracle_random_scores(_p(out), ctypes.c_int64(out.size), ctypes.c_uint64(seed & ((1 << 64) - 1)))
+    return out
+
+
 def accumulate(acc: np.ndarray, Q, K, bias=None, causal: bool = False, scale: float | None = None):
     """Eq. 1 as a running sum: acc[H,Lq,Lk] (float64, in place) += sum_b softmax(Q_b K_b^T*scale + bias)."""
     Q, K = _f32(Q), _f32(K)

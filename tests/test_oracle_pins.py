@@ -597,3 +597,40 @@ def test_mac_fraction_closed_form():
     assert metrics.attention_macs_fraction(768, 384, 0.9) == pytest.approx(3494.4 / 3840)
     assert metrics.effective_flops(10, 2, 64) == 4 * 64 * 10 * 2
     assert metrics.tile_flops(3, 2, 64) == 4 * 64 * 128 * 128 * 3 * 2
+
+
+# --------------------------------------------------------------- random-pruning control
+
+
+def test_random_scores_follow_the_published_generator_outputs():
+    """Score n is the top 24 bits of SplitMix64 output n + 1: checked against the generator's
+    published first outputs (tests/golden/splitmix64.txt)."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "splitmix64.txt")
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        seed, *outs = [int(t) for t in line.split()]
+        got = orc.random_scores(1, 1, len(outs), seed)[0, 0]
+        want = np.array([(z >> 40) / 16777216.0 for z in outs], dtype=np.float32)
+        np.testing.assert_array_equal(got, want)
+        # the value of entry n does not depend on the shape it is asked in
+        np.testing.assert_array_equal(orc.random_scores(len(outs), 1, 1, seed).ravel(), want)
+
+
+def test_random_scores_are_uniform_and_give_a_mask_of_the_exact_count():
+    H, L = 2, 256
+    u = orc.random_scores(H, L, L, seed=99)
+    assert u.min() >= 0.0 and u.max() < 1.0
+    assert abs(u.mean() - 0.5) < 4 * (1 / 12 / u.size) ** 0.5
+    assert abs(u.var() - 1 / 12) < 2e-3
+    hist = np.histogram(u, bins=64, range=(0, 1))[0]
+    expect = u.size / 64
+    assert ((hist - expect) ** 2 / expect).sum() < 64 + 5 * (2 * 64) ** 0.5      # chi-square, 63 d.o.f.
+    assert abs(np.corrcoef(u.ravel()[:-1], u.ravel()[1:])[0, 1]) < 0.01          # neighbours uncorrelated
+    assert not np.array_equal(u, orc.random_scores(H, L, L, seed=100))
+    # pruning random entries = Eq. 2's selection applied to the scores: same count as a tailored mask
+    mask, nnz = orc.build_mask(u, 0.2, causal=True, keep_diag=True)
+    k = orc.keep_count(L * (L + 1) // 2, L, 0.2)
+    assert nnz.tolist() == [k, k] and mask[:, np.arange(L), np.arange(L)].all()
+    rows = mask[0].sum(1) / (np.arange(L) + 1)                                    # kept share per row
+    assert abs(rows[64:].mean() - 0.2) < 0.02                                     # spread evenly over rows
