@@ -181,6 +181,16 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Scores for the random-pruning control (the paper's comparison of tailored masks with
+ * pruning random entries): scores[n], n = (h*Lq + i)*Lk + j, is the top 24 bits of the
+ * (n+1)-th output of the SplitMix64 generator seeded with `seed`, scaled to [0, 1).
+ * ap_build_mask[_layer] on these scores gives a random mask with exactly the count, the
+ * domain and the forced entries of a tailored mask of the same keep_frac.
+ *   scores  [H,Lq,Lk] fp32, written
+ */
+ap_status ap_random_scores(float *scores, int H, int Lq, int Lk, uint64_t seed, void *stream);
+
+/*
  * Tile list of an arbitrary element mask (uint8 [H,Lq,Lk], non-zero = kept):
  * the same encoding ap_build_mask emits, for masks made elsewhere (random
  * masks as in the paper's control experiment, all-ones, hand-made).

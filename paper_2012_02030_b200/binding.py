@@ -57,6 +57,7 @@ def _load() -> ctypes.CDLL:
         "ap_accumulate_attention": (i, [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp]),
         "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_build_mask_layer": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
+        "ap_random_scores": (i, [vp, i, i, i, ctypes.c_uint64, vp]),
         "ap_mask_to_tiles": (i, [vp, i, i, i, tp, vp, sz, vp]),
         "ap_dense_tiles": (i, [i, i, i, i, tp, vp]),
         "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
@@ -72,7 +73,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
-           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer",
+           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
            "ap_sparse_attention_fwd_host", "ap_device_status")
 
@@ -212,6 +213,15 @@ def ap_build_mask_layer(acc, keep_frac, causal=False, keep_diag=True, mask=None,
                         nnz_per_head=None, workspace=None, stream=None) -> None:
     _build_mask(lib.ap_build_mask_layer, "ap_build_mask_layer", acc, keep_frac, causal, keep_diag, mask, tiles,
                 nnz_per_head, workspace, stream)
+
+
+def ap_random_scores(scores, seed: int, stream=None) -> None:
+    _dev(scores, "scores")
+    H, Lq, Lk = scores.shape
+    if scores.dtype != torch.float32:
+        raise ValueError("scores must be float32")
+    _check(lib.ap_random_scores(_ptr(scores), H, Lq, Lk, int(seed) & ((1 << 64) - 1), _stream(stream)),
+           "ap_random_scores")
 
 
 def ap_mask_to_tiles(mask, tiles: Tiles, workspace=None, stream=None) -> None:

@@ -203,6 +203,14 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                          workspace_bytes, stream, 1);
 }
 
+ap_status ap_random_scores(float *scores, int H, int Lq, int Lk, uint64_t seed, void *stream) {
+  if (!scores || !aligned16(scores) || !shape_ok(H, Lq, Lk)) return AP_ERR_INVALID_ARG;
+  if (!have_device()) return AP_ERR_CUDA;
+  return launch_random_scores(scores, (int64_t)H * Lq * Lk, seed, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? AP_OK
+             : AP_ERR_CUDA;
+}
+
 ap_status ap_mask_to_tiles(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles *tiles, void *workspace,
                            size_t workspace_bytes, void *stream) {
   if (!mask || !shape_ok(H, Lq, Lk)) return AP_ERR_INVALID_ARG;

@@ -101,6 +101,10 @@ def test_accumulate_and_mask_reject_bad_arguments():
     big = [FAKE, 64, 8192, 8192, 0.5, 0, 1, FAKE, None, FAKE, FAKE, ap.ap_build_mask_workspace_bytes(64, 8192, 8192),
            None]
     assert ap.lib.ap_build_mask_layer(*big) == ap.AP_ERR_UNSUPPORTED
+    rs = ap.lib.ap_random_scores
+    assert rs(None, 1, 8, 8, 1, None) == ap.AP_ERR_INVALID_ARG
+    assert rs(FAKE + 4, 1, 8, 8, 1, None) == ap.AP_ERR_INVALID_ARG
+    assert rs(FAKE, 1, 0, 8, 1, None) == ap.AP_ERR_INVALID_ARG
     m = ap.lib.ap_mask_to_tiles
     assert m(None, 1, 8, 8, ctypes.byref(t), FAKE, 1 << 20, None) == ap.AP_ERR_INVALID_ARG
     assert m(FAKE, 1, 8, 8, ctypes.byref(t), FAKE, 16, None) == ap.AP_ERR_WORKSPACE

@@ -288,6 +288,21 @@ def test_build_mask_layer_full_size_long(ap):
         assert int(last_kept) < int(first_pruned)
 
 
+# ------------------------------------------------------------------- random-pruning control
+
+
+@pytest.mark.parametrize("shape", [(2, 128, 128), (3, 67, 201), (1, 1, 5), (2, 1024, 1024)])
+def test_random_scores_bit_exact_and_mask_of_exact_count(ap, shape):
+    H, Lq, Lk = shape
+    for seed in (0, 1234567, 2**63 + 5):
+        got = torch.full((H, Lq, Lk), -1.0, dtype=torch.float32, device="cuda")
+        ap.ap_random_scores(got, seed)
+        np.testing.assert_array_equal(got.cpu().numpy(), orc.random_scores(H, Lq, Lk, seed))
+    if Lq == Lk:  # pruning random entries: Eq. 2's selection on the scores
+        w = W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=True, keep_frac=0.2)
+        _check_build_mask(ap, got.cpu().numpy(), w)
+
+
 # ------------------------------------------------------------------------------ accumulate
 
 
