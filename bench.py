@@ -148,9 +148,10 @@ class ClockSampler:
 # --------------------------------------------------------------------------- CPU oracle legs
 
 
-def oracle_sample_step(w, units, calib_seqs=1):
-    """One pass of the path on the CPU oracle for a bounded sample: `units` heads of
-    batch element 0.  Returns per-stage seconds and the FLOPs (4*d*nnz) of the forward."""
+def oracle_sample_step(w, units, calib_seqs=1, batch=1):
+    """One pass of the path on the CPU oracle for a bounded sample: `units` heads, `calib_seqs`
+    calibration sequences, the forward on `batch` batch elements.  Returns per-stage seconds and
+    the FLOPs (4*d*nnz per batch element) of the forward."""
     from oracle import ap_oracle as orc
 
     heads = list(range(units))
@@ -164,11 +165,11 @@ def oracle_sample_step(w, units, calib_seqs=1):
     mask, nnz = orc.build_mask(acc64.astype(np.float32), w.keep_frac, w.causal, w.keep_diag)
     t2 = time.perf_counter()
     eq, ek, ev = inputs.eval_qkv(w)
-    eq, ek, ev = (inputs.widen(t[:1, heads]) for t in (eq, ek, ev))
+    eq, ek, ev = (inputs.widen(t[:batch, heads]) for t in (eq, ek, ev))
     t3 = time.perf_counter()
     orc.attention_fwd(eq, ek, ev, mask)
     t4 = time.perf_counter()
-    flops = 4.0 * w.d * float(nnz.sum())
+    flops = 4.0 * w.d * float(nnz.sum()) * batch
     return dict(acc_s=t1 - t0, mask_s=t2 - t1, fwd_s=t4 - t3, flops=flops, cores=min(orc.num_threads(), units))
 
 
@@ -334,7 +335,34 @@ def run_gpu(args, w):
     h2d = 3 * 0 + (hq.numel() + hk.numel() + hv.numel()) * elem
     d2h = ho.numel() * elem
 
+    # ---- Eq. 2 with one threshold for the layer (outside the step: the workloads prescribe per head) ----
+    tiles_layer = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    nnz_layer = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+    layer_ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    layer_ms = [0.0, 0.0]
+    n_layer = 5
+    for it in range(2 + n_layer):
+        layer_ev[0].record()
+        ap.ap_build_mask_layer(acc, w.keep_frac, w.causal, w.keep_diag, mask, tiles_layer, nnz_layer, ws)
+        layer_ev[1].record()
+        ap.ap_sparse_attention_fwd(q, k, v, tiles_layer, out)
+        layer_ev[2].record()
+        torch.cuda.synchronize()
+        if it >= 2:
+            layer_ms[0] += layer_ev[0].elapsed_time(layer_ev[1]) / n_layer
+            layer_ms[1] += layer_ev[1].elapsed_time(layer_ev[2]) / n_layer
+    if ap.ap_device_status() != ap.AP_OK:
+        raise RuntimeError("device status not OK after the layer-threshold runs")
+    k_layer = metrics.keep_count(w.n_valid * w.H, w.n_forced * w.H, w.keep_frac)
+    assert int(nnz_layer.sum().item()) == k_layer
+    layer = {"build_mask_layer_ms": layer_ms[0], "sparse_fwd_ms": layer_ms[1], "tiles_kept": tiles_layer.n_tiles(),
+             "nnz_per_head_min": int(nnz_layer.min().item()), "nnz_per_head_max": int(nnz_layer.max().item()),
+             "effective_tflops": metrics.effective_flops(k_layer, w.B, w.d) / (layer_ms[1] * 1e-3) / 1e12,
+             "note": "one threshold over all heads of the layer; %d runs after 2 warm-up runs, outside the step"
+                     % n_layer}
+
     # ---- the same step replayed from a CUDA graph (launch gaps of the ~25 kernels of a step removed) ----
+    # (last: the replays add one calibration batch over and over, which skews the accumulator)
     graph_ms = None
     try:
         side = torch.cuda.Stream(device=dev)
@@ -362,32 +390,6 @@ def run_gpu(args, w):
             raise RuntimeError("device status not OK after the graph replays")
     except RuntimeError as exc:  # capture refused: reported, not fatal
         graph_ms = "unavailable: %s" % str(exc).splitlines()[0][:120]
-
-    # ---- Eq. 2 with one threshold for the layer (outside the step: the workloads prescribe per head) ----
-    tiles_layer = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
-    nnz_layer = torch.zeros((w.H,), dtype=torch.int64, device=dev)
-    layer_ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-    layer_ms = [0.0, 0.0]
-    n_layer = 5
-    for it in range(2 + n_layer):
-        layer_ev[0].record()
-        ap.ap_build_mask_layer(acc, w.keep_frac, w.causal, w.keep_diag, mask, tiles_layer, nnz_layer, ws)
-        layer_ev[1].record()
-        ap.ap_sparse_attention_fwd(q, k, v, tiles_layer, out)
-        layer_ev[2].record()
-        torch.cuda.synchronize()
-        if it >= 2:
-            layer_ms[0] += layer_ev[0].elapsed_time(layer_ev[1]) / n_layer
-            layer_ms[1] += layer_ev[1].elapsed_time(layer_ev[2]) / n_layer
-    if ap.ap_device_status() != ap.AP_OK:
-        raise RuntimeError("device status not OK after the layer-threshold runs")
-    k_layer = metrics.keep_count(w.n_valid * w.H, w.n_forced * w.H, w.keep_frac)
-    assert int(nnz_layer.sum().item()) == k_layer
-    layer = {"build_mask_layer_ms": layer_ms[0], "sparse_fwd_ms": layer_ms[1], "tiles_kept": tiles_layer.n_tiles(),
-             "nnz_per_head_min": int(nnz_layer.min().item()), "nnz_per_head_max": int(nnz_layer.max().item()),
-             "effective_tflops": metrics.effective_flops(k_layer, w.B, w.d) / (layer_ms[1] * 1e-3) / 1e12,
-             "note": "one threshold over all heads of the layer; %d runs after 2 warm-up runs, outside the step"
-                     % n_layer}
 
     if rank != 0:
         return
@@ -433,11 +435,11 @@ def run_gpu(args, w):
     # ---- CPU baseline (bounded sample) -----------------------------------------------------
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        units = min(w.H, 8)
-        r = oracle_sample_step(w, units)
+        units, seqs = min(w.H, 16), min(w.B, 4)
+        r = oracle_sample_step(w, units, calib_seqs=seqs, batch=seqs)
         cpu = {"value": r["flops"] / r["fwd_s"] / 1e12, "unit": UNIT, "cores": r["cores"], "kind": "oracle",
-               "sample": "forward of heads 0..%d of batch element 0 (%d of %d (b,h) units), mask from one "
-                         "calibration sequence" % (units - 1, units, w.B * w.H),
+               "sample": "forward of heads 0..%d of batch elements 0..%d (%d of %d (b,h) units), mask from %d "
+                         "calibration sequences" % (units - 1, seqs - 1, units * seqs, w.B * w.H, seqs),
                "stage_seconds": {"accumulate": r["acc_s"], "build_mask": r["mask_s"], "sparse_fwd": r["fwd_s"]}}
 
     line = {
