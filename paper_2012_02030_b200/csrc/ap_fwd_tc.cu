@@ -119,7 +119,7 @@ __device__ __noinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volat
   for (uint32_t i = 0; i < kMaxPolls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (i > 64) __nanosleep(64);
+    if (i > 1024) __nanosleep(64);
   }
   *abort_flag = 1;
   atomicOr(err, kDevErrTimeout);
@@ -224,22 +224,23 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     // of this CTA is half t & 1 of unit blockIdx.x + (t >> 1) * gridDim.x.
     const int n_half = (n_qt + 1) / 2, n_units = B * H * n_half;
     struct ItemRef {
-      int bh, qt, rho0, n_rounds;  // n_rounds < 0: no such item (the unit's halves coincide)
-      bool in_range;
+      int bh, qt, rho0, rho1;  // rounds [rho0, rho1): loaded here, first read when the item begins
+      bool in_range, exists;   // !exists: no such item (the unit's halves coincide)
     };
     auto item_ref = [&](int t) {
       ItemRef it;
       const int u = (int)blockIdx.x + (t >> 1) * item_step;
       it.in_range = u < n_units;
-      it.bh = 0, it.qt = 0, it.rho0 = 0, it.n_rounds = -1;
+      it.bh = 0, it.qt = 0, it.rho0 = 0, it.rho1 = 0, it.exists = false;
       if (it.in_range) {
         const int j = u % n_half;
         it.bh = u / n_half;
         it.qt = (t & 1) ? j : n_qt - 1 - j;
         if (!(t & 1) || j != n_qt - 1 - j) {
           const int lr = (it.bh % H) * n_qt + it.qt;
-          it.rho0 = round_ptr[lr];
-          it.n_rounds = round_ptr[lr + 1] - it.rho0;
+          it.rho0 = (int)ldg_now_u32(round_ptr + lr);
+          it.rho1 = (int)ldg_now_u32(round_ptr + lr + 1);
+          it.exists = true;
         }
       }
       return it;
@@ -291,16 +292,19 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       load_run(v_s + pv_st * C::kTileBytes, maps.v, &sh->v_full[pv_st], pv_row, pv_run, pv_bh);
       pv_valid = false;
     };
-    // the rounds of an item are looked up one item ahead
+    // the rounds of an item are looked up two items ahead: the loads of item t + 2 are issued when
+    // item t begins and their results first touched when item t + 1 does
     ItemRef next = item_ref(0);
+    ItemRef next2 = item_ref(1);
     // ... and the slot rows and info byte of its first round while the current item is under way
     int pf_t = -1, pf_row = -1;
     uint32_t pf_info = 0u;
     for (int t = 0; next.in_range && ok; ++t) {
       const ItemRef cur = next;
-      next = item_ref(t + 1);
-      const int bh = cur.bh, qt = cur.qt, rho0 = cur.rho0, n_rounds = cur.n_rounds;
-      if (n_rounds < 0) continue;
+      next = next2;
+      next2 = item_ref(t + 2);
+      if (!cur.exists) continue;
+      const int bh = cur.bh, qt = cur.qt, rho0 = cur.rho0, n_rounds = cur.rho1 - cur.rho0;
       if (n_rounds == 0) {
         // nothing kept in this query tile: its output rows are zero (nobody else sees the item)
         const int rows = min(kTile, Lq - qt * kTile);
@@ -335,7 +339,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         if (v + 1 < n_rounds) {
           next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)(rho0 + v + 1) * 8 + lane) : -1;
           next_info = ldg_now_u8(round_info + rho0 + v + 1);
-        } else if (next.n_rounds > 0) {
+        } else if (next.exists && next.rho1 > next.rho0) {
           pf_t = t + 1;
           pf_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)next.rho0 * 8 + lane) : -1;
           pf_info = ldg_now_u8(round_info + next.rho0);
