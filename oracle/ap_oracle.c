@@ -162,6 +162,49 @@ int64_t oracle_keep_count(int64_t n_valid, int64_t n_forced, double keep_frac) {
 }
 
 /*
+ * Block-structured pruning (the hardware section applies the method with sparseness
+ * patterns "structured around blocks", block size 16, without saying how entries are
+ * grouped).  Reading: a block's score is the mean of the averaged attention over the
+ * block's entries inside the domain; Eq. 2's selection then runs over blocks
+ * (oracle_build_mask on the pooled array, which has the same causal structure at block
+ * level when Lq and Lk are multiples of the block size), and a kept block keeps all
+ * of its entries inside the domain.
+ *   pooled[h,I,J] = mean of acc[h,i,j] over I*bs <= i < (I+1)*bs, J*bs <= j < (J+1)*bs,
+ *                   (i,j) in the domain; 0 for blocks without such entries
+ * Needs Lq % bs == 0 and Lk % bs == 0.
+ */
+void oracle_pool_scores(const float *acc, int H, int Lq, int Lk, int bs, int causal, double *pooled) {
+  int nI = Lq / bs, nJ = Lk / bs;
+  for (int h = 0; h < H; ++h)
+    for (int I = 0; I < nI; ++I)
+      for (int J = 0; J < nJ; ++J) {
+        double sum = 0.0;
+        int64_t count = 0;
+        for (int i = I * bs; i < (I + 1) * bs; ++i) {
+          int jend = row_domain_end(i, Lq, Lk, causal);
+          for (int j = J * bs; j < (J + 1) * bs && j < jend; ++j) {
+            sum += (double)acc[((size_t)h * Lq + i) * Lk + j];
+            ++count;
+          }
+        }
+        pooled[((size_t)h * nI + I) * nJ + J] = count ? sum / (double)count : 0.0;
+      }
+}
+
+/* A kept block keeps its entries inside the domain: mask[h,i,j] = block_mask[h,i/bs,j/bs] there, else 0. */
+void oracle_expand_block_mask(const uint8_t *block_mask, int H, int Lq, int Lk, int bs, int causal,
+                              uint8_t *mask) {
+  int nI = Lq / bs, nJ = Lk / bs;
+  for (int h = 0; h < H; ++h)
+    for (int i = 0; i < Lq; ++i) {
+      int jend = row_domain_end(i, Lq, Lk, causal);
+      for (int j = 0; j < Lk; ++j)
+        mask[((size_t)h * Lq + i) * Lk + j] =
+            (j < jend && block_mask[((size_t)h * nI + i / bs) * nJ + j / bs]) ? 1 : 0;
+    }
+}
+
+/*
  * Scores for the random-pruning control (the section that compares tailored masks
  * with pruning random entries): score n, n = (h*Lq + i)*Lk + j, is the top 24 bits
  * of the (n+1)-th output of the SplitMix64 generator seeded with `seed`, scaled to

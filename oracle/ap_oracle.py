@@ -75,6 +75,34 @@ def _check_domain(Lq: int, Lk: int, causal: bool) -> None:
         raise ValueError("the causal domain needs Lk >= Lq")
 
 
+def pool_scores(acc32, block: int, causal: bool = False) -> np.ndarray:
+    """Block scores for block-structured pruning: float64 [H, Lq/block, Lk/block], the mean of acc over
+    each block's entries inside the domain (0 for blocks outside it)."""
+    acc32 = _f32(acc32)
+    H, Lq, Lk = acc32.shape
+    _check_domain(Lq, Lk, causal)
+    if block < 1 or Lq % block or Lk % block:
+        raise ValueError("Lq and Lk must be multiples of the block size")
+    out = np.zeros((H, Lq // block, Lk // block), dtype=np.float64)
+    lib = _load()
+    lib.oracle_pool_scores.restype = None
+    lib.oracle_pool_scores(_p(acc32), H, Lq, Lk, block, int(bool(causal)), _p(out))
+    return out
+
+
+def expand_block_mask(block_mask, block: int, causal: bool = False) -> np.ndarray:
+    """Element mask of a block mask: uint8 [H, R*block, C*block]; a kept block keeps its entries inside the domain."""
+    bm = np.ascontiguousarray(np.asarray(block_mask, dtype=np.uint8))
+    H, R, C = bm.shape
+    Lq, Lk = R * block, C * block
+    _check_domain(Lq, Lk, causal)
+    out = np.zeros((H, Lq, Lk), dtype=np.uint8)
+    lib = _load()
+    lib.oracle_expand_block_mask.restype = None
+    lib.oracle_expand_block_mask(_p(bm), H, Lq, Lk, block, int(bool(causal)), _p(out))
+    return out
+
+
 def random_scores(H: int, Lq: int, Lk: int, seed: int) -> np.ndarray:
     """Scores of the random-pruning control: float32 [H,Lq,Lk] in [0,1), entry n = (h*Lq+i)*Lk+j from
     the (n+1)-th SplitMix64 output for `seed` (top 24 bits)."""

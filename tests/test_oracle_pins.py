@@ -634,3 +634,48 @@ def test_random_scores_are_uniform_and_give_a_mask_of_the_exact_count():
     assert nnz.tolist() == [k, k] and mask[:, np.arange(L), np.arange(L)].all()
     rows = mask[0].sum(1) / (np.arange(L) + 1)                                    # kept share per row
     assert abs(rows[64:].mean() - 0.2) < 0.02                                     # spread evenly over rows
+
+
+# ------------------------------------------------------------- block-structured pruning
+
+
+@pytest.mark.parametrize("block", [4, 16])
+def test_pool_scores_equal_a_reshaped_mean_and_expansion_equals_a_kronecker_product(block):
+    """Away from the causal boundary the block mean is a reshape + mean, and the expansion of a
+    block mask is its Kronecker product with a block of ones (library routines)."""
+    rng = np.random.default_rng(60)
+    H, R, C = 2, 5, 7
+    acc = rng.random((H, R * block, C * block), dtype=np.float32)
+    got = orc.pool_scores(acc, block)
+    want = acc.astype(np.float64).reshape(H, R, block, C, block).mean(axis=(2, 4))
+    np.testing.assert_allclose(got, want, rtol=1e-14)
+    bm = (rng.random((H, R, C)) < 0.4).astype(np.uint8)
+    np.testing.assert_array_equal(orc.expand_block_mask(bm, block), np.kron(bm, np.ones((block, block), dtype=np.uint8)))
+
+
+@pytest.mark.parametrize("mem_blocks", [0, 2])
+def test_pool_scores_and_expansion_respect_the_causal_domain(mem_blocks):
+    rng = np.random.default_rng(61)
+    H, R, block = 2, 6, 8
+    Lq, Lk = R * block, (R + mem_blocks) * block
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    dom = np.tril(np.ones((Lq, Lk), dtype=bool), Lk - Lq)
+    got = orc.pool_scores(acc, block, causal=True)
+    a = np.where(dom, acc.astype(np.float64), 0.0).reshape(H, R, block, R + mem_blocks, block).sum(axis=(2, 4))
+    n = dom.reshape(R, block, R + mem_blocks, block).sum(axis=(1, 3))
+    np.testing.assert_allclose(got, np.where(n > 0, a / np.maximum(n, 1), 0.0), rtol=1e-14)
+    assert n[0, mem_blocks] == block * (block + 1) // 2          # a diagonal block holds a triangle
+    assert np.all(got[:, n == 0] == 0.0)
+    bm = np.ones((H, R, R + mem_blocks), dtype=np.uint8)
+    np.testing.assert_array_equal(orc.expand_block_mask(bm, block, causal=True), np.broadcast_to(dom, (H, Lq, Lk)))
+    # the whole route: pooled scores -> Eq. 2 over blocks -> element mask made of whole blocks
+    bmask, nnz = orc.build_mask(got.astype(np.float32), 0.5, causal=True, keep_diag=True)
+    mask = orc.expand_block_mask(bmask, block, causal=True)
+    n_blocks = R * (R + 1) // 2 + R * mem_blocks
+    assert nnz.tolist() == [orc.keep_count(n_blocks, R, 0.5)] * H
+    for h in range(H):
+        blocks = mask[h].reshape(R, block, R + mem_blocks, block).sum(axis=(1, 3))
+        assert np.all((blocks == 0) | (blocks == n))               # a block is kept whole or not at all
+        assert np.all(mask[h][np.arange(Lq), np.arange(Lq) + Lk - Lq] == 1)
+    with pytest.raises(ValueError):
+        orc.pool_scores(acc[:, :-1], block, causal=False)
