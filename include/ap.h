@@ -181,6 +181,24 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Block-structured pruning (the paper's hardware section uses sparseness patterns made of
+ * blocks of 16; how entries are grouped is not stated).  Three steps:
+ *   ap_pool_scores         pooled[h,I,J] = mean of acc over the entries of block (I,J) that lie
+ *                          inside the domain (0 if none), [H, Lq/block, Lk/block] fp32
+ *   ap_build_mask[_layer]  on the pooled array with the same causal / keep_diag arguments:
+ *                          Eq. 2 over blocks (the pooled array has the element domain's shape
+ *                          at block level)
+ *   ap_expand_block_mask   mask[h,i,j] = block_mask[h, i/block, j/block] inside the domain,
+ *                          0 outside; then ap_mask_to_tiles for the forward pass
+ * block is 16, 32, 64 or 128 and must divide Lq and Lk (AP_ERR_UNSUPPORTED otherwise).  With
+ * block = 128 every stored tile is fully kept, except where the causal boundary cuts it.
+ */
+ap_status ap_pool_scores(const float *acc, int H, int Lq, int Lk, int block, int causal, float *pooled,
+                         void *stream);
+ap_status ap_expand_block_mask(const uint8_t *block_mask, int H, int Lq, int Lk, int block, int causal,
+                               uint8_t *mask, void *stream);
+
+/*
  * Scores for the random-pruning control (the paper's comparison of tailored masks with
  * pruning random entries): scores[n], n = (h*Lq + i)*Lk + j, is the top 24 bits of the
  * (n+1)-th output of the SplitMix64 generator seeded with `seed`, scaled to [0, 1).

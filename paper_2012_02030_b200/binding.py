@@ -58,6 +58,8 @@ def _load() -> ctypes.CDLL:
         "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_build_mask_layer": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_random_scores": (i, [vp, i, i, i, ctypes.c_uint64, vp]),
+        "ap_pool_scores": (i, [vp, i, i, i, i, i, vp, vp]),
+        "ap_expand_block_mask": (i, [vp, i, i, i, i, i, vp, vp]),
         "ap_mask_to_tiles": (i, [vp, i, i, i, tp, vp, sz, vp]),
         "ap_dense_tiles": (i, [i, i, i, i, tp, vp]),
         "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
@@ -73,7 +75,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
-           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores",
+           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
            "ap_sparse_attention_fwd_host", "ap_device_status")
 
@@ -213,6 +215,31 @@ def ap_build_mask_layer(acc, keep_frac, causal=False, keep_diag=True, mask=None,
                         nnz_per_head=None, workspace=None, stream=None) -> None:
     _build_mask(lib.ap_build_mask_layer, "ap_build_mask_layer", acc, keep_frac, causal, keep_diag, mask, tiles,
                 nnz_per_head, workspace, stream)
+
+
+def ap_pool_scores(acc, block: int, causal=False, pooled=None, stream=None):
+    _dev(acc, "acc")
+    H, Lq, Lk = acc.shape
+    if acc.dtype != torch.float32:
+        raise ValueError("acc must be float32")
+    if pooled is None:
+        pooled = torch.empty((H, max(Lq // max(block, 1), 1), max(Lk // max(block, 1), 1)), dtype=torch.float32,
+                             device=acc.device)
+    _check(lib.ap_pool_scores(_ptr(acc), H, Lq, Lk, int(block), int(bool(causal)), _ptr(pooled), _stream(stream)),
+           "ap_pool_scores")
+    return pooled
+
+
+def ap_expand_block_mask(block_mask, block: int, causal=False, mask=None, stream=None):
+    _dev(block_mask, "block_mask")
+    H, R, C = block_mask.shape
+    if block_mask.dtype != torch.uint8:
+        raise ValueError("block_mask must be uint8")
+    if mask is None:
+        mask = torch.empty((H, R * block, C * block), dtype=torch.uint8, device=block_mask.device)
+    _check(lib.ap_expand_block_mask(_ptr(block_mask), H, R * block, C * block, int(block), int(bool(causal)),
+                                    _ptr(mask), _stream(stream)), "ap_expand_block_mask")
+    return mask
 
 
 def ap_random_scores(scores, seed: int, stream=None) -> None:

@@ -203,6 +203,36 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                          workspace_bytes, stream, 1);
 }
 
+namespace {
+bool block_ok(int Lq, int Lk, int block) {
+  return (block == 16 || block == 32 || block == 64 || block == 128) && Lq % block == 0 && Lk % block == 0;
+}
+}  // namespace
+
+ap_status ap_pool_scores(const float *acc, int H, int Lq, int Lk, int block, int causal, float *pooled,
+                         void *stream) {
+  if (!acc || !pooled || !aligned16(acc) || !aligned16(pooled) || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq))
+    return AP_ERR_INVALID_ARG;
+  if (!block_ok(Lq, Lk, block)) return AP_ERR_UNSUPPORTED;
+  if (!have_device()) return AP_ERR_CUDA;
+  return launch_pool_scores(acc, H, Lq, Lk, block, causal ? 1 : 0, pooled, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? AP_OK
+             : AP_ERR_CUDA;
+}
+
+ap_status ap_expand_block_mask(const uint8_t *block_mask, int H, int Lq, int Lk, int block, int causal,
+                               uint8_t *mask, void *stream) {
+  if (!block_mask || !mask || !aligned16(mask) || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq))
+    return AP_ERR_INVALID_ARG;
+  if (!block_ok(Lq, Lk, block)) return AP_ERR_UNSUPPORTED;
+  if (!have_device()) return AP_ERR_CUDA;
+  return launch_expand_block_mask(block_mask, H, Lq, Lk, block, causal ? 1 : 0, mask,
+                                  static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? AP_OK
+             : AP_ERR_CUDA;
+}
+
 ap_status ap_random_scores(float *scores, int H, int Lq, int Lk, uint64_t seed, void *stream) {
   if (!scores || !aligned16(scores) || !shape_ok(H, Lq, Lk)) return AP_ERR_INVALID_ARG;
   if (!have_device()) return AP_ERR_CUDA;

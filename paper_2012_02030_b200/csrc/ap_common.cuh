@@ -93,6 +93,10 @@ bool make_split_map_bf16_d128(CUtensorMap *m, const void *base, int BH, int L, i
 bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk);
 
 // bf16 tensors: tcgen05 tensor-core kernel
+cudaError_t launch_pool_scores(const float *acc, int H, int Lq, int Lk, int bs, int causal, float *pooled,
+                               cudaStream_t s);
+cudaError_t launch_expand_block_mask(const uint8_t *block_mask, int H, int Lq, int Lk, int bs, int causal,
+                                     uint8_t *mask, cudaStream_t s);
 cudaError_t launch_random_scores(float *out, int64_t count, uint64_t seed, cudaStream_t s);
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
                           int B, int H, int Lq, int Lk, int d, int f16, float scale, cudaStream_t s);

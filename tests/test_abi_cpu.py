@@ -101,6 +101,15 @@ def test_accumulate_and_mask_reject_bad_arguments():
     big = [FAKE, 64, 8192, 8192, 0.5, 0, 1, FAKE, None, FAKE, FAKE, ap.ap_build_mask_workspace_bytes(64, 8192, 8192),
            None]
     assert ap.lib.ap_build_mask_layer(*big) == ap.AP_ERR_UNSUPPORTED
+    ps, eb = ap.lib.ap_pool_scores, ap.lib.ap_expand_block_mask
+    assert ps(None, 1, 128, 128, 16, 0, FAKE, None) == ap.AP_ERR_INVALID_ARG
+    assert ps(FAKE, 1, 128, 128, 16, 0, None, None) == ap.AP_ERR_INVALID_ARG
+    assert ps(FAKE, 1, 128, 128, 24, 0, FAKE, None) == ap.AP_ERR_UNSUPPORTED   # block size
+    assert ps(FAKE, 1, 128, 136, 16, 0, FAKE, None) == ap.AP_ERR_UNSUPPORTED   # Lk not a multiple
+    assert ps(FAKE, 1, 256, 128, 16, 1, FAKE, None) == ap.AP_ERR_INVALID_ARG   # causal with Lk < Lq
+    assert eb(None, 1, 128, 128, 16, 0, FAKE, None) == ap.AP_ERR_INVALID_ARG
+    assert eb(FAKE, 1, 128, 128, 16, 0, FAKE + 4, None) == ap.AP_ERR_INVALID_ARG
+    assert eb(FAKE, 1, 120, 128, 16, 0, FAKE, None) == ap.AP_ERR_UNSUPPORTED
     rs = ap.lib.ap_random_scores
     assert rs(None, 1, 8, 8, 1, None) == ap.AP_ERR_INVALID_ARG
     assert rs(FAKE + 4, 1, 8, 8, 1, None) == ap.AP_ERR_INVALID_ARG

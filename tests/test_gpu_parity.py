@@ -288,6 +288,47 @@ def test_build_mask_layer_full_size_long(ap):
         assert int(last_kept) < int(first_pruned)
 
 
+# ------------------------------------------------------------------ block-structured pruning
+
+
+@pytest.mark.parametrize("causal,shape", [(False, (2, 256, 384)), (True, (2, 384, 384)), (True, (3, 256, 640)),
+                                          (False, (1, 128, 128)), (True, (2, 1024, 1024))])
+@pytest.mark.parametrize("block", [16, 32, 128])
+def test_block_structured_pruning(ap, shape, causal, block):
+    """Pooled block scores against the oracle (fp32 sums against fp64: relative 1e-5); Eq. 2 over the
+    blocks on the GPU's own pooled bits, the expansion and the tile list bit for bit; every block kept
+    whole or not at all; and the forward pass under the block mask."""
+    H, Lq, Lk = shape
+    rng = np.random.default_rng(77 + block)
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc[0] *= np.linspace(0.1, 2.0, Lk, dtype=np.float32)[None, :]
+    acc_dev = torch.from_numpy(acc).cuda()
+    pooled = ap.ap_pool_scores(acc_dev, block, causal)
+    np.testing.assert_allclose(pooled.cpu().numpy(), orc.pool_scores(acc, block, causal), rtol=1e-5, atol=1e-7)
+    R, C = Lq // block, Lk // block
+    bmask = torch.full((H, R, C), 7, dtype=torch.uint8, device="cuda")
+    keep_diag = Lq == Lk or causal
+    ap.ap_build_mask(pooled, 0.3, causal, keep_diag, mask=bmask)
+    want_b, _ = orc.build_mask(pooled.cpu().numpy(), 0.3, causal, keep_diag)
+    np.testing.assert_array_equal(bmask.cpu().numpy(), want_b)
+    mask = torch.full((H, Lq, Lk), 7, dtype=torch.uint8, device="cuda")
+    ap.ap_expand_block_mask(bmask, block, causal, mask=mask)
+    want = orc.expand_block_mask(want_b, block, causal)
+    np.testing.assert_array_equal(mask.cpu().numpy(), want)
+    tiles = ap.Tiles(H, Lq, Lk)
+    ap.ap_mask_to_tiles(mask, tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    host = tiles.to_host()
+    pu.assert_tiles_equal(host, orc.mask_to_tiles(want))
+    if block == 128 and not causal:
+        assert host["flags"].all()                       # every stored tile is fully kept
+    w = W["tiny"].scaled(B=2, H=H, Lq=Lq, Lk=Lk, d=64, dtype="bf16")
+    q, k, v = inputs.eval_qkv(w)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles)
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), want)
+    pu.assert_close_attention(out, ref, "bf16", "block mask")
+
+
 # ------------------------------------------------------------------- random-pruning control
 
 
