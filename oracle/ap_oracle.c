@@ -17,6 +17,8 @@
  *   oracle_attention_fwd   the masked attention equation of Section 3.2,
  *                          softmax((Q K^T + M_p)/sqrt(d_k)) V with M_p = -inf
  *                          on pruned entries.
+ *   oracle_attention_bwd   its derivative with respect to Q, K and V (what step 4 of
+ *                          the procedure, retraining under the mask, needs).
  *
  * Parity status: every function here is pinned by tests that do not go through
  * this file's own formulas (library SDPA, closed forms, brute force, invariants,
@@ -417,5 +419,76 @@ void oracle_attention_rows(const float *Q, const float *K, const float *V, const
     size_t bh = (size_t)b * H + h;
     attention_row(out + (size_t)r * d, Q + (bh * Lq + i) * d, K + bh * (size_t)Lk * d,
                   V + bh * (size_t)Lk * d, mask + ((size_t)h * Lq + i) * Lk, Lk, d, scale);
+  }
+}
+
+/*
+ * Derivative of the masked attention of Section 3.2 (step 4 of the procedure retrains the
+ * model under the mask, so gradients flow through exactly this function).  For one query
+ * row i with kept keys j:
+ *   s_j = scale * q_i.k_j,  p = softmax over the kept j,  o_i = sum_j p_j v_j
+ * and an incoming gradient g = dL/do_i:
+ *   dL/dv_j += p_j g
+ *   dL/dp_j  = g.v_j
+ *   dL/ds_j  = p_j (dL/dp_j - sum_k p_k dL/dp_k)          (softmax Jacobian)
+ *   dL/dq_i += scale * sum_j dL/ds_j k_j,   dL/dk_j += scale * dL/ds_j q_i
+ * Pruned entries have p = 0 and receive no gradient; a row without kept entries outputs 0
+ * and passes no gradient.  dQ[B,H,Lq,d], dK,dV[B,H,Lk,d] are overwritten.
+ */
+void oracle_attention_bwd(const float *Q, const float *K, const float *V, const float *dO,
+                          const uint8_t *mask, double *dQ, double *dK, double *dV, int B, int H,
+                          int Lq, int Lk, int d, double scale) {
+  memset(dQ, 0, sizeof(double) * (size_t)B * H * Lq * d);
+  memset(dK, 0, sizeof(double) * (size_t)B * H * Lk * d);
+  memset(dV, 0, sizeof(double) * (size_t)B * H * Lk * d);
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int bh = 0; bh < B * H; ++bh) {
+    int h = bh % H;
+    const float *Kh = K + (size_t)bh * Lk * d, *Vh = V + (size_t)bh * Lk * d;
+    double *dKh = dK + (size_t)bh * Lk * d, *dVh = dV + (size_t)bh * Lk * d;
+    double *p = (double *)malloc(sizeof(double) * (size_t)Lk);
+    double *dp = (double *)malloc(sizeof(double) * (size_t)Lk);
+    for (int i = 0; i < Lq; ++i) {
+      const float *q = Q + ((size_t)bh * Lq + i) * d, *g = dO + ((size_t)bh * Lq + i) * d;
+      const uint8_t *mrow = mask + ((size_t)h * Lq + i) * Lk;
+      double *dq = dQ + ((size_t)bh * Lq + i) * d;
+      double m = -INFINITY;
+      int kept = 0;
+      for (int j = 0; j < Lk; ++j) {
+        if (!mrow[j]) continue;
+        double dot = 0.0;
+        for (int t = 0; t < d; ++t) dot += (double)q[t] * (double)Kh[(size_t)j * d + t];
+        p[j] = dot * scale;
+        if (p[j] > m) m = p[j];
+        ++kept;
+      }
+      if (!kept) continue;
+      double z = 0.0;
+      for (int j = 0; j < Lk; ++j)
+        if (mrow[j]) {
+          p[j] = exp(p[j] - m);
+          z += p[j];
+        }
+      double pdp = 0.0;
+      for (int j = 0; j < Lk; ++j)
+        if (mrow[j]) {
+          p[j] /= z;
+          double a = 0.0;
+          for (int t = 0; t < d; ++t) a += (double)g[t] * (double)Vh[(size_t)j * d + t];
+          dp[j] = a;
+          pdp += p[j] * a;
+        }
+      for (int j = 0; j < Lk; ++j)
+        if (mrow[j]) {
+          double ds = p[j] * (dp[j] - pdp);
+          for (int t = 0; t < d; ++t) {
+            dVh[(size_t)j * d + t] += p[j] * (double)g[t];
+            dq[t] += scale * ds * (double)Kh[(size_t)j * d + t];
+            dKh[(size_t)j * d + t] += scale * ds * (double)q[t];
+          }
+        }
+    }
+    free(p);
+    free(dp);
   }
 }

@@ -216,6 +216,25 @@ def attention_fwd(Q, K, V, mask, scale: float | None = None) -> np.ndarray:
     return O
 
 
+def attention_bwd(Q, K, V, dO, mask, scale: float | None = None):
+    """Derivative of the masked attention of Section 3.2 in fp64: (dQ, dK, dV) for an incoming dO."""
+    Q, K, V, dO = _f32(Q), _f32(K), _f32(V), _f32(dO)
+    mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    assert K.shape == (B, H, Lk, d) and V.shape == (B, H, Lk, d) and dO.shape == Q.shape
+    assert mask.shape == (H, Lq, Lk)
+    dQ = np.zeros((B, H, Lq, d), dtype=np.float64)
+    dK = np.zeros((B, H, Lk, d), dtype=np.float64)
+    dV = np.zeros((B, H, Lk, d), dtype=np.float64)
+    s = 1.0 / np.sqrt(d) if scale is None else scale
+    lib = _load()
+    lib.oracle_attention_bwd.restype = None
+    lib.oracle_attention_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(mask), _p(dQ), _p(dK), _p(dV), B, H, Lq, Lk, d,
+                             ctypes.c_double(s))
+    return dQ, dK, dV
+
+
 def attention_rows(Q, K, V, mask, rows, scale: float | None = None) -> np.ndarray:
     """Masked attention for sampled (b, h, i) rows only; returns float64 [len(rows), d]."""
     Q, K, V = _f32(Q), _f32(K), _f32(V)

@@ -679,3 +679,71 @@ def test_pool_scores_and_expansion_respect_the_causal_domain(mem_blocks):
         assert np.all(mask[h][np.arange(Lq), np.arange(Lq) + Lk - Lq] == 1)
     with pytest.raises(ValueError):
         orc.pool_scores(acc[:, :-1], block, causal=False)
+
+
+# ------------------------------------------------------------------------------ backward
+
+
+@pytest.mark.parametrize("shape", [(2, 2, 37, 37, 16), (1, 2, 20, 45, 8)])
+def test_bwd_equals_library_autograd(shape):
+    """Gradients of a library softmax over an additive -inf mask, by reverse-mode differentiation
+    in fp64 (rows without kept entries are left out of the library graph: they output 0)."""
+    B, H, Lq, Lk, d = shape
+    q, k, v, g = (_rand(s, 70 + n) for n, s in enumerate(((B, H, Lq, d), (B, H, Lk, d), (B, H, Lk, d), (B, H, Lq, d))))
+    mask = inputs.random_mask(H, Lq, Lk, 0.3, seed=74, empty_rows=(3,))
+    qd, kd, vd = (t.double().requires_grad_(True) for t in (q, k, v))
+    s = torch.einsum("bhid,bhjd->bhij", qd, kd) * 0.31
+    s = s.masked_fill(mask.bool().unsqueeze(0) == 0, float("-inf"))
+    has = (mask.sum(-1) > 0)
+    p = torch.where(has.unsqueeze(0).unsqueeze(-1), torch.softmax(torch.where(has.unsqueeze(0).unsqueeze(-1), s, torch.zeros_like(s)), -1), torch.zeros_like(s))
+    p = p * mask.bool().unsqueeze(0)
+    out = p @ vd
+    (out * g.double()).sum().backward()
+    dq, dk, dv = orc.attention_bwd(q.numpy(), k.numpy(), v.numpy(), g.numpy(), mask.numpy(), scale=0.31)
+    np.testing.assert_allclose(out.detach().numpy(), orc.attention_fwd(q.numpy(), k.numpy(), v.numpy(), mask.numpy(), scale=0.31), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(dq, qd.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(dk, kd.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(dv, vd.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.all(dq[:, :, 3] == 0.0)                        # the row without kept entries passes no gradient
+
+
+def test_bwd_matches_central_differences_of_the_forward():
+    """Independent of any formula for the derivative: (L(x + e) - L(x - e)) / 2e of the oracle's own
+    forward (pinned above), for a few coordinates of Q, K and V."""
+    B, H, L, d = 1, 2, 9, 4
+    rng = np.random.default_rng(75)
+    q, k, v, g = (rng.standard_normal((B, H, L, d)).astype(np.float32) for _ in range(4))
+    mask = inputs.random_mask(H, L, L, 0.5, seed=76).numpy()
+    mask[:, :, 0] = 1
+    dq, dk, dv = orc.attention_bwd(q, k, v, g, mask)
+    loss = lambda a, b, c: float((orc.attention_fwd(a, b, c, mask) * g).sum())
+    eps = 2.0 ** -10                                          # exact in fp32 next to values of order 1
+    for arr, grad, which in ((q, dq, 0), (k, dk, 1), (v, dv, 2)):
+        for idx in ((0, 0, 2, 1), (0, 1, 7, 3), (0, 1, 0, 0)):
+            hi, lo = arr.copy(), arr.copy()
+            hi[idx] += eps
+            lo[idx] -= eps
+            args_hi = [q, k, v]; args_lo = [q, k, v]
+            args_hi[which], args_lo[which] = hi, lo
+            fd = (loss(*args_hi) - loss(*args_lo)) / (float(hi[idx]) - float(lo[idx]))
+            assert abs(fd - grad[idx]) <= 1e-5 * max(1.0, abs(fd)), (which, idx, fd, grad[idx])
+
+
+def test_bwd_closed_forms():
+    """One kept entry per row: p = 1, so dV is the scattered dO, and dQ = dK = 0.  Q = 0 with all
+    entries kept: uniform weights, dV_j = mean-weighted sum of dO."""
+    B, H, L, d = 1, 1, 6, 4
+    rng = np.random.default_rng(77)
+    q, k, v, g = (rng.standard_normal((B, H, L, d)).astype(np.float32) for _ in range(4))
+    cols = np.array([2, 0, 5, 5, 1, 3])
+    mask = np.zeros((H, L, L), dtype=np.uint8)
+    mask[0, np.arange(L), cols] = 1
+    dq, dk, dv = orc.attention_bwd(q, k, v, g, mask)
+    assert np.all(dq == 0.0) and np.all(dk == 0.0)
+    want = np.zeros((L, d))
+    for i, j in enumerate(cols):
+        want[j] += g[0, 0, i]
+    np.testing.assert_allclose(dv[0, 0], want, rtol=1e-15)
+    ones = np.ones((H, L, L), dtype=np.uint8)
+    dq, dk, dv = orc.attention_bwd(np.zeros_like(q), k, v, g, ones)
+    np.testing.assert_allclose(dv[0, 0], np.broadcast_to(g[0, 0].astype(np.float64).sum(0) / L, (L, d)), rtol=1e-13)
