@@ -181,6 +181,23 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Derivative of ap_sparse_attention_fwd with respect to Q, K and V (retraining under the
+ * mask, step 4 of the paper's procedure, differentiates exactly this function).  With
+ * S = scale*Q.K^T, P = softmax of S over the kept entries of a row, O = P.V and dO given:
+ *   dV = P^T.dO,  dP = dO.V^T,  dS = P o (dP - rowsum(dO o O)),  dQ = scale*dS.K,  dK = scale*dS^T.Q
+ * Pruned entries receive no gradient; a row without kept entries passes none.
+ *   Q, O, dO, dQ  [B,H,Lq,d];  K, V, dK, dV  [B,H,Lk,d], all of type dt (AP_BF16 or AP_F16;
+ *   AP_F32 is AP_ERR_UNSUPPORTED); O is the forward's output for the same inputs and tiles.
+ *   dQ, dK, dV are overwritten (every element written once: reproducible bit for bit).
+ *   workspace     ap_sparse_attention_bwd_workspace_bytes(B, H, Lq) bytes (row statistics)
+ */
+size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq);
+ap_status ap_sparse_attention_bwd(const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                                  const ap_tiles *tiles, void *dQ, void *dK, void *dV, int B, int H,
+                                  int Lq, int Lk, int d, ap_dtype dt, float scale, void *workspace,
+                                  size_t workspace_bytes, void *stream);
+
+/*
  * Block-structured pruning (the paper's hardware section uses sparseness patterns made of
  * blocks of 16; how entries are grouped is not stated).  Three steps:
  *   ap_pool_scores         pooled[h,I,J] = mean of acc over the entries of block (I,J) that lie

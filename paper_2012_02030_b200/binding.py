@@ -65,6 +65,8 @@ def _load() -> ctypes.CDLL:
         "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
         "ap_sparse_attention_fwd": (i, [vp, vp, vp, tp, vp, i, i, i, i, i, i, f, vp]),
         "ap_sparse_attention_fwd_host": (i, [vp, vp, vp, tp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, vp]),
+        "ap_sparse_attention_bwd_workspace_bytes": (sz, [i, i, i]),
+        "ap_sparse_attention_bwd": (i, [vp, vp, vp, vp, vp, tp, vp, vp, vp, i, i, i, i, i, i, f, vp, sz, vp]),
         "ap_device_status": (i, [vp]),
     }
     for name, (res, args) in sig.items():
@@ -77,7 +79,8 @@ lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
            "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
-           "ap_sparse_attention_fwd_host", "ap_device_status")
+           "ap_sparse_attention_fwd_host", "ap_sparse_attention_bwd_workspace_bytes", "ap_sparse_attention_bwd",
+           "ap_device_status")
 
 
 def status_string(status: int) -> str:
@@ -291,6 +294,31 @@ def ap_sparse_attention_fwd(Q, K, V, tiles: Tiles, O=None, scale=0.0, stream=Non
                                        B, H, Lq, Lk, d, _dtype_code(Q), float(scale), _stream(stream)),
            "ap_sparse_attention_fwd")
     return O
+
+
+def ap_sparse_attention_bwd_workspace_bytes(B: int, H: int, Lq: int) -> int:
+    return int(lib.ap_sparse_attention_bwd_workspace_bytes(B, H, Lq))
+
+
+def ap_sparse_attention_bwd(Q, K, V, O, dO, tiles: Tiles, dQ=None, dK=None, dV=None, scale=0.0, workspace=None,
+                            stream=None):
+    for t, name in ((Q, "Q"), (K, "K"), (V, "V"), (O, "O"), (dO, "dO")):
+        _dev(t, name)
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    if (K.shape != (B, H, Lk, d) or V.shape != K.shape or O.shape != Q.shape or dO.shape != Q.shape
+            or any(t.dtype != Q.dtype for t in (K, V, O, dO))):
+        raise ValueError("shape/dtype mismatch")
+    dQ = torch.empty_like(Q) if dQ is None else _dev(dQ, "dQ")
+    dK = torch.empty_like(K) if dK is None else _dev(dK, "dK")
+    dV = torch.empty_like(V) if dV is None else _dev(dV, "dV")
+    if workspace is None:
+        workspace = torch.empty(ap_sparse_attention_bwd_workspace_bytes(B, H, Lq), dtype=torch.uint8, device=Q.device)
+    _check(lib.ap_sparse_attention_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), ctypes.byref(tiles.c),
+                                       _ptr(dQ), _ptr(dK), _ptr(dV), B, H, Lq, Lk, d, _dtype_code(Q), float(scale),
+                                       _ptr(workspace), workspace.numel(), _stream(stream)),
+           "ap_sparse_attention_bwd")
+    return dQ, dK, dV
 
 
 def ap_sparse_attention_fwd_host(hQ, hK, hV, tiles: Tiles, hO, dQ, dK, dV, dO, scale=0.0, stream=None):

@@ -291,6 +291,32 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V, c
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
+size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq) {
+  if (B < 1 || H < 1 || Lq < 1) return 0;
+  return bwd_workspace_bytes(B, H, Lq);
+}
+
+ap_status ap_sparse_attention_bwd(const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                                  const ap_tiles *tiles, void *dQ, void *dK, void *dV, int B, int H, int Lq,
+                                  int Lk, int d, ap_dtype dt, float scale, void *workspace,
+                                  size_t workspace_bytes, void *stream) {
+  const void *ptrs[] = {Q, K, V, O, dO, dQ, dK, dV, workspace};
+  for (const void *p : ptrs)
+    if (!p || !aligned16(p)) return AP_ERR_INVALID_ARG;
+  if (B < 1 || !shape_ok(H, Lq, Lk) || !(scale >= 0.f) || isinf(scale)) return AP_ERR_INVALID_ARG;
+  if ((int64_t)B * H * ceil_div(Lq > Lk ? Lq : Lk, kTile) > (int64_t)0x7fffffff) return AP_ERR_INVALID_ARG;
+  ap_status st = check_tiles(tiles, H, Lq, Lk, true);
+  if (st != AP_OK) return st;
+  if ((d != 64 && d != 128) || (dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
+  if (workspace_bytes < bwd_workspace_bytes(B, H, Lq)) return AP_ERR_WORKSPACE;
+  if (!have_device()) return AP_ERR_CUDA;
+  const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
+  return launch_bwd_tc(Q, K, V, O, dO, *tiles, dQ, dK, dV, workspace, B, H, Lq, Lk, d, dt == AP_F16 ? 1 : 0, sc,
+                       static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? AP_OK
+             : AP_ERR_CUDA;
+}
+
 ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const void *hV, const ap_tiles *tiles,
                                        void *hO, void *dQ, void *dK, void *dV, void *dO, int B, int H, int Lq,
                                        int Lk, int d, ap_dtype dt, float scale, void *stream) {

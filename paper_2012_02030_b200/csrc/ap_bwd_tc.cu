@@ -1,0 +1,562 @@
+// Derivative of the masked attention of Section 3.2 (what retraining under the mask, step 4 of
+// the procedure, needs) for bf16 / fp16 tensors, on the tcgen05 tensor cores.
+//
+// With S = scale Q K^T, P = softmax of S over the kept entries of a row, O = P V and an incoming dO:
+//   dV = P^T dO,   dP = dO V^T,   dS = P o (dP - D),  D_i = dO_i . O_i,
+//   dQ = scale dS K,   dK = scale dS^T Q.
+// Two kernels follow the tile list, both tile by tile and without overlap between their steps (a
+// first, plain version: one CTA of 128 threads, thread r = row r of the tile; one thread issues the
+// copies and the MMAs, everybody waits on two mbarriers):
+//   rows kernel     one CTA per (b, h, query tile).  Sweep 1 over the row's tiles: S on the tensor
+//                   cores, running maximum and sum of the kept entries -> L_i = log2 sum_j 2^(c S_ij)
+//                   (c = log2 e), and D_i from dO and O; both go to the workspace.  Sweep 2: S and dP
+//                   on the tensor cores, dS by the threads (P = 2^(c S - L), rounded to the tensors'
+//                   16-bit type and written to shared memory in the operand layout), dQ += dS K on the
+//                   tensor cores (accumulator in TMEM).
+//   columns kernel  one CTA per (b, h, key tile), looping over the query tiles whose list row holds
+//                   that key tile: S, dP, then P and dS to shared memory, dV += P^T dO and
+//                   dK += dS^T Q on the tensor cores.
+// Every output element is written once, by the thread that owns its row: no atomics, results are
+// reproducible bit for bit.  All tiles are staged by TMA with the 128-byte swizzle, one layout
+// ([64-element slab][row][128 bytes]) serving as K-major and as MN-major operand; P and dS are
+// written by the threads in that same layout.  Every wait is bounded.
+#include <math_constants.h>
+
+#include "ap_common.cuh"
+#include "ap_sm100.cuh"
+
+namespace ap {
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kThreads = 128;
+constexpr int kSubBytes = 128 * 128;  // one slab: 128 rows x 64 elements of 2 bytes
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kMaxPolls = 1u << 22;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct Bars {
+  uint64_t tma, mma;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <bool kF16>
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  if constexpr (kF16) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+  } else {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+  }
+}
+template <bool kF16>
+__device__ __forceinline__ float2 unpack2(uint32_t pk) {
+  if constexpr (kF16) {
+    return __half22float2(*reinterpret_cast<const __half2 *>(&pk));
+  } else {
+    return make_float2(__uint_as_float(pk << 16), __uint_as_float(pk & 0xffff0000u));
+  }
+}
+
+// Bounded wait of the whole CTA on one barrier phase; the outcome is the same for every thread.
+__device__ __forceinline__ bool cta_wait(uint64_t *bar, uint32_t parity, Bars *bars, unsigned *err) {
+  bool ok = false;
+  volatile int *abort_flag = &bars->abort_flag;
+  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+    if (mbar_try_wait(bar, parity)) {
+      ok = true;
+      break;
+    }
+    if (*abort_flag) break;
+    if (i > 1024) __nanosleep(64);
+  }
+  if (!ok && !*abort_flag) {
+    *abort_flag = 1;
+    atomicOr(err, kDevErrTimeout);
+  }
+  return __syncthreads_and(ok ? 1 : 0) != 0;
+}
+
+// Address of 16-byte piece `piece` (0..7) of row r in slab `slab` of a staged tile.
+__device__ __forceinline__ unsigned char *piece_ptr(unsigned char *tile, int slab, int r, int piece) {
+  return tile + slab * kSubBytes + r * 128 + ((piece ^ (r & 7)) << 4);
+}
+
+// One thread: copies rows [row0, row0 + 128) of (batch, head) index bh into a staged tile of D columns.
+template <int D>
+__device__ __forceinline__ void load_tile(unsigned char *dst, const CUtensorMap *m, uint64_t *bar, int row0, int bh) {
+#pragma unroll
+  for (int s = 0; s < D / 64; ++s) tma_load_3d(dst + s * kSubBytes, m, bar, 64 * s, row0, bh);
+}
+
+// One thread: C[128 x 128] = A B^T with A and B staged tiles of D columns (rows x D, D contiguous).
+template <int D>
+__device__ __forceinline__ void mma_abt(uint32_t d_tmem, const unsigned char *a, const unsigned char *b, uint32_t idesc) {
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    const int sub = ks / 4, off = (ks % 4) * 32;
+    mma_ss(d_tmem, smem_desc_sw128(smem_u32(a + sub * kSubBytes + off), 16, 1024),
+           smem_desc_sw128(smem_u32(b + sub * kSubBytes + off), 16, 1024), idesc, ks > 0);
+  }
+}
+
+// One thread: C[128 x D] (+)= A^T B, A a staged 128 x 128 tile (rows = contraction index), B a staged
+// tile of D columns with the same rows.
+template <int D>
+__device__ __forceinline__ void mma_atb(uint32_t d_tmem, const unsigned char *a, const unsigned char *b, uint32_t idesc,
+                                        bool accumulate) {
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks)  // 16 rows of the contraction per step
+    mma_ss(d_tmem, smem_desc_sw128(smem_u32(a + ks * 2048), kSubBytes, 1024),
+           smem_desc_sw128(smem_u32(b + ks * 2048), kSubBytes, 1024), idesc, accumulate || ks > 0);
+}
+
+// One thread: C[128 x D] (+)= A B, A a staged 128 x 128 tile (columns = contraction index), B a staged
+// tile of D columns whose rows are the contraction index.
+template <int D>
+__device__ __forceinline__ void mma_ab(uint32_t d_tmem, const unsigned char *a, const unsigned char *b, uint32_t idesc,
+                                       bool accumulate) {
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const int sub = ks / 4, off = (ks % 4) * 32;
+    mma_ss(d_tmem, smem_desc_sw128(smem_u32(a + sub * kSubBytes + off), 16, 1024),
+           smem_desc_sw128(smem_u32(b + ks * 2048), kSubBytes, 1024), idesc, accumulate || ks > 0);
+  }
+}
+
+struct BwdMaps {
+  CUtensorMap q, k, v, o, d_o;
+};
+
+template <int D>
+struct Cfg {
+  static constexpr int kTileBytes = (D / 64) * kSubBytes;  // a staged tile of D columns
+  static constexpr int kSquareBytes = 2 * kSubBytes;       // a staged 128 x 128 tile (P, dS)
+  // rows kernel: Q, dO, K, V, dS (O is staged in the dS area first)
+  static constexpr int kRowsSmem = 4 * kTileBytes + kSquareBytes + 1024 + 256;
+  // columns kernel: K, V, Q, dO, P, dS
+  static constexpr int kColsSmem = 4 * kTileBytes + 2 * kSquareBytes + 1024 + 256;
+};
+
+// Thread r's 32 values of one chunk -> 16-bit pairs in row r of a staged 128 x 128 tile, columns [32c, 32c+32).
+__device__ __forceinline__ void store_chunk(unsigned char *tile, int r, int c, const uint32_t pk[16]) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    *reinterpret_cast<uint4 *>(piece_ptr(tile, c >> 1, r, (c & 1) * 4 + q)) =
+        make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+}
+
+// ------------------------------------------------------------------------------------------ rows kernel
+
+template <int D, bool kF16>
+__global__ void __launch_bounds__(kThreads, 1)
+bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ, float *__restrict__ stat_l,
+                float *__restrict__ stat_d, const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
+                const uint32_t *__restrict__ bitmap, int H, int Lq, int n_qt, float scale, unsigned *err) {
+  using C = Cfg<D>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char *smem =
+      reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char *q_s = smem, *do_s = smem + C::kTileBytes, *k_s = smem + 2 * C::kTileBytes,
+                *v_s = smem + 3 * C::kTileBytes, *ds_s = smem + 4 * C::kTileBytes;
+  Bars *bars = reinterpret_cast<Bars *>(smem + 4 * C::kTileBytes + C::kSquareBytes);
+
+  const int qt = blockIdx.x % n_qt, bh = blockIdx.x / n_qt, h = bh % H;
+  const int r = threadIdx.x, warp = r >> 5;
+  const int i = qt * kTile + r;
+  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  const int t0 = row_ptr[h * n_qt + qt], t1 = row_ptr[h * n_qt + qt + 1];
+  const float c = scale * kLog2e;
+
+  if (r == 0) {
+    mbar_init(&bars->tma, 1);
+    mbar_init(&bars->mma, 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&bars->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = bars->tmem_base;
+  const uint32_t tmem_s = tmem, tmem_dp = tmem + 128, tmem_dq = tmem + 256;
+  uint32_t tma_n = 0, mma_n = 0;  // phases used so far
+  bool ok = true;
+
+  // Q, dO and O of the query tile; D_i = dO_i . O_i
+  if (r == 0) {
+    mbar_arrive_expect_tx(&bars->tma, 3 * C::kTileBytes);
+    load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
+    load_tile<D>(do_s, &maps.d_o, &bars->tma, qt * kTile, bh);
+    load_tile<D>(ds_s, &maps.o, &bars->tma, qt * kTile, bh);
+  }
+  ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+  float dsum = 0.f;
+  if (ok) {
+#pragma unroll
+    for (int s = 0; s < D / 64; ++s)
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        const uint4 a = *reinterpret_cast<const uint4 *>(piece_ptr(do_s, s, r, p));
+        const uint4 b = *reinterpret_cast<const uint4 *>(piece_ptr(ds_s, s, r, p));
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 x = unpack2<kF16>(aw[e]), y = unpack2<kF16>(bw[e]);
+          dsum = fmaf(x.x, y.x, dsum);
+          dsum = fmaf(x.y, y.y, dsum);
+        }
+      }
+  }
+  __syncthreads();  // O is read: its area becomes dS
+
+  constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, false, false, kF16);
+  constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, false, true, kF16);
+
+  // ---- sweep 1: row maximum and sum over the kept entries
+  float m = -CUDART_INF_F, l = 0.f;
+  for (int t = t0; t < t1 && ok; ++t) {
+    if (r == 0) {
+      mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
+      load_tile<D>(k_s, &maps.k, &bars->tma, col_idx[t] * kTile, bh);
+    }
+    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+    if (!ok) break;
+    if (r == 0) {
+      tc_fence_after_sync();
+      mma_abt<D>(tmem_s, q_s, k_s, idesc_s);
+      mma_commit(&bars->mma);
+    }
+    const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
+    const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
+    if (!ok) break;
+    tc_fence_after_sync();
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ++ch) {
+      uint32_t x[32];
+      tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
+      tmem_wait_ld();
+      float cm = -CUDART_INF_F;
+#pragma unroll
+      for (int e = 0; e < 32; ++e)
+        if ((w[ch] >> e) & 1u) cm = fmaxf(cm, __uint_as_float(x[e]));
+      if (cm > m) {
+        l *= ex2_approx((m - cm) * c);  // 0 when m was -inf
+        m = cm;
+      }
+      if (m > -CUDART_INF_F) {
+        const float neg = -m * c;
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if ((w[ch] >> e) & 1u) l += ex2_approx(fmaf(__uint_as_float(x[e]), c, neg));
+      }
+    }
+    tc_fence_before_sync();
+    __syncthreads();  // S and K may be overwritten
+  }
+  // L_i = log2 of the row's sum of 2^(c S); +inf for a row without kept entries (then P = 0 everywhere)
+  const float big_l = l > 0.f ? fmaf(m, c, lg2_approx(l)) : CUDART_INF_F;
+  if (ok && i < Lq) {
+    stat_l[(size_t)bh * Lq + i] = big_l;
+    stat_d[(size_t)bh * Lq + i] = dsum;
+  }
+
+  // ---- sweep 2: dS and dQ
+  bool started = false;
+  for (int t = t0; t < t1 && ok; ++t) {
+    if (r == 0) {
+      mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+      load_tile<D>(k_s, &maps.k, &bars->tma, col_idx[t] * kTile, bh);
+      load_tile<D>(v_s, &maps.v, &bars->tma, col_idx[t] * kTile, bh);
+    }
+    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+    if (!ok) break;
+    if (r == 0) {
+      tc_fence_after_sync();
+      mma_abt<D>(tmem_s, q_s, k_s, idesc_s);
+      mma_abt<D>(tmem_dp, do_s, v_s, idesc_s);
+      mma_commit(&bars->mma);
+    }
+    const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
+    const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
+    if (!ok) break;
+    tc_fence_after_sync();
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ++ch) {
+      uint32_t x[32], y[32], pk[16];
+      tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
+      tmem_ld32(tmem_dp + lane_addr + 32 * ch, y);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        float ds[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int col = 2 * e + u;
+          const bool kept = (w[ch] >> col) & 1u;
+          const float p = kept ? ex2_approx(fmaf(__uint_as_float(x[col]), c, -big_l)) : 0.f;
+          ds[u] = p * (__uint_as_float(y[col]) - dsum);
+        }
+        pk[e] = pack2<kF16>(ds[0], ds[1]);
+      }
+      store_chunk(ds_s, r, ch, pk);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (r == 0) {
+      tc_fence_after_sync();
+      mma_ab<D>(tmem_dq, ds_s, k_s, idesc_dq, started);
+      mma_commit(&bars->mma);
+    }
+    started = true;
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);  // K, V, dS may be overwritten
+  }
+
+  // ---- dQ rows, scaled and rounded once (the loads are warp-wide: rows beyond Lq take part and store nothing)
+  if (ok) {
+    uint16_t *out = dQ + ((size_t)bh * Lq + i) * D;
+    tc_fence_after_sync();
+#pragma unroll 1
+    for (int ch = 0; ch < D / 32; ++ch) {
+      uint32_t x[32];
+      if (started) {  // the same for every thread
+        tmem_ld32(tmem_dq + lane_addr + 32 * ch, x);
+        tmem_wait_ld();
+      }
+      if (i < Lq) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            pk[e] = started ? pack2<kF16>(__uint_as_float(x[8 * q + 2 * e]) * scale,
+                                          __uint_as_float(x[8 * q + 2 * e + 1]) * scale)
+                            : 0u;
+          *reinterpret_cast<uint4 *>(out + 32 * ch + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// --------------------------------------------------------------------------------------- columns kernel
+
+template <int D, bool kF16>
+__global__ void __launch_bounds__(kThreads, 1)
+bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK, uint16_t *__restrict__ dV,
+                const float *__restrict__ stat_l, const float *__restrict__ stat_d,
+                const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
+                const uint32_t *__restrict__ bitmap, int H, int Lq, int Lk, int n_qt, int n_kt, float scale,
+                unsigned *err) {
+  using C = Cfg<D>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char *smem =
+      reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char *k_s = smem, *v_s = smem + C::kTileBytes, *q_s = smem + 2 * C::kTileBytes,
+                *do_s = smem + 3 * C::kTileBytes, *p_s = smem + 4 * C::kTileBytes,
+                *ds_s = smem + 4 * C::kTileBytes + C::kSquareBytes;
+  Bars *bars = reinterpret_cast<Bars *>(smem + 4 * C::kTileBytes + 2 * C::kSquareBytes);
+
+  const int kt = blockIdx.x % n_kt, bh = blockIdx.x / n_kt, h = bh % H;
+  const int r = threadIdx.x, warp = r >> 5;
+  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  const float c = scale * kLog2e;
+
+  if (r == 0) {
+    mbar_init(&bars->tma, 1);
+    mbar_init(&bars->mma, 1);
+    bars->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&bars->tmem_base, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = bars->tmem_base;
+  const uint32_t tmem_s = tmem, tmem_dp = tmem + 128, tmem_dv = tmem + 256, tmem_dk = tmem + 256 + D;
+  uint32_t tma_n = 0, mma_n = 0;
+  bool ok = true;
+
+  if (r == 0) {
+    mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+    load_tile<D>(k_s, &maps.k, &bars->tma, kt * kTile, bh);
+    load_tile<D>(v_s, &maps.v, &bars->tma, kt * kTile, bh);
+  }
+  ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+
+  constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, false, false, kF16);
+  constexpr uint32_t idesc_t = idesc_bf16_f32(128, D, true, true, kF16);
+
+  bool started = false;
+  for (int qt = 0; qt < n_qt && ok; ++qt) {
+    // the tile (qt, kt) in the list row of qt, if it is stored (key tiles ascend inside a row)
+    int lo = row_ptr[h * n_qt + qt], hi = row_ptr[h * n_qt + qt + 1];
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (col_idx[mid] < kt) lo = mid + 1; else hi = mid;
+    }
+    if (lo >= row_ptr[h * n_qt + qt + 1] || col_idx[lo] != kt) continue;
+    const int t = lo;
+    if (r == 0) {
+      mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+      load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
+      load_tile<D>(do_s, &maps.d_o, &bars->tma, qt * kTile, bh);
+    }
+    const int i = qt * kTile + r;
+    const float big_l = i < Lq ? stat_l[(size_t)bh * Lq + i] : CUDART_INF_F;
+    const float dsum = i < Lq ? stat_d[(size_t)bh * Lq + i] : 0.f;
+    const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
+    const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
+    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+    if (!ok) break;
+    if (r == 0) {
+      tc_fence_after_sync();
+      mma_abt<D>(tmem_s, q_s, k_s, idesc_s);
+      mma_abt<D>(tmem_dp, do_s, v_s, idesc_s);
+      mma_commit(&bars->mma);
+    }
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
+    if (!ok) break;
+    tc_fence_after_sync();
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ++ch) {
+      uint32_t x[32], y[32], pp[16], pd[16];
+      tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
+      tmem_ld32(tmem_dp + lane_addr + 32 * ch, y);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        float p[2], ds[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int col = 2 * e + u;
+          const bool kept = (w[ch] >> col) & 1u;
+          p[u] = kept ? ex2_approx(fmaf(__uint_as_float(x[col]), c, -big_l)) : 0.f;
+          ds[u] = p[u] * (__uint_as_float(y[col]) - dsum);
+        }
+        pp[e] = pack2<kF16>(p[0], p[1]);
+        pd[e] = pack2<kF16>(ds[0], ds[1]);
+      }
+      store_chunk(p_s, r, ch, pp);
+      store_chunk(ds_s, r, ch, pd);
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (r == 0) {
+      tc_fence_after_sync();
+      mma_atb<D>(tmem_dv, p_s, do_s, idesc_t, started);
+      mma_atb<D>(tmem_dk, ds_s, q_s, idesc_t, started);
+      mma_commit(&bars->mma);
+    }
+    started = true;
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);  // Q, dO, P, dS may be overwritten
+  }
+
+  // ---- dV and dK rows of this key tile (thread r = key row), rounded once
+  const int j = kt * kTile + r;
+  if (ok) {
+    tc_fence_after_sync();
+#pragma unroll 1
+    for (int which = 0; which < 2; ++which) {
+      uint16_t *out = (which ? dK : dV) + ((size_t)bh * Lk + j) * D;
+      const float f = which ? scale : 1.f;
+#pragma unroll 1
+      for (int ch = 0; ch < D / 32; ++ch) {
+        uint32_t x[32];
+        if (started) {  // the same for every thread; the loads are warp-wide
+          tmem_ld32((which ? tmem_dk : tmem_dv) + lane_addr + 32 * ch, x);
+          tmem_wait_ld();
+        }
+        if (j < Lk) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              pk[e] = started ? pack2<kF16>(__uint_as_float(x[8 * q + 2 * e]) * f,
+                                            __uint_as_float(x[8 * q + 2 * e + 1]) * f)
+                              : 0u;
+            *reinterpret_cast<uint4 *>(out + 32 * ch + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+template <int D, bool kF16>
+cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *stat_l, float *stat_d, const ap_tiles &t,
+                   int B, int H, int Lq, int Lk, float scale, unsigned *err, cudaStream_t s) {
+  using C = Cfg<D>;
+  auto rows = bwd_rows_kernel<D, kF16>;
+  auto cols = bwd_cols_kernel<D, kF16>;
+  cudaError_t e = cudaFuncSetAttribute(rows, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kRowsSmem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(cols, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kColsSmem);
+  if (e != cudaSuccess) return e;
+  rows<<<B * H * t.n_qt, kThreads, C::kRowsSmem, s>>>(maps, static_cast<uint16_t *>(dQ), stat_l, stat_d, t.row_ptr,
+                                                      t.col_idx, t.bitmap, H, Lq, t.n_qt, scale, err);
+  count_launches(1);
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  cols<<<B * H * t.n_kt, kThreads, C::kColsSmem, s>>>(maps, static_cast<uint16_t *>(dK), static_cast<uint16_t *>(dV),
+                                                      stat_l, stat_d, t.row_ptr, t.col_idx, t.bitmap, H, Lq, Lk,
+                                                      t.n_qt, t.n_kt, scale, err);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t bwd_workspace_bytes(int B, int H, int Lq) { return 2 * sizeof(float) * (size_t)B * H * Lq; }
+
+cudaError_t launch_bwd_tc(const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                          const ap_tiles &t, void *dQ, void *dK, void *dV, void *workspace, int B, int H, int Lq,
+                          int Lk, int d, int f16, float scale, cudaStream_t s) {
+  unsigned *err = device_error_word();
+  if (!err) return cudaErrorUnknown;
+  BwdMaps maps;
+  if (!make_tile_map_bf16(&maps.q, Q, B * H, Lq, d) || !make_tile_map_bf16(&maps.k, K, B * H, Lk, d) ||
+      !make_tile_map_bf16(&maps.v, V, B * H, Lk, d) || !make_tile_map_bf16(&maps.o, O, B * H, Lq, d) ||
+      !make_tile_map_bf16(&maps.d_o, dO, B * H, Lq, d))
+    return cudaErrorUnknown;
+  float *stat_l = static_cast<float *>(workspace);
+  float *stat_d = stat_l + (size_t)B * H * Lq;
+  if (d == 64)
+    return f16 ? launch<64, true>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s)
+               : launch<64, false>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s);
+  return f16 ? launch<128, true>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s)
+             : launch<128, false>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s);
+}
+
+}  // namespace ap

@@ -77,6 +77,26 @@ def test_forward_rejects_bad_arguments_before_any_device_work():
     assert call(a3=ctypes.byref(tn)) == ap.AP_ERR_INVALID_ARG
 
 
+def test_backward_rejects_bad_arguments():
+    f = ap.lib.ap_sparse_attention_bwd
+    t = _tiles()
+    ws = ap.ap_sparse_attention_bwd_workspace_bytes(1, 2, 128)
+    assert ws == 2 * 4 * 2 * 128 and ap.ap_sparse_attention_bwd_workspace_bytes(0, 1, 128) == 0
+    ok = [FAKE, FAKE, FAKE, FAKE, FAKE, ctypes.byref(t), FAKE, FAKE, FAKE, 1, 2, 128, 128, 64, 1, 0.0, FAKE, ws, None]
+    for idx in (0, 1, 2, 3, 4, 6, 7, 8, 16):
+        a = list(ok)
+        a[idx] = None
+        assert f(*a) == ap.AP_ERR_INVALID_ARG, idx
+    a = list(ok); a[14] = 0
+    assert f(*a) == ap.AP_ERR_UNSUPPORTED                      # fp32 tensors: no backward
+    a = list(ok); a[13] = 96
+    assert f(*a) == ap.AP_ERR_UNSUPPORTED
+    a = list(ok); a[17] = ws - 1
+    assert f(*a) == ap.AP_ERR_WORKSPACE
+    a = list(ok); a[11] = 129
+    assert f(*a) == ap.AP_ERR_INVALID_ARG                      # tiles built for another Lq
+
+
 def test_accumulate_and_mask_reject_bad_arguments():
     f = ap.lib.ap_accumulate_attention
     assert f(None, FAKE, FAKE, None, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG

@@ -488,6 +488,60 @@ def test_forward_single_kept_entry_copies_value_rows_exactly(ap):
     assert torch.equal(out.cpu(), v)
 
 
+# ------------------------------------------------------------------------------ backward
+
+
+def _rel_l2(got, ref):
+    return float(np.linalg.norm(got.astype(np.float64) - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def _bwd_case(ap, w, mask: torch.Tensor, tol):
+    """dQ, dK, dV of the masked attention against the oracle's derivative, for dO ~ N(0,1)."""
+    q, k, v = inputs.eval_qkv(w)
+    g = torch.Generator().manual_seed(w.seed0 + 77)
+    d_o = torch.randn(q.shape, generator=g).to(q.dtype)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles)
+    poison = [torch.full_like(t, float("nan"), device="cuda") for t in (q, k, v)]
+    dq, dk, dv = ap.ap_sparse_attention_bwd(q.cuda(), k.cuda(), v.cuda(), out, d_o.cuda(), tiles, *poison)
+    assert ap.ap_device_status() == ap.AP_OK
+    again = ap.ap_sparse_attention_bwd(q.cuda(), k.cuda(), v.cuda(), out, d_o.cuda(), tiles)
+    assert all(torch.equal(a, b) for a, b in zip((dq, dk, dv), again))      # no atomics: bit-reproducible
+    want = orc.attention_bwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), inputs.widen(d_o), mask.numpy())
+    for name, got, ref in zip(("dQ", "dK", "dV"), (dq, dk, dv), want):
+        got = got.float().cpu().numpy()
+        assert np.isfinite(got).all(), name
+        err = _rel_l2(got, ref)
+        assert err <= tol, (name, err)
+    return dq, dk, dv
+
+
+@pytest.mark.parametrize("dtype,tol", [("bf16", 1e-2), ("f16", 2e-3)])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("shape", [(2, 2, 128, 128), (1, 2, 200, 333), (2, 1, 513, 130), (1, 1, 5, 7)])
+def test_backward_random_masks_ragged_shapes(ap, shape, d, dtype, tol):
+    B, H, Lq, Lk = shape
+    w = W["tiny"].scaled(B=B, H=H, Lq=Lq, Lk=Lk, d=d, dtype=dtype)
+    mask = inputs.random_mask(H, Lq, Lk, 0.3, seed=95, empty_rows=(1,) if Lq > 1 else ())
+    dq, _, _ = _bwd_case(ap, w, mask, tol)
+    if Lq > 1:
+        assert torch.all(dq[:, :, 1] == 0)               # a row without kept entries passes no gradient
+
+
+def test_backward_causal_band_and_absent_tiles(ap):
+    """A causal band: most (query tile, key tile) pairs are not in the list; key tiles that no
+    query tile keeps get zero gradients."""
+    H, L = 2, 640
+    i = torch.arange(L)[:, None]
+    j = torch.arange(L)[None, :]
+    mask = ((j <= i) & (i - j < 100)).to(torch.uint8).expand(H, L, L).contiguous().clone()
+    mask[1, :, 512:] = 0                                 # head 1 never looks at the last key tile
+    w = W["tiny"].scaled(B=2, H=H, Lq=L, Lk=L, d=128, dtype="bf16")
+    _, dk, dv = _bwd_case(ap, w, mask, 1e-2)
+    assert torch.all(dk[:, 1, 512:] == 0) and torch.all(dv[:, 1, 512:] == 0)
+
+
 # ------------------------------------------------------------------- the five workloads
 
 
