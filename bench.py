@@ -361,6 +361,34 @@ def run_gpu(args, w):
              "note": "one threshold over all heads of the layer; %d runs after 2 warm-up runs, outside the step"
                      % n_layer}
 
+    # ---- derivative of the masked attention under the step's mask (outside the step) ----
+    backward = None
+    if w.dtype != "f32":
+        gen = torch.Generator(device="cpu")
+        gen.manual_seed(w.seed0 + 77)
+        d_out = torch.randn(q.shape, generator=gen).to(q.dtype).to(dev)
+        ap.ap_sparse_attention_fwd(q, k, v, tiles, out)
+        grads = ap.ap_sparse_attention_bwd(q, k, v, out, d_out, tiles)
+        bws = torch.empty(ap.ap_sparse_attention_bwd_workspace_bytes(w.B, w.H, w.Lq), dtype=torch.uint8, device=dev)
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_bwd = 5
+        torch.cuda.synchronize()
+        b0.record()
+        for _ in range(n_bwd):
+            ap.ap_sparse_attention_bwd(q, k, v, out, d_out, tiles, *grads, workspace=bws)
+        b1.record()
+        torch.cuda.synchronize()
+        if ap.ap_device_status() != ap.AP_OK:
+            raise RuntimeError("device status not OK after the backward runs")
+        bwd_ms = b0.elapsed_time(b1) / n_bwd
+        # executed: per stored tile and batch element eight 128 x 128 x d products (S twice, dP twice,
+        # S for the row statistics, dQ, dK, dV); effective: 10*d per kept entry (2.5 x the forward's 4*d)
+        bwd_tile_fl = 8 * 2.0 * 128 * 128 * w.d * tiles.n_tiles() * w.B
+        backward = {"ms": bwd_ms, "effective_tflops": 10.0 * w.d * float(nnz.sum().item()) * w.B / (bwd_ms * 1e-3) / 1e12,
+                    "executed_tile_tflops": bwd_tile_fl / (bwd_ms * 1e-3) / 1e12,
+                    "frac_of_bf16_sustained": bwd_tile_fl / (bwd_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
+                    "note": "ap_sparse_attention_bwd (rows kernel + columns kernel), %d runs outside the step" % n_bwd}
+
     # ---- the same step replayed from a CUDA graph (launch gaps of the ~25 kernels of a step removed) ----
     # (last: the replays add one calibration batch over and over, which skews the accumulator)
     graph_ms = None
@@ -461,7 +489,7 @@ def run_gpu(args, w):
         "roofline": roof, "roofline_by_stage": by_stage, "cpu_baseline": cpu,
         "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer,
+        "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer, "backward": backward,
         "graph_replay": {"ms_per_step": graph_ms, "note": "the same step (same calibration batch every replay) "
                          "captured once in a CUDA graph; steps replays timed with one pair of events"},
     }
