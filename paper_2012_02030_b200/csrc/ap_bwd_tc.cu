@@ -104,14 +104,21 @@ __device__ __forceinline__ void load_tile(unsigned char *dst, const CUtensorMap 
   for (int s = 0; s < D / 64; ++s) tma_load_3d(dst + s * kSubBytes, m, bar, 64 * s, row0, bh);
 }
 
-// One thread: C[128 x 128] = A B^T with A and B staged tiles of D columns (rows x D, D contiguous).
-template <int D>
-__device__ __forceinline__ void mma_abt(uint32_t d_tmem, const unsigned char *a, const unsigned char *b, uint32_t idesc) {
+// One thread: C[128 x 128] = A B^T with A and B staged tiles of D columns (rows x D, D contiguous),
+// restricted to the span of 16-column groups of C from the first to the last one named in `groups`
+// (bit g: columns [16g, 16g+16), i.e. rows [16g, 16g+16) of B); columns outside the span are left as they
+// are.  One product per step of the contraction: its cost hardly depends on the width, so the span is
+// not split further.
+template <int D, bool kF16>
+__device__ __forceinline__ void mma_abt_span(uint32_t d_tmem, const unsigned char *a, const unsigned char *b,
+                                             uint32_t groups) {
+  const int first = __ffs((int)groups) - 1, last = 31 - __clz((int)groups);
+  const uint32_t idesc = idesc_bf16_f32(128, 16 * (last - first + 1), false, false, kF16);
 #pragma unroll
   for (int ks = 0; ks < D / 16; ++ks) {
     const int sub = ks / 4, off = (ks % 4) * 32;
-    mma_ss(d_tmem, smem_desc_sw128(smem_u32(a + sub * kSubBytes + off), 16, 1024),
-           smem_desc_sw128(smem_u32(b + sub * kSubBytes + off), 16, 1024), idesc, ks > 0);
+    mma_ss(d_tmem + 16 * first, smem_desc_sw128(smem_u32(a + sub * kSubBytes + off), 16, 1024),
+           smem_desc_sw128(smem_u32(b + sub * kSubBytes + first * 2048 + off), 16, 1024), idesc, ks > 0);
   }
 }
 
@@ -128,14 +135,18 @@ __device__ __forceinline__ void mma_atb(uint32_t d_tmem, const unsigned char *a,
 
 // One thread: C[128 x D] (+)= A B, A a staged 128 x 128 tile (columns = contraction index), B a staged
 // tile of D columns whose rows are the contraction index.
+// Only the contraction steps named in `groups` are taken (bit g: columns [16g, 16g+16) of A).
 template <int D>
 __device__ __forceinline__ void mma_ab(uint32_t d_tmem, const unsigned char *a, const unsigned char *b, uint32_t idesc,
-                                       bool accumulate) {
+                                       bool accumulate, uint32_t groups) {
+  bool acc = accumulate;
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) {
+    if (!((groups >> ks) & 1u)) continue;
     const int sub = ks / 4, off = (ks % 4) * 32;
     mma_ss(d_tmem, smem_desc_sw128(smem_u32(a + sub * kSubBytes + off), 16, 1024),
-           smem_desc_sw128(smem_u32(b + ks * 2048), kSubBytes, 1024), idesc, accumulate || ks > 0);
+           smem_desc_sw128(smem_u32(b + ks * 2048), kSubBytes, 1024), idesc, acc);
+    acc = true;
   }
 }
 
@@ -147,8 +158,9 @@ template <int D>
 struct Cfg {
   static constexpr int kTileBytes = (D / 64) * kSubBytes;  // a staged tile of D columns
   static constexpr int kSquareBytes = 2 * kSubBytes;       // a staged 128 x 128 tile (P, dS)
-  // rows kernel: Q, dO, K, V, dS (O is staged in the dS area first)
-  static constexpr int kRowsSmem = 4 * kTileBytes + kSquareBytes + 1024 + 256;
+  // rows kernel: Q, dO, two (K, V) pairs (the next tile's pair is copied while this one is used), dS
+  // (O is staged in the dS area first)
+  static constexpr int kRowsSmem = 6 * kTileBytes + kSquareBytes + 1024 + 256;
   // columns kernel: K, V, Q, dO, P, dS
   static constexpr int kColsSmem = 4 * kTileBytes + 2 * kSquareBytes + 1024 + 256;
 };
@@ -167,16 +179,18 @@ template <int D, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ, float *__restrict__ stat_l,
                 float *__restrict__ stat_d, const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
+                const uint8_t *__restrict__ flags, const uint8_t *__restrict__ groups,
                 const uint32_t *__restrict__ bitmap, int H, int Lq, int n_qt, float scale, unsigned *err) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
       reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char *q_s = smem, *do_s = smem + C::kTileBytes, *k_s = smem + 2 * C::kTileBytes,
-                *v_s = smem + 3 * C::kTileBytes, *ds_s = smem + 4 * C::kTileBytes;
-  Bars *bars = reinterpret_cast<Bars *>(smem + 4 * C::kTileBytes + C::kSquareBytes);
+  unsigned char *q_s = smem, *do_s = smem + C::kTileBytes, *kv_s = smem + 2 * C::kTileBytes,
+                *ds_s = smem + 6 * C::kTileBytes;
+  Bars *bars = reinterpret_cast<Bars *>(smem + 6 * C::kTileBytes + C::kSquareBytes);
 
-  const int qt = blockIdx.x % n_qt, bh = blockIdx.x / n_qt, h = bh % H;
+  // late query tiles (the longest list rows under a causal mask) first
+  const int qt = n_qt - 1 - (int)(blockIdx.x / (gridDim.x / n_qt)), bh = blockIdx.x % (gridDim.x / n_qt), h = bh % H;
   const int r = threadIdx.x, warp = r >> 5;
   const int i = qt * kTile + r;
   const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
@@ -228,21 +242,26 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
   }
   __syncthreads();  // O is read: its area becomes dS
 
-  constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, false, false, kF16);
   constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, false, true, kF16);
 
   // ---- sweep 1: row maximum and sum over the kept entries
   float m = -CUDART_INF_F, l = 0.f;
+  if (r == 0 && ok && t0 < t1) {
+    mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
+    load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
+  }
   for (int t = t0; t < t1 && ok; ++t) {
-    if (r == 0) {
-      mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
-      load_tile<D>(k_s, &maps.k, &bars->tma, col_idx[t] * kTile, bh);
-    }
+    unsigned char *k_s = kv_s + ((t - t0) & 1) * 2 * C::kTileBytes;
+    const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];  // non-empty 16-column groups of the tile
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
     if (r == 0) {
+      if (t + 1 < t1) {  // the other pair was last read by the MMA of tile t - 1, which has completed
+        mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
+        load_tile<D>(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, &maps.k, &bars->tma, col_idx[t + 1] * kTile, bh);
+      }
       tc_fence_after_sync();
-      mma_abt<D>(tmem_s, q_s, k_s, idesc_s);
+      mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
       mma_commit(&bars->mma);
     }
     const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
@@ -252,6 +271,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     tc_fence_after_sync();
 #pragma unroll 1
     for (int ch = 0; ch < 4; ++ch) {
+      if (!((gm >> (2 * ch)) & 3u)) continue;  // nothing kept in these 32 columns (the same for every thread)
       uint32_t x[32];
       tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
       tmem_wait_ld();
@@ -282,18 +302,26 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
 
   // ---- sweep 2: dS and dQ
   bool started = false;
+  if (r == 0 && ok && t0 < t1) {
+    mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+    load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
+    load_tile<D>(kv_s + C::kTileBytes, &maps.v, &bars->tma, col_idx[t0] * kTile, bh);
+  }
   for (int t = t0; t < t1 && ok; ++t) {
-    if (r == 0) {
-      mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
-      load_tile<D>(k_s, &maps.k, &bars->tma, col_idx[t] * kTile, bh);
-      load_tile<D>(v_s, &maps.v, &bars->tma, col_idx[t] * kTile, bh);
-    }
+    unsigned char *k_s = kv_s + ((t - t0) & 1) * 2 * C::kTileBytes, *v_s = k_s + C::kTileBytes;
+    const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
     if (r == 0) {
+      if (t + 1 < t1) {  // the other pair was last read by dQ += dS K of tile t - 1, which has completed
+        unsigned char *nk = kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes;
+        mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+        load_tile<D>(nk, &maps.k, &bars->tma, col_idx[t + 1] * kTile, bh);
+        load_tile<D>(nk + C::kTileBytes, &maps.v, &bars->tma, col_idx[t + 1] * kTile, bh);
+      }
       tc_fence_after_sync();
-      mma_abt<D>(tmem_s, q_s, k_s, idesc_s);
-      mma_abt<D>(tmem_dp, do_s, v_s, idesc_s);
+      mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
+      mma_abt_span<D, kF16>(tmem_dp, do_s, v_s, gm);
       mma_commit(&bars->mma);
     }
     const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
@@ -303,6 +331,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     tc_fence_after_sync();
 #pragma unroll 1
     for (int ch = 0; ch < 4; ++ch) {
+      if (!((gm >> (2 * ch)) & 3u)) continue;  // dS of these columns is not read: their steps of dQ += dS K are skipped
       uint32_t x[32], y[32], pk[16];
       tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
       tmem_ld32(tmem_dp + lane_addr + 32 * ch, y);
@@ -314,8 +343,8 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
         for (int u = 0; u < 2; ++u) {
           const int col = 2 * e + u;
           const bool kept = (w[ch] >> col) & 1u;
-          const float p = kept ? ex2_approx(fmaf(__uint_as_float(x[col]), c, -big_l)) : 0.f;
-          ds[u] = p * (__uint_as_float(y[col]) - dsum);
+          // columns of an empty group hold whatever an earlier tile left in S and dP: never used
+          ds[u] = kept ? ex2_approx(fmaf(__uint_as_float(x[col]), c, -big_l)) * (__uint_as_float(y[col]) - dsum) : 0.f;
         }
         pk[e] = pack2<kF16>(ds[0], ds[1]);
       }
@@ -326,7 +355,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     __syncthreads();
     if (r == 0) {
       tc_fence_after_sync();
-      mma_ab<D>(tmem_dq, ds_s, k_s, idesc_dq, started);
+      mma_ab<D>(tmem_dq, ds_s, k_s, idesc_dq, started, gm);
       mma_commit(&bars->mma);
     }
     started = true;
@@ -370,6 +399,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK, uint16_t *__restrict__ dV,
                 const float *__restrict__ stat_l, const float *__restrict__ stat_d,
                 const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
+                const uint8_t *__restrict__ flags, const uint8_t *__restrict__ groups,
                 const uint32_t *__restrict__ bitmap, int H, int Lq, int Lk, int n_qt, int n_kt, float scale,
                 unsigned *err) {
   using C = Cfg<D>;
@@ -411,7 +441,6 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
   }
   ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
 
-  constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, false, false, kF16);
   constexpr uint32_t idesc_t = idesc_bf16_f32(128, D, true, true, kF16);
 
   bool started = false;
@@ -424,6 +453,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     }
     if (lo >= row_ptr[h * n_qt + qt + 1] || col_idx[lo] != kt) continue;
     const int t = lo;
+    const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
     if (r == 0) {
       mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
       load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
@@ -438,8 +468,8 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     if (!ok) break;
     if (r == 0) {
       tc_fence_after_sync();
-      mma_abt<D>(tmem_s, q_s, k_s, idesc_s);
-      mma_abt<D>(tmem_dp, do_s, v_s, idesc_s);
+      mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
+      mma_abt_span<D, kF16>(tmem_dp, do_s, v_s, gm);
       mma_commit(&bars->mma);
     }
     ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
@@ -448,6 +478,14 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
 #pragma unroll 1
     for (int ch = 0; ch < 4; ++ch) {
       uint32_t x[32], y[32], pp[16], pd[16];
+      if (!((gm >> (2 * ch)) & 3u)) {
+        // nothing kept in these 32 key columns: P and dS are zero there (the products below read all 128)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) pp[e] = 0u;
+        store_chunk(p_s, r, ch, pp);
+        store_chunk(ds_s, r, ch, pp);
+        continue;
+      }
       tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
       tmem_ld32(tmem_dp + lane_addr + 32 * ch, y);
       tmem_wait_ld();
@@ -459,7 +497,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
           const int col = 2 * e + u;
           const bool kept = (w[ch] >> col) & 1u;
           p[u] = kept ? ex2_approx(fmaf(__uint_as_float(x[col]), c, -big_l)) : 0.f;
-          ds[u] = p[u] * (__uint_as_float(y[col]) - dsum);
+          ds[u] = kept ? p[u] * (__uint_as_float(y[col]) - dsum) : 0.f;
         }
         pp[e] = pack2<kF16>(p[0], p[1]);
         pd[e] = pack2<kF16>(ds[0], ds[1]);
@@ -526,12 +564,13 @@ cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *sta
   e = cudaFuncSetAttribute(cols, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kColsSmem);
   if (e != cudaSuccess) return e;
   rows<<<B * H * t.n_qt, kThreads, C::kRowsSmem, s>>>(maps, static_cast<uint16_t *>(dQ), stat_l, stat_d, t.row_ptr,
-                                                      t.col_idx, t.bitmap, H, Lq, t.n_qt, scale, err);
+                                                      t.col_idx, t.flags, t.groups, t.bitmap, H, Lq, t.n_qt, scale,
+                                                      err);
   count_launches(1);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cols<<<B * H * t.n_kt, kThreads, C::kColsSmem, s>>>(maps, static_cast<uint16_t *>(dK), static_cast<uint16_t *>(dV),
-                                                      stat_l, stat_d, t.row_ptr, t.col_idx, t.bitmap, H, Lq, Lk,
-                                                      t.n_qt, t.n_kt, scale, err);
+                                                      stat_l, stat_d, t.row_ptr, t.col_idx, t.flags, t.groups,
+                                                      t.bitmap, H, Lq, Lk, t.n_qt, t.n_kt, scale, err);
   count_launches(1);
   return cudaGetLastError();
 }
