@@ -542,6 +542,28 @@ def test_backward_causal_band_and_absent_tiles(ap):
     assert torch.all(dk[:, 1, 512:] == 0) and torch.all(dv[:, 1, 512:] == 0)
 
 
+def test_backward_long_full_size(ap):
+    """The long workload at full size under its own calibrated mask (the configuration the benchmark
+    times): all of dQ, dK, dV against the oracle's derivative."""
+    w = W["long"]
+    bias = inputs.calib_bias(w).cuda()
+    acc = pu.gpu_accumulate(ap, w, 2, bias)
+    del bias
+    mask, tiles, _ = pu.gpu_build_mask(ap, acc, w)
+    del acc
+    q, k, v = inputs.eval_qkv(w)
+    g = torch.Generator().manual_seed(w.seed0 + 77)
+    d_o = torch.randn(q.shape, generator=g).to(q.dtype)
+    out = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles)
+    dq, dk, dv = ap.ap_sparse_attention_bwd(q.cuda(), k.cuda(), v.cuda(), out, d_o.cuda(), tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    want = orc.attention_bwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), inputs.widen(d_o),
+                             mask.cpu().numpy())
+    for name, got, ref in zip(("dQ", "dK", "dV"), (dq, dk, dv), want):
+        err = _rel_l2(got.float().cpu().numpy(), ref)
+        assert err <= 1e-2, (name, err)
+
+
 # ------------------------------------------------------------------- the five workloads
 
 
