@@ -5,8 +5,9 @@
 //   dV = P^T dO,   dP = dO V^T,   dS = P o (dP - D),  D_i = dO_i . O_i,
 //   dQ = scale dS K,   dK = scale dS^T Q.
 // Two kernels follow the tile list, both tile by tile and without overlap between their steps (a
-// first, plain version: one CTA of 128 threads, thread r = row r of the tile; one thread issues the
-// copies and the MMAs, everybody waits on two mbarriers):
+// first, plain version: one CTA of 256 threads, two threads per row of the tile, each with two of
+// the four 32-column chunks; one thread issues the copies and the MMAs, everybody waits on two
+// mbarriers):
 //   rows kernel     one CTA per (b, h, query tile).  Sweep 1 over the row's tiles: S on the tensor
 //                   cores, running maximum and sum of the kept entries -> L_i = log2 sum_j 2^(c S_ij)
 //                   (c = log2 e), and D_i from dO and O; both go to the workspace.  Sweep 2: S and dP
@@ -31,7 +32,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;  // thread (half, r): row r of the tile, chunks 2 half and 2 half + 1
 constexpr int kSubBytes = 128 * 128;  // one slab: 128 rows x 64 elements of 2 bytes
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kMaxPolls = 1u << 22;
@@ -191,13 +192,14 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
 
   // late query tiles (the longest list rows under a causal mask) first
   const int qt = n_qt - 1 - (int)(blockIdx.x / (gridDim.x / n_qt)), bh = blockIdx.x % (gridDim.x / n_qt), h = bh % H;
-  const int r = threadIdx.x, warp = r >> 5;
+  const int r = threadIdx.x & 127, half = threadIdx.x >> 7, warp = threadIdx.x >> 5;
   const int i = qt * kTile + r;
-  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+  const bool leader = threadIdx.x == 0;
   const int t0 = row_ptr[h * n_qt + qt], t1 = row_ptr[h * n_qt + qt + 1];
   const float c = scale * kLog2e;
 
-  if (r == 0) {
+  if (leader) {
     mbar_init(&bars->tma, 1);
     mbar_init(&bars->mma, 1);
     bars->abort_flag = 0;
@@ -216,19 +218,21 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
   bool ok = true;
 
   // Q, dO and O of the query tile; D_i = dO_i . O_i
-  if (r == 0) {
+  if (leader) {
     mbar_arrive_expect_tx(&bars->tma, 3 * C::kTileBytes);
     load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
     load_tile<D>(do_s, &maps.d_o, &bars->tma, qt * kTile, bh);
     load_tile<D>(ds_s, &maps.o, &bars->tma, qt * kTile, bh);
   }
   ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+  // each of the row's two threads takes half of every 128-byte line; the halves are added in a fixed order
   float dsum = 0.f;
+  float *xch = reinterpret_cast<float *>(kv_s);  // [half][row]; the K / V area is not in use yet
   if (ok) {
 #pragma unroll
     for (int s = 0; s < D / 64; ++s)
 #pragma unroll
-      for (int p = 0; p < 8; ++p) {
+      for (int p = 4 * half; p < 4 * half + 4; ++p) {
         const uint4 a = *reinterpret_cast<const uint4 *>(piece_ptr(do_s, s, r, p));
         const uint4 b = *reinterpret_cast<const uint4 *>(piece_ptr(ds_s, s, r, p));
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
@@ -240,13 +244,17 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
         }
       }
   }
+  xch[half * 128 + r] = dsum;
   __syncthreads();  // O is read: its area becomes dS
+  dsum = xch[r] + xch[128 + r];
+  fence_proxy_async_smem();  // the area is written by the copy engine next
+  __syncthreads();
 
   constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, false, true, kF16);
 
   // ---- sweep 1: row maximum and sum over the kept entries
   float m = -CUDART_INF_F, l = 0.f;
-  if (r == 0 && ok && t0 < t1) {
+  if (leader && ok && t0 < t1) {
     mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
     load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
   }
@@ -255,7 +263,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];  // non-empty 16-column groups of the tile
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
-    if (r == 0) {
+    if (leader) {
       if (t + 1 < t1) {  // the other pair was last read by the MMA of tile t - 1, which has completed
         mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
         load_tile<D>(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, &maps.k, &bars->tma, col_idx[t + 1] * kTile, bh);
@@ -270,8 +278,8 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     if (!ok) break;
     tc_fence_after_sync();
 #pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
-      if (!((gm >> (2 * ch)) & 3u)) continue;  // nothing kept in these 32 columns (the same for every thread)
+    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
+      if (!((gm >> (2 * ch)) & 3u)) continue;  // nothing kept in these 32 columns (the same for the whole warp)
       uint32_t x[32];
       tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
       tmem_wait_ld();
@@ -294,15 +302,25 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     __syncthreads();  // S and K may be overwritten
   }
   // L_i = log2 of the row's sum of 2^(c S); +inf for a row without kept entries (then P = 0 everywhere)
+  {
+    // the row's two partial (maximum, sum) pairs, merged the same way by both threads
+    float2 *ml = reinterpret_cast<float2 *>(ds_s);  // [half][row]; the dS area is not in use yet
+    ml[half * 128 + r] = make_float2(m, l);
+    __syncthreads();
+    const float2 a = ml[r], b = ml[128 + r];
+    m = fmaxf(a.x, b.x);
+    l = (a.y > 0.f ? a.y * ex2_approx((a.x - m) * c) : 0.f) + (b.y > 0.f ? b.y * ex2_approx((b.x - m) * c) : 0.f);
+    __syncthreads();
+  }
   const float big_l = l > 0.f ? fmaf(m, c, lg2_approx(l)) : CUDART_INF_F;
-  if (ok && i < Lq) {
+  if (ok && i < Lq && half == 0) {
     stat_l[(size_t)bh * Lq + i] = big_l;
     stat_d[(size_t)bh * Lq + i] = dsum;
   }
 
   // ---- sweep 2: dS and dQ
   bool started = false;
-  if (r == 0 && ok && t0 < t1) {
+  if (leader && ok && t0 < t1) {
     mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
     load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
     load_tile<D>(kv_s + C::kTileBytes, &maps.v, &bars->tma, col_idx[t0] * kTile, bh);
@@ -312,7 +330,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
-    if (r == 0) {
+    if (leader) {
       if (t + 1 < t1) {  // the other pair was last read by dQ += dS K of tile t - 1, which has completed
         unsigned char *nk = kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes;
         mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
@@ -330,7 +348,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     if (!ok) break;
     tc_fence_after_sync();
 #pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
+    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
       if (!((gm >> (2 * ch)) & 3u)) continue;  // dS of these columns is not read: their steps of dQ += dS K are skipped
       uint32_t x[32], y[32], pk[16];
       tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
@@ -353,7 +371,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
-    if (r == 0) {
+    if (leader) {
       tc_fence_after_sync();
       mma_ab<D>(tmem_dq, ds_s, k_s, idesc_dq, started, gm);
       mma_commit(&bars->mma);
@@ -367,7 +385,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     uint16_t *out = dQ + ((size_t)bh * Lq + i) * D;
     tc_fence_after_sync();
 #pragma unroll 1
-    for (int ch = 0; ch < D / 32; ++ch) {
+    for (int ch = half; ch < D / 32; ch += 2) {
       uint32_t x[32];
       if (started) {  // the same for every thread
         tmem_ld32(tmem_dq + lane_addr + 32 * ch, x);
@@ -412,11 +430,12 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
   Bars *bars = reinterpret_cast<Bars *>(smem + 4 * C::kTileBytes + 2 * C::kSquareBytes);
 
   const int kt = blockIdx.x % n_kt, bh = blockIdx.x / n_kt, h = bh % H;
-  const int r = threadIdx.x, warp = r >> 5;
-  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+  const int r = threadIdx.x & 127, half = threadIdx.x >> 7, warp = threadIdx.x >> 5;
+  const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+  const bool leader = threadIdx.x == 0;
   const float c = scale * kLog2e;
 
-  if (r == 0) {
+  if (leader) {
     mbar_init(&bars->tma, 1);
     mbar_init(&bars->mma, 1);
     bars->abort_flag = 0;
@@ -434,7 +453,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
   uint32_t tma_n = 0, mma_n = 0;
   bool ok = true;
 
-  if (r == 0) {
+  if (leader) {
     mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
     load_tile<D>(k_s, &maps.k, &bars->tma, kt * kTile, bh);
     load_tile<D>(v_s, &maps.v, &bars->tma, kt * kTile, bh);
@@ -454,7 +473,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     if (lo >= row_ptr[h * n_qt + qt + 1] || col_idx[lo] != kt) continue;
     const int t = lo;
     const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
-    if (r == 0) {
+    if (leader) {
       mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
       load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
       load_tile<D>(do_s, &maps.d_o, &bars->tma, qt * kTile, bh);
@@ -466,7 +485,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
-    if (r == 0) {
+    if (leader) {
       tc_fence_after_sync();
       mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
       mma_abt_span<D, kF16>(tmem_dp, do_s, v_s, gm);
@@ -476,7 +495,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     if (!ok) break;
     tc_fence_after_sync();
 #pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
+    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
       uint32_t x[32], y[32], pp[16], pd[16];
       if (!((gm >> (2 * ch)) & 3u)) {
         // nothing kept in these 32 key columns: P and dS are zero there (the products below read all 128)
@@ -508,7 +527,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
-    if (r == 0) {
+    if (leader) {
       tc_fence_after_sync();
       mma_atb<D>(tmem_dv, p_s, do_s, idesc_t, started);
       mma_atb<D>(tmem_dk, ds_s, q_s, idesc_t, started);
@@ -527,7 +546,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
       uint16_t *out = (which ? dK : dV) + ((size_t)bh * Lk + j) * D;
       const float f = which ? scale : 1.f;
 #pragma unroll 1
-      for (int ch = 0; ch < D / 32; ++ch) {
+      for (int ch = half; ch < D / 32; ch += 2) {
         uint32_t x[32];
         if (started) {  // the same for every thread; the loads are warp-wide
           tmem_ld32((which ? tmem_dk : tmem_dv) + lane_addr + 32 * ch, x);
