@@ -369,7 +369,7 @@ def run_gpu(args, w):
         d_out = torch.randn(q.shape, generator=gen).to(q.dtype).to(dev)
         ap.ap_sparse_attention_fwd(q, k, v, tiles, out)
         grads = ap.ap_sparse_attention_bwd(q, k, v, out, d_out, tiles)
-        bws = torch.empty(ap.ap_sparse_attention_bwd_workspace_bytes(w.B, w.H, w.Lq), dtype=torch.uint8, device=dev)
+        bws = torch.empty(ap.ap_sparse_attention_bwd_workspace_bytes(w.B, w.H, w.Lq, w.Lk), dtype=torch.uint8, device=dev)
         b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n_bwd = 5
         torch.cuda.synchronize()

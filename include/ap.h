@@ -189,9 +189,10 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
  *   Q, O, dO, dQ  [B,H,Lq,d];  K, V, dK, dV  [B,H,Lk,d], all of type dt (AP_BF16 or AP_F16;
  *   AP_F32 is AP_ERR_UNSUPPORTED); O is the forward's output for the same inputs and tiles.
  *   dQ, dK, dV are overwritten (every element written once: reproducible bit for bit).
- *   workspace     ap_sparse_attention_bwd_workspace_bytes(B, H, Lq) bytes (row statistics)
+ *   workspace     ap_sparse_attention_bwd_workspace_bytes(B, H, Lq, Lk) bytes (row statistics and a
+ *                 table from (query tile, key tile) to the tile's position in the list)
  */
-size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq);
+size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq, int Lk);
 ap_status ap_sparse_attention_bwd(const void *Q, const void *K, const void *V, const void *O, const void *dO,
                                   const ap_tiles *tiles, void *dQ, void *dK, void *dV, int B, int H,
                                   int Lq, int Lk, int d, ap_dtype dt, float scale, void *workspace,

@@ -65,7 +65,7 @@ def _load() -> ctypes.CDLL:
         "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
         "ap_sparse_attention_fwd": (i, [vp, vp, vp, tp, vp, i, i, i, i, i, i, f, vp]),
         "ap_sparse_attention_fwd_host": (i, [vp, vp, vp, tp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, vp]),
-        "ap_sparse_attention_bwd_workspace_bytes": (sz, [i, i, i]),
+        "ap_sparse_attention_bwd_workspace_bytes": (sz, [i, i, i, i]),
         "ap_sparse_attention_bwd": (i, [vp, vp, vp, vp, vp, tp, vp, vp, vp, i, i, i, i, i, i, f, vp, sz, vp]),
         "ap_device_status": (i, [vp]),
     }
@@ -296,8 +296,8 @@ def ap_sparse_attention_fwd(Q, K, V, tiles: Tiles, O=None, scale=0.0, stream=Non
     return O
 
 
-def ap_sparse_attention_bwd_workspace_bytes(B: int, H: int, Lq: int) -> int:
-    return int(lib.ap_sparse_attention_bwd_workspace_bytes(B, H, Lq))
+def ap_sparse_attention_bwd_workspace_bytes(B: int, H: int, Lq: int, Lk: int) -> int:
+    return int(lib.ap_sparse_attention_bwd_workspace_bytes(B, H, Lq, Lk))
 
 
 def ap_sparse_attention_bwd(Q, K, V, O, dO, tiles: Tiles, dQ=None, dK=None, dV=None, scale=0.0, workspace=None,
@@ -313,7 +313,8 @@ def ap_sparse_attention_bwd(Q, K, V, O, dO, tiles: Tiles, dQ=None, dK=None, dV=N
     dK = torch.empty_like(K) if dK is None else _dev(dK, "dK")
     dV = torch.empty_like(V) if dV is None else _dev(dV, "dV")
     if workspace is None:
-        workspace = torch.empty(ap_sparse_attention_bwd_workspace_bytes(B, H, Lq), dtype=torch.uint8, device=Q.device)
+        workspace = torch.empty(ap_sparse_attention_bwd_workspace_bytes(B, H, Lq, Lk), dtype=torch.uint8,
+                                device=Q.device)
     _check(lib.ap_sparse_attention_bwd(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), ctypes.byref(tiles.c),
                                        _ptr(dQ), _ptr(dK), _ptr(dV), B, H, Lq, Lk, d, _dtype_code(Q), float(scale),
                                        _ptr(workspace), workspace.numel(), _stream(stream)),

@@ -291,9 +291,9 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V, c
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
-size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq) {
-  if (B < 1 || H < 1 || Lq < 1) return 0;
-  return bwd_workspace_bytes(B, H, Lq);
+size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq, int Lk) {
+  if (B < 1 || !shape_ok(H, Lq, Lk)) return 0;
+  return bwd_workspace_bytes(B, H, Lq, Lk);
 }
 
 ap_status ap_sparse_attention_bwd(const void *Q, const void *K, const void *V, const void *O, const void *dO,
@@ -308,7 +308,7 @@ ap_status ap_sparse_attention_bwd(const void *Q, const void *K, const void *V, c
   ap_status st = check_tiles(tiles, H, Lq, Lk, true);
   if (st != AP_OK) return st;
   if ((d != 64 && d != 128) || (dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
-  if (workspace_bytes < bwd_workspace_bytes(B, H, Lq)) return AP_ERR_WORKSPACE;
+  if (workspace_bytes < bwd_workspace_bytes(B, H, Lq, Lk)) return AP_ERR_WORKSPACE;
   if (!have_device()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
   return launch_bwd_tc(Q, K, V, O, dO, *tiles, dQ, dK, dV, workspace, B, H, Lq, Lk, d, dt == AP_F16 ? 1 : 0, sc,

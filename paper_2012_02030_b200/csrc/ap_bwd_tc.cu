@@ -15,8 +15,9 @@
 //                   16-bit type and written to shared memory in the operand layout), dQ += dS K on the
 //                   tensor cores (accumulator in TMEM).
 //   columns kernel  one CTA per (b, h, key tile), looping over the query tiles whose list row holds
-//                   that key tile: S, dP, then P and dS to shared memory, dV += P^T dO and
-//                   dK += dS^T Q on the tensor cores.
+//                   that key tile (the next one's Q and dO are copied ahead): S, dP, then P to shared
+//                   memory and dV += P^T dO, then dS to the same area and dK += dS^T Q, which runs
+//                   under the next query tile's S and dP.
 // Every output element is written once, by the thread that owns its row: no atomics, results are
 // reproducible bit for bit.  All tiles are staged by TMA with the 128-byte swizzle, one layout
 // ([64-element slab][row][128 bytes]) serving as K-major and as MN-major operand; P and dS are
@@ -39,7 +40,7 @@ constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct Bars {
-  uint64_t tma, mma;
+  uint64_t tma, mma, mma2;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -91,6 +92,13 @@ __device__ __forceinline__ bool cta_wait(uint64_t *bar, uint32_t parity, Bars *b
     atomicOr(err, kDevErrTimeout);
   }
   return __syncthreads_and(ok ? 1 : 0) != 0;
+}
+
+// After a wait has given up: lets a copy that may still be in flight (the phase after the last one
+// waited for) land before the CTA returns; bounded.
+__device__ __forceinline__ void drain_copies(Bars *bars, uint32_t phases_waited) {
+  if (threadIdx.x == 0) mbar_wait(&bars->tma, phases_waited & 1u, 1u << 16);
+  __syncthreads();
 }
 
 // Address of 16-byte piece `piece` (0..7) of row r in slab `slab` of a staged tile.
@@ -162,8 +170,8 @@ struct Cfg {
   // rows kernel: Q, dO, two (K, V) pairs (the next tile's pair is copied while this one is used), dS
   // (O is staged in the dS area first)
   static constexpr int kRowsSmem = 6 * kTileBytes + kSquareBytes + 1024 + 256;
-  // columns kernel: K, V, Q, dO, P, dS
-  static constexpr int kColsSmem = 4 * kTileBytes + 2 * kSquareBytes + 1024 + 256;
+  // columns kernel: K, V, two (Q, dO) pairs, one area for P and then dS, the staged lookup column
+  static constexpr int kColsSmem = 6 * kTileBytes + kSquareBytes + 1024 + 256 + 1024;
 };
 
 // Thread r's 32 values of one chunk -> 16-bit pairs in row r of a staged 128 x 128 tile, columns [32c, 32c+32).
@@ -405,6 +413,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
       }
     }
   }
+  if (!ok) drain_copies(bars, tma_n);  // ok is the same for every thread
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
@@ -412,22 +421,37 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
 
 // --------------------------------------------------------------------------------------- columns kernel
 
+// tile_id[(h * n_qt + qt) * n_kt + kt] = position of tile (qt, kt) in head h's list, -1 if it is not
+// stored: what the columns kernel walks (the list itself is ordered by query tile).
+__global__ void tile_lookup_kernel(const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
+                                   int n_rows, int n_kt, int32_t *__restrict__ tile_id) {
+  const int row = blockIdx.x;  // h * n_qt + qt
+  if (row >= n_rows) return;
+  for (int kt = threadIdx.x; kt < n_kt; kt += blockDim.x) tile_id[(size_t)row * n_kt + kt] = -1;
+  __syncthreads();
+  const int t0 = row_ptr[row], t1 = row_ptr[row + 1];
+  for (int t = t0 + (int)threadIdx.x; t < t1; t += blockDim.x) tile_id[(size_t)row * n_kt + col_idx[t]] = t;
+}
+
+constexpr int kMaxIds = 256;  // query tiles whose lookup entries are staged in shared memory
+
 template <int D, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK, uint16_t *__restrict__ dV,
                 const float *__restrict__ stat_l, const float *__restrict__ stat_d,
-                const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
-                const uint8_t *__restrict__ flags, const uint8_t *__restrict__ groups,
-                const uint32_t *__restrict__ bitmap, int H, int Lq, int Lk, int n_qt, int n_kt, float scale,
-                unsigned *err) {
+                const int32_t *__restrict__ tile_id, const uint8_t *__restrict__ flags,
+                const uint8_t *__restrict__ groups, const uint32_t *__restrict__ bitmap, int H, int Lq, int Lk,
+                int n_qt, int n_kt, float scale, unsigned *err) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
       reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char *k_s = smem, *v_s = smem + C::kTileBytes, *q_s = smem + 2 * C::kTileBytes,
-                *do_s = smem + 3 * C::kTileBytes, *p_s = smem + 4 * C::kTileBytes,
-                *ds_s = smem + 4 * C::kTileBytes + C::kSquareBytes;
-  Bars *bars = reinterpret_cast<Bars *>(smem + 4 * C::kTileBytes + 2 * C::kSquareBytes);
+  // K, V of the key tile; two (Q, dO) pairs (the next query tile's pair is copied while this one is
+  // used); one 128 x 128 area that holds P for dV += P^T dO and then dS for dK += dS^T Q
+  unsigned char *k_s = smem, *v_s = smem + C::kTileBytes, *qd_s = smem + 2 * C::kTileBytes,
+                *x_s = smem + 6 * C::kTileBytes;
+  Bars *bars = reinterpret_cast<Bars *>(smem + 6 * C::kTileBytes + C::kSquareBytes);
+  int32_t *ids = reinterpret_cast<int32_t *>(smem + 6 * C::kTileBytes + C::kSquareBytes + 256);  // [kMaxIds]
 
   const int kt = blockIdx.x % n_kt, bh = blockIdx.x / n_kt, h = bh % H;
   const int r = threadIdx.x & 127, half = threadIdx.x >> 7, warp = threadIdx.x >> 5;
@@ -438,6 +462,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
   if (leader) {
     mbar_init(&bars->tma, 1);
     mbar_init(&bars->mma, 1);
+    mbar_init(&bars->mma2, 1);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -450,35 +475,47 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
   tc_fence_after_sync();
   const uint32_t tmem = bars->tmem_base;
   const uint32_t tmem_s = tmem, tmem_dp = tmem + 128, tmem_dv = tmem + 256, tmem_dk = tmem + 256 + D;
-  uint32_t tma_n = 0, mma_n = 0;
+  uint32_t tma_n = 0, mma_n = 0, dk_n = 0;
   bool ok = true;
 
-  if (leader) {
-    mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+  // this key tile's column of the lookup table: one entry per query tile, staged once
+  for (int qt = threadIdx.x; qt < n_qt && qt < kMaxIds; qt += kThreads)
+    ids[qt] = tile_id[((size_t)h * n_qt + qt) * n_kt + kt];
+  __syncthreads();
+  // The next query tile at or after qt0 whose list row holds this key tile; n_qt if there is none.
+  // The same for every thread.
+  auto find_from = [&](int qt0, int &t_out) {
+    for (int qt = qt0; qt < n_qt; ++qt) {
+      const int t = qt < kMaxIds ? ids[qt] : tile_id[((size_t)h * n_qt + qt) * n_kt + kt];
+      if (t >= 0) {
+        t_out = t;
+        return qt;
+      }
+    }
+    t_out = -1;
+    return n_qt;
+  };
+
+  int t_cur = -1;
+  int qt_cur = find_from(0, t_cur);
+  if (leader && qt_cur < n_qt) {  // K, V and the first query tile's Q, dO in one go
+    mbar_arrive_expect_tx(&bars->tma, 4 * C::kTileBytes);
     load_tile<D>(k_s, &maps.k, &bars->tma, kt * kTile, bh);
     load_tile<D>(v_s, &maps.v, &bars->tma, kt * kTile, bh);
+    load_tile<D>(qd_s, &maps.q, &bars->tma, qt_cur * kTile, bh);
+    load_tile<D>(qd_s + C::kTileBytes, &maps.d_o, &bars->tma, qt_cur * kTile, bh);
   }
-  ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
 
   constexpr uint32_t idesc_t = idesc_bf16_f32(128, D, true, true, kF16);
 
   bool started = false;
-  for (int qt = 0; qt < n_qt && ok; ++qt) {
-    // the tile (qt, kt) in the list row of qt, if it is stored (key tiles ascend inside a row)
-    int lo = row_ptr[h * n_qt + qt], hi = row_ptr[h * n_qt + qt + 1];
-    while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
-      if (col_idx[mid] < kt) lo = mid + 1; else hi = mid;
-    }
-    if (lo >= row_ptr[h * n_qt + qt + 1] || col_idx[lo] != kt) continue;
-    const int t = lo;
+  for (uint32_t n = 0; qt_cur < n_qt && ok; ++n) {
+    int t_nxt = -1;
+    const int qt_nxt = find_from(qt_cur + 1, t_nxt);
+    unsigned char *q_s = qd_s + (n & 1u) * 2 * C::kTileBytes, *do_s = q_s + C::kTileBytes;
+    const int t = t_cur;
     const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
-    if (leader) {
-      mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
-      load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
-      load_tile<D>(do_s, &maps.d_o, &bars->tma, qt * kTile, bh);
-    }
-    const int i = qt * kTile + r;
+    const int i = qt_cur * kTile + r;
     const float big_l = i < Lq ? stat_l[(size_t)bh * Lq + i] : CUDART_INF_F;
     const float dsum = i < Lq ? stat_d[(size_t)bh * Lq + i] : 0.f;
     const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
@@ -491,20 +528,29 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
       mma_abt_span<D, kF16>(tmem_dp, do_s, v_s, gm);
       mma_commit(&bars->mma);
     }
+    // products complete in order: with S and dP, dK += dS^T Q of the previous query tile is over too,
+    // so its (Q, dO) pair and the P / dS area are free
     ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
     if (!ok) break;
+    if (leader && qt_nxt < n_qt) {
+      unsigned char *nq = qd_s + ((n + 1u) & 1u) * 2 * C::kTileBytes;
+      mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
+      load_tile<D>(nq, &maps.q, &bars->tma, qt_nxt * kTile, bh);
+      load_tile<D>(nq + C::kTileBytes, &maps.d_o, &bars->tma, qt_nxt * kTile, bh);
+    }
     tc_fence_after_sync();
-#pragma unroll 1
-    for (int ch = 2 * half; ch < 2 * half + 2; ++ch) {
-      uint32_t x[32], y[32], pp[16], pd[16];
-      if (!((gm >> (2 * ch)) & 3u)) {
-        // nothing kept in these 32 key columns: P and dS are zero there (the products below read all 128)
+    // this thread's two chunks of P and dS, rounded to the tensors' type; zero where nothing is kept
+    // (the products below read all 128 key columns)
+    uint32_t pp[2][16], pd[2][16];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) pp[e] = 0u;
-        store_chunk(p_s, r, ch, pp);
-        store_chunk(ds_s, r, ch, pp);
+    for (int cc = 0; cc < 2; ++cc) {
+      const int ch = 2 * half + cc;
+      if (!((gm >> (2 * ch)) & 3u)) {  // the same for the whole warp
+#pragma unroll
+        for (int e = 0; e < 16; ++e) pp[cc][e] = pd[cc][e] = 0u;
         continue;
       }
+      uint32_t x[32], y[32];
       tmem_ld32(tmem_s + lane_addr + 32 * ch, x);
       tmem_ld32(tmem_dp + lane_addr + 32 * ch, y);
       tmem_wait_ld();
@@ -515,27 +561,41 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
         for (int u = 0; u < 2; ++u) {
           const int col = 2 * e + u;
           const bool kept = (w[ch] >> col) & 1u;
+          // columns of an empty group hold whatever an earlier tile left in S and dP: never used
           p[u] = kept ? ex2_approx(fmaf(__uint_as_float(x[col]), c, -big_l)) : 0.f;
           ds[u] = kept ? p[u] * (__uint_as_float(y[col]) - dsum) : 0.f;
         }
-        pp[e] = pack2<kF16>(p[0], p[1]);
-        pd[e] = pack2<kF16>(ds[0], ds[1]);
+        pp[cc][e] = pack2<kF16>(p[0], p[1]);
+        pd[cc][e] = pack2<kF16>(ds[0], ds[1]);
       }
-      store_chunk(p_s, r, ch, pp);
-      store_chunk(ds_s, r, ch, pd);
     }
+    store_chunk(x_s, r, 2 * half, pp[0]);
+    store_chunk(x_s, r, 2 * half + 1, pp[1]);
     fence_proxy_async_smem();
     tc_fence_before_sync();
     __syncthreads();
     if (leader) {
       tc_fence_after_sync();
-      mma_atb<D>(tmem_dv, p_s, do_s, idesc_t, started);
-      mma_atb<D>(tmem_dk, ds_s, q_s, idesc_t, started);
+      mma_atb<D>(tmem_dv, x_s, do_s, idesc_t, started);
       mma_commit(&bars->mma);
     }
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);  // P is read: the area takes dS
+    if (!ok) break;
+    store_chunk(x_s, r, 2 * half, pd[0]);
+    store_chunk(x_s, r, 2 * half + 1, pd[1]);
+    fence_proxy_async_smem();
+    __syncthreads();
+    if (leader) {
+      tc_fence_after_sync();
+      mma_atb<D>(tmem_dk, x_s, q_s, idesc_t, started);
+      mma_commit(&bars->mma2);  // waited for through the next tile's S and dP, or below
+    }
+    ++dk_n;
     started = true;
-    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);  // Q, dO, P, dS may be overwritten
+    qt_cur = qt_nxt;
+    t_cur = t_nxt;
   }
+  if (ok && started) ok = cta_wait(&bars->mma2, (dk_n - 1u) & 1u, bars, err);
 
   // ---- dV and dK rows of this key tile (thread r = key row), rounded once
   const int j = kt * kTile + r;
@@ -567,14 +627,15 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
       }
     }
   }
+  if (!ok) drain_copies(bars, tma_n);  // ok is the same for every thread
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
 template <int D, bool kF16>
-cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *stat_l, float *stat_d, const ap_tiles &t,
-                   int B, int H, int Lq, int Lk, float scale, unsigned *err, cudaStream_t s) {
+cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *stat_l, float *stat_d, int32_t *tile_id,
+                   const ap_tiles &t, int B, int H, int Lq, int Lk, float scale, unsigned *err, cudaStream_t s) {
   using C = Cfg<D>;
   auto rows = bwd_rows_kernel<D, kF16>;
   auto cols = bwd_cols_kernel<D, kF16>;
@@ -585,18 +646,23 @@ cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *sta
   rows<<<B * H * t.n_qt, kThreads, C::kRowsSmem, s>>>(maps, static_cast<uint16_t *>(dQ), stat_l, stat_d, t.row_ptr,
                                                       t.col_idx, t.flags, t.groups, t.bitmap, H, Lq, t.n_qt, scale,
                                                       err);
-  count_launches(1);
+  tile_lookup_kernel<<<H * t.n_qt, 128, 0, s>>>(t.row_ptr, t.col_idx, H * t.n_qt, t.n_kt, tile_id);
+  count_launches(2);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cols<<<B * H * t.n_kt, kThreads, C::kColsSmem, s>>>(maps, static_cast<uint16_t *>(dK), static_cast<uint16_t *>(dV),
-                                                      stat_l, stat_d, t.row_ptr, t.col_idx, t.flags, t.groups,
-                                                      t.bitmap, H, Lq, Lk, t.n_qt, t.n_kt, scale, err);
+                                                      stat_l, stat_d, tile_id, t.flags, t.groups, t.bitmap, H, Lq, Lk,
+                                                      t.n_qt, t.n_kt, scale, err);
   count_launches(1);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-size_t bwd_workspace_bytes(int B, int H, int Lq) { return 2 * sizeof(float) * (size_t)B * H * Lq; }
+// row statistics (L and D, one float each per query row) and the (query tile, key tile) -> list position table
+size_t bwd_workspace_bytes(int B, int H, int Lq, int Lk) {
+  const size_t stats = (2 * sizeof(float) * (size_t)B * H * Lq + 255) / 256 * 256;
+  return stats + sizeof(int32_t) * (size_t)H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile);
+}
 
 cudaError_t launch_bwd_tc(const void *Q, const void *K, const void *V, const void *O, const void *dO,
                           const ap_tiles &t, void *dQ, void *dK, void *dV, void *workspace, int B, int H, int Lq,
@@ -610,11 +676,13 @@ cudaError_t launch_bwd_tc(const void *Q, const void *K, const void *V, const voi
     return cudaErrorUnknown;
   float *stat_l = static_cast<float *>(workspace);
   float *stat_d = stat_l + (size_t)B * H * Lq;
+  int32_t *tile_id = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) +
+                                                 (2 * sizeof(float) * (size_t)B * H * Lq + 255) / 256 * 256);
   if (d == 64)
-    return f16 ? launch<64, true>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s)
-               : launch<64, false>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s);
-  return f16 ? launch<128, true>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s)
-             : launch<128, false>(maps, dQ, dK, dV, stat_l, stat_d, t, B, H, Lq, Lk, scale, err, s);
+    return f16 ? launch<64, true>(maps, dQ, dK, dV, stat_l, stat_d, tile_id, t, B, H, Lq, Lk, scale, err, s)
+               : launch<64, false>(maps, dQ, dK, dV, stat_l, stat_d, tile_id, t, B, H, Lq, Lk, scale, err, s);
+  return f16 ? launch<128, true>(maps, dQ, dK, dV, stat_l, stat_d, tile_id, t, B, H, Lq, Lk, scale, err, s)
+             : launch<128, false>(maps, dQ, dK, dV, stat_l, stat_d, tile_id, t, B, H, Lq, Lk, scale, err, s);
 }
 
 }  // namespace ap

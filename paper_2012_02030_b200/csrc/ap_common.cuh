@@ -97,7 +97,7 @@ cudaError_t launch_pool_scores(const float *acc, int H, int Lq, int Lk, int bs, 
                                cudaStream_t s);
 cudaError_t launch_expand_block_mask(const uint8_t *block_mask, int H, int Lq, int Lk, int bs, int causal,
                                      uint8_t *mask, cudaStream_t s);
-size_t bwd_workspace_bytes(int B, int H, int Lq);
+size_t bwd_workspace_bytes(int B, int H, int Lq, int Lk);
 cudaError_t launch_bwd_tc(const void *Q, const void *K, const void *V, const void *O, const void *dO,
                           const ap_tiles &t, void *dQ, void *dK, void *dV, void *workspace, int B, int H, int Lq,
                           int Lk, int d, int f16, float scale, cudaStream_t s);

@@ -80,8 +80,8 @@ def test_forward_rejects_bad_arguments_before_any_device_work():
 def test_backward_rejects_bad_arguments():
     f = ap.lib.ap_sparse_attention_bwd
     t = _tiles()
-    ws = ap.ap_sparse_attention_bwd_workspace_bytes(1, 2, 128)
-    assert ws == 2 * 4 * 2 * 128 and ap.ap_sparse_attention_bwd_workspace_bytes(0, 1, 128) == 0
+    ws = ap.ap_sparse_attention_bwd_workspace_bytes(1, 2, 128, 128)
+    assert ws == 2 * 4 * 2 * 128 + 4 * 2 and ap.ap_sparse_attention_bwd_workspace_bytes(0, 1, 128, 128) == 0
     ok = [FAKE, FAKE, FAKE, FAKE, FAKE, ctypes.byref(t), FAKE, FAKE, FAKE, 1, 2, 128, 128, 64, 1, 0.0, FAKE, ws, None]
     for idx in (0, 1, 2, 3, 4, 6, 7, 8, 16):
         a = list(ok)
