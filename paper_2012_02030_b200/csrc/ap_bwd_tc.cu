@@ -75,7 +75,8 @@ __device__ __forceinline__ float2 unpack2(uint32_t pk) {
   }
 }
 
-// Bounded wait of the whole CTA on one barrier phase; the outcome is the same for every thread.
+// Bounded wait of the whole CTA on one barrier phase; the outcome is the same for every thread.  (Every
+// thread polls: with one polling thread and the others parked at the CTA barrier the kernels were 4 % slower.)
 __device__ __forceinline__ bool cta_wait(uint64_t *bar, uint32_t parity, Bars *bars, unsigned *err) {
   bool ok = false;
   volatile int *abort_flag = &bars->abort_flag;
@@ -99,6 +100,13 @@ __device__ __forceinline__ bool cta_wait(uint64_t *bar, uint32_t parity, Bars *b
 __device__ __forceinline__ void drain_copies(Bars *bars, uint32_t phases_waited) {
   if (threadIdx.x == 0) mbar_wait(&bars->tma, phases_waited & 1u, 1u << 16);
   __syncthreads();
+}
+
+// Non-empty 16-column groups of list tile t (all eight for a tile flagged as fully kept); loaded where
+// it is written, one tile ahead of its use.
+__device__ __forceinline__ uint32_t group_mask(const uint8_t *flags, const uint8_t *groups, int t) {
+  const uint32_t f = ldg_now_u8(flags + t), g = ldg_now_u8(groups + t);
+  return (f & 1u) ? 0xffu : g;
 }
 
 // Address of 16-byte piece `piece` (0..7) of row r in slab `slab` of a staged tile.
@@ -266,15 +274,20 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
     load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
   }
+  uint32_t gm_next = t0 < t1 ? group_mask(flags, groups, t0) : 0u;
+  int kt_ahead = t0 + 1 < t1 ? (int)ldg_now_u32(col_idx + t0 + 1) : 0;  // key tile of list tile t + 1
   for (int t = t0; t < t1 && ok; ++t) {
     unsigned char *k_s = kv_s + ((t - t0) & 1) * 2 * C::kTileBytes;
-    const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];  // non-empty 16-column groups of the tile
+    const uint32_t gm = gm_next;  // non-empty 16-column groups of the tile
+    const int kt_next = kt_ahead;
+    if (t + 1 < t1) gm_next = group_mask(flags, groups, t + 1);
+    if (t + 2 < t1) kt_ahead = (int)ldg_now_u32(col_idx + t + 2);
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
     if (leader) {
       if (t + 1 < t1) {  // the other pair was last read by the MMA of tile t - 1, which has completed
         mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
-        load_tile<D>(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, &maps.k, &bars->tma, col_idx[t + 1] * kTile, bh);
+        load_tile<D>(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, &maps.k, &bars->tma, kt_next * kTile, bh);
       }
       tc_fence_after_sync();
       mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
@@ -333,17 +346,22 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
     load_tile<D>(kv_s + C::kTileBytes, &maps.v, &bars->tma, col_idx[t0] * kTile, bh);
   }
+  gm_next = t0 < t1 ? group_mask(flags, groups, t0) : 0u;
+  kt_ahead = t0 + 1 < t1 ? (int)ldg_now_u32(col_idx + t0 + 1) : 0;
   for (int t = t0; t < t1 && ok; ++t) {
     unsigned char *k_s = kv_s + ((t - t0) & 1) * 2 * C::kTileBytes, *v_s = k_s + C::kTileBytes;
-    const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
+    const uint32_t gm = gm_next;
+    const int kt_next = kt_ahead;
+    if (t + 1 < t1) gm_next = group_mask(flags, groups, t + 1);
+    if (t + 2 < t1) kt_ahead = (int)ldg_now_u32(col_idx + t + 2);
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
     if (leader) {
       if (t + 1 < t1) {  // the other pair was last read by dQ += dS K of tile t - 1, which has completed
         unsigned char *nk = kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes;
         mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
-        load_tile<D>(nk, &maps.k, &bars->tma, col_idx[t + 1] * kTile, bh);
-        load_tile<D>(nk + C::kTileBytes, &maps.v, &bars->tma, col_idx[t + 1] * kTile, bh);
+        load_tile<D>(nk, &maps.k, &bars->tma, kt_next * kTile, bh);
+        load_tile<D>(nk + C::kTileBytes, &maps.v, &bars->tma, kt_next * kTile, bh);
       }
       tc_fence_after_sync();
       mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
@@ -509,12 +527,14 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
   constexpr uint32_t idesc_t = idesc_bf16_f32(128, D, true, true, kF16);
 
   bool started = false;
+  uint32_t gm_next = qt_cur < n_qt ? group_mask(flags, groups, t_cur) : 0u;
   for (uint32_t n = 0; qt_cur < n_qt && ok; ++n) {
     int t_nxt = -1;
     const int qt_nxt = find_from(qt_cur + 1, t_nxt);
     unsigned char *q_s = qd_s + (n & 1u) * 2 * C::kTileBytes, *do_s = q_s + C::kTileBytes;
     const int t = t_cur;
-    const uint32_t gm = (flags[t] & 1) ? 0xffu : (uint32_t)groups[t];
+    const uint32_t gm = gm_next;
+    if (qt_nxt < n_qt) gm_next = group_mask(flags, groups, t_nxt);
     const int i = qt_cur * kTile + r;
     const float big_l = i < Lq ? stat_l[(size_t)bh * Lq + i] : CUDART_INF_F;
     const float dsum = i < Lq ? stat_d[(size_t)bh * Lq + i] : 0.f;
