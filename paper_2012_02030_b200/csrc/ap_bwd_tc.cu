@@ -8,7 +8,9 @@
 // first, plain version: one CTA of 256 threads, two threads per row of the tile, each with two of
 // the four 32-column chunks; one thread issues the copies and the MMAs, everybody waits on two
 // mbarriers):
-//   rows kernel     one CTA per (b, h, query tile).  Sweep 1 over the row's tiles: S on the tensor
+//   rows kernel     one CTA per (b, h, query tile), following the query tile's ROUNDS (the forward's
+//                   schedule: up to eight non-empty 16-column groups gathered from its key tiles, so
+//                   the work follows the slots, not the stored tiles).  Sweep 1 over the rounds: S on the tensor
 //                   cores, running maximum and sum of the kept entries -> L_i = log2 sum_j 2^(c S_ij)
 //                   (c = log2 e), and D_i from dO and O; both go to the workspace.  Sweep 2: S and dP
 //                   on the tensor cores, dS by the threads (P = 2^(c S - L), rounded to the tensors'
@@ -168,7 +170,8 @@ __device__ __forceinline__ void mma_ab(uint32_t d_tmem, const unsigned char *a, 
 }
 
 struct BwdMaps {
-  CUtensorMap q, k, v, o, d_o;
+  CUtensorMap q, k, v, o, d_o;  // boxes of 128 rows
+  CUtensorMap kbox[4], vbox[4];  // boxes of 16, 32, 64, 128 rows: runs of 1, 2, 4, 8 slots of a round
 };
 
 template <int D>
@@ -195,9 +198,9 @@ __device__ __forceinline__ void store_chunk(unsigned char *tile, int r, int c, c
 template <int D, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ, float *__restrict__ stat_l,
-                float *__restrict__ stat_d, const int32_t *__restrict__ row_ptr, const int32_t *__restrict__ col_idx,
-                const uint8_t *__restrict__ flags, const uint8_t *__restrict__ groups,
-                const uint32_t *__restrict__ bitmap, int H, int Lq, int n_qt, float scale, unsigned *err) {
+                float *__restrict__ stat_d, const int32_t *__restrict__ round_ptr,
+                const int32_t *__restrict__ round_rows, const uint8_t *__restrict__ round_info,
+                const uint32_t *__restrict__ round_bitmap, int H, int Lq, int n_qt, float scale, unsigned *err) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -212,7 +215,45 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
   const int i = qt * kTile + r;
   const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
   const bool leader = threadIdx.x == 0;
-  const int t0 = row_ptr[h * n_qt + qt], t1 = row_ptr[h * n_qt + qt + 1];
+  // the query tile's rounds: up to eight non-empty 16-column groups (slots) each, gathered from its
+  // key tiles, as the forward pass visits them
+  const int t0 = round_ptr[h * n_qt + qt], t1 = round_ptr[h * n_qt + qt + 1];
+  struct RoundMeta {
+    uint4 lo, hi;   // first key row of slots 0..3 and 4..7
+    uint32_t info;  // bits 0..3: slots; bit 7: every entry kept
+  };
+  auto meta_of = [&](int t) {
+    RoundMeta mt;
+    mt.lo = ldg_now_v4(round_rows + (size_t)t * 8);
+    mt.hi = ldg_now_v4(round_rows + (size_t)t * 8 + 4);
+    mt.info = ldg_now_u8(round_info + t);
+    return mt;
+  };
+  // One thread: copies the key rows (and value rows) of a round's slots, slot q to rows [16q, 16q+16).
+  // Slots whose key rows follow one another are copied together, in boxes of 8, 4, 2 or 1 slots.
+  auto load_round = [&](unsigned char *kb, const RoundMeta &mt, bool with_v) {
+    const int ng = (int)(mt.info & 15u);
+    const int first[8] = {(int)mt.lo.x, (int)mt.lo.y, (int)mt.lo.z, (int)mt.lo.w,
+                          (int)mt.hi.x, (int)mt.hi.y, (int)mt.hi.z, (int)mt.hi.w};
+    mbar_arrive_expect_tx(&bars->tma, (uint32_t)((with_v ? 2 : 1) * ng * 16 * D * 2));
+    int q = 0;
+    while (q < ng) {
+      int run = 1;
+      while (q + run < ng && first[q + run] == first[q] + 16 * run) ++run;
+      for (int done = 0; done < run;) {
+        const int left = run - done;
+        const int lg = left >= 8 ? 3 : left >= 4 ? 2 : left >= 2 ? 1 : 0;
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) {
+          unsigned char *dst = kb + sl * kSubBytes + (q + done) * 2048;
+          tma_load_3d(dst, &maps.kbox[lg], &bars->tma, 64 * sl, first[q] + 16 * done, bh);
+          if (with_v) tma_load_3d(dst + C::kTileBytes, &maps.vbox[lg], &bars->tma, 64 * sl, first[q] + 16 * done, bh);
+        }
+        done += 1 << lg;
+      }
+      q += run;
+    }
+  };
   const float c = scale * kLog2e;
 
   if (leader) {
@@ -270,30 +311,25 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
 
   // ---- sweep 1: row maximum and sum over the kept entries
   float m = -CUDART_INF_F, l = 0.f;
-  if (leader && ok && t0 < t1) {
-    mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
-    load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
-  }
-  uint32_t gm_next = t0 < t1 ? group_mask(flags, groups, t0) : 0u;
-  int kt_ahead = t0 + 1 < t1 ? (int)ldg_now_u32(col_idx + t0 + 1) : 0;  // key tile of list tile t + 1
+  RoundMeta cur = meta_of(t0 < t1 ? t0 : 0), nxt = meta_of(t0 + 1 < t1 ? t0 + 1 : 0);  // fetched ahead of their use
+  if (leader && ok && t0 < t1) load_round(kv_s, cur, false);
   for (int t = t0; t < t1 && ok; ++t) {
     unsigned char *k_s = kv_s + ((t - t0) & 1) * 2 * C::kTileBytes;
-    const uint32_t gm = gm_next;  // non-empty 16-column groups of the tile
-    const int kt_next = kt_ahead;
-    if (t + 1 < t1) gm_next = group_mask(flags, groups, t + 1);
-    if (t + 2 < t1) kt_ahead = (int)ldg_now_u32(col_idx + t + 2);
+    const RoundMeta me = cur, after = nxt;
+    cur = nxt;
+    if (t + 2 < t1) nxt = meta_of(t + 2);
+    const uint32_t gm = (1u << (me.info & 15u)) - 1u;  // the round's slots, packed from slot 0
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
     if (leader) {
-      if (t + 1 < t1) {  // the other pair was last read by the MMA of tile t - 1, which has completed
-        mbar_arrive_expect_tx(&bars->tma, C::kTileBytes);
-        load_tile<D>(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, &maps.k, &bars->tma, kt_next * kTile, bh);
-      }
+      // the other pair was last read by the MMA of round t - 1, which has completed
+      if (t + 1 < t1) load_round(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, after, false);
       tc_fence_after_sync();
       mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
       mma_commit(&bars->mma);
     }
-    const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
+    uint4 bw = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+    if (!(me.info & 0x80u)) bw = *reinterpret_cast<const uint4 *>(round_bitmap + ((size_t)t * kTile + r) * 4);
     const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
     ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
     if (!ok) break;
@@ -341,34 +377,27 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
 
   // ---- sweep 2: dS and dQ
   bool started = false;
-  if (leader && ok && t0 < t1) {
-    mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
-    load_tile<D>(kv_s, &maps.k, &bars->tma, col_idx[t0] * kTile, bh);
-    load_tile<D>(kv_s + C::kTileBytes, &maps.v, &bars->tma, col_idx[t0] * kTile, bh);
-  }
-  gm_next = t0 < t1 ? group_mask(flags, groups, t0) : 0u;
-  kt_ahead = t0 + 1 < t1 ? (int)ldg_now_u32(col_idx + t0 + 1) : 0;
+  cur = meta_of(t0 < t1 ? t0 : 0);
+  nxt = meta_of(t0 + 1 < t1 ? t0 + 1 : 0);
+  if (leader && ok && t0 < t1) load_round(kv_s, cur, true);
   for (int t = t0; t < t1 && ok; ++t) {
     unsigned char *k_s = kv_s + ((t - t0) & 1) * 2 * C::kTileBytes, *v_s = k_s + C::kTileBytes;
-    const uint32_t gm = gm_next;
-    const int kt_next = kt_ahead;
-    if (t + 1 < t1) gm_next = group_mask(flags, groups, t + 1);
-    if (t + 2 < t1) kt_ahead = (int)ldg_now_u32(col_idx + t + 2);
+    const RoundMeta me = cur, after = nxt;
+    cur = nxt;
+    if (t + 2 < t1) nxt = meta_of(t + 2);
+    const uint32_t gm = (1u << (me.info & 15u)) - 1u;
     ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
     if (!ok) break;
     if (leader) {
-      if (t + 1 < t1) {  // the other pair was last read by dQ += dS K of tile t - 1, which has completed
-        unsigned char *nk = kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes;
-        mbar_arrive_expect_tx(&bars->tma, 2 * C::kTileBytes);
-        load_tile<D>(nk, &maps.k, &bars->tma, kt_next * kTile, bh);
-        load_tile<D>(nk + C::kTileBytes, &maps.v, &bars->tma, kt_next * kTile, bh);
-      }
+      // the other pair was last read by dQ += dS K of round t - 1, which has completed
+      if (t + 1 < t1) load_round(kv_s + ((t + 1 - t0) & 1) * 2 * C::kTileBytes, after, true);
       tc_fence_after_sync();
       mma_abt_span<D, kF16>(tmem_s, q_s, k_s, gm);
       mma_abt_span<D, kF16>(tmem_dp, do_s, v_s, gm);
       mma_commit(&bars->mma);
     }
-    const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
+    uint4 bw = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+    if (!(me.info & 0x80u)) bw = *reinterpret_cast<const uint4 *>(round_bitmap + ((size_t)t * kTile + r) * 4);
     const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
     ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
     if (!ok) break;
@@ -663,9 +692,9 @@ cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *sta
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(cols, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kColsSmem);
   if (e != cudaSuccess) return e;
-  rows<<<B * H * t.n_qt, kThreads, C::kRowsSmem, s>>>(maps, static_cast<uint16_t *>(dQ), stat_l, stat_d, t.row_ptr,
-                                                      t.col_idx, t.flags, t.groups, t.bitmap, H, Lq, t.n_qt, scale,
-                                                      err);
+  rows<<<B * H * t.n_qt, kThreads, C::kRowsSmem, s>>>(maps, static_cast<uint16_t *>(dQ), stat_l, stat_d, t.round_ptr,
+                                                      t.round_rows, t.round_info, t.round_bitmap, H, Lq, t.n_qt,
+                                                      scale, err);
   tile_lookup_kernel<<<H * t.n_qt, 128, 0, s>>>(t.row_ptr, t.col_idx, H * t.n_qt, t.n_kt, tile_id);
   count_launches(2);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -694,6 +723,10 @@ cudaError_t launch_bwd_tc(const void *Q, const void *K, const void *V, const voi
       !make_tile_map_bf16(&maps.v, V, B * H, Lk, d) || !make_tile_map_bf16(&maps.o, O, B * H, Lq, d) ||
       !make_tile_map_bf16(&maps.d_o, dO, B * H, Lq, d))
     return cudaErrorUnknown;
+  for (int lg = 0; lg < 4; ++lg)
+    if (!make_tile_map_bf16(&maps.kbox[lg], K, B * H, Lk, d, 16 << lg) ||
+        !make_tile_map_bf16(&maps.vbox[lg], V, B * H, Lk, d, 16 << lg))
+      return cudaErrorUnknown;
   float *stat_l = static_cast<float *>(workspace);
   float *stat_d = stat_l + (size_t)B * H * Lq;
   int32_t *tile_id = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) +
