@@ -381,13 +381,18 @@ def run_gpu(args, w):
         if ap.ap_device_status() != ap.AP_OK:
             raise RuntimeError("device status not OK after the backward runs")
         bwd_ms = b0.elapsed_time(b1) / n_bwd
-        # executed: per stored tile and batch element eight 128 x 128 x d products (S twice, dP twice,
-        # S for the row statistics, dQ, dK, dV); effective: 10*d per kept entry (2.5 x the forward's 4*d)
-        bwd_tile_fl = 8 * 2.0 * 128 * 128 * w.d * tiles.n_tiles() * w.B
+        # executed (upper bound): the rows kernel works on rounds, four products per slot (S twice, dP, dQ:
+        # 128 rows x 16 columns x d each); the columns kernel on stored tiles, four 128 x 128 x d products
+        # per tile (S, dP over the span of non-empty groups at most, dV, dK in full);
+        # effective: 10*d per kept entry (2.5 x the forward's 4*d)
+        n_rounds_b = int(tiles.round_ptr[-1].item())
+        n_slots_b = int((tiles.round_info[:n_rounds_b] & 15).sum().item())
+        bwd_fl = (4 * 2.0 * 128 * 16 * w.d * n_slots_b + 4 * 2.0 * 128 * 128 * w.d * tiles.n_tiles()) * w.B
         backward = {"ms": bwd_ms, "effective_tflops": 10.0 * w.d * float(nnz.sum().item()) * w.B / (bwd_ms * 1e-3) / 1e12,
-                    "executed_tile_tflops": bwd_tile_fl / (bwd_ms * 1e-3) / 1e12,
-                    "frac_of_bf16_sustained": bwd_tile_fl / (bwd_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
-                    "note": "ap_sparse_attention_bwd (rows kernel + columns kernel), %d runs outside the step" % n_bwd}
+                    "executed_tflops": bwd_fl / (bwd_ms * 1e-3) / 1e12,
+                    "frac_of_bf16_sustained": bwd_fl / (bwd_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
+                    "note": "ap_sparse_attention_bwd (rows kernel on rounds + columns kernel on tiles), %d runs "
+                            "outside the step" % n_bwd}
 
     # ---- the same step replayed from a CUDA graph (launch gaps of the ~25 kernels of a step removed) ----
     # (last: the replays add one calibration batch over and over, which skews the accumulator)
