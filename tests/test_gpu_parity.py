@@ -512,8 +512,14 @@ def _bwd_case(ap, w, mask: torch.Tensor, tol):
     for name, got, ref in zip(("dQ", "dK", "dV"), (dq, dk, dv), want):
         got = got.float().cpu().numpy()
         assert np.isfinite(got).all(), name
-        err = _rel_l2(got, ref)
-        assert err <= tol, (name, err)
+        # Relative in the L2 norm, plus an absolute floor that matters only for concentrated rows:
+        # D_i = dO_i . O_i is formed from the rounded O, an error of about |dO_i| |O_i| ulp / 2, which
+        # stays in dS = P o (dP - D) in proportion to P.  Where a row keeps one entry (P = 1, exact
+        # dS = 0) that is 5e-3 per element of dQ, dK in bf16; it falls off like 1 / (kept entries).
+        conc = float((1.0 / np.maximum(mask.numpy().sum(-1), 1)).mean())
+        floor = (5e-3 if tol >= 1e-2 else 1e-3) * conc * np.sqrt(ref.size)
+        diff = float(np.linalg.norm(got.astype(np.float64) - ref))
+        assert diff <= tol * float(np.linalg.norm(ref)) + floor, (name, diff, float(np.linalg.norm(ref)))
     return dq, dk, dv
 
 
@@ -562,6 +568,38 @@ def test_backward_long_full_size(ap):
     for name, got, ref in zip(("dQ", "dK", "dV"), (dq, dk, dv), want):
         err = _rel_l2(got.float().cpu().numpy(), ref)
         assert err <= 1e-2, (name, err)
+
+
+# -------------------------------------------------------------------------- seeded sweeps
+
+
+def test_seeded_sweep_of_small_shapes(ap):
+    """Forty seeded random configurations (shape, domain, fraction, value distribution, dtype, density):
+    mask builders bit for bit, forward and backward within their tolerances.  Shapes stay small so
+    that the oracle finishes at once; they straddle tile edges (1..300 rows and columns)."""
+    rng = np.random.default_rng(2024)
+    for case in range(40):
+        H = int(rng.integers(1, 4))
+        Lq = int(rng.integers(1, 301))
+        causal = bool(rng.integers(0, 2))
+        Lk = Lq + int(rng.integers(0, 200)) * int(rng.integers(0, 2)) if causal else int(rng.integers(1, 301))
+        keep_diag = bool(rng.integers(0, 2))
+        keep = float(rng.choice([0.01, 0.07, 0.3, 0.5, 0.93, 1.0]))
+        acc = rng.random((H, Lq, Lk), dtype=np.float32)
+        kind = int(rng.integers(0, 3))
+        if kind == 1:
+            acc = np.round(acc * 5) / 5                      # six distinct values
+        elif kind == 2:
+            acc[:] = 0.5                                     # one value
+        w = W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=causal, keep_diag=keep_diag, keep_frac=keep)
+        want = _check_build_mask(ap, acc, w, layer=bool(rng.integers(0, 2)))
+        d = int(rng.choice([64, 128]))
+        dtype = str(rng.choice(["bf16", "f16"]))
+        B = int(rng.integers(1, 3))
+        wf = w.scaled(B=B, d=d, dtype=dtype, seed0=w.seed0 + case)
+        mask = torch.from_numpy(want.copy())
+        _fwd_case(ap, wf, mask)
+        _bwd_case(ap, wf, mask, 1e-2 if dtype == "bf16" else 2e-3)
 
 
 # ------------------------------------------------------------------- the five workloads
