@@ -602,6 +602,40 @@ def test_seeded_sweep_of_small_shapes(ap):
         _bwd_case(ap, wf, mask, 1e-2 if dtype == "bf16" else 2e-3)
 
 
+def test_seeded_sweep_of_accumulate_and_tile_lists(ap):
+    """Thirty seeded random configurations of the calibration sum (shape, domain, dtype, bias or not,
+    one to nine samples) and of the tile-list builders on random masks of random density."""
+    rng = np.random.default_rng(2025)
+    for case in range(30):
+        H = int(rng.integers(1, 4))
+        Lq = int(rng.integers(1, 301))
+        causal = bool(rng.integers(0, 2))
+        Lk = Lq + int(rng.integers(0, 200)) * int(rng.integers(0, 2)) if causal else int(rng.integers(1, 301))
+        d = int(rng.choice([64, 128]))
+        dtype = str(rng.choice(["bf16", "f16", "f32"]))
+        B = int(rng.integers(1, 10))
+        w = W["tiny"].scaled(B=B, H=H, Lq=Lq, Lk=Lk, d=d, dtype=dtype, causal=causal, seed0=7000 + case)
+        bias = None
+        if rng.integers(0, 2):
+            g = torch.Generator().manual_seed(7100 + case)
+            bias = torch.randn((H, Lq, Lk), generator=g)
+        acc = pu.gpu_accumulate(ap, w, 1, None if bias is None else bias.cuda())
+        want = pu.oracle_accumulate(w, 1, bias)
+        np.testing.assert_allclose(acc.cpu().numpy(), want, rtol=2e-5, atol=1e-7 * B, err_msg=str(w))
+        density = float(rng.choice([0.0, 0.02, 0.3, 0.9, 1.0]))
+        mask = inputs.random_mask(H, Lq, Lk, density, seed=7200 + case, causal=causal)
+        tiles = ap.Tiles(H, Lq, Lk)
+        ap.ap_mask_to_tiles(mask.cuda(), tiles)
+        assert ap.ap_device_status() == ap.AP_OK
+        pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(mask.numpy()))
+        dense = ap.Tiles(H, Lq, Lk)
+        ap.ap_dense_tiles(dense, causal=causal)
+        dom = torch.ones((H, Lq, Lk), dtype=torch.uint8)
+        if causal:
+            dom = torch.tril(dom, diagonal=Lk - Lq)
+        pu.assert_tiles_equal(dense.to_host(), orc.mask_to_tiles(dom.numpy()))
+
+
 # ------------------------------------------------------------------- the five workloads
 
 
