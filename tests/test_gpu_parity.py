@@ -548,6 +548,17 @@ def test_backward_causal_band_and_absent_tiles(ap):
     assert torch.all(dk[:, 1, 512:] == 0) and torch.all(dv[:, 1, 512:] == 0)
 
 
+def test_backward_more_query_tiles_than_the_staged_lookup_holds(ap):
+    """A key tile's column of the (query tile, key tile) table is staged for 256 query tiles; beyond
+    that the columns kernel reads the table directly."""
+    H, Lq, Lk = 1, 260 * 128 + 17, 200
+    w = W["tiny"].scaled(B=1, H=H, Lq=Lq, Lk=Lk, d=64, dtype="bf16")
+    mask = inputs.random_mask(H, Lq, Lk, 0.05, seed=96)
+    mask[:, 258 * 128:, :] = 0
+    mask[:, 259 * 128 + 3, 150] = 1            # a lone stored tile far beyond the staged part
+    _bwd_case(ap, w, mask, 1e-2)
+
+
 def test_backward_long_full_size(ap):
     """The long workload at full size under its own calibrated mask (the configuration the benchmark
     times): all of dQ, dK, dV against the oracle's derivative."""
