@@ -37,7 +37,7 @@
 // Warp roles (480 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
 // TMEM lane), warp 8 producer, warp 9 issuer of S = Q K^T and TMEM owner, warp 10 issuer of
 // O += P V, warps 11-14 epilogue (the softmax groups hand (m, l) over and go on with the next
-// item while the epilogue warps wait for the item's last O += P V, merge and write).  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384.  Every wait is bounded; a wait that expires
+// item while the epilogue warps wait for the item's last O += P V, merge and write).  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384 (d = 128); at d = 64 the pair (O_0, O_1) takes 128 columns and two items' pairs alternate at 256 and 384.  Every wait is bounded; a wait that expires
 // raises the device status word and the CTA winds down.
 #include <math_constants.h>
 
@@ -98,7 +98,8 @@ struct Shared {
   uint64_t k_empty[kMaxStages], v_empty[kMaxStages];  // S = Q K^T / O += P V of the stage has completed
   uint64_t s_full[2], p_full[2];                      // per S buffer
   uint64_t pv_done[2];                                // O += P V of a round has completed, per S buffer
-  uint64_t o_done, o_free;                            // per item: O complete / O read out by the epilogue
+  uint64_t o_done[2], o_free[2];                      // per item: O complete / O read out by the epilogue
+                                                      // (one pair per set of accumulators)
   uint64_t ml_ready[4];                               // per item: both groups have handed over (m, l)
   float2 ml[4][2][kTile];                             // [item % 4][group][row] = (m, l)
   int32_t ml_item[4];                                 // the item handed over, -1: no more items
@@ -189,8 +190,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     for (int s = 0; s < kMaxStages; ++s) mbar_init(&sh->b_full[s], 1);
     mbar_init(&sh->pv_done[0], 1);
     mbar_init(&sh->pv_done[1], 1);
-    mbar_init(&sh->o_done, 1);
-    mbar_init(&sh->o_free, 4);  // epilogue warps
+    for (int i = 0; i < 2; ++i) mbar_init(&sh->o_done[i], 1);
+    for (int i = 0; i < 2; ++i) mbar_init(&sh->o_free[i], 4);  // epilogue warps
     for (int i = 0; i < 4; ++i) mbar_init(&sh->ml_ready[i], kSoftmaxWarps);
     sh->abort_flag = 0;
     fence_mbar_init();
@@ -203,7 +204,13 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sh->tmem_base;
+  // The two groups' accumulators of an item.  At d = 64 they take 128 columns together and TMEM has
+  // room for two items' worth: items alternate between them, so that the next item's first
+  // O += P V need not wait until the epilogue has read this item's result.
+  constexpr uint32_t kOBufs = D == 64 ? 2u : 1u;
+  constexpr uint32_t kOGroup = D == 64 ? 64u : 128u;  // columns from group 0's accumulator to group 1's
   const uint32_t tmem_o = tmem + 256;
+  auto o_of_item = [&](uint32_t n) { return tmem_o + (kOBufs == 2u ? 128u * (n & 1u) : 0u); };
   volatile int *abort_flag = &sh->abort_flag;
   const int item_step = (int)gridDim.x;
 
@@ -462,7 +469,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       // (what is ready early first; P, which the softmax has just finished, last)
       ok = warp_wait<31>(&sh->v_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
       // the first round of an item overwrites O: the epilogue of the previous item must have read it
-      if (ok && first && n > 0) ok = warp_wait<31>(&sh->o_free, (n - 1u) & 1u, lane, abort_flag, err);
+      if (ok && first && n >= kOBufs)
+        ok = warp_wait<31>(&sh->o_free[kOBufs == 2u ? (n & 1u) : 0u], ((n / kOBufs) - 1u) & 1u, lane, abort_flag, err);
       if (ok) ok = warp_wait<31>(&sh->p_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
@@ -480,13 +488,13 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
           if (ks < ng) {
             const int grp = (ks >> 1) & 1;
             const uint32_t acc = ks == 0 ? started0 : ks == 2 ? started1 : 1u;  // slots 0 / 2 open their group
-            mma_ts(tmem_o + 128u * grp, p_base + 32 * (ks >> 1) + 8 * (ks & 1),
+            mma_ts(o_of_item(n) + kOGroup * grp, p_base + 32 * (ks >> 1) + 8 * (ks & 1),
                    smem_desc_sw128(v_stage + ks * C::kSlotStride, C::kHalfStride, C::kSbo), idesc_pv, acc);
           }
         }
         mma_commit(&sh->v_empty[st]);
         mma_commit(&sh->pv_done[sb]);
-        if (last) mma_commit(&sh->o_done);
+        if (last) mma_commit(&sh->o_done[kOBufs == 2u ? (n & 1u) : 0u]);
       }
       __syncwarp();
       started0 = 1u;
@@ -498,7 +506,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     const int grp = warp >> 2;               // softmax group: chunks grp and grp + 2 of every round
     const int r = (warp & 3) * 32 + lane;    // row of the query tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tmem_og = tmem_o + 128u * grp;  // this group's output accumulator
+    uint32_t tmem_og = tmem_o + kOGroup * grp;  // this group's output accumulator (of the current item)
     const float ref_slack = 8.f / scale_log2;
     bool ok = true;
     uint32_t n = 0;
@@ -521,6 +529,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         m = -CUDART_INF_F;
         l = 0.f;
         o_started = false;
+        tmem_og = o_of_item(n) + kOGroup * grp;
       }
       // this group's 32-column chunks of the round: grp and grp + 2, as far as the round reaches
       const int n_mine = ((ng + 1) >> 1) > grp + 2 ? 2 : ((ng + 1) >> 1) > grp ? 1 : 0;
@@ -673,19 +682,19 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       const float l_tot = g0.y * a0 + g1.y * a1;
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
       const float f0 = a0 * inv, f1 = a1 * inv;
-      ok = warp_wait(&sh->o_done, n & 1u, lane, abort_flag, err);
+      ok = warp_wait(&sh->o_done[kOBufs == 2u ? (n & 1u) : 0u], (n / kOBufs) & 1u, lane, abort_flag, err);
       if (!ok) break;
       tc_fence_after_sync();
 #pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {
         uint32_t o0[32], o1[32];
-        tmem_ld32(tmem_o + lane_addr + 32 * c, o0);
-        tmem_ld32(tmem_o + 128u + lane_addr + 32 * c, o1);
+        tmem_ld32(o_of_item(n) + lane_addr + 32 * c, o0);
+        tmem_ld32(o_of_item(n) + kOGroup + lane_addr + 32 * c, o1);
         tmem_wait_ld();
         if (c == D / 32 - 1) {  // this thread's rows of O are in registers: the next item may overwrite them
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh->o_free);
+          if (lane == 0) mbar_arrive(&sh->o_free[kOBufs == 2u ? (n & 1u) : 0u]);
         }
         if (i < Lq) {
 #pragma unroll
