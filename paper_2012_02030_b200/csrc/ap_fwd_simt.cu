@@ -23,26 +23,12 @@ template <>
 __device__ __forceinline__ float4 load4<float>(const float *p) {
   return *reinterpret_cast<const float4 *>(p);
 }
-template <>
-__device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16 *p) {
-  uint2 u = *reinterpret_cast<const uint2 *>(p);
-  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u),
-                     __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
-}
 
 template <typename T>
 __device__ __forceinline__ void store4(T *p, float4 v);
 template <>
 __device__ __forceinline__ void store4<float>(float *p, float4 v) {
   *reinterpret_cast<float4 *>(p) = v;
-}
-template <>
-__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 *p, float4 v) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
-  uint2 u;
-  u.x = *reinterpret_cast<uint32_t *>(&a);
-  u.y = *reinterpret_cast<uint32_t *>(&b);
-  *reinterpret_cast<uint2 *>(p) = u;
 }
 
 template <typename T, int D>
