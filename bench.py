@@ -45,6 +45,9 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the ncu
 # captures summarised under profiles/ (None until a capture exists).
 NCU_FWD_TRAFFIC_BYTES = {"long": 255.8e6}  # profiles/long_workload_ncu.md (209.3 MB read + 46.5 MB written)
+# the other stages on the same workload, same file: accumulate 2137.7 MB read + 509.8 MB written per call;
+# build_mask = collecting pass (541 MB read) + emit pass (541 MB read + 275 MB written) + small kernels
+NCU_STAGE_TRAFFIC_BYTES = {"long": {"accumulate": 2647.5e6, "build_mask": 1.40e9}}
 
 
 def load_peaks():
@@ -462,8 +465,16 @@ def run_gpu(args, w):
         "dense_fwd": {"bound": "tensor", "unit": "TFLOP/s", "peak": peaks["bf16_sustained"],
                       "achieved": metrics.tile_flops(T_dense, w.B, w.d) / (stage_ms["dense_fwd"] * 1e-3) / 1e12},
     }
-    for r in by_stage.values():
+    for name, r in by_stage.items():
         r["frac"] = r["achieved"] / r["peak"]
+        r["traffic"] = NCU_STAGE_TRAFFIC_BYTES.get(w.name, {}).get(name)
+    by_stage["accumulate"]["algorithmic_bytes"] = acc_bytes
+    by_stage["build_mask"]["algorithmic_bytes"] = mask_bytes
+    # the kernel with the largest share of the step's device time is not the metric's kernel
+    share = {k: v / sum(stage_ms.values()) for k, v in stage_ms.items()}
+    roof["step_share"] = share["sparse_fwd"]
+    roof["largest_stage"] = {"stage": max(share, key=share.get), "share": max(share.values()),
+                             "roofline": "roofline_by_stage"}
 
     # ---- CPU baseline (bounded sample) -----------------------------------------------------
     cpu = None
