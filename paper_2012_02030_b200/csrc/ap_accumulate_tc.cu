@@ -69,6 +69,26 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Two independent IEEE fp32 operations per instruction (the packed forms of sm_100): the results are
+// those of the scalar fmaf / add, the instruction count is half.
+__device__ __forceinline__ void ffma2(float &d0, float &d1, float a0, float a1, float b, float c0, float c1) {
+  asm("{\n .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %4};\n mov.b64 rc, {%5, %6};\n"
+      " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0, %1}, rd;\n}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void fadd2(float &d0, float &d1, float a0, float a1, float b0, float b1) {
+  asm("{\n .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n"
+      " add.rn.f32x2 rd, ra, rb;\n mov.b64 {%0, %1}, rd;\n}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 __device__ __forceinline__ float lg2_approx(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -279,7 +299,9 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         float t[32];
         if (interior) {  // the usual case: nothing to mask, no per-entry comparison
 #pragma unroll
-          for (int e = 0; e < 32; ++e) t[e] = fmaf(__uint_as_float(x[e]), scale_log2, bias2[32 * c + e]);
+          for (int e = 0; e < 32; e += 2)
+            ffma2(t[e], t[e + 1], __uint_as_float(x[e]), __uint_as_float(x[e + 1]), scale_log2, bias2[32 * c + e],
+                  bias2[32 * c + e + 1]);
         } else {
 #pragma unroll
           for (int e = 0; e < 32; ++e)
@@ -289,21 +311,24 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // four independent chains each for the maximum and for the sum
           float m0 = st.x, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
 #pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            m0 = fmaxf(m0, t[e]);
-            m1 = fmaxf(m1, t[e + 1]);
-            m2 = fmaxf(m2, t[e + 2]);
-            m3 = fmaxf(m3, t[e + 3]);
+          for (int e = 0; e < 32; e += 8) {  // three-input maxima: half the instructions
+            m0 = fmax3(m0, t[e], t[e + 4]);
+            m1 = fmax3(m1, t[e + 1], t[e + 5]);
+            m2 = fmax3(m2, t[e + 2], t[e + 6]);
+            m3 = fmax3(m3, t[e + 3], t[e + 7]);
           }
           const float cm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
           const float cm_safe = cm == -CUDART_INF_F ? 0.f : cm;
           float z0 = st.y * ex2_approx(st.x - cm_safe), z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
+          const float neg_cm = -cm_safe;
+#pragma unroll
           for (int e = 0; e < 32; e += 4) {
-            z0 += ex2_approx(t[e] - cm_safe);
-            z1 += ex2_approx(t[e + 1] - cm_safe);
-            z2 += ex2_approx(t[e + 2] - cm_safe);
-            z3 += ex2_approx(t[e + 3] - cm_safe);
+            float a0, a1, a2, a3;
+            fadd2(a0, a1, t[e], t[e + 1], neg_cm, neg_cm);
+            fadd2(a2, a3, t[e + 2], t[e + 3], neg_cm, neg_cm);
+            fadd2(z0, z1, z0, z1, ex2_approx(a0), ex2_approx(a1));
+            fadd2(z2, z3, z2, z3, ex2_approx(a2), ex2_approx(a3));
           }
           st = make_float2(cm, (z0 + z1) + (z2 + z3));
         } else {
@@ -314,10 +339,15 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             tmem_ld32(ps_addr, ps);
             tmem_wait_ld();
           }
+          const float neg_ref = -ref;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const float p = ex2_approx(t[e] - ref);
-            ps[e] = __float_as_uint(b == 0 ? p : __uint_as_float(ps[e]) + p);
+          for (int e = 0; e < 32; e += 2) {
+            float a0, a1;
+            fadd2(a0, a1, t[e], t[e + 1], neg_ref, neg_ref);
+            float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+            if (b > 0) fadd2(p0, p1, __uint_as_float(ps[e]), __uint_as_float(ps[e + 1]), p0, p1);
+            ps[e] = __float_as_uint(p0);
+            ps[e + 1] = __float_as_uint(p1);
           }
           if (b < Bc - 1) {
             tmem_st32(ps_addr, ps);
