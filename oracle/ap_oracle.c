@@ -19,6 +19,9 @@
  *                          on pruned entries.
  *   oracle_attention_bwd   its derivative with respect to Q, K and V (what step 4 of
  *                          the procedure, retraining under the mask, needs).
+ *   oracle_entmax15, oracle_accumulate_entmax15, oracle_attention_entmax15_fwd
+ *                          the same average and masked attention with 1.5-entmax as the
+ *                          normaliser (the section on sparse normalisation).
  *
  * Parity status: every function here is pinned by tests that do not go through
  * this file's own formulas (library SDPA, closed forms, brute force, invariants,
@@ -490,5 +493,150 @@ void oracle_attention_bwd(const float *Q, const float *K, const float *V, const 
     }
     free(p);
     free(dp);
+  }
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Sparse normalisation: 1.5-entmax in place of the softmax (the section on sparse
+ * normalisation runs the whole procedure with alpha-entmax, alpha = 1.5, as the normaliser).
+ *
+ * alpha-entmax maps a score vector z to the point p of the probability simplex that maximises
+ * p.z + H_alpha(p), H_alpha the Tsallis entropy sum_j (p_j - p_j^alpha) / (alpha (alpha - 1)).
+ * Stationarity on the support and complementary slackness off it give, for alpha = 1.5,
+ *   p_j = max(z_j / 2 - tau, 0)^2      with tau the one number for which sum_j p_j = 1.
+ * (alpha -> 1 is the softmax, alpha = 2 the Euclidean projection onto the simplex.)
+ *
+ * Solved exactly here: with x = z / 2 sorted in descending order, if the support is the k
+ * largest entries then tau solves sum_{j<=k} (x_(j) - tau)^2 = 1 below x_(k), i.e.
+ *   tau_k = mean_k - sqrt((1 - k var_k) / k),  mean_k, var_k = mean and variance of x_(1..k),
+ * and the support is the largest k for which that number exists and lies below x_(k).
+ * Values are taken relative to the largest one (p is invariant to a shift of z).
+ * ------------------------------------------------------------------------------------------ */
+static int descending(const void *a, const void *b) {
+  double x = *(const double *)a, y = *(const double *)b;
+  return (x < y) - (x > y);
+}
+
+/* p[0..n) = 1.5-entmax(z[0..n)); n >= 1; p may alias z. */
+void oracle_entmax15(const double *z, int n, double *p) {
+  double *x = (double *)malloc(sizeof(double) * (size_t)n);
+  double top = -INFINITY;
+  for (int j = 0; j < n; ++j)
+    if (z[j] > top) top = z[j];
+  for (int j = 0; j < n; ++j) x[j] = (z[j] - top) / 2.0; /* <= 0, the largest is 0 */
+  qsort(x, (size_t)n, sizeof(double), descending);
+  double sum = 0.0, sumsq = 0.0, tau = -1.0; /* k = 1: (0 - tau)^2 = 1 */
+  for (int k = 1; k <= n; ++k) {
+    sum += x[k - 1];
+    sumsq += x[k - 1] * x[k - 1];
+    double mean = sum / k, var = sumsq / k - mean * mean;
+    double disc = (1.0 - k * var) / k;
+    if (disc < 0.0) continue;
+    double t = mean - sqrt(disc);
+    if (t < x[k - 1]) tau = t;
+  }
+  for (int j = 0; j < n; ++j) {
+    double u = (z[j] - top) / 2.0 - tau;
+    p[j] = u > 0.0 ? u * u : 0.0;
+  }
+  free(x);
+}
+
+/* Eq. 1 (sum form) with the 1.5-entmax attention matrix: one row (h, i), as accumulate_row. */
+static void accumulate_row_entmax15(double *arow, const float *Q, const float *K, const float *bias,
+                                    int h, int i, int B, int H, int Lq, int Lk, int d, int causal,
+                                    double scale) {
+  int jend = row_domain_end(i, Lq, Lk, causal);
+  if (jend <= 0) return;
+  double *s = (double *)malloc(sizeof(double) * (size_t)jend);
+  for (int b = 0; b < B; ++b) {
+    const float *q = Q + (((size_t)b * H + h) * Lq + i) * d;
+    const float *Kh = K + ((size_t)b * H + h) * (size_t)Lk * d;
+    for (int j = 0; j < jend; ++j) {
+      double dot = 0.0;
+      for (int t = 0; t < d; ++t) dot += (double)q[t] * (double)Kh[(size_t)j * d + t];
+      s[j] = dot * scale;
+      if (bias) s[j] += (double)bias[((size_t)h * Lq + i) * Lk + j];
+    }
+    oracle_entmax15(s, jend, s);
+    for (int j = 0; j < jend; ++j) arow[j] += s[j];
+  }
+  free(s);
+}
+
+/* acc[H,Lq,Lk] += sum_b entmax15 rows of (Q_b K_b^T * scale + bias) over each row's domain. */
+void oracle_accumulate_entmax15(double *acc, const float *Q, const float *K, const float *bias, int B,
+                                int H, int Lq, int Lk, int d, int causal, double scale) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int hi = 0; hi < H * Lq; ++hi) {
+    int h = hi / Lq, i = hi % Lq;
+    accumulate_row_entmax15(acc + ((size_t)h * Lq + i) * Lk, Q, K, bias, h, i, B, H, Lq, Lk, d,
+                            causal, scale);
+  }
+}
+
+/* The same for sampled rows: rows[r] = (h, i), out[r, 0..Lk) += the row's sum. */
+void oracle_accumulate_entmax15_rows(double *out, const int32_t *rows, int n_rows, const float *Q,
+                                     const float *K, const float *bias, int B, int H, int Lq, int Lk,
+                                     int d, int causal, double scale) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int r = 0; r < n_rows; ++r)
+    accumulate_row_entmax15(out + (size_t)r * Lk, Q, K, bias, rows[2 * r], rows[2 * r + 1], B, H, Lq,
+                            Lk, d, causal, scale);
+}
+
+/*
+ * Masked attention of Section 3.2 with the 1.5-entmax normaliser, one output row: pruned
+ * entries are at -inf before the normaliser, so they are outside its argument;
+ *   J = { j : mrow[j] = 1 },  p = entmax15((q . k_j) * scale, j in J),  o = sum_J p_j v_j,
+ * and exactly 0 when J is empty.
+ */
+static void attention_row_entmax15(double *o, const float *q, const float *Kh, const float *Vh,
+                                   const uint8_t *mrow, int Lk, int d, double scale) {
+  double *s = (double *)malloc(sizeof(double) * (size_t)(Lk > 0 ? Lk : 1));
+  int *idx = (int *)malloc(sizeof(int) * (size_t)(Lk > 0 ? Lk : 1));
+  int n = 0;
+  for (int t = 0; t < d; ++t) o[t] = 0.0;
+  for (int j = 0; j < Lk; ++j) {
+    if (!mrow[j]) continue;
+    double dot = 0.0;
+    for (int t = 0; t < d; ++t) dot += (double)q[t] * (double)Kh[(size_t)j * d + t];
+    s[n] = dot * scale;
+    idx[n++] = j;
+  }
+  if (n > 0) {
+    oracle_entmax15(s, n, s);
+    for (int c = 0; c < n; ++c)
+      for (int t = 0; t < d; ++t) o[t] += s[c] * (double)Vh[(size_t)idx[c] * d + t];
+  }
+  free(s);
+  free(idx);
+}
+
+/* All rows: Q[B,H,Lq,d], K,V[B,H,Lk,d], mask[H,Lq,Lk] -> O[B,H,Lq,d]. */
+void oracle_attention_entmax15_fwd(const float *Q, const float *K, const float *V,
+                                   const uint8_t *mask, double *O, int B, int H, int Lq, int Lk,
+                                   int d, double scale) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int bh = 0; bh < B * H; ++bh) {
+    int h = bh % H;
+    for (int i = 0; i < Lq; ++i)
+      attention_row_entmax15(O + ((size_t)bh * Lq + i) * d, Q + ((size_t)bh * Lq + i) * d,
+                             K + (size_t)bh * Lk * d, V + (size_t)bh * Lk * d,
+                             mask + ((size_t)h * Lq + i) * Lk, Lk, d, scale);
+  }
+}
+
+/* Sampled rows: rows[r] = (b, h, i), out[r, 0..d). */
+void oracle_attention_entmax15_rows(const float *Q, const float *K, const float *V,
+                                    const uint8_t *mask, double *out, const int32_t *rows,
+                                    int n_rows, int B, int H, int Lq, int Lk, int d, double scale) {
+  (void)B;
+#pragma omp parallel for schedule(dynamic, 8)
+  for (int r = 0; r < n_rows; ++r) {
+    int b = rows[3 * r], h = rows[3 * r + 1], i = rows[3 * r + 2];
+    size_t bh = (size_t)b * H + h;
+    attention_row_entmax15(out + (size_t)r * d, Q + (bh * Lq + i) * d, K + bh * (size_t)Lk * d,
+                           V + bh * (size_t)Lk * d, mask + ((size_t)h * Lq + i) * Lk, Lk, d, scale);
   }
 }

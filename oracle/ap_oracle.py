@@ -247,3 +247,86 @@ def attention_rows(Q, K, V, mask, rows, scale: float | None = None) -> np.ndarra
     _load().oracle_attention_rows(_p(Q), _p(K), _p(V), _p(mask), _p(out), _p(rows),
                                   rows.shape[0], B, H, Lq, Lk, d, ctypes.c_double(s))
     return out
+
+
+def entmax15(z) -> np.ndarray:
+    """1.5-entmax of a score vector (float64): p_j = max(z_j/2 - tau, 0)^2 with sum p = 1."""
+    z = np.ascontiguousarray(np.asarray(z, dtype=np.float64).reshape(-1))
+    assert z.size >= 1
+    p = np.zeros_like(z)
+    lib = _load()
+    lib.oracle_entmax15.restype = None
+    lib.oracle_entmax15(_p(z), int(z.size), _p(p))
+    return p
+
+
+def accumulate_entmax15(acc: np.ndarray, Q, K, bias=None, causal: bool = False, scale: float | None = None):
+    """Eq. 1 as a running sum with the 1.5-entmax attention matrix: acc[H,Lq,Lk] (float64, in place)."""
+    Q, K = _f32(Q), _f32(K)
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    assert K.shape == (B, H, Lk, d) and acc.shape == (H, Lq, Lk)
+    assert acc.dtype == np.float64 and acc.flags.c_contiguous
+    _check_domain(Lq, Lk, causal)
+    if bias is not None:
+        bias = _f32(bias)
+        assert bias.shape == (H, Lq, Lk)
+    s = 1.0 / np.sqrt(d) if scale is None else scale
+    lib = _load()
+    lib.oracle_accumulate_entmax15.restype = None
+    lib.oracle_accumulate_entmax15(
+        _p(acc), _p(Q), _p(K), _p(bias) if bias is not None else None,
+        B, H, Lq, Lk, d, int(bool(causal)), ctypes.c_double(s),
+    )
+    return acc
+
+
+def accumulate_entmax15_rows(rows, Q, K, bias=None, causal: bool = False, scale: float | None = None):
+    """The 1.5-entmax sum for sampled (h, i) rows only; returns float64 [len(rows), Lk]."""
+    Q, K = _f32(Q), _f32(K)
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    _check_domain(Lq, Lk, causal)
+    rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int32).reshape(-1, 2))
+    out = np.zeros((rows.shape[0], Lk), dtype=np.float64)
+    if bias is not None:
+        bias = _f32(bias)
+    s = 1.0 / np.sqrt(d) if scale is None else scale
+    lib = _load()
+    lib.oracle_accumulate_entmax15_rows.restype = None
+    lib.oracle_accumulate_entmax15_rows(
+        _p(out), _p(rows), rows.shape[0], _p(Q), _p(K), _p(bias) if bias is not None else None,
+        B, H, Lq, Lk, d, int(bool(causal)), ctypes.c_double(s),
+    )
+    return out
+
+
+def attention_entmax15_fwd(Q, K, V, mask, scale: float | None = None) -> np.ndarray:
+    """Masked attention with the 1.5-entmax normaliser in fp64: O[B,H,Lq,d]; rows with no kept key are 0."""
+    Q, K, V = _f32(Q), _f32(K), _f32(V)
+    mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    assert K.shape == (B, H, Lk, d) and V.shape == (B, H, Lk, d) and mask.shape == (H, Lq, Lk)
+    O = np.zeros((B, H, Lq, d), dtype=np.float64)
+    s = 1.0 / np.sqrt(d) if scale is None else scale
+    lib = _load()
+    lib.oracle_attention_entmax15_fwd.restype = None
+    lib.oracle_attention_entmax15_fwd(_p(Q), _p(K), _p(V), _p(mask), _p(O), B, H, Lq, Lk, d, ctypes.c_double(s))
+    return O
+
+
+def attention_entmax15_rows(Q, K, V, mask, rows, scale: float | None = None) -> np.ndarray:
+    """The same for sampled (b, h, i) rows only; returns float64 [len(rows), d]."""
+    Q, K, V = _f32(Q), _f32(K), _f32(V)
+    mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    rows = np.ascontiguousarray(np.asarray(rows, dtype=np.int32).reshape(-1, 3))
+    out = np.zeros((rows.shape[0], d), dtype=np.float64)
+    s = 1.0 / np.sqrt(d) if scale is None else scale
+    lib = _load()
+    lib.oracle_attention_entmax15_rows.restype = None
+    lib.oracle_attention_entmax15_rows(_p(Q), _p(K), _p(V), _p(mask), _p(out), _p(rows),
+                                       rows.shape[0], B, H, Lq, Lk, d, ctypes.c_double(s))
+    return out

@@ -747,3 +747,137 @@ def test_bwd_closed_forms():
     ones = np.ones((H, L, L), dtype=np.uint8)
     dq, dk, dv = orc.attention_bwd(np.zeros_like(q), k, v, g, ones)
     np.testing.assert_allclose(dv[0, 0], np.broadcast_to(g[0, 0].astype(np.float64).sum(0) / L, (L, d)), rtol=1e-13)
+
+
+# --------------------------------------------------------------------------- 1.5-entmax (sparse normalisation)
+
+
+def _entmax15_by_bisection(z):
+    """Independent route to the same vector: tau is the root of the decreasing function
+    sum_j max(z_j/2 - tau, 0)^2 - 1, bracketed by [max/2 - 1, max/2] and found by bisection."""
+    x = np.asarray(z, dtype=np.float64) / 2.0
+    lo, hi = x.max() - 1.0, x.max()
+    for _ in range(200):
+        mid = 0.5 * (lo + hi)
+        if (np.maximum(x - mid, 0.0) ** 2).sum() >= 1.0:
+            lo = mid
+        else:
+            hi = mid
+    return np.maximum(x - 0.5 * (lo + hi), 0.0) ** 2
+
+
+def test_entmax15_two_scores_closed_form():
+    """Two scores a >= b with g = (a - b)/2: u^2 + (u - g)^2 = 1 gives u = (g + sqrt(2 - g^2))/2 while
+    g < 1; from g = 1 on the whole mass sits on the larger score."""
+    for a, b in ((0.0, 0.0), (0.3, -0.4), (1.0, 0.0), (2.5, 0.9), (-1.0, -2.99), (4.0, 2.0), (5.0, 1.0)):
+        g = (a - b) / 2.0
+        if g < 1.0:
+            u = (g + math.sqrt(2.0 - g * g)) / 2.0
+            want = np.array([u * u, (u - g) ** 2])
+        else:
+            want = np.array([1.0, 0.0])
+        np.testing.assert_allclose(orc.entmax15([a, b]), want, rtol=0, atol=1e-15)
+        np.testing.assert_allclose(orc.entmax15([b, a]), want[::-1], rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 7, 64, 1000, 4096])
+@pytest.mark.parametrize("spread", [0.05, 1.0, 4.0])
+def test_entmax15_against_bisection(n, spread):
+    rng = np.random.default_rng(1000 * n + int(100 * spread))
+    z = rng.standard_normal(n) * spread + rng.uniform(-30, 30)
+    if n >= 7:
+        z[3] = z[5] = z.max()                     # ties at the top
+    p = orc.entmax15(z)
+    assert abs(p.sum() - 1.0) <= 1e-12 and np.all(p >= 0.0)
+    np.testing.assert_allclose(p, _entmax15_by_bisection(z), rtol=0, atol=1e-12)
+
+
+def test_entmax15_invariants_and_special_cases():
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal(50) * 2.0
+    p = orc.entmax15(z)
+    np.testing.assert_allclose(orc.entmax15(z + 17.25), p, rtol=0, atol=1e-13)      # shift invariance
+    perm = rng.permutation(50)
+    np.testing.assert_allclose(orc.entmax15(z[perm]), p[perm], rtol=0, atol=1e-15)   # no dependence on position
+    assert np.all(np.diff(p[np.argsort(z)]) >= 0.0)                                 # order preserving
+    assert 0 < np.count_nonzero(p) < 50                                             # sparse, unlike a softmax
+    np.testing.assert_allclose(orc.entmax15(np.full(9, -3.5)), np.full(9, 1.0 / 9.0), rtol=1e-15)
+    np.testing.assert_array_equal(orc.entmax15([1.0, 3.0, -2.0, 0.999]), [0.0, 1.0, 0.0, 0.0])  # gap of 2
+    np.testing.assert_allclose(orc.entmax15([0.0, 0.0, -5.0]), [0.5, 0.5, 0.0], rtol=1e-15)
+    # every score outside the support lies at or below the threshold: z_j / 2 <= tau
+    x = z / 2.0
+    tau = x[p > 0].min() - math.sqrt(p[p > 0].min())
+    assert np.all(x[p == 0] <= tau + 1e-15)
+
+
+def test_entmax15_maximises_its_objective():
+    """The defining property: p maximises p.z + H(p) over the simplex, H the Tsallis entropy of order 1.5,
+    sum_j (p_j - p_j^1.5) / 0.75.  The objective is concave, so it is enough that no move towards another
+    point of the simplex raises it."""
+    rng = np.random.default_rng(6)
+
+    def objective(p, z):
+        return float(p @ z + (p - p ** 1.5).sum() / 0.75)
+
+    for n in (3, 10, 40):
+        z = rng.standard_normal(n) * 1.5
+        p = orc.entmax15(z)
+        best = objective(p, z)
+        for _ in range(200):
+            q = rng.dirichlet(np.full(n, 0.3))
+            for eps in (1e-3, 0.05, 1.0):
+                assert objective((1 - eps) * p + eps * q, z) <= best + 1e-12
+        # and a wrong exponent, a missing 1/2 or a wrong normalisation would not pass:
+        soft = np.exp(z - z.max()); soft /= soft.sum()
+        assert objective(soft, z) < best - 1e-6
+
+
+def _entmax15_rows_np(s, valid):
+    """Row-wise 1.5-entmax over the entries marked valid (numpy + the bisection above)."""
+    out = np.zeros_like(s)
+    for idx in np.ndindex(s.shape[:-1]):
+        keep = valid[idx]
+        if keep.any():
+            out[idx][keep] = _entmax15_by_bisection(s[idx][keep])
+    return out
+
+
+@pytest.mark.parametrize("causal,Lq,Lk", [(False, 9, 14), (True, 11, 11), (True, 6, 13)])
+def test_accumulate_entmax15_equals_row_wise_composition(causal, Lq, Lk):
+    B, H, d = 3, 2, 8
+    q, k = _rand((B, H, Lq, d), 21).numpy(), _rand((B, H, Lk, d), 22).numpy()
+    bias = np.random.default_rng(23).standard_normal((H, Lq, Lk)).astype(np.float32)
+    scale = 0.7
+    s = np.einsum("bhid,bhjd->bhij", q.astype(np.float64), k.astype(np.float64)) * scale + bias[None].astype(np.float64)
+    valid = np.ones((Lq, Lk), dtype=bool)
+    if causal:
+        valid = np.tril(valid, k=Lk - Lq)
+    want = _entmax15_rows_np(s, np.broadcast_to(valid, s.shape)).sum(0)
+    acc = np.full((H, Lq, Lk), 0.25, dtype=np.float64)        # the call adds to what is there
+    orc.accumulate_entmax15(acc, q, k, bias, causal=causal, scale=scale)
+    np.testing.assert_allclose(acc - 0.25, want, rtol=0, atol=1e-12)
+    assert np.all((acc == 0.25) | np.broadcast_to(valid, acc.shape))   # nothing outside the domain is touched
+    rows = [(0, 0), (1, Lq - 1), (1, 3)]
+    got = orc.accumulate_entmax15_rows(rows, q, k, bias, causal=causal, scale=scale)
+    for r, (h, i) in enumerate(rows):
+        np.testing.assert_allclose(got[r], want[h, i], rtol=0, atol=1e-12)
+
+
+def test_attention_entmax15_equals_row_wise_composition():
+    B, H, Lq, Lk, d = 2, 2, 10, 17, 8
+    q, k, v = _rand((B, H, Lq, d), 31).numpy(), _rand((B, H, Lk, d), 32).numpy(), _rand((B, H, Lk, d), 33).numpy()
+    rng = np.random.default_rng(34)
+    mask = (rng.random((H, Lq, Lk)) < 0.4).astype(np.uint8)
+    mask[0, 2] = 0                                             # a row with nothing kept
+    mask[1, 4] = 0; mask[1, 4, 9] = 1                          # a row with a single kept key
+    s = np.einsum("bhid,bhjd->bhij", q.astype(np.float64), k.astype(np.float64)) / math.sqrt(d)
+    p = _entmax15_rows_np(s, np.broadcast_to(mask.astype(bool), s.shape))
+    want = np.einsum("bhij,bhjd->bhid", p, v.astype(np.float64))
+    got = orc.attention_entmax15_fwd(q, k, v, mask)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
+    assert np.all(got[:, 0, 2] == 0.0)
+    np.testing.assert_array_equal(got[:, 1, 4], v[:, 1, 9].astype(np.float64))
+    rows = [(0, 0, 0), (1, 1, 4), (1, 0, 9)]
+    sub = orc.attention_entmax15_rows(q, k, v, mask, rows)
+    for r, (b, h, i) in enumerate(rows):
+        np.testing.assert_allclose(sub[r], want[b, h, i], rtol=0, atol=1e-12)
