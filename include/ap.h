@@ -145,6 +145,21 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
                                   float scale, void *stream);
 
 /*
+ * Eq. 1 for a model whose normaliser is 1.5-entmax instead of the softmax (the section on
+ * sparse normalisation): the same running sum with
+ *   p = entmax15_j( Q[b,h,i,:].K[b,h,j,:] * scale + bias[h,i,j] ),
+ *   entmax15(z)_j = max(z_j / 2 - tau, 0)^2,  tau such that the row sums to 1,
+ * over the row's domain.  Entries outside the domain, and entries inside it that no sample
+ * gives weight, keep their value.  tau is found by Newton's iteration in fp32 from below,
+ * until the step falls under 1e-6 max(1, |tau|).
+ * Arguments, layout, ordering of the sum and error behaviour as ap_accumulate_attention,
+ * except that dt must be AP_BF16 or AP_F16 (AP_ERR_UNSUPPORTED otherwise).
+ */
+ap_status ap_accumulate_attention_entmax15(float *acc, const void *Q, const void *K, const float *bias,
+                                           int B, int H, int Lq, int Lk, int d, ap_dtype dt, int causal,
+                                           float scale, void *stream);
+
+/*
  * Eq. 2 with one threshold per head, as an exact top-k: an entry is pruned
  * unless it is among the k largest of its head.
  *   domain  all (i,j), or the causal domain; n_valid = its size

@@ -55,6 +55,7 @@ def _load() -> ctypes.CDLL:
         "ap_build_mask_workspace_bytes": (sz, [i, i, i]),
         "ap_mask_to_tiles_workspace_bytes": (sz, [i, i, i]),
         "ap_accumulate_attention": (i, [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp]),
+        "ap_accumulate_attention_entmax15": (i, [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp]),
         "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_build_mask_layer": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_random_scores": (i, [vp, i, i, i, ctypes.c_uint64, vp]),
@@ -77,7 +78,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
-           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
+           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_accumulate_attention_entmax15", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
            "ap_sparse_attention_fwd_host", "ap_sparse_attention_bwd_workspace_bytes", "ap_sparse_attention_bwd",
            "ap_device_status")
@@ -194,6 +195,19 @@ def ap_accumulate_attention(acc, Q, K, bias=None, causal=False, scale=0.0, strea
     _check(lib.ap_accumulate_attention(_ptr(acc), _ptr(Q), _ptr(K), _ptr(bias), B, H, Lq, Lk, d,
                                        _dtype_code(Q), int(bool(causal)), float(scale), _stream(stream)),
            "ap_accumulate_attention")
+
+
+def ap_accumulate_attention_entmax15(acc, Q, K, bias=None, causal=False, scale=0.0, stream=None) -> None:
+    _dev(acc, "acc"), _dev(Q, "Q"), _dev(K, "K")
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    if K.shape != (B, H, Lk, d) or acc.shape != (H, Lq, Lk) or acc.dtype != torch.float32 or K.dtype != Q.dtype:
+        raise ValueError("shape/dtype mismatch")
+    if bias is not None and (_dev(bias, "bias").shape != (H, Lq, Lk) or bias.dtype != torch.float32):
+        raise ValueError("bias must be float32 [H,Lq,Lk]")
+    _check(lib.ap_accumulate_attention_entmax15(_ptr(acc), _ptr(Q), _ptr(K), _ptr(bias), B, H, Lq, Lk, d,
+                                                _dtype_code(Q), int(bool(causal)), float(scale), _stream(stream)),
+           "ap_accumulate_attention_entmax15")
 
 
 def _build_mask(fn, name, acc, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head, workspace, stream) -> None:

@@ -53,6 +53,7 @@ struct Cfg {
   static constexpr int kStatsBytes = 2 * kMaxB * 128 * 8;  // [wg][b][row] (max, sum)
   static constexpr int kBarOffset = kStatsOffset + kStatsBytes;
   static constexpr int kSmemBytes = kBarOffset + 256 + 1024;
+  static_assert(kSmemBytes <= 227 * 1024, "within the shared memory of one CTA");
 };
 
 struct Barriers {
@@ -69,26 +70,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Two independent IEEE fp32 operations per instruction (the packed forms of sm_100): the results are
-// those of the scalar fmaf / add, the instruction count is half.
-__device__ __forceinline__ void ffma2(float &d0, float &d1, float a0, float a1, float b, float c0, float c1) {
-  asm("{\n .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %4};\n mov.b64 rc, {%5, %6};\n"
-      " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0, %1}, rd;\n}"
-      : "=f"(d0), "=f"(d1)
-      : "f"(a0), "f"(a1), "f"(b), "f"(c0), "f"(c1));
-}
-__device__ __forceinline__ void fadd2(float &d0, float &d1, float a0, float a1, float b0, float b1) {
-  asm("{\n .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n"
-      " add.rn.f32x2 rd, ra, rb;\n mov.b64 {%0, %1}, rd;\n}"
-      : "=f"(d0), "=f"(d1)
-      : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
-}
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-
 __device__ __forceinline__ float lg2_approx(float x) {
   float y;
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -320,7 +301,6 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           const float cm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
           const float cm_safe = cm == -CUDART_INF_F ? 0.f : cm;
           float z0 = st.y * ex2_approx(st.x - cm_safe), z1 = 0.f, z2 = 0.f, z3 = 0.f;
-#pragma unroll
           const float neg_cm = -cm_safe;
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {

@@ -141,6 +141,21 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
+ap_status ap_accumulate_attention_entmax15(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
+                                           int Lq, int Lk, int d, ap_dtype dt, int causal, float scale,
+                                           void *stream) {
+  if (!acc || !Q || !K || !aligned16(acc) || !aligned16(Q) || !aligned16(K) || (bias && !aligned16(bias)))
+    return AP_ERR_INVALID_ARG;
+  if (B < 1 || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq) || !(scale >= 0.f) || isinf(scale))
+    return AP_ERR_INVALID_ARG;
+  if ((d != 64 && d != 128) || (dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
+  if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
+  const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
+  cudaError_t e = launch_accumulate_entmax_tc(acc, Q, K, bias, B, H, Lq, Lk, d, causal ? 1 : 0, dt == AP_F16 ? 1 : 0,
+                                              sc, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
+}
+
 namespace {
 ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
                           uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,

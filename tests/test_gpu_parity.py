@@ -393,6 +393,91 @@ def test_accumulate_without_bias_and_custom_scale(ap):
     np.testing.assert_allclose(acc.cpu().numpy(), want, rtol=2e-5, atol=1e-7)
 
 
+# ------------------------------------------------------------------------------ accumulate, 1.5-entmax
+
+
+def _entmax_acc(ap, w, n_batches, bias_dev, scale=0.0):
+    acc = torch.zeros((w.H, w.Lq, w.Lk), dtype=torch.float32, device="cuda")
+    for t in range(n_batches):
+        q, k = inputs.calib_qk(w, t)
+        ap.ap_accumulate_attention_entmax15(acc, q.cuda(), k.cuda(), bias_dev, causal=w.causal, scale=scale)
+    assert ap.ap_device_status() == ap.AP_OK
+    return acc
+
+
+def _entmax_want(w, n_batches, bias, scale=None):
+    acc64 = np.zeros((w.H, w.Lq, w.Lk))
+    for t in range(n_batches):
+        q, k = inputs.calib_qk(w, t)
+        orc.accumulate_entmax15(acc64, inputs.widen(q), inputs.widen(k), None if bias is None else bias.numpy(),
+                                causal=w.causal, scale=scale)
+    return acc64
+
+
+# A weight is p = u^2 with u = x - tau; the fp32 threshold is off by at most a few 1e-6 (the stopping rule of
+# the iteration plus the rounding of x, |x| of order 10), so p is off by 2 u dtau <= 2e-5 per sample
+# whatever its size: an absolute bound per sample, plus the relative error of the fp32 square.
+ENTMAX_ATOL, ENTMAX_RTOL = 2e-5, 1e-4
+
+
+@pytest.mark.parametrize("name,over,n_batches", [
+    ("tiny", {}, 3),
+    ("tiny", dict(Lq=77, Lk=77, B=3), 2),            # ragged, bias through direct loads (Lk % 4 != 0)
+    ("tiny", dict(Lq=50, Lk=300, d=128), 2),
+    ("tiny", dict(B=18, H=2), 1),                    # more samples than one launch holds (8)
+    ("bert", dict(B=4, H=3), 2),
+    ("lm", dict(B=2, H=2, Lq=300, Lk=300), 2),       # causal
+    ("long", dict(B=1, H=2, Lq=640, Lk=640), 2),
+    ("txl", dict(B=2, H=2, Lq=200, Lk=333), 2),      # causal with memory keys
+    ("s2s_cross", dict(B=3, H=2, dtype="f16"), 2),
+])
+def test_accumulate_entmax15_matches_oracle(ap, name, over, n_batches):
+    w = W[name].scaled(**over)
+    if w.dtype == "f32":
+        w = w.scaled(dtype="bf16")
+    bias = inputs.calib_bias(w)
+    acc = _entmax_acc(ap, w, n_batches, bias.cuda())
+    assert torch.equal(acc, _entmax_acc(ap, w, n_batches, bias.cuda()))  # fixed order: bit-reproducible
+    got, want = acc.cpu().numpy(), _entmax_want(w, n_batches, bias)
+    total = n_batches * w.B
+    np.testing.assert_allclose(got, want, rtol=ENTMAX_RTOL, atol=ENTMAX_ATOL * total)
+    if w.causal:
+        assert np.all(got[:, ~np.tril(np.ones((w.Lq, w.Lk), dtype=bool), w.Lk - w.Lq)] == 0.0)
+    np.testing.assert_allclose(got.sum(-1), total, rtol=2e-5)
+    # sparse, unlike the softmax average: entries no sample gives weight stay exactly zero
+    clear = want == 0.0
+    assert clear.any() and np.count_nonzero(got[clear]) <= 1e-3 * clear.sum()
+
+
+def test_accumulate_entmax15_special_rows(ap):
+    """Closed forms through the kernel: equal scores give the uniform row (the longest Newton run: the
+    threshold has to travel from max - 1 to max - 1/sqrt(n)); a gap of 2 between the best and the second
+    best score gives a one-hot row."""
+    H, L, d = 1, 1024, 64
+    q = torch.zeros((1, H, L, d), dtype=torch.bfloat16, device="cuda")
+    k = torch.randn((1, H, L, d), generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).cuda()
+    acc = torch.zeros((H, L, L), device="cuda")
+    ap.ap_accumulate_attention_entmax15(acc, q, k, None, causal=True)
+    rows = torch.arange(1, L + 1, dtype=torch.float32, device="cuda")[:, None]
+    want = torch.tril(torch.ones((L, L), device="cuda")) / rows
+    assert torch.allclose(acc[0], want, rtol=2e-4, atol=1e-8)
+    # one-hot: q_i = k_i = 8 e_(i mod d) ... use a bias instead: +4 on the diagonal, 0 elsewhere, q = 0
+    bias = torch.zeros((H, L, L), device="cuda")
+    bias[0].fill_diagonal_(4.0)
+    acc.zero_()
+    ap.ap_accumulate_attention_entmax15(acc, q, k, bias, causal=False)
+    assert torch.equal(acc[0], torch.eye(L, device="cuda"))
+    assert ap.ap_device_status() == ap.AP_OK
+
+
+def test_accumulate_entmax15_sharp_scores_custom_scale(ap):
+    w = W["tiny"].scaled(Lq=40, Lk=90, dtype="bf16")
+    for scale in (0.05, 1.5):
+        got = _entmax_acc(ap, w, 1, None, scale=scale).cpu().numpy()
+        want = _entmax_want(w, 1, None, scale=scale)
+        np.testing.assert_allclose(got, want, rtol=ENTMAX_RTOL, atol=ENTMAX_ATOL * w.B)
+
+
 # ------------------------------------------------------------------------------ forward
 
 
