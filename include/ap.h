@@ -150,8 +150,8 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
  *   p = entmax15_j( Q[b,h,i,:].K[b,h,j,:] * scale + bias[h,i,j] ),
  *   entmax15(z)_j = max(z_j / 2 - tau, 0)^2,  tau such that the row sums to 1,
  * over the row's domain.  Entries outside the domain, and entries inside it that no sample
- * gives weight, keep their value.  tau is found by Newton's iteration in fp32 from below,
- * until the step falls under 1e-6 max(1, |tau|).
+ * gives weight, keep their value.  tau is found in fp32 by solving the row's equation on the
+ * support of a trial threshold and repeating until the step falls under 2e-6 max(1, |tau|).
  * Arguments, layout, ordering of the sum and error behaviour as ap_accumulate_attention,
  * except that dt must be AP_BF16 or AP_F16 (AP_ERR_UNSUPPORTED otherwise).
  */
@@ -298,6 +298,21 @@ ap_status ap_dense_tiles(int H, int Lq, int Lk, int causal, ap_tiles *tiles, voi
 ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V,
                                   const ap_tiles *tiles, void *O, int B, int H, int Lq, int Lk,
                                   int d, ap_dtype dt, float scale, void *stream);
+
+/*
+ * The same masked attention for a model whose normaliser is 1.5-entmax (the section on sparse
+ * normalisation): pruned entries are outside the normaliser's argument,
+ *   O[b,h,i,:] = sum_j p_j V[b,h,j,:],  p = entmax15( scale * Q[b,h,i,:].K[b,h,j,:] : j kept ),
+ *   entmax15(z)_j = max(z_j / 2 - tau, 0)^2,  tau such that the row sums to 1
+ * (found in fp32 as in ap_accumulate_attention_entmax15, to a step under 2e-6 max(1, |tau|)); a row
+ * without kept entries outputs exactly 0.  The weights are rounded to dt before they multiply V
+ * and the row is divided by the sum of the rounded weights.  Reads the tile list's row_ptr,
+ * col_idx, flags and bitmap.  Arguments and error behaviour as ap_sparse_attention_fwd, except
+ * that dt must be AP_BF16 or AP_F16 (AP_ERR_UNSUPPORTED otherwise).
+ */
+ap_status ap_sparse_attention_entmax15_fwd(const void *Q, const void *K, const void *V, const ap_tiles *tiles,
+                                           void *O, int B, int H, int Lq, int Lk, int d, ap_dtype dt,
+                                           float scale, void *stream);
 
 /*
  * The same call for HOST tensors (pinned memory recommended): copies Q, K, V to

@@ -65,6 +65,7 @@ def _load() -> ctypes.CDLL:
         "ap_dense_tiles": (i, [i, i, i, i, tp, vp]),
         "ap_mask_to_tiles_static": (i, [vp, i, i, i, tp, vp]),
         "ap_sparse_attention_fwd": (i, [vp, vp, vp, tp, vp, i, i, i, i, i, i, f, vp]),
+        "ap_sparse_attention_entmax15_fwd": (i, [vp, vp, vp, tp, vp, i, i, i, i, i, i, f, vp]),
         "ap_sparse_attention_fwd_host": (i, [vp, vp, vp, tp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, vp]),
         "ap_sparse_attention_bwd_workspace_bytes": (sz, [i, i, i, i]),
         "ap_sparse_attention_bwd": (i, [vp, vp, vp, vp, vp, tp, vp, vp, vp, i, i, i, i, i, i, f, vp, sz, vp]),
@@ -79,7 +80,7 @@ def _load() -> ctypes.CDLL:
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
            "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_accumulate_attention_entmax15", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
-           "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd",
+           "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd", "ap_sparse_attention_entmax15_fwd",
            "ap_sparse_attention_fwd_host", "ap_sparse_attention_bwd_workspace_bytes", "ap_sparse_attention_bwd",
            "ap_device_status")
 
@@ -307,6 +308,20 @@ def ap_sparse_attention_fwd(Q, K, V, tiles: Tiles, O=None, scale=0.0, stream=Non
     _check(lib.ap_sparse_attention_fwd(_ptr(Q), _ptr(K), _ptr(V), ctypes.byref(tiles.c), _ptr(_dev(O, "O")),
                                        B, H, Lq, Lk, d, _dtype_code(Q), float(scale), _stream(stream)),
            "ap_sparse_attention_fwd")
+    return O
+
+
+def ap_sparse_attention_entmax15_fwd(Q, K, V, tiles: Tiles, O=None, scale=0.0, stream=None):
+    _dev(Q, "Q"), _dev(K, "K"), _dev(V, "V")
+    B, H, Lq, d = Q.shape
+    Lk = K.shape[2]
+    if K.shape != (B, H, Lk, d) or V.shape != K.shape or K.dtype != Q.dtype or V.dtype != Q.dtype:
+        raise ValueError("shape/dtype mismatch")
+    if O is None:
+        O = torch.empty_like(Q)
+    _check(lib.ap_sparse_attention_entmax15_fwd(_ptr(Q), _ptr(K), _ptr(V), ctypes.byref(tiles.c), _ptr(_dev(O, "O")),
+                                                B, H, Lq, Lk, d, _dtype_code(Q), float(scale), _stream(stream)),
+           "ap_sparse_attention_entmax15_fwd")
     return O
 
 

@@ -3,14 +3,19 @@
 //
 // 1.5-entmax of a row of scores z is p_j = max(z_j / 2 - tau, 0)^2 with tau the one number for
 // which the row sums to 1.  f(tau) = sum_j max(x_j - tau, 0)^2 - 1 (x = z / 2) is convex and
-// decreasing, its root lies in [max x - 1, max x), and Newton's iteration started at max x - 1
-// stays left of the root and rises to it:
-//     tau <- tau + (S2 - 1) / (2 S1),   S1 = sum_j max(x_j - tau, 0),  S2 = sum_j max(x_j - tau, 0)^2.
+// decreasing and its root lies in [max x - 1, max x).  On the support of a trial threshold c (the
+// n entries with x_j > c) f is the parabola sum (x_j - tau)^2 - 1, whose smaller root is
+//     c + (S2 - 1) / (S1 + sqrt(S1^2 - n (S2 - 1))),   S1 = sum (x_j - c), S2 = sum (x_j - c)^2 over the support.
+// That root is the answer when the support is the right one; otherwise it lies on the other side
+// of the answer than c (too many entries in the support push it right, too few left), the trial
+// thresholds left of the answer rise and those right of it fall, so the iteration started at
+// max x - 1 ends after a few supports.  Where the parabola has no root (a support far too wide)
+// the step is Newton's, (S2 - 1) / (2 S1), which stays left of the answer.
 // The scores of a row (up to Lk of them, for every sample) do not fit on the chip, but QK^T is
 // cheap on the tensor cores, so the CTA recomputes them: one (head, 128-row query tile) per CTA,
 // up to 8 samples per launch,
 //   sweep 0          S = Q_b K_b(kt)^T for every key tile and sample -> row maxima, tau = max - 1
-//   sweeps 1 .. n    the same visits -> S1, S2 of every (sample, row) -> one Newton step; repeated
+//   sweeps 1 .. n    the same visits -> n, S1, S2 of every (sample, row) -> one step; repeated
 //                    until no row of the CTA moves any more (or kMaxNewton sweeps)
 //   last sweep       p = max(x - tau, 0)^2; the sum over samples is kept in TMEM and added to the
 //                    accumulator once per key tile (one red.global.add per entry and launch).
@@ -18,7 +23,7 @@
 // warps 0-7 normalise (thread (wg, r) owns row r and columns [64 wg, 64 wg + 64) of every key
 // tile), warp 8 copies with TMA, warp 9 issues the products.  The two column halves of a row meet
 // in shared memory at the end of every sweep; the copy and product warps learn there whether
-// another Newton sweep follows.  Every mbarrier wait is bounded.
+// another sweep of the iteration follows.  Every mbarrier wait is bounded.
 #include <math_constants.h>
 
 #include "ap_common.cuh"
@@ -36,7 +41,7 @@ constexpr int kSubBytes = 128 * 128;
 constexpr uint32_t kTmemCols = 512;  // S x 2 (columns 0..255), running sum over b (columns 256..383)
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr int kMaxB = 8;         // samples per launch (row statistics and thresholds live in shared memory)
-constexpr int kMaxNewton = 30;   // Newton sweeps at most (fp32 steps stop moving long before)
+constexpr int kMaxNewton = 30;   // sweeps of the iteration at most (fp32 steps stop moving long before)
 constexpr int kBiasBytes = 128 * 128 * 4;
 
 template <int D>
@@ -47,7 +52,9 @@ struct Cfg {
   static constexpr int kBiasOffset = 2 * kStages * kTileBytes;
   static constexpr int kStatsOffset = kBiasOffset + kBiasBytes;
   static constexpr int kStatsBytes = 2 * kMaxB * 128 * 8;  // [wg][b][row] (max, -) or (S1, S2)
-  static constexpr int kTauOffset = kStatsOffset + kStatsBytes;
+  static constexpr int kCntOffset = kStatsOffset + kStatsBytes;
+  static constexpr int kCntBytes = 2 * kMaxB * 128 * 4;    // [wg][b][row] support size n
+  static constexpr int kTauOffset = kCntOffset + kCntBytes;
   static constexpr int kTauBytes = 2 * kMaxB * 128 * 4;    // [wg][b][row]: each half keeps its own copy
   static constexpr int kBarOffset = kTauOffset + kTauBytes;
   static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
@@ -77,7 +84,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
   return false;
 }
 
-// Sweep s + 1 is the last one when sweep s was a Newton sweep after which nothing moved.
+// Sweep s + 1 is the last one when sweep s was a sweep of the iteration after which nothing moved.
 __device__ __forceinline__ bool last_follows(const Barriers *bars, int s) {
   return s >= 1 && (s >= kMaxNewton || *reinterpret_cast<const volatile int *>(&bars->more[s]) == 0);
 }
@@ -94,6 +101,7 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
       reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char *bias_s = smem + C::kBiasOffset;
   float2 *stats = reinterpret_cast<float2 *>(smem + C::kStatsOffset);  // [wg][b][row]
+  float *cnts = reinterpret_cast<float *>(smem + C::kCntOffset);       // [wg][b][row]
   float *taus = reinterpret_cast<float *>(smem + C::kTauOffset);       // [wg][b][row]
   Barriers *bars = reinterpret_cast<Barriers *>(smem + C::kBarOffset);
 
@@ -211,13 +219,14 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int jend = causal ? min(Lk, i + 1 + off) : Lk;  // first key outside this row's domain
     const bool vec = (Lk & 3) == 0;
     float2 *my_stats = stats + (size_t)wg * kMaxB * 128 + r;  // + b * 128
+    float *my_cnt = cnts + (size_t)wg * kMaxB * 128 + r;      // + b * 128
     float *my_tau = taus + (size_t)wg * kMaxB * 128 + r;      // + b * 128
 
     float hbias[64];  // half the bias of this thread's 64 columns of the current key tile
     int v = 0, tl = 0;
     bool last = false, ok = true;
     for (int sw = 0; ok; ++sw) {
-      const int kind = sw == 0 ? 0 : (last ? 2 : 1);  // 0 maxima, 1 Newton sums, 2 weights
+      const int kind = sw == 0 ? 0 : (last ? 2 : 1);  // 0 maxima, 1 sums over the support, 2 weights
       for (int vv = 0; vv < visits_per_sweep && ok; ++vv, ++v) {
         const int kt = vv / Bc, b = vv % Bc;
         const int buf = v & 1;
@@ -258,6 +267,7 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const float neg_tau = kind == 0 ? 0.f : -my_tau[b * 128];
         // statistics of (sample b, this half of the row): fresh at the first key tile of a sweep
         float2 st = kt == 0 ? make_float2(kind == 0 ? -CUDART_INF_F : 0.f, 0.f) : my_stats[b * 128];
+        float cnt = (kind != 1 || kt == 0) ? 0.f : my_cnt[b * 128];
         ok = wait_or_abort(&bars->s_full[buf], (uint32_t)(v >> 1) & 1u, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
@@ -302,6 +312,7 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
               fadd2(a2, a3, a2, a3, u2, u3);
               ffma2v(q0, q1, u0, u1, u0, u1, q0, q1);
               ffma2v(q2, q3, u2, u3, u2, u3, q2, q3);
+              cnt += ((u0 > 0.f ? 1.f : 0.f) + (u1 > 0.f ? 1.f : 0.f)) + ((u2 > 0.f ? 1.f : 0.f) + (u3 > 0.f ? 1.f : 0.f));
             }
             st = make_float2((a0 + a1) + (a2 + a3), (q0 + q1) + (q2 + q3));
           } else {
@@ -357,6 +368,7 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         tc_fence_before_sync();
         mbar_arrive(&bars->s_empty[buf]);
         if (kind != 2) my_stats[b * 128] = st;
+        if (kind == 1) my_cnt[b * 128] = cnt;
       }
       if (!ok || last) break;
       // ---- end of a sweep: the two halves of every row meet, every (sample, row) takes its step
@@ -372,12 +384,13 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         } else {
           tau = my_tau[b * 128];
           const float S1 = s0.x + s1.x, S2 = s0.y + s1.y;
-          const float step = S1 > 0.f ? (S2 - 1.f) / (2.f * S1) : 0.f;
+          const float n = cnts[(size_t)b * 128 + r] + cnts[(size_t)(kMaxB + b) * 128 + r];
+          // root of the support's parabola; Newton's step where it has none
+          const float disc = S1 * S1 - n * (S2 - 1.f);
+          const float step = S1 > 0.f ? (S2 - 1.f) / (S1 + (disc >= 0.f ? sqrtf(disc) : S1)) : 0.f;
+          tau += step;
           // below the resolution of tau itself a step is rounding noise of the sums
-          if (step > 1e-6f * fmaxf(1.f, fabsf(tau))) {
-            tau += step;
-            moved = true;
-          }
+          moved = moved || fabsf(step) > 2e-6f * fmaxf(1.f, fabsf(tau));
         }
         my_tau[b * 128] = tau;
       }

@@ -306,6 +306,23 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V, c
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
+ap_status ap_sparse_attention_entmax15_fwd(const void *Q, const void *K, const void *V, const ap_tiles *tiles,
+                                           void *O, int B, int H, int Lq, int Lk, int d, ap_dtype dt, float scale,
+                                           void *stream) {
+  if (!Q || !K || !V || !O || !aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O))
+    return AP_ERR_INVALID_ARG;
+  if (B < 1 || !shape_ok(H, Lq, Lk) || !(scale >= 0.f) || isinf(scale)) return AP_ERR_INVALID_ARG;
+  if ((int64_t)B * H * ceil_div(Lq, kTile) > (int64_t)0x7fffffff) return AP_ERR_INVALID_ARG;
+  ap_status st = check_tiles(tiles, H, Lq, Lk, true);
+  if (st != AP_OK) return st;
+  if ((d != 64 && d != 128) || (dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
+  if (!have_device()) return AP_ERR_CUDA;
+  const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
+  cudaError_t e = launch_fwd_entmax_tc(Q, K, V, *tiles, O, B, H, Lq, Lk, d, dt == AP_F16 ? 1 : 0, sc,
+                                       static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
+}
+
 size_t ap_sparse_attention_bwd_workspace_bytes(int B, int H, int Lq, int Lk) {
   if (B < 1 || !shape_ok(H, Lq, Lk)) return 0;
   return bwd_workspace_bytes(B, H, Lq, Lk);

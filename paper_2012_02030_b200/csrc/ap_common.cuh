@@ -89,6 +89,9 @@ cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const
 cudaError_t launch_accumulate_entmax_tc(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
                                         int Lq, int Lk, int d, int causal, int f16, float scale, cudaStream_t s);
 
+cudaError_t launch_fwd_entmax_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O, int B, int H,
+                                 int Lq, int Lk, int d, int f16, float scale, cudaStream_t s);
+
 // Tensor map of a [B*H, L, d] tensor of 16-bit elements (bf16 or fp16: the copy engine moves them
 // unchanged and fills out-of-range elements with zero bits) for box_rows-row x 64-element swizzled boxes.
 bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d, int box_rows = 128);

@@ -509,6 +509,68 @@ def test_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
     assert np.all(o[:, empty] == 0.0)
 
 
+# ---- the same attention with the 1.5-entmax normaliser
+
+
+def _entmax_fwd_case(ap, w, mask: torch.Tensor, scale=0.0):
+    q, k, v = inputs.eval_qkv(w)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    out = torch.full_like(q, 3.0).cuda()          # poison: every element must be written
+    ap.ap_sparse_attention_entmax15_fwd(q.cuda(), k.cuda(), v.cuda(), tiles, out, scale=scale)
+    assert ap.ap_device_status() == ap.AP_OK
+    ref = orc.attention_entmax15_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy(),
+                                     scale=None if scale == 0.0 else scale)
+    # Sparse rows average few rows of V, so |O| reaches the size of single values of V (up to 4 and more):
+    # the output's own rounding (half an ulp: 2^-9 |O| in bf16, 2^-12 |O| in fp16) no longer fits under a fixed
+    # absolute bound.  Bound: that rounding plus the absolute part of the softmax path's tolerance.
+    got = out.float().cpu().numpy()
+    rtol, atol = (2.0 ** -8, 6e-3) if w.dtype == "bf16" else (2.0 ** -11, 1.5e-3)
+    np.testing.assert_allclose(got, ref, rtol=rtol, atol=atol)
+    rel_l2 = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30))
+    assert rel_l2 <= pu.TOL[w.dtype]["rel_l2"], (w.name, rel_l2)
+    return out, ref
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("shape", [(2, 2, 128, 128), (1, 2, 200, 333), (2, 1, 513, 130), (1, 1, 5, 7),
+                                   (1, 2, 384, 1200)])
+def test_entmax_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
+    B, H, Lq, Lk = shape
+    w = W["tiny"].scaled(B=B, H=H, Lq=Lq, Lk=Lk, d=d, dtype=dtype)
+    mask = inputs.random_mask(H, Lq, Lk, 0.15, seed=81, empty_rows=(0, Lq - 1) if Lq > 2 else ())
+    mask[0, : min(128, Lq), : min(128, Lk)] = 1   # a fully kept (or edge-full) tile next to partial ones
+    if Lq > 256:
+        mask[H - 1, 128:256] = 0                   # a query tile with no kept tile at all
+    out, _ = _entmax_fwd_case(ap, w, mask)
+    o = out.float().cpu().numpy()
+    empty = mask.numpy().sum(-1) == 0
+    assert np.all(o[:, empty] == 0.0)
+
+
+def test_entmax_forward_closed_forms_and_scale(ap):
+    """One kept entry per row: the output is that row of V, bit for bit.  Everything kept and Q = 0: the mean of
+    V.  A sharp custom scale: rows close to one-hot."""
+    w = W["tiny"].scaled(B=1, H=2, Lq=256, Lk=256, d=64, dtype="bf16")
+    q, k, v = inputs.eval_qkv(w)
+    cols = torch.randint(0, w.Lk, (w.H, w.Lq), generator=torch.Generator().manual_seed(9))
+    mask = torch.zeros((w.H, w.Lq, w.Lk), dtype=torch.uint8)
+    mask.scatter_(2, cols[..., None], 1)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    out = ap.ap_sparse_attention_entmax15_fwd(q.cuda(), k.cuda(), v.cuda(), tiles).cpu()
+    want = torch.gather(v, 2, cols[None, ..., None].expand(1, w.H, w.Lq, w.d))
+    assert torch.equal(out, want)
+    ones = torch.ones_like(mask)
+    ap.ap_mask_to_tiles(ones.cuda(), tiles)
+    out = ap.ap_sparse_attention_entmax15_fwd(torch.zeros_like(q).cuda(), k.cuda(), v.cuda(), tiles).float().cpu()
+    mean = v.float().mean(2, keepdim=True).expand_as(out)
+    assert float((out - mean).abs().max()) <= 1e-2
+    for scale in (0.02, 2.0):
+        _entmax_fwd_case(ap, w, inputs.random_mask(w.H, w.Lq, w.Lk, 0.3, seed=5), scale=scale)
+
+
 @pytest.mark.parametrize("d", [64, 128])
 @pytest.mark.parametrize("case", [
     # (B, H, Lq, Lk, group_frac, fill, full_tile_frac, causal)
