@@ -397,6 +397,38 @@ def run_gpu(args, w):
                     "note": "ap_sparse_attention_bwd (rows kernel on rounds + columns kernel on tiles), %d runs "
                             "outside the step" % n_bwd}
 
+    # ---- the same two stages for a model normalised by 1.5-entmax (outside the step) ----
+    entmax = None
+    if w.dtype != "f32":
+        acc_e = torch.zeros_like(acc)
+        cq, ck = calib[0]
+        n_ent = 3
+        ent_ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ent_ms = [0.0, 0.0]
+        for it in range(2 + n_ent):
+            ent_ev[0].record()
+            ap.ap_accumulate_attention_entmax15(acc_e, cq, ck, bias, causal=w.causal)
+            ent_ev[1].record()
+            ap.ap_sparse_attention_entmax15_fwd(q, k, v, tiles, out)
+            ent_ev[2].record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                ent_ms[0] += ent_ev[0].elapsed_time(ent_ev[1]) / n_ent
+                ent_ms[1] += ent_ev[1].elapsed_time(ent_ev[2]) / n_ent
+        if ap.ap_device_status() != ap.AP_OK:
+            raise RuntimeError("device status not OK after the entmax runs")
+        support = float((acc_e != 0).sum().item()) / float(w.n_valid * w.H)
+        del acc_e
+        # algorithmic work: one pass of Q K^T over the domain (accumulate), 4*d per kept entry (forward);
+        # the kernels recompute Q K^T once per sweep of the threshold iteration
+        entmax = {"accumulate_ms": ent_ms[0], "sparse_fwd_ms": ent_ms[1],
+                  "accumulate_one_pass_tflops": 2.0 * w.d * w.n_valid * w.H * w.B / (ent_ms[0] * 1e-3) / 1e12,
+                  "fwd_effective_tflops": metrics.effective_flops(int(nnz.sum().item()), w.B, w.d) / (ent_ms[1] * 1e-3) / 1e12,
+                  "entries_given_weight": support,
+                  "note": "ap_accumulate_attention_entmax15 on one calibration batch into a scratch accumulator and "
+                          "ap_sparse_attention_entmax15_fwd under the step's mask, %d runs after 2 warm-up runs; "
+                          "entries_given_weight = fraction of the domain that received weight from any sample" % n_ent}
+
     # ---- the same step replayed from a CUDA graph (launch gaps of the ~25 kernels of a step removed) ----
     # (last: the replays add one calibration batch over and over, which skews the accumulator)
     graph_ms = None
@@ -506,6 +538,7 @@ def run_gpu(args, w):
         "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer, "backward": backward,
+        "entmax15": entmax,
         "graph_replay": {"ms_per_step": graph_ms, "note": "the same step (same calibration batch every replay) "
                          "captured once in a CUDA graph; steps replays timed with one pair of events"},
     }

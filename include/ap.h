@@ -306,8 +306,8 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V,
  *   entmax15(z)_j = max(z_j / 2 - tau, 0)^2,  tau such that the row sums to 1
  * (found in fp32 as in ap_accumulate_attention_entmax15, to a step under 2e-6 max(1, |tau|)); a row
  * without kept entries outputs exactly 0.  The weights are rounded to dt before they multiply V
- * and the row is divided by the sum of the rounded weights.  Reads the tile list's row_ptr,
- * col_idx, flags and bitmap.  Arguments and error behaviour as ap_sparse_attention_fwd, except
+ * and the row is divided by the sum of the rounded weights.  Follows the tile list's rounds
+ * (round_ptr, round_rows, round_info, round_bitmap).  Arguments and error behaviour as ap_sparse_attention_fwd, except
  * that dt must be AP_BF16 or AP_F16 (AP_ERR_UNSUPPORTED otherwise).
  */
 ap_status ap_sparse_attention_entmax15_fwd(const void *Q, const void *K, const void *V, const ap_tiles *tiles,

@@ -4,8 +4,10 @@
 //   entmax15(z)_j = max(z_j / 2 - tau, 0)^2 with tau such that the row sums to 1; a row without
 //   kept entries outputs 0.
 // Unlike a softmax, the weights cannot be formed in one pass with a running correction: tau depends
-// on all kept scores of the row.  One CTA owns one (b, h, 128-row query tile) and sweeps the kept
-// tiles of its list row several times, recomputing S = Q K^T on the tensor cores each time:
+// on all kept scores of the row.  One CTA owns one (b, h, 128-row query tile) and sweeps the rounds
+// of its list row (the schedule of the tile list: up to eight non-empty groups of 16 key columns,
+// taken from one or several key tiles, per round) several times, recomputing S = Q K^T on the tensor
+// cores each time:
 //   sweep 0          row maxima over the kept entries, tau = max - 1 (left of the root)
 //   sweeps 1 .. n    over the support of the trial threshold (the n entries with x > tau):
 //                    S1 = sum (x - tau), S2 = sum (x - tau)^2 -> tau moves to the smaller root of the
@@ -16,8 +18,10 @@
 //   last sweep       P = max(x - tau, 0)^2 rounded to the tensors' type, written over S in TMEM;
 //                    O += P V (A operand from TMEM); the epilogue divides by the sum of the rounded
 //                    weights, so that O is an exact convex combination of V rows.
-// Warps 0-7 normalise (thread (wg, r) owns row r and columns [64 wg, 64 wg + 64) of every tile),
-// warp 8 copies with TMA (Q once; K every sweep; V in the last sweep), warp 9 issues the products.
+// Warps 0-7 normalise (thread (wg, r) owns row r and columns [64 wg, 64 wg + 64) of every round),
+// warp 8 copies with TMA (Q once; the rounds' K rows every sweep, in boxes of 16 rows per group or
+// one box of 128 rows for eight adjacent groups, into a ring of 4 to 6 stages; V rows in the last
+// sweep), warp 9 issues the products.
 // Every mbarrier wait is bounded.
 #include <math_constants.h>
 
@@ -41,10 +45,13 @@ template <int D>
 struct Cfg {
   static constexpr int kSub = D / 64;
   static constexpr int kTileBytes = kSub * kSubBytes;
-  static constexpr int kStages = D == 64 ? 4 : 2;         // (K, V) pairs in flight
+  // K is copied again in every sweep and a list row is a few rounds long: a ring deep enough to hold
+  // a short row whole keeps the copies several visits ahead of the products.  V is needed once.
+  static constexpr int kStages = D == 64 ? 6 : 4;         // K ring
+  static constexpr int kVStages = D == 64 ? 2 : 1;        // V ring (last sweep)
   static constexpr int kKOffset = kTileBytes;             // after Q
   static constexpr int kVOffset = kKOffset + kStages * kTileBytes;
-  static constexpr int kStatsOffset = kVOffset + kStages * kTileBytes;
+  static constexpr int kStatsOffset = kVOffset + kVStages * kTileBytes;
   static constexpr int kStatsBytes = 2 * 128 * 8;         // [wg][row] (max, -), (S1, S2) or (sum of weights, -)
   static constexpr int kCntOffset = kStatsOffset + kStatsBytes;
   static constexpr int kCntBytes = 2 * 128 * 4;           // [wg][row] support size n
@@ -58,8 +65,10 @@ struct Cfg {
 struct Barriers {
   uint64_t q_full;
   uint64_t s_full[2], s_empty[2];
-  uint64_t in_full[4], in_empty[4];
-  uint64_t sweep_done, decided;
+  uint64_t in_full[6], in_empty[6];  // K ring: rows landed / S = Q K^T of the visit completed
+  uint64_t v_full[2], v_empty[2];    // V ring: rows landed / O += P V of the visit completed
+  uint64_t sweep_done;  // all statistics of the sweep are in shared memory
+  uint64_t decided;     // every row has moved its threshold and said whether it needs another sweep
   uint64_t o_done;
   uint32_t tmem_base;
   int abort_flag;
@@ -67,8 +76,39 @@ struct Barriers {
 };
 
 struct Maps {
-  CUtensorMap q, k, v;
+  CUtensorMap q;
+  CUtensorMap k16, k128, v16, v128;  // K and V in boxes of 16 and of 128 rows
 };
+
+// A round's descriptor as loaded (nothing is computed from it here, so that the loads of the next
+// round's descriptor stay in flight while the current round is worked on) ...
+struct RawRound {
+  uint32_t info;
+  int4 a, b;
+};
+__device__ __forceinline__ RawRound load_round(const int32_t *round_rows, const uint8_t *round_info, int t) {
+  RawRound r;
+  r.info = __ldg(round_info + t);
+  r.a = __ldg(reinterpret_cast<const int4 *>(round_rows + (size_t)t * 8));
+  r.b = __ldg(reinterpret_cast<const int4 *>(round_rows + (size_t)t * 8) + 1);
+  return r;
+}
+// ... and decoded: its groups and whether they are eight adjacent ones (one box of 128 rows brings them).
+struct Round {
+  int ng;
+  bool run;
+  int rows[8];
+};
+__device__ __forceinline__ Round decode_round(const RawRound &r) {
+  Round rd;
+  rd.ng = (int)(r.info & 15u);
+  rd.rows[0] = r.a.x; rd.rows[1] = r.a.y; rd.rows[2] = r.a.z; rd.rows[3] = r.a.w;
+  rd.rows[4] = r.b.x; rd.rows[5] = r.b.y; rd.rows[6] = r.b.z; rd.rows[7] = r.b.w;
+  rd.run = rd.ng == 8;
+#pragma unroll
+  for (int q = 1; q < 8; ++q) rd.run = rd.run && rd.rows[q] == rd.rows[0] + 16 * q;
+  return rd;
+}
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                               unsigned *err) {
@@ -84,6 +124,13 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
 
 __device__ __forceinline__ bool last_follows(const Barriers *bars, int s) {
   return s >= 1 && (s >= kMaxNewton || *reinterpret_cast<const volatile int *>(&bars->more[s]) == 0);
+}
+
+// v when sel < 0, -inf otherwise (one select instruction on the sign of an integer).
+__device__ __forceinline__ float keep_if_negative(float v, int sel) {
+  float d;
+  asm("slct.f32.s32 %0, %1, %2, %3;" : "=f"(d) : "f"(-CUDART_INF_F), "f"(v), "r"(sel));
+  return d;
 }
 
 template <bool kF16>
@@ -107,9 +154,9 @@ __device__ __forceinline__ float2 unpack2(uint32_t v) {
 
 template <int D, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
-fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, const int32_t *__restrict__ row_ptr,
-                  const int32_t *__restrict__ col_idx, const uint8_t *__restrict__ flags,
-                  const uint32_t *__restrict__ bitmap, int BH, int H, int Lq, int n_qt, float half_scale,
+fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, const int32_t *__restrict__ round_ptr,
+                  const int32_t *__restrict__ round_rows, const uint8_t *__restrict__ round_info,
+                  const uint32_t *__restrict__ round_bitmap, int BH, int H, int Lq, int n_qt, float half_scale,
                   unsigned *err) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
@@ -124,8 +171,8 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
   const int qt = n_qt - 1 - (int)(blockIdx.x / BH);  // late query tiles (the longest list rows when causal) first
   const int h = bh % H;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int t0 = row_ptr[h * n_qt + qt];
-  const int T = row_ptr[h * n_qt + qt + 1] - t0;  // kept tiles of this query tile: visits per sweep
+  const int t0 = round_ptr[h * n_qt + qt];
+  const int T = round_ptr[h * n_qt + qt + 1] - t0;  // rounds of this query tile: visits per sweep
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
@@ -137,8 +184,12 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
       mbar_init(&bars->in_full[s], 1);
       mbar_init(&bars->in_empty[s], 1);
     }
+    for (int s = 0; s < C::kVStages; ++s) {
+      mbar_init(&bars->v_full[s], 1);
+      mbar_init(&bars->v_empty[s], 1);
+    }
     mbar_init(&bars->sweep_done, kNormThreads);
-    mbar_init(&bars->decided, kNormThreads);
+    mbar_init(&bars->decided, kNormThreads + 2);  // + the copy and product threads, which run ahead of it
     mbar_init(&bars->o_done, 1);
     bars->abort_flag = 0;
     for (int s = 0; s < kMaxNewton + 2; ++s) bars->more[s] = 0;
@@ -167,90 +218,151 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
     }
   } else if (warp == 8) {
     // ------------------------------------------------------------ TMA producer
+    // K of visit v goes to stage v % kStages of its ring; V of the j-th visit of the last sweep to stage
+    // j % kVStages of its own.  A sweep that is not the last is always followed by another, so the K
+    // rows of the first visits of the next sweep are copied before the rows have decided whether that
+    // sweep is the last one: the decision costs no copy latency.
     if (lane == 0) {
       prefetch_tensormap(&maps.q);
-      prefetch_tensormap(&maps.k);
-      prefetch_tensormap(&maps.v);
+      prefetch_tensormap(&maps.k16);
+      prefetch_tensormap(&maps.k128);
+      prefetch_tensormap(&maps.v16);
+      prefetch_tensormap(&maps.v128);
       mbar_arrive_expect_tx(&bars->q_full, C::kTileBytes);
 #pragma unroll
       for (int s = 0; s < C::kSub; ++s) tma_load_3d(smem + s * kSubBytes, &maps.q, &bars->q_full, 64 * s, qt * kTile, bh);
-      int v = 0;
-      bool last = false, ok = true;
-      int kt_next = __ldg(col_idx + t0);
-      for (int sw = 0; ok; ++sw) {
-        for (int vv = 0; vv < T; ++vv, ++v) {
-          const int st = v % C::kStages;
-          const uint32_t ph = (uint32_t)(v / C::kStages) & 1u;
-          const int kt = kt_next;
-          kt_next = __ldg(col_idx + t0 + (vv + 1 == T ? 0 : vv + 1));
-          if (!wait_or_abort(&bars->in_empty[st], ph ^ 1u, abort_flag, err)) { ok = false; break; }
-          unsigned char *k_s = smem + C::kKOffset + st * C::kTileBytes, *v_s = smem + C::kVOffset + st * C::kTileBytes;
-          mbar_arrive_expect_tx(&bars->in_full[st], (last ? 2 : 1) * C::kTileBytes);
+      // rows of group q of a round land at rows [16 q, 16 q + 16) of the stage: 2048 bytes per group and half
+      auto copy_rows = [&](const Round &rd, unsigned char *dst, const CUtensorMap *m16, const CUtensorMap *m128,
+                           uint64_t *bar) {
+        mbar_arrive_expect_tx(bar, (uint32_t)(rd.ng * 2048 * C::kSub));
+        if (rd.run) {
 #pragma unroll
-          for (int s = 0; s < C::kSub; ++s) {
-            tma_load_3d(k_s + s * kSubBytes, &maps.k, &bars->in_full[st], 64 * s, kt * kTile, bh);
-            if (last) tma_load_3d(v_s + s * kSubBytes, &maps.v, &bars->in_full[st], 64 * s, kt * kTile, bh);
-          }
+          for (int s = 0; s < C::kSub; ++s) tma_load_3d(dst + s * kSubBytes, m128, bar, 64 * s, rd.rows[0], bh);
+        } else {
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            if (q < rd.ng) {
+#pragma unroll
+              for (int s = 0; s < C::kSub; ++s) tma_load_3d(dst + s * kSubBytes + q * 2048, m16, bar, 64 * s, rd.rows[q], bh);
+            }
         }
-        if (!ok || last) break;
+      };
+      int v = 0;        // visits whose K copy has been issued
+      int v_loads = 0;  // V copies issued
+      bool ok = true;
+      RawRound next = load_round(round_rows, round_info, t0);  // rounds are visited in order, again and again
+      int vv_next = 0;
+      auto copy_k = [&]() -> bool {
+        const Round rd = decode_round(next);
+        vv_next = vv_next + 1 == T ? 0 : vv_next + 1;
+        next = load_round(round_rows, round_info, t0 + vv_next);
+        const int st = v % C::kStages;
+        if (!wait_or_abort(&bars->in_empty[st], ((uint32_t)(v / C::kStages) & 1u) ^ 1u, abort_flag, err)) return false;
+        copy_rows(rd, smem + C::kKOffset + st * C::kTileBytes, &maps.k16, &maps.k128, &bars->in_full[st]);
+        ++v;
+        return true;
+      };
+      auto copy_v = [&](int vv) -> bool {  // V of round vv, the v_loads-th visit of the last sweep
+        const int st = v_loads % C::kVStages;
+        const Round rd = decode_round(load_round(round_rows, round_info, t0 + vv));
+        if (!wait_or_abort(&bars->v_empty[st], ((uint32_t)(v_loads / C::kVStages) & 1u) ^ 1u, abort_flag, err)) return false;
+        copy_rows(rd, smem + C::kVOffset + st * C::kTileBytes, &maps.v16, &maps.v128, &bars->v_full[st]);
+        ++v_loads;
+        return true;
+      };
+      const int n_ahead = T < C::kStages ? T : C::kStages;
+      for (int vv = 0; vv < T && ok; ++vv) ok = copy_k();  // sweep 0
+      for (int sw = 0; ok; ++sw) {
+        // sweep sw is issued and is not the last: the head of sweep sw + 1, before the decision
+        for (int vv = 0; vv < n_ahead && ok; ++vv) ok = copy_k();
+        if (!ok) break;
+        // (a participant of the barrier: a short sweep could otherwise complete the next phase
+        // before this thread has seen this one)
+        mbar_arrive(&bars->decided);
         if (!wait_or_abort(&bars->decided, (uint32_t)sw & 1u, abort_flag, err)) break;
-        last = last_follows(bars, sw);
+        const bool last = last_follows(bars, sw);
+        for (int vv = 0; vv < T && ok; ++vv) {
+          if (vv >= n_ahead) ok = copy_k();
+          if (ok && last) ok = copy_v(vv);
+        }
+        if (last) break;
       }
       if (*abort_flag) {  // winding down: let the copies in flight land (bounded)
         mbar_wait(&bars->q_full, 0u, kMaxPolls);
         for (int j = max(0, v - C::kStages); j < v; ++j)
           mbar_wait(&bars->in_full[j % C::kStages], (uint32_t)(j / C::kStages) & 1u, kMaxPolls);
+        for (int j = max(0, v_loads - C::kVStages); j < v_loads; ++j)
+          mbar_wait(&bars->v_full[j % C::kVStages], (uint32_t)(j / C::kVStages) & 1u, kMaxPolls);
       }
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
+    // S = Q K^T of the first two visits of the next sweep is issued before the decision as well
+    // (S is double-buffered).
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, 128, false, false, kF16);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true, kF16);
       const uint32_t q_addr = smem_u32(smem), k_addr = smem_u32(smem + C::kKOffset), v_addr = smem_u32(smem + C::kVOffset);
-      bool last = false, ok = wait_or_abort(&bars->q_full, 0u, abort_flag, err);
-      int v = 0;
-      // O += P V of visit u (last sweep): P of the visit is in S[u & 1] once the normalising threads
-      // have arrived; afterwards the visit's stage (K and V) is free
-      auto issue_pv = [&](int u, bool first) -> bool {
-        const int sb = u & 1, su = u % C::kStages;
+      bool ok = wait_or_abort(&bars->q_full, 0u, abort_flag, err);
+      int v = 0;  // visits whose S has been issued
+      auto ng_of = [&](int vv) { return (int)(__ldg(round_info + t0 + vv) & 15u); };
+      uint32_t info_next = __ldg(round_info + t0);  // used one visit later: the load stays in flight
+      int vv_next = 0;
+      auto issue_qk = [&]() -> bool {
+        const int st = v % C::kStages, buf = v & 1;
+        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * (int)(info_next & 15u), false, false, kF16);
+        vv_next = vv_next + 1 == T ? 0 : vv_next + 1;
+        info_next = __ldg(round_info + t0 + vv_next);
+        if (!wait_or_abort(&bars->in_full[st], (uint32_t)(v / C::kStages) & 1u, abort_flag, err)) return false;
+        // S[buf] was read (and, in the last sweep, its P consumed by a product issued earlier by
+        // this thread: products execute in issue order) two visits ago
+        if (!wait_or_abort(&bars->s_empty[buf], ((uint32_t)(v >> 1) & 1u) ^ 1u, abort_flag, err)) return false;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const int sub = ks / 4, o = (ks % 4) * 32;
+          mma_ss(tmem + 128 * buf, smem_desc_sw128(q_addr + sub * kSubBytes + o, 16, 1024),
+                 smem_desc_sw128(k_addr + st * C::kTileBytes + sub * kSubBytes + o, 16, 1024), idesc_qk, ks > 0);
+        }
+        mma_commit(&bars->in_empty[st]);
+        mma_commit(&bars->s_full[buf]);
+        ++v;
+        return true;
+      };
+      // O += P V of visit u = round j of the last sweep: P is in S[u & 1] once the normalising
+      // threads have arrived; one contraction step of 16 keys per group; then the V stage is free
+      auto issue_pv = [&](int u, int j) -> bool {
+        const int sb = u & 1, sv = j % C::kVStages, ng_u = ng_of(j);
+        if (!wait_or_abort(&bars->v_full[sv], (uint32_t)(j / C::kVStages) & 1u, abort_flag, err)) return false;
         if (!wait_or_abort(&bars->s_empty[sb], (uint32_t)(u >> 1) & 1u, abort_flag, err)) return false;
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          mma_ts(tmem + 256, tmem + 128 * sb + 32 * (ks >> 1) + 8 * (ks & 1),
-                 smem_desc_sw128(v_addr + su * C::kTileBytes + ks * 2048, kSubBytes, 1024), idesc_pv,
-                 (first && ks == 0) ? 0u : 1u);
-        mma_commit(&bars->in_empty[su]);
+          if (ks < ng_u)
+            mma_ts(tmem + 256, tmem + 128 * sb + 32 * (ks >> 1) + 8 * (ks & 1),
+                   smem_desc_sw128(v_addr + sv * C::kTileBytes + ks * 2048, kSubBytes, 1024), idesc_pv,
+                   (j == 0 && ks == 0) ? 0u : 1u);
+        mma_commit(&bars->v_empty[sv]);
         return true;
       };
+      const int n_ahead = T < 2 ? T : 2;
+      for (int vv = 0; vv < T && ok; ++vv) ok = issue_qk();  // sweep 0
       for (int sw = 0; ok; ++sw) {
-        for (int vv = 0; vv < T; ++vv, ++v) {
-          const int st = v % C::kStages;
-          const uint32_t ph = (uint32_t)(v / C::kStages) & 1u;
-          const int buf = v & 1;
-          if (!wait_or_abort(&bars->in_full[st], ph, abort_flag, err)) { ok = false; break; }
-          // S[buf] was read (and, in the last sweep, its P consumed by a product issued earlier by
-          // this thread: products execute in issue order) two visits ago
-          if (!wait_or_abort(&bars->s_empty[buf], ((uint32_t)(v >> 1) & 1u) ^ 1u, abort_flag, err)) { ok = false; break; }
-          tc_fence_after_sync();
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const int sub = ks / 4, o = (ks % 4) * 32;
-            mma_ss(tmem + 128 * buf, smem_desc_sw128(q_addr + sub * kSubBytes + o, 16, 1024),
-                   smem_desc_sw128(k_addr + st * C::kTileBytes + sub * kSubBytes + o, 16, 1024), idesc_qk, ks > 0);
-          }
-          if (!last) mma_commit(&bars->in_empty[st]);
-          mma_commit(&bars->s_full[buf]);
-          if (last && vv > 0 && !issue_pv(v - 1, vv == 1)) { ok = false; break; }
-        }
+        const int v_head = v;
+        for (int vv = 0; vv < n_ahead && ok; ++vv) ok = issue_qk();
         if (!ok) break;
-        if (last) {
-          if (issue_pv(v - 1, T == 1)) mma_commit(&bars->o_done);
+        mbar_arrive(&bars->decided);
+        if (!wait_or_abort(&bars->decided, (uint32_t)sw & 1u, abort_flag, err)) break;
+        if (!last_follows(bars, sw)) {
+          for (int vv = n_ahead; vv < T && ok; ++vv) ok = issue_qk();
+        } else {
+          // visit by visit: S of the visit (unless issued above), then O += P V of the one before
+          for (int vv = 0; vv < T && ok; ++vv) {
+            if (vv >= n_ahead) ok = issue_qk();
+            if (ok && vv > 0) ok = issue_pv(v_head + vv - 1, vv - 1);
+          }
+          if (ok && issue_pv(v_head + T - 1, T - 1)) mma_commit(&bars->o_done);
           break;
         }
-        if (!wait_or_abort(&bars->decided, (uint32_t)sw & 1u, abort_flag, err)) break;
-        last = last_follows(bars, sw);
       }
     }
   } else {
@@ -264,15 +376,17 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
     float *my_tau = taus + wg * 128 + r;
     float cnt = 0.f;
 
-    // kept-entry bits of this thread's 64 columns, fetched one visit ahead
-    auto fetch = [&](int vv, bool &full, uint2 &bits) {
+    // kept-entry bits of this thread's 64 columns of the round (0 for the columns of unused groups),
+    // fetched one visit ahead
+    // (raw: nothing is computed from the loaded values before the visit that uses them)
+    auto fetch = [&](int vv, uint32_t &info, uint2 &bits) {
       const int t = t0 + vv;
-      full = (__ldg(flags + t) & 1u) != 0u;
-      bits = __ldg(reinterpret_cast<const uint2 *>(bitmap + ((size_t)t * kTile + r) * 4 + 2 * wg));
+      info = __ldg(round_info + t);
+      bits = __ldg(reinterpret_cast<const uint2 *>(round_bitmap + ((size_t)t * kTile + r) * 4 + 2 * wg));
     };
-    bool full_next;
+    uint32_t info_next;
     uint2 bits_next;
-    fetch(0, full_next, bits_next);
+    fetch(0, info_next, bits_next);
 
     int v = 0;
     bool last = false, ok = true;
@@ -284,9 +398,9 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
       cnt = 0.f;
       for (int vv = 0; vv < T && ok; ++vv, ++v) {
         const int buf = v & 1;
-        const bool full = full_next;
+        const bool full = (info_next & 0x80u) != 0u;  // every entry of the round is kept
         const uint2 bits = bits_next;
-        fetch(vv + 1 == T ? 0 : vv + 1, full_next, bits_next);
+        fetch(vv + 1 == T ? 0 : vv + 1, info_next, bits_next);
         ok = wait_or_abort(&bars->s_full[buf], (uint32_t)(v >> 1) & 1u, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
@@ -298,12 +412,13 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
           tmem_wait_ld();
           const uint32_t w = c == 0 ? bits.x : bits.y;
           float t[32];  // x_j = scale * q.k_j / 2, -inf for pruned entries
-          if (full) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) t[e] = __uint_as_float(x[e]) * half_scale;
-          } else {
+          for (int e = 0; e < 32; e += 2)
+            ffma2(t[e], t[e + 1], __uint_as_float(x[e]), __uint_as_float(x[e + 1]), half_scale, 0.f, 0.f);
+          if (!full) {
+            // bit e of w moved to the sign position selects between the score and -inf
 #pragma unroll
-            for (int e = 0; e < 32; ++e) t[e] = (w >> e) & 1u ? __uint_as_float(x[e]) * half_scale : -CUDART_INF_F;
+            for (int e = 0; e < 32; ++e) t[e] = keep_if_negative(t[e], (int)(w << (31 - e)));
           }
           if (kind == 0) {
             float m0 = st.x, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
@@ -425,8 +540,9 @@ cudaError_t launch(const Maps &maps, const ap_tiles &t, void *O, int B, int H, i
   auto kern = fwd_entmax_kernel<D, kF16>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
-  kern<<<B * H * t.n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(maps, static_cast<uint16_t *>(O), t.row_ptr, t.col_idx,
-                                                           t.flags, t.bitmap, B * H, H, Lq, t.n_qt, 0.5f * scale, err);
+  kern<<<B * H * t.n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(maps, static_cast<uint16_t *>(O), t.round_ptr, t.round_rows,
+                                                           t.round_info, t.round_bitmap, B * H, H, Lq, t.n_qt,
+                                                           0.5f * scale, err);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -438,8 +554,9 @@ cudaError_t launch_fwd_entmax_tc(const void *Q, const void *K, const void *V, co
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   Maps maps;
-  if (!make_tile_map_bf16(&maps.q, Q, B * H, Lq, d) || !make_tile_map_bf16(&maps.k, K, B * H, Lk, d) ||
-      !make_tile_map_bf16(&maps.v, V, B * H, Lk, d))
+  if (!make_tile_map_bf16(&maps.q, Q, B * H, Lq, d) || !make_tile_map_bf16(&maps.k16, K, B * H, Lk, d, 16) ||
+      !make_tile_map_bf16(&maps.k128, K, B * H, Lk, d, 128) || !make_tile_map_bf16(&maps.v16, V, B * H, Lk, d, 16) ||
+      !make_tile_map_bf16(&maps.v128, V, B * H, Lk, d, 128))
     return cudaErrorUnknown;
   if (d == 64)
     return f16 ? launch<64, true>(maps, t, O, B, H, Lq, scale, err, s) : launch<64, false>(maps, t, O, B, H, Lq, scale, err, s);
