@@ -405,7 +405,7 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
         if (!ok) break;
         tc_fence_after_sync();
         float psum0 = 0.f, psum1 = 0.f;
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < 2; ++c) {
           uint32_t x[32];
           tmem_ld32(tmem + 128 * buf + 64 * wg + 32 * c + lane_addr, x);
