@@ -12,6 +12,7 @@
  *                          Section 3.1, softmax(Q K^T / sqrt(d_k)).
  *   oracle_build_mask      Eq. 2 read as an exact top-k selection per head.
  *   oracle_build_mask_layer  Eq. 2 with one threshold for all heads of the layer.
+ *   oracle_build_mask_ties   Eq. 2 with its strict inequality: ties with the threshold all stay.
  *   oracle_mask_to_tiles   the 128x128 tile list + bitmaps (an encoding of the
  *                          mask of Eq. 2; no counterpart in the paper).
  *   oracle_attention_fwd   the masked attention equation of Section 3.2,
@@ -314,6 +315,57 @@ int oracle_build_mask_layer(const float *acc, int H, int Lq, int Lk, double keep
   for (int64_t r = 0; r < k; ++r) {
     mask[(size_t)e[r].index] = 1;
     nnz[e[r].index / ((int64_t)Lq * Lk)] += 1;
+  }
+  free(e);
+  return 0;
+}
+
+/*
+ * Eq. 2 with its strict inequality taken literally: an entry is pruned iff its average lies
+ * strictly BELOW the threshold, so every entry equal to the threshold stays and the kept count
+ * can exceed k.  The threshold tau is the value of the last entry the exact top-k above would
+ * keep (the k-th in the order forced first, value descending); when the forced entries alone
+ * fill k there is no threshold and only they are kept.
+ *   mask[h,i,j] = 1  iff  (i,j) is forced, or in the domain with acc[h,i,j] >= tau (as fp32)
+ * per_layer = 0: one population, k and tau per head; per_layer = 1: one for all heads together
+ * (the layer rule above).  nnz[h] = entries kept in head h.  Returns 0, or -1 on a failed allocation.
+ */
+int oracle_build_mask_ties(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal,
+                           int keep_diag, int per_layer, uint8_t *mask, int64_t *nnz) {
+  memset(mask, 0, (size_t)H * Lq * Lk);
+  int64_t n_valid = 0;
+  for (int i = 0; i < Lq; ++i) n_valid += row_domain_end(i, Lq, Lk, causal);
+  int heads_per_pop = per_layer ? H : 1, n_pop = per_layer ? 1 : H;
+  int64_t N = n_valid * heads_per_pop;
+  ap_entry *e = (ap_entry *)malloc(sizeof(ap_entry) * (size_t)(N > 0 ? N : 1));
+  if (!e) return -1;
+  for (int h = 0; h < H; ++h) nnz[h] = 0;
+  for (int pop = 0; pop < n_pop; ++pop) {
+    int64_t n = 0, n_forced = 0;
+    for (int hh = 0; hh < heads_per_pop; ++hh) {
+      int h = pop * heads_per_pop + hh;
+      for (int i = 0; i < Lq; ++i) {
+        int jend = row_domain_end(i, Lq, Lk, causal);
+        for (int j = 0; j < jend; ++j) {
+          e[n].value = acc[((size_t)h * Lq + i) * Lk + j];
+          e[n].forced = is_forced(i, j, Lq, Lk, causal, keep_diag);
+          e[n].index = ((int64_t)h * Lq + i) * Lk + j;
+          n_forced += e[n].forced;
+          ++n;
+        }
+      }
+    }
+    int64_t k = oracle_keep_count(N, n_forced, keep_frac);
+    qsort(e, (size_t)n, sizeof(ap_entry), entry_before);
+    int64_t kept = k;
+    if (k > n_forced) {
+      float tau = e[k - 1].value;
+      while (kept < n && e[kept].value >= tau) ++kept; /* sorted: the rest of the ties follow */
+    }
+    for (int64_t r = 0; r < kept; ++r) {
+      mask[(size_t)e[r].index] = 1;
+      nnz[e[r].index / ((int64_t)Lq * Lk)] += 1;
+    }
   }
   free(e);
   return 0;

@@ -185,6 +185,25 @@ def build_mask_layer(acc32, keep_frac: float, causal: bool = False, keep_diag: b
     return mask, nnz
 
 
+def build_mask_ties(acc32, keep_frac: float, causal: bool = False, keep_diag: bool = True, per_layer: bool = False):
+    """Eq. 2 with its strict inequality: the threshold is the exact top-k's last kept value and every entry
+    equal to it stays; returns (mask uint8 [H,Lq,Lk], nnz int64 [H])."""
+    acc32 = _f32(acc32)
+    H, Lq, Lk = acc32.shape
+    _check_domain(Lq, Lk, causal)
+    mask = np.zeros((H, Lq, Lk), dtype=np.uint8)
+    nnz = np.zeros((H,), dtype=np.int64)
+    lib = _load()
+    lib.oracle_build_mask_ties.restype = ctypes.c_int
+    rc = lib.oracle_build_mask_ties(
+        _p(acc32), H, Lq, Lk, ctypes.c_double(keep_frac), int(bool(causal)), int(bool(keep_diag)),
+        int(bool(per_layer)), _p(mask), _p(nnz),
+    )
+    if rc != 0:
+        raise MemoryError("oracle_build_mask_ties")
+    return mask, nnz
+
+
 def mask_to_tiles(mask):
     """Tile list of a mask: dict(row_ptr, col_idx, flags, bitmap) trimmed to the T non-empty tiles."""
     mask = np.ascontiguousarray(np.asarray(mask, dtype=np.uint8))

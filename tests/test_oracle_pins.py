@@ -881,3 +881,65 @@ def test_attention_entmax15_equals_row_wise_composition():
     sub = orc.attention_entmax15_rows(q, k, v, mask, rows)
     for r, (b, h, i) in enumerate(rows):
         np.testing.assert_allclose(sub[r], want[b, h, i], rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- Eq. 2 with ties kept
+
+
+@pytest.mark.parametrize("per_layer", [False, True])
+def test_ties_mask_is_a_threshold_on_the_kth_largest_value(per_layer):
+    """Without a domain restriction or forced entries the rule is one line of numpy: tau = the k-th largest
+    value of the population, mask = (acc >= tau).  Values on a coarse grid, so ties at tau are the rule."""
+    rng = np.random.default_rng(41)
+    H, Lq, Lk = 3, 9, 14
+    acc = (rng.integers(0, 12, size=(H, Lq, Lk)) / 8.0).astype(np.float32)
+    for keep in (0.1, 0.37, 0.8, 1.0):
+        mask, nnz = orc.build_mask_ties(acc, keep, causal=False, keep_diag=False, per_layer=per_layer)
+        pops = [acc] if per_layer else [acc[h:h + 1] for h in range(H)]
+        want = []
+        for pop in pops:
+            k = orc.keep_count(pop.size, 0, keep)
+            tau = np.partition(pop.reshape(-1), pop.size - k)[pop.size - k]
+            want.append(pop >= tau)
+        want = np.concatenate(want, axis=0)
+        np.testing.assert_array_equal(mask.astype(bool), want)
+        np.testing.assert_array_equal(nnz, want.reshape(H, -1).sum(1))
+        assert nnz.sum() >= (orc.keep_count(acc.size, 0, keep) if per_layer else H * orc.keep_count(Lq * Lk, 0, keep))
+
+
+@pytest.mark.parametrize("causal,Lq,Lk", [(True, 11, 11), (True, 6, 13), (False, 8, 8)])
+@pytest.mark.parametrize("per_layer", [False, True])
+def test_ties_mask_against_the_exact_count_mask(causal, Lq, Lk, per_layer):
+    """With a domain and forced entries: the exact-count mask (pinned above) fixes tau as its smallest kept
+    value that is not forced; the ties rule keeps the forced entries and everything in the domain >= tau.
+    Distinct values: the two masks coincide."""
+    rng = np.random.default_rng(43)
+    H = 2
+    exact = orc.build_mask_layer if per_layer else orc.build_mask
+    dom = np.tril(np.ones((Lq, Lk), dtype=bool), Lk - Lq) if causal else np.ones((Lq, Lk), dtype=bool)
+    forced = np.zeros((Lq, Lk), dtype=bool)
+    forced[np.arange(Lq), np.arange(Lq) + Lk - Lq] = True
+    acc = (rng.integers(0, 6, size=(H, Lq, Lk)) / 4.0).astype(np.float32)
+    for keep in (0.15, 0.5, 0.9):
+        base, _ = exact(acc, keep, causal=causal, keep_diag=True)
+        mask, nnz = orc.build_mask_ties(acc, keep, causal=causal, keep_diag=True, per_layer=per_layer)
+        want = np.zeros_like(base, dtype=bool)
+        groups = [slice(0, H)] if per_layer else [slice(h, h + 1) for h in range(H)]
+        for g in groups:
+            kept_free = base[g].astype(bool) & ~forced[None]
+            w = np.broadcast_to(forced[None], base[g].shape).copy()
+            if kept_free.any():
+                w |= (acc[g] >= acc[g][kept_free].min()) & dom[None]
+            want[g] = w
+        np.testing.assert_array_equal(mask.astype(bool), want)
+        np.testing.assert_array_equal(nnz, want.reshape(H, -1).sum(1))
+        assert np.all(mask >= base)                                   # a superset of the exact-count mask
+    distinct = rng.permutation(H * Lq * Lk).reshape(H, Lq, Lk).astype(np.float32)
+    for keep in (0.2, 0.6):
+        base, n0 = exact(distinct, keep, causal=causal, keep_diag=True)
+        mask, n1 = orc.build_mask_ties(distinct, keep, causal=causal, keep_diag=True, per_layer=per_layer)
+        np.testing.assert_array_equal(mask, base)
+        np.testing.assert_array_equal(n0, n1)
+    flat = np.full((H, Lq, Lk), 0.5, dtype=np.float32)                # all equal: nothing is strictly below
+    mask, _ = orc.build_mask_ties(flat, 0.3, causal=causal, keep_diag=True, per_layer=per_layer)
+    np.testing.assert_array_equal(mask.astype(bool), np.broadcast_to(dom, mask.shape))
