@@ -196,6 +196,22 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Both rules with Eq. 2's strict inequality taken literally.  flags is a sum of
+ *   AP_MASK_PER_LAYER  one selection over all heads (ap_build_mask_layer) instead of one per head
+ *   AP_MASK_KEEP_TIES  an entry is pruned iff its average lies strictly below the threshold, the
+ *                      value of the last entry the exact top-k would keep: every entry equal to
+ *                      it stays, so a head (the layer) may keep more than k entries.  Where the
+ *                      forced entries alone fill k there is no threshold and only they are kept.
+ * With flags = 0 this is ap_build_mask.  nnz_per_head[h] = entries kept in head h.  Other
+ * arguments, outputs and errors as above; unknown flag bits are AP_ERR_INVALID_ARG.
+ */
+#define AP_MASK_PER_LAYER 1
+#define AP_MASK_KEEP_TIES 2
+ap_status ap_build_mask_ex(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal,
+                           int keep_diag, int flags, uint8_t *mask, ap_tiles *tiles,
+                           int64_t *nnz_per_head, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Derivative of ap_sparse_attention_fwd with respect to Q, K and V (retraining under the
  * mask, step 4 of the paper's procedure, differentiates exactly this function).  With
  * S = scale*Q.K^T, P = softmax of S over the kept entries of a row, O = P.V and dO given:

@@ -58,6 +58,7 @@ def _load() -> ctypes.CDLL:
         "ap_accumulate_attention_entmax15": (i, [vp, vp, vp, vp, i, i, i, i, i, i, i, f, vp]),
         "ap_build_mask": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_build_mask_layer": (i, [vp, i, i, i, d, i, i, vp, tp, vp, vp, sz, vp]),
+        "ap_build_mask_ex": (i, [vp, i, i, i, d, i, i, i, vp, tp, vp, vp, sz, vp]),
         "ap_random_scores": (i, [vp, i, i, i, ctypes.c_uint64, vp]),
         "ap_pool_scores": (i, [vp, i, i, i, i, i, vp, vp]),
         "ap_expand_block_mask": (i, [vp, i, i, i, i, i, vp, vp]),
@@ -79,7 +80,7 @@ def _load() -> ctypes.CDLL:
 
 lib = _load()
 EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
-           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_accumulate_attention_entmax15", "ap_build_mask", "ap_build_mask_layer", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
+           "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_accumulate_attention_entmax15", "ap_build_mask", "ap_build_mask_layer", "ap_build_mask_ex", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd", "ap_sparse_attention_entmax15_fwd",
            "ap_sparse_attention_fwd_host", "ap_sparse_attention_bwd_workspace_bytes", "ap_sparse_attention_bwd",
            "ap_device_status")
@@ -233,6 +234,23 @@ def ap_build_mask_layer(acc, keep_frac, causal=False, keep_diag=True, mask=None,
                         nnz_per_head=None, workspace=None, stream=None) -> None:
     _build_mask(lib.ap_build_mask_layer, "ap_build_mask_layer", acc, keep_frac, causal, keep_diag, mask, tiles,
                 nnz_per_head, workspace, stream)
+
+
+AP_MASK_PER_LAYER, AP_MASK_KEEP_TIES = 1, 2
+
+
+def ap_build_mask_ex(acc, keep_frac, causal=False, keep_diag=True, flags=0, mask=None, tiles: Tiles | None = None,
+                     nnz_per_head=None, workspace=None, stream=None) -> None:
+    _dev(acc, "acc")
+    H, Lq, Lk = acc.shape
+    if acc.dtype != torch.float32:
+        raise ValueError("acc must be float32")
+    if workspace is None:
+        workspace = torch.empty(ap_build_mask_workspace_bytes(H, Lq, Lk), dtype=torch.uint8, device=acc.device)
+    _check(lib.ap_build_mask_ex(_ptr(acc), H, Lq, Lk, float(keep_frac), int(bool(causal)), int(bool(keep_diag)),
+                                int(flags), _ptr(mask), ctypes.byref(tiles.c) if tiles is not None else None,
+                                _ptr(nnz_per_head), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "ap_build_mask_ex")
 
 
 def ap_pool_scores(acc, block: int, causal=False, pooled=None, stream=None):

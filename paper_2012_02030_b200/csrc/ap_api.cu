@@ -159,7 +159,7 @@ ap_status ap_accumulate_attention_entmax15(float *acc, const void *Q, const void
 namespace {
 ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
                           uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
-                          size_t workspace_bytes, void *stream, int per_layer) {
+                          size_t workspace_bytes, void *stream, int per_layer, int keep_ties = 0) {
   if (!acc || !aligned16(acc) || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq)) return AP_ERR_INVALID_ARG;
   if (!(keep_frac > 0.0) || !(keep_frac <= 1.0)) return AP_ERR_INVALID_ARG;
   if (mask && !aligned16(mask)) return AP_ERR_INVALID_ARG;
@@ -184,6 +184,7 @@ ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_f
   a.causal = causal ? 1 : 0;
   a.keep_diag = keep_diag ? 1 : 0;
   a.per_layer = per_layer;
+  a.keep_ties = keep_ties;
   // population of one selection: a head's domain, or the union of the heads' domains
   const int64_t heads = per_layer ? H : 1;
   const int64_t n_valid = domain_size(Lq, Lk, a.causal) * heads;
@@ -216,6 +217,15 @@ ap_status ap_build_mask_layer(const float *acc, int H, int Lq, int Lk, double ke
                               size_t workspace_bytes, void *stream) {
   return build_mask_impl(acc, H, Lq, Lk, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head, workspace,
                          workspace_bytes, stream, 1);
+}
+
+ap_status ap_build_mask_ex(const float *acc, int H, int Lq, int Lk, double keep_frac, int causal, int keep_diag,
+                           int flags, uint8_t *mask, ap_tiles *tiles, int64_t *nnz_per_head, void *workspace,
+                           size_t workspace_bytes, void *stream) {
+  if (flags & ~(AP_MASK_PER_LAYER | AP_MASK_KEEP_TIES)) return AP_ERR_INVALID_ARG;
+  return build_mask_impl(acc, H, Lq, Lk, keep_frac, causal, keep_diag, mask, tiles, nnz_per_head, workspace,
+                         workspace_bytes, stream, (flags & AP_MASK_PER_LAYER) ? 1 : 0,
+                         (flags & AP_MASK_KEEP_TIES) ? 1 : 0);
 }
 
 namespace {

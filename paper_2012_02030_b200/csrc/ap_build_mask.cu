@@ -794,9 +794,10 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
 // element mask, the tile's bitmap and popcount into the staging area.  Values are
 // compared with the threshold as floats (the same order as their keys).  per_layer:
 // all heads share selection 0, ties are ordered by (h*Lq + i)*Lk + j, and the
-// tiles' popcounts are added up into nnz[h].
+// tiles' popcounts are added up into nnz[h].  keep_ties: every entry equal to the threshold is
+// kept (no ranking), and the popcounts are added up as well (the count is not known beforehand).
 __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_qt, int n_kt,
-                                                   int causal, int diag, int per_layer,
+                                                   int causal, int diag, int per_layer, int keep_ties,
                                                    const SelectState *__restrict__ state,
                                                    const uint32_t *__restrict__ tie_prefix,
                                                    uint8_t *__restrict__ mask, uint32_t *__restrict__ stage_bitmap,
@@ -834,7 +835,7 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   EmitSel sel;
   sel.thr_f = float_of_key(st.thr);
   sel.ties_kept = st.ties_kept;
-  sel.all_ties = st.all_ties_kept != 0u;
+  sel.all_ties = st.all_ties_kept != 0u || keep_ties != 0;
   sel.have_cut = st.have_cut != 0u;
   sel.tie_cut = st.tie_cut;
   sel.first_row = per_layer ? (uint32_t)h * (uint32_t)Lq : 0u;
@@ -852,7 +853,7 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
   if (threadIdx.x == 0) {
     const int total = warp_count[0] + warp_count[1] + warp_count[2] + warp_count[3];
     if (stage_count) stage_count[tile] = total;
-    if (per_layer && nnz && total)
+    if ((per_layer || keep_ties) && nnz && total)
       atomicAdd(reinterpret_cast<unsigned long long *>(nnz + h), (unsigned long long)total);
   }
 }
@@ -892,9 +893,10 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   const int rows = a.per_layer ? a.H * a.Lq : a.Lq;
   const int period = a.Lq;
   cudaError_t e;
-  // per head nnz = k; per layer the emit pass counts it
+  // per head nnz = k; per layer, or with all ties kept, the emit pass counts it
+  const bool count_nnz = a.per_layer || a.keep_ties;
   init_state_kernel<<<ceil_div(max(n_sel * kBins, a.H), 256), 256, 0, s>>>(
-      sc.state, sc.hist, n_sel, (unsigned long long)a.k_rest, a.H, a.per_layer ? 0ll : (long long)a.k, a.nnz);
+      sc.state, sc.hist, n_sel, (unsigned long long)a.k_rest, a.H, count_nnz ? 0ll : (long long)a.k, a.nnz);
   count_launches(1);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   // enough CTAs per selection to fill the GPU, at most one warp-row each
@@ -940,16 +942,19 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
-    // both return at once for selections whose ties with the threshold are all kept
-    tie_count_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, n_kt, a.causal, diag, sc.state,
-                                               sc.tie_count);
-    count_launches(1);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    tie_scan_kernel<<<n_sel, 1024, 0, s>>>(sc.tie_count, rows * n_kt, sc.state);
-    count_launches(1);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if (!a.keep_ties) {  // the ties' ranks are needed only where some of them are pruned
+      // both return at once for selections whose ties with the threshold are all kept
+      tie_count_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, n_kt, a.causal, diag, sc.state,
+                                                 sc.tie_count);
+      count_launches(1);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      tie_scan_kernel<<<n_sel, 1024, 0, s>>>(sc.tie_count, rows * n_kt, sc.state);
+      count_launches(1);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
   }
-  emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer, sc.state,
+  emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer,
+                                                a.keep_ties, sc.state,
                                                 sc.tie_count, a.mask, a.stage_bitmap, a.stage_count, a.nnz);
   count_launches(1);
   return cudaGetLastError();

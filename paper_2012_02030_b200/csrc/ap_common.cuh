@@ -64,6 +64,7 @@ struct BuildMaskArgs {
   const float *acc;
   int H, Lq, Lk, causal, keep_diag;
   int per_layer;   // one selection over all heads instead of one per head
+  int keep_ties;   // every entry equal to the threshold is kept (the kept count may exceed k)
   int64_t k_rest;  // entries to select among the non-forced entries of the selection's population
   int64_t k;       // entries kept per selection (per head, or in the whole layer)
   uint8_t *mask;   // may be NULL

@@ -124,6 +124,15 @@ def test_accumulate_and_mask_reject_bad_arguments():
         a = list(base)
         a[2], a[5] = 9, 1  # causal with Lk < Lq
         assert g(*a) == ap.AP_ERR_INVALID_ARG
+    ex = ap.lib.ap_build_mask_ex  # flags: per layer = 1, keep ties = 2; anything else is refused
+    ok = [FAKE, 1, 8, 8, 0.5, 0, 1, 3, FAKE, ctypes.byref(t), FAKE, FAKE, ws, None]
+    for bad in (4, 8, -1):
+        a = list(ok); a[7] = bad
+        assert ex(*a) == ap.AP_ERR_INVALID_ARG
+    a = list(ok); a[12] = ws - 1
+    assert ex(*a) == ap.AP_ERR_WORKSPACE
+    a = list(ok); a[0] = None
+    assert ex(*a) == ap.AP_ERR_INVALID_ARG
     # one selection over the layer ranks ties by a 32-bit index over all heads
     big = [FAKE, 64, 8192, 8192, 0.5, 0, 1, FAKE, None, FAKE, FAKE, ap.ap_build_mask_workspace_bytes(64, 8192, 8192),
            None]

@@ -7,7 +7,7 @@ import pytest
 import torch
 
 from oracle import ap_oracle as orc
-from paper_2012_02030_b200 import inputs
+from paper_2012_02030_b200 import inputs, metrics
 from tests import parity_util as pu
 
 pytestmark = pytest.mark.gpu
@@ -93,6 +93,58 @@ def test_build_mask_random_values_with_ties(ap, shape, causal, keep_diag):
     for keep in (0.1, 0.5, 1.0):
         _check_build_mask(ap, acc, W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=causal, keep_diag=keep_diag,
                                                      keep_frac=keep))
+
+
+def _check_build_mask_ties(ap, acc32: np.ndarray, w, layer):
+    H, Lq, Lk = acc32.shape
+    mask = torch.full((H, Lq, Lk), 7, dtype=torch.uint8, device="cuda")  # poison: every byte must be written
+    nnz = torch.full((H,), -1, dtype=torch.int64, device="cuda")
+    tiles = ap.Tiles(H, Lq, Lk)
+    flags = ap.AP_MASK_KEEP_TIES | (ap.AP_MASK_PER_LAYER if layer else 0)
+    ap.ap_build_mask_ex(torch.from_numpy(acc32).cuda(), w.keep_frac, w.causal, w.keep_diag, flags, mask, tiles, nnz)
+    assert ap.ap_device_status() == ap.AP_OK
+    want_mask, want_nnz = orc.build_mask_ties(acc32, w.keep_frac, w.causal, w.keep_diag, per_layer=layer)
+    np.testing.assert_array_equal(nnz.cpu().numpy(), want_nnz)
+    np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
+    pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
+    return want_nnz
+
+
+@pytest.mark.parametrize("layer", [False, True])
+@pytest.mark.parametrize("causal,keep_diag", [(False, False), (True, True), (False, True)])
+@pytest.mark.parametrize("shape", [(3, 67, 67), (2, 300, 300), (2, 100, 260), (1, 5, 5)])
+def test_build_mask_keeping_all_ties(ap, shape, causal, keep_diag, layer):
+    """Eq. 2 with its strict inequality: entries equal to the threshold all stay."""
+    H, Lq, Lk = shape
+    if causal and Lk < Lq:
+        pytest.skip("the causal domain needs Lk >= Lq")
+    rng = np.random.default_rng(72)
+    acc = rng.random((H, Lq, Lk), dtype=np.float32)
+    acc[0].flat[::3] = 0.5                      # a third of head 0 ties at one value
+    acc[-1] = np.round(acc[-1] * 8) / 8         # 9 distinct values: the threshold is always tied
+    acc[0, 0, :3] = [-1.0, -0.0, 0.0]
+    more = 0
+    for keep in (1e-6, 0.1, 0.5, 1.0):
+        w = W["tiny"].scaled(H=H, Lq=Lq, Lk=Lk, causal=causal, keep_diag=keep_diag, keep_frac=keep)
+        nnz = _check_build_mask_ties(ap, acc, w, layer)
+        k = metrics.keep_count(w.n_valid * (H if layer else 1), w.n_forced * (H if layer else 1), keep)
+        more += int(nnz.sum() > (k if layer else k * H))
+    assert more > 0 or Lq < 8                   # the case is exercised: ties pushed the count past k
+    flags = ap.AP_MASK_KEEP_TIES | (ap.AP_MASK_PER_LAYER if layer else 0)
+    assert flags  # with flags = 0 the entry point is ap_build_mask: checked below
+
+
+def test_build_mask_ex_without_flags_is_build_mask(ap):
+    acc = np.random.default_rng(73).random((2, 130, 130), dtype=np.float32)
+    acc[1] = np.round(acc[1] * 4) / 4
+    dev = torch.from_numpy(acc).cuda()
+    for flags, want in ((0, orc.build_mask), (ap.AP_MASK_PER_LAYER, orc.build_mask_layer)):
+        mask = torch.empty((2, 130, 130), dtype=torch.uint8, device="cuda")
+        nnz = torch.empty((2,), dtype=torch.int64, device="cuda")
+        ap.ap_build_mask_ex(dev, 0.3, True, True, flags, mask, None, nnz)
+        want_mask, want_nnz = want(acc, 0.3, True, True)
+        np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
+        np.testing.assert_array_equal(nnz.cpu().numpy(), want_nnz)
 
 
 @pytest.mark.parametrize("shape", [(2, 100, 260), (1, 257, 31)])
