@@ -152,8 +152,8 @@ ap_status ap_accumulate_attention(float *acc, const void *Q, const void *K, cons
  * over the row's domain.  Entries outside the domain, and entries inside it that no sample
  * gives weight, keep their value.  tau is found in fp32 by solving the row's equation on the
  * support of a trial threshold and repeating until the step falls under 2e-6 max(1, |tau|).
- * Arguments, layout, ordering of the sum and error behaviour as ap_accumulate_attention,
- * except that dt must be AP_BF16 or AP_F16 (AP_ERR_UNSUPPORTED otherwise).
+ * (5e-7 for fp32 tensors, which run on the CUDA cores).
+ * Arguments, layout, ordering of the sum and error behaviour as ap_accumulate_attention.
  */
 ap_status ap_accumulate_attention_entmax15(float *acc, const void *Q, const void *K, const float *bias,
                                            int B, int H, int Lq, int Lk, int d, ap_dtype dt, int causal,
@@ -323,8 +323,9 @@ ap_status ap_sparse_attention_fwd(const void *Q, const void *K, const void *V,
  * (found in fp32 as in ap_accumulate_attention_entmax15, to a step under 2e-6 max(1, |tau|)); a row
  * without kept entries outputs exactly 0.  The weights are rounded to dt before they multiply V
  * and the row is divided by the sum of the rounded weights.  Follows the tile list's rounds
- * (round_ptr, round_rows, round_info, round_bitmap).  Arguments and error behaviour as ap_sparse_attention_fwd, except
- * that dt must be AP_BF16 or AP_F16 (AP_ERR_UNSUPPORTED otherwise).
+ * (round_ptr, round_rows, round_info, round_bitmap); fp32 tensors run on the CUDA cores over
+ * the stored tiles (row_ptr, col_idx, flags, bitmap), with fp32 weights and a step bound of
+ * 5e-7.  Arguments and error behaviour as ap_sparse_attention_fwd.
  */
 ap_status ap_sparse_attention_entmax15_fwd(const void *Q, const void *K, const void *V, const ap_tiles *tiles,
                                            void *O, int B, int H, int Lq, int Lk, int d, ap_dtype dt,

@@ -7,6 +7,14 @@
 // memory, then one warp per row takes the row maximum, the sum of exponentials
 // and adds the normalised row to the accumulator with coalesced read-modify-
 // writes.  Used for fp32 inputs, where tensor-core precision would not do.
+//
+// kEntmax: the same sum with 1.5-entmax as the normaliser (the section on sparse normalisation),
+// p_j = max(s_j / 2 - tau, 0)^2 with tau such that the row sums to 1.  The row's scores are in
+// shared memory, so the warp iterates on tau there: from max/2 - 1 (left of the root) to the
+// smaller root of the parabola of the current support, tau + (S2 - 1) / (S1 + sqrt(S1^2 - n (S2 - 1)))
+// with n, S1, S2 the support's size and its sums of (s_j/2 - tau) and of its square (Newton's
+// step (S2 - 1) / (2 S1) where the parabola has no root), until the step falls under
+// 5e-7 max(1, |tau|) (at most 30 steps).
 #include <math_constants.h>
 
 #include "ap_common.cuh"
@@ -39,7 +47,7 @@ __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16 *p, flo
   }
 }
 
-template <typename T, int D>
+template <typename T, int D, bool kEntmax>
 __global__ void __launch_bounds__(kThreads) accumulate_simt_kernel(float *__restrict__ acc, const T *__restrict__ Q,
                                                                    const T *__restrict__ K,
                                                                    const float *__restrict__ bias, int B, int H,
@@ -102,18 +110,47 @@ __global__ void __launch_bounds__(kThreads) accumulate_simt_kernel(float *__rest
       for (int j = lane; j < jend; j += 32) m = fmaxf(m, srow[j]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      float *arow = acc + ((size_t)h * Lq + i) * Lk;
+      if (kEntmax) {
+        float tau = 0.5f * m - 1.f;
+        for (int it = 0; it < 30; ++it) {
+          float n = 0.f, S1 = 0.f, S2 = 0.f;
+          for (int j = lane; j < jend; j += 32) {
+            const float u = fmaf(0.5f, srow[j], -tau);
+            if (u > 0.f) {
+              n += 1.f;
+              S1 += u;
+              S2 = fmaf(u, u, S2);
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {  // every lane ends with the same bits
+            n += __shfl_xor_sync(0xffffffffu, n, o);
+            S1 += __shfl_xor_sync(0xffffffffu, S1, o);
+            S2 += __shfl_xor_sync(0xffffffffu, S2, o);
+          }
+          const float disc = S1 * S1 - n * (S2 - 1.f);
+          const float step = S1 > 0.f ? (S2 - 1.f) / (S1 + (disc >= 0.f ? sqrtf(disc) : S1)) : 0.f;
+          tau += step;
+          if (fabsf(step) <= 5e-7f * fmaxf(1.f, fabsf(tau))) break;
+        }
+        for (int j = lane; j < jend; j += 32) {
+          const float u = fmaf(0.5f, srow[j], -tau);
+          if (u > 0.f) arow[j] += u * u;
+        }
+        continue;
+      }
       float z = 0.f;
       for (int j = lane; j < jend; j += 32) z += expf(srow[j] - m);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-      float *arow = acc + ((size_t)h * Lq + i) * Lk;
       for (int j = lane; j < jend; j += 32) arow[j] += expf(srow[j] - m) / z;
     }
     __syncthreads();
   }
 }
 
-template <typename T, int D>
+template <typename T, int D, bool kEntmax>
 cudaError_t launch(float *acc, const void *Q, const void *K, const float *bias, int B, int H, int Lq, int Lk,
                    int causal, float scale, cudaStream_t s) {
   // as many rows per CTA (up to 8) as the score rows allow in shared memory
@@ -122,7 +159,7 @@ cudaError_t launch(float *acc, const void *Q, const void *K, const float *bias, 
   while (rows > 1 && (size_t)(kRows * D + (size_t)rows * Lk) * sizeof(float) > budget) rows >>= 1;
   const size_t smem = (size_t)(kRows * D + (size_t)rows * Lk) * sizeof(float);
   if (smem > budget) return cudaErrorInvalidValue;
-  auto kern = accumulate_simt_kernel<T, D>;
+  auto kern = accumulate_simt_kernel<T, D, kEntmax>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(ceil_div(Lq, rows), H);
@@ -136,13 +173,17 @@ cudaError_t launch(float *acc, const void *Q, const void *K, const float *bias, 
 
 cudaError_t launch_accumulate_simt(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
                                    int Lq, int Lk, int d, ap_dtype dt, int causal, float scale,
-                                   cudaStream_t s) {
-  if (dt == AP_F32) {
-    return d == 64 ? launch<float, 64>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s)
-                   : launch<float, 128>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s);
+                                   cudaStream_t s, int entmax) {
+  if (entmax) {  // fp32 tensors only
+    return d == 64 ? launch<float, 64, true>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s)
+                   : launch<float, 128, true>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s);
   }
-  return d == 64 ? launch<__nv_bfloat16, 64>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s)
-                 : launch<__nv_bfloat16, 128>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s);
+  if (dt == AP_F32) {
+    return d == 64 ? launch<float, 64, false>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s)
+                   : launch<float, 128, false>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s);
+  }
+  return d == 64 ? launch<__nv_bfloat16, 64, false>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s)
+                 : launch<__nv_bfloat16, 128, false>(acc, Q, K, bias, B, H, Lq, Lk, causal, scale, s);
 }
 
 }  // namespace ap

@@ -148,11 +148,15 @@ ap_status ap_accumulate_attention_entmax15(float *acc, const void *Q, const void
     return AP_ERR_INVALID_ARG;
   if (B < 1 || !shape_ok(H, Lq, Lk) || (causal && Lk < Lq) || !(scale >= 0.f) || isinf(scale))
     return AP_ERR_INVALID_ARG;
-  if ((d != 64 && d != 128) || (dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
   if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
-  cudaError_t e = launch_accumulate_entmax_tc(acc, Q, K, bias, B, H, Lq, Lk, d, causal ? 1 : 0, dt == AP_F16 ? 1 : 0,
-                                              sc, static_cast<cudaStream_t>(stream));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = dt == AP_F32
+                      ? launch_accumulate_simt(acc, Q, K, bias, B, H, Lq, Lk, d, dt, causal ? 1 : 0, sc, s, 1)
+                      : launch_accumulate_entmax_tc(acc, Q, K, bias, B, H, Lq, Lk, d, causal ? 1 : 0,
+                                                    dt == AP_F16 ? 1 : 0, sc, s);
+  if (e == cudaErrorInvalidValue) return AP_ERR_UNSUPPORTED;  // key length beyond the shared-memory budget
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 
@@ -325,11 +329,12 @@ ap_status ap_sparse_attention_entmax15_fwd(const void *Q, const void *K, const v
   if ((int64_t)B * H * ceil_div(Lq, kTile) > (int64_t)0x7fffffff) return AP_ERR_INVALID_ARG;
   ap_status st = check_tiles(tiles, H, Lq, Lk, true);
   if (st != AP_OK) return st;
-  if ((d != 64 && d != 128) || (dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
+  if ((d != 64 && d != 128) || (dt != AP_F32 && dt != AP_BF16 && dt != AP_F16)) return AP_ERR_UNSUPPORTED;
   if (!have_device()) return AP_ERR_CUDA;
   const float sc = scale == 0.f ? (float)(1.0 / sqrt((double)d)) : scale;
-  cudaError_t e = launch_fwd_entmax_tc(Q, K, V, *tiles, O, B, H, Lq, Lk, d, dt == AP_F16 ? 1 : 0, sc,
-                                       static_cast<cudaStream_t>(stream));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = dt == AP_F32 ? launch_fwd_entmax_simt(Q, K, V, *tiles, O, B, H, Lq, Lk, d, sc, s)
+                               : launch_fwd_entmax_tc(Q, K, V, *tiles, O, B, H, Lq, Lk, d, dt == AP_F16 ? 1 : 0, sc, s);
   return e == cudaSuccess ? AP_OK : AP_ERR_CUDA;
 }
 

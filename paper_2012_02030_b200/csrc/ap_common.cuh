@@ -76,13 +76,16 @@ struct BuildMaskArgs {
 size_t select_scratch_bytes(int H, int Lq, int Lk);
 cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s);
 
+// (entmax: the 1.5-entmax normaliser instead of the softmax; fp32 tensors)
 cudaError_t launch_accumulate_simt(float *acc, const void *Q, const void *K, const float *bias, int B,
                                    int H, int Lq, int Lk, int d, ap_dtype dt, int causal, float scale,
-                                   cudaStream_t s);
+                                   cudaStream_t s, int entmax = 0);
 
 // fp32 tensors: CUDA-core kernel
 cudaError_t launch_fwd_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
                             int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
+cudaError_t launch_fwd_entmax_simt(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O,
+                                   int B, int H, int Lq, int Lk, int d, float scale, cudaStream_t s);
 cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const float *bias, int B, int H,
                                  int Lq, int Lk, int d, int causal, int f16, float scale, cudaStream_t s);
 

@@ -103,13 +103,13 @@ def test_accumulate_and_mask_reject_bad_arguments():
     assert f(FAKE, FAKE, FAKE, FAKE + 4, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 9, 8, 64, 1, 1, 0.0, None) == ap.AP_ERR_INVALID_ARG  # causal, Lk < Lq
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 32, 1, 0, 0.0, None) == ap.AP_ERR_UNSUPPORTED
-    f = ap.lib.ap_accumulate_attention_entmax15  # same checks; tensor-core types only
+    f = ap.lib.ap_accumulate_attention_entmax15  # same checks
     assert f(None, FAKE, FAKE, None, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, FAKE + 4, 1, 1, 8, 8, 64, 1, 0, 0.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 9, 8, 64, 1, 1, 0.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 64, 1, 0, -1.0, None) == ap.AP_ERR_INVALID_ARG
     assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 32, 1, 0, 0.0, None) == ap.AP_ERR_UNSUPPORTED
-    assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 64, ap.AP_F32, 0, 0.0, None) == ap.AP_ERR_UNSUPPORTED
+    assert f(FAKE, FAKE, FAKE, None, 1, 1, 8, 8, 64, 7, 0, 0.0, None) == ap.AP_ERR_UNSUPPORTED  # no such dtype
     t = _tiles(H=1, Lq=8, Lk=8, cap=1)
     ws = ap.ap_build_mask_workspace_bytes(1, 8, 8)
     for g in (ap.lib.ap_build_mask, ap.lib.ap_build_mask_layer):
