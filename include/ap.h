@@ -332,9 +332,15 @@ ap_status ap_sparse_attention_entmax15_fwd(const void *Q, const void *K, const v
                                            float scale, void *stream);
 
 /*
- * The same call for HOST tensors (pinned memory recommended): copies Q, K, V to
- * the caller's device staging buffers, runs ap_sparse_attention_fwd and copies
- * O back, all on `stream`.  dQ..dO are device buffers of the tensors' sizes.
+ * The same call for HOST tensors (pinned memory, or the copies are not asynchronous): copies
+ * Q, K, V to the caller's device staging buffers, runs ap_sparse_attention_fwd and copies O
+ * back.  dQ..dO are device buffers of the tensors' sizes.  The batch is cut into up to 8 chunks
+ * of batch elements that are copied in, computed and copied out as a pipeline, so that the two
+ * directions of the host link work at the same time: the kernels run on `stream`, the copies on
+ * two streams the library keeps per device (created on the first call, with 18 events, and never
+ * destroyed), ordered after the work already in `stream`; when the call returns, `stream` is
+ * ordered after the last output copy, so synchronising `stream` is enough.  Calls on one device
+ * share those streams and events: issue them from one host thread at a time.
  */
 ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const void *hV,
                                        const ap_tiles *tiles, void *hO, void *dQ, void *dK,

@@ -3,6 +3,7 @@
 #include <math.h>
 
 #include <atomic>
+#include <mutex>
 
 #include "ap_common.cuh"
 
@@ -364,6 +365,40 @@ ap_status ap_sparse_attention_bwd(const void *Q, const void *K, const void *V, c
              : AP_ERR_CUDA;
 }
 
+namespace {
+// Streams and events of ap_sparse_attention_fwd_host, one set per device, created on first use and
+// kept for the life of the process: an input-copy stream, an output-copy stream and one event pair
+// per chunk of batch elements.
+constexpr int kMaxChunks = 8;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, out_done = nullptr;
+  cudaEvent_t in_done[kMaxChunks] = {}, fwd_done[kMaxChunks] = {};
+};
+HostPipe g_pipe[kMaxDevices];
+std::mutex g_pipe_mutex;
+
+HostPipe *host_pipe() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe &p = g_pipe[dev];
+  if (!p.ready) {
+    bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.out_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; ok && c < kMaxChunks; ++c)
+      ok = cudaEventCreateWithFlags(&p.in_done[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&p.fwd_done[c], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    p.ready = true;
+  }
+  return &p;
+}
+}  // namespace
+
 ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const void *hV, const ap_tiles *tiles,
                                        void *hO, void *dQ, void *dK, void *dV, void *dO, int B, int H, int Lq,
                                        int Lk, int d, ap_dtype dt, float scale, void *stream) {
@@ -377,14 +412,40 @@ ap_status ap_sparse_attention_fwd_host(const void *hQ, const void *hK, const voi
   if (!have_device()) return AP_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t elem = dt == AP_F32 ? 4 : 2;
-  const size_t q_bytes = elem * B * H * (size_t)Lq * d, k_bytes = elem * B * H * (size_t)Lk * d;
-  if (cudaMemcpyAsync(dQ, hQ, q_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AP_ERR_CUDA;
-  if (cudaMemcpyAsync(dK, hK, k_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AP_ERR_CUDA;
-  if (cudaMemcpyAsync(dV, hV, k_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AP_ERR_CUDA;
-  st = ap_sparse_attention_fwd(dQ, dK, dV, tiles, dO, B, H, Lq, Lk, d, dt, scale, stream);
+  // The batch is cut into chunks of batch elements (the masks are per head, so any subset of the
+  // batch is a valid call): chunk c + 1 is copied in while chunk c is computed and chunk c - 1 is
+  // copied out, so the two directions of the host link work at the same time.
+  HostPipe *pipe = host_pipe();
+  if (!pipe) return AP_ERR_CUDA;
+  const int per_chunk = ceil_div(B, kMaxChunks), n_chunks = ceil_div(B, per_chunk);
+  const size_t q_one = elem * H * (size_t)Lq * d, k_one = elem * H * (size_t)Lk * d;  // bytes of one batch element
+  bool ok = cudaEventRecord(pipe->start, s) == cudaSuccess &&  // the staging buffers are free once s gets here
+            cudaStreamWaitEvent(pipe->in, pipe->start, 0) == cudaSuccess;
+  for (int c = 0; ok && c < n_chunks; ++c) {
+    const int b0 = c * per_chunk, nb = B - b0 < per_chunk ? B - b0 : per_chunk;
+    const size_t qo = q_one * b0, ko = k_one * b0;
+    const char *hq = static_cast<const char *>(hQ) + qo, *hk = static_cast<const char *>(hK) + ko,
+               *hv = static_cast<const char *>(hV) + ko;
+    char *q = static_cast<char *>(dQ) + qo, *k = static_cast<char *>(dK) + ko, *v = static_cast<char *>(dV) + ko,
+         *o = static_cast<char *>(dO) + qo;
+    ok = cudaMemcpyAsync(q, hq, q_one * nb, cudaMemcpyHostToDevice, pipe->in) == cudaSuccess &&
+         cudaMemcpyAsync(k, hk, k_one * nb, cudaMemcpyHostToDevice, pipe->in) == cudaSuccess &&
+         cudaMemcpyAsync(v, hv, k_one * nb, cudaMemcpyHostToDevice, pipe->in) == cudaSuccess &&
+         cudaEventRecord(pipe->in_done[c], pipe->in) == cudaSuccess &&
+         cudaStreamWaitEvent(s, pipe->in_done[c], 0) == cudaSuccess;
+    if (!ok) break;
+    st = ap_sparse_attention_fwd(q, k, v, tiles, o, nb, H, Lq, Lk, d, dt, scale, stream);
+    if (st != AP_OK) break;
+    ok = cudaEventRecord(pipe->fwd_done[c], s) == cudaSuccess &&
+         cudaStreamWaitEvent(pipe->out, pipe->fwd_done[c], 0) == cudaSuccess &&
+         cudaMemcpyAsync(static_cast<char *>(hO) + qo, o, q_one * nb, cudaMemcpyDeviceToHost, pipe->out) == cudaSuccess;
+  }
+  // whatever happened, s rejoins the output stream: the caller synchronises s only
+  // (s has already waited for every input copy issued above)
+  const bool joined = cudaEventRecord(pipe->out_done, pipe->out) == cudaSuccess &&
+                      cudaStreamWaitEvent(s, pipe->out_done, 0) == cudaSuccess;
   if (st != AP_OK) return st;
-  if (cudaMemcpyAsync(hO, dO, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return AP_ERR_CUDA;
-  return AP_OK;
+  return ok && joined ? AP_OK : AP_ERR_CUDA;
 }
 
 ap_status ap_device_status(void *stream) {

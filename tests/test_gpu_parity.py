@@ -967,3 +967,25 @@ def test_host_buffer_entry_point(ap):
     assert ap.ap_device_status() == ap.AP_OK
     ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy())
     pu.assert_close_attention(ho, ref, "bf16")
+
+
+def test_host_buffer_entry_point_pipelines_batch_chunks(ap):
+    """More batch elements than chunks (11 -> 6 chunks of 2, the last of 1), two calls back to back on the
+    same staging buffers: each result equals the device-tensor call bit for bit (batch elements are
+    independent), and the second call's input copies wait for the first call's kernels."""
+    w = W["bert"].scaled(B=11, H=2, Lq=200, Lk=200)
+    mask = inputs.random_mask(w.H, w.Lq, w.Lk, 0.3, seed=92)
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    q, k, v = (t.pin_memory() for t in inputs.eval_qkv(w))
+    q2, k2, v2 = (t.pin_memory() for t in inputs.eval_qkv(w.scaled(seed0=w.seed0 + 5)))
+    ho, ho2 = torch.empty_like(q).pin_memory(), torch.empty_like(q).pin_memory()
+    dq, dk, dv, do = (torch.empty_like(t, device="cuda") for t in (q, k, v, q))
+    ap.ap_sparse_attention_fwd_host(q, k, v, tiles, ho, dq, dk, dv, do)
+    ap.ap_sparse_attention_fwd_host(q2, k2, v2, tiles, ho2, dq, dk, dv, do)
+    torch.cuda.current_stream().synchronize()      # the caller's stream is all there is to wait for
+    assert ap.ap_device_status() == ap.AP_OK
+    want = ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles).cpu()
+    want2 = ap.ap_sparse_attention_fwd(q2.cuda(), k2.cuda(), v2.cuda(), tiles).cpu()
+    assert torch.equal(ho, want) and torch.equal(ho2, want2)
+    assert not torch.equal(ho, ho2)
