@@ -8,13 +8,13 @@
 //     c + (S2 - 1) / (S1 + sqrt(S1^2 - n (S2 - 1))),   S1 = sum (x_j - c), S2 = sum (x_j - c)^2 over the support.
 // That root is the answer when the support is the right one; otherwise it lies on the other side
 // of the answer than c (too many entries in the support push it right, too few left), the trial
-// thresholds left of the answer rise and those right of it fall, so the iteration started at
-// max x - 1 ends after a few supports.  Where the parabola has no root (a support far too wide)
+// thresholds left of the answer rise and those right of it fall, so the iteration ends after a
+// few supports wherever in [max x - 1, max x) it starts (it starts at max x - 0.625).  Where the parabola has no root (a support far too wide)
 // the step is Newton's, (S2 - 1) / (2 S1), which stays left of the answer.
 // The scores of a row (up to Lk of them, for every sample) do not fit on the chip, but QK^T is
 // cheap on the tensor cores, so the CTA recomputes them: one (head, 128-row query tile) per CTA,
 // up to 8 samples per launch,
-//   sweep 0          S = Q_b K_b(kt)^T for every key tile and sample -> row maxima, tau = max - 1
+//   sweep 0          S = Q_b K_b(kt)^T for every key tile and sample -> row maxima, tau = max - 0.625
 //   sweeps 1 .. n    the same visits -> n, S1, S2 of every (sample, row) -> one step; repeated
 //                    until no row of the CTA moves any more (or kMaxNewton sweeps)
 //   last sweep       p = max(x - tau, 0)^2; the sum over samples is kept in TMEM and added to the
@@ -43,6 +43,10 @@ constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr int kMaxB = 8;         // samples per launch (row statistics and thresholds live in shared memory)
 constexpr int kMaxNewton = 30;   // sweeps of the iteration at most (fp32 steps stop moving long before)
 constexpr int kBiasBytes = 128 * 128 * 4;
+// The first trial threshold: this far below the row maximum.  The root lies between max - 1 (all the
+// weight on one entry) and max; from either side of it the iteration below lands on the other side
+// or on the root, and starting in the middle of that range saves a sweep on most rows.
+constexpr float kFirstGap = 0.625f;
 
 template <int D>
 struct Cfg {
@@ -380,7 +384,7 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const float2 s0 = stats[(size_t)b * 128 + r], s1 = stats[(size_t)(kMaxB + b) * 128 + r];
         float tau;
         if (sw == 0) {
-          tau = fmaxf(s0.x, s1.x) - 1.f;  // f(max - 1) >= 0: left of the root
+          tau = fmaxf(s0.x, s1.x) - kFirstGap;
         } else {
           tau = my_tau[b * 128];
           const float S1 = s0.x + s1.x, S2 = s0.y + s1.y;

@@ -10,7 +10,7 @@
 //
 // kEntmax: the same sum with 1.5-entmax as the normaliser (the section on sparse normalisation),
 // p_j = max(s_j / 2 - tau, 0)^2 with tau such that the row sums to 1.  The row's scores are in
-// shared memory, so the warp iterates on tau there: from max/2 - 1 (left of the root) to the
+// shared memory, so the warp iterates on tau there: from max/2 - 0.625 (the root lies in [max/2 - 1, max/2)) to the
 // smaller root of the parabola of the current support, tau + (S2 - 1) / (S1 + sqrt(S1^2 - n (S2 - 1)))
 // with n, S1, S2 the support's size and its sums of (s_j/2 - tau) and of its square (Newton's
 // step (S2 - 1) / (2 S1) where the parabola has no root), until the step falls under
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(kThreads) accumulate_simt_kernel(float *__rest
       for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
       float *arow = acc + ((size_t)h * Lq + i) * Lk;
       if (kEntmax) {
-        float tau = 0.5f * m - 1.f;
+        float tau = 0.5f * m - 0.625f;  // the root lies in [max/2 - 1, max/2)
         for (int it = 0; it < 30; ++it) {
           float n = 0.f, S1 = 0.f, S2 = 0.f;
           for (int j = lane; j < jend; j += 32) {

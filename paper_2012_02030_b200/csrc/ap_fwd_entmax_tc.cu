@@ -8,7 +8,7 @@
 // of its list row (the schedule of the tile list: up to eight non-empty groups of 16 key columns,
 // taken from one or several key tiles, per round) several times, recomputing S = Q K^T on the tensor
 // cores each time:
-//   sweep 0          row maxima over the kept entries, tau = max - 1 (left of the root)
+//   sweep 0          row maxima over the kept entries, tau = max - 0.625 (the root lies in [max - 1, max))
 //   sweeps 1 .. n    over the support of the trial threshold (the n entries with x > tau):
 //                    S1 = sum (x - tau), S2 = sum (x - tau)^2 -> tau moves to the smaller root of the
 //                    support's parabola, tau + (S2 - 1) / (S1 + sqrt(S1^2 - n (S2 - 1))), which is the
@@ -40,6 +40,9 @@ constexpr int kSubBytes = 128 * 128;
 constexpr uint32_t kTmemCols = 512;  // S x 2 (columns 0..255), O (columns 256..256 + d)
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr int kMaxNewton = 30;
+// The first trial threshold: this far below the row maximum (the root lies in [max - 1, max); from
+// either side of it the iteration lands on the other side or on the root).
+constexpr float kFirstGap = 0.625f;
 
 template <int D>
 struct Cfg {
@@ -508,8 +511,8 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
       float tau;
       if (sw == 0) {
         const float m = fmaxf(s0.x, s1.x);
-        // f(max - 1) >= 0: left of the root.  No kept entry: every weight is 0 whatever the score
-        tau = m == -CUDART_INF_F ? CUDART_INF_F : m - 1.f;
+        // No kept entry: every weight is 0 whatever the score
+        tau = m == -CUDART_INF_F ? CUDART_INF_F : m - kFirstGap;
       } else {
         tau = *my_tau;
         const float S1 = s0.x + s1.x, S2 = s0.y + s1.y, n = cnts[r] + cnts[128 + r];

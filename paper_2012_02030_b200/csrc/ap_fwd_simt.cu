@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(kThreads) fwd_simt_kernel(const T *__restrict_
 // The same attention with 1.5-entmax as the normaliser (the section on sparse normalisation):
 // p_j = max(s_j / 2 - tau, 0)^2 over the kept keys, tau such that the row sums to 1.  tau depends
 // on all kept scores of a row, so the CTA walks its tiles once per sweep: row maxima first
-// (tau = max/2 - 1 is left of the root), then sweeps that collect the size n of the support of the
+// (tau = max/2 - 0.625; the root lies in [max/2 - 1, max/2)), then sweeps that collect the size n of the support of the
 // trial threshold and its sums S1, S2 of (s_j/2 - tau) and of its square and move tau to the smaller
 // root of the support's parabola, tau + (S2 - 1) / (S1 + sqrt(S1^2 - n (S2 - 1))) (Newton's step
 // (S2 - 1) / (2 S1) where it has none), until no row of the CTA moves by more than
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(kThreads) fwd_entmax_simt_kernel(const T *__re
     bool moved = false;
     if (kind == 0) {
       // no kept key: every weight is 0 whatever the threshold
-      tau = m == -CUDART_INF_F ? CUDART_INF_F : m - 1.f;
+      tau = m == -CUDART_INF_F ? CUDART_INF_F : m - 0.625f;
     } else {
       const float disc = S1 * S1 - n * (S2 - 1.f);
       const float step = S1 > 0.f ? (S2 - 1.f) / (S1 + (disc >= 0.f ? sqrtf(disc) : S1)) : 0.f;
