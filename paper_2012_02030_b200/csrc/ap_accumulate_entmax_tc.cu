@@ -308,10 +308,11 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             float a0 = st.x, a1 = 0.f, a2 = 0.f, a3 = 0.f, q0 = st.y, q1 = 0.f, q2 = 0.f, q3 = 0.f;
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
-              float u0, u1, u2, u3;
-              fadd2(u0, u1, t[e], t[e + 1], neg_tau, neg_tau);
-              fadd2(u2, u3, t[e + 2], t[e + 3], neg_tau, neg_tau);
-              u0 = fmaxf(u0, 0.f); u1 = fmaxf(u1, 0.f); u2 = fmaxf(u2, 0.f); u3 = fmaxf(u3, 0.f);
+              // max(x - tau, 0) as a saturating add: every trial threshold is at least max - 1 (the
+              // root's lower bound), so x - tau <= 1 and clamping to [0, 1] clamps at 0 only; the add
+              // runs on the FMA pipe, a separate maximum would load the half-rate ALU pipe
+              const float u0 = __saturatef(t[e] + neg_tau), u1 = __saturatef(t[e + 1] + neg_tau);
+              const float u2 = __saturatef(t[e + 2] + neg_tau), u3 = __saturatef(t[e + 3] + neg_tau);
               fadd2(a0, a1, a0, a1, u0, u1);
               fadd2(a2, a3, a2, a3, u2, u3);
               ffma2v(q0, q1, u0, u1, u0, u1, q0, q1);
@@ -329,9 +330,8 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
-              float u0, u1, p0, p1;
-              fadd2(u0, u1, t[e], t[e + 1], neg_tau, neg_tau);
-              u0 = fmaxf(u0, 0.f); u1 = fmaxf(u1, 0.f);
+              float p0, p1;
+              const float u0 = __saturatef(t[e] + neg_tau), u1 = __saturatef(t[e + 1] + neg_tau);
               if (b > 0) {
                 ffma2v(p0, p1, u0, u1, u0, u1, __uint_as_float(ps[e]), __uint_as_float(ps[e + 1]));
               } else {

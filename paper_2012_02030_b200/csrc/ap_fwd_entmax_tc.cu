@@ -37,7 +37,8 @@ using namespace sm100;
 constexpr int kThreads = 320;
 constexpr int kNormThreads = 256;
 constexpr int kSubBytes = 128 * 128;
-constexpr uint32_t kTmemCols = 512;  // S x 2 (columns 0..255), O (columns 256..256 + d)
+constexpr uint32_t kTmemCols = 512;  // S x 3 (columns 0..383), O (columns 384..384 + d)
+constexpr int kSBufs = 3;            // S buffers in flight: a visit's hand-offs take longer than its work
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr int kMaxNewton = 30;
 // The first trial threshold: this far below the row maximum (the root lies in [max - 1, max); from
@@ -67,7 +68,7 @@ struct Cfg {
 
 struct Barriers {
   uint64_t q_full;
-  uint64_t s_full[2], s_empty[2];
+  uint64_t s_full[kSBufs], s_empty[kSBufs];
   uint64_t in_full[6], in_empty[6];  // K ring: rows landed / S = Q K^T of the visit completed
   uint64_t v_full[2], v_empty[2];    // V ring: rows landed / O += P V of the visit completed
   uint64_t sweep_done;  // all statistics of the sweep are in shared memory
@@ -179,7 +180,7 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kSBufs; ++s) {
       mbar_init(&bars->s_full[s], 1);
       mbar_init(&bars->s_empty[s], kNormThreads);
     }
@@ -300,8 +301,8 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------ MMA issuer
-    // S = Q K^T of the first two visits of the next sweep is issued before the decision as well
-    // (S is double-buffered).
+    // S = Q K^T of the first visits of the next sweep is issued before the decision as well
+    // (three S buffers).
     if (lane == 0) {
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true, kF16);
       const uint32_t q_addr = smem_u32(smem), k_addr = smem_u32(smem + C::kKOffset), v_addr = smem_u32(smem + C::kVOffset);
@@ -311,14 +312,14 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
       uint32_t info_next = __ldg(round_info + t0);  // used one visit later: the load stays in flight
       int vv_next = 0;
       auto issue_qk = [&]() -> bool {
-        const int st = v % C::kStages, buf = v & 1;
+        const int st = v % C::kStages, buf = v % kSBufs;
         const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * (int)(info_next & 15u), false, false, kF16);
         vv_next = vv_next + 1 == T ? 0 : vv_next + 1;
         info_next = __ldg(round_info + t0 + vv_next);
         if (!wait_or_abort(&bars->in_full[st], (uint32_t)(v / C::kStages) & 1u, abort_flag, err)) return false;
         // S[buf] was read (and, in the last sweep, its P consumed by a product issued earlier by
-        // this thread: products execute in issue order) two visits ago
-        if (!wait_or_abort(&bars->s_empty[buf], ((uint32_t)(v >> 1) & 1u) ^ 1u, abort_flag, err)) return false;
+        // this thread: products execute in issue order) kSBufs visits ago
+        if (!wait_or_abort(&bars->s_empty[buf], ((uint32_t)(v / kSBufs) & 1u) ^ 1u, abort_flag, err)) return false;
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
@@ -334,20 +335,20 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
       // O += P V of visit u = round j of the last sweep: P is in S[u & 1] once the normalising
       // threads have arrived; one contraction step of 16 keys per group; then the V stage is free
       auto issue_pv = [&](int u, int j) -> bool {
-        const int sb = u & 1, sv = j % C::kVStages, ng_u = ng_of(j);
+        const int sb = u % kSBufs, sv = j % C::kVStages, ng_u = ng_of(j);
         if (!wait_or_abort(&bars->v_full[sv], (uint32_t)(j / C::kVStages) & 1u, abort_flag, err)) return false;
-        if (!wait_or_abort(&bars->s_empty[sb], (uint32_t)(u >> 1) & 1u, abort_flag, err)) return false;
+        if (!wait_or_abort(&bars->s_empty[sb], (uint32_t)(u / kSBufs) & 1u, abort_flag, err)) return false;
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
           if (ks < ng_u)
-            mma_ts(tmem + 256, tmem + 128 * sb + 32 * (ks >> 1) + 8 * (ks & 1),
+            mma_ts(tmem + 128 * kSBufs, tmem + 128 * sb + 32 * (ks >> 1) + 8 * (ks & 1),
                    smem_desc_sw128(v_addr + sv * C::kTileBytes + ks * 2048, kSubBytes, 1024), idesc_pv,
                    (j == 0 && ks == 0) ? 0u : 1u);
         mma_commit(&bars->v_empty[sv]);
         return true;
       };
-      const int n_ahead = T < 2 ? T : 2;
+      const int n_ahead = T < kSBufs ? T : kSBufs;
       for (int vv = 0; vv < T && ok; ++vv) ok = issue_qk();  // sweep 0
       for (int sw = 0; ok; ++sw) {
         const int v_head = v;
@@ -400,11 +401,11 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
       st = make_float2(kind == 0 ? -CUDART_INF_F : 0.f, 0.f);
       cnt = 0.f;
       for (int vv = 0; vv < T && ok; ++vv, ++v) {
-        const int buf = v & 1;
+        const int buf = v % kSBufs;
         const bool full = (info_next & 0x80u) != 0u;  // every entry of the round is kept
         const uint2 bits = bits_next;
         fetch(vv + 1 == T ? 0 : vv + 1, info_next, bits_next);
-        ok = wait_or_abort(&bars->s_full[buf], (uint32_t)(v >> 1) & 1u, abort_flag, err);
+        ok = wait_or_abort(&bars->s_full[buf], (uint32_t)(v / kSBufs) & 1u, abort_flag, err);
         if (!ok) break;
         tc_fence_after_sync();
         float psum0 = 0.f, psum1 = 0.f;
@@ -437,10 +438,11 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
             float a0 = st.x, a1 = 0.f, a2 = 0.f, a3 = 0.f, q0 = st.y, q1 = 0.f, q2 = 0.f, q3 = 0.f;
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
-              float u0, u1, u2, u3;
-              fadd2(u0, u1, t[e], t[e + 1], neg_tau, neg_tau);
-              fadd2(u2, u3, t[e + 2], t[e + 3], neg_tau, neg_tau);
-              u0 = fmaxf(u0, 0.f); u1 = fmaxf(u1, 0.f); u2 = fmaxf(u2, 0.f); u3 = fmaxf(u3, 0.f);
+              // max(x - tau, 0) as a saturating add: every trial threshold is at least max - 1 (the
+              // root's lower bound), so x - tau <= 1 and clamping to [0, 1] clamps at 0 only; the add
+              // runs on the FMA pipe, a separate maximum would load the half-rate ALU pipe
+              const float u0 = __saturatef(t[e] + neg_tau), u1 = __saturatef(t[e + 1] + neg_tau);
+              const float u2 = __saturatef(t[e + 2] + neg_tau), u3 = __saturatef(t[e + 3] + neg_tau);
               fadd2(a0, a1, a0, a1, u0, u1);
               fadd2(a2, a3, a2, a3, u2, u3);
               ffma2v(q0, q1, u0, u1, u0, u1, q0, q1);
@@ -453,9 +455,7 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
             uint32_t pk[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              float u0, u1;
-              fadd2(u0, u1, t[2 * e], t[2 * e + 1], neg_tau, neg_tau);
-              u0 = fmaxf(u0, 0.f); u1 = fmaxf(u1, 0.f);
+              const float u0 = __saturatef(t[2 * e] + neg_tau), u1 = __saturatef(t[2 * e + 1] + neg_tau);
               pk[e] = pack2<kF16>(u0 * u0, u1 * u1);
               const float2 pr = unpack2<kF16>(pk[e]);  // the weights the product will use
               psum0 += pr.x;
@@ -490,7 +490,7 @@ fwd_entmax_kernel(const __grid_constant__ Maps maps, uint16_t *__restrict__ O, c
 #pragma unroll
         for (int c = 0; c < D / 64; ++c) {
           uint32_t o[32];
-          tmem_ld32(tmem + 256 + wg * (D / 2) + 32 * c + lane_addr, o);
+          tmem_ld32(tmem + 128 * kSBufs + wg * (D / 2) + 32 * c + lane_addr, o);
           tmem_wait_ld();
           if (row_ok) {
             uint4 *dst = reinterpret_cast<uint4 *>(O + ((size_t)bh * Lq + i) * D + wg * (D / 2) + 32 * c);
