@@ -887,6 +887,36 @@ def _pipeline(ap, w, n_batches, oracle_acc=True):
     return pu.assert_close_attention(out, ref, w.dtype, w.name)
 
 
+def _pipeline_entmax(ap, w, n_batches):
+    """The procedure for a model normalised by 1.5-entmax: entmax average -> Eq. 2 on the GPU's own
+    accumulator bits (stage-exact; the average is sparse, so zeros tie in great numbers and the
+    threshold may be 0) -> entmax forward under that mask against the oracle."""
+    bias = inputs.calib_bias(w)
+    acc = _entmax_acc(ap, w, n_batches, bias.cuda())
+    acc_host = acc.cpu().numpy()
+    np.testing.assert_allclose(acc_host, _entmax_want(w, n_batches, bias), rtol=ENTMAX_RTOL,
+                               atol=ENTMAX_ATOL * n_batches * w.B)
+    for layer in (False, True):
+        mask, tiles, nnz = pu.gpu_build_mask(ap, acc, w, layer=layer)
+        want_mask, want_nnz = (orc.build_mask_layer if layer else orc.build_mask)(acc_host, w.keep_frac, w.causal,
+                                                                                   w.keep_diag)
+        np.testing.assert_array_equal(mask.cpu().numpy(), want_mask)
+        np.testing.assert_array_equal(nnz.cpu().numpy(), want_nnz)
+        pu.assert_tiles_equal(tiles.to_host(), orc.mask_to_tiles(want_mask))
+    return _entmax_fwd_case(ap, w, torch.from_numpy(want_mask))
+
+
+@pytest.mark.parametrize("name,over,n_batches", [
+    ("bert", dict(B=4, H=3), 2),
+    ("lm", dict(B=2, H=2, Lq=300, Lk=300), 2),
+    ("s2s_cross", dict(B=3, H=2, dtype="f16"), 2),
+    ("tiny", dict(keep_frac=0.6), 2),            # fp32; keeps more than the average's support: the threshold is 0
+    ("long", dict(B=1, H=2, Lq=640, Lk=640), 2),
+])
+def test_workload_with_entmax_normaliser(ap, name, over, n_batches):
+    _pipeline_entmax(ap, W[name].scaled(**over), n_batches)
+
+
 def test_workload_tiny_full(ap):
     _pipeline(ap, W["tiny"], W["tiny"].calib_batches)
 
