@@ -231,8 +231,14 @@ accumulate_entmax_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     bool last = false, ok = true;
     for (int sw = 0; ok; ++sw) {
       const int kind = sw == 0 ? 0 : (last ? 2 : 1);  // 0 maxima, 1 sums over the support, 2 weights
+      // (key tile, sample) of the visit, stepped rather than divided out of vv: an integer division per
+      // visit is a hundred cycles on this thread's critical path
+      int kt = 0, b = -1;
       for (int vv = 0; vv < visits_per_sweep && ok; ++vv, ++v) {
-        const int kt = vv / Bc, b = vv % Bc;
+        if (++b == Bc) {
+          b = 0;
+          ++kt;
+        }
         const int buf = v & 1;
         const int j0 = kt * kTile + 64 * wg;  // first column of this thread's slice
         if (b == 0) {  // new key tile: fetch this thread's bias slice once for all samples

@@ -213,10 +213,17 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     float bias2[64];  // bias * log2(e) of this thread's 64 columns of the current key tile
     float ref = 0.f;  // sweep 2: max + log2(sum) of the current sample's row
     bool ok = true;
+    // (sweep, key tile, sample) of the visit, stepped rather than divided out of v: an integer
+    // division per visit is a hundred cycles on this thread's critical path
+    int sweep = 0, kt = 0, b = -1;
     for (int v = 0; v < n_visits && ok; ++v) {
-      const int sweep = v >= visits_per_sweep ? 1 : 0;
-      const int vv = v - sweep * visits_per_sweep;
-      const int kt = vv / Bc, b = vv % Bc;
+      if (++b == Bc) {
+        b = 0;
+        if (++kt == n_k) {
+          kt = 0;
+          sweep = 1;
+        }
+      }
       const int buf = v & 1;
       const int j0 = kt * kTile + 64 * wg;  // first column of this thread's slice
       if (v == visits_per_sweep) {
