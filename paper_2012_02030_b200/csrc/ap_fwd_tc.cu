@@ -234,17 +234,34 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       int bh, qt, rho0, rho1;  // rounds [rho0, rho1): loaded here, first read when the item begins
       bool in_range, exists;   // !exists: no such item (the unit's halves coincide)
     };
+    // (called for t = 0, 1, 2, ... in turn: the unit's (j, bh, h = bh % H) are stepped from one unit
+    // of this CTA to the next instead of divided out of the unit number every time; this warp's
+    // instruction stream is what short items wait for)
+    int cur_u = (int)blockIdx.x, cur_j = cur_u % n_half, cur_bh = cur_u / n_half, cur_h = cur_bh % H;
+    const int step_j = item_step % n_half, step_bh = item_step / n_half, step_h = step_bh % H;
     auto item_ref = [&](int t) {
       ItemRef it;
-      const int u = (int)blockIdx.x + (t >> 1) * item_step;
+      if (t >= 2 && !(t & 1)) {  // the next unit
+        cur_u += item_step;
+        cur_j += step_j;
+        cur_bh += step_bh;
+        cur_h += step_h;
+        if (cur_j >= n_half) {
+          cur_j -= n_half;
+          ++cur_bh;
+          ++cur_h;
+        }
+        if (cur_h >= H) cur_h -= H;
+      }
+      const int u = cur_u;
       it.in_range = u < n_units;
       it.bh = 0, it.qt = 0, it.rho0 = 0, it.rho1 = 0, it.exists = false;
       if (it.in_range) {
-        const int j = u % n_half;
-        it.bh = u / n_half;
+        const int j = cur_j;
+        it.bh = cur_bh;
         it.qt = (t & 1) ? j : n_qt - 1 - j;
         if (!(t & 1) || j != n_qt - 1 - j) {
-          const int lr = (it.bh % H) * n_qt + it.qt;
+          const int lr = cur_h * n_qt + it.qt;
           it.rho0 = (int)ldg_now_u32(round_ptr + lr);
           it.rho1 = (int)ldg_now_u32(round_ptr + lr + 1);
           it.exists = true;
