@@ -102,9 +102,9 @@ struct Shared {
                                                       // (one pair per set of accumulators)
   uint64_t ml_ready[4];                               // per item: both groups have handed over (m, l)
   float2 ml[4][2][kTile];                             // [item % 4][group][row] = (m, l)
-  int32_t ml_item[4];                                 // the item handed over, -1: no more items
+  int32_t ml_bh[4], ml_qt[4];                         // the item handed over (b * H + h, query tile); qt = -1: no more items
   uint32_t info[kMaxStages];
-  int32_t item[kMaxStages];                           // the item a stage's round belongs to
+  int32_t item_bh[kMaxStages], item_qt[kMaxStages];   // the item a stage's round belongs to
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -386,7 +386,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         if (lane == 0) {
           sh->info[si] = (uint32_t)ng | (v == 0 ? kInfoFirst : 0u) | (v + 1 == n_rounds ? kInfoLast : 0u) |
                          (full ? kInfoFull : 0u);
-          sh->item[si] = bh * n_qt + qt;
+          sh->item_bh[si] = bh;
+          sh->item_qt[si] = qt;
           mbar_arrive_expect_tx(&sh->k_full[st], bytes);
           if (full) {
             mbar_arrive(&sh->b_full[si]);
@@ -529,7 +530,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     uint32_t n = 0;
     float m = -CUDART_INF_F, l = 0.f;       // this group's exponent reference and running sum of weights
     bool o_started = false;                  // an earlier round of the item added to this group's accumulator
-    int cur_item = 0;
+    int cur_bh = 0, cur_qt = 0;
     for (uint32_t g = 0; ok; ++g) {
       const int st = (int)(g % kMaxStages);  // info / bitmap slot of the round
       const uint32_t sb = g & 1u;
@@ -542,7 +543,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
       const bool tile_full = (info & kInfoFull) != 0u;
       if (first) {
-        cur_item = sh->item[st];  // (b * H + h) * n_qt + qt
+        cur_bh = sh->item_bh[st];
+        cur_qt = sh->item_qt[st];
         m = -CUDART_INF_F;
         l = 0.f;
         o_started = false;
@@ -666,14 +668,17 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       // with the next item; the slot of the hand-over ring was read by the epilogue of item n - 4,
       // which is over (this item's S needed O += P V of item n - 2, that the epilogue of item n - 3).
       sh->ml[n & 3u][grp][r] = make_float2(m, l);
-      if (threadIdx.x == 0) sh->ml_item[n & 3u] = cur_item;
+      if (threadIdx.x == 0) {
+        sh->ml_bh[n & 3u] = cur_bh;
+        sh->ml_qt[n & 3u] = cur_qt;
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->ml_ready[n & 3u]);
       ++n;
     }
     // no more items: tell the epilogue warps
     if (ok) {
-      if (threadIdx.x == 0) sh->ml_item[n & 3u] = -1;
+      if (threadIdx.x == 0) sh->ml_qt[n & 3u] = -1;
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->ml_ready[n & 3u]);
     }
@@ -686,11 +691,11 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     for (uint32_t n = 0; ok; ++n) {
       ok = warp_wait(&sh->ml_ready[n & 3u], (n >> 2) & 1u, lane, abort_flag, err);
       if (!ok) break;
-      const int item = sh->ml_item[n & 3u];  // (b * H + h) * n_qt + qt
-      if (item < 0) break;
+      const int item_qt = sh->ml_qt[n & 3u], item_bh = sh->ml_bh[n & 3u];
+      if (item_qt < 0) break;
       const float2 g0 = sh->ml[n & 3u][0][r], g1 = sh->ml[n & 3u][1][r];
-      const int i = (item % n_qt) * kTile + r;
-      uint16_t *orow = O + ((size_t)(item / n_qt) * Lq + i) * D;
+      const int i = item_qt * kTile + r;
+      uint16_t *orow = O + ((size_t)item_bh * Lq + i) * D;
       const float m_tot = fmaxf(g0.x, g1.x);
       // weight of a partial result; 0 for a group that saw no kept entry of this row (m = -inf),
       // whose accumulator is then never read into the sum (it may hold a previous item's data)
