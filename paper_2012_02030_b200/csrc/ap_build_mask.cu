@@ -357,7 +357,6 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
   const int h = blockIdx.x, t = threadIdx.x;
   if (t == 0) n_valid_s = 0u;
   __syncthreads();
-  const unsigned long long cells = (unsigned long long)Lq * Lk;
   const int off = (causal || diag) ? Lk - period : 0;
   constexpr int kDraws = kSamples / 1024;  // per thread, all loads in flight at once
   float drawn[kDraws];
@@ -365,8 +364,11 @@ __global__ void __launch_bounds__(1024) sample_pivots_kernel(const float *__rest
 #pragma unroll
   for (int u = 0; u < kDraws; ++u) {
     const int s = t + 1024 * u;
-    const unsigned long long idx = mix64(((unsigned long long)h << 32) | (unsigned)s) % cells;
-    const int i = (int)(idx / Lk), j = (int)(idx % Lk);
+    // row and column from the two halves of one 64-bit draw, scaled by multiplication (64-bit
+    // divisions, emulated in dozens of instructions each, made up most of this kernel's time)
+    const unsigned long long m = mix64(((unsigned long long)h << 32) | (unsigned)s);
+    const int i = (int)(((m >> 32) * (unsigned long long)Lq) >> 32);
+    const int j = (int)(((m & 0xffffffffull) * (unsigned long long)Lk) >> 32);
     const int own = i % period + off;
     valid[u] = !((causal && j > own) || (diag && j == own));
     drawn[u] = valid[u] ? acc[((size_t)h * Lq + i) * Lk + j] : 0.f;
