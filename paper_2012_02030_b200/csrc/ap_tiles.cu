@@ -94,15 +94,20 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
     __syncthreads();
     const int carry = carry_s;
     int before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - mine;
+    int row = idx0 / n_kt, kt = idx0 - row * n_kt;  // list row and key tile of the tile, stepped below
 #pragma unroll
     for (int e = 0; e < kPer; ++e) {
       const int idx = idx0 + e;
       const int flag = cnt[e] > 0 ? 1 : 0;
       if (idx < n_tiles) {
         stage_pos[idx] = flag ? before : -1;
-        if (idx % n_kt == n_kt - 1) row_ptr[idx / n_kt + 1] = min(before + flag, cap);
+        if (kt == n_kt - 1) row_ptr[row + 1] = min(before + flag, cap);
       }
       before += flag;
+      if (++kt == n_kt) {
+        kt = 0;
+        ++row;
+      }
     }
     __syncthreads();
     if (threadIdx.x == 1023) carry_s = carry + warp_sums[31];
