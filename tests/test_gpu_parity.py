@@ -525,6 +525,18 @@ def test_accumulate_entmax15_special_rows(ap):
     assert ap.ap_device_status() == ap.AP_OK
 
 
+def test_accumulate_entmax15_large_scores(ap):
+    """Scores in the hundreds: fp32 resolves x = z/2 to about 1e-5 there, so the threshold and with it
+    the weights are coarser (2 u dtau with dtau of that order), but the iteration still ends, rows still sum
+    to 1 and almost every row is one-hot or close to it."""
+    w = W["tiny"].scaled(Lq=200, Lk=333, dtype="bf16", B=2)
+    got = _entmax_acc(ap, w, 1, None, scale=25.0).cpu().numpy()
+    want = _entmax_want(w, 1, None, scale=25.0)
+    assert np.isfinite(got).all()
+    np.testing.assert_allclose(got.sum(-1), w.B, rtol=1e-4)
+    np.testing.assert_allclose(got, want, rtol=1e-3, atol=2e-3)
+
+
 def test_accumulate_entmax15_sharp_scores_custom_scale(ap):
     w = W["tiny"].scaled(Lq=40, Lk=90, dtype="bf16")
     for scale in (0.05, 1.5):
