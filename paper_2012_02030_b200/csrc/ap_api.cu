@@ -28,24 +28,6 @@ bool shape_ok(int H, int Lq, int Lk) {
   return true;
 }
 
-ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shape_must_match) {
-  if (!t) return AP_ERR_INVALID_ARG;
-  if (!t->row_ptr || !t->col_idx || !t->flags || !t->bitmap || !t->groups || !t->round_ptr || !t->round_rows ||
-      !t->round_info || !t->round_bitmap)
-    return AP_ERR_INVALID_ARG;
-  if (!aligned16(t->bitmap) || !aligned16(t->round_bitmap) || !aligned16(t->round_rows) ||
-      (reinterpret_cast<uintptr_t>(t->row_ptr) & 3u) || (reinterpret_cast<uintptr_t>(t->col_idx) & 3u) ||
-      (reinterpret_cast<uintptr_t>(t->round_ptr) & 3u))
-    return AP_ERR_INVALID_ARG;
-  if (t->cap < 1) return AP_ERR_WORKSPACE;
-  if (shape_must_match) {
-    if (t->H != H || t->Lq != Lq || t->Lk != Lk || t->n_qt != ceil_div(Lq, kTile) ||
-        t->n_kt != ceil_div(Lk, kTile))
-      return AP_ERR_INVALID_ARG;
-  }
-  return AP_OK;
-}
-
 void fill_tiles_shape(ap_tiles *t, int H, int Lq, int Lk) {
   t->H = H;
   t->Lq = Lq;

@@ -23,6 +23,28 @@ unsigned *device_error_word();
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// The checks every entry point that fills or reads a tile list applies to the descriptor before
+// anything is enqueued: all arrays present, the arrays that kernels access with 16-byte vectors
+// (bitmap, round_bitmap, round_rows) 16-byte aligned, the 32-bit arrays 4-byte aligned, a capacity
+// of at least one tile, and (for readers) the recorded shape equal to the call's.
+inline ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shape_must_match) {
+  auto misaligned = [](const void *p, uintptr_t mask) { return (reinterpret_cast<uintptr_t>(p) & mask) != 0; };
+  if (!t) return AP_ERR_INVALID_ARG;
+  if (!t->row_ptr || !t->col_idx || !t->flags || !t->bitmap || !t->groups || !t->round_ptr || !t->round_rows ||
+      !t->round_info || !t->round_bitmap)
+    return AP_ERR_INVALID_ARG;
+  if (misaligned(t->bitmap, 15u) || misaligned(t->round_bitmap, 15u) || misaligned(t->round_rows, 15u) ||
+      misaligned(t->row_ptr, 3u) || misaligned(t->col_idx, 3u) || misaligned(t->round_ptr, 3u))
+    return AP_ERR_INVALID_ARG;
+  if (t->cap < 1) return AP_ERR_WORKSPACE;
+  if (shape_must_match) {
+    if (t->H != H || t->Lq != Lq || t->Lk != Lk || t->n_qt != ceil_div(Lq, kTile) ||
+        t->n_kt != ceil_div(Lk, kTile))
+      return AP_ERR_INVALID_ARG;
+  }
+  return AP_OK;
+}
+
 // Kernels launched by this library in this process (see ap_launch_count in ap.h).
 void count_launches(int n);
 

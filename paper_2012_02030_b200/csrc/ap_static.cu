@@ -46,11 +46,8 @@ using namespace ap;
 extern "C" ap_status ap_mask_to_tiles_static(const uint8_t *mask, int H, int Lq, int Lk, ap_tiles *tiles,
                                              void *stream) {
   if (!mask || H < 1 || Lq < 1 || Lk < 1) return AP_ERR_INVALID_ARG;
-  if (!tiles || !tiles->row_ptr || !tiles->col_idx || !tiles->flags || !tiles->bitmap || !tiles->groups || !tiles->round_ptr || !tiles->round_rows ||
-      !tiles->round_info || !tiles->round_bitmap ||
-      (reinterpret_cast<uintptr_t>(tiles->bitmap) & 15u))
-    return AP_ERR_INVALID_ARG;
-  if (tiles->cap < 1) return AP_ERR_WORKSPACE;
+  const ap_status st = check_tiles(tiles, H, Lq, Lk, false);
+  if (st != AP_OK) return st;
   const int64_t n_tiles = (int64_t)H * ceil_div(Lq, kTile) * ceil_div(Lk, kTile);
   if (n_tiles > kStaticMaxTiles) return AP_ERR_WORKSPACE;  // beyond the built-in scratch
   if (stage_bytes(H, Lq, Lk) > kStaticBytes) return AP_ERR_WORKSPACE;

@@ -29,6 +29,23 @@ def test_static_variant_rejects_shapes_beyond_its_scratch_before_touching_a_devi
     assert ap.lib.ap_mask_to_tiles_static(None, 1, 8, 8, ctypes.byref(t), None) == ap.AP_ERR_INVALID_ARG
 
 
+def test_static_variant_rejects_misaligned_tile_arrays_like_the_workspace_variant():
+    """The kernels behind both entry points store 16-byte vectors to bitmap, round_bitmap and
+    round_rows and 32-bit words to row_ptr, col_idx and round_ptr: a misaligned array must come back as
+    an argument error from the host, not as a misaligned-address fault from the device."""
+    from paper_2012_02030_b200 import binding as ap
+
+    names = [f[0] for f in ap.ap_tiles._fields_]
+    for field, off in (("bitmap", 8), ("round_bitmap", 4), ("round_rows", 8), ("row_ptr", 2), ("col_idx", 1),
+                       ("round_ptr", 2)):
+        t = ap.ap_tiles(1, 128, 128, 1, 1, 4, *([FAKE] * 9))
+        assert field in names
+        setattr(t, field, FAKE + off)
+        assert ap.lib.ap_mask_to_tiles_static(FAKE, 1, 128, 128, ctypes.byref(t), None) == ap.AP_ERR_INVALID_ARG, field
+        assert ap.lib.ap_mask_to_tiles(FAKE, 1, 128, 128, ctypes.byref(t), FAKE, 1 << 30, None) == \
+            ap.AP_ERR_INVALID_ARG, field
+
+
 @pytest.mark.gpu
 def test_static_variant_matches_workspace_variant_on_two_calls_in_a_row():
     from paper_2012_02030_b200 import binding as ap
@@ -43,7 +60,11 @@ def test_static_variant_matches_workspace_variant_on_two_calls_in_a_row():
         ap.ap_mask_to_tiles(mask, want)
         got = ap.Tiles(H, Lq, Lk)
         before = ap.ap_launch_count()
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         ap.ap_mask_to_tiles_static(mask, got)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before  # the call took no device memory
         assert ap.ap_launch_count() - before == 6  # bitmaps, scan, gather; rounds: count, scan, fill
         assert ap.ap_device_status() == ap.AP_OK
         a, b = got.to_host(), want.to_host()
