@@ -25,7 +25,10 @@
  *     enqueued.  Nothing throws, aborts or traps.  Conditions only the device
  *     can see (a tile list that outgrew its capacity, a bounded wait that
  *     expired) set a sticky device word that ap_device_status() returns.
- *   - d is 64 or 128.  Any Lq, Lk >= 1 is accepted.
+ *   - d is 64 or 128.  Any Lq, Lk >= 1 is accepted by the 16-bit paths; the fp32
+ *     accumulate keeps a row of Lk scores in shared memory and returns
+ *     AP_ERR_UNSUPPORTED beyond roughly Lk = 45 000.  ap_build_mask (one
+ *     selection per head) takes at most 65 535 heads.
  *   - `causal` != 0 restricts query i to the keys j <= i + (Lk - Lq) and needs
  *     Lk >= Lq.  With Lq == Lk that is the usual autoregressive mask; with
  *     Lk = mem + Lq the first `mem` keys are cached positions of earlier segments,
@@ -118,6 +121,18 @@ int ap_version(void);
 /* Kernels this library has launched so far in this process (a diagnostic counter). */
 uint64_t ap_launch_count(void);
 
+/*
+ * Test hook for the failure path (no counterpart in the paper).  Every wait inside the tensor-core
+ * kernels polls a bounded number of times; when a wait runs out the kernel raises the device status
+ * word, every role leaves its loop, copies in flight are waited for (bounded), tensor memory is
+ * freed and the kernel returns, after which ap_device_status() reports AP_ERR_TIMEOUT once.
+ * With on != 0, the following launches of ap_sparse_attention_fwd (16-bit types) run on ONE
+ * thread block with a poll limit of a few thousand and leave out one producer arrival, so that
+ * this path runs within a millisecond without faulting or hanging anything; their output is
+ * undefined.  on == 0 restores normal operation.  Process-wide; not for production use.
+ */
+void ap_debug_expire_waits(int on);
+
 /* Static, human-readable name of a status code. */
 const char *ap_status_string(ap_status s);
 
@@ -134,8 +149,9 @@ size_t ap_mask_to_tiles_workspace_bytes(int H, int Lq, int Lk);
  * over the row's domain (all j, or the causal domain above); entries outside the
  * domain are not touched.  The 1/n of Eq. 1 is left to the caller, who counts
  * the samples: the selection of Eq. 2 does not depend on it.
- *   acc    [H,Lq,Lk] fp32, in/out.  The sum over b is taken in ascending b with no
- *          floating-point atomics, so results are reproducible bit for bit.
+ *   acc    [H,Lq,Lk] fp32, in/out.  The sum over b is taken in ascending b inside the
+ *          kernel and added to acc with one reduction per entry and launch, ordered by
+ *          the stream, so results are reproducible bit for bit.
  *   Q, K   [B,H,Lq,d], [B,H,Lk,d] of type dt (AP_BF16 and AP_F16 run on the tensor cores)
  *   bias   [H,Lq,Lk] fp32 added after scaling, or NULL
  *   scale  multiplier of Q.K^T; 0 selects 1/sqrt(d)

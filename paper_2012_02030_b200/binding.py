@@ -18,7 +18,8 @@ AP_OK, AP_ERR_INVALID_ARG, AP_ERR_UNSUPPORTED, AP_ERR_WORKSPACE, AP_ERR_CUDA, AP
 AP_F32, AP_BF16, AP_F16 = 0, 1, 2
 AP_STATIC_MAX_TILES = 1024
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libap_b200.so")
+# AP_B200_LIB names another build of the same library (e.g. one compiled with development aids)
+_LIB_PATH = os.environ.get("AP_B200_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libap_b200.so")
 
 
 class ApError(RuntimeError):
@@ -50,6 +51,7 @@ def _load() -> ctypes.CDLL:
     sig = {
         "ap_version": (i, []),
         "ap_launch_count": (ctypes.c_uint64, []),
+        "ap_debug_expire_waits": (None, [i]),
         "ap_status_string": (ctypes.c_char_p, [i]),
         "ap_tiles_capacity": (i64, [i, i, i]),
         "ap_build_mask_workspace_bytes": (sz, [i, i, i]),
@@ -79,7 +81,7 @@ def _load() -> ctypes.CDLL:
 
 
 lib = _load()
-EXPORTS = ("ap_version", "ap_launch_count", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
+EXPORTS = ("ap_version", "ap_launch_count", "ap_debug_expire_waits", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
            "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_accumulate_attention_entmax15", "ap_build_mask", "ap_build_mask_layer", "ap_build_mask_ex", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd", "ap_sparse_attention_entmax15_fwd",
            "ap_sparse_attention_fwd_host", "ap_sparse_attention_bwd_workspace_bytes", "ap_sparse_attention_bwd",
@@ -99,6 +101,10 @@ def ap_version() -> int:
 
 def ap_launch_count() -> int:
     return int(lib.ap_launch_count())
+
+
+def ap_debug_expire_waits(on: bool) -> None:
+    lib.ap_debug_expire_waits(1 if on else 0)
 
 
 def ap_tiles_capacity(H: int, Lq: int, Lk: int) -> int:

@@ -1,6 +1,6 @@
 // Eq. 1 as a running sum for bf16 and fp16 tensors, on the tcgen05 tensor cores.
 //
-// One CTA owns one (head, 128-row query tile) and adds, for up to 32 samples b,
+// One CTA owns one (head, 128-row query tile) and adds, for up to 16 samples b per launch,
 // the normalised softmax rows to the accumulator.  A softmax row needs its
 // maximum and its sum of exponentials over ALL keys before any entry can be
 // normalised, and the sum over b needs each sample normalised separately, so

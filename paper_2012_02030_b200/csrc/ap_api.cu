@@ -43,6 +43,13 @@ bool have_device() {
 
 }  // namespace
 
+std::atomic<int> g_expire_waits{0};
+
+DebugKnobs debug_knobs() {
+  const int on = g_expire_waits.load(std::memory_order_relaxed);
+  return DebugKnobs{on ? (1u << 12) : (1u << 22), on};
+}
+
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 unsigned *device_error_word() {
@@ -75,7 +82,9 @@ using namespace ap;
 
 extern "C" {
 
-int ap_version(void) { return 100; }
+int ap_version(void) { return 200; }
+
+void ap_debug_expire_waits(int on) { ap::g_expire_waits.store(on ? 1 : 0, std::memory_order_relaxed); }
 
 uint64_t ap_launch_count(void) { return (uint64_t)g_launches.load(std::memory_order_relaxed); }
 
@@ -159,6 +168,8 @@ ap_status build_mask_impl(const float *acc, int H, int Lq, int Lk, double keep_f
   if (workspace_bytes < ap_build_mask_workspace_bytes(H, Lq, Lk)) return AP_ERR_WORKSPACE;
   // the selection over a whole layer ranks ties by a 32-bit global index (h*Lq + i)*Lk + j
   if (per_layer && (int64_t)H * Lq * Lk > (int64_t)0xffffffffLL) return AP_ERR_UNSUPPORTED;
+  // one selection per head is one grid row per head (65 535 grid rows at most)
+  if (!per_layer && H > 65535) return AP_ERR_UNSUPPORTED;
   if (!have_device() || !device_error_word()) return AP_ERR_CUDA;
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -45,6 +45,15 @@ inline ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shap
   return AP_OK;
 }
 
+// Poll limit of the kernels' bounded waits and the test hook that makes one wait run out (see
+// ap_debug_expire_waits in ap.h): skip_arrive != 0 asks the next launches' producers to leave out
+// one arrival on a single-CTA grid.
+struct DebugKnobs {
+  uint32_t max_polls;
+  int skip_arrive;
+};
+DebugKnobs debug_knobs();
+
 // Kernels launched by this library in this process (see ap_launch_count in ap.h).
 void count_launches(int n);
 

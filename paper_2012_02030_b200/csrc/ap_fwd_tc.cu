@@ -1,44 +1,41 @@
-// Masked attention of Section 3.2 for bf16 tensors on the tcgen05 tensor cores.
+// Masked attention of Section 3.2 for bf16 / fp16 tensors on the tcgen05 tensor cores.
 //
-// Persistent kernel, one CTA per SM.  A work item is one (b, h, query tile of 128 rows); items
-// are handed out in pairs (a late and an early query tile of the same head), CTA c taking pairs
-// c, c + gridDim.x, ...  The CTA follows the schedule stored
-// with the tile list: the ROUNDS of the item's (h, qt) list row.  A round holds up to eight
-// non-empty groups of 16 key columns (slots), taken in list order from one or several key tiles,
-// together with the bitmap of exactly those columns; groups without a kept entry never appear, so
-// leaving them out is exact.  Per round:
+// Persistent kernel, one CTA per SM, TWO query tiles in flight per CTA.  A work item is one
+// (b, h, query tile of 128 rows).  The CTA runs two independent STREAMS; each stream owns one item
+// at a time, with its own Q tile, K/V stages and bitmaps in shared memory, its own score buffer S
+// and output accumulator O in tensor memory, its own producer warp, MMA-issuing warp and group of
+// four softmax warps.  Nothing but the tensor pipe, the special-function units and a work counter
+// is shared, so one stream's MMAs run under the other stream's softmax, and an item's first loads
+// and its epilogue run under the other stream's rounds.
+//
+// A stream follows the schedule stored with the tile list: the ROUNDS of the item's (h, qt) list
+// row.  A round holds up to eight non-empty groups of 16 key columns (slots), taken in list order
+// from one or several key tiles, together with the bitmap of exactly those columns; groups without
+// a kept entry never appear, so leaving them out is exact.  Per round:
 //   S  = Q K_round^T         tcgen05.mma, N = 16 * slots, fp32 accumulator in TMEM
-//   P  = exp2(c*S - c*m)     one thread per query row reads its S row from TMEM, replaces pruned
-//                            entries by -inf (the round's bitmap decides, exactly), keeps the
-//                            running reference m and sum l of an online softmax, rescales O when m
-//                            moved, and writes P as bf16 over S in TMEM
+//   P  = exp2(c*S - c*m)     one thread per query row reads its S row from TMEM in two halves of
+//                            64 columns (each an online-softmax step of its own), replaces pruned entries by -inf (the round's bitmap
+//                            decides, exactly), keeps the running reference m and sum l of an
+//                            online softmax, rescales O when m moved, and writes P as bf16 over S
 //   O += P V_round           tcgen05.mma, A = P from TMEM, B = V (MN-major), one K step of 16 keys
-//                            per slot
-// and at the item's last round O / l is written (zeros for rows that never saw a kept entry).
+//                            per slot; the first half's steps are issued as soon as the first
+//                            half of P is written, i.e. under the softmax of the second half
+// and after the item's last round O / l is written by the epilogue warps (zeros for rows that
+// never saw a kept entry) while the stream goes on with its next item.
 //
-// Everything a round needs arrives through one ring of stages in shared memory, filled by the
-// producer warp: the K and V rows of the round's slots (TMA boxes of 16..128 rows, slots whose key
-// rows follow one another are copied as one box), the round's bitmap (one bulk copy) and a word
-// that says how many slots there are and whether the round starts or ends an item.  The producer
-// runs ahead across item boundaries, so an item's first loads are hidden behind the previous
-// item's last rounds.  S is double-buffered in TMEM and the two kinds of MMA are issued by two
-// warps, each held back only by what it really depends on: S(g) = Q K^T waits for K(g) and for
-// O += P V of round g - 2 (the previous user of that S buffer), O += P(g) V for P(g) and V(g).
-// So the softmax threads find the next S ready when they finish a round.
+// Work distribution.  Items are numbered per CTA: item t is half t & 1 of unit
+// blockIdx.x + (t >> 1) * gridDim.x, a unit being the pair (query tile n_qt-1-j, query tile j) of
+// one (b, h).  The two producers draw item numbers from a counter in shared memory, so the stream
+// that finishes first takes the next item (a causal late tile has a long list and an early one a
+// short list).  Consecutive units belong to the same (b, h), so the CTAs running at any time share
+// a few heads' K and V in L2.
 //
-//
-// The softmax is shared by two groups of four warps.  The 32-column chunks of a round alternate
-// between them (chunk c belongs to group c & 1), and each group is an online softmax of its own:
-// its own reference m and sum l per query row and its own output accumulator in TMEM (O += P V
-// of a slot goes to the accumulator of the slot's group), so the groups never exchange anything
-// inside a round.  The item's epilogue merges the two partial results
-//   O = (a_0 O_0 + a_1 O_1) / (a_0 l_0 + a_1 l_1),   a_i = exp2(c (m_i - max(m_0, m_1))).
-//
-// Warp roles (480 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
-// TMEM lane), warp 8 producer, warp 9 issuer of S = Q K^T and TMEM owner, warp 10 issuer of
-// O += P V, warps 11-14 epilogue (the softmax groups hand (m, l) over and go on with the next
-// item while the epilogue warps wait for the item's last O += P V, merge and write).  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384 (d = 128); at d = 64 the pair (O_0, O_1) takes 128 columns and two items' pairs alternate at 256 and 384.  Every wait is bounded; a wait that expires
-// raises the device status word and the CTA winds down.
+// Warp roles (512 threads): warps 0-3 softmax of stream 0, warps 4-7 softmax of stream 1 (thread =
+// query row = TMEM lane), warps 8-11 epilogue (both streams), warps 12/13 producers, warps 14/15
+// MMA issuers (warp 14 owns the TMEM allocation).  TMEM (512 columns): S of stream x at column
+// 128 x, O of stream x at column 256 + 128 x (at d = 64 two accumulators of 64 columns alternate
+// there, so the next item's first O += P V need not wait for the epilogue).  Every wait is
+// bounded; a wait that expires raises the device status word and the CTA winds down.
 #include <math_constants.h>
 
 #include "ap_common.cuh"
@@ -50,37 +47,48 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 480;
-constexpr int kSoftmaxWarps = 8;       // two groups of four; barriers the softmax warps arrive on count warps
+constexpr int kThreads = 512;
 constexpr int kSubBytes = 128 * 128;  // one [128 rows][64 bf16] swizzled sub-tile
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kMaxPolls = 1u << 22;
-constexpr int kMaxStages = 4;
+constexpr bool kStagger = true;        // the streams' softmax phases keep apart (see the softmax warps)
+#ifndef AP_STAGGER_CYCLES
+#define AP_STAGGER_CYCLES 1200
+#endif
+constexpr uint32_t kStaggerCycles = AP_STAGGER_CYCLES;
+constexpr int kRing = 4;              // per stream: slots for the rounds' info words and bitmaps
 
-// per-stage word published by the producer
+// per-round word published by the producer
 constexpr uint32_t kInfoSlots = 15u;       // bits 0..3: slots of the round
 constexpr uint32_t kInfoFirst = 1u << 4;   // first round of its item
 constexpr uint32_t kInfoLast = 1u << 5;    // last round of its item
 constexpr uint32_t kInfoFull = 1u << 6;    // every entry of the round is kept: no bitmap was copied
-constexpr uint32_t kInfoStop = 1u << 7;    // no more work for this CTA
+constexpr uint32_t kInfoStop = 1u << 7;    // no more work for this stream
 
 // Shared-memory layout of a K or V stage.  Rows are the round's keys, a row's d elements are cut
 // into halves of 64 (128 bytes, the swizzle span).
 //   kSplit = false: [half][row / 8][8 rows][128 B]   one TMA box per half (3-D tensor map)
 //   kSplit = true:  [row / 8][half][8 rows][128 B]   d = 128 only: one box brings both halves (5-D map)
+// Per stream: kQBufs Q tiles, kStages K stages, kStages V stages.  Within a stream the chain
+// S(g) -> softmax(g) -> O += P V(g) -> S(g+1) is serial (P lives in S's columns), so one stage is
+// enough to keep the copies ahead: K(g+1) is copied under softmax(g), V(g+1) under S(g+1) and
+// softmax(g+1).  d = 64 has room for two.
 template <int D, bool kSplit>
 struct Cfg {
   static_assert(!kSplit || D == 128, "the split layout is for d = 128");
   static constexpr int kSub = D / 64;                 // halves per row
   static constexpr int kTileBytes = kSub * kSubBytes;
-  static constexpr int kStages = D == 64 ? 4 : 2;     // ring depth
-  static constexpr int kKOffset = 2 * kTileBytes;     // after the two Q buffers
+  static constexpr int kStages = D == 64 ? 2 : 1;     // K / V ring depth of a stream
+  static constexpr int kQBufs = D == 64 ? 2 : 1;
+  static constexpr int kOBufs = D == 64 ? 2 : 1;      // output accumulators of a stream in TMEM
+  static constexpr int kQOffset = 0;
+  static constexpr int kKOffset = kQBufs * kTileBytes;
   static constexpr int kVOffset = kKOffset + kStages * kTileBytes;
-  static constexpr int kBarOffset = kVOffset + kStages * kTileBytes;
-  static constexpr int kSmemBytes = kBarOffset + 17 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
+  static constexpr int kStreamBytes = kVOffset + kStages * kTileBytes;
+  static constexpr int kBarOffset = 2 * kStreamBytes;
   static constexpr int kHalfStride = kSplit ? 1024 : kSubBytes;          // half 0 -> half 1 of the same rows
   static constexpr int kSbo = kSplit ? 2048 : 1024;                      // one group of 8 rows -> the next
   static constexpr int kSlotStride = 2 * kSbo;                           // 16 rows (one slot) -> the next
+  static_assert(kRing >= kStages + 2, "info / bitmap ring too short for the K ring");
 };
 
 // Tensor maps of one launch: Q in whole-tile boxes; K and V in boxes of 16, 32, 64 and 128 rows.
@@ -90,24 +98,57 @@ struct FwdMaps {
   CUtensorMap v[4];
 };
 
-struct Shared {
-  alignas(16) uint32_t bitmap[kMaxStages][kTile][4];  // the round's bitmap, row r = words [r][0..3]
+struct StreamShared {
+  alignas(16) uint32_t bitmap[kRing][kTile][4];  // the round's bitmap, row r = words [r][0..3]
   uint64_t q_full[2], q_empty[2];
-  uint64_t k_full[kMaxStages], v_full[kMaxStages];    // K / V rows of the stage have landed
-  uint64_t b_full[kMaxStages];                        // info word and bitmap of the stage are valid
-  uint64_t k_empty[kMaxStages], v_empty[kMaxStages];  // S = Q K^T / O += P V of the stage has completed
-  uint64_t s_full[2], p_full[2];                      // per S buffer
-  uint64_t pv_done[2];                                // O += P V of a round has completed, per S buffer
-  uint64_t o_done[2], o_free[2];                      // per item: O complete / O read out by the epilogue
-                                                      // (one pair per set of accumulators)
-  uint64_t ml_ready[4];                               // per item: both groups have handed over (m, l)
-  float2 ml[4][2][kTile];                             // [item % 4][group][row] = (m, l)
-  int32_t ml_bh[4], ml_qt[4];                         // the item handed over (b * H + h, query tile); qt = -1: no more items
-  uint32_t info[kMaxStages];
-  int32_t item_bh[kMaxStages], item_qt[kMaxStages];   // the item a stage's round belongs to
+  uint64_t k_full[2], v_full[2];                 // K / V rows of the stage have landed
+  uint64_t k_empty[2], v_empty[2];               // S = Q K^T / O += P V of the stage has completed
+  uint64_t b_full[kRing];                        // info word and bitmap of the round are valid
+  uint64_t s_full;                               // S of a round is complete
+  uint64_t p_full[2];                            // P of a half round is written (one arrival per softmax warp)
+  uint64_t pv_done;                              // O += P V of a half round has completed
+  uint64_t o_done[2], o_free[2];                 // per accumulator: O complete / O read out by the epilogue
+  uint64_t ml_ready[4];                          // per item: the softmax warps have handed over l
+  float l[4][kTile];                             // [item % 4][row]: sum of the row's weights
+  int32_t ml_bh[4], ml_qt[4];                    // the item handed over (b * H + h, query tile); qt = -1: no more items
+  uint32_t info[kRing];
+  int32_t item_bh[kRing], item_qt[kRing];        // the item a round belongs to
+};
+
+struct Shared {
+  StreamShared st[2];
   uint32_t tmem_base;
   int abort_flag;
+  int next_item;  // work counter of the CTA
+  uint32_t sm_start[2];  // cycle count (low word) at which stream x's softmax warps last began a round
 };
+
+// Development aid: with -DAP_FWD_TRACE thread block 0 records cycle stamps of its roles
+// ([stream][role][round][point]; roles: 0 producer, 1 MMA issuer, 2..5 softmax warps), read back
+// through ap_debug_fwd_trace.  Compiled out otherwise.
+#ifdef AP_FWD_TRACE
+constexpr int kTraceRounds = 256, kTracePoints = 16;
+__device__ long long g_fwd_trace[2][6][kTraceRounds][kTracePoints];
+#define AP_TRACE(x, role, g, k)                                                              \
+  do {                                                                                       \
+    if (blockIdx.x == 0 && lane == 0 && (g) < (uint32_t)kTraceRounds) g_fwd_trace[x][role][g][k] = clock64(); \
+  } while (0)
+#else
+#define AP_TRACE(x, role, g, k) \
+  do {                          \
+  } while (0)
+#endif
+// the same from inside a single elected thread
+#ifdef AP_FWD_TRACE
+#define AP_TRACE1(x, role, g, k)                                                                      \
+  do {                                                                                                \
+    if (blockIdx.x == 0 && (g) < (uint32_t)kTraceRounds) g_fwd_trace[x][role][g][k] = clock64();      \
+  } while (0)
+#else
+#define AP_TRACE1(x, role, g, k) \
+  do {                           \
+  } while (0)
+#endif
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -115,25 +156,40 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
-// Bounded wait that also gives up as soon as another thread of the CTA has.
-__device__ __noinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag, unsigned *err) {
-  for (uint32_t i = 0; i < kMaxPolls; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (i > 1024) __nanosleep(64);
+__device__ __forceinline__ uint32_t lds_volatile(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_volatile(uint32_t addr, uint32_t v) {
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
+// What every bounded wait needs.
+struct WaitCtx {
+  volatile int *abort_flag;
+  unsigned *err;
+  uint32_t max_polls;
+};
+
+// Bounded wait that also gives up as soon as another thread of the CTA has.  Each poll lets the
+// hardware suspend the thread for up to a microsecond, so a waiting thread costs few issue slots.
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, const WaitCtx &w) {
+  for (uint32_t i = 0; i < w.max_polls; ++i) {
+    if (mbar_try_wait_for(bar, parity, 1000u)) return true;
+    if (*w.abort_flag) return false;
   }
-  *abort_flag = 1;
-  atomicOr(err, kDevErrTimeout);
+  *w.abort_flag = 1;
+  atomicOr(w.err, kDevErrTimeout);
   return false;
 }
 
 // The same wait for a whole (converged) warp: one lane polls - 32 lanes polling one barrier would
 // serialise - and the outcome is shared.
 template <int kPollLane = 0>
-__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag,
-                                          unsigned *err) {
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int lane, const WaitCtx &w) {
   bool ok = true;
-  if (lane == kPollLane && !mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, abort_flag, err);
+  if (lane == kPollLane && !mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, w);
   return __shfl_sync(0xffffffffu, ok ? 1 : 0, kPollLane) != 0;
 }
 
@@ -158,45 +214,107 @@ __device__ __forceinline__ float2 unpack16x2(uint32_t pk) {
   }
 }
 
+// One online-softmax step of a thread's query row over kChunks 32-column chunks of S at `tmem_b`:
+// pruned entries (bitmap bit 0) are replaced by -inf (exp2 of -inf is exactly 0), the row maximum
+// is taken over kept entries, the exponent's reference follows it lazily, P = exp2(c*S - c*m) is
+// written as 16-bit values over the first half of each chunk's columns of S (not yet waited for).
+// Returns the new reference, the new sum and the factor by which the old sum (and the output
+// accumulated so far) had to be scaled.
+struct HalfStep {
+  float m, l, alpha;
+};
+template <int kChunks, bool kMasked, bool kF16>
+__device__ __forceinline__ HalfStep softmax_half(uint32_t tmem_b, uint2 bw, float m, float l, float scale_log2,
+                                                 float ref_slack) {
+  uint32_t xs[32 * kChunks];
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) tmem_ld32(tmem_b + 32 * c, &xs[32 * c]);
+  tmem_wait_ld();
+  if (kMasked) {
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      const uint32_t w = c == 0 ? bw.x : bw.y;
+#pragma unroll
+      for (int e = 0; e < 32; ++e) xs[32 * c + e] = ((w >> e) & 1u) ? xs[32 * c + e] : 0xff800000u;  // -inf
+    }
+  }
+  float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
+#pragma unroll
+  for (int e = 0; e < 32 * kChunks; e += 8) {
+    mx0 = fmax3(mx0, __uint_as_float(xs[e]), __uint_as_float(xs[e + 1]));
+    mx1 = fmax3(mx1, __uint_as_float(xs[e + 2]), __uint_as_float(xs[e + 3]));
+    mx2 = fmax3(mx2, __uint_as_float(xs[e + 4]), __uint_as_float(xs[e + 5]));
+    mx3 = fmax3(mx3, __uint_as_float(xs[e + 6]), __uint_as_float(xs[e + 7]));
+  }
+  const float half_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+  // The reference moves only when the maximum outgrows it by more than 2^8 in the exp2 domain
+  // (weights stay <= 256, well inside bf16 and fp32 range), which saves most rescales of O.
+  // O / l does not depend on the reference.
+  const bool move = half_max > m + ref_slack;   // also true for the first kept entry (m = -inf)
+  const float m_new = move ? half_max : m;
+  const float m_safe = m_new == -CUDART_INF_F ? 0.f : m_new;
+  const float alpha = move ? ex2_approx((m - m_safe) * scale_log2) : 1.f;  // 0 when m was -inf
+  const float neg_mc = -m_safe * scale_log2;
+  float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const float p0 = ex2_approx(fmaf(__uint_as_float(xs[32 * c + 2 * e]), scale_log2, neg_mc));
+      const float p1 = ex2_approx(fmaf(__uint_as_float(xs[32 * c + 2 * e + 1]), scale_log2, neg_mc));
+      pk[e] = pack16x2<kF16>(p0, p1);
+      // the row sum is taken over the rounded weights the MMA will use, so that
+      // O / l is an exact convex combination of V rows whatever the rounding of P
+      const float2 pr = unpack16x2<kF16>(pk[e]);
+      sum0 += pr.x;
+      sum1 += pr.y;
+    }
+    tmem_st16(tmem_b + 32 * c, pk);
+  }
+  return HalfStep{m_new, l * alpha + (sum0 + sum1), alpha};
+}
+
+// dbg_skip != 0 (test hook, see ap_debug_expire_waits): the producer of stream 0 leaves out the
+// copies and the arrival of its first round, so that the waits on it run out.
 template <int D, bool kSplit, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
               const int32_t *__restrict__ round_ptr, const int32_t *__restrict__ round_rows,
               const uint8_t *__restrict__ round_info, const uint32_t *__restrict__ round_bitmap, int B, int H,
-              int Lq, int n_qt, float scale_log2, unsigned *err) {
+              int Lq, int n_qt, float scale_log2, unsigned *err, uint32_t max_polls, int dbg_skip) {
   using C = Cfg<D, kSplit>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
       reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char *q_s = smem;
-  unsigned char *k_s = smem + C::kKOffset;
-  unsigned char *v_s = smem + C::kVOffset;
   Shared *sh = reinterpret_cast<Shared *>(smem + C::kBarOffset);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&sh->q_full[i], 1);
-      mbar_init(&sh->q_empty[i], 1);
-      mbar_init(&sh->s_full[i], 1);
-      mbar_init(&sh->p_full[i], kSoftmaxWarps);
+    for (int x = 0; x < 2; ++x) {
+      StreamShared &ss = sh->st[x];
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&ss.q_full[i], 1);
+        mbar_init(&ss.q_empty[i], 1);
+        mbar_init(&ss.k_full[i], 1);
+        mbar_init(&ss.v_full[i], 1);
+        mbar_init(&ss.k_empty[i], 1);
+        mbar_init(&ss.v_empty[i], 1);
+        mbar_init(&ss.p_full[i], 4);  // softmax warps of the stream
+        mbar_init(&ss.o_done[i], 1);
+        mbar_init(&ss.o_free[i], 4);  // epilogue warps
+      }
+      for (int i = 0; i < kRing; ++i) mbar_init(&ss.b_full[i], 1);
+      mbar_init(&ss.s_full, 1);
+      mbar_init(&ss.pv_done, 1);
+      for (int i = 0; i < 4; ++i) mbar_init(&ss.ml_ready[i], 4);
     }
-    for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(&sh->k_full[s], 1);
-      mbar_init(&sh->v_full[s], 1);
-      mbar_init(&sh->k_empty[s], 1);
-      mbar_init(&sh->v_empty[s], 1);
-    }
-    for (int s = 0; s < kMaxStages; ++s) mbar_init(&sh->b_full[s], 1);
-    mbar_init(&sh->pv_done[0], 1);
-    mbar_init(&sh->pv_done[1], 1);
-    for (int i = 0; i < 2; ++i) mbar_init(&sh->o_done[i], 1);
-    for (int i = 0; i < 2; ++i) mbar_init(&sh->o_free[i], 4);  // epilogue warps
-    for (int i = 0; i < 4; ++i) mbar_init(&sh->ml_ready[i], kSoftmaxWarps);
     sh->abort_flag = 0;
+    sh->next_item = 0;
+    sh->sm_start[0] = sh->sm_start[1] = (uint32_t)clock64() - 0x40000000u;
     fence_mbar_init();
   }
-  if (warp == 9) {
+  if (warp == 14) {
     tmem_alloc(&sh->tmem_base, kTmemCols);
     tmem_relinquish();
   }
@@ -204,44 +322,46 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sh->tmem_base;
-  // The two groups' accumulators of an item.  At d = 64 they take 128 columns together and TMEM has
-  // room for two items' worth: items alternate between them, so that the next item's first
-  // O += P V need not wait until the epilogue has read this item's result.
-  constexpr uint32_t kOBufs = D == 64 ? 2u : 1u;
-  constexpr uint32_t kOGroup = D == 64 ? 64u : 128u;  // columns from group 0's accumulator to group 1's
-  const uint32_t tmem_o = tmem + 256;
-  auto o_of_item = [&](uint32_t n) { return tmem_o + (kOBufs == 2u ? 128u * (n & 1u) : 0u); };
-  volatile int *abort_flag = &sh->abort_flag;
-  const int item_step = (int)gridDim.x;
+  // Output accumulator of the n-th item of stream x.
+  auto o_addr = [&](int x, uint32_t n) {
+    return tmem + 256u + 128u * (uint32_t)x + (C::kOBufs == 2 ? 64u * (n & 1u) : 0u);
+  };
+  const WaitCtx wc{&sh->abort_flag, err, max_polls};
+  // producers: the copies armed last (round numbers; -1: none), for the wind-down after an expired wait
+  int armed_q = -1, armed_k = -1, armed_v = -1;
 
-  if (warp == 8) {
-    // ------------------------------------------------------------ producer
+  if (warp == 12 || warp == 13) {
+    // ------------------------------------------------------------ producer of stream x
+    const int x = warp - 12;
+    StreamShared &ss = sh->st[x];
+    unsigned char *q_s = smem + x * C::kStreamBytes + C::kQOffset;
+    unsigned char *k_s = smem + x * C::kStreamBytes + C::kKOffset;
+    unsigned char *v_s = smem + x * C::kStreamBytes + C::kVOffset;
     if (lane < 4) {
       prefetch_tensormap(&maps.k[lane]);
       prefetch_tensormap(&maps.v[lane]);
     }
     if (lane == 4) prefetch_tensormap(&maps.q);
     bool ok = true;
-    uint32_t g = 0, n = 0;   // rounds / non-empty items so far
-    int armed_q = -1;        // non-empty item whose Q copy was armed last
-    // Work is handed out in units of two items of one (b, h): query tile n_qt - 1 - j and query
-    // tile j.  Under a causal mask a late tile has a long list and an early one a short list, so
-    // units weigh about the same; and because consecutive units belong to the same (b, h), the
-    // CTAs running at any time share a few heads' K and V, which then stay in L2.  The t-th item
-    // of this CTA is half t & 1 of unit blockIdx.x + (t >> 1) * gridDim.x.
+    uint32_t g = 0, n = 0;   // rounds / non-empty items of this stream so far
     const int n_half = (n_qt + 1) / 2, n_units = B * H * n_half;
+    const int item_step = (int)gridDim.x;
     struct ItemRef {
       int bh, qt, rho0, rho1;  // rounds [rho0, rho1): loaded here, first read when the item begins
       bool in_range, exists;   // !exists: no such item (the unit's halves coincide)
     };
-    // (called for t = 0, 1, 2, ... in turn: the unit's (j, bh, h = bh % H) are stepped from one unit
-    // of this CTA to the next instead of divided out of the unit number every time; this warp's
-    // instruction stream is what short items wait for)
-    int cur_u = (int)blockIdx.x, cur_j = cur_u % n_half, cur_bh = cur_u / n_half, cur_h = cur_bh % H;
+    // The unit's (j, bh, h = bh % H) are stepped from the unit last looked at to the one wanted
+    // instead of divided out of the unit number (item numbers only grow).
+    int cur_k = 0, cur_u = (int)blockIdx.x, cur_j = cur_u % n_half, cur_bh = cur_u / n_half, cur_h = cur_bh % H;
     const int step_j = item_step % n_half, step_bh = item_step / n_half, step_h = step_bh % H;
-    auto item_ref = [&](int t) {
-      ItemRef it;
-      if (t >= 2 && !(t & 1)) {  // the next unit
+    // Draws the next item number of the CTA and looks its rounds up.
+    auto next_item = [&]() {
+      int t = 0;
+      if (lane == 0) t = atomicAdd(&sh->next_item, 1);
+      t = __shfl_sync(0xffffffffu, t, 0);
+      const int k = t >> 1;
+      while (cur_k < k && cur_u < n_units) {
+        ++cur_k;
         cur_u += item_step;
         cur_j += step_j;
         cur_bh += step_bh;
@@ -253,8 +373,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         }
         if (cur_h >= H) cur_h -= H;
       }
-      const int u = cur_u;
-      it.in_range = u < n_units;
+      ItemRef it;
+      it.in_range = cur_k == k && cur_u < n_units;
       it.bh = 0, it.qt = 0, it.rho0 = 0, it.rho1 = 0, it.exists = false;
       if (it.in_range) {
         const int j = cur_j;
@@ -279,15 +399,8 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
           tma_load_3d(stage + s * kSubBytes + q * C::kSlotStride, m, bar, 64 * s, row, bh);
       }
     };
-    // Ring discipline.  K and V of round g go to stage g % kStages, its info word and bitmap to
-    // slot g % kMaxStages.  K may be overwritten once S = Q K^T of round g - kStages has completed
-    // (k_empty), V once O += P V of that round has (v_empty).  The info slot last served round
-    // g - kMaxStages, whose softmax must be over: with kStages == kMaxStages that is what v_empty
-    // says; with a ring of two, S of round g - 2 could only be computed after O += P V of round
-    // g - 4 was issued, i.e. after that round's softmax, so k_empty implies it.
-    static_assert(C::kStages == kMaxStages || C::kStages == 2, "ring discipline");
     auto wait_free = [&](uint64_t *bar, uint32_t ph) {
-      if (lane == 0) ok = wait_or_abort(bar, ph ^ 1u, abort_flag, err);
+      if (lane == 0) ok = wait_or_abort(bar, ph ^ 1u, wc);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     };
     // A run of slots (key rows following one another) is copied by the lane of its first slot, in
@@ -302,49 +415,33 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         left -= 1 << lg;
       }
     };
-    // V of a round is copied one round later than its K: K only needs S = Q K^T of the round that
-    // used the stage before to be over, V needs that round's O += P V, which comes much later;
-    // issued in round order, the V copy would hold back the next round's K.
-    bool pv_valid = false;
-    int pv_st = 0, pv_ng = 0, pv_row = 0, pv_run = 0, pv_bh = 0;
-    uint32_t pv_ph = 0;
-    auto issue_v = [&]() {
-      if (C::kStages != kMaxStages) wait_free(&sh->v_empty[pv_st], pv_ph);
-      if (!ok) return;
-      if (lane == 0) mbar_arrive_expect_tx(&sh->v_full[pv_st], (uint32_t)pv_ng * 16u * D * 2u);
-      __syncwarp();
-      load_run(v_s + pv_st * C::kTileBytes, maps.v, &sh->v_full[pv_st], pv_row, pv_run, pv_bh);
-      pv_valid = false;
-    };
-    // the rounds of an item are looked up two items ahead: the loads of item t + 2 are issued when
-    // item t begins and their results first touched when item t + 1 does
-    ItemRef next = item_ref(0);
-    ItemRef next2 = item_ref(1);
-    // ... and the slot rows and info byte of its first round while the current item is under way
-    int pf_t = -1, pf_row = -1;
+    // Items are drawn one ahead: the look-ups of the next item are in flight while this one runs,
+    // and the slot rows and info byte of its first round are fetched during this item's last round.
+    ItemRef next = next_item();
+    int pf_valid = 0, pf_row = -1;
     uint32_t pf_info = 0u;
-    for (int t = 0; next.in_range && ok; ++t) {
+    while (next.in_range && ok) {
       const ItemRef cur = next;
-      next = next2;
-      next2 = item_ref(t + 2);
+      next = next_item();
       if (!cur.exists) continue;
       const int bh = cur.bh, qt = cur.qt, rho0 = cur.rho0, n_rounds = cur.rho1 - cur.rho0;
       if (n_rounds == 0) {
         // nothing kept in this query tile: its output rows are zero (nobody else sees the item)
         const int rows = min(kTile, Lq - qt * kTile);
         uint4 *dst = reinterpret_cast<uint4 *>(O + ((size_t)bh * Lq + (size_t)qt * kTile) * D);
-        for (int x = lane; x < rows * (D / 8); x += 32) dst[x] = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = lane; i < rows * (D / 8); i += 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
         continue;
       }
-      // Q of this item into its buffer (free once the last S = Q K^T of item n - 2 has completed)
-      const int qb = (int)(n & 1u);
+      // Q of this item into its buffer (free once the last S = Q K^T of item n - kQBufs has completed)
+      const int qb = (int)(n % C::kQBufs);
+      const uint32_t q_use = n / C::kQBufs;
       if (lane == 0) {
-        ok = wait_or_abort(&sh->q_empty[qb], ((n >> 1) & 1u) ^ 1u, abort_flag, err);
+        ok = wait_or_abort(&ss.q_empty[qb], (q_use & 1u) ^ 1u, wc);
         if (ok) {
-          mbar_arrive_expect_tx(&sh->q_full[qb], C::kTileBytes);
+          mbar_arrive_expect_tx(&ss.q_full[qb], C::kTileBytes);
 #pragma unroll
           for (int s = 0; s < C::kSub; ++s)
-            tma_load_3d(q_s + qb * C::kTileBytes + s * kSubBytes, &maps.q, &sh->q_full[qb], 64 * s, qt * kTile, bh);
+            tma_load_3d(q_s + qb * C::kTileBytes + s * kSubBytes, &maps.q, &ss.q_full[qb], 64 * s, qt * kTile, bh);
           armed_q = (int)n;
         }
       }
@@ -353,18 +450,19 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       // slot rows (lanes 0..7) and info byte of a round are fetched one round ahead
       int next_row = pf_row;
       uint32_t next_info = pf_info;
-      if (pf_t != t) {
+      if (!pf_valid) {
         next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)rho0 * 8 + lane) : -1;
         next_info = ldg_now_u8(round_info + rho0);
       }
+      pf_valid = 0;
       for (int v = 0; v < n_rounds && ok; ++v, ++g) {
         const int row = next_row;
         const uint32_t rinfo = next_info;
         if (v + 1 < n_rounds) {
           next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)(rho0 + v + 1) * 8 + lane) : -1;
           next_info = ldg_now_u8(round_info + rho0 + v + 1);
-        } else if (next.exists && next.rho1 > next.rho0) {
-          pf_t = t + 1;
+        } else if (next.in_range && next.exists && next.rho1 > next.rho0) {
+          pf_valid = 1;
           pf_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)next.rho0 * 8 + lane) : -1;
           pf_info = ldg_now_u8(round_info + next.rho0);
         }
@@ -378,345 +476,367 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         const uint32_t heads = __ballot_sync(0xffffffffu, head);
         const uint32_t later = lane < 31 ? heads >> (lane + 1) : 0u;
         const int run = head ? (later ? __ffs((int)later) : ng - lane) : 0;  // slots in this lane's run
-        const int si = (int)(g % kMaxStages);
-        wait_free(&sh->k_empty[st], ph);
-        if (ok && C::kStages == kMaxStages) wait_free(&sh->v_empty[st], ph);
+        const int si = (int)(g % kRing);
+        // K of round g: its stage is free once S of round g - kStages has completed.  The info slot
+        // last served round g - kRing, whose softmax was over before S of round g - kStages was issued.
+        wait_free(&ss.k_empty[st], ph);
         if (!ok) break;
+        AP_TRACE(x, 0, g, 0);
         const uint32_t bytes = (uint32_t)ng * 16u * D * 2u;
+        const bool skip = dbg_skip != 0 && x == 0 && g == 0;
         if (lane == 0) {
-          sh->info[si] = (uint32_t)ng | (v == 0 ? kInfoFirst : 0u) | (v + 1 == n_rounds ? kInfoLast : 0u) |
-                         (full ? kInfoFull : 0u);
-          sh->item_bh[si] = bh;
-          sh->item_qt[si] = qt;
-          mbar_arrive_expect_tx(&sh->k_full[st], bytes);
-          if (full) {
-            mbar_arrive(&sh->b_full[si]);
-          } else {
-            mbar_arrive_expect_tx(&sh->b_full[si], kBitmapWords * 4);
-            bulk_load(&sh->bitmap[si][0][0], round_bitmap + (size_t)(rho0 + v) * kBitmapWords, kBitmapWords * 4,
-                      &sh->b_full[si]);
+          ss.info[si] = (uint32_t)ng | (v == 0 ? kInfoFirst : 0u) | (v + 1 == n_rounds ? kInfoLast : 0u) |
+                        (full ? kInfoFull : 0u);
+          ss.item_bh[si] = bh;
+          ss.item_qt[si] = qt;
+          if (!skip) {
+            mbar_arrive_expect_tx(&ss.k_full[st], bytes);
+            armed_k = (int)g;
+            if (full) {
+              mbar_arrive(&ss.b_full[si]);
+            } else {
+              mbar_arrive_expect_tx(&ss.b_full[si], kBitmapWords * 4);
+              bulk_load(&ss.bitmap[si][0][0], round_bitmap + (size_t)(rho0 + v) * kBitmapWords, kBitmapWords * 4,
+                        &ss.b_full[si]);
+            }
           }
         }
         __syncwarp();
-        load_run(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st], row, run, bh);
-        if (pv_valid) issue_v();
+        if (!skip) load_run(k_s + st * C::kTileBytes, maps.k, &ss.k_full[st], row, run, bh);
+        AP_TRACE(x, 0, g, 1);
+        // V of round g: its stage is free once O += P V of round g - kStages has completed, which is
+        // before S of round g + 1 - kStages, the next thing this warp waits for
+        wait_free(&ss.v_empty[st], ph);
         if (!ok) break;
-        pv_valid = true;
-        pv_st = st, pv_ph = ph, pv_ng = ng, pv_row = row, pv_run = run, pv_bh = bh;
+        AP_TRACE(x, 0, g, 2);
+        if (!skip) {
+          if (lane == 0) {
+            mbar_arrive_expect_tx(&ss.v_full[st], bytes);
+            armed_v = (int)g;
+          }
+          __syncwarp();
+          load_run(v_s + st * C::kTileBytes, maps.v, &ss.v_full[st], row, run, bh);
+        }
+        AP_TRACE(x, 0, g, 3);
       }
       ++n;
     }
-    if (ok && pv_valid) issue_v();
-    // no more work: one more stage carries the stop word
+    // no more work: one more round carries the stop word
     if (ok) {
       const int st = (int)(g % C::kStages);
       const uint32_t ph = (g / C::kStages) & 1u;
-      wait_free(&sh->k_empty[st], ph);
-      if (ok && C::kStages == kMaxStages) wait_free(&sh->v_empty[st], ph);
+      wait_free(&ss.k_empty[st], ph);
       if (ok && lane == 0) {
-        sh->info[g % kMaxStages] = kInfoStop;
-        mbar_arrive(&sh->k_full[st]);
-        mbar_arrive(&sh->b_full[g % kMaxStages]);
+        ss.info[g % kRing] = kInfoStop;
+        mbar_arrive(&ss.k_full[st]);
+        mbar_arrive(&ss.b_full[g % kRing]);
       }
     }
-    if (lane == 0 && *abort_flag) {
-      // winding down: wait (bounded) for the copies armed most recently
-      if (armed_q >= 0) mbar_wait(&sh->q_full[armed_q & 1], ((uint32_t)armed_q >> 1) & 1u, 1u << 16);
-      for (uint32_t a = g > (uint32_t)C::kStages ? g - C::kStages : 0; a <= g; ++a) {
-        mbar_wait(&sh->k_full[a % C::kStages], (a / C::kStages) & 1u, 1u << 16);
-        mbar_wait(&sh->v_full[a % C::kStages], (a / C::kStages) & 1u, 1u << 16);
-        mbar_wait(&sh->b_full[a % kMaxStages], (a / kMaxStages) & 1u, 1u << 16);
+  } else if (warp >= 14) {
+    // ------------------------------------------------------------ MMA issuer of stream x
+    // One thread walks the stream's rounds.  Per round it issues O += P V in two halves as the
+    // softmax hands P over, and right behind the second half the next round's S = Q K^T, whose
+    // operands it has checked for while the softmax was busy.  The tensor pipe runs one thread's
+    // instructions in order, so that S may overwrite the columns P was read from without a wait in
+    // between.  Every instruction between a hand-over and the MMAs it releases is on the stream's
+    // critical path, so this thread's code is kept short: descriptors are prepared once, nothing is
+    // shared with other lanes.
+    const int x = warp - 14;
+    if (lane == 0) {
+      StreamShared &ss = sh->st[x];
+      const uint32_t q_addr = smem_u32(smem + x * C::kStreamBytes + C::kQOffset);
+      const uint32_t k_addr = smem_u32(smem + x * C::kStreamBytes + C::kKOffset);
+      const uint32_t v_addr = smem_u32(smem + x * C::kStreamBytes + C::kVOffset);
+      const uint32_t tmem_s = tmem + 128u * (uint32_t)x;
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true, kF16);
+      bool ok = true;
+      uint32_t n = 0;  // non-empty items finished so far
+      auto wait = [&](uint64_t *bar, uint32_t parity) {
+        if (!mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, wc);
+        return ok;
+      };
+      // waits for K of round g (and Q if the round opens an item) and returns the round's info word
+      auto operands_of = [&](uint32_t g) {
+        if (!wait(&ss.k_full[g % C::kStages], (g / C::kStages) & 1u)) return kInfoStop;
+        const uint32_t info = ss.info[g % kRing];
+        if (!(info & kInfoStop) && (info & kInfoFirst)) {
+          // the item this round opens: item n, or n + 1 while item n's last round is still under way
+          const uint32_t item = n + (g > 0 && (ss.info[(g - 1) % kRing] & kInfoLast) ? 1u : 0u);
+          if (!wait(&ss.q_full[item % C::kQBufs], (item / C::kQBufs) & 1u)) return kInfoStop;
+        }
+        return info;
+      };
+      // Low descriptor words of every operand tile this thread will ever name (the stages are few).
+      uint32_t q_lo[C::kQBufs][D / 16], k_lo[C::kStages][D / 16], v_lo[C::kStages][8];
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) {
+        const int sub = ks / 4, off = (ks % 4) * 32;  // D/16 steps of K = 16 (32 bytes inside the swizzled rows)
+#pragma unroll
+        for (int b = 0; b < C::kQBufs; ++b)
+          q_lo[b][ks] = smem_desc_lo(q_addr + b * C::kTileBytes + sub * kSubBytes + off, 16);
+#pragma unroll
+        for (int b = 0; b < C::kStages; ++b)
+          k_lo[b][ks] = smem_desc_lo(k_addr + b * C::kTileBytes + sub * C::kHalfStride + off, 16);
       }
-    }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------ issuer of S = Q K^T
-    // The whole warp walks the rounds in lockstep (one lane polls the barriers, another, elected
-    // one issues the tcgen05 instructions; the state is warp-uniform).
-    const uint32_t q_addr = smem_u32(q_s), k_addr = smem_u32(k_s);
-    bool ok = true;
-    uint32_t n = 0;  // non-empty items started so far
-    for (uint32_t g = 0; ok; ++g) {
-      const int st = (int)(g % C::kStages);
-      const uint32_t sb = g & 1u;
-      ok = warp_wait<31>(&sh->k_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
-      if (!ok) break;
-      const uint32_t info = sh->info[g % kMaxStages];
-      if (info & kInfoStop) break;
-      const int ng = (int)(info & kInfoSlots);
-      const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
-      const int qb = (int)(n & 1u);
-      if (first) ok = warp_wait<31>(&sh->q_full[qb], (n >> 1) & 1u, lane, abort_flag, err);
-      // S[sb] still holds P of round g - 2 until that round's O += P V (issued by another warp) has
-      // completed
-      if (ok && g >= 2) ok = warp_wait<31>(&sh->pv_done[sb], ((g >> 1) - 1u) & 1u, lane, abort_flag, err);
-      if (!ok) break;
-      tc_fence_after_sync();
-      // N = 16 ng, D/16 steps of K = 16 (32 bytes inside the swizzled rows)
-      if (elect_one()) {
-        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false, kF16);
-        const uint32_t q_buf = q_addr + qb * C::kTileBytes, k_stage = k_addr + st * C::kTileBytes;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+        for (int b = 0; b < C::kStages; ++b)
+          v_lo[b][ks] = smem_desc_lo(v_addr + b * C::kTileBytes + ks * C::kSlotStride, C::kHalfStride);
+      constexpr uint32_t q_hi = smem_desc_hi_sw128(1024), kv_hi = smem_desc_hi_sw128(C::kSbo);
+      // S = Q K^T of round g of item `item` (N = 16 ng), announced on s_full first: the softmax waits for it
+      auto issue_s = [&](uint32_t g, uint32_t info, uint32_t item) {
+        const int st = (int)(g % C::kStages), qb = (int)(item % C::kQBufs);
+        const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * (int)(info & kInfoSlots), false, false, kF16);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const int sub = ks / 4, off = (ks % 4) * 32;
-          mma_ss(tmem + 128u * sb, smem_desc_sw128(q_buf + sub * kSubBytes + off, 16, 1024),
-                 smem_desc_sw128(k_stage + sub * C::kHalfStride + off, 16, C::kSbo), idesc_qk, ks > 0);
+          const uint32_t ql = C::kQBufs == 2 && qb ? q_lo[C::kQBufs - 1][ks] : q_lo[0][ks];
+          const uint32_t kl = C::kStages == 2 && st ? k_lo[C::kStages - 1][ks] : k_lo[0][ks];
+          mma_ss(tmem_s, smem_desc_join(ql, q_hi), smem_desc_join(kl, kv_hi), idesc_qk, ks > 0);
         }
-        mma_commit(&sh->k_empty[st]);
-        if (last) mma_commit(&sh->q_empty[qb]);
-        mma_commit(&sh->s_full[sb]);
+        mma_commit(&ss.s_full);
+        mma_commit(&ss.k_empty[st]);
+        if (info & kInfoLast) mma_commit(&ss.q_empty[qb]);
+      };
+      uint32_t info = operands_of(0);
+      if (ok && !(info & kInfoStop)) {
+        tc_fence_after_sync();
+        issue_s(0, info, 0);
+        AP_TRACE1(x, 1, 0u, 0);
       }
-      __syncwarp();
-      if (last) ++n;
-    }
-  } else if (warp == 10) {
-    // ------------------------------------------------------------ issuer of O += P V
-    constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true, kF16);
-    const uint32_t v_addr = smem_u32(v_s);
-    bool ok = true;
-    uint32_t n = 0;                          // non-empty items started so far
-    uint32_t started0 = 0u, started1 = 0u;  // the item's O_0 / O_1 holds a partial result already
-    for (uint32_t g = 0; ok; ++g) {
-      const int st = (int)(g % C::kStages);
-      const uint32_t sb = g & 1u;
-      ok = warp_wait<31>(&sh->b_full[g % kMaxStages], (g / kMaxStages) & 1u, lane, abort_flag, err);
-      if (!ok) break;
-      const uint32_t info = sh->info[g % kMaxStages];
-      if (info & kInfoStop) break;
-      const int ng = (int)(info & kInfoSlots);
-      const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
-      // (what is ready early first; P, which the softmax has just finished, last)
-      ok = warp_wait<31>(&sh->v_full[st], (g / C::kStages) & 1u, lane, abort_flag, err);
-      // the first round of an item overwrites O: the epilogue of the previous item must have read it
-      if (ok && first && n >= kOBufs)
-        ok = warp_wait<31>(&sh->o_free[kOBufs == 2u ? (n & 1u) : 0u], ((n / kOBufs) - 1u) & 1u, lane, abort_flag, err);
-      if (ok) ok = warp_wait<31>(&sh->p_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
-      if (!ok) break;
-      tc_fence_after_sync();
-      // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
-      // 16 columns of that chunk of S (each group stays inside its own chunks), so slot q's
-      // eight columns of P start at column 32 (q / 2) + 8 (q % 2).
-      // Slots 0, 1, 4, 5 (chunks 0 and 2) belong to softmax group 0 and add to O_0, the others to
-      // O_1; a group's first step of an item overwrites its accumulator.
-      if (first) started0 = started1 = 0u;
-      if (elect_one()) {
-        const uint32_t v_stage = v_addr + st * C::kTileBytes;
-        const uint32_t p_base = tmem + 128u * sb;
+      for (uint32_t g = 0; ok && !(info & kInfoStop); ++g) {
+        const int st = (int)(g % C::kStages);
+        const uint32_t ph = (g / C::kStages) & 1u;
+        const int ng = (int)(info & kInfoSlots);
+        const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
+        // O += P V.  What is ready early first; P, which the softmax has just finished, last.
+        if (!wait(&ss.v_full[st], ph)) break;
+        // the first round of an item overwrites O: the epilogue of the item that used the accumulator
+        // before must have read it
+        const uint32_t ob = C::kOBufs == 2 ? (n & 1u) : 0u;
+        if (first && n >= (uint32_t)C::kOBufs && !wait(&ss.o_free[ob], ((n / C::kOBufs) - 1u) & 1u)) break;
+        const uint32_t o_acc = o_addr(x, n);
+        AP_TRACE1(x, 1, g, 2);
+        // One K step of 16 keys per slot.  P (16-bit) of a 32-column chunk is written over the
+        // first 16 columns of that chunk of S, so slot q's eight columns of P start at column
+        // 32 (q / 2) + 8 (q % 2).  The item's first step overwrites the accumulator.
+        auto issue_pv = [&](int half) {
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          if (ks < ng) {
-            const int grp = (ks >> 1) & 1;
-            const uint32_t acc = ks == 0 ? started0 : ks == 2 ? started1 : 1u;  // slots 0 / 2 open their group
-            mma_ts(o_of_item(n) + kOGroup * grp, p_base + 32 * (ks >> 1) + 8 * (ks & 1),
-                   smem_desc_sw128(v_stage + ks * C::kSlotStride, C::kHalfStride, C::kSbo), idesc_pv, acc);
+          for (int ks = 4 * half; ks < 4 * half + 4; ++ks) {
+            const uint32_t vl = C::kStages == 2 && st ? v_lo[C::kStages - 1][ks] : v_lo[0][ks];
+            if (ks < ng)
+              mma_ts(o_acc, tmem_s + 32 * (ks >> 1) + 8 * (ks & 1), smem_desc_join(vl, kv_hi), idesc_pv,
+                     (first && ks == 0) ? 0u : 1u);
           }
-        }
-        mma_commit(&sh->v_empty[st]);
-        mma_commit(&sh->pv_done[sb]);
-        if (last) mma_commit(&sh->o_done[kOBufs == 2u ? (n & 1u) : 0u]);
+        };
+        if (!wait(&ss.p_full[0], g & 1u)) break;
+        AP_TRACE1(x, 1, g, 3);
+        tc_fence_after_sync();
+        issue_pv(0);
+        mma_commit(&ss.pv_done);
+        // while the softmax works on the second half: the next round's operands (they do not
+        // depend on this round's P)
+        const uint32_t info_next = operands_of(g + 1);
+        if (!ok) break;
+        AP_TRACE1(x, 1, g, 6);
+        if (last) ++n;
+        if (!wait(&ss.p_full[1], g & 1u)) break;
+        AP_TRACE1(x, 1, g, 4);
+        tc_fence_after_sync();
+        issue_pv(1);
+        if (!(info_next & kInfoStop)) issue_s(g + 1, info_next, n);
+        AP_TRACE1(x, 1, g + 1, 0);
+        // (completion of these is signalled once the MMAs issued so far, S included, are through:
+        // nobody waits for them as urgently as the softmax for S)
+        mma_commit(&ss.pv_done);
+        mma_commit(&ss.v_empty[st]);
+        if (last) mma_commit(&ss.o_done[ob]);
+        AP_TRACE1(x, 1, g, 5);
+        info = info_next;
       }
-      __syncwarp();
-      started0 = 1u;
-      if (ng > 2) started1 = 1u;
-      if (last) ++n;
     }
+    __syncwarp();
   } else if (warp < 8) {
-    // ------------------------------------------------------------ softmax
-    const int grp = warp >> 2;               // softmax group: chunks grp and grp + 2 of every round
+    // ------------------------------------------------------------ softmax of stream x
+    const int x = warp >> 2;
+    StreamShared &ss = sh->st[x];
     const int r = (warp & 3) * 32 + lane;    // row of the query tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-    uint32_t tmem_og = tmem_o + kOGroup * grp;  // this group's output accumulator (of the current item)
+    const uint32_t tmem_s = tmem + 128u * (uint32_t)x + lane_addr;
+    uint32_t tmem_og = o_addr(x, 0) + lane_addr;  // the current item's output accumulator
     const float ref_slack = 8.f / scale_log2;
+    const uint32_t start_mine = smem_u32(&sh->sm_start[x]), start_other = smem_u32(&sh->sm_start[1 - x]);
+    const bool flag_writer = (warp & 3) == 0 && lane == 0;
     bool ok = true;
     uint32_t n = 0;
-    float m = -CUDART_INF_F, l = 0.f;       // this group's exponent reference and running sum of weights
-    bool o_started = false;                  // an earlier round of the item added to this group's accumulator
+    float m = -CUDART_INF_F, l = 0.f;       // exponent reference and running sum of weights of this row
+    bool o_started = false;                  // an earlier half round of the item added to the accumulator
     int cur_bh = 0, cur_qt = 0;
     for (uint32_t g = 0; ok; ++g) {
-      const int st = (int)(g % kMaxStages);  // info / bitmap slot of the round
-      const uint32_t sb = g & 1u;
-      const uint32_t tmem_s = tmem + 128u * sb;
-      ok = warp_wait(&sh->b_full[st], (g / kMaxStages) & 1u, lane, abort_flag, err);
+      const int si = (int)(g % kRing);       // info / bitmap slot of the round
+      ok = warp_wait(&ss.b_full[si], (g / kRing) & 1u, lane, wc);
       if (!ok) break;
-      const uint32_t info = sh->info[st];
+      const uint32_t info = ss.info[si];
       if (info & kInfoStop) break;
       const int ng = (int)(info & kInfoSlots);
       const bool first = (info & kInfoFirst) != 0u, last = (info & kInfoLast) != 0u;
       const bool tile_full = (info & kInfoFull) != 0u;
       if (first) {
-        cur_bh = sh->item_bh[st];
-        cur_qt = sh->item_qt[st];
+        cur_bh = ss.item_bh[si];
+        cur_qt = ss.item_qt[si];
         m = -CUDART_INF_F;
         l = 0.f;
         o_started = false;
-        tmem_og = o_of_item(n) + kOGroup * grp;
+        tmem_og = o_addr(x, n) + lane_addr;
       }
-      // this group's 32-column chunks of the round: grp and grp + 2, as far as the round reaches
-      const int n_mine = ((ng + 1) >> 1) > grp + 2 ? 2 : ((ng + 1) >> 1) > grp ? 1 : 0;
-      float alpha = 1.f;
-      if (n_mine > 0) {
-      uint32_t w0 = 0xffffffffu, w1 = 0xffffffffu;   // bitmap words of chunks grp and grp + 2
-      if (!tile_full) {
-        const uint32_t *brow = &sh->bitmap[st][r][0];
-        w0 = brow[grp];
-        w1 = brow[grp + 2];
-      }
-      // chunks in which none of this warp's 32 rows keeps anything are skipped (their P is
-      // written as zeros without reading S)
-      const uint32_t active = (__any_sync(0xffffffffu, w0 != 0u) ? 1u : 0u) | (__any_sync(0xffffffffu, w1 != 0u) ? 2u : 0u);
-      ok = warp_wait(&sh->s_full[sb], (g >> 1) & 1u, lane, abort_flag, err);
+      AP_TRACE(x, 2 + (warp & 3), g, 0);
+      ok = warp_wait(&ss.s_full, g & 1u, lane, wc);
       if (!ok) break;
+      AP_TRACE(x, 2 + (warp & 3), g, 1);
+      // The two streams keep their softmax phases apart by at least half a round.  Left alone they
+      // fall into lockstep (their MMAs share the tensor pipe and complete together), and then
+      // both compute while the tensor pipe idles and both wait while it works.  Started a
+      // half round apart, one stream's MMAs run under the other's exponentials, while two
+      // warps per scheduler still overlap enough to hide each other's latencies.  A hint only: the
+      // wait is short and bounded, and nothing depends on it.  (Stream 1 looks a moment later, so
+      // that of two streams arriving together stream 0 goes first.)
+      if (kStagger) {
+        if (x == 1) __nanosleep(64);
+        for (int i = 0; i < 48; ++i) {  // (one read serves the warp)
+          if ((uint32_t)clock64() - lds_volatile(start_other) >= kStaggerCycles) break;
+          __nanosleep(32);
+        }
+        if (flag_writer) sts_volatile(start_mine, (uint32_t)clock64());
+      }
+      AP_TRACE(x, 2 + (warp & 3), g, 2);
       tc_fence_after_sync();
-      // pass 1: the group's (up to) two chunks of S come into registers and stay there; pruned
-      // entries are replaced by -inf (exp2 of -inf is exactly 0); row maximum over kept entries
-      // (four independent chains)
-      uint32_t xa[32], xb[32];
-      const bool act0 = (active & 1u) != 0u, act1 = n_mine > 1 && (active & 2u) != 0u;
-      if (act0) tmem_ld32(tmem_s + lane_addr + 32 * grp, xa);
-      if (act1) tmem_ld32(tmem_s + lane_addr + 32 * (grp + 2), xb);
-      tmem_wait_ld();
-      float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F, mx2 = -CUDART_INF_F, mx3 = -CUDART_INF_F;
-      if (act0) {
-        if (!tile_full) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (!((w0 >> e) & 1u)) xa[e] = 0xff800000u;  // -inf
-        }
-#pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(xa[e]));
-          mx1 = fmaxf(mx1, __uint_as_float(xa[e + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(xa[e + 2]));
-          mx3 = fmaxf(mx3, __uint_as_float(xa[e + 3]));
-        }
-      }
-      if (act1) {
-        if (!tile_full) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e)
-            if (!((w1 >> e) & 1u)) xb[e] = 0xff800000u;
-        }
-#pragma unroll
-        for (int e = 0; e < 32; e += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(xb[e]));
-          mx1 = fmaxf(mx1, __uint_as_float(xb[e + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(xb[e + 2]));
-          mx3 = fmaxf(mx3, __uint_as_float(xb[e + 3]));
-        }
-      }
-      const float tile_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      // The exponent's reference m follows the running maximum lazily: it moves only when
-      // the maximum outgrows it by more than 2^8 in the exp2 domain (weights stay <= 256,
-      // well inside bf16 and fp32 range), which saves most rescales of O.  O / l does not
-      // depend on the reference.
-      const bool move = tile_max > m + ref_slack;   // also true for the first kept entry (m = -inf)
-      const float m_new = move ? tile_max : m;
-      const float m_safe = m_new == -CUDART_INF_F ? 0.f : m_new;
-      alpha = move ? ex2_approx((m - m_safe) * scale_log2) : 1.f;  // 0 when m was -inf
-      const float neg_mc = -m_safe * scale_log2;
-      m = m_new;
-      // Rescale the group's running output where the reference moved.  O += P V of the previous
-      // round may still be running (this round's S was computed ahead of it): wait for it first.
-      if (o_started && __any_sync(0xffffffffu, alpha != 1.f)) {
-        ok = warp_wait(&sh->pv_done[(g - 1u) & 1u], ((g - 1u) >> 1) & 1u, lane, abort_flag, err);
-        if (!ok) break;
-        tc_fence_after_sync();
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tmem_og + lane_addr + 32 * c, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(tmem_og + lane_addr + 32 * c, o);
-        }
-      }
-      // pass 2: P = exp2(c*S - c*m); pruned entries are -inf by now and give exactly 0; bf16 P over
-      // the first half of the chunk's columns of S
-      float sum0 = 0.f, sum1 = 0.f;
-      auto emit = [&](const uint32_t (&x)[32], bool act, int c) {
-        uint32_t pk[16];
-        if (!act) {
-#pragma unroll
-          for (int e = 0; e < 16; ++e) pk[e] = 0u;
-        } else {
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = ex2_approx(fmaf(__uint_as_float(x[2 * e]), scale_log2, neg_mc));
-            const float p1 = ex2_approx(fmaf(__uint_as_float(x[2 * e + 1]), scale_log2, neg_mc));
-            pk[e] = pack16x2<kF16>(p0, p1);
-            // the row sum is taken over the rounded weights the MMA will use, so that
-            // O / l is an exact convex combination of V rows whatever the rounding of P
-            const float2 pr = unpack16x2<kF16>(pk[e]);
-            sum0 += pr.x;
-            sum1 += pr.y;
+      for (int half = 0; half < 2; ++half) {
+        // this half's slots 4 half .. 4 half + n_sl - 1: one or two 32-column chunks
+        const int n_sl = min(max(ng - 4 * half, 0), 4);
+        if (n_sl > 0) {
+          const uint32_t tmem_b = tmem_s + 64u * (uint32_t)half;
+          uint2 bw = make_uint2(0xffffffffu, 0xffffffffu);   // bitmap words of the two chunks
+          if (!tile_full) bw = *reinterpret_cast<const uint2 *>(&ss.bitmap[si][r][2 * half]);
+          // Straight-line code per case (one or two chunks, masked or not): the chunks' loads,
+          // maxima, exponentials and stores interleave freely, which is worth far more than
+          // skipping the occasional chunk in which a warp's 32 rows keep nothing.
+          HalfStep st{m, l, 1.f};
+          if (n_sl > 2) {
+            if (tile_full) st = softmax_half<2, false, kF16>(tmem_b, bw, m, l, scale_log2, ref_slack);
+            else st = softmax_half<2, true, kF16>(tmem_b, bw, m, l, scale_log2, ref_slack);
+          } else {
+            st = softmax_half<1, true, kF16>(tmem_b, bw, m, l, scale_log2, ref_slack);
           }
+          // Rescale the running output where the reference moved (rare: the reference is lazy).
+          // O += P V of the half round before may still be running: wait for it first.  (It cannot
+          // be further ahead: the step after it needs the P being handed over below.)  P of this
+          // half is already in TMEM but not handed over yet, so the order is free.
+          if (o_started && __any_sync(0xffffffffu, st.alpha != 1.f)) {
+            ok = warp_wait(&ss.pv_done, (2u * g + (uint32_t)half - 1u) & 1u, lane, wc);
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t o[32];
+              tmem_ld32(tmem_og + 32 * c, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * st.alpha);
+              tmem_st32(tmem_og + 32 * c, o);
+            }
+          }
+          m = st.m;
+          l = st.l;
+          o_started = true;
+          tmem_wait_st();
         }
-        tmem_st16(tmem_s + lane_addr + 32 * c, pk);
-      };
-      emit(xa, act0, grp);
-      if (n_mine > 1) emit(xb, act1, grp + 2);
-      l = l * alpha + (sum0 + sum1);
-      o_started = true;
-      tmem_wait_st();
-      }  // n_mine > 0
-      // one arrival per warp (32 lanes arriving one by one would take hundreds of cycles)
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->p_full[sb]);
+        // one arrival per warp (32 lanes arriving one by one would take hundreds of cycles)
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ss.p_full[half]);
+        AP_TRACE(x, 2 + (warp & 3), g, 3 + half);
+      }
+      if (!ok) break;
       if (!last) continue;
-      // The item's rounds are over for this group: it hands (m, l) to the epilogue warps and goes on
-      // with the next item; the slot of the hand-over ring was read by the epilogue of item n - 4,
-      // which is over (this item's S needed O += P V of item n - 2, that the epilogue of item n - 3).
-      sh->ml[n & 3u][grp][r] = make_float2(m, l);
-      if (threadIdx.x == 0) {
-        sh->ml_bh[n & 3u] = cur_bh;
-        sh->ml_qt[n & 3u] = cur_qt;
+      // The item's rounds are over for these warps: they hand l to the epilogue warps and go on with
+      // the stream's next item.  The slot of the hand-over ring was last used by item n - 4, whose
+      // epilogue read it before it released that item's accumulator, which the first O += P V of
+      // item n - 4 + kOBufs waited for; that step was issued before S of this item.
+      ss.l[n & 3u][r] = l;
+      if ((threadIdx.x & 127) == 0) {
+        ss.ml_bh[n & 3u] = cur_bh;
+        ss.ml_qt[n & 3u] = cur_qt;
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->ml_ready[n & 3u]);
+      if (lane == 0) mbar_arrive(&ss.ml_ready[n & 3u]);
       ++n;
     }
-    // no more items: tell the epilogue warps
+    // no more items: tell the epilogue warps (the slot is free by the argument above)
     if (ok) {
-      if (threadIdx.x == 0) sh->ml_qt[n & 3u] = -1;
+      if ((threadIdx.x & 127) == 0) ss.ml_qt[n & 3u] = -1;
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->ml_ready[n & 3u]);
+      if (lane == 0) mbar_arrive(&ss.ml_ready[n & 3u]);
     }
-  } else if (warp >= 11) {
-    // ------------------------------------------------------------ epilogue
-    // Per item: merge the two groups' accumulators and write O / l, rounded once to bf16.
+  } else if (warp < 12) {
+    // ------------------------------------------------------------ epilogue (both streams)
+    // Per finished item: O / l, rounded once to the tensors' type.  Each warp serves its 32 rows of
+    // whichever stream hands an item over next.
     const int r = (warp & 3) * 32 + lane;    // row of the query tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    uint32_t n0 = 0u, n1 = 0u;             // items of stream 0 / 1 taken so far
+    bool live0 = true, live1 = true;       // the stream has not sent its end marker yet
     bool ok = true;
-    for (uint32_t n = 0; ok; ++n) {
-      ok = warp_wait(&sh->ml_ready[n & 3u], (n >> 2) & 1u, lane, abort_flag, err);
-      if (!ok) break;
-      const int item_qt = sh->ml_qt[n & 3u], item_bh = sh->ml_bh[n & 3u];
-      if (item_qt < 0) break;
-      const float2 g0 = sh->ml[n & 3u][0][r], g1 = sh->ml[n & 3u][1][r];
+    while (ok && (live0 || live1)) {
+      // lane 0 polls the two streams' hand-over barriers in turn
+      int x = -1;
+      if (lane == 0) {
+        for (uint32_t i = 0; i < wc.max_polls && x < 0; ++i) {
+          if (live0 && mbar_try_wait(&sh->st[0].ml_ready[n0 & 3u], (n0 >> 2) & 1u)) x = 0;
+          if (x < 0 && live1 && mbar_try_wait(&sh->st[1].ml_ready[n1 & 3u], (n1 >> 2) & 1u)) x = 1;
+          if (x < 0) {
+            if (*wc.abort_flag) break;
+            if (i > 1024) __nanosleep(64);
+          }
+        }
+        if (x < 0 && !*wc.abort_flag) {
+          *wc.abort_flag = 1;
+          atomicOr(err, kDevErrTimeout);
+        }
+      }
+      x = __shfl_sync(0xffffffffu, x, 0);
+      if (x < 0) {
+        ok = false;
+        break;
+      }
+      StreamShared &ss = sh->st[x];
+      const uint32_t n = x == 0 ? n0 : n1;
+      if (x == 0) ++n0; else ++n1;
+      const int item_qt = ss.ml_qt[n & 3u], item_bh = ss.ml_bh[n & 3u];
+      if (item_qt < 0) {
+        if (x == 0) live0 = false; else live1 = false;
+        continue;
+      }
+      const float l = ss.l[n & 3u][r];
       const int i = item_qt * kTile + r;
       uint16_t *orow = O + ((size_t)item_bh * Lq + i) * D;
-      const float m_tot = fmaxf(g0.x, g1.x);
-      // weight of a partial result; 0 for a group that saw no kept entry of this row (m = -inf),
-      // whose accumulator is then never read into the sum (it may hold a previous item's data)
-      const float a0 = g0.x == -CUDART_INF_F ? 0.f : ex2_approx((g0.x - m_tot) * scale_log2);
-      const float a1 = g1.x == -CUDART_INF_F ? 0.f : ex2_approx((g1.x - m_tot) * scale_log2);
-      const float l_tot = g0.y * a0 + g1.y * a1;
-      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-      const float f0 = a0 * inv, f1 = a1 * inv;
-      ok = warp_wait(&sh->o_done[kOBufs == 2u ? (n & 1u) : 0u], (n / kOBufs) & 1u, lane, abort_flag, err);
+      // a row without kept entries has l = 0 and P = 0 throughout: exact zeros (its accumulator may
+      // never have been written)
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const uint32_t ob = C::kOBufs == 2 ? (n & 1u) : 0u;
+      ok = warp_wait(&ss.o_done[ob], (n / C::kOBufs) & 1u, lane, wc);
       if (!ok) break;
       tc_fence_after_sync();
+      const uint32_t o_acc = o_addr(x, n) + lane_addr;
 #pragma unroll 1
       for (int c = 0; c < D / 32; ++c) {
-        uint32_t o0[32], o1[32];
-        tmem_ld32(o_of_item(n) + lane_addr + 32 * c, o0);
-        tmem_ld32(o_of_item(n) + kOGroup + lane_addr + 32 * c, o1);
+        uint32_t o[32];
+        tmem_ld32(o_acc + 32 * c, o);
         tmem_wait_ld();
         if (c == D / 32 - 1) {  // this thread's rows of O are in registers: the next item may overwrite them
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh->o_free[kOBufs == 2u ? (n & 1u) : 0u]);
+          if (lane == 0) mbar_arrive(&ss.o_free[ob]);
         }
         if (i < Lq) {
 #pragma unroll
@@ -724,11 +844,9 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
             uint32_t pk[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              // a row without kept entries has l = 0 and P = 0 throughout: write exact zeros
               const int j = 8 * q + 2 * e;
-              const float x0 = (f0 > 0.f ? __uint_as_float(o0[j]) * f0 : 0.f) + (f1 > 0.f ? __uint_as_float(o1[j]) * f1 : 0.f);
-              const float x1 = (f0 > 0.f ? __uint_as_float(o0[j + 1]) * f0 : 0.f) +
-                               (f1 > 0.f ? __uint_as_float(o1[j + 1]) * f1 : 0.f);
+              const float x0 = inv > 0.f ? __uint_as_float(o[j]) * inv : 0.f;
+              const float x1 = inv > 0.f ? __uint_as_float(o[j + 1]) * inv : 0.f;
               pk[e] = pack16x2<kF16>(x0, x1);
             }
             *reinterpret_cast<uint4 *>(orow + 32 * c + 8 * q) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -739,7 +857,22 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, kTmemCols);
+  if ((warp == 12 || warp == 13) && lane == 0 && *wc.abort_flag) {
+    // A wait expired somewhere in the CTA and every role has left its loop.  Copies this producer
+    // armed may still be in flight: wait (bounded) for the most recent ones before the CTA's shared
+    // memory is given up (earlier ones completed before these were armed).
+    StreamShared &ss = sh->st[warp - 12];
+    if (armed_q >= 0) mbar_wait(&ss.q_full[armed_q % C::kQBufs], ((uint32_t)armed_q / C::kQBufs) & 1u, 1u << 16);
+    for (int a = armed_k - 1; a <= armed_k; ++a)
+      if (a >= 0) {
+        mbar_wait(&ss.k_full[a % C::kStages], ((uint32_t)a / C::kStages) & 1u, 1u << 16);
+        mbar_wait(&ss.b_full[a % kRing], ((uint32_t)a / kRing) & 1u, 1u << 16);
+      }
+    for (int a = armed_v - 1; a <= armed_v; ++a)
+      if (a >= 0) mbar_wait(&ss.v_full[a % C::kStages], ((uint32_t)a / C::kStages) & 1u, 1u << 16);
+  }
+  __syncthreads();
+  if (warp == 14) tmem_dealloc(tmem, kTmemCols);
 }
 
 int sm_count() {
@@ -758,24 +891,31 @@ template <int D, bool kSplit, bool kF16>
 cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
                    unsigned *err, cudaStream_t s) {
   using C = Cfg<D, kSplit>;
-  static_assert(sizeof(Shared) <= 17 * 1024, "shared bookkeeping outgrew its reservation");
-  static_assert(C::kStages <= kMaxStages, "ring deeper than its barriers");
-  static_assert(C::kSmemBytes > 114 * 1024 && C::kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
+  constexpr int kSmemBytes = C::kBarOffset + (int)sizeof(Shared) + 1024;  // + alignment slack
+  static_assert(kSmemBytes > 114 * 1024 && kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
   auto kern = fwd_tc_kernel<D, kSplit, kF16>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   const int n_units = B * H * ((t.n_qt + 1) / 2);  // pairs of query tiles, see the producer
   const float scale_log2 = scale * 1.4426950408889634f;
-  kern<<<n_units < sms ? n_units : sms, kThreads, C::kSmemBytes, s>>>(
+  const DebugKnobs dbg = debug_knobs();
+  // the test hook runs on one CTA only (a tiny grid is all it is meant for)
+  kern<<<dbg.skip_arrive ? 1 : (n_units < sms ? n_units : sms), kThreads, kSmemBytes, s>>>(
       maps, static_cast<uint16_t *>(O), t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, B, H, Lq,
-      t.n_qt, scale_log2, err);
+      t.n_qt, scale_log2, err, dbg.max_polls, dbg.skip_arrive);
   count_launches(1);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+#ifdef AP_FWD_TRACE
+extern "C" int ap_debug_fwd_trace(long long *host_out, size_t bytes) {
+  return (int)cudaMemcpyFromSymbol(host_out, g_fwd_trace, bytes < sizeof(g_fwd_trace) ? bytes : sizeof(g_fwd_trace));
+}
+#endif
 
 cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_tiles &t, void *O, int B, int H,
                           int Lq, int Lk, int d, int f16, float scale, cudaStream_t s) {

@@ -1,0 +1,39 @@
+"""The bounded waits of the tensor-core kernels, exercised without faulting or hanging anything.
+
+ap_debug_expire_waits(1) makes the next launches run on one thread block with a short poll limit
+and leave out one producer arrival: a wait runs out, the kernel must return by itself with the
+device status word raised, and the library must work normally afterwards.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ap_oracle as orc
+from paper_2012_02030_b200 import inputs
+from tests.parity_util import assert_close_attention
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [64, 128])
+def test_forward_expired_wait_returns_timeout_once_and_the_next_call_is_correct(d):
+    from paper_2012_02030_b200 import binding as ap
+
+    B, H, L = 1, 2, 256
+    gen = torch.Generator().manual_seed(4100 + d)
+    q, k, v = (torch.randn((B, H, L, d), generator=gen).to(torch.bfloat16) for _ in range(3))
+    mask = inputs.random_mask(H, L, L, 0.3, seed=77, causal=True)
+    tiles = ap.Tiles(H, L, L)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    ap.ap_debug_expire_waits(True)
+    try:
+        ap.ap_sparse_attention_fwd(qd, kd, vd, tiles)          # returns by itself: every wait is bounded
+        assert ap.ap_device_status() == ap.AP_ERR_TIMEOUT      # raised once ...
+    finally:
+        ap.ap_debug_expire_waits(False)
+    assert ap.ap_device_status() == ap.AP_OK                   # ... and cleared by the read
+    out = ap.ap_sparse_attention_fwd(qd, kd, vd, tiles)        # tensor memory was freed, barriers are fresh
+    assert ap.ap_device_status() == ap.AP_OK
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy())
+    assert_close_attention(out, ref, "bf16", "after an expired wait")
