@@ -111,3 +111,39 @@ def gpu_build_mask(ap, acc_dev, w, want_tiles=True, layer=False):
     build(acc_dev, w.keep_frac, w.causal, w.keep_diag, mask, tiles, nnz)
     assert ap.ap_device_status() == ap.AP_OK
     return mask, tiles, nnz
+
+
+def backward_bounds(q, k, v, d_o, mask, ulp, scale=None, tiny=0.0):
+    """Element-wise absolute error bounds for dQ, dK, dV of the tensor-core backward, from a model of
+    where it rounds (fp64 numpy, small shapes only).  With P the masked softmax, dP = dO V^T,
+    D_i = dO_i . O_i and dS = P o (dP - D):
+      * P and dS are each rounded once to the 16-bit type before they enter a product (relative ulp / 2
+        each), so every term of dQ = c dS K, dK = c dS^T Q, dV = P^T dO is off by at most ulp times its
+        size: the sum of the terms' absolute values bounds the effect;
+      * D_i is formed from the rounded output O, an error of at most (ulp / 2) sum_c |dO_ic O_ic|, which
+        enters dS_ij as P_ij dD_i and from there dQ_i (times c |K_j|) and dK_j (times c |Q_i|);
+      * dV has no D in it.
+    ulp = 2^-8 for bf16, 2^-11 for fp16 (one unit in the last place at 1.0); tiny = the absolute
+    rounding step at the bottom of the 16-bit type's range (fp16: weights below 2^-24 vanish), 0 where
+    that is out of reach (bf16 has fp32's exponent range)."""
+    B, H, Lq, d = q.shape
+    Lk = k.shape[2]
+    c = 1.0 / np.sqrt(d) if scale is None else scale
+    keep = mask.astype(bool)[None]                                   # [1, H, Lq, Lk]
+    s = np.einsum("bhid,bhjd->bhij", q, k) * c
+    s = np.where(keep, s, -np.inf)
+    m = s.max(-1, keepdims=True)
+    m = np.where(np.isfinite(m), m, 0.0)
+    e = np.where(keep, np.exp(s - m), 0.0)
+    den = e.sum(-1, keepdims=True)
+    p = np.divide(e, den, out=np.zeros_like(e), where=den > 0)
+    o = np.einsum("bhij,bhjd->bhid", p, v)
+    dp = np.einsum("bhid,bhjd->bhij", d_o, v)
+    dd = (d_o * o).sum(-1, keepdims=True)
+    ds = p * (dp - dd)
+    d_dd = 0.5 * ulp * (np.abs(d_o) * np.abs(o)).sum(-1, keepdims=True)       # [B, H, Lq, 1]
+    ads = ulp * np.abs(ds) + p * d_dd + tiny * (1.0 + np.abs(dp - dd))         # per entry of dS
+    b_dq = c * np.einsum("bhij,bhjd->bhid", ads, np.abs(k))
+    b_dk = c * np.einsum("bhij,bhid->bhjd", ads, np.abs(q))
+    b_dv = np.einsum("bhij,bhid->bhjd", ulp * p + tiny, np.abs(d_o))
+    return b_dq, b_dk, b_dv
