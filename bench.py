@@ -42,12 +42,17 @@ from paper_2012_02030_b200 import inputs, metrics, replicas  # noqa: E402
 METRIC = "sparse-attention fwd effective TFLOP/s (4*d*nnz)"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per forward launch from the ncu
-# captures summarised under profiles/ (None until a capture exists).
-NCU_FWD_TRAFFIC_BYTES = {"long": 255.8e6}  # profiles/long_workload_ncu.md (209.3 MB read + 46.5 MB written)
-# the other stages on the same workload, same file: accumulate 2137.7 MB read + 509.8 MB written per call;
-# build_mask = collecting pass (541 MB read) + emit pass (541 MB read + 275 MB written) + small kernels
-NCU_STAGE_TRAFFIC_BYTES = {"long": {"accumulate": 2647.5e6, "build_mask": 1.40e9}}
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each stage's kernels, from ncu
+# captures of a REDUCED case of the same workload (fewer batch elements, so that the capture is small),
+# scaled to the full launch by the units it processes; `source` says which capture and how it was scaled.
+# A stage without a capture reports null.
+NCU_TRAFFIC = {
+    "long": {
+        "sparse_fwd": None,
+        "accumulate": None,
+        "build_mask": None,
+    },
+}
 
 
 def load_peaks():
@@ -214,6 +219,123 @@ def workload_config(w):
 # ------------------------------------------------------------------------------- GPU arm
 
 
+def _stats(ms):
+    ms = [float(x) for x in ms]
+    return {"mean": float(np.mean(ms)), "median": float(np.median(ms)), "best": float(np.min(ms))}
+
+
+def _time_back_to_back(fn, n):
+    """n launches of fn(i) back to back between one pair of events: ms per launch."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n
+
+
+def workloads_section(ap, dev, peaks, with_cpu):
+    """Short runs of the small workloads: forward under the calibrated mask and under the dense list.
+    Their tensors fit in L2, so the figure for the HBM roofline rotates over enough copies of the
+    tensors to exceed L2 twice over (every launch finds its inputs in DRAM); the L2-warm figure (one
+    set of tensors reused) is given beside it.  With with_cpu, the oracle's forward on a bounded
+    sample is timed on one thread and on all threads."""
+    out = {}
+    for name in ("tiny", "bert", "lm", "s2s_self", "s2s_cross"):
+        w = inputs.WORKLOADS[name]
+        elem = 4 if w.dtype == "f32" else 2
+        bias = inputs.calib_bias(w).to(dev)
+        acc = torch.zeros((w.H, w.Lq, w.Lk), dtype=torch.float32, device=dev)
+        for t in range(w.calib_batches):
+            cq, ck = inputs.calib_qk(w, t)
+            ap.ap_accumulate_attention(acc, cq.to(dev), ck.to(dev), bias, causal=w.causal)
+        tiles = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+        dense = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+        nnz = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+        mask = torch.empty((w.H, w.Lq, w.Lk), dtype=torch.uint8, device=dev)
+        ap.ap_build_mask(acc, w.keep_frac, w.causal, w.keep_diag, mask, tiles, nnz)
+        ap.ap_dense_tiles(dense, causal=w.causal)
+        q, k, v = (t.to(dev) for t in inputs.eval_qkv(w))
+        set_bytes = 4 * q.numel() * elem
+        n_sets = max(2, int(np.ceil(2.5 * 126e6 / set_bytes)))
+        sets = [(q, k, v, torch.empty_like(q))] + [(q.clone(), k.clone(), v.clone(), torch.empty_like(q))
+                                                   for _ in range(n_sets - 1)]
+        n = max(20, 2 * n_sets)
+        res = {}
+        for label, tl in (("sparse", tiles), ("dense", dense)):
+            for i in range(n_sets):   # warm-up: every set once
+                ap.ap_sparse_attention_fwd(*sets[i][:3], tl, sets[i][3])
+            cold = _time_back_to_back(lambda i: ap.ap_sparse_attention_fwd(*sets[i % n_sets][:3], tl, sets[i % n_sets][3]), n)
+            warm = _time_back_to_back(lambda i: ap.ap_sparse_attention_fwd(*sets[0][:3], tl, sets[0][3]), n)
+            res[label] = (cold, warm)
+        if ap.ap_device_status() != ap.AP_OK:
+            raise RuntimeError("device status not OK in the workloads section (%s)" % name)
+        nnz_total = int(nnz.sum().item())
+        comp = metrics.compulsory_bytes(w.B, w.H, w.Lq, w.Lk, w.d, elem)
+        entry = {
+            "shape": {"B": w.B, "H": w.H, "Lq": w.Lq, "Lk": w.Lk, "d": w.d, "dtype": w.dtype, "keep_frac": w.keep_frac,
+                      "calib_batches": w.calib_batches},
+            "sparse_fwd_ms": res["sparse"][0], "dense_fwd_ms": res["dense"][0],
+            "sparse_fwd_ms_l2_warm": res["sparse"][1], "dense_fwd_ms_l2_warm": res["dense"][1],
+            "speedup_vs_dense_path": res["dense"][0] / res["sparse"][0],
+            "effective_tflops": metrics.effective_flops(nnz_total, w.B, w.d) / (res["sparse"][0] * 1e-3) / 1e12,
+            "tokens_per_s": w.B * w.Lq / (res["sparse"][0] * 1e-3),
+            "frac_of_hbm_on_compulsory_bytes": comp / (res["sparse"][0] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "tiles_kept": tiles.n_tiles(), "tiles_domain": dense.n_tiles(), "rounds": int(tiles.round_ptr[-1].item()),
+            "buffer_sets": n_sets, "launches_timed": n,
+        }
+        if with_cpu:
+            from oracle import ap_oracle as orc
+
+            units, seqs = min(w.H, 4), min(w.B, 2)
+            eq, ek, ev = (inputs.widen(t[:seqs, :units]) for t in inputs.eval_qkv(w))
+            m_host = mask[:units].cpu().numpy()
+            fl = 4.0 * w.d * float(m_host.sum()) * seqs
+            all_threads = orc.num_threads()
+            cpu = {}
+            for label, nt in (("threads_1", 1), ("threads_all", all_threads)):
+                orc.set_num_threads(nt)
+                t0 = time.perf_counter()
+                orc.attention_fwd(eq, ek, ev, m_host)
+                cpu[label] = {"tflops": fl / (time.perf_counter() - t0) / 1e12, "threads": min(nt, units * seqs)}
+            orc.set_num_threads(all_threads)
+            cpu["sample"] = "oracle forward of heads 0..%d of batch elements 0..%d" % (units - 1, seqs - 1)
+            entry["cpu_oracle"] = cpu
+        out[name] = entry
+        del sets, acc, mask, bias
+    return out
+
+
+def density_section(ap, w, acc, q, k, v, out, ws, dense_ms, dense_tiles, peaks, dev):
+    """The forward on the bench's own shape and accumulator at several kept fractions: time, what the
+    schedule holds, speedup over the dense list, fractions of the burst bf16 peak."""
+    rows = []
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    nnz = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+    for keep in (0.10, 0.05, 0.02):
+        ap.ap_build_mask(acc, keep, w.causal, w.keep_diag, None, tiles, nnz, ws)
+        for _ in range(3):
+            ap.ap_sparse_attention_fwd(q, k, v, tiles, out)
+        ms = _time_back_to_back(lambda i: ap.ap_sparse_attention_fwd(q, k, v, tiles, out), 10)
+        n_rounds = int(tiles.round_ptr[-1].item())
+        slots = int((tiles.round_info[:n_rounds] & 15).sum().item())
+        n_tiles = tiles.n_tiles()
+        kept = int(nnz.sum().item())
+        rows.append({
+            "keep_frac": keep, "kept_entries_per_head": kept // w.H, "fwd_ms": ms, "tiles": n_tiles, "rounds": n_rounds,
+            "slots": slots, "speedup_vs_dense_path": dense_ms / ms,
+            "effective_tflops": metrics.effective_flops(kept, w.B, w.d) / (ms * 1e-3) / 1e12,
+            "frac_of_bf16_burst_on_kept_tile_flops": metrics.tile_flops(n_tiles, w.B, w.d) / (ms * 1e-3) / 1e12 / peaks["bf16"],
+            "frac_of_bf16_burst_on_executed_flops": metrics.slot_flops(slots, w.B, w.d) / (ms * 1e-3) / 1e12 / peaks["bf16"],
+        })
+    if ap.ap_device_status() != ap.AP_OK:
+        raise RuntimeError("device status not OK in the density section")
+    return {"shape": w.name, "dense_path_ms": dense_ms, "dense_tiles": dense_tiles,
+            "timing": "10 launches back to back after 3 warm-up launches; the tensors exceed L2", "rows": rows}
+
+
+
 def run_gpu(args, w):
     from paper_2012_02030_b200 import binding as ap
 
@@ -303,8 +425,9 @@ def run_gpu(args, w):
     if status != ap.AP_OK:
         raise RuntimeError("device status %d after the timed steps" % status)
     total_ms = start.elapsed_time(end)
-    stage_ms = {s: float(np.mean([events[i][j].elapsed_time(events[i][j + 1]) for i in range(args.steps)]))
-                for j, s in enumerate(stages)}
+    stage_all = {s: _stats([events[i][j].elapsed_time(events[i][j + 1]) for i in range(args.steps)])
+                 for j, s in enumerate(stages)}
+    stage_ms = {s: stage_all[s]["mean"] for s in stages}
     total_ms, fwd_ms_max = replicas.max_over_ranks(info, [total_ms, stage_ms["sparse_fwd"]], dev)
 
     # ---- counts -----------------------------------------------------------------------------
@@ -393,6 +516,7 @@ def run_gpu(args, w):
         bwd_fl = (4 * 2.0 * 128 * 16 * w.d * n_slots_b + 4 * 2.0 * 128 * 128 * w.d * tiles.n_tiles()) * w.B
         backward = {"ms": bwd_ms, "effective_tflops": 10.0 * w.d * float(nnz.sum().item()) * w.B / (bwd_ms * 1e-3) / 1e12,
                     "executed_tflops": bwd_fl / (bwd_ms * 1e-3) / 1e12,
+                    "frac_of_bf16_burst": bwd_fl / (bwd_ms * 1e-3) / 1e12 / peaks["bf16"],
                     "frac_of_bf16_sustained": bwd_fl / (bwd_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
                     "note": "ap_sparse_attention_bwd (rows kernel on rounds + columns kernel on tiles), %d runs "
                             "outside the step" % n_bwd}
@@ -428,6 +552,14 @@ def run_gpu(args, w):
                   "note": "ap_accumulate_attention_entmax15 on one calibration batch into a scratch accumulator and "
                           "ap_sparse_attention_entmax15_fwd under the step's mask, %d runs after 2 warm-up runs; "
                           "entries_given_weight = fraction of the domain that received weight from any sample" % n_ent}
+
+    # ---- the forward at other kept fractions on this shape, and the small workloads (outside the step) ----
+    density = workloads = None
+    if not args.no_extras:
+        if w.dtype != "f32":
+            density = density_section(ap, w, acc, q, k, v, out, ws, stage_ms["dense_fwd"], T_dense, peaks, dev)
+        if world == 1:
+            workloads = workloads_section(ap, dev, peaks, not args.no_cpu_baseline)
 
     # ---- the same step replayed from a CUDA graph (launch gaps of the ~25 kernels of a step removed) ----
     # (last: the replays add one calibration batch over and over, which skews the accumulator)
@@ -472,17 +604,22 @@ def run_gpu(args, w):
     comp_bytes = metrics.compulsory_bytes(w.B, w.H, w.Lq, w.Lk, w.d, elem)
     tensor_bound = w.dtype == "bf16" and slot_fl / comp_bytes > peaks["bf16_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
     if tensor_bound:
-        roof = {"bound": "tensor", "achieved": slot_fl / fwd_s / 1e12, "peak": peaks["bf16_sustained"],
-                "unit": "TFLOP/s", "peak_kind": "bf16 sustained, of " + peaks["source"]}
+        roof = {"bound": "tensor", "achieved": slot_fl / fwd_s / 1e12, "peak": peaks["bf16"],
+                "unit": "TFLOP/s", "peak_kind": "bf16 burst (the forward is timed alone between events), of " + peaks["source"]}
     else:
         roof = {"bound": "hbm", "achieved": comp_bytes / fwd_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "peak_kind": "copy bandwidth, of " + peaks["source"]}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_FWD_TRAFFIC_BYTES.get(w.name)
+    traffic = NCU_TRAFFIC.get(w.name, {}) if (w.B, w.H) == (inputs.WORKLOADS[w.name].B, inputs.WORKLOADS[w.name].H) else {}
+    roof["traffic"] = (traffic.get("sparse_fwd") or {}).get("bytes")
+    roof["traffic_source"] = (traffic.get("sparse_fwd") or {}).get("source")
     roof["kernel"] = "sparse_fwd (fwd_tc_kernel)" if w.dtype == "bf16" else "sparse_fwd (fwd_simt_kernel)"
     roof["algorithmic"] = {"slot_flops": slot_fl, "slots_per_launch": n_slots * w.B, "rounds_per_launch": n_rounds * w.B,
                            "kept_tile_flops": tile_fl, "compulsory_bytes": comp_bytes, "tiles_per_step": T_sparse}
-    roof["other_views"] = {"kept_tile_flops_frac_of_bf16_sustained": tile_fl / fwd_s / 1e12 / peaks["bf16_sustained"],
+    roof["other_views"] = {"executed_flops_frac_of_bf16_sustained": slot_fl / fwd_s / 1e12 / peaks["bf16_sustained"],
+                           "kept_tile_flops_frac_of_bf16_burst": tile_fl / fwd_s / 1e12 / peaks["bf16"],
+                           "kept_tile_flops_frac_of_bf16_sustained": tile_fl / fwd_s / 1e12 / peaks["bf16_sustained"],
+                           "effective_flops_frac_of_bf16_burst": eff_flops / fwd_s / 1e12 / peaks["bf16"],
                            "compulsory_bytes_frac_of_hbm": comp_bytes / fwd_s / 1e9 / peaks["hbm_gbs"]}
     # other stages, HBM view: accumulate = acc read+write over the domain + bias + Q,K;
     # build_mask = 2 reads of acc + mask bytes + bitmap bits over H*Lq*Lk
@@ -494,12 +631,14 @@ def run_gpu(args, w):
                        "peak": peaks["hbm_gbs"], "unit": "GB/s"},
         "build_mask": {"bound": "hbm", "achieved": mask_bytes / (stage_ms["build_mask"] * 1e-3) / 1e9,
                        "peak": peaks["hbm_gbs"], "unit": "GB/s"},
-        "dense_fwd": {"bound": "tensor", "unit": "TFLOP/s", "peak": peaks["bf16_sustained"],
+        "dense_fwd": {"bound": "tensor", "unit": "TFLOP/s", "peak": peaks["bf16"],
                       "achieved": metrics.tile_flops(T_dense, w.B, w.d) / (stage_ms["dense_fwd"] * 1e-3) / 1e12},
     }
     for name, r in by_stage.items():
         r["frac"] = r["achieved"] / r["peak"]
-        r["traffic"] = NCU_STAGE_TRAFFIC_BYTES.get(w.name, {}).get(name)
+        r["traffic"] = (traffic.get(name) or {}).get("bytes")
+        r["traffic_source"] = (traffic.get(name) or {}).get("source")
+    by_stage["dense_fwd"]["frac_of_bf16_sustained"] = by_stage["dense_fwd"]["achieved"] / peaks["bf16_sustained"]
     by_stage["accumulate"]["algorithmic_bytes"] = acc_bytes
     by_stage["build_mask"]["algorithmic_bytes"] = mask_bytes
     # the kernel with the largest share of the step's device time is not the metric's kernel
@@ -526,6 +665,8 @@ def run_gpu(args, w):
                        l2="inputs exceed L2" if flush is None else "256 MiB flush write between steps",
                        value_scope="sparse forward's device time inside the step; ms_per_step is the whole step"),
         "stage_ms": stage_ms,
+        "stage_ms_median": {s_: stage_all[s_]["median"] for s_ in stages},
+        "stage_ms_best": {s_: stage_all[s_]["best"] for s_ in stages},
         "tokens_per_s": replicas.job_throughput(info, w.B * w.Lq, fwd_ms_max * 1e-3),
         "speedup_vs_dense_path": stage_ms["dense_fwd"] / stage_ms["sparse_fwd"],
         "density": {"kept_fraction": nnz_total / float(dom), "tiles_kept": T_sparse, "tiles_domain": T_dense,
@@ -538,7 +679,7 @@ def run_gpu(args, w):
         "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer, "backward": backward,
-        "entmax15": entmax,
+        "entmax15": entmax, "workloads": workloads, "density": density,
         "graph_replay": {"ms_per_step": graph_ms, "note": "the same step (same calibration batch every replay) "
                          "captured once in a CUDA graph; steps replays timed with one pair of events"},
     }
@@ -639,10 +780,16 @@ def main():
     p.add_argument("--calib-batches", type=int, default=0,
                    help="calibration batches accumulated before the timed steps (0 = the workload's own count); "
                         "profiling runs use a small number to keep the launch list short")
+    p.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling runs use a small case)")
+    p.add_argument("--H", type=int, default=0, help="override the workload's head count")
+    p.add_argument("--no-extras", action="store_true",
+                   help="leave out the sections measured outside the step (other densities, the small workloads)")
     p.add_argument("--density-sweep", action="store_true",
                    help="instead of the bench line: forward time vs kept fraction on the workload's shape")
     args = p.parse_args()
     w = inputs.WORKLOADS[args.workload]
+    if args.B > 0 or args.H > 0:
+        w = w.scaled(**({"B": args.B} if args.B > 0 else {}), **({"H": args.H} if args.H > 0 else {}))
     if args.density_sweep:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
