@@ -16,13 +16,24 @@
 // 128-byte swizzle, so that a thread reads its own row without bank conflicts),
 // copied to registers and reused for all b.  Samples are added in ascending b by
 // a fixed thread and every accumulator entry receives exactly one addition per
-// launch (a fire-and-forget red.global.add), so results are reproducible bit for bit.
+// launch, so results are reproducible bit for bit.  Where the accumulator's rows are
+// 16-byte multiples that addition is a TMA reduction: each softmax warp stages its
+// 32 rows x 32 columns in shared memory (128-byte swizzle again) and one lane issues
+// cp.reduce.async.bulk.tensor ... add, which updates whole 128-byte lines in L2;
+// a lane per row adding 16 bytes at a time would touch 32 lines per instruction.  Inside
+// a tile that straddles the edge of a causal domain the reduction adds exact zeros to the
+// entries outside the domain (boxes wholly outside are skipped).  Other shapes keep the
+// per-row red.global.add.
 //
 // Warp roles (320 threads, one CTA per SM): warps 0-7 softmax; thread (wg, r)
 // with wg = warp / 4 owns row r of the tile and columns [64 wg, 64 wg + 64) of
 // every key tile; warp 8 TMA producer; warp 9 MMA issuer and TMEM owner.  S is
 // double-buffered in TMEM (2 x 128 columns) so the MMA of the next visit runs
-// under the softmax of the current one.  Every mbarrier wait is bounded.
+// under the softmax of the current one; a visit's 64 columns are copied to registers in one
+// go and S is handed back before the arithmetic starts.  TMEM columns 256-383 hold the running
+// sum over b, columns 384-511 the per-sample (maximum, sum) pairs of both column halves, which
+// a thread reads back for its own row (lane) at the start of sweep 2.  Every mbarrier wait is
+// bounded.
 #include <math_constants.h>
 
 #include "ap_common.cuh"
@@ -36,30 +47,32 @@ using namespace sm100;
 
 constexpr int kThreads = 320;
 constexpr int kSoftmaxThreads = 256;
+constexpr int kSoftmaxWarps = kSoftmaxThreads / 32;
 constexpr int kSubBytes = 128 * 128;
-constexpr uint32_t kTmemCols = 512;  // S x 2 (columns 0..255), running sum over b (columns 256..383)
-constexpr uint32_t kMaxPolls = 1u << 22;
-constexpr int kMaxB = 16;  // samples per launch (statistics live in shared memory)
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kSumCol = 256;    // running sum over b: 128 columns
+constexpr uint32_t kStatsCol = 384;  // (max, sum) pairs: 32 columns per column half, 2 per sample
+constexpr int kMaxB = 16;            // samples per launch
 constexpr int kBiasBytes = 128 * 128 * 4;  // one fp32 bias tile: 4 boxes of 128 rows x 32 columns
+constexpr int kRedBytes = 32 * 128;        // per softmax warp: 32 rows x 32 fp32 columns on their way to the accumulator
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
 struct Cfg {
   static constexpr int kSub = D / 64;
   static constexpr int kTileBytes = kSub * kSubBytes;    // one operand tile (Q or K)
-  static constexpr int kStages = D == 64 ? 3 : 2;        // (Q, K) pairs in flight
+  static constexpr int kStages = D == 64 ? 4 : 2;        // (Q, K) pairs in flight
   static constexpr int kBiasOffset = 2 * kStages * kTileBytes;
-  static constexpr int kStatsOffset = kBiasOffset + kBiasBytes;
-  static constexpr int kStatsBytes = 2 * kMaxB * 128 * 8;  // [wg][b][row] (max, sum)
-  static constexpr int kBarOffset = kStatsOffset + kStatsBytes;
+  static constexpr int kRedOffset = kBiasOffset + kBiasBytes;
+  static constexpr int kBarOffset = kRedOffset + kSoftmaxWarps * kRedBytes;
   static constexpr int kSmemBytes = kBarOffset + 256 + 1024;
   static_assert(kSmemBytes <= 227 * 1024, "within the shared memory of one CTA");
 };
 
 struct Barriers {
   uint64_t s_full[2], s_empty[2];
-  uint64_t in_full[3], in_empty[3];
-  uint64_t sweep1_done;  // all 256 softmax threads have stored their sweep-1 statistics
+  uint64_t in_full[4], in_empty[4];
+  uint64_t sweep1_done;  // all softmax warps have stored their sweep-1 statistics
   uint64_t bias_full, bias_empty;
   uint32_t tmem_base;
   int abort_flag;
@@ -76,30 +89,42 @@ __device__ __forceinline__ float lg2_approx(float x) {
   return y;
 }
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
-                                              unsigned *err) {
-  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+// Bounded wait that also gives up as soon as another thread of the CTA has.
+__device__ __noinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag, unsigned *err,
+                                           uint32_t max_polls) {
+  for (uint32_t i = 0; i < max_polls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (i > 64) __nanosleep(64);
+    if (i > 1024) __nanosleep(64);
   }
   *abort_flag = 1;
   atomicOr(err, kDevErrTimeout);
   return false;
 }
 
+// The same wait for a whole (converged) warp: one lane polls - 32 lanes polling one barrier would
+// serialise - and the outcome is shared.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int lane, volatile int *abort_flag,
+                                          unsigned *err, uint32_t max_polls) {
+  bool ok = true;
+  if (lane == 0 && !mbar_try_wait(bar, parity)) ok = wait_or_abort(bar, parity, abort_flag, err, max_polls);
+  return __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+}
+
+// dbg_skip != 0 (test hook): the copies of the first visit are never issued, so the MMA issuer's
+// first wait runs out and the CTA leaves through its error path.
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                     const __grid_constant__ CUtensorMap map_bias, int bias_by_tma, float *__restrict__ acc,
-                     const float *__restrict__ bias, int b0, int Bc, int H, int Lq, int Lk,
-                     int n_qt, int n_kt, int causal, int f16, float scale_log2, unsigned *err) {
+                     const __grid_constant__ CUtensorMap map_bias, const __grid_constant__ CUtensorMap map_acc,
+                     int bias_by_tma, int acc_by_tma, float *__restrict__ acc, const float *__restrict__ bias, int b0,
+                     int Bc, int H, int Lq, int Lk, int n_qt, int n_kt, int causal, int f16, float scale_log2,
+                     unsigned *err, uint32_t max_polls, int dbg_skip) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
       reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char *bias_s = smem + C::kBiasOffset;
-  float2 *stats = reinterpret_cast<float2 *>(smem + C::kStatsOffset);  // [wg][b][row]
   Barriers *bars = reinterpret_cast<Barriers *>(smem + C::kBarOffset);
 
   // late query tiles (most key tiles under a causal mask) first
@@ -115,15 +140,15 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bars->s_full[s], 1);
-      mbar_init(&bars->s_empty[s], kSoftmaxThreads);
+      mbar_init(&bars->s_empty[s], kSoftmaxWarps);  // one arrival per softmax warp
     }
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->in_full[s], 1);
       mbar_init(&bars->in_empty[s], 1);
     }
-    mbar_init(&bars->sweep1_done, kSoftmaxThreads);
+    mbar_init(&bars->sweep1_done, kSoftmaxWarps);
     mbar_init(&bars->bias_full, 1);
-    mbar_init(&bars->bias_empty, kSoftmaxThreads);
+    mbar_init(&bars->bias_empty, kSoftmaxWarps);
     bars->abort_flag = 0;
     fence_mbar_init();
   }
@@ -153,14 +178,15 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           // bias tile of the key tile whose visits start here; the buffer is free once all
           // softmax threads have copied the previous tile to registers
           const int tl = v / Bc;
-          if (!wait_or_abort(&bars->bias_empty, ((uint32_t)tl & 1u) ^ 1u, abort_flag, err)) break;
+          if (!wait_or_abort(&bars->bias_empty, ((uint32_t)tl & 1u) ^ 1u, abort_flag, err, max_polls)) break;
           mbar_arrive_expect_tx(&bars->bias_full, kBiasBytes);
 #pragma unroll
           for (int q = 0; q < 4; ++q)
             tma_load_3d(bias_s + q * (kBiasBytes / 4), &map_bias, &bars->bias_full, kt * kTile + 32 * q, qt * kTile, h);
           bias_loads = tl + 1;
         }
-        if (!wait_or_abort(&bars->in_empty[st], ph ^ 1u, abort_flag, err)) break;
+        if (!wait_or_abort(&bars->in_empty[st], ph ^ 1u, abort_flag, err, max_polls)) break;
+        if (dbg_skip != 0 && v == 0) continue;
         unsigned char *q_s = smem + (2 * st) * C::kTileBytes, *k_s = q_s + C::kTileBytes;
         mbar_arrive_expect_tx(&bars->in_full[st], 2 * C::kTileBytes);
 #pragma unroll
@@ -170,9 +196,11 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
       }
       if (*abort_flag) {  // winding down: let the copies in flight land (bounded)
-        for (int j = max(0, v - C::kStages); j < v; ++j)
-          mbar_wait(&bars->in_full[j % C::kStages], (uint32_t)(j / C::kStages) & 1u, kMaxPolls);
-        if (bias_loads > 0) mbar_wait(&bars->bias_full, (uint32_t)(bias_loads - 1) & 1u, kMaxPolls);
+        for (int j = max(0, v - C::kStages); j < v; ++j) {
+          if (dbg_skip != 0 && j == 0) continue;
+          mbar_wait(&bars->in_full[j % C::kStages], (uint32_t)(j / C::kStages) & 1u, max_polls);
+        }
+        if (bias_loads > 0) mbar_wait(&bars->bias_full, (uint32_t)(bias_loads - 1) & 1u, max_polls);
       }
     }
   } else if (warp == 9) {
@@ -183,8 +211,8 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int st = v % C::kStages;
         const uint32_t ph = (uint32_t)(v / C::kStages) & 1u;
         const int buf = v & 1;
-        if (!wait_or_abort(&bars->in_full[st], ph, abort_flag, err)) break;
-        if (!wait_or_abort(&bars->s_empty[buf], ((uint32_t)(v >> 1) & 1u) ^ 1u, abort_flag, err)) break;
+        if (!wait_or_abort(&bars->in_full[st], ph, abort_flag, err, max_polls)) break;
+        if (!wait_or_abort(&bars->s_empty[buf], ((uint32_t)(v >> 1) & 1u) ^ 1u, abort_flag, err, max_polls)) break;
         tc_fence_after_sync();
         const unsigned char *q_s = smem + (2 * st) * C::kTileBytes, *k_s = q_s + C::kTileBytes;
 #pragma unroll
@@ -207,140 +235,197 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const int jend = causal ? min(Lk, i + 1 + off) : Lk;  // first key outside this row's domain
     const bool vec = (Lk & 3) == 0;
-    float2 *my_stats = stats + (size_t)wg * kMaxB * 128 + r;  // + b * 128
-    for (int b = 0; b < Bc; ++b) my_stats[b * 128] = make_float2(-CUDART_INF_F, 0.f);
+    const uint32_t s_addr = tmem + lane_addr + 64 * wg;                   // + 128 * buf
+    const uint32_t sum_addr = tmem + lane_addr + kSumCol + 64 * wg;       // + 32 * c
+    const uint32_t my_stats = tmem + lane_addr + kStatsCol + 32 * wg;     // + 2 * b
+    const uint32_t other_stats = tmem + lane_addr + kStatsCol + 32 * (1 - wg);
+    // this warp's 32 rows x 32 columns on their way to the accumulator, and the rows' place in it
+    unsigned char *red_s = smem + C::kRedOffset + warp * kRedBytes;
+    const int red_y = qt * kTile + (warp & 3) * 32;
+    const int red_jend = causal ? min(Lk, red_y + 32 + off) : Lk;  // first key outside the domain of all 32 rows
+
+    for (int b = 0; b < Bc; ++b) tmem_st2(my_stats + 2 * b, __float_as_uint(-CUDART_INF_F), 0u);
 
     float bias2[64];  // bias * log2(e) of this thread's 64 columns of the current key tile
-    float ref = 0.f;  // sweep 2: max + log2(sum) of the current sample's row
     bool ok = true;
-    // (sweep, key tile, sample) of the visit, stepped rather than divided out of v: an integer
-    // division per visit is a hundred cycles on this thread's critical path
-    int sweep = 0, kt = 0, b = -1;
-    for (int v = 0; v < n_visits && ok; ++v) {
-      if (++b == Bc) {
-        b = 0;
-        if (++kt == n_k) {
-          kt = 0;
-          sweep = 1;
+    // the bias slice of key tile kt (tl: how many tiles were staged before it), once for all samples
+    auto fetch_bias = [&](int kt, int tl) {
+      const int j0 = kt * kTile + 64 * wg;
+      if (bias_by_tma) {
+        ok = warp_wait(&bars->bias_full, (uint32_t)tl & 1u, lane, abort_flag, err, max_polls);
+        if (!ok) return;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const unsigned char *box = bias_s + (2 * wg + q) * (kBiasBytes / 4) + r * 128;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {  // 16-byte chunk k of the row sits at position k ^ (r % 8)
+            const float4 t = *reinterpret_cast<const float4 *>(box + ((k ^ (r & 7)) << 4));
+            bias2[32 * q + 4 * k] = t.x * kLog2e; bias2[32 * q + 4 * k + 1] = t.y * kLog2e;
+            bias2[32 * q + 4 * k + 2] = t.z * kLog2e; bias2[32 * q + 4 * k + 3] = t.w * kLog2e;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->bias_empty);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+          const int j = j0 + 4 * c;
+          if (bias && row_ok) {
+            const float *brow = bias + ((size_t)h * Lq + i) * Lk;
+            if (j < Lk) t.x = brow[j];
+            if (j + 1 < Lk) t.y = brow[j + 1];
+            if (j + 2 < Lk) t.z = brow[j + 2];
+            if (j + 3 < Lk) t.w = brow[j + 3];
+          }
+          bias2[4 * c] = t.x * kLog2e; bias2[4 * c + 1] = t.y * kLog2e;
+          bias2[4 * c + 2] = t.z * kLog2e; bias2[4 * c + 3] = t.w * kLog2e;
         }
       }
+    };
+    // S of visit v is ready: copy this thread's 64 columns to registers and hand S back.  The MMA of
+    // visit v + 2 may then overwrite the buffer while the arithmetic on the copy is still going on
+    // (one arrival per warp: 256 threads arriving one by one would take longer than a visit's MMAs).
+    auto take_s = [&](int v, uint32_t (&xs)[64]) {
       const int buf = v & 1;
-      const int j0 = kt * kTile + 64 * wg;  // first column of this thread's slice
-      if (v == visits_per_sweep) {
-        // every statistic of sweep 1 is final once both column halves of every row are done
-        mbar_arrive(&bars->sweep1_done);
-        ok = wait_or_abort(&bars->sweep1_done, 0, abort_flag, err);
-        if (!ok) break;
-      }
-      if (b == 0) {  // new key tile: fetch this thread's bias slice once for all samples
-        if (bias_by_tma) {
-          const int tl = sweep * n_k + kt;
-          ok = wait_or_abort(&bars->bias_full, (uint32_t)tl & 1u, abort_flag, err);
-          if (!ok) break;
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            const unsigned char *box = bias_s + (2 * wg + q) * (kBiasBytes / 4) + r * 128;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {  // 16-byte chunk k of the row sits at position k ^ (r % 8)
-              const float4 t = *reinterpret_cast<const float4 *>(box + ((k ^ (r & 7)) << 4));
-              bias2[32 * q + 4 * k] = t.x * kLog2e; bias2[32 * q + 4 * k + 1] = t.y * kLog2e;
-              bias2[32 * q + 4 * k + 2] = t.z * kLog2e; bias2[32 * q + 4 * k + 3] = t.w * kLog2e;
-            }
-          }
-          mbar_arrive(&bars->bias_empty);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-            const int j = j0 + 4 * c;
-            if (bias && row_ok) {
-              const float *brow = bias + ((size_t)h * Lq + i) * Lk;
-              if (j < Lk) t.x = brow[j];
-              if (j + 1 < Lk) t.y = brow[j + 1];
-              if (j + 2 < Lk) t.z = brow[j + 2];
-              if (j + 3 < Lk) t.w = brow[j + 3];
-            }
-            bias2[4 * c] = t.x * kLog2e; bias2[4 * c + 1] = t.y * kLog2e;
-            bias2[4 * c + 2] = t.z * kLog2e; bias2[4 * c + 3] = t.w * kLog2e;
-          }
-        }
-      }
-      if (sweep == 1) {
-        // combine the two column halves' statistics of sample b: max + log2(sum)
-        const float2 s0 = stats[(size_t)b * 128 + r], s1 = stats[(size_t)(kMaxB + b) * 128 + r];
-        const float mm = fmaxf(s0.x, s1.x);
-        const float z = s0.y * ex2_approx(s0.x - mm) + s1.y * ex2_approx(s1.x - mm);
-        ref = mm + lg2_approx(z);
-      }
-      ok = wait_or_abort(&bars->s_full[buf], (uint32_t)(v >> 1) & 1u, abort_flag, err);
-      if (!ok) break;
+      ok = warp_wait(&bars->s_full[buf], (uint32_t)(v >> 1) & 1u, lane, abort_flag, err, max_polls);
+      if (!ok) return;
       tc_fence_after_sync();
+      tmem_ld32(s_addr + 128 * buf, xs);
+      tmem_ld32(s_addr + 128 * buf + 32, xs + 32);
+    };
+    auto release_s = [&](int v) {
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->s_empty[v & 1]);
+    };
+
+    // ---- sweep 1: per sample and row, the maximum and the sum of exp2 over this thread's columns
+    int v = 0;
+    for (int kt = 0; kt < n_k && ok; ++kt) {
+      fetch_bias(kt, kt);
+      if (!ok) break;
       // columns of this slice inside the row's domain; whole warp inside => no masking
+      const int n_valid = max(0, min(64, jend - (kt * kTile + 64 * wg)));
+      const bool interior = __all_sync(0xffffffffu, n_valid == 64);
+      for (int b = 0; b < Bc; ++b, ++v) {
+        uint32_t xs[64], sv[2];
+        take_s(v, xs);
+        if (!ok) break;
+        tmem_wait_st();  // this sample's pair as the previous key tile left it
+        tmem_ld2(my_stats + 2 * b, sv);
+        tmem_wait_ld();
+        release_s(v);
+        float t[64];
+#pragma unroll
+        for (int e = 0; e < 64; e += 2)
+          ffma2(t[e], t[e + 1], __uint_as_float(xs[e]), __uint_as_float(xs[e + 1]), scale_log2, bias2[e], bias2[e + 1]);
+        if (!interior) {
+#pragma unroll
+          for (int e = 0; e < 64; ++e) t[e] = e < n_valid ? t[e] : -CUDART_INF_F;
+        }
+        const float m_old = __uint_as_float(sv[0]);
+        // four independent chains each for the maximum and for the sum
+        float m0 = m_old, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
+#pragma unroll
+        for (int e = 0; e < 64; e += 8) {  // three-input maxima: half the instructions
+          m0 = fmax3(m0, t[e], t[e + 4]);
+          m1 = fmax3(m1, t[e + 1], t[e + 5]);
+          m2 = fmax3(m2, t[e + 2], t[e + 6]);
+          m3 = fmax3(m3, t[e + 3], t[e + 7]);
+        }
+        const float cm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        const float cm_safe = cm == -CUDART_INF_F ? 0.f : cm;
+        float z0 = __uint_as_float(sv[1]) * ex2_approx(m_old - cm_safe), z1 = 0.f, z2 = 0.f, z3 = 0.f;
+        const float neg_cm = -cm_safe;
+#pragma unroll
+        for (int e = 0; e < 64; e += 4) {
+          float a0, a1, a2, a3;
+          fadd2(a0, a1, t[e], t[e + 1], neg_cm, neg_cm);
+          fadd2(a2, a3, t[e + 2], t[e + 3], neg_cm, neg_cm);
+          fadd2(z0, z1, z0, z1, ex2_approx(a0), ex2_approx(a1));
+          fadd2(z2, z3, z2, z3, ex2_approx(a2), ex2_approx(a3));
+        }
+        tmem_st2(my_stats + 2 * b, __float_as_uint(cm), __float_as_uint((z0 + z1) + (z2 + z3)));
+      }
+    }
+    if (ok) {
+      // every statistic of sweep 1 is final once both column halves of every row are done
+      tmem_wait_st();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->sweep1_done);
+      ok = warp_wait(&bars->sweep1_done, 0, lane, abort_flag, err, max_polls);
+      tc_fence_after_sync();
+    }
+
+    // ---- sweep 2: normalised weights, summed over b in TMEM, added to the accumulator per key tile
+    for (int kt = 0; kt < n_k && ok; ++kt) {
+      fetch_bias(kt, n_k + kt);
+      if (!ok) break;
+      const int j0 = kt * kTile + 64 * wg;  // first column of this thread's slice
       const int n_valid = max(0, min(64, jend - j0));
       const bool interior = __all_sync(0xffffffffu, n_valid == 64);
-      float2 st = sweep == 0 ? my_stats[b * 128] : make_float2(0.f, 0.f);
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t x[32];
-        tmem_ld32(tmem + 128 * buf + 64 * wg + 32 * c + lane_addr, x);
+      for (int b = 0; b < Bc; ++b, ++v) {
+        uint32_t xs[64], s0[2], s1[2];
+        take_s(v, xs);
+        if (!ok) break;
+        tmem_ld2(my_stats + 2 * b, s0);
+        tmem_ld2(other_stats + 2 * b, s1);
         tmem_wait_ld();
-        float t[32];
-        if (interior) {  // the usual case: nothing to mask, no per-entry comparison
+        release_s(v);
+        // both column halves' statistics of sample b combined: max + log2(sum).  A row without any key
+        // in its domain (possible when Lk < Lq) gets weight 0 everywhere.
+        const float mm = fmaxf(__uint_as_float(s0[0]), __uint_as_float(s1[0]));
+        const float z = __uint_as_float(s0[1]) * ex2_approx(__uint_as_float(s0[0]) - mm) +
+                        __uint_as_float(s1[1]) * ex2_approx(__uint_as_float(s1[0]) - mm);
+        const float neg_ref = jend > 0 ? -(mm + lg2_approx(z)) : -CUDART_INF_F;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          float p[32];
 #pragma unroll
           for (int e = 0; e < 32; e += 2)
-            ffma2(t[e], t[e + 1], __uint_as_float(x[e]), __uint_as_float(x[e + 1]), scale_log2, bias2[32 * c + e],
-                  bias2[32 * c + e + 1]);
-        } else {
+            ffma2(p[e], p[e + 1], __uint_as_float(xs[32 * c + e]), __uint_as_float(xs[32 * c + e + 1]), scale_log2,
+                  bias2[32 * c + e], bias2[32 * c + e + 1]);
+          if (!interior) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
-            t[e] = 32 * c + e < n_valid ? fmaf(__uint_as_float(x[e]), scale_log2, bias2[32 * c + e]) : -CUDART_INF_F;
-        }
-        if (sweep == 0) {
-          // four independent chains each for the maximum and for the sum
-          float m0 = st.x, m1 = -CUDART_INF_F, m2 = -CUDART_INF_F, m3 = -CUDART_INF_F;
-#pragma unroll
-          for (int e = 0; e < 32; e += 8) {  // three-input maxima: half the instructions
-            m0 = fmax3(m0, t[e], t[e + 4]);
-            m1 = fmax3(m1, t[e + 1], t[e + 5]);
-            m2 = fmax3(m2, t[e + 2], t[e + 6]);
-            m3 = fmax3(m3, t[e + 3], t[e + 7]);
+            for (int e = 0; e < 32; ++e) p[e] = 32 * c + e < n_valid ? p[e] : -CUDART_INF_F;
           }
-          const float cm = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-          const float cm_safe = cm == -CUDART_INF_F ? 0.f : cm;
-          float z0 = st.y * ex2_approx(st.x - cm_safe), z1 = 0.f, z2 = 0.f, z3 = 0.f;
-          const float neg_cm = -cm_safe;
-#pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            float a0, a1, a2, a3;
-            fadd2(a0, a1, t[e], t[e + 1], neg_cm, neg_cm);
-            fadd2(a2, a3, t[e + 2], t[e + 3], neg_cm, neg_cm);
-            fadd2(z0, z1, z0, z1, ex2_approx(a0), ex2_approx(a1));
-            fadd2(z2, z3, z2, z3, ex2_approx(a2), ex2_approx(a3));
-          }
-          st = make_float2(cm, (z0 + z1) + (z2 + z3));
-        } else {
-          // running sum over b of the normalised weights, kept in TMEM next to S
-          const uint32_t ps_addr = tmem + 256 + 64 * wg + 32 * c + lane_addr;
           uint32_t ps[32];
           if (b > 0) {
-            tmem_ld32(ps_addr, ps);
+            tmem_ld32(sum_addr + 32 * c, ps);
             tmem_wait_ld();
           }
-          const float neg_ref = -ref;
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             float a0, a1;
-            fadd2(a0, a1, t[e], t[e + 1], neg_ref, neg_ref);
+            fadd2(a0, a1, p[e], p[e + 1], neg_ref, neg_ref);
             float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
             if (b > 0) fadd2(p0, p1, __uint_as_float(ps[e]), __uint_as_float(ps[e + 1]), p0, p1);
             ps[e] = __float_as_uint(p0);
             ps[e + 1] = __float_as_uint(p1);
           }
           if (b < Bc - 1) {
-            tmem_st32(ps_addr, ps);
+            tmem_st32(sum_addr + 32 * c, ps);
+          } else if (acc_by_tma) {
+            // last sample of this key tile: one addition per accumulator entry and launch, performed
+            // in L2 by a TMA reduction of this warp's 32 x 32 block
+            if (lane == 0) bulk_wait_group_read0();  // the block staged before has been read
+            __syncwarp();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)  // 16-byte chunk k of row `lane` goes to position k ^ (lane % 8)
+              *reinterpret_cast<uint4 *>(red_s + lane * 128 + ((k ^ (lane & 7)) << 4)) =
+                  make_uint4(ps[4 * k], ps[4 * k + 1], ps[4 * k + 2], ps[4 * k + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            const int x = j0 + 32 * c;
+            if (lane == 0 && red_y < Lq && x < red_jend) {
+              tma_reduce_add_3d(&map_acc, red_s, x, red_y, h);
+              bulk_commit_group();
+            }
           } else if (row_ok) {
-            // last sample of this key tile: one addition per accumulator entry and launch,
-            // performed in L2 (entries outside the domain are not touched)
+            // accumulator rows that are no 16-byte multiples: one red per entry (entries outside the
+            // domain are not touched)
             float *arow = acc + ((size_t)h * Lq + i) * Lk + j0 + 32 * c;
             const int nv = n_valid - 32 * c;
 #pragma unroll
@@ -362,13 +447,11 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
           }
         }
+        // the sums must be in TMEM before the next visit reads them
+        if (b < Bc - 1) tmem_wait_st();
       }
-      // S[buf] is consumed: the MMA of visit v + 2 may overwrite it
-      if (sweep == 1 && b < Bc - 1) tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(&bars->s_empty[buf]);
-      if (sweep == 0) my_stats[b * 128] = st;
     }
+    if (lane == 0) bulk_wait_group0();  // shared memory stays valid until the reductions have read it
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -376,18 +459,20 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 }
 
 template <int D>
-cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mb, int bias_by_tma, float *acc,
-                   const float *bias, int B, int H, int Lq, int Lk, int causal, int f16, float scale, unsigned *err,
-                   cudaStream_t s) {
+cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mb, const CUtensorMap &ma,
+                   int bias_by_tma, int acc_by_tma, float *acc, const float *bias, int B, int H, int Lq, int Lk,
+                   int causal, int f16, float scale, unsigned *err, cudaStream_t s) {
   auto kern = accumulate_tc_kernel<D>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int n_qt = ceil_div(Lq, kTile), n_kt = ceil_div(Lk, kTile);
+  const DebugKnobs knobs = debug_knobs();
   // samples in ascending order, at most kMaxB per launch; launches on one stream run in order
   for (int b0 = 0; b0 < B; b0 += kMaxB) {
     const int Bc = B - b0 < kMaxB ? B - b0 : kMaxB;
-    kern<<<H * n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(mq, mk, mb, bias_by_tma, acc, bias, b0, Bc, H, Lq, Lk, n_qt,
-                                                       n_kt, causal, f16, scale * kLog2e, err);
+    kern<<<knobs.skip_arrive ? 1 : H * n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(
+        mq, mk, mb, ma, bias_by_tma, acc_by_tma, acc, bias, b0, Bc, H, Lq, Lk, n_qt, n_kt, causal, f16, scale * kLog2e,
+        err, knobs.max_polls, knobs.skip_arrive);
     count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -406,8 +491,13 @@ cudaError_t launch_accumulate_tc(float *acc, const void *Q, const void *K, const
   CUtensorMap mb = mq;
   const int bias_by_tma = (bias && (Lk & 3) == 0) ? 1 : 0;
   if (bias_by_tma && !make_tile_map_f32(&mb, bias, H, Lq, Lk)) return cudaErrorUnknown;
-  return d == 64 ? launch<64>(mq, mk, mb, bias_by_tma, acc, bias, B, H, Lq, Lk, causal, f16, scale, err, s)
-                 : launch<128>(mq, mk, mb, bias_by_tma, acc, bias, B, H, Lq, Lk, causal, f16, scale, err, s);
+  // so does the accumulator's update (32-row boxes, one per softmax warp)
+  CUtensorMap ma = mq;
+  const int acc_by_tma = (Lk & 3) == 0 ? 1 : 0;
+  if (acc_by_tma && !make_tile_map_f32(&ma, acc, H, Lq, Lk, 32)) return cudaErrorUnknown;
+  return d == 64
+             ? launch<64>(mq, mk, mb, ma, bias_by_tma, acc_by_tma, acc, bias, B, H, Lq, Lk, causal, f16, scale, err, s)
+             : launch<128>(mq, mk, mb, ma, bias_by_tma, acc_by_tma, acc, bias, B, H, Lq, Lk, causal, f16, scale, err, s);
 }
 
 }  // namespace ap

@@ -131,8 +131,9 @@ cudaError_t launch_fwd_entmax_tc(const void *Q, const void *K, const void *V, co
 // unchanged and fills out-of-range elements with zero bits) for box_rows-row x 64-element swizzled boxes.
 bool make_tile_map_bf16(CUtensorMap *m, const void *base, int BH, int L, int d, int box_rows = 128);
 bool make_split_map_bf16_d128(CUtensorMap *m, const void *base, int BH, int L, int box_rows);
-// Tensor map of an [H, Lq, Lk] fp32 tensor for 128-row x 32-column swizzled boxes (Lk % 4 == 0).
-bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk);
+// Tensor map of an [H, Lq, Lk] fp32 tensor for box_rows x 32-column swizzled boxes (Lk % 4 == 0,
+// base 16-byte aligned).
+bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk, int box_rows = 128);
 
 // bf16 tensors: tcgen05 tensor-core kernel
 cudaError_t launch_pool_scores(const float *acc, int H, int Lq, int Lk, int bs, int causal, float *pooled,

@@ -57,12 +57,12 @@ bool make_split_map_bf16_d128(CUtensorMap *m, const void *base, int BH, int L, i
 
 // [H, Lq, Lk] fp32 tensor, boxes of 128 rows x 32 columns (128 bytes), 128-byte swizzle, zero fill outside.
 // Needs Lk % 4 == 0 (row pitch a multiple of 16 bytes).
-bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk) {
+bool make_tile_map_f32(CUtensorMap *m, const void *base, int H, int Lq, int Lk, int box_rows) {
   EncodeTiledFn enc = encode_fn();
   if (!enc) return false;
   cuuint64_t dims[3] = {(cuuint64_t)Lk, (cuuint64_t)Lq, (cuuint64_t)H};
   cuuint64_t strides[2] = {(cuuint64_t)Lk * 4, (cuuint64_t)Lq * Lk * 4};
-  cuuint32_t box[3] = {32, 128, 1};
+  cuuint32_t box[3] = {32, (cuuint32_t)box_rows, 1};
   cuuint32_t elem_strides[3] = {1, 1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, elem_strides,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
