@@ -37,3 +37,30 @@ def test_forward_expired_wait_returns_timeout_once_and_the_next_call_is_correct(
     assert ap.ap_device_status() == ap.AP_OK
     ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy())
     assert_close_attention(out, ref, "bf16", "after an expired wait")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [64, 128])
+def test_accumulate_expired_wait_returns_timeout_once_and_the_next_call_is_correct(d):
+    from paper_2012_02030_b200 import binding as ap
+
+    B, H, L = 2, 2, 256
+    gen = torch.Generator().manual_seed(4200 + d)
+    q, k = (torch.randn((B, H, L, d), generator=gen).to(torch.bfloat16) for _ in range(2))
+    bias = 0.5 * torch.randn((H, L, L), generator=gen)
+    qd, kd, bd = q.cuda(), k.cuda(), bias.cuda()
+    scratch = torch.zeros((H, L, L), device="cuda")
+    assert ap.ap_device_status() == ap.AP_OK
+    ap.ap_debug_expire_waits(True)
+    try:
+        ap.ap_accumulate_attention(scratch, qd, kd, bd, causal=True)   # the first visit's operands never arrive
+        assert ap.ap_device_status() == ap.AP_ERR_TIMEOUT
+    finally:
+        ap.ap_debug_expire_waits(False)
+    assert ap.ap_device_status() == ap.AP_OK
+    acc = torch.zeros((H, L, L), device="cuda")
+    ap.ap_accumulate_attention(acc, qd, kd, bd, causal=True)
+    assert ap.ap_device_status() == ap.AP_OK
+    want = np.zeros((H, L, L))
+    orc.accumulate(want, inputs.widen(q), inputs.widen(k), bias.numpy(), causal=True)
+    np.testing.assert_allclose(acc.cpu().numpy(), want, rtol=2e-5, atol=1e-7 * B)
