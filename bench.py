@@ -338,6 +338,52 @@ def density_section(ap, w, acc, q, k, v, out, ws, dense_ms, dense_tiles, peaks, 
     return {"shape": w.name, "dense_path_ms": dense_ms, "dense_tiles": dense_tiles,
             "timing": "10 launches back to back after 3 warm-up launches; the tensors exceed L2", "rows": rows}
 
+def gathered_section(ap, w, acc, q, k, v, out, ws, dev):
+    """The tile list's second schedule (rounds of individually gathered key columns) against the rounds, on the
+    bench's shape: under the method's own masks (where the builders' rule decides per list row) and under
+    column-structured synthetic masks (single key columns shared by the rows of a query tile)."""
+    rows = []
+    tiles = ap.Tiles(w.H, w.Lq, w.Lk, device=dev, gathered=True)
+    nnz = torch.zeros((w.H,), dtype=torch.int64, device=dev)
+
+    def measure(label, build):
+        row = {"mask": label}
+        for mode, key in ((1, "rounds"), (0, "gathered_where_the_rule_allows"), (2, "gathered_everywhere")):
+            ap.ap_debug_schedule(mode)
+            try:
+                build()
+                for _ in range(3):
+                    ap.ap_sparse_attention_fwd(q, k, v, tiles, out)
+                row[key + "_ms"] = _time_back_to_back(lambda i: ap.ap_sparse_attention_fwd(q, k, v, tiles, out), 10)
+            finally:
+                ap.ap_debug_schedule(0)
+            rp, gp = tiles.round_ptr.diff(), tiles.ground_ptr.diff()
+            if mode == 1:
+                row["rounds"] = int(rp.sum().item())
+            else:
+                row[key + "_rounds_followed"] = int(torch.where(gp > 0, gp, rp).sum().item())
+                row[key + "_list_rows"] = int((gp > 0).sum().item())
+        rows.append(row)
+
+    for keep in (0.10, 0.05):
+        measure("method's mask, keep %g" % keep,
+                lambda: ap.ap_build_mask(acc, keep, w.causal, w.keep_diag, None, tiles, nnz, ws))
+    gen = torch.Generator(device=dev).manual_seed(11)
+    i = torch.arange(w.Lq, device=dev)[:, None]
+    inside = (torch.arange(w.Lk, device=dev)[None, :] <= i + (w.Lk - w.Lq)) if w.causal else None
+    for frac in (0.05, 0.3):
+        sel = torch.rand((w.H, -(-w.Lq // 128), w.Lk), device=dev, generator=gen) < frac
+        mask = sel.repeat_interleave(128, dim=1)[:, :w.Lq]
+        if inside is not None:
+            mask = mask & inside[None]
+        mask = mask.to(torch.uint8)
+        del sel
+        measure("single columns per query tile, %g of the keys" % frac, lambda: ap.ap_mask_to_tiles(mask, tiles))
+        del mask
+    if ap.ap_device_status() != ap.AP_OK:
+        raise RuntimeError("device status not OK in the gathered section")
+    return {"shape": w.name, "list_rows": w.H * (-(-w.Lq // 128)),
+            "timing": "10 launches back to back after 3 warm-up launches; the tensors exceed L2", "rows": rows}
 
 
 def run_gpu(args, w):
@@ -558,10 +604,11 @@ def run_gpu(args, w):
                           "entries_given_weight = fraction of the domain that received weight from any sample" % n_ent}
 
     # ---- the forward at other kept fractions on this shape, and the small workloads (outside the step) ----
-    density = workloads = None
+    density = workloads = gathered = None
     if not args.no_extras:
         if w.dtype != "f32":
             density = density_section(ap, w, acc, q, k, v, out, ws, stage_ms["dense_fwd"], T_dense, peaks, dev)
+            gathered = gathered_section(ap, w, acc, q, k, v, out, ws, dev)
         if world == 1:
             workloads = workloads_section(ap, dev, peaks, not args.no_cpu_baseline)
 
@@ -673,7 +720,7 @@ def run_gpu(args, w):
         "stage_ms_best": {s_: stage_all[s_]["best"] for s_ in stages},
         "tokens_per_s": replicas.job_throughput(info, w.B * w.Lq, fwd_ms_max * 1e-3),
         "speedup_vs_dense_path": stage_ms["dense_fwd"] / stage_ms["sparse_fwd"],
-        "density": {"kept_fraction": nnz_total / float(dom), "tiles_kept": T_sparse, "tiles_domain": T_dense,
+        "mask": {"kept_fraction": nnz_total / float(dom), "tiles_kept": T_sparse, "tiles_domain": T_dense,
                     "tile_fill": nnz_total / (T_sparse * 128.0 * 128.0) if T_sparse else None},
         "pct_of_bf16_roofline": {"effective_flops_burst": 100 * eff_flops / fwd_s / 1e12 / peaks["bf16"],
                                  "tile_flops_burst": 100 * tile_fl / fwd_s / 1e12 / peaks["bf16"],
@@ -683,7 +730,7 @@ def run_gpu(args, w):
         "e2e": {"value": replicas.job_throughput(info, eff_flops, e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": int(launches), "clocks": clocks, "layer_threshold": layer, "backward": backward,
-        "entmax15": entmax, "workloads": workloads, "density": density,
+        "entmax15": entmax, "workloads": workloads, "density": density, "gathered_rounds": gathered,
         "graph_replay": {"ms_per_step": graph_ms, "note": "the same step (same calibration batch every replay) "
                          "captured once in a CUDA graph; steps replays timed with one pair of events"},
     }

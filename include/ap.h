@@ -98,6 +98,30 @@ typedef enum { AP_F32 = 0, AP_BF16 = 1, AP_F16 = 2 } ap_dtype; /* AP_F16: IEEE h
  * ap_dense_tiles) writes groups and the round arrays along with the tile list; a
  * list assembled by hand must provide them too for ap_sparse_attention_fwd.
  *
+ * Gathered rounds: an optional second schedule (all four pointers null, or all four
+ * set; the CSR arrays and the rounds above do not depend on it).  A list row's ACTIVE
+ * KEY COLUMNS - the keys that at least one of the 128 query rows keeps - are put in
+ * this order: first the columns of the 16-column groups [16g, 16g+16) in which every
+ * column is active, then all other active columns, ascending in each part; gathered
+ * round k of the list row consists of columns [128k, 128k+128) of that order, whatever
+ * key tiles they come from, so a list row with c active columns has ceil(c/128)
+ * gathered rounds (never more than its rounds above).  The builders give a list row
+ * gathered rounds only where the forward is expected to gain from them: with r rounds,
+ * g = ceil(c/128) and s = ceil((c - 16 w)/16), w the number of those whole groups, if
+ * 2 r > 4 g + s; other list rows have none.
+ *   ground_ptr[H*n_qt + 1]      offsets into the gathered-round arrays, per list row;
+ *                               all zero: no gathered schedule (ap_dense_tiles)
+ *   ground_keys[cap][128]       key index of each column of a gathered round; the unused
+ *                               tail of a row's last round repeats its last key
+ *   ground_info[cap]            bits 0..3: ceil(columns / 16), 1..8 (the forward computes
+ *                               that many 16-column slots); bit 7: 128 columns, all kept
+ *   ground_bitmap[cap][128][4]  bit p of the 128-bit row r: query row r keeps column p
+ *                               of the round; 0 for unused columns
+ * ap_sparse_attention_fwd follows the gathered rounds of a list row that has some (a
+ * slot of 16 keys that follow one another from a multiple of 8 on is fetched as one box,
+ * the rows of other slots one by one), the rounds otherwise; the result is the same
+ * masked attention either way.
+ *
  * cap is the capacity in tiles; ap_tiles_capacity() always suffices.
  */
 typedef struct ap_tiles {
@@ -113,6 +137,10 @@ typedef struct ap_tiles {
   int32_t *round_rows;
   uint8_t *round_info;
   uint32_t *round_bitmap;
+  int32_t *ground_ptr;
+  int32_t *ground_keys;
+  uint8_t *ground_info;
+  uint32_t *ground_bitmap;
 } ap_tiles;
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -132,6 +160,17 @@ uint64_t ap_launch_count(void);
  * undefined.  on == 0 restores normal operation.  Process-wide; not for production use.
  */
 void ap_debug_expire_waits(int on);
+
+/*
+ * Test and measurement hook (no counterpart in the paper) for the two schedules of a tile list.
+ * 0 (the default): the builders give a list row gathered rounds where they are expected to pay, and
+ * ap_sparse_attention_fwd (16-bit types) follows them where a list row has some.  1: the forward
+ * follows the rounds only.  2: the builders give every list row with a kept entry its gathered
+ * rounds (and the forward follows them).  The forward's output is the same masked attention in
+ * every mode (the exponentials are summed in a different order, so the last bit may differ).
+ * Process-wide.
+ */
+void ap_debug_schedule(int mode);
 
 /* Static, human-readable name of a status code. */
 const char *ap_status_string(ap_status s);

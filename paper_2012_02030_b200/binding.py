@@ -36,6 +36,8 @@ class ap_tiles(ctypes.Structure):
         ("flags", ctypes.c_void_p), ("bitmap", ctypes.c_void_p), ("groups", ctypes.c_void_p),
         ("round_ptr", ctypes.c_void_p), ("round_rows", ctypes.c_void_p), ("round_info", ctypes.c_void_p),
         ("round_bitmap", ctypes.c_void_p),
+        ("ground_ptr", ctypes.c_void_p), ("ground_keys", ctypes.c_void_p), ("ground_info", ctypes.c_void_p),
+        ("ground_bitmap", ctypes.c_void_p),
     ]
 
 
@@ -52,6 +54,7 @@ def _load() -> ctypes.CDLL:
         "ap_version": (i, []),
         "ap_launch_count": (ctypes.c_uint64, []),
         "ap_debug_expire_waits": (None, [i]),
+        "ap_debug_schedule": (None, [i]),
         "ap_status_string": (ctypes.c_char_p, [i]),
         "ap_tiles_capacity": (i64, [i, i, i]),
         "ap_build_mask_workspace_bytes": (sz, [i, i, i]),
@@ -81,7 +84,7 @@ def _load() -> ctypes.CDLL:
 
 
 lib = _load()
-EXPORTS = ("ap_version", "ap_launch_count", "ap_debug_expire_waits", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
+EXPORTS = ("ap_version", "ap_launch_count", "ap_debug_expire_waits", "ap_debug_schedule", "ap_status_string", "ap_tiles_capacity", "ap_build_mask_workspace_bytes",
            "ap_mask_to_tiles_workspace_bytes", "ap_accumulate_attention", "ap_accumulate_attention_entmax15", "ap_build_mask", "ap_build_mask_layer", "ap_build_mask_ex", "ap_random_scores", "ap_pool_scores", "ap_expand_block_mask",
            "ap_mask_to_tiles", "ap_mask_to_tiles_static", "ap_dense_tiles", "ap_sparse_attention_fwd", "ap_sparse_attention_entmax15_fwd",
            "ap_sparse_attention_fwd_host", "ap_sparse_attention_bwd_workspace_bytes", "ap_sparse_attention_bwd",
@@ -105,6 +108,12 @@ def ap_launch_count() -> int:
 
 def ap_debug_expire_waits(on: bool) -> None:
     lib.ap_debug_expire_waits(1 if on else 0)
+
+
+def ap_debug_schedule(mode: int) -> None:
+    """0: gathered rounds where the builders expect them to pay; 1: the forward follows the rounds only;
+    2: the builders give every list row its gathered rounds."""
+    lib.ap_debug_schedule(int(mode))
 
 
 def ap_tiles_capacity(H: int, Lq: int, Lk: int) -> int:
@@ -153,7 +162,7 @@ def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
 class Tiles:
     """Device buffers of a tile list plus the ap_tiles descriptor that points at them."""
 
-    def __init__(self, H: int, Lq: int, Lk: int, device="cuda", cap: int | None = None):
+    def __init__(self, H: int, Lq: int, Lk: int, device="cuda", cap: int | None = None, gathered: bool = False):
         self.H, self.Lq, self.Lk = H, Lq, Lk
         self.n_qt, self.n_kt = -(-Lq // TILE), -(-Lk // TILE)
         self.cap = ap_tiles_capacity(H, Lq, Lk) if cap is None else cap
@@ -167,10 +176,20 @@ class Tiles:
         self.round_rows = torch.zeros((max(self.cap, 1), 8), dtype=torch.int32, device=device)
         self.round_info = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
         self.round_bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
+        # the optional second schedule (rounds of 128 individually gathered key columns)
+        self.gathered = gathered
+        g = [None] * 4
+        if gathered:
+            self.ground_ptr = torch.zeros(H * self.n_qt + 1, dtype=torch.int32, device=device)
+            self.ground_keys = torch.zeros((max(self.cap, 1), TILE), dtype=torch.int32, device=device)
+            self.ground_info = torch.zeros(max(self.cap, 1), dtype=torch.uint8, device=device)
+            self.ground_bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
+            g = [self.ground_ptr.data_ptr(), self.ground_keys.data_ptr(), self.ground_info.data_ptr(),
+                 self.ground_bitmap.data_ptr()]
         self.c = ap_tiles(H, Lq, Lk, self.n_qt, self.n_kt, self.cap, self.row_ptr.data_ptr(),
                           self.col_idx.data_ptr(), self.flags.data_ptr(), self.bitmap.data_ptr(),
                           self.groups.data_ptr(), self.round_ptr.data_ptr(), self.round_rows.data_ptr(),
-                          self.round_info.data_ptr(), self.round_bitmap.data_ptr())
+                          self.round_info.data_ptr(), self.round_bitmap.data_ptr(), *g)
 
     def n_tiles(self) -> int:
         """Number of stored tiles (synchronises)."""
@@ -183,6 +202,13 @@ class Tiles:
                     flags=self.flags[:T].cpu().numpy(), groups=self.groups[:T].cpu().numpy(),
                     bitmap=self.bitmap[:T].cpu().numpy().view("uint32"), n_qt=self.n_qt, n_kt=self.n_kt,
                     **self.rounds_to_host())
+
+    def grounds_to_host(self):
+        """The gathered-round arrays trimmed to the stored gathered rounds (synchronises)."""
+        R = int(self.ground_ptr[-1].item())
+        return dict(ground_ptr=self.ground_ptr.cpu().numpy(), ground_keys=self.ground_keys[:R].cpu().numpy(),
+                    ground_info=self.ground_info[:R].cpu().numpy(),
+                    ground_bitmap=self.ground_bitmap[:R].cpu().numpy().view("uint32"))
 
     def rounds_to_host(self):
         """The round arrays trimmed to the stored rounds (synchronises)."""

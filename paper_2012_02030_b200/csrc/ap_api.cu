@@ -44,10 +44,11 @@ bool have_device() {
 }  // namespace
 
 std::atomic<int> g_expire_waits{0};
+std::atomic<int> g_schedule{0};
 
 DebugKnobs debug_knobs() {
   const int on = g_expire_waits.load(std::memory_order_relaxed);
-  return DebugKnobs{on ? (1u << 12) : (1u << 22), on};
+  return DebugKnobs{on ? (1u << 12) : (1u << 22), on, g_schedule.load(std::memory_order_relaxed)};
 }
 
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
@@ -85,6 +86,10 @@ extern "C" {
 int ap_version(void) { return 200; }
 
 void ap_debug_expire_waits(int on) { ap::g_expire_waits.store(on ? 1 : 0, std::memory_order_relaxed); }
+
+void ap_debug_schedule(int mode) {
+  ap::g_schedule.store(mode == 1 || mode == 2 ? mode : 0, std::memory_order_relaxed);
+}
 
 uint64_t ap_launch_count(void) { return (uint64_t)g_launches.load(std::memory_order_relaxed); }
 

@@ -36,6 +36,12 @@ inline ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shap
   if (misaligned(t->bitmap, 15u) || misaligned(t->round_bitmap, 15u) || misaligned(t->round_rows, 15u) ||
       misaligned(t->row_ptr, 3u) || misaligned(t->col_idx, 3u) || misaligned(t->round_ptr, 3u))
     return AP_ERR_INVALID_ARG;
+  // the gathered rounds are optional: all four arrays or none
+  const int n_g = (t->ground_ptr != nullptr) + (t->ground_keys != nullptr) + (t->ground_info != nullptr) +
+                  (t->ground_bitmap != nullptr);
+  if (n_g != 0 && n_g != 4) return AP_ERR_INVALID_ARG;
+  if (n_g == 4 && (misaligned(t->ground_bitmap, 15u) || misaligned(t->ground_keys, 15u) || misaligned(t->ground_ptr, 3u)))
+    return AP_ERR_INVALID_ARG;
   if (t->cap < 1) return AP_ERR_WORKSPACE;
   if (shape_must_match) {
     if (t->H != H || t->Lq != Lq || t->Lk != Lk || t->n_qt != ceil_div(Lq, kTile) ||
@@ -51,6 +57,7 @@ inline ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shap
 struct DebugKnobs {
   uint32_t max_polls;
   int skip_arrive;
+  int schedule;  // ap_debug_schedule: 0 = gathered rounds where they pay, 1 = never followed, 2 = built for every list row
 };
 DebugKnobs debug_knobs();
 

@@ -76,7 +76,7 @@ struct Cfg {
   static constexpr int kKOffset = 2 * kTileBytes;     // after the two Q buffers
   static constexpr int kVOffset = kKOffset + kStages * kTileBytes;
   static constexpr int kBarOffset = kVOffset + kStages * kTileBytes;
-  static constexpr int kSmemBytes = kBarOffset + 17 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
+  static constexpr int kSmemBytes = kBarOffset + 18 * 1024 + 1024;  // + bitmaps/barriers + alignment slack
   static constexpr int kHalfStride = kSplit ? 1024 : kSubBytes;          // half 0 -> half 1 of the same rows
   static constexpr int kSbo = kSplit ? 2048 : 1024;                      // one group of 8 rows -> the next
   static constexpr int kSlotStride = 2 * kSbo;                           // 16 rows (one slot) -> the next
@@ -87,6 +87,17 @@ struct FwdMaps {
   CUtensorMap q;
   CUtensorMap k[4];
   CUtensorMap v[4];
+};
+
+// The second schedule of a tile list, followed for the list rows that have gathered rounds.
+struct Gathered {
+  const int32_t *ptr;
+  const int32_t *keys;
+  const uint8_t *info;
+  const uint32_t *bitmap;
+  const uint16_t *K, *V;  // the tensors themselves: single key rows are fetched with plain asynchronous copies
+  int Lk;
+  int mode;
 };
 
 struct Shared {
@@ -102,6 +113,7 @@ struct Shared {
   uint64_t ml_ready[4];                               // per item: both groups have handed over (m, l)
   float2 ml[4][2][kTile];                             // [item % 4][group][row] = (m, l)
   int32_t ml_bh[4], ml_qt[4];                         // the item handed over (b * H + h, query tile); qt = -1: no more items
+  alignas(16) int32_t keys[2][kTile];                 // producer's scratch: keys of a gathered round (two rounds in flight)
   uint32_t info[kMaxStages];
   int32_t item_bh[kMaxStages], item_qt[kMaxStages];   // the item a stage's round belongs to
   uint32_t tmem_base;
@@ -160,12 +172,15 @@ __device__ __forceinline__ float2 unpack16x2(uint32_t pk) {
   }
 }
 
-template <int D, bool kSplit, bool kF16>
+// kGath: the launch may follow gathered rounds (a second instantiation, so that the code for them
+// costs lists without a gathered schedule nothing).
+template <int D, bool kSplit, bool kF16, bool kGath>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
               const int32_t *__restrict__ round_ptr, const int32_t *__restrict__ round_rows,
-              const uint8_t *__restrict__ round_info, const uint32_t *__restrict__ round_bitmap, int B, int H,
-              int Lq, int n_qt, float scale_log2, unsigned *err, uint32_t max_polls, int dbg_skip) {
+              const uint8_t *__restrict__ round_info, const uint32_t *__restrict__ round_bitmap,
+              const Gathered gth, int B, int H, int Lq, int n_qt, float scale_log2, unsigned *err,
+              uint32_t max_polls, int dbg_skip) {
   using C = Cfg<D, kSplit>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -236,6 +251,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     const int n_half = (n_qt + 1) / 2, n_units = B * H * n_half;
     struct ItemRef {
       int bh, qt, rho0, rho1;  // rounds [rho0, rho1): loaded here, first read when the item begins
+      int gr0, gr1;            // the list row's gathered rounds (equal: none)
       bool in_range, exists;   // !exists: no such item (the unit's halves coincide)
     };
     // (called for t = 0, 1, 2, ... in turn: the unit's (j, bh, h = bh % H) are stepped from one unit
@@ -259,7 +275,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       }
       const int u = cur_u;
       it.in_range = u < n_units;
-      it.bh = 0, it.qt = 0, it.rho0 = 0, it.rho1 = 0, it.exists = false;
+      it.bh = 0, it.qt = 0, it.rho0 = 0, it.rho1 = 0, it.gr0 = 0, it.gr1 = 0, it.exists = false;
       if (it.in_range) {
         const int j = cur_j;
         it.bh = cur_bh;
@@ -268,6 +284,10 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
           const int lr = cur_h * n_qt + it.qt;
           it.rho0 = (int)ldg_now_u32(round_ptr + lr);
           it.rho1 = (int)ldg_now_u32(round_ptr + lr + 1);
+          if constexpr (kGath) {
+            it.gr0 = (int)ldg_now_u32(gth.ptr + lr);
+            it.gr1 = (int)ldg_now_u32(gth.ptr + lr + 1);
+          }
           it.exists = true;
         }
       }
@@ -306,18 +326,91 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         left -= 1 << lg;
       }
     };
+    // Gathered round: lane l holds the keys k4 of the stage's rows 4l .. 4l+3, lanes 4q .. 4q+3 those of
+    // slot q.  A slot whose 16 keys follow one another from a multiple of 8 on is one box (most slots of
+    // a gathered schedule are of that kind); the other slots' rows are fetched one by one.  The copy
+    // engine spends some 60 cycles on every copy whatever its size, so a row-by-row slot would cost it
+    // sixteen times a box with four-row gathers; instead the whole warp copies such a slot in 16-byte
+    // pieces (cp.async) to where the 128-byte swizzle puts them, and ties those copies to the stage's
+    // barrier before that barrier gets the producer's own arrival.
+    auto box_slots = [&](int4 k4, int ng) {  // bit q: slot q is a box
+      const int before = __shfl_up_sync(0xffffffffu, k4.w, 1);
+      const bool chained = k4.y == k4.x + 1 && k4.z == k4.x + 2 && k4.w == k4.x + 3 &&
+                           ((lane & 3) == 0 ? (k4.x & 7) == 0 : k4.x == before + 1);
+      uint32_t chain = __ballot_sync(0xffffffffu, chained);
+      chain &= chain >> 1;
+      chain &= chain >> 2;  // bit 4q: lanes 4q .. 4q+3 all chained
+      uint32_t boxes = 0u;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) boxes |= ((chain >> (4 * q)) & 1u) << q;
+      return boxes & ((1u << ng) - 1u);
+    };
+    // keys of the gathered round being copied and of the one before (whose V copies come a round later)
+    auto load_scattered = [&](unsigned char *stage, const uint16_t *src, uint64_t *bar, const int32_t *keys_s,
+                              uint32_t slots, int bh) {
+      constexpr int kChunks = D / 8;             // 16-byte pieces per key row
+      constexpr int kRowsPerStep = 32 / kChunks; // rows the warp covers per step: lane -> (row, piece)
+      const uint16_t *rows = src + (size_t)bh * gth.Lk * D;
+      const int c = lane % kChunks, r0 = lane / kChunks, half = c >> 3;
+      unsigned char *dst_lane = stage + half * C::kHalfStride;
+      while (slots) {
+        const int q = __ffs((int)slots) - 1;
+        slots &= slots - 1u;
+#pragma unroll
+        for (int i = 0; i < 16 / kRowsPerStep; ++i) {
+          const int R = 16 * q + r0 + kRowsPerStep * i;
+          const int key = keys_s[R];
+          unsigned char *dst = dst_lane + (kSplit ? (R >> 3) * 2048 + (R & 7) * 128 : R * 128) + (((c ^ R) & 7) << 4);
+          cp_async16(dst, rows + (size_t)key * D + 8 * c);
+        }
+      }
+      cp_async_arrive_on(bar);
+    };
+    // The box slots of a gathered round, runs of them that continue one another as one copy.
+    auto load_boxes = [&](unsigned char *stage, const CUtensorMap *m4, uint64_t *bar, int4 k4, uint32_t boxes,
+                          int bh) {
+      const int row_q = __shfl_sync(0xffffffffu, k4.x, (lane & 7) * 4);  // lanes 0..7: first key of slot `lane`
+      const int row_before = __shfl_up_sync(0xffffffffu, row_q, 1);
+      const bool is_box = lane < 8 && ((boxes >> lane) & 1u);
+      const bool after_box = lane > 0 && ((boxes >> (lane - 1)) & 1u);
+      const bool head = is_box && (!after_box || row_q != row_before + 16);
+      const uint32_t heads = __ballot_sync(0xffffffffu, head);
+      const uint32_t stop = ((heads | ~boxes) >> (lane + 1)) & 0x7fu;
+      const int run = head ? (stop ? __ffs((int)stop) : 8 - lane) : 0;
+      load_run(stage, m4, bar, row_q, run, bh);
+    };
+    // which schedule an item follows
+    auto use_gathered = [&](const ItemRef &it) {
+      if constexpr (!kGath) return false;
+      return it.gr1 > it.gr0;  // the list's builder decided where they pay
+    };
     // V of a round is copied one round later than its K: K only needs S = Q K^T of the round that
     // used the stage before to be over, V needs that round's O += P V, which comes much later;
     // issued in round order, the V copy would hold back the next round's K.
-    bool pv_valid = false;
+    bool pv_valid = false, pv_gathered = false;
+    uint32_t pv_boxes = 0u;
+    int pv_kb = 0;
     int pv_st = 0, pv_ng = 0, pv_row = 0, pv_run = 0, pv_bh = 0;
+    int4 pv_keys = make_int4(0, 0, 0, 0);
     uint32_t pv_ph = 0;
     auto issue_v = [&]() {
       if (C::kStages != kMaxStages) wait_free(&sh->v_empty[pv_st], pv_ph);
       if (!ok) return;
-      if (lane == 0) mbar_arrive_expect_tx(&sh->v_full[pv_st], (uint32_t)pv_ng * 16u * D * 2u);
+      if constexpr (kGath) {
+        const uint32_t scattered = pv_gathered ? ((1u << pv_ng) - 1u) & ~pv_boxes : 0u;
+        if (scattered)
+          load_scattered(v_s + pv_st * C::kTileBytes, gth.V, &sh->v_full[pv_st], sh->keys[pv_kb], scattered, pv_bh);
+        __syncwarp();
+      }
+      if (lane == 0)
+        mbar_arrive_expect_tx(&sh->v_full[pv_st],
+                              (uint32_t)(kGath && pv_gathered ? __popc(pv_boxes) : pv_ng) * 16u * D * 2u);
       __syncwarp();
-      load_run(v_s + pv_st * C::kTileBytes, maps.v, &sh->v_full[pv_st], pv_row, pv_run, pv_bh);
+      if (kGath && pv_gathered) {
+        load_boxes(v_s + pv_st * C::kTileBytes, maps.v, &sh->v_full[pv_st], pv_keys, pv_boxes, pv_bh);
+      } else {
+        load_run(v_s + pv_st * C::kTileBytes, maps.v, &sh->v_full[pv_st], pv_row, pv_run, pv_bh);
+      }
       pv_valid = false;
     };
     // the rounds of an item are looked up two items ahead: the loads of item t + 2 are issued when
@@ -326,13 +419,28 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     ItemRef next2 = item_ref(1);
     // ... and the slot rows and info byte of its first round while the current item is under way
     int pf_t = -1, pf_row = -1;
+    int4 pf_keys = make_int4(0, 0, 0, 0);
     uint32_t pf_info = 0u;
+    // slot rows (lanes 0..7) or, for a gathered round, this lane's four keys, and the info byte
+    auto fetch_round = [&](bool gathered, int rho, int &row, int4 &keys, uint32_t &info) {
+      if (kGath && gathered) {
+        const uint4 k = ldg_now_v4(gth.keys + (size_t)rho * kTile + 4 * lane);
+        keys = make_int4((int)k.x, (int)k.y, (int)k.z, (int)k.w);
+        info = ldg_now_u8(gth.info + rho);
+      } else {
+        row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)rho * 8 + lane) : -1;
+        info = ldg_now_u8(round_info + rho);
+      }
+    };
     for (int t = 0; next.in_range && ok; ++t) {
       const ItemRef cur = next;
       next = next2;
       next2 = item_ref(t + 2);
       if (!cur.exists) continue;
-      const int bh = cur.bh, qt = cur.qt, rho0 = cur.rho0, n_rounds = cur.rho1 - cur.rho0;
+      const bool gathered = use_gathered(cur);
+      const int bh = cur.bh, qt = cur.qt, rho0 = gathered ? cur.gr0 : cur.rho0;
+      const int n_rounds = gathered ? cur.gr1 - cur.gr0 : cur.rho1 - cur.rho0;
+      const uint32_t *bitmaps = gathered ? gth.bitmap : round_bitmap;
       if (n_rounds == 0) {
         // nothing kept in this query tile: its output rows are zero (nobody else sees the item)
         const int rows = min(kTile, Lq - qt * kTile);
@@ -354,23 +462,21 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
-      // slot rows (lanes 0..7) and info byte of a round are fetched one round ahead
+      // a round's rows or keys and its info byte are fetched one round ahead
       int next_row = pf_row;
+      int4 next_keys = pf_keys;
       uint32_t next_info = pf_info;
-      if (pf_t != t) {
-        next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)rho0 * 8 + lane) : -1;
-        next_info = ldg_now_u8(round_info + rho0);
-      }
+      if (pf_t != t) fetch_round(gathered, rho0, next_row, next_keys, next_info);
       for (int v = 0; v < n_rounds && ok; ++v, ++g) {
         const int row = next_row;
+        const int4 keys = next_keys;
         const uint32_t rinfo = next_info;
         if (v + 1 < n_rounds) {
-          next_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)(rho0 + v + 1) * 8 + lane) : -1;
-          next_info = ldg_now_u8(round_info + rho0 + v + 1);
+          fetch_round(gathered, rho0 + v + 1, next_row, next_keys, next_info);
         } else if (next.exists && next.rho1 > next.rho0) {
           pf_t = t + 1;
-          pf_row = lane < 8 ? (int)ldg_now_u32(round_rows + (size_t)next.rho0 * 8 + lane) : -1;
-          pf_info = ldg_now_u8(round_info + next.rho0);
+          const bool g_next = use_gathered(next);
+          fetch_round(g_next, g_next ? next.gr0 : next.rho0, pf_row, pf_keys, pf_info);
         }
         const int st = (int)(g % C::kStages);
         const uint32_t ph = (g / C::kStages) & 1u;
@@ -386,8 +492,24 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
         wait_free(&sh->k_empty[st], ph);
         if (ok && C::kStages == kMaxStages) wait_free(&sh->v_empty[st], ph);
         if (!ok) break;
-        const uint32_t bytes = (uint32_t)ng * 16u * D * 2u;
         const bool skip = dbg_skip != 0 && g == 0;   // (test hook: this round's copies and arrivals are left out)
+        uint32_t boxes = 0u;
+        uint32_t bytes = (uint32_t)ng * 16u * D * 2u;
+        const int kb = (int)(g & 1u);
+        if constexpr (kGath) {
+          if (gathered) {
+            boxes = box_slots(keys, ng);
+            bytes = (uint32_t)__popc(boxes) * 16u * D * 2u;
+            const uint32_t scattered = ((1u << ng) - 1u) & ~boxes;
+            if (scattered && !skip) {
+              // (V of the round before last, which used this buffer, was issued a round ago)
+              *reinterpret_cast<int4 *>(&sh->keys[kb][4 * lane]) = keys;
+              __syncwarp();
+              load_scattered(k_s + st * C::kTileBytes, gth.K, &sh->k_full[st], sh->keys[kb], scattered, bh);
+            }
+            __syncwarp();
+          }
+        }
         if (lane == 0 && !skip) {
           sh->info[si] = (uint32_t)ng | (v == 0 ? kInfoFirst : 0u) | (v + 1 == n_rounds ? kInfoLast : 0u) |
                          (full ? kInfoFull : 0u);
@@ -398,16 +520,24 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
             mbar_arrive(&sh->b_full[si]);
           } else {
             mbar_arrive_expect_tx(&sh->b_full[si], kBitmapWords * 4);
-            bulk_load(&sh->bitmap[si][0][0], round_bitmap + (size_t)(rho0 + v) * kBitmapWords, kBitmapWords * 4,
+            bulk_load(&sh->bitmap[si][0][0], bitmaps + (size_t)(rho0 + v) * kBitmapWords, kBitmapWords * 4,
                       &sh->b_full[si]);
           }
         }
         __syncwarp();
-        if (!skip) load_run(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st], row, run, bh);
+        if (!skip) {
+          if (kGath && gathered) {
+            load_boxes(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st], keys, boxes, bh);
+          } else {
+            load_run(k_s + st * C::kTileBytes, maps.k, &sh->k_full[st], row, run, bh);
+          }
+        }
         if (pv_valid) issue_v();
         if (!ok) break;
         pv_valid = !skip;
-        pv_st = st, pv_ph = ph, pv_ng = ng, pv_row = row, pv_run = run, pv_bh = bh;
+        pv_gathered = gathered;
+        pv_st = st, pv_ph = ph, pv_ng = ng, pv_row = row, pv_run = run, pv_bh = bh, pv_keys = keys, pv_boxes = boxes;
+        pv_kb = kb;
       }
       ++n;
     }
@@ -457,6 +587,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       if (ok && g >= 2) ok = warp_wait<31>(&sh->pv_done[sb], ((g >> 1) - 1u) & 1u, lane, abort_flag, err, max_polls);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (kGath) fence_proxy_async_smem();  // rows of a gathered round may come from plain asynchronous copies
       // N = 16 ng, D/16 steps of K = 16 (32 bytes inside the swizzled rows)
       if (elect_one()) {
         const uint32_t idesc_qk = idesc_bf16_f32(128, 16 * ng, false, false, kF16);
@@ -498,6 +629,7 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       if (ok) ok = warp_wait<31>(&sh->p_full[sb], (g >> 1) & 1u, lane, abort_flag, err, max_polls);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (kGath) fence_proxy_async_smem();  // rows of a gathered round may come from plain asynchronous copies
       // One K step of 16 keys per slot.  P (bf16) of a 32-column chunk is written over the first
       // 16 columns of that chunk of S (each group stays inside its own chunks), so slot q's
       // eight columns of P start at column 32 (q / 2) + 8 (q % 2).
@@ -736,27 +868,39 @@ int sm_count() {
   return cached[dev];
 }
 
-template <int D, bool kSplit, bool kF16>
-cudaError_t launch(const FwdMaps &maps, void *O, const ap_tiles &t, int B, int H, int Lq, float scale,
-                   unsigned *err, cudaStream_t s) {
+template <int D, bool kSplit, bool kF16, bool kGath>
+cudaError_t launch_kernel(const FwdMaps &maps, const void *K, const void *V, void *O, const ap_tiles &t, int B, int H,
+                          int Lq, int Lk, const DebugKnobs &dbg, float scale, unsigned *err, cudaStream_t s) {
   using C = Cfg<D, kSplit>;
-  static_assert(sizeof(Shared) <= 17 * 1024, "shared bookkeeping outgrew its reservation");
+  static_assert(sizeof(Shared) <= 18 * 1024, "shared bookkeeping outgrew its reservation");
   static_assert(C::kStages <= kMaxStages, "ring deeper than its barriers");
   static_assert(C::kSmemBytes > 114 * 1024 && C::kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
-  auto kern = fwd_tc_kernel<D, kSplit, kF16>;
+  auto kern = fwd_tc_kernel<D, kSplit, kF16, kGath>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   const int n_units = B * H * ((t.n_qt + 1) / 2);  // pairs of query tiles, see the producer
   const float scale_log2 = scale * 1.4426950408889634f;
-  const DebugKnobs dbg = debug_knobs();
+  Gathered gth = {nullptr, nullptr, nullptr, nullptr, static_cast<const uint16_t *>(K), static_cast<const uint16_t *>(V),
+                  Lk, dbg.schedule};
+  if (kGath) gth.ptr = t.ground_ptr, gth.keys = t.ground_keys, gth.info = t.ground_info, gth.bitmap = t.ground_bitmap;
   // the test hook runs on one CTA only (a tiny grid is all it is meant for)
   kern<<<dbg.skip_arrive ? 1 : (n_units < sms ? n_units : sms), kThreads, C::kSmemBytes, s>>>(
-      maps, static_cast<uint16_t *>(O), t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, B, H, Lq,
+      maps, static_cast<uint16_t *>(O), t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, gth, B, H, Lq,
       t.n_qt, scale_log2, err, dbg.max_polls, dbg.skip_arrive);
   count_launches(1);
   return cudaGetLastError();
+}
+
+// Lists that carry a gathered schedule get the instantiation that can follow it.
+template <int D, bool kSplit, bool kF16>
+cudaError_t launch(const FwdMaps &maps, const void *K, const void *V, void *O, const ap_tiles &t, int B, int H, int Lq,
+                   int Lk, bool, float scale, unsigned *err, cudaStream_t s) {
+  const DebugKnobs dbg = debug_knobs();
+  if (t.ground_ptr != nullptr && dbg.schedule != 1)
+    return launch_kernel<D, kSplit, kF16, true>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
+  return launch_kernel<D, kSplit, kF16, false>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
 }
 
 }  // namespace
@@ -777,14 +921,15 @@ cudaError_t launch_fwd_tc(const void *Q, const void *K, const void *V, const ap_
                      make_tile_map_bf16(&maps.v[i], V, B * H, Lk, d, rows);
   }
   if (!ok) return cudaErrorUnknown;
+  const bool gm = t.ground_ptr != nullptr;
   if (f16) {
-    if (d == 64) return launch<64, false, true>(maps, O, t, B, H, Lq, scale, err, s);
-    return split ? launch<128, true, true>(maps, O, t, B, H, Lq, scale, err, s)
-                 : launch<128, false, true>(maps, O, t, B, H, Lq, scale, err, s);
+    if (d == 64) return launch<64, false, true>(maps, K, V, O, t, B, H, Lq, Lk, gm, scale, err, s);
+    return split ? launch<128, true, true>(maps, K, V, O, t, B, H, Lq, Lk, gm, scale, err, s)
+                 : launch<128, false, true>(maps, K, V, O, t, B, H, Lq, Lk, gm, scale, err, s);
   }
-  if (d == 64) return launch<64, false, false>(maps, O, t, B, H, Lq, scale, err, s);
-  return split ? launch<128, true, false>(maps, O, t, B, H, Lq, scale, err, s)
-               : launch<128, false, false>(maps, O, t, B, H, Lq, scale, err, s);
+  if (d == 64) return launch<64, false, false>(maps, K, V, O, t, B, H, Lq, Lk, gm, scale, err, s);
+  return split ? launch<128, true, false>(maps, K, V, O, t, B, H, Lq, Lk, gm, scale, err, s)
+               : launch<128, false, false>(maps, K, V, O, t, B, H, Lq, Lk, gm, scale, err, s);
 }
 
 }  // namespace ap

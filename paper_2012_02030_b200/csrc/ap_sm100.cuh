@@ -129,6 +129,18 @@ __device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *m
       : "memory");
 }
 
+// 16 bytes global -> shared memory by the calling thread, asynchronously (cached in L2 only).  Both
+// addresses 16-byte aligned.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+// Ties the calling thread's cp.async copies issued so far to `bar`: the barrier's pending count goes
+// up by one now and comes down again when those copies have landed, so a phase that is still open
+// when this executes cannot complete before they have.
+__device__ __forceinline__ void cp_async_arrive_on(uint64_t *bar) {
+  asm volatile("cp.async.mbarrier.arrive.shared.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
 // 5-D tiled load: box at coordinates (c0..c4) -> shared memory, completion on `bar`.
 __device__ __forceinline__ void tma_load_5d(void *smem_dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1,
                                             int c2, int c3, int c4) {

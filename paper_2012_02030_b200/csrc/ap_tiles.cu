@@ -365,15 +365,195 @@ __global__ void __launch_bounds__(128) fill_rounds_kernel(const int32_t *__restr
   }
 }
 
+// ---- gathered rounds: a list row's active key columns, 128 per round ----------------------------
+
+// The 128-bit column summary of one stored tile (bit c: some row keeps column c), by one warp:
+// lane l ORs rows l, l + 32, l + 64, l + 96.  Every lane returns the four words.
+__device__ __forceinline__ uint4 column_summary(const uint32_t *__restrict__ bitmap, int t, int lane) {
+  uint4 m = make_uint4(0u, 0u, 0u, 0u);
+  const uint4 *rows = reinterpret_cast<const uint4 *>(bitmap + (size_t)t * kBitmapWords);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint4 w = rows[lane + 32 * k];
+    m.x |= w.x, m.y |= w.y, m.z |= w.z, m.w |= w.w;
+  }
+  m.x = __reduce_or_sync(0xffffffffu, m.x);
+  m.y = __reduce_or_sync(0xffffffffu, m.y);
+  m.z = __reduce_or_sync(0xffffffffu, m.z);
+  m.w = __reduce_or_sync(0xffffffffu, m.w);
+  return m;
+}
+
+// How many of a summary word's two 16-column groups have every column active.
+__device__ __forceinline__ int whole_groups(uint32_t m) {
+  return ((m & 0xffffu) == 0xffffu ? 1 : 0) + ((m >> 16) == 0xffffu ? 1 : 0);
+}
+
+// One warp per list row: ground_ptr[row + 1] = ceil(active columns / 128) (scanned afterwards), or 0
+// where gathered rounds would not pay.  Measured on the forward: a gathered round takes 1.1 to 1.3
+// times a round of the same width (the copy warp has more to do), a slot whose 16 key rows are
+// fetched one by one costs a quarter of a round and more on top, and the kernel that can follow
+// gathered rounds is some 10 % slower on every round; so a list row of r rounds gets its g gathered
+// rounds, s of whose slots are of that kind, only where they halve the work: r > 2 g + s / 2.
+__global__ void __launch_bounds__(128) count_grounds_kernel(const int32_t *__restrict__ row_ptr,
+                                                            const uint32_t *__restrict__ bitmap,
+                                                            const int32_t *__restrict__ round_ptr, int n_rows,
+                                                            int always, int32_t *__restrict__ ground_ptr) {
+  const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= n_rows) return;
+  int cols = 0, whole = 0;
+  for (int t = row_ptr[row]; t < row_ptr[row + 1]; ++t) {
+    const uint4 m = column_summary(bitmap, t, lane);
+    cols += __popc(m.x) + __popc(m.y) + __popc(m.z) + __popc(m.w);
+    whole += whole_groups(m.x) + whole_groups(m.y) + whole_groups(m.z) + whole_groups(m.w);
+  }
+  if (lane == 0) {
+    const int r = round_ptr[row + 1] - round_ptr[row];
+    const int g = (cols + kTile - 1) / kTile;
+    const int s = (cols - 16 * whole + 15) / 16;
+    ground_ptr[row + 1] = (always || 2 * r > 4 * g + s) ? g : 0;
+    if (row == 0) ground_ptr[0] = 0;
+  }
+}
+
+// One CTA per list row, thread r = bitmap row r (and column p of the round being written).  The
+// row's tiles are taken 32 at a time, twice: first the 16-column groups in which every column is
+// active are listed in shared memory (a slot of such a group is 16 key rows that follow one another
+// from a multiple of 16 on, which the forward fetches as one box), then the active columns of the
+// other groups, each time in ascending key order; every complete set of 128 listed columns (plus
+// the remainder at the end) is written out as a gathered round.
+__global__ void __launch_bounds__(128) fill_grounds_kernel(const int32_t *__restrict__ row_ptr,
+                                                           const int32_t *__restrict__ col_idx,
+                                                           const uint32_t *__restrict__ bitmap,
+                                                           const int32_t *__restrict__ ground_ptr, int cap,
+                                                           int32_t *__restrict__ ground_keys,
+                                                           uint8_t *__restrict__ ground_info,
+                                                           uint32_t *__restrict__ ground_bitmap) {
+  constexpr int kSeg = 32;                         // tiles per pass
+  __shared__ uint32_t summary[kSeg * 4];           // column summaries of the pass's tiles
+  __shared__ int32_t tile_kt[kSeg];
+  __shared__ int32_t col_key[kSeg * kTile + kTile];  // key index of each listed column
+  __shared__ uint32_t col_src[kSeg * kTile + kTile]; // tile index << 7 | column inside the tile
+  __shared__ int warp_sums[4];
+  const int row = blockIdx.x, r = threadIdx.x, lane = r & 31, warp = r >> 5;
+  const int t_begin = row_ptr[row], t_end = row_ptr[row + 1];
+  int rho = ground_ptr[row];
+  if (ground_ptr[row + 1] == rho) return;  // no gathered rounds for this list row
+  int pending = 0;  // columns carried over from the previous pass (fewer than 128)
+  for (int phase = 0; phase < 2; ++phase)
+  for (int base = t_begin; base < t_end; base += kSeg) {
+    const int n_here = min(kSeg, t_end - base);
+    for (int k = warp; k < kSeg; k += 4) {  // warp w summarises tiles w, w + 4, ...
+      uint4 m = make_uint4(0u, 0u, 0u, 0u);
+      if (k < n_here) m = column_summary(bitmap, base + k, lane);
+      if (lane == 0) {
+        summary[4 * k] = m.x, summary[4 * k + 1] = m.y, summary[4 * k + 2] = m.z, summary[4 * k + 3] = m.w;
+        tile_kt[k] = k < n_here ? col_idx[base + k] : 0;
+      }
+    }
+    __syncthreads();
+    // thread r owns summary word r (tile r / 4, columns 32 (r % 4) ...), of which this phase takes the
+    // halves that are all ones, or the others: exclusive prefix of the popcounts
+    uint32_t m = summary[r];
+    const uint32_t whole = ((m & 0xffffu) == 0xffffu ? 0xffffu : 0u) | ((m >> 16) == 0xffffu ? 0xffff0000u : 0u);
+    m = phase == 0 ? whole : m & ~whole;
+    const int cnt = __popc(m);
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      if (w < warp) before += warp_sums[w];
+      total += warp_sums[w];
+    }
+    int s = pending + before + incl - cnt;
+    const int tile = base + (r >> 2), kt = tile_kt[r >> 2];
+    while (m) {
+      const int c = 32 * (r & 3) + __ffs((int)m) - 1;
+      m &= m - 1u;
+      col_key[s] = kt * kTile + c;
+      col_src[s] = ((uint32_t)tile << 7) | (uint32_t)c;
+      ++s;
+    }
+    __syncthreads();
+    const int avail = pending + total;
+    const bool last_pass = phase == 1 && base + kSeg >= t_end;
+    const int n_emit = last_pass ? (avail + kTile - 1) / kTile : avail / kTile;
+    for (int k = 0; k < n_emit; ++k) {
+      const int nc = min(kTile, avail - kTile * k);  // columns of this round
+      // row r of the round's bitmap: bit p = bit (column of p) of row r of (tile of p)
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      uint32_t cur_word_id = 0xffffffffu, cur_word = 0u;
+      for (int p = 0; p < nc; ++p) {
+        const uint32_t src = col_src[kTile * k + p];
+        const uint32_t word_id = ((src >> 7) << 2) | ((src & 127u) >> 5);  // (tile, word of the row)
+        if (word_id != cur_word_id) {
+          cur_word_id = word_id;
+          cur_word = bitmap[(size_t)(src >> 7) * kBitmapWords + r * 4 + ((src & 127u) >> 5)];
+        }
+        w[p >> 5] |= ((cur_word >> (src & 31u)) & 1u) << (p & 31);
+      }
+      const bool mine_full = (w[0] & w[1] & w[2] & w[3]) == 0xffffffffu;
+      const int all_full = __syncthreads_and(mine_full ? 1 : 0);
+      const int out = rho + k;
+      if (out < cap) {
+        reinterpret_cast<uint4 *>(ground_bitmap + (size_t)out * kBitmapWords)[r] = make_uint4(w[0], w[1], w[2], w[3]);
+        ground_keys[(size_t)out * kTile + r] = col_key[kTile * k + min(r, nc - 1)];
+        if (r == 0) ground_info[out] = (uint8_t)(((nc + 15) / 16) | ((all_full && nc == kTile) ? 0x80 : 0));
+      }
+    }
+    rho += n_emit;
+    __syncthreads();
+    // fewer than 128 columns are left over; they move to the front (no overlap: they start at or
+    // beyond index 128 unless nothing was written out, in which case they are in place already)
+    const int left = avail - kTile * n_emit;
+    int32_t a = 0;
+    uint32_t b = 0u;
+    const bool move = !last_pass && n_emit > 0 && r < left;
+    if (move) a = col_key[kTile * n_emit + r], b = col_src[kTile * n_emit + r];
+    __syncthreads();
+    if (move) col_key[r] = a, col_src[r] = b;
+    pending = last_pass ? 0 : left;
+    __syncthreads();
+  }
+}
+
+// No gathered schedule (dense lists): every list row has zero gathered rounds.
+__global__ void clear_grounds_kernel(int32_t *__restrict__ ground_ptr, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) ground_ptr[i] = 0;
+}
+
 }  // namespace
 
-// Writes the round arrays of a finished tile list (row_ptr, col_idx, flags, groups, bitmap).
-cudaError_t launch_build_rounds(const ap_tiles &t, cudaStream_t s) {
+// Writes the round arrays of a finished tile list (row_ptr, col_idx, flags, groups, bitmap), and the
+// gathered rounds where the list has room for them (gathered == false: an empty gathered schedule).
+cudaError_t launch_build_rounds(const ap_tiles &t, cudaStream_t s, bool gathered) {
   const int n_rows = t.H * t.n_qt;
   count_rounds_kernel<<<ceil_div(n_rows, 4), 128, 0, s>>>(t.row_ptr, t.flags, t.groups, n_rows, t.round_ptr);
   scan_rounds_kernel<<<1, 1024, 0, s>>>(t.round_ptr, n_rows);
   fill_rounds_kernel<<<n_rows, 128, 0, s>>>(t.row_ptr, t.col_idx, t.flags, t.groups, t.bitmap, t.round_ptr, t.cap,
                                             t.round_rows, t.round_info, t.round_bitmap);
+  count_launches(3);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || !t.ground_ptr) return e;
+  if (!gathered) {
+    clear_grounds_kernel<<<ceil_div(n_rows + 1, 256), 256, 0, s>>>(t.ground_ptr, n_rows + 1);
+    count_launches(1);
+    return cudaGetLastError();
+  }
+  // (test hook: every list row gets its gathered rounds, see ap_debug_schedule)
+  count_grounds_kernel<<<ceil_div(n_rows, 4), 128, 0, s>>>(t.row_ptr, t.bitmap, t.round_ptr, n_rows,
+                                                           debug_knobs().schedule == 2 ? 1 : 0, t.ground_ptr);
+  scan_rounds_kernel<<<1, 1024, 0, s>>>(t.ground_ptr, n_rows);
+  fill_grounds_kernel<<<n_rows, 128, 0, s>>>(t.row_ptr, t.col_idx, t.bitmap, t.ground_ptr, t.cap, t.ground_keys,
+                                             t.ground_info, t.ground_bitmap);
   count_launches(3);
   return cudaGetLastError();
 }
@@ -403,7 +583,7 @@ cudaError_t launch_compact_tiles(const uint32_t *stage_bitmap, const int32_t *st
   count_launches(1);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  return launch_build_rounds(t, s);
+  return launch_build_rounds(t, s, true);
 }
 
 cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
@@ -414,7 +594,7 @@ cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
   count_launches(1);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  return launch_build_rounds(t, s);
+  return launch_build_rounds(t, s, false);
 }
 
 }  // namespace ap
