@@ -51,7 +51,9 @@ NCU_TRAFFIC = {
         "sparse_fwd": {"bytes": 4 * 70.5e6,
                        "source": "ncu on the B=1 case (68.0 MB read + 2.5 MB written per launch), times 4 batch elements; "
                                  "O is still in L2 when the kernel ends"},
-        "accumulate": {"bytes": 2.69e9, "source": "ncu on the full workload, one launch (2.18 GB read + 0.51 GB written)"},
+        "accumulate": {"bytes": 2.27e9,
+                       "source": "ncu on the B=1 case (1.72 GB read + 0.50 GB written per launch: the accumulator, the bias "
+                                 "and their traffic have no batch dimension) plus Q and K of three more samples"},
         "build_mask": {"bytes": 1.39e9,
                        "source": "ncu on the full workload: collecting pass 542 MB read + 31 MB written, emit pass "
                                  "541 MB read + 278 MB written; the call's other kernels move a few MB"},
