@@ -26,6 +26,12 @@
 // O += P V of round g - 2 (the previous user of that S buffer), O += P(g) V for P(g) and V(g).
 // So the softmax threads find the next S ready when they finish a round.
 //
+// A list row that carries GATHERED ROUNDS (the tile list's second schedule: the row's active key
+// columns, those of whole 16-column groups first, 128 per round, with the bitmap re-packed per
+// column) is followed through those instead, by the kernel's second instantiation: a slot of 16
+// keys that follow one another is still one box; the rows of any other slot are copied one by one
+// (see the producer).  Everything after the copies is the same: N = 16 * slots, the round's
+// bitmap, the same softmax.
 //
 // The softmax is shared by two groups of four warps.  The 32-column chunks of a round alternate
 // between them (chunk c belongs to group c & 1), and each group is an online softmax of its own:
@@ -37,8 +43,14 @@
 // Warp roles (480 threads): warps 0-3 softmax group 0, warps 4-7 group 1 (thread = query row =
 // TMEM lane), warp 8 producer, warp 9 issuer of S = Q K^T and TMEM owner, warp 10 issuer of
 // O += P V, warps 11-14 epilogue (the softmax groups hand (m, l) over and go on with the next
-// item while the epilogue warps wait for the item's last O += P V, merge and write).  TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384 (d = 128); at d = 64 the pair (O_0, O_1) takes 128 columns and two items' pairs alternate at 256 and 384.  Every wait is bounded; a wait that expires
-// raises the device status word and the CTA winds down.
+// item while the epilogue warps wait for the item's last O += P V, merge and write).  The softmax
+// body of a round is straight-line code: both 32-column chunks of the group are always loaded, and
+// the mask is applied by select (branches around the tensor-memory loads cost more than the loads).
+// TMEM (512 columns): S[0] at column 0, S[1] at 128, O_0 at 256, O_1 at 384 (d = 128); at d = 64
+// the pair (O_0, O_1) takes 128 columns and two items' pairs alternate at 256 and 384.  Every wait
+// is bounded, with the poll limit a kernel argument; a wait that expires raises the device status
+// word and the CTA winds down (the end of a CTA's work reaches the epilogue warps through a word of
+// its own, not through the ring that hands (m, l) over).
 #include <math_constants.h>
 
 #include "ap_common.cuh"
