@@ -154,10 +154,11 @@ uint64_t ap_launch_count(void);
  * kernels polls a bounded number of times; when a wait runs out the kernel raises the device status
  * word, every role leaves its loop, copies in flight are waited for (bounded), tensor memory is
  * freed and the kernel returns, after which ap_device_status() reports AP_ERR_TIMEOUT once.
- * With on != 0, the following launches of ap_sparse_attention_fwd (16-bit types) run on ONE
- * thread block with a poll limit of a few thousand and leave out one producer arrival, so that
- * this path runs within a millisecond without faulting or hanging anything; their output is
- * undefined.  on == 0 restores normal operation.  Process-wide; not for production use.
+ * With on != 0, the following launches of ap_sparse_attention_fwd, ap_accumulate_attention and
+ * ap_sparse_attention_bwd (16-bit types) poll a few thousand times only and leave out the first
+ * copies of a thread block (forward and accumulate: on a grid of ONE thread block), so that this path
+ * runs within milliseconds without faulting or hanging anything; their output is undefined.
+ * on == 0 restores normal operation.  Process-wide; not for production use.
  */
 void ap_debug_expire_waits(int on);
 

@@ -38,7 +38,6 @@ using namespace sm100;
 constexpr int kThreads = 256;  // thread (half, r): row r of the tile, chunks 2 half and 2 half + 1
 constexpr int kSubBytes = 128 * 128;  // one slab: 128 rows x 64 elements of 2 bytes
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct Bars {
@@ -79,10 +78,11 @@ __device__ __forceinline__ float2 unpack2(uint32_t pk) {
 
 // Bounded wait of the whole CTA on one barrier phase; the outcome is the same for every thread.  (Every
 // thread polls: with one polling thread and the others parked at the CTA barrier the kernels were 4 % slower.)
-__device__ __forceinline__ bool cta_wait(uint64_t *bar, uint32_t parity, Bars *bars, unsigned *err) {
+__device__ __forceinline__ bool cta_wait(uint64_t *bar, uint32_t parity, Bars *bars, unsigned *err,
+                                         uint32_t max_polls) {
   bool ok = false;
   volatile int *abort_flag = &bars->abort_flag;
-  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+  for (uint32_t i = 0; i < max_polls; ++i) {
     if (mbar_try_wait(bar, parity)) {
       ok = true;
       break;
@@ -200,7 +200,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ, float *__restrict__ stat_l,
                 float *__restrict__ stat_d, const int32_t *__restrict__ round_ptr,
                 const int32_t *__restrict__ round_rows, const uint8_t *__restrict__ round_info,
-                const uint32_t *__restrict__ round_bitmap, int H, int Lq, int n_qt, float scale, unsigned *err) {
+                const uint32_t *__restrict__ round_bitmap, int H, int Lq, int n_qt, float scale, unsigned *err,
+                uint32_t max_polls, int dbg_skip) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -274,14 +275,14 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
   uint32_t tma_n = 0, mma_n = 0;  // phases used so far
   bool ok = true;
 
-  // Q, dO and O of the query tile; D_i = dO_i . O_i
-  if (leader) {
+  // Q, dO and O of the query tile; D_i = dO_i . O_i  (test hook: the copies are left out, the wait below runs out)
+  if (leader && dbg_skip == 0) {
     mbar_arrive_expect_tx(&bars->tma, 3 * C::kTileBytes);
     load_tile<D>(q_s, &maps.q, &bars->tma, qt * kTile, bh);
     load_tile<D>(do_s, &maps.d_o, &bars->tma, qt * kTile, bh);
     load_tile<D>(ds_s, &maps.o, &bars->tma, qt * kTile, bh);
   }
-  ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+  ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err, max_polls);
   // each of the row's two threads takes half of every 128-byte line; the halves are added in a fixed order
   float dsum = 0.f;
   float *xch = reinterpret_cast<float *>(kv_s);  // [half][row]; the K / V area is not in use yet
@@ -319,7 +320,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     cur = nxt;
     if (t + 2 < t1) nxt = meta_of(t + 2);
     const uint32_t gm = (1u << (me.info & 15u)) - 1u;  // the round's slots, packed from slot 0
-    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err, max_polls);
     if (!ok) break;
     if (leader) {
       // the other pair was last read by the MMA of round t - 1, which has completed
@@ -331,7 +332,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     uint4 bw = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
     if (!(me.info & 0x80u)) bw = *reinterpret_cast<const uint4 *>(round_bitmap + ((size_t)t * kTile + r) * 4);
     const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
-    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err, max_polls);
     if (!ok) break;
     tc_fence_after_sync();
 #pragma unroll 1
@@ -386,7 +387,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     cur = nxt;
     if (t + 2 < t1) nxt = meta_of(t + 2);
     const uint32_t gm = (1u << (me.info & 15u)) - 1u;
-    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err, max_polls);
     if (!ok) break;
     if (leader) {
       // the other pair was last read by dQ += dS K of round t - 1, which has completed
@@ -399,7 +400,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
     uint4 bw = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
     if (!(me.info & 0x80u)) bw = *reinterpret_cast<const uint4 *>(round_bitmap + ((size_t)t * kTile + r) * 4);
     const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
-    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err, max_polls);
     if (!ok) break;
     tc_fence_after_sync();
 #pragma unroll 1
@@ -432,7 +433,7 @@ bwd_rows_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dQ,
       mma_commit(&bars->mma);
     }
     started = true;
-    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);  // K, V, dS may be overwritten
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err, max_polls);  // K, V, dS may be overwritten
   }
 
   // ---- dQ rows, scaled and rounded once (the loads are warp-wide: rows beyond Lq take part and store nothing)
@@ -488,7 +489,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
                 const float *__restrict__ stat_l, const float *__restrict__ stat_d,
                 const int32_t *__restrict__ tile_id, const uint8_t *__restrict__ flags,
                 const uint8_t *__restrict__ groups, const uint32_t *__restrict__ bitmap, int H, int Lq, int Lk,
-                int n_qt, int n_kt, float scale, unsigned *err) {
+                int n_qt, int n_kt, float scale, unsigned *err, uint32_t max_polls, int dbg_skip) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -545,7 +546,8 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
 
   int t_cur = -1;
   int qt_cur = find_from(0, t_cur);
-  if (leader && qt_cur < n_qt) {  // K, V and the first query tile's Q, dO in one go
+  // (test hook: these copies are left out, so the first wait runs out)
+  if (leader && qt_cur < n_qt && dbg_skip == 0) {  // K, V and the first query tile's Q, dO in one go
     mbar_arrive_expect_tx(&bars->tma, 4 * C::kTileBytes);
     load_tile<D>(k_s, &maps.k, &bars->tma, kt * kTile, bh);
     load_tile<D>(v_s, &maps.v, &bars->tma, kt * kTile, bh);
@@ -569,7 +571,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     const float dsum = i < Lq ? stat_d[(size_t)bh * Lq + i] : 0.f;
     const uint4 bw = *reinterpret_cast<const uint4 *>(bitmap + ((size_t)t * kTile + r) * 4);
     const uint32_t w[4] = {bw.x, bw.y, bw.z, bw.w};
-    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err);
+    ok = cta_wait(&bars->tma, tma_n++ & 1u, bars, err, max_polls);
     if (!ok) break;
     if (leader) {
       tc_fence_after_sync();
@@ -579,7 +581,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     }
     // products complete in order: with S and dP, dK += dS^T Q of the previous query tile is over too,
     // so its (Q, dO) pair and the P / dS area are free
-    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err, max_polls);
     if (!ok) break;
     if (leader && qt_nxt < n_qt) {
       unsigned char *nq = qd_s + ((n + 1u) & 1u) * 2 * C::kTileBytes;
@@ -628,7 +630,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
       mma_atb<D>(tmem_dv, x_s, do_s, idesc_t, started);
       mma_commit(&bars->mma);
     }
-    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err);  // P is read: the area takes dS
+    ok = cta_wait(&bars->mma, mma_n++ & 1u, bars, err, max_polls);  // P is read: the area takes dS
     if (!ok) break;
     store_chunk(x_s, r, 2 * half, pd[0]);
     store_chunk(x_s, r, 2 * half + 1, pd[1]);
@@ -644,7 +646,7 @@ bwd_cols_kernel(const __grid_constant__ BwdMaps maps, uint16_t *__restrict__ dK,
     qt_cur = qt_nxt;
     t_cur = t_nxt;
   }
-  if (ok && started) ok = cta_wait(&bars->mma2, (dk_n - 1u) & 1u, bars, err);
+  if (ok && started) ok = cta_wait(&bars->mma2, (dk_n - 1u) & 1u, bars, err, max_polls);
 
   // ---- dV and dK rows of this key tile (thread r = key row), rounded once
   const int j = kt * kTile + r;
@@ -686,6 +688,7 @@ template <int D, bool kF16>
 cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *stat_l, float *stat_d, int32_t *tile_id,
                    const ap_tiles &t, int B, int H, int Lq, int Lk, float scale, unsigned *err, cudaStream_t s) {
   using C = Cfg<D>;
+  const DebugKnobs knobs = debug_knobs();  // poll limit; test hook of the failure path
   auto rows = bwd_rows_kernel<D, kF16>;
   auto cols = bwd_cols_kernel<D, kF16>;
   cudaError_t e = cudaFuncSetAttribute(rows, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kRowsSmem);
@@ -694,13 +697,13 @@ cudaError_t launch(const BwdMaps &maps, void *dQ, void *dK, void *dV, float *sta
   if (e != cudaSuccess) return e;
   rows<<<B * H * t.n_qt, kThreads, C::kRowsSmem, s>>>(maps, static_cast<uint16_t *>(dQ), stat_l, stat_d, t.round_ptr,
                                                       t.round_rows, t.round_info, t.round_bitmap, H, Lq, t.n_qt,
-                                                      scale, err);
+                                                      scale, err, knobs.max_polls, knobs.skip_arrive);
   tile_lookup_kernel<<<H * t.n_qt, 128, 0, s>>>(t.row_ptr, t.col_idx, H * t.n_qt, t.n_kt, tile_id);
   count_launches(2);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cols<<<B * H * t.n_kt, kThreads, C::kColsSmem, s>>>(maps, static_cast<uint16_t *>(dK), static_cast<uint16_t *>(dV),
                                                       stat_l, stat_d, tile_id, t.flags, t.groups, t.bitmap, H, Lq, Lk,
-                                                      t.n_qt, t.n_kt, scale, err);
+                                                      t.n_qt, t.n_kt, scale, err, knobs.max_polls, knobs.skip_arrive);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -64,3 +64,33 @@ def test_accumulate_expired_wait_returns_timeout_once_and_the_next_call_is_corre
     want = np.zeros((H, L, L))
     orc.accumulate(want, inputs.widen(q), inputs.widen(k), bias.numpy(), causal=True)
     np.testing.assert_allclose(acc.cpu().numpy(), want, rtol=2e-5, atol=1e-7 * B)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d", [64, 128])
+def test_backward_expired_wait_returns_timeout_once_and_the_next_call_is_correct(d):
+    from paper_2012_02030_b200 import binding as ap
+    from tests import parity_util as pu
+
+    B, H, L = 1, 2, 256
+    gen = torch.Generator().manual_seed(4300 + d)
+    q, k, v, d_o = (torch.randn((B, H, L, d), generator=gen).to(torch.bfloat16) for _ in range(4))
+    mask = inputs.random_mask(H, L, L, 0.3, seed=78, causal=True)
+    tiles = ap.Tiles(H, L, L)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    qd, kd, vd, dod = q.cuda(), k.cuda(), v.cuda(), d_o.cuda()
+    out = ap.ap_sparse_attention_fwd(qd, kd, vd, tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    ap.ap_debug_expire_waits(True)
+    try:
+        ap.ap_sparse_attention_bwd(qd, kd, vd, out, dod, tiles)    # both kernels' first waits run out
+        assert ap.ap_device_status() == ap.AP_ERR_TIMEOUT
+    finally:
+        ap.ap_debug_expire_waits(False)
+    assert ap.ap_device_status() == ap.AP_OK
+    dq, dk, dv = ap.ap_sparse_attention_bwd(qd, kd, vd, out, dod, tiles)
+    assert ap.ap_device_status() == ap.AP_OK
+    ref = orc.attention_bwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), inputs.widen(d_o), mask.numpy())
+    for got, want, name in zip((dq, dk, dv), ref, ("dQ", "dK", "dV")):
+        err = np.linalg.norm(got.float().cpu().numpy() - want) / np.linalg.norm(want)
+        assert err < 1e-2, (name, err)
