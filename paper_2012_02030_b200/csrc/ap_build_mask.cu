@@ -462,7 +462,9 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
       for (int u = 0; u < 4; ++u) {
         const int j0 = base + 128 * u + 4 * lane;
         if (j0 + 4 <= jend && !(diag && own >= j0 && own < j0 + 4)) {
-          // four entries of the domain: nothing to check per entry
+          // four entries of the domain: nothing to check per entry, and nothing to do at all where all
+          // four lie below the bracket (most pieces of a row: the bracket sits near the top of the values)
+          if (v[u][0] < lo_f && v[u][1] < lo_f && v[u][2] < lo_f && v[u][3] < lo_f) continue;
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const float f = v[u][c];
@@ -715,10 +717,13 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
       if (kInterior || i < Lq) {  // warp-uniform
         uint32_t tie_bits = 0u, gt_bits = 0u;
         if (kInterior) {
+          // (most pieces of a row lie wholly below the threshold: one test instead of eight)
+          if (!(v[u][0] < thr_f && v[u][1] < thr_f && v[u][2] < thr_f && v[u][3] < thr_f)) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
-            tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
+            for (int c = 0; c < 4; ++c) {
+              gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
+              tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
+            }
           }
         } else {
           const int jend = causal ? min(Lk, i + 1 + off) : Lk;
