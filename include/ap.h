@@ -189,9 +189,11 @@ size_t ap_mask_to_tiles_workspace_bytes(int H, int Lq, int Lk);
  * over the row's domain (all j, or the causal domain above); entries outside the
  * domain are not touched.  The 1/n of Eq. 1 is left to the caller, who counts
  * the samples: the selection of Eq. 2 does not depend on it.
- *   acc    [H,Lq,Lk] fp32, in/out.  The sum over b is taken in ascending b inside the
- *          kernel and added to acc with one reduction per entry and launch, ordered by
- *          the stream, so results are reproducible bit for bit.
+ *   acc    [H,Lq,Lk] fp32, in/out.  The samples are summed in ascending b inside the kernel,
+ *          in chunks whose size depends only on the shape and the device's SM count (all B
+ *          samples at once for shapes with many (head, query tile) pairs), and every chunk's
+ *          sum is added to acc in ascending order of the chunks, so results are reproducible
+ *          bit for bit on a given device.
  *   Q, K   [B,H,Lq,d], [B,H,Lk,d] of type dt (AP_BF16 and AP_F16 run on the tensor cores)
  *   bias   [H,Lq,Lk] fp32 added after scaling, or NULL
  *   scale  multiplier of Q.K^T; 0 selects 1/sqrt(d)

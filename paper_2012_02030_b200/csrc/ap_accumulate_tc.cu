@@ -1,6 +1,6 @@
 // Eq. 1 as a running sum for bf16 and fp16 tensors, on the tcgen05 tensor cores.
 //
-// One CTA owns one (head, 128-row query tile) and adds, for up to 16 samples b per launch,
+// One CTA owns one (head, 128-row query tile) and adds, for up to 32 samples b per launch,
 // the normalised softmax rows to the accumulator.  A softmax row needs its
 // maximum and its sum of exponentials over ALL keys before any entry can be
 // normalised, and the sum over b needs each sample normalised separately, so
@@ -15,8 +15,13 @@
 // The bias tile of a key tile is staged once per sweep and key tile by TMA (fp32,
 // 128-byte swizzle, so that a thread reads its own row without bank conflicts),
 // copied to registers and reused for all b.  Samples are added in ascending b by
-// a fixed thread and every accumulator entry receives exactly one addition per
-// launch, so results are reproducible bit for bit.  Where the accumulator's rows are
+// a fixed thread and every accumulator entry receives exactly one addition per CTA that
+// owns it, so results are reproducible bit for bit.  Shapes with few (head, query tile)
+// pairs would leave most SMs idle; for them a launch's samples are cut into chunks, one
+// CTA per (chunk, head, query tile), and the chunks' sums are added to the accumulator
+// in ascending chunk order: per key tile a counter in global memory says how many warps
+// of lower chunks have finished their addition, and a CTA waits (bounded) for its turn
+// before it issues its own.  Where the accumulator's rows are
 // 16-byte multiples that addition is a TMA reduction: each softmax warp stages its
 // 32 rows x 32 columns in shared memory (128-byte swizzle again) and one lane issues
 // cp.reduce.async.bulk.tensor ... add, which updates whole 128-byte lines in L2;
@@ -36,6 +41,8 @@
 // bounded.
 #include <math_constants.h>
 
+#include <atomic>
+
 #include "ap_common.cuh"
 #include "ap_sm100.cuh"
 
@@ -51,8 +58,8 @@ constexpr int kSoftmaxWarps = kSoftmaxThreads / 32;
 constexpr int kSubBytes = 128 * 128;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kSumCol = 256;    // running sum over b: 128 columns
-constexpr uint32_t kStatsCol = 384;  // (max, sum) pairs: 32 columns per column half, 2 per sample
-constexpr int kMaxB = 16;            // samples per launch
+constexpr uint32_t kStatsCol = 384;  // (max, sum) pairs: 64 columns per column half, 2 per sample
+constexpr int kMaxB = 32;            // samples per launch (what the spare tensor-memory columns hold)
 constexpr int kBiasBytes = 128 * 128 * 4;  // one fp32 bias tile: 4 boxes of 128 rows x 32 columns
 constexpr int kRedBytes = 32 * 128;        // per softmax warp: 32 rows x 32 fp32 columns on their way to the accumulator
 constexpr float kLog2e = 1.4426950408889634f;
@@ -89,6 +96,32 @@ __device__ __forceinline__ float lg2_approx(float x) {
   return y;
 }
 
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Turn counters of the chunked launches: one word per (head, query tile, key tile), zeroed before every
+// such launch.  Launches that overlap on the GPU (different streams) take different sets.
+constexpr size_t kTurnWords = 8192;
+constexpr int kTurnSets = 8;
+constexpr int kMinChunk = 2;  // samples per CTA at least
+__device__ unsigned g_turn[kTurnSets][kTurnWords];
+
+unsigned *turn_words() {
+  static std::atomic<unsigned> next{0};
+  static unsigned *base[16] = {nullptr};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return nullptr;
+  if (!base[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_turn) != cudaSuccess) return nullptr;
+    base[dev] = static_cast<unsigned *>(p);
+  }
+  return base[dev] + (size_t)(next.fetch_add(1) % kTurnSets) * kTurnWords;
+}
+
 // Bounded wait that also gives up as soon as another thread of the CTA has.
 __device__ __noinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag, unsigned *err,
                                            uint32_t max_polls) {
@@ -113,13 +146,15 @@ __device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, int la
 
 // dbg_skip != 0 (test hook): the copies of the first visit are never issued, so the MMA issuer's
 // first wait runs out and the CTA leaves through its error path.
-template <int D>
+// kChunked: the instantiation for launches whose samples are cut into chunks (see below); a
+// separate one so that its extra code costs the plain launches nothing.
+template <int D, bool kChunked>
 __global__ void __launch_bounds__(kThreads, 1)
 accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_bias, const __grid_constant__ CUtensorMap map_acc,
                      int bias_by_tma, int acc_by_tma, float *__restrict__ acc, const float *__restrict__ bias, int b0,
-                     int Bc, int H, int Lq, int Lk, int n_qt, int n_kt, int causal, int f16, float scale_log2,
-                     unsigned *err, uint32_t max_polls, int dbg_skip) {
+                     int Bc_all, int chunk_samples, unsigned *__restrict__ turn, int H, int Lq, int Lk, int n_qt,
+                     int n_kt, int causal, int f16, float scale_log2, unsigned *err, uint32_t max_polls, int dbg_skip) {
   using C = Cfg<D>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char *smem =
@@ -127,9 +162,17 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   unsigned char *bias_s = smem + C::kBiasOffset;
   Barriers *bars = reinterpret_cast<Barriers *>(smem + C::kBarOffset);
 
+  // Small shapes have fewer (head, query tile) pairs than the GPU has SMs; the launch's samples are
+  // then cut into chunks, CTA (chunk, head, query tile) takes chunk_samples of them, and the chunks'
+  // sums are added to the accumulator in ascending order of the chunks (turn[], see below), so that
+  // the result does not depend on which CTA finishes first.  Lower chunks have lower block indices.
+  const int unit = kChunked ? (int)blockIdx.x % (H * n_qt) : (int)blockIdx.x;
+  const int chunk = kChunked ? (int)blockIdx.x / (H * n_qt) : 0;
+  if (kChunked) b0 += chunk * chunk_samples;
+  const int Bc = kChunked ? min(chunk_samples, Bc_all - chunk * chunk_samples) : Bc_all;
   // late query tiles (most key tiles under a causal mask) first
-  const int qt = n_qt - 1 - (int)(blockIdx.x / H);
-  const int h = blockIdx.x % H;
+  const int qt = n_qt - 1 - unit / H;
+  const int h = unit % H;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // causal: row i looks at keys j <= i + (Lk - Lq), i.e. Lk - Lq memory keys, then its own segment
   const int off = causal ? Lk - Lq : 0;
@@ -237,8 +280,8 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const bool vec = (Lk & 3) == 0;
     const uint32_t s_addr = tmem + lane_addr + 64 * wg;                   // + 128 * buf
     const uint32_t sum_addr = tmem + lane_addr + kSumCol + 64 * wg;       // + 32 * c
-    const uint32_t my_stats = tmem + lane_addr + kStatsCol + 32 * wg;     // + 2 * b
-    const uint32_t other_stats = tmem + lane_addr + kStatsCol + 32 * (1 - wg);
+    const uint32_t my_stats = tmem + lane_addr + kStatsCol + 64 * wg;     // + 2 * b
+    const uint32_t other_stats = tmem + lane_addr + kStatsCol + 64 * (1 - wg);
     // this warp's 32 rows x 32 columns on their way to the accumulator, and the rows' place in it
     unsigned char *red_s = smem + C::kRedOffset + warp * kRedBytes;
     const int red_y = qt * kTile + (warp & 3) * 32;
@@ -419,9 +462,37 @@ accumulate_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             fence_proxy_async_smem();
             __syncwarp();
             const int x = j0 + 32 * c;
+            if (kChunked && c == 0) {
+              // this key tile's entries have received the sums of all lower chunks once their eight
+              // warps each have counted themselves in (bounded wait)
+              if (lane == 0) {
+                const unsigned *flag = turn + ((size_t)h * n_qt + qt) * n_kt + kt;
+                const unsigned want = (unsigned)chunk * kSoftmaxWarps;
+                uint32_t polls = 0;
+                while (ld_acquire_gpu(flag) < want && ok) {
+                  if (*abort_flag || ++polls > max_polls) {
+                    if (!*abort_flag) {
+                      *abort_flag = 1;
+                      atomicOr(err, kDevErrTimeout);
+                    }
+                    ok = false;
+                  } else if (polls > 64) {
+                    __nanosleep(128);
+                  }
+                }
+              }
+              ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+              if (!ok) break;
+            }
             if (lane == 0 && red_y < Lq && x < red_jend) {
               tma_reduce_add_3d(&map_acc, red_s, x, red_y, h);
               bulk_commit_group();
+            }
+            if (kChunked && c == 1 && lane == 0) {
+              // both blocks of this warp are in the accumulator: count this warp in for the next chunk
+              bulk_wait_group0();
+              __threadfence();
+              atomicAdd(turn + ((size_t)h * n_qt + qt) * n_kt + kt, 1u);
             }
           } else if (row_ok) {
             // accumulator rows that are no 16-byte multiples: one red per entry (entries outside the
@@ -462,19 +533,42 @@ template <int D>
 cudaError_t launch(const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mb, const CUtensorMap &ma,
                    int bias_by_tma, int acc_by_tma, float *acc, const float *bias, int B, int H, int Lq, int Lk,
                    int causal, int f16, float scale, unsigned *err, cudaStream_t s) {
-  auto kern = accumulate_tc_kernel<D>;
+  auto kern = accumulate_tc_kernel<D, false>;
+  auto kern_chunked = accumulate_tc_kernel<D, true>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(kern_chunked, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int n_qt = ceil_div(Lq, kTile), n_kt = ceil_div(Lk, kTile);
   const DebugKnobs knobs = debug_knobs();
-  // samples in ascending order, at most kMaxB per launch; launches on one stream run in order
-  for (int b0 = 0; b0 < B; b0 += kMaxB) {
-    const int Bc = B - b0 < kMaxB ? B - b0 : kMaxB;
-    kern<<<knobs.skip_arrive ? 1 : H * n_qt, kThreads, Cfg<D>::kSmemBytes, s>>>(
-        mq, mk, mb, ma, bias_by_tma, acc_by_tma, acc, bias, b0, Bc, H, Lq, Lk, n_qt, n_kt, causal, f16, scale * kLog2e,
-        err, knobs.max_polls, knobs.skip_arrive);
+  // Shapes with at most half as many (head, query tile) pairs as SMs: several CTAs per pair, each with
+  // a chunk of the samples, taking turns at the accumulator (one wave of CTAs, one per SM).
+  const int n_units = H * n_qt, sms = sm_count();
+  int max_chunks = 1;
+  unsigned *turn = nullptr;
+  if (acc_by_tma && !knobs.skip_arrive && sms > 0 && 2 * n_units <= sms && (size_t)n_units * n_kt <= kTurnWords) {
+    turn = turn_words();
+    if (turn) max_chunks = sms / n_units;
+  }
+  // samples in ascending order, at most kMaxB per CTA and launch; launches on one stream run in order
+  for (int b0 = 0; b0 < B;) {
+    const int left = B - b0;
+    int chunks = 1, per = left < kMaxB ? left : kMaxB;
+    if (max_chunks > 1 && left >= 2 * kMinChunk) {
+      chunks = left / kMinChunk < max_chunks ? left / kMinChunk : max_chunks;
+      per = ceil_div(left, chunks);
+      if (per > kMaxB) per = kMaxB;
+      chunks = ceil_div(left < chunks * per ? left : chunks * per, per);
+    }
+    const int Bc = left < chunks * per ? left : chunks * per;
+    unsigned *t = chunks > 1 ? turn : nullptr;
+    if (t && (e = cudaMemsetAsync(t, 0, (size_t)n_units * n_kt * sizeof(unsigned), s)) != cudaSuccess) return e;
+    (t ? kern_chunked : kern)<<<knobs.skip_arrive ? 1 : n_units * chunks, kThreads, Cfg<D>::kSmemBytes, s>>>(
+        mq, mk, mb, ma, bias_by_tma, acc_by_tma, acc, bias, b0, Bc, per, t, H, Lq, Lk, n_qt, n_kt, causal, f16,
+        scale * kLog2e, err, knobs.max_polls, knobs.skip_arrive);
     count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    b0 += Bc;
   }
   return cudaSuccess;
 }

@@ -61,6 +61,9 @@ struct DebugKnobs {
 };
 DebugKnobs debug_knobs();
 
+// SMs of the current device (0 if it cannot be queried).
+int sm_count();
+
 // Kernels launched by this library in this process (see ap_launch_count in ap.h).
 void count_launches(int n);
 

@@ -868,18 +868,6 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
   if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
-int sm_count() {
-  static int cached[64] = {0};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-  if (cached[dev] == 0) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    cached[dev] = n;
-  }
-  return cached[dev];
-}
-
 template <int D, bool kSplit, bool kF16, bool kGath>
 cudaError_t launch_kernel(const FwdMaps &maps, const void *K, const void *V, void *O, const ap_tiles &t, int B, int H,
                           int Lq, int Lk, const DebugKnobs &dbg, float scale, unsigned *err, cudaStream_t s) {
