@@ -576,6 +576,31 @@ def test_forward_random_masks_ragged_shapes(ap, shape, d, dtype):
     assert np.all(o[:, empty] == 0.0)
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_forward_many_one_round_items_per_cta_poisoned_output(ap, d):
+    """Far more items than four per SM, each of one round (one query tile, one key tile): the softmax
+    warps run ahead of the epilogue warps as far as the hand-over ring lets them, and the end of a
+    CTA's work follows a row of very short items.  Every output element must have been written."""
+    B, H, L = 64, 16, 128  # 1024 items of one round on 148 CTAs
+    w = W["tiny"].scaled(B=B, H=H, Lq=L, Lk=L, d=d, dtype="bf16")
+    q, k, v = inputs.eval_qkv(w)
+    mask = inputs.random_mask(H, L, L, 0.8, seed=91, causal=True)  # (dense rows: the fixed absolute tolerance applies)
+    tiles = ap.Tiles(H, L, L)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    out = torch.full_like(q, float("nan")).cuda()
+    for _ in range(3):  # the race, if there were one, would not show on every launch
+        out.fill_(float("nan"))
+        ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles, out)
+        assert ap.ap_device_status() == ap.AP_OK
+        assert not torch.isnan(out).any()
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy())
+    # (a million rows, the first of each head with one or two kept entries: |O| reaches the largest single
+    # values of V, whose bf16 rounding alone exceeds the fixed absolute bound; so bound by value as well)
+    got = out.float().cpu().numpy()
+    np.testing.assert_allclose(got, ref, rtol=2.0 ** -8, atol=6e-3)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= pu.TOL["bf16"]["rel_l2"]
+
+
 # ---- the same attention with the 1.5-entmax normaliser
 
 
