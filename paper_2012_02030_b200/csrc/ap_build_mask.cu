@@ -281,7 +281,9 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
 struct Picked {
   uint32_t key, count, rank_in_ties;
 };
-__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch) {
+// scan(fn) calls fn(key) once for every key, the keys spread over the CTA's threads in any way.
+template <typename Scan>
+__device__ Picked block_select_over(uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch, Scan scan) {
   __shared__ uint32_t warp_sums[32];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   uint32_t prefix = 0u, hi_mask = 0u, count = n;
@@ -291,17 +293,9 @@ __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, 
     hist[t] = 0u;
     hist[t + 1024] = 0u;
     __syncthreads();
-    for (uint32_t idx0 = t; idx0 < n; idx0 += 8 * 1024) {  // eight loads in flight per thread
-      uint32_t kk[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const uint32_t idx = idx0 + u * 1024;
-        kk[u] = idx < n ? keys[idx] : 0xffffffffu;
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (idx0 + u * 1024 < n && (kk[u] & hi_mask) == prefix) atomicAdd(&hist[(kk[u] >> shift) & dmask], 1u);
-    }
+    scan([&](uint32_t key) {
+      if ((key & hi_mask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+    });
     __syncthreads();
     // thread t owns bins 2047 - 2t and 2046 - 2t (descending order of keys)
     const uint32_t c0 = hist[kBins - 1 - 2 * t], c1 = hist[kBins - 2 - 2 * t];
@@ -334,6 +328,21 @@ __device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, 
   p.count = count;
   p.rank_in_ties = rank;
   return p;
+}
+__device__ Picked block_select(const uint32_t *keys, uint32_t n, uint32_t rank, uint32_t *hist, uint32_t *xch) {
+  return block_select_over(n, rank, hist, xch, [&](auto fn) {
+    for (uint32_t idx0 = threadIdx.x; idx0 < n; idx0 += 8 * 1024) {  // eight loads in flight per thread
+      uint32_t kk[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t idx = idx0 + u * 1024;
+        kk[u] = idx < n ? keys[idx] : 0xffffffffu;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (idx0 + u * 1024 < n) fn(kk[u]);
+    }
+  });
 }
 
 __device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
@@ -594,6 +603,108 @@ __global__ void __launch_bounds__(1024) cand_finish_kernel(SelectState *state, c
     state[h].prefix = st.prefix + st.lo;
     state[h].done = 1u;
   }
+}
+
+// ---- small selections: everything in one CTA ----------------------------------------------------
+
+constexpr long long kSelectSmallEntries = 1ll << 15;  // rows x Lk of a selection, at most
+
+// One CTA of 1024 threads per selection of at most kSelectSmallEntries entries: sets up the
+// selection's state (and nnz), finds the threshold with the CTA-wide radix select straight over
+// the selection's domain, and where only some of the entries equal to the threshold are kept, the
+// linear index of the last kept one (tie_cut): by ranking the ties when there are at most
+// kMaxCutTies of them, else by bisection on the index (each probe counts the ties up to it).  Such a
+// selection needs no other kernel before the emit pass.
+__global__ void __launch_bounds__(1024) select_small_kernel(const float *__restrict__ acc, int rows, int Lk,
+                                                            int period, int causal, int diag,
+                                                            unsigned long long k_rest, SelectState *state, int H,
+                                                            long long nnz_init, int64_t *nnz) {
+  __shared__ uint32_t hist[kBins];
+  __shared__ uint32_t xch[4];
+  __shared__ uint32_t tie_idx[kMaxCutTies];
+  __shared__ uint32_t tie_n_s, cut_s;
+  const int h = blockIdx.x;
+  if (nnz && h == 0)
+    for (int x = threadIdx.x; x < H; x += 1024) nnz[x] = nnz_init;
+  SelectState st;
+  st.prefix = 0u, st.thr = 0xffffffffu, st.remaining = k_rest, st.ties_kept = 0ull, st.all_ties_kept = 0u;
+  st.done = 1u, st.lo = 0u, st.hi = 0xffffffffu, st.above_hi = 0ull, st.n_cand = 0u, st.use_shortcut = 0u;
+  st.tie_cut = 0u, st.have_cut = 0u, st.cand_select = 0u, st.thr_count = 0u, st.tie_n = 0u;
+  if (k_rest == 0ull) {  // nothing but the forced entries is kept
+    if (threadIdx.x == 0) state[h] = st;
+    return;
+  }
+  const float *base = acc + (size_t)h * rows * Lk;
+  const int off = (causal || diag) ? Lk - period : 0;
+  const uint32_t n = (uint32_t)rows * (uint32_t)Lk;
+  const bool vec = (Lk & 3) == 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // fn(key, linear index) for every selectable entry of rows [0, row_end): a warp takes a row at a time,
+  // its lanes four consecutive entries each, two loads in flight
+  auto scan_rows = [&](int row_end, auto fn) {
+    for (int i = warp; i < row_end; i += 32) {
+      const float *row = base + (size_t)i * Lk;
+      const int own = i % period + off;  // the row's own position among the keys
+      const int jend = causal ? min(Lk, own + 1) : Lk;
+      for (int j00 = 0; j00 < jend; j00 += 256) {
+        float v[2][4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int j0 = j00 + 128 * u + 4 * lane;
+          v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0.f;
+          if (j0 < jend) load4(row, j0, jend, vec, v[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int j = j00 + 128 * u + 4 * lane + c;
+            if (j < jend && !(diag && j == own)) fn(key_of(v[u][c]), (uint32_t)i * (uint32_t)Lk + (uint32_t)j);
+          }
+      }
+    }
+  };
+  const Picked p = block_select_over(n, (uint32_t)k_rest, hist, xch, [&](auto fn) {
+    scan_rows(rows, [&](uint32_t key, uint32_t) { fn(key); });
+  });
+  st.prefix = st.thr = p.key;
+  st.remaining = st.ties_kept = p.rank_in_ties;
+  st.thr_count = p.count;
+  st.all_ties_kept = p.rank_in_ties == p.count ? 1u : 0u;
+  if (!st.all_ties_kept) {
+    if (p.count <= (uint32_t)kMaxCutTies) {
+      if (threadIdx.x == 0) tie_n_s = 0u;
+      __syncthreads();
+      scan_rows(rows, [&](uint32_t key, uint32_t idx) {
+        if (key == p.key) tie_idx[atomicAdd(&tie_n_s, 1u)] = idx;
+      });
+      __syncthreads();
+      rank_ties(tie_idx, p.count, p.rank_in_ties, &cut_s);
+    } else {
+      // the smallest index L with rank_in_ties ties at indices <= L
+      uint32_t lo = 0u, hi = n - 1u;
+      while (lo < hi) {  // the same for every thread
+        const uint32_t mid = lo + (hi - lo) / 2u;
+        uint32_t mine = 0u;
+        scan_rows((int)(mid / (uint32_t)Lk) + 1, [&](uint32_t key, uint32_t idx) {
+          mine += (key == p.key && idx <= mid) ? 1u : 0u;
+        });
+        if (threadIdx.x == 0) tie_n_s = 0u;
+        __syncthreads();
+        mine = __reduce_add_sync(0xffffffffu, mine);
+        if (lane == 0 && mine) atomicAdd(&tie_n_s, mine);
+        __syncthreads();
+        const uint32_t upto = tie_n_s;
+        __syncthreads();
+        if (upto >= p.rank_in_ties) hi = mid; else lo = mid + 1u;
+      }
+      if (threadIdx.x == 0) cut_s = lo;
+      __syncthreads();
+    }
+    st.tie_cut = cut_s;
+    st.have_cut = 1u;
+  }
+  if (threadIdx.x == 0) state[h] = st;
 }
 
 // Entries equal to the threshold key per (row, 128-column segment); only for heads
@@ -902,6 +1013,23 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
   cudaError_t e;
   // per head nnz = k; per layer, or with all ties kept, the emit pass counts it
   const bool count_nnz = a.per_layer || a.keep_ties;
+  {
+    // very small selections: one kernel instead of the passes below (measured: one CTA per selection
+    // beats the ten launches of the passes up to about 2^15 entries per selection: 0.085 -> 0.065 ms on
+    // B32 H12 L128; at 2^17 and more it loses, the passes spread a selection over many CTAs)
+    if ((long long)rows * a.Lk <= kSelectSmallEntries) {
+      select_small_kernel<<<n_sel, 1024, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
+                                                 (unsigned long long)a.k_rest, sc.state, a.H,
+                                                 count_nnz ? 0ll : (long long)a.k, a.nnz);
+      count_launches(1);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer,
+                                                    a.keep_ties, sc.state, sc.tie_count, a.mask, a.stage_bitmap,
+                                                    a.stage_count, a.nnz);
+      count_launches(1);
+      return cudaGetLastError();
+    }
+  }
   init_state_kernel<<<ceil_div(max(n_sel * kBins, a.H), 256), 256, 0, s>>>(
       sc.state, sc.hist, n_sel, (unsigned long long)a.k_rest, a.H, count_nnz ? 0ll : (long long)a.k, a.nnz);
   count_launches(1);
