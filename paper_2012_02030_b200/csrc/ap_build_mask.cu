@@ -67,7 +67,26 @@ struct SelectState {  // per selection
   uint32_t cand_select;          // the bracket holds the threshold: the passes over the collected keys run
   uint32_t thr_count;            // entries equal to the threshold key
   uint32_t tie_n;                // entries gathered in the tie list
+  // CTAs of the running kernel that have finished their share of this selection: the last one goes on
+  // with the step that needs all of them (digit pick, tie scan, finish) and puts the count back to zero
+  uint32_t ticket;
 };
+
+// Called by all threads of a CTA when its share of selection h is done (its global writes issued):
+// true in exactly the CTA that finishes last, which then sees everything the others wrote.
+__device__ __forceinline__ bool last_cta_of(SelectState *state, int h, uint32_t n_ctas) {
+  __shared__ uint32_t last_s;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool last = atomicAdd(&state[h].ticket, 1u) == n_ctas - 1u;
+    if (last) state[h].ticket = 0u;
+    last_s = last ? 1u : 0u;
+  }
+  __syncthreads();
+  if (last_s) __threadfence();
+  return last_s != 0u;
+}
 
 // Selection among the keys the one-pass shortcut collected (see below).
 // The bracket holds the threshold (the (k_rest - above_hi)-th largest collected key) and every key
@@ -135,11 +154,15 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int n_sel,
     state[idx].cand_select = 0u;
     state[idx].thr_count = 0u;
     state[idx].tie_n = 0u;
+    state[idx].ticket = 0u;
   }
 }
 
+__device__ void pick_digit(SelectState *state, uint32_t *hist, int h, int pass, int from_cand, uint32_t cand_cap,
+                           unsigned long long k_rest);
+
 // Histogram of one digit over the non-forced domain entries whose higher digits
-// equal the prefix found so far.  grid = (row blocks, selections); a warp takes a row at
+// equal the prefix found so far; the CTA that finishes last picks the digit.  grid = (row blocks, selections); a warp takes a row at
 // a time and its lanes stride over the row, two float4 loads in flight each.
 // Here and in the kernels below Lq counts the rows of the selection and row i has
 // the domain of row i % period of a head (period == Lq unless heads are stacked).
@@ -148,8 +171,7 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int n_sel,
 // is the forced entry when the diagonal is kept.
 __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *__restrict__ acc, int Lq, int Lk,
                                                                    int period, int causal, int diag, int pass,
-                                                                   const SelectState *__restrict__ state,
-                                                                   uint32_t *__restrict__ hist) {
+                                                                   SelectState *state, uint32_t *hist) {
   __shared__ uint32_t sh[kBins];
   const int h = blockIdx.y;
   if (state[h].done) return;  // resolved by the shortcut
@@ -199,6 +221,7 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
     const uint32_t s = sh[b];
     if (s) atomicAdd(&hist[h * kBins + b], s);
   }
+  if (last_cta_of(state, h, gridDim.x)) pick_digit(state, hist, h, pass, 0, 0u, 0ull);
 }
 
 // One CTA per head: picks the digit whose bin contains the wanted rank.  Thread t
@@ -206,10 +229,10 @@ __global__ void __launch_bounds__(kThreads) digit_histogram_kernel(const float *
 // threads' sums locates the owner, which then walks its eight bins.
 // from_cand: the histogram came from the collected keys (offsets from the lower pivot); the first
 // such pass opens the selection among them if the bracket holds the threshold.
-__global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uint32_t *hist, int pass, int from_cand,
-                                                         uint32_t cand_cap, unsigned long long k_rest) {
+// Run by the last CTA (256 threads) of the histogram pass that filled hist.
+__device__ void pick_digit(SelectState *state, uint32_t *hist, int h, int pass, int from_cand, uint32_t cand_cap,
+                           unsigned long long k_rest) {
   __shared__ uint32_t warp_sums[8];
-  const int h = blockIdx.x;
   if (!from_cand && state[h].done) return;  // resolved by the shortcut
   if (from_cand) {
     const SelectState cur = state[h];
@@ -229,7 +252,7 @@ __global__ void __launch_bounds__(256) pick_digit_kernel(SelectState *state, uin
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
     const int bin = kBins - 1 - (8 * (int)threadIdx.x + e);
-    cnt[e] = hist[h * kBins + bin];
+    cnt[e] = __ldcg(hist + h * kBins + bin);
     hist[h * kBins + bin] = 0u;
     mine += cnt[e];
   }
@@ -507,14 +530,17 @@ __global__ void __launch_bounds__(kThreads) collect_kernel(const float *__restri
 
 
 // grid = (CTAs, selections)
-__global__ void __launch_bounds__(kThreads) cand_histogram_kernel(const SelectState *__restrict__ state,
-                                                                  const uint2 *__restrict__ cand, uint32_t cand_cap,
-                                                                  unsigned long long k_rest, int pass,
-                                                                  uint32_t *__restrict__ hist) {
+__global__ void __launch_bounds__(kThreads) cand_histogram_kernel(SelectState *state, const uint2 *__restrict__ cand,
+                                                                  uint32_t cand_cap, unsigned long long k_rest,
+                                                                  int pass, uint32_t *hist) {
   __shared__ uint32_t sh[kBins];
   const int h = blockIdx.y;
   const SelectState st = state[h];
-  if (!(pass == 0 ? bracket_holds(st, cand_cap, k_rest) : st.cand_select != 0u) || digit_is_zero(st, pass)) return;
+  if (!(pass == 0 ? bracket_holds(st, cand_cap, k_rest) : st.cand_select != 0u)) return;
+  if (digit_is_zero(st, pass)) {  // no pass needed; the first CTA lets the pick open the selection
+    if (blockIdx.x == 0) pick_digit(state, hist, h, pass, 1, cand_cap, k_rest);
+    return;
+  }
   const int lane = threadIdx.x & 31;
   for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0u;
   __syncthreads();
@@ -548,30 +574,13 @@ __global__ void __launch_bounds__(kThreads) cand_histogram_kernel(const SelectSt
     const uint32_t s = sh[b];
     if (s) atomicAdd(&hist[h * kBins + b], s);
   }
-}
-
-// Gathers the linear indices of the collected entries equal to the threshold, when they must be
-// ranked and are few enough.  grid = (CTAs, selections)
-__global__ void __launch_bounds__(kThreads) cand_ties_kernel(SelectState *state, const uint2 *__restrict__ cand,
-                                                             uint32_t cand_cap, uint32_t *__restrict__ tie_list) {
-  const int h = blockIdx.y;
-  const SelectState st = state[h];
-  if (!st.cand_select || st.all_ties_kept || st.thr_count > (uint32_t)kMaxCutTies) return;
-  const uint32_t want = st.prefix + st.lo;
-  const uint2 *mine = cand + (size_t)h * cand_cap;
-  for (uint32_t idx = blockIdx.x * kThreads + threadIdx.x; idx < st.n_cand; idx += gridDim.x * kThreads) {
-    const uint2 c = mine[idx];
-    if (c.x == want) {
-      const uint32_t pos = atomicAdd(&state[h].tie_n, 1u);
-      if (pos < (uint32_t)kMaxCutTies) tie_list[(size_t)h * kMaxCutTies + pos] = c.y;
-    }
-  }
+  if (last_cta_of(state, h, gridDim.x)) pick_digit(state, hist, h, pass, 1, cand_cap, k_rest);
 }
 
 // Ranks `count` <= kMaxCutTies distinct linear indices: returns (in *cut_s, after a barrier) the one
-// with exactly rank - 1 smaller ones.  CTA of 1024 threads.
+// with exactly rank - 1 smaller ones.  By all threads of a CTA.
 __device__ void rank_ties(const uint32_t *tie_idx, uint32_t count, uint32_t rank, uint32_t *cut_s) {
-  for (uint32_t e = threadIdx.x; e < count; e += 1024) {
+  for (uint32_t e = threadIdx.x; e < count; e += blockDim.x) {
     const uint32_t me = tie_idx[e];
     uint32_t smaller = 0u;
     for (uint32_t f = 0; f < count; ++f) smaller += tie_idx[f] < me ? 1u : 0u;
@@ -580,25 +589,39 @@ __device__ void rank_ties(const uint32_t *tie_idx, uint32_t count, uint32_t rank
   __syncthreads();
 }
 
-// One CTA per selection: turns the digits found among the collected keys into the threshold,
-// ranks its ties when not all of them are kept (the lowest linear indices are), and closes the
-// selection.
-__global__ void __launch_bounds__(1024) cand_finish_kernel(SelectState *state, const uint32_t *__restrict__ tie_list) {
+// Closes the selection among the collected keys.  grid = (CTAs, selections).  First the linear indices
+// of the collected entries equal to the threshold are gathered, when they must be ranked and are few
+// enough; the CTA that finishes last then turns the digits found among the collected keys into the
+// threshold, ranks those ties (the lowest linear indices are kept) and marks the selection as done.
+__global__ void __launch_bounds__(kThreads) cand_finish_kernel(SelectState *state, const uint2 *__restrict__ cand,
+                                                               uint32_t cand_cap, uint32_t *tie_list) {
   __shared__ uint32_t tie_idx[kMaxCutTies];
   __shared__ uint32_t cut_s;
-  const int h = blockIdx.x;
+  const int h = blockIdx.y;
   const SelectState st = state[h];
   if (!st.cand_select) return;
-  bool have_cut = false;
-  if (!st.all_ties_kept && st.thr_count <= (uint32_t)kMaxCutTies) {
-    for (uint32_t e = threadIdx.x; e < st.thr_count; e += 1024) tie_idx[e] = tie_list[(size_t)h * kMaxCutTies + e];
+  const bool rank_them = !st.all_ties_kept && st.thr_count <= (uint32_t)kMaxCutTies;
+  if (rank_them) {
+    const uint32_t want = st.prefix + st.lo;
+    const uint2 *mine = cand + (size_t)h * cand_cap;
+    for (uint32_t idx = blockIdx.x * kThreads + threadIdx.x; idx < st.n_cand; idx += gridDim.x * kThreads) {
+      const uint2 c = mine[idx];
+      if (c.x == want) {
+        const uint32_t pos = atomicAdd(&state[h].tie_n, 1u);
+        if (pos < (uint32_t)kMaxCutTies) tie_list[(size_t)h * kMaxCutTies + pos] = c.y;
+      }
+    }
+  }
+  if (!last_cta_of(state, h, gridDim.x)) return;
+  if (rank_them) {
+    for (uint32_t e = threadIdx.x; e < st.thr_count; e += kThreads)
+      tie_idx[e] = __ldcg(tie_list + (size_t)h * kMaxCutTies + e);
     __syncthreads();
     rank_ties(tie_idx, st.thr_count, (uint32_t)st.ties_kept, &cut_s);
-    have_cut = true;
   }
   if (threadIdx.x == 0) {
-    state[h].tie_cut = have_cut ? cut_s : 0u;
-    state[h].have_cut = have_cut ? 1u : 0u;
+    state[h].tie_cut = rank_them ? cut_s : 0u;
+    state[h].have_cut = rank_them ? 1u : 0u;
     state[h].thr = st.prefix + st.lo;
     state[h].prefix = st.prefix + st.lo;
     state[h].done = 1u;
@@ -629,7 +652,7 @@ __global__ void __launch_bounds__(1024) select_small_kernel(const float *__restr
   SelectState st;
   st.prefix = 0u, st.thr = 0xffffffffu, st.remaining = k_rest, st.ties_kept = 0ull, st.all_ties_kept = 0u;
   st.done = 1u, st.lo = 0u, st.hi = 0xffffffffu, st.above_hi = 0ull, st.n_cand = 0u, st.use_shortcut = 0u;
-  st.tie_cut = 0u, st.have_cut = 0u, st.cand_select = 0u, st.thr_count = 0u, st.tie_n = 0u;
+  st.tie_cut = 0u, st.have_cut = 0u, st.cand_select = 0u, st.thr_count = 0u, st.tie_n = 0u, st.ticket = 0u;
   if (k_rest == 0ull) {  // nothing but the forced entries is kept
     if (threadIdx.x == 0) state[h] = st;
     return;
@@ -708,11 +731,11 @@ __global__ void __launch_bounds__(1024) select_small_kernel(const float *__restr
 }
 
 // Entries equal to the threshold key per (row, 128-column segment); only for heads
-// where the ties must be ranked.  grid = (row blocks, H); a warp takes a row.
+// where the ties must be ranked.  grid = (row blocks, H); a warp takes a row.  The CTA that finishes
+// last turns the head's counts into their exclusive prefix sum, in place.
 __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__restrict__ acc, int Lq, int Lk, int period,
-                                                             int n_kt, int causal, int diag,
-                                                             const SelectState *__restrict__ state,
-                                                             uint32_t *__restrict__ tie_count) {
+                                                             int n_kt, int causal, int diag, SelectState *state,
+                                                             uint32_t *tie_count) {
   const int h = blockIdx.y;
   if (state[h].all_ties_kept || state[h].have_cut) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -740,21 +763,16 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
       if (lane == 0) tie_count[((size_t)h * Lq + i) * n_kt + kt] = (uint32_t)ties;
     }
   }
-}
-
-// One CTA per head: in-place exclusive prefix sum over the head's (row, segment) tie counts.
-__global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ tie_count, int n_per_head,
-                                                        const SelectState *__restrict__ state) {
-  if (state[blockIdx.x].all_ties_kept || state[blockIdx.x].have_cut) return;
-  __shared__ uint32_t warp_sums[32];
+  if (!last_cta_of(state, h, gridDim.x)) return;
+  __shared__ uint32_t warp_sums[kWarps];
   __shared__ uint32_t carry_s;
-  uint32_t *a = tie_count + (size_t)blockIdx.x * n_per_head;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n_per_head = Lq * n_kt;
+  uint32_t *a = tie_count + (size_t)h * n_per_head;
   if (threadIdx.x == 0) carry_s = 0u;
   __syncthreads();
-  for (int base = 0; base < n_per_head; base += 1024) {
+  for (int base = 0; base < n_per_head; base += kThreads) {
     const int idx = base + threadIdx.x;
-    const uint32_t x = idx < n_per_head ? a[idx] : 0u;
+    const uint32_t x = idx < n_per_head ? __ldcg(a + idx) : 0u;
     uint32_t incl = x;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -763,20 +781,16 @@ __global__ void __launch_bounds__(1024) tie_scan_kernel(uint32_t *__restrict__ t
     }
     if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
-    if (warp == 0) {
-      uint32_t v = warp_sums[lane];
+    uint32_t before = 0u, total = 0u;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        uint32_t u = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= o) v += u;
-      }
-      warp_sums[lane] = v;
+    for (int w = 0; w < kWarps; ++w) {
+      if (w < warp) before += warp_sums[w];
+      total += warp_sums[w];
     }
-    __syncthreads();
     const uint32_t carry = carry_s;
-    if (idx < n_per_head) a[idx] = carry + (warp ? warp_sums[warp - 1] : 0u) + incl - x;
+    if (idx < n_per_head) a[idx] = carry + before + incl - x;
     __syncthreads();
-    if (threadIdx.x == 1023) carry_s = carry + warp_sums[31];
+    if (threadIdx.x == 0) carry_s = carry + total;
     __syncthreads();
   }
 }
@@ -1060,12 +1074,9 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
       for (int pass = 0; pass < kPasses; ++pass) {
         cand_histogram_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap,
                                                              (unsigned long long)a.k_rest, pass, sc.hist);
-        pick_digit_kernel<<<n_sel, 256, 0, s>>>(sc.state, sc.hist, pass, 1, (uint32_t)cap,
-                                                (unsigned long long)a.k_rest);
       }
-      cand_ties_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, sc.tie_list);
-      cand_finish_kernel<<<n_sel, 1024, 0, s>>>(sc.state, sc.tie_list);
-      count_launches(4 + 2 * kPasses);
+      cand_finish_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, sc.tie_list);
+      count_launches(3 + kPasses);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     for (int pass = 0; pass < kPasses; ++pass) {
@@ -1073,17 +1084,11 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
                                                        sc.hist);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
-      pick_digit_kernel<<<n_sel, 256, 0, s>>>(sc.state, sc.hist, pass, 0, 0u, 0ull);
-      count_launches(1);
-      if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     if (!a.keep_ties) {  // the ties' ranks are needed only where some of them are pruned
       // both return at once for selections whose ties with the threshold are all kept
       tie_count_kernel<<<grid, kThreads, 0, s>>>(a.acc, rows, a.Lk, period, n_kt, a.causal, diag, sc.state,
                                                  sc.tie_count);
-      count_launches(1);
-      if ((e = cudaGetLastError()) != cudaSuccess) return e;
-      tie_scan_kernel<<<n_sel, 1024, 0, s>>>(sc.tie_count, rows * n_kt, sc.state);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
