@@ -54,9 +54,10 @@ NCU_TRAFFIC = {
         "accumulate": {"bytes": 2.27e9,
                        "source": "ncu on the B=1 case (1.72 GB read + 0.50 GB written per launch: the accumulator, the bias "
                                  "and their traffic have no batch dimension) plus Q and K of three more samples"},
-        "build_mask": {"bytes": 1.39e9,
-                       "source": "ncu on the full workload: collecting pass 542 MB read + 31 MB written, emit pass "
-                                 "541 MB read + 278 MB written; the call's other kernels move a few MB"},
+        "build_mask": {"bytes": 1.04e9,
+                       "source": "ncu on the B=1 case (the accumulator and the mask have no batch dimension): the "
+                                 "classifying pass 541 MB read + 304 MB written, the passes over the collected entries "
+                                 "3 x 35 MB read, the patch pass 58 MB read + 13 MB written, the pivots' sample 17 MB read"},
     },
 }
 

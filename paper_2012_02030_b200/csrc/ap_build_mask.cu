@@ -67,6 +67,9 @@ struct SelectState {  // per selection
   uint32_t cand_select;          // the bracket holds the threshold: the passes over the collected keys run
   uint32_t thr_count;            // entries equal to the threshold key
   uint32_t tie_n;                // entries gathered in the tie list
+  // the classifying pass and the patch pass have written this selection's mask and tile bitmaps: the
+  // emit pass has nothing left to do for it
+  uint32_t emitted;
   // CTAs of the running kernel that have finished their share of this selection: the last one goes on
   // with the step that needs all of them (digit pick, tie scan, finish) and puts the count back to zero
   uint32_t ticket;
@@ -154,6 +157,7 @@ __global__ void init_state_kernel(SelectState *state, uint32_t *hist, int n_sel,
     state[idx].cand_select = 0u;
     state[idx].thr_count = 0u;
     state[idx].tie_n = 0u;
+    state[idx].emitted = 0u;
     state[idx].ticket = 0u;
   }
 }
@@ -594,7 +598,8 @@ __device__ void rank_ties(const uint32_t *tie_idx, uint32_t count, uint32_t rank
 // enough; the CTA that finishes last then turns the digits found among the collected keys into the
 // threshold, ranks those ties (the lowest linear indices are kept) and marks the selection as done.
 __global__ void __launch_bounds__(kThreads) cand_finish_kernel(SelectState *state, const uint2 *__restrict__ cand,
-                                                               uint32_t cand_cap, uint32_t *tie_list) {
+                                                               uint32_t cand_cap, uint32_t *tie_list,
+                                                               int classified) {
   __shared__ uint32_t tie_idx[kMaxCutTies];
   __shared__ uint32_t cut_s;
   const int h = blockIdx.y;
@@ -625,6 +630,9 @@ __global__ void __launch_bounds__(kThreads) cand_finish_kernel(SelectState *stat
     state[h].thr = st.prefix + st.lo;
     state[h].prefix = st.prefix + st.lo;
     state[h].done = 1u;
+    // with the classifying pass before it, the patch pass can finish the mask unless the ties would
+    // have to be ranked by their counts per row segment
+    state[h].emitted = (classified && (st.all_ties_kept || rank_them)) ? 1u : 0u;
   }
 }
 
@@ -653,6 +661,7 @@ __global__ void __launch_bounds__(1024) select_small_kernel(const float *__restr
   st.prefix = 0u, st.thr = 0xffffffffu, st.remaining = k_rest, st.ties_kept = 0ull, st.all_ties_kept = 0u;
   st.done = 1u, st.lo = 0u, st.hi = 0xffffffffu, st.above_hi = 0ull, st.n_cand = 0u, st.use_shortcut = 0u;
   st.tie_cut = 0u, st.have_cut = 0u, st.cand_select = 0u, st.thr_count = 0u, st.tie_n = 0u, st.ticket = 0u;
+  st.emitted = 0u;
   if (k_rest == 0ull) {  // nothing but the forced entries is kept
     if (threadIdx.x == 0) state[h] = st;
     return;
@@ -795,9 +804,44 @@ __global__ void __launch_bounds__(kThreads) tie_count_kernel(const float *__rest
   }
 }
 
+// A warp's way into a selection's buffer of collected entries: staged in shared memory and appended
+// with one reservation per flush (an entry that finds the stage full goes straight to the buffer).
+struct Collector {
+  uint2 *stage;        // this warp's kWarpStage entries of shared memory
+  uint32_t *stage_n;   // entries pushed since the last flush (may run past the stage)
+  uint2 *out;          // the selection's buffer
+  uint32_t *n_cand;    // entries reserved in it so far (may exceed the capacity: then the shortcut fails)
+  uint32_t cap;
+  __device__ __forceinline__ void push(float f, uint32_t index) {
+    const uint2 entry = make_uint2(key_of(f), index);
+    const uint32_t pos = atomicAdd(stage_n, 1u);
+    if (pos < (uint32_t)kWarpStage) {
+      stage[pos] = entry;
+    } else {
+      const uint32_t g = atomicAdd(n_cand, 1u);
+      if (g < cap) out[g] = entry;
+    }
+  }
+  __device__ __forceinline__ void flush(uint32_t at_least, int lane) {  // by the whole warp
+    __syncwarp();
+    const uint32_t n = min(*stage_n, (uint32_t)kWarpStage);
+    if (n >= at_least && n > 0u) {
+      uint32_t dst = 0u;
+      if (lane == 0) dst = atomicAdd(n_cand, n);
+      dst = __shfl_sync(0xffffffffu, dst, 0);
+      for (uint32_t e = lane; e < n; e += 32)
+        if (dst + e < cap) out[dst + e] = stage[e];
+      __syncwarp();
+      if (lane == 0) *stage_n = 0u;
+      __syncwarp();
+    }
+  }
+};
+
 // What the emit pass needs of a selection.
 struct EmitSel {
   float thr_f;  // the threshold as a float (NaN when nothing but the forced entries is kept)
+  float lo_f;   // classifying pass: thr_f is the bracket's upper pivot, lo_f its lower one
   unsigned long long ties_kept;
   bool all_ties, have_cut;
   uint32_t tie_cut;
@@ -807,11 +851,14 @@ struct EmitSel {
 // The rows of one tile; returns this lane's share of the tile's popcount (lanes 0, 8, 16, 24).
 // kInterior: every row and column of the tile exists and lies in the domain and none is forced,
 // so nothing is checked per entry.
-template <bool kInterior>
+// kClassify: the classifying pass of the one-pass shortcut instead of the emit pass proper.  Entries
+// above the bracket are kept, entries inside it are collected (col) and left out for the patch pass
+// to decide, entries above the bracket are counted (above).
+template <bool kInterior, bool kClassify>
 __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int Lq, int Lk, int n_kt, int h, int qt,
                                               int kt, int tile, int causal, int diag, const EmitSel &sel,
                                               const uint32_t *__restrict__ tie_prefix, uint8_t *__restrict__ mask,
-                                              uint32_t *__restrict__ stage_bitmap) {
+                                              uint32_t *__restrict__ stage_bitmap, Collector &col, uint32_t &above) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const bool vec = (Lk & 3) == 0;
   const int j0 = kt * kTile + 4 * lane;
@@ -841,13 +888,16 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
       uint32_t nib = 0u;
       if (kInterior || i < Lq) {  // warp-uniform
         uint32_t tie_bits = 0u, gt_bits = 0u;
+        // the lowest value that needs a closer look: the threshold, or the bracket's lower pivot
+        const float floor_f = kClassify ? sel.lo_f : thr_f;
+        uint32_t forced_bits = 0u;
         if (kInterior) {
-          // (most pieces of a row lie wholly below the threshold: one test instead of eight)
-          if (!(v[u][0] < thr_f && v[u][1] < thr_f && v[u][2] < thr_f && v[u][3] < thr_f)) {
+          // (most pieces of a row lie wholly below it: one test instead of eight)
+          if (!(v[u][0] < floor_f && v[u][1] < floor_f && v[u][2] < floor_f && v[u][3] < floor_f)) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
               gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
-              tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
+              tie_bits |= ((kClassify ? !(v[u][c] < floor_f) && !(v[u][c] > thr_f) : v[u][c] == thr_f) ? 1u : 0u) << c;
             }
           }
         } else {
@@ -857,16 +907,24 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
             const int j = j0 + c;
             if (j < jend) {
               if (diag && j == i + off) {
-                gt_bits |= 1u << c;
+                forced_bits |= 1u << c;
               } else {
                 gt_bits |= (v[u][c] > thr_f ? 1u : 0u) << c;
-                tie_bits |= (v[u][c] == thr_f ? 1u : 0u) << c;
+                tie_bits |= ((kClassify ? !(v[u][c] < floor_f) && !(v[u][c] > thr_f) : v[u][c] == thr_f) ? 1u : 0u) << c;
               }
             }
           }
         }
-        nib = gt_bits;
-        if (sel.all_ties) {
+        nib = gt_bits | forced_bits;
+        if (kClassify) {
+          above += (uint32_t)__popc(gt_bits);
+          if (tie_bits) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              if (tie_bits & (1u << c))
+                col.push(v[u][c], (sel.first_row + (uint32_t)i) * (uint32_t)Lk + (uint32_t)(j0 + c));
+          }
+        } else if (sel.all_ties) {
           nib |= tie_bits;
         } else if (sel.have_cut) {
           if (tie_bits) {
@@ -917,7 +975,9 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
         if (stage_bitmap) stage_bitmap[(size_t)tile * kBitmapWords + 4 * r + (lane >> 3)] = w;
       }
     }
+    if (kClassify) col.flush(kWarpStage / 2, lane);
   }
+  if (kClassify) col.flush(1u, lane);
   return count;
 }
 
@@ -928,18 +988,28 @@ __device__ __forceinline__ int emit_tile_rows(const float *__restrict__ acc, int
 // all heads share selection 0, ties are ordered by (h*Lq + i)*Lk + j, and the
 // tiles' popcounts are added up into nnz[h].  keep_ties: every entry equal to the threshold is
 // kept (no ranking), and the popcounts are added up as well (the count is not known beforehand).
+// kClassify: the shortcut's one pass over the accumulator, which does the collecting pass's work
+// (entries above the upper pivot counted, entries inside the bracket appended to the selection's
+// buffer) and most of the emit pass's at once: everything above the bracket is kept, everything else
+// left out, and patch_kernel adds the collected entries that turn out to be kept.  Only for exact
+// per-head selections (the kept count is known beforehand, nothing is counted here).
+template <bool kClassify>
 __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc, int Lq, int Lk, int n_qt, int n_kt,
                                                    int causal, int diag, int per_layer, int keep_ties,
-                                                   const SelectState *__restrict__ state,
-                                                   const uint32_t *__restrict__ tie_prefix,
+                                                   SelectState *state, const uint32_t *__restrict__ tie_prefix,
                                                    uint8_t *__restrict__ mask, uint32_t *__restrict__ stage_bitmap,
-                                                   int32_t *__restrict__ stage_count, int64_t *__restrict__ nnz) {
+                                                   int32_t *__restrict__ stage_count, int64_t *__restrict__ nnz,
+                                                   uint2 *__restrict__ cand, uint32_t cand_cap) {
   const int tile = blockIdx.x;
   const int kt = tile % n_kt;
   const int qt = (tile / n_kt) % n_qt;
   const int h = tile / (n_kt * n_qt);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ int warp_count[4];
+  __shared__ uint2 stage_all[kClassify ? 4 : 1][kClassify ? kWarpStage : 1];
+  __shared__ uint32_t stage_n_all[4];
+  SelectState &st = state[per_layer ? 0 : h];
+  if (kClassify ? !st.use_shortcut : st.emitted != 0u) return;  // not this pass's selection
   // own positions of the tile's rows among the keys: columns own_lo .. own_hi
   const int own_lo = qt * kTile + ((causal || diag) ? Lk - Lq : 0), own_hi = own_lo + kTile - 1;
   if (causal && kt * kTile > own_hi) {
@@ -963,30 +1033,80 @@ __global__ void __launch_bounds__(128) emit_kernel(const float *__restrict__ acc
     if (stage_count && threadIdx.x == 0) stage_count[tile] = 0;
     return;
   }
-  const SelectState &st = state[per_layer ? 0 : h];
   EmitSel sel;
-  sel.thr_f = float_of_key(st.thr);
+  sel.thr_f = float_of_key(kClassify ? st.hi : st.thr);
+  sel.lo_f = float_of_key(st.lo);
   sel.ties_kept = st.ties_kept;
   sel.all_ties = st.all_ties_kept != 0u || keep_ties != 0;
   sel.have_cut = st.have_cut != 0u;
   sel.tie_cut = st.tie_cut;
   sel.first_row = per_layer ? (uint32_t)h * (uint32_t)Lq : 0u;
+  Collector col;
+  col.stage = stage_all[kClassify ? warp : 0];
+  col.stage_n = &stage_n_all[warp];
+  col.out = cand + (size_t)(per_layer ? 0 : h) * cand_cap;
+  col.n_cand = &st.n_cand;
+  col.cap = cand_cap;
+  if (lane == 0) stage_n_all[warp] = 0u;
+  __syncwarp();
+  uint32_t above = 0u;
   const bool below = !causal || kt * kTile + kTile - 1 <= own_lo;  // every column in every row's domain
   const bool has_diag = diag && own_lo <= kt * kTile + kTile - 1 && own_hi >= kt * kTile;
   const bool interior = (qt + 1) * kTile <= Lq && (kt + 1) * kTile <= Lk && (Lk & 3) == 0 && below && !has_diag;
-  int count = interior ? emit_tile_rows<true>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel, tie_prefix, mask,
-                                              stage_bitmap)
-                       : emit_tile_rows<false>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel, tie_prefix, mask,
-                                               stage_bitmap);
+  int count = interior ? emit_tile_rows<true, kClassify>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel,
+                                                         tie_prefix, mask, stage_bitmap, col, above)
+                       : emit_tile_rows<false, kClassify>(acc, Lq, Lk, n_kt, h, qt, kt, tile, causal, diag, sel,
+                                                          tie_prefix, mask, stage_bitmap, col, above);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xffffffffu, count, o);
+  if (kClassify) {
+    above = __reduce_add_sync(0xffffffffu, above);
+    if (lane == 0 && above) atomicAdd(&st.above_hi, (unsigned long long)above);
+  }
   if (lane == 0) warp_count[warp] = count;
   __syncthreads();
   if (threadIdx.x == 0) {
     const int total = warp_count[0] + warp_count[1] + warp_count[2] + warp_count[3];
     if (stage_count) stage_count[tile] = total;
-    if ((per_layer || keep_ties) && nnz && total)
+    if (!kClassify && (per_layer || keep_ties) && nnz && total)
       atomicAdd(reinterpret_cast<unsigned long long *>(nnz + h), (unsigned long long)total);
+  }
+}
+
+// The collected entries of a selection that the classifying pass left out and that are kept after all:
+// above the threshold, or equal to it and within the ties that are kept.  grid = (CTAs, selections).
+__global__ void __launch_bounds__(kThreads) patch_kernel(const SelectState *__restrict__ state,
+                                                         const uint2 *__restrict__ cand, uint32_t cand_cap, int Lq,
+                                                         int Lk, int n_qt, int n_kt, uint8_t *__restrict__ mask,
+                                                         uint32_t *__restrict__ stage_bitmap,
+                                                         int32_t *__restrict__ stage_count) {
+  const int h = blockIdx.y;
+  const SelectState st = state[h];
+  if (!st.emitted) return;
+  const uint2 *mine = cand + (size_t)h * cand_cap;
+  const int lane = threadIdx.x & 31;
+  const uint32_t n = st.n_cand;
+  // (warp-uniform trip count; entries that follow one another in the buffer were collected by one warp
+  // from one stretch of a tile, so lanes that hit the same bitmap word or tile combine their updates)
+  for (uint32_t base = blockIdx.x * kThreads; base < n; base += gridDim.x * kThreads) {
+    const uint32_t idx = base + threadIdx.x;
+    uint2 c = make_uint2(0u, 0u);
+    if (idx < n) c = mine[idx];
+    const bool keep = idx < n && (c.x > st.thr || (c.x == st.thr && (st.all_ties_kept != 0u || c.y <= st.tie_cut)));
+    const uint32_t i = c.y / (uint32_t)Lk, j = c.y - i * (uint32_t)Lk;
+    if (keep && mask) mask[((size_t)h * Lq + i) * Lk + j] = 1;
+    if (stage_bitmap) {
+      const uint32_t tile = (uint32_t)((h * n_qt + (int)(i >> 7)) * n_kt + (int)(j >> 7));
+      const uint32_t word = tile * (uint32_t)kBitmapWords + 4u * (i & 127u) + ((j & 127u) >> 5);
+      const unsigned voters = __ballot_sync(0xffffffffu, keep);
+      if (keep) {
+        const unsigned same_word = __match_any_sync(voters, word);
+        const uint32_t all_bits = __reduce_or_sync(same_word, 1u << (j & 31u));
+        if (lane == __ffs((int)same_word) - 1) atomicOr(stage_bitmap + word, all_bits);
+        const unsigned same_tile = __match_any_sync(voters, tile);
+        if (lane == __ffs((int)same_tile) - 1) atomicAdd(stage_count + tile, __popc(same_tile));
+      }
+    }
   }
 }
 
@@ -1037,9 +1157,9 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
                                                  count_nnz ? 0ll : (long long)a.k, a.nnz);
       count_launches(1);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
-      emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer,
-                                                    a.keep_ties, sc.state, sc.tie_count, a.mask, a.stage_bitmap,
-                                                    a.stage_count, a.nnz);
+      emit_kernel<false><<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag,
+                                                           a.per_layer, a.keep_ties, sc.state, sc.tie_count, a.mask,
+                                                           a.stage_bitmap, a.stage_count, a.nnz, nullptr, 0u);
       count_launches(1);
       return cudaGetLastError();
     }
@@ -1064,19 +1184,36 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
       if (e != cudaSuccess) return e;
       sample_pivots_kernel<<<dim3(n_sel, 2), 1024, smem, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
                                                      (unsigned long long)a.k_rest, (unsigned long long)n_rest, sc.state);
-      // one wave of CTAs (five fit an SM), so that no SM idles while a second, partial wave runs
-      int collect_blocks = ceil_div(rows, kWarps);
-      if (collect_blocks > 148 * 5 / n_sel) collect_blocks = max(148 * 5 / n_sel, 1);
-      collect_kernel<<<dim3(collect_blocks, n_sel), kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
-                                                                     sc.state, sc.cand, (uint32_t)cap);
+      // Exact per-head selections: the one pass over the accumulator also writes what is certain of the
+      // mask and the tile bitmaps (the patch pass below adds the collected entries that are kept), so
+      // the emit pass at the end has nothing to read for the selections the shortcut resolves.  Other
+      // selections count what they keep in the emit pass, which therefore has to see every entry.
+      const bool classify = !a.per_layer && !a.keep_ties;
+      if (classify) {
+        emit_kernel<true><<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, 0, 0,
+                                                            sc.state, sc.tie_count, a.mask, a.stage_bitmap,
+                                                            a.stage_count, a.nnz, sc.cand, (uint32_t)cap);
+      } else {
+        // one wave of CTAs (five fit an SM), so that no SM idles while a second, partial wave runs
+        int collect_blocks = ceil_div(rows, kWarps);
+        if (collect_blocks > 148 * 5 / n_sel) collect_blocks = max(148 * 5 / n_sel, 1);
+        collect_kernel<<<dim3(collect_blocks, n_sel), kThreads, 0, s>>>(a.acc, rows, a.Lk, period, a.causal, diag,
+                                                                       sc.state, sc.cand, (uint32_t)cap);
+      }
       // the threshold among the collected keys: the same three digits, on offsets from the lower pivot
       const dim3 cand_grid(ceil_div(148 * 8, n_sel), n_sel);
       for (int pass = 0; pass < kPasses; ++pass) {
         cand_histogram_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap,
                                                              (unsigned long long)a.k_rest, pass, sc.hist);
       }
-      cand_finish_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, sc.tie_list);
+      cand_finish_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, sc.tie_list,
+                                                        classify ? 1 : 0);
       count_launches(3 + kPasses);
+      if (classify) {
+        patch_kernel<<<cand_grid, kThreads, 0, s>>>(sc.state, sc.cand, (uint32_t)cap, a.Lq, a.Lk, n_qt, n_kt, a.mask,
+                                                    a.stage_bitmap, a.stage_count);
+        count_launches(1);
+      }
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     for (int pass = 0; pass < kPasses; ++pass) {
@@ -1093,9 +1230,9 @@ cudaError_t launch_build_mask(const BuildMaskArgs &a, cudaStream_t s) {
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
   }
-  emit_kernel<<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer,
-                                                a.keep_ties, sc.state,
-                                                sc.tie_count, a.mask, a.stage_bitmap, a.stage_count, a.nnz);
+  emit_kernel<false><<<a.H * n_qt * n_kt, 128, 0, s>>>(a.acc, a.Lq, a.Lk, n_qt, n_kt, a.causal, diag, a.per_layer,
+                                                       a.keep_ties, sc.state, sc.tie_count, a.mask, a.stage_bitmap,
+                                                       a.stage_count, a.nnz, nullptr, 0u);
   count_launches(1);
   return cudaGetLastError();
 }
