@@ -164,13 +164,20 @@ __global__ void __launch_bounds__(128) gather_tiles_kernel(const uint32_t *__res
 }
 
 // One CTA per grid tile, thread r = tile row r: writes the list of the full
-// (optionally causal) domain in closed form.
+// (optionally causal) domain in closed form, rounds included: in such a list only the last tile of
+// a list row can have fewer than eight non-empty groups (the others lie inside the domain of the
+// tile's last row), and its groups are the first ones of the tile, so round k of a list row is its
+// k-th tile - same key rows, same bitmap.
 __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk, int n_qt, int n_kt, int causal,
                                                           int cap, int32_t *__restrict__ row_ptr,
                                                           int32_t *__restrict__ col_idx,
                                                           uint8_t *__restrict__ flags,
                                                           uint32_t *__restrict__ bitmap,
-                                                          uint8_t *__restrict__ groups, unsigned *err) {
+                                                          uint8_t *__restrict__ groups,
+                                                          int32_t *__restrict__ round_ptr,
+                                                          int32_t *__restrict__ round_rows,
+                                                          uint8_t *__restrict__ round_info,
+                                                          uint32_t *__restrict__ round_bitmap, unsigned *err) {
   const int tile = blockIdx.x;
   const int kt = tile % n_kt;
   const int qt = (tile / n_kt) % n_qt;
@@ -178,9 +185,9 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
   const int per_head = (int)dense_row_start(n_qt, n_kt, Lq, Lk, causal);
   const int row_start = h * per_head + (int)dense_row_start(qt, n_kt, Lq, Lk, causal);
   if (threadIdx.x == 0 && kt == 0) {
-    row_ptr[h * n_qt + qt] = min(row_start, cap);
+    row_ptr[h * n_qt + qt] = round_ptr[h * n_qt + qt] = min(row_start, cap);
     if (h == H - 1 && qt == n_qt - 1) {
-      row_ptr[H * n_qt] = min(H * per_head, cap);
+      row_ptr[H * n_qt] = round_ptr[H * n_qt] = min(H * per_head, cap);
       if (H * per_head > cap) atomicOr(err, kDevErrCapacity);
     }
   }
@@ -201,13 +208,17 @@ __global__ void __launch_bounds__(128) dense_tiles_kernel(int H, int Lq, int Lk,
     }
   }
   reinterpret_cast<uint4 *>(bitmap + (size_t)pos * kBitmapWords)[r] = make_uint4(w[0], w[1], w[2], w[3]);
+  reinterpret_cast<uint4 *>(round_bitmap + (size_t)pos * kBitmapWords)[r] = make_uint4(w[0], w[1], w[2], w[3]);
   const int full = __syncthreads_and(w[0] == 0xffffffffu && w[1] == 0xffffffffu &&
                                      w[2] == 0xffffffffu && w[3] == 0xffffffffu);
   const uint32_t gm = group_mask_of_tile(make_uint4(w[0], w[1], w[2], w[3]));
+  const int ng = __popc(gm);  // the tile's first ng groups
+  if (r < 8) round_rows[(size_t)pos * 8 + r] = r < ng ? kt * kTile + 16 * r : -1;
   if (r == 0) {
     col_idx[pos] = kt;
     flags[pos] = full ? 1 : 0;
     groups[pos] = (uint8_t)gm;
+    round_info[pos] = (uint8_t)(ng | ((full && ng == 8) ? 0x80 : 0));
   }
 }
 
@@ -590,11 +601,16 @@ cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
   unsigned *err = device_error_word();
   if (!err) return cudaErrorUnknown;
   dense_tiles_kernel<<<t.H * t.n_qt * t.n_kt, 128, 0, s>>>(t.H, t.Lq, t.Lk, t.n_qt, t.n_kt, causal, t.cap,
-                                                         t.row_ptr, t.col_idx, t.flags, t.bitmap, t.groups, err);
+                                                         t.row_ptr, t.col_idx, t.flags, t.bitmap, t.groups,
+                                                         t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, err);
   count_launches(1);
   const cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  return launch_build_rounds(t, s, false);
+  if (e != cudaSuccess || !t.ground_ptr) return e;
+  // no gathered schedule for a dense list
+  const int n_rows = t.H * t.n_qt;
+  clear_grounds_kernel<<<ceil_div(n_rows + 1, 256), 256, 0, s>>>(t.ground_ptr, n_rows + 1);
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 }  // namespace ap
