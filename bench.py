@@ -319,8 +319,13 @@ def density_section(ap, w, acc, q, k, v, out, ws, dense_ms, dense_tiles, peaks, 
     schedule holds, speedup over the dense list, fractions of the burst bf16 peak."""
     rows = []
     tiles = ap.Tiles(w.H, w.Lq, w.Lk, device=dev)
+    paired = ap.Tiles(w.H, w.Lq, w.Lk, device=dev, paired=True)  # units of work balanced by the list's builder
     nnz = torch.zeros((w.H,), dtype=torch.int64, device=dev)
     for keep in (0.10, 0.05, 0.02):
+        ap.ap_build_mask(acc, keep, w.causal, w.keep_diag, None, paired, nnz, ws)
+        for _ in range(3):
+            ap.ap_sparse_attention_fwd(q, k, v, paired, out)
+        ms_paired = _time_back_to_back(lambda i: ap.ap_sparse_attention_fwd(q, k, v, paired, out), 10)
         ap.ap_build_mask(acc, keep, w.causal, w.keep_diag, None, tiles, nnz, ws)
         for _ in range(3):
             ap.ap_sparse_attention_fwd(q, k, v, tiles, out)
@@ -330,7 +335,8 @@ def density_section(ap, w, acc, q, k, v, out, ws, dense_ms, dense_tiles, peaks, 
         n_tiles = tiles.n_tiles()
         kept = int(nnz.sum().item())
         rows.append({
-            "keep_frac": keep, "kept_entries_per_head": kept // w.H, "fwd_ms": ms, "tiles": n_tiles, "rounds": n_rounds,
+            "keep_frac": keep, "kept_entries_per_head": kept // w.H, "fwd_ms": ms,
+            "fwd_ms_with_balanced_units": ms_paired, "tiles": n_tiles, "rounds": n_rounds,
             "slots": slots, "speedup_vs_dense_path": dense_ms / ms,
             "effective_tflops": metrics.effective_flops(kept, w.B, w.d) / (ms * 1e-3) / 1e12,
             "frac_of_bf16_burst_on_kept_tile_flops": metrics.tile_flops(n_tiles, w.B, w.d) / (ms * 1e-3) / 1e12 / peaks["bf16"],

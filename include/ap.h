@@ -117,6 +117,15 @@ typedef enum { AP_F32 = 0, AP_BF16 = 1, AP_F16 = 2 } ap_dtype; /* AP_F16: IEEE h
  *                               that many 16-column slots); bit 7: 128 columns, all kept
  *   ground_bitmap[cap][128][4]  bit p of the 128-bit row r: query row r keeps column p
  *                               of the round; 0 for unused columns
+ * Work units: optional (null: the forward pairs query tile n_qt-1-j with query tile j).
+ *   unit_qt[H][ceil(n_qt/2)][2]  the two query tiles of each unit of work of a head; every query
+ *                               tile of the head appears exactly once, the second entry of at most
+ *                               one unit is -1 (odd n_qt).  The builders pair the list row with the
+ *                               most rounds with the one with the fewest, the second with the
+ *                               second fewest, and so on (ties by lower index first), so that a
+ *                               head's units weigh about the same; ap_sparse_attention_fwd hands
+ *                               whole units to its thread blocks.
+ *
  * ap_sparse_attention_fwd follows the gathered rounds of a list row that has some (a
  * slot of 16 keys that follow one another from a multiple of 8 on is fetched as one box,
  * the rows of other slots one by one), the rounds otherwise; the result is the same
@@ -141,6 +150,7 @@ typedef struct ap_tiles {
   int32_t *ground_keys;
   uint8_t *ground_info;
   uint32_t *ground_bitmap;
+  int32_t *unit_qt;
 } ap_tiles;
 
 /* Library version (major*10000 + minor*100 + patch). */

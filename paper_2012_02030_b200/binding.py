@@ -37,7 +37,7 @@ class ap_tiles(ctypes.Structure):
         ("round_ptr", ctypes.c_void_p), ("round_rows", ctypes.c_void_p), ("round_info", ctypes.c_void_p),
         ("round_bitmap", ctypes.c_void_p),
         ("ground_ptr", ctypes.c_void_p), ("ground_keys", ctypes.c_void_p), ("ground_info", ctypes.c_void_p),
-        ("ground_bitmap", ctypes.c_void_p),
+        ("ground_bitmap", ctypes.c_void_p), ("unit_qt", ctypes.c_void_p),
     ]
 
 
@@ -162,7 +162,8 @@ def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
 class Tiles:
     """Device buffers of a tile list plus the ap_tiles descriptor that points at them."""
 
-    def __init__(self, H: int, Lq: int, Lk: int, device="cuda", cap: int | None = None, gathered: bool = False):
+    def __init__(self, H: int, Lq: int, Lk: int, device="cuda", cap: int | None = None, gathered: bool = False,
+                 paired: bool = False):
         self.H, self.Lq, self.Lk = H, Lq, Lk
         self.n_qt, self.n_kt = -(-Lq // TILE), -(-Lk // TILE)
         self.cap = ap_tiles_capacity(H, Lq, Lk) if cap is None else cap
@@ -186,10 +187,13 @@ class Tiles:
             self.ground_bitmap = torch.zeros((max(self.cap, 1), TILE, 4), dtype=torch.int32, device=device)
             g = [self.ground_ptr.data_ptr(), self.ground_keys.data_ptr(), self.ground_info.data_ptr(),
                  self.ground_bitmap.data_ptr()]
+        # the forward's units of work: pairs of query tiles of a head, balanced by the builders
+        self.unit_qt = torch.zeros((H, (self.n_qt + 1) // 2, 2), dtype=torch.int32, device=device) if paired else None
         self.c = ap_tiles(H, Lq, Lk, self.n_qt, self.n_kt, self.cap, self.row_ptr.data_ptr(),
                           self.col_idx.data_ptr(), self.flags.data_ptr(), self.bitmap.data_ptr(),
                           self.groups.data_ptr(), self.round_ptr.data_ptr(), self.round_rows.data_ptr(),
-                          self.round_info.data_ptr(), self.round_bitmap.data_ptr(), *g)
+                          self.round_info.data_ptr(), self.round_bitmap.data_ptr(), *g,
+                          self.unit_qt.data_ptr() if paired else None)
 
     def n_tiles(self) -> int:
         """Number of stored tiles (synchronises)."""

@@ -42,6 +42,7 @@ inline ap_status check_tiles(const ap_tiles *t, int H, int Lq, int Lk, bool shap
   if (n_g != 0 && n_g != 4) return AP_ERR_INVALID_ARG;
   if (n_g == 4 && (misaligned(t->ground_bitmap, 15u) || misaligned(t->ground_keys, 15u) || misaligned(t->ground_ptr, 3u)))
     return AP_ERR_INVALID_ARG;
+  if (t->unit_qt && misaligned(t->unit_qt, 7u)) return AP_ERR_INVALID_ARG;
   if (t->cap < 1) return AP_ERR_WORKSPACE;
   if (shape_must_match) {
     if (t->H != H || t->Lq != Lq || t->Lk != Lk || t->n_qt != ceil_div(Lq, kTile) ||

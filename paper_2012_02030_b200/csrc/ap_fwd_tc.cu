@@ -110,6 +110,7 @@ struct Gathered {
   const uint16_t *K, *V;  // the tensors themselves: single key rows are fetched with plain asynchronous copies
   int Lk;
   int mode;
+  const int32_t *unit_qt;  // [H][ceil(n_qt/2)][2]: the query tiles of each unit of work (kPairs)
 };
 
 struct Shared {
@@ -185,8 +186,9 @@ __device__ __forceinline__ float2 unpack16x2(uint32_t pk) {
 }
 
 // kGath: the launch may follow gathered rounds (a second instantiation, so that the code for them
-// costs lists without a gathered schedule nothing).
-template <int D, bool kSplit, bool kF16, bool kGath>
+// costs lists without a gathered schedule nothing).  kPairs: the units of work are the pairs of query
+// tiles the list's builder chose (balanced by their rounds) instead of (n_qt - 1 - j, j).
+template <int D, bool kSplit, bool kF16, bool kGath, bool kPairs>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
               const int32_t *__restrict__ round_ptr, const int32_t *__restrict__ round_rows,
@@ -271,19 +273,38 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
     // instruction stream is what short items wait for)
     int cur_u = (int)blockIdx.x, cur_j = cur_u % n_half, cur_bh = cur_u / n_half, cur_h = cur_bh % H;
     const int step_j = item_step % n_half, step_bh = item_step / n_half, step_h = step_bh % H;
+    auto next_unit = [&](int &u, int &j, int &bh, int &h) {
+      u += item_step;
+      j += step_j;
+      bh += step_bh;
+      h += step_h;
+      if (j >= n_half) {
+        j -= n_half;
+        ++bh;
+        ++h;
+      }
+      if (h >= H) h -= H;
+    };
+    // kPairs: a unit's two query tiles come from the list's table, fetched one unit ahead of their use
+    // (the address of the rounds' offsets depends on them)
+    uint2 cur_pair = make_uint2(0u, 0u), ahead_pair = make_uint2(0u, 0u);
+    auto fetch_pair_after = [&]() {  // the pair of the unit after the current one
+      int u = cur_u, j = cur_j, bh = cur_bh, h = cur_h;
+      next_unit(u, j, bh, h);
+      if (u < n_units) ahead_pair = ldg_now_v2(gth.unit_qt + ((size_t)h * n_half + j) * 2);
+    };
+    if constexpr (kPairs) {
+      if (cur_u < n_units) cur_pair = ldg_now_v2(gth.unit_qt + ((size_t)cur_h * n_half + cur_j) * 2);
+      fetch_pair_after();
+    }
     auto item_ref = [&](int t) {
       ItemRef it;
       if (t >= 2 && !(t & 1)) {  // the next unit
-        cur_u += item_step;
-        cur_j += step_j;
-        cur_bh += step_bh;
-        cur_h += step_h;
-        if (cur_j >= n_half) {
-          cur_j -= n_half;
-          ++cur_bh;
-          ++cur_h;
+        next_unit(cur_u, cur_j, cur_bh, cur_h);
+        if constexpr (kPairs) {
+          cur_pair = ahead_pair;
+          fetch_pair_after();
         }
-        if (cur_h >= H) cur_h -= H;
       }
       const int u = cur_u;
       it.in_range = u < n_units;
@@ -291,8 +312,15 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
       if (it.in_range) {
         const int j = cur_j;
         it.bh = cur_bh;
-        it.qt = (t & 1) ? j : n_qt - 1 - j;
-        if (!(t & 1) || j != n_qt - 1 - j) {
+        bool there = !(t & 1) || j != n_qt - 1 - j;
+        if constexpr (kPairs) {
+          it.qt = (t & 1) ? (int)cur_pair.y : (int)cur_pair.x;
+          there = it.qt >= 0;
+          if (!there) it.qt = 0;
+        } else {
+          it.qt = (t & 1) ? j : n_qt - 1 - j;
+        }
+        if (there) {
           const int lr = cur_h * n_qt + it.qt;
           it.rho0 = (int)ldg_now_u32(round_ptr + lr);
           it.rho1 = (int)ldg_now_u32(round_ptr + lr + 1);
@@ -868,14 +896,14 @@ fwd_tc_kernel(const __grid_constant__ FwdMaps maps, uint16_t *__restrict__ O,
   if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
-template <int D, bool kSplit, bool kF16, bool kGath>
+template <int D, bool kSplit, bool kF16, bool kGath, bool kPairs>
 cudaError_t launch_kernel(const FwdMaps &maps, const void *K, const void *V, void *O, const ap_tiles &t, int B, int H,
                           int Lq, int Lk, const DebugKnobs &dbg, float scale, unsigned *err, cudaStream_t s) {
   using C = Cfg<D, kSplit>;
   static_assert(sizeof(Shared) <= 18 * 1024, "shared bookkeeping outgrew its reservation");
   static_assert(C::kStages <= kMaxStages, "ring deeper than its barriers");
   static_assert(C::kSmemBytes > 114 * 1024 && C::kSmemBytes <= 227 * 1024, "one CTA per SM, within the limit");
-  auto kern = fwd_tc_kernel<D, kSplit, kF16, kGath>;
+  auto kern = fwd_tc_kernel<D, kSplit, kF16, kGath, kPairs>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
   if (e != cudaSuccess) return e;
   const int sms = sm_count();
@@ -883,7 +911,7 @@ cudaError_t launch_kernel(const FwdMaps &maps, const void *K, const void *V, voi
   const int n_units = B * H * ((t.n_qt + 1) / 2);  // pairs of query tiles, see the producer
   const float scale_log2 = scale * 1.4426950408889634f;
   Gathered gth = {nullptr, nullptr, nullptr, nullptr, static_cast<const uint16_t *>(K), static_cast<const uint16_t *>(V),
-                  Lk, dbg.schedule};
+                  Lk, dbg.schedule, kPairs ? t.unit_qt : nullptr};
   if (kGath) gth.ptr = t.ground_ptr, gth.keys = t.ground_keys, gth.info = t.ground_info, gth.bitmap = t.ground_bitmap;
   // the test hook runs on one CTA only (a tiny grid is all it is meant for)
   kern<<<dbg.skip_arrive ? 1 : (n_units < sms ? n_units : sms), kThreads, C::kSmemBytes, s>>>(
@@ -899,8 +927,10 @@ cudaError_t launch(const FwdMaps &maps, const void *K, const void *V, void *O, c
                    int Lk, bool, float scale, unsigned *err, cudaStream_t s) {
   const DebugKnobs dbg = debug_knobs();
   if (t.ground_ptr != nullptr && dbg.schedule != 1)
-    return launch_kernel<D, kSplit, kF16, true>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
-  return launch_kernel<D, kSplit, kF16, false>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
+    return launch_kernel<D, kSplit, kF16, true, false>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
+  if (t.unit_qt != nullptr && !dbg.skip_arrive)
+    return launch_kernel<D, kSplit, kF16, false, true>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
+  return launch_kernel<D, kSplit, kF16, false, false>(maps, K, V, O, t, B, H, Lq, Lk, dbg, scale, err, s);
 }
 
 }  // namespace

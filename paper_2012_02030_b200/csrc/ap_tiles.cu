@@ -535,6 +535,41 @@ __global__ void __launch_bounds__(128) fill_grounds_kernel(const int32_t *__rest
   }
 }
 
+// ---- units of work of the forward: balanced pairs of a head's query tiles ------------------------
+
+// One CTA per head.  The head's list rows are ranked by their number of rounds (more first, ties by
+// lower index); unit j pairs rank j with rank n_qt - 1 - j.  Heads of more than kMaxPairTiles query
+// tiles keep the plain pairing (n_qt - 1 - j, j).
+constexpr int kMaxPairTiles = 2048;
+__global__ void __launch_bounds__(256) pair_units_kernel(const int32_t *__restrict__ round_ptr, int n_qt,
+                                                         int32_t *__restrict__ unit_qt) {
+  __shared__ int32_t rounds[kMaxPairTiles];
+  __shared__ int32_t sorted[kMaxPairTiles];
+  const int h = blockIdx.x, n_half = (n_qt + 1) / 2;
+  int32_t *out = unit_qt + (size_t)h * n_half * 2;
+  if (n_qt > kMaxPairTiles) {
+    for (int j = threadIdx.x; j < n_half; j += blockDim.x) {
+      out[2 * j] = n_qt - 1 - j;
+      out[2 * j + 1] = j != n_qt - 1 - j ? j : -1;
+    }
+    return;
+  }
+  for (int q = threadIdx.x; q < n_qt; q += blockDim.x)
+    rounds[q] = round_ptr[h * n_qt + q + 1] - round_ptr[h * n_qt + q];
+  __syncthreads();
+  for (int q = threadIdx.x; q < n_qt; q += blockDim.x) {
+    const int32_t mine = rounds[q];
+    int rank = 0;
+    for (int p = 0; p < n_qt; ++p) rank += (rounds[p] > mine || (rounds[p] == mine && p < q)) ? 1 : 0;
+    sorted[rank] = q;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < n_half; j += blockDim.x) {
+    out[2 * j] = sorted[j];
+    out[2 * j + 1] = j != n_qt - 1 - j ? sorted[n_qt - 1 - j] : -1;
+  }
+}
+
 // No gathered schedule (dense lists): every list row has zero gathered rounds.
 __global__ void clear_grounds_kernel(int32_t *__restrict__ ground_ptr, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -553,7 +588,13 @@ cudaError_t launch_build_rounds(const ap_tiles &t, cudaStream_t s, bool gathered
                                             t.round_rows, t.round_info, t.round_bitmap);
   count_launches(3);
   cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || !t.ground_ptr) return e;
+  if (e != cudaSuccess) return e;
+  if (t.unit_qt) {
+    pair_units_kernel<<<t.H, 256, 0, s>>>(t.round_ptr, t.n_qt, t.unit_qt);
+    count_launches(1);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  if (!t.ground_ptr) return e;
   if (!gathered) {
     clear_grounds_kernel<<<ceil_div(n_rows + 1, 256), 256, 0, s>>>(t.ground_ptr, n_rows + 1);
     count_launches(1);
@@ -604,8 +645,14 @@ cudaError_t launch_dense_tiles(const ap_tiles &t, int causal, cudaStream_t s) {
                                                          t.row_ptr, t.col_idx, t.flags, t.bitmap, t.groups,
                                                          t.round_ptr, t.round_rows, t.round_info, t.round_bitmap, err);
   count_launches(1);
-  const cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || !t.ground_ptr) return e;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (t.unit_qt) {
+    pair_units_kernel<<<t.H, 256, 0, s>>>(t.round_ptr, t.n_qt, t.unit_qt);
+    count_launches(1);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  if (!t.ground_ptr) return e;
   // no gathered schedule for a dense list
   const int n_rows = t.H * t.n_qt;
   clear_grounds_kernel<<<ceil_div(n_rows + 1, 256), 256, 0, s>>>(t.ground_ptr, n_rows + 1);

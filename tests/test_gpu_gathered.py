@@ -130,3 +130,39 @@ def test_list_without_gathered_arrays_is_unchanged():
     ha, hb = a.to_host(), b.to_host()
     for key in ha:
         assert np.array_equal(ha[key], hb[key]), key
+
+
+@pytest.mark.parametrize("H,Lq,Lk,d,causal", [(2, 1024, 1024, 128, True), (3, 640, 900, 64, False), (1, 128, 128, 64, True)])
+def test_balanced_units_table_and_forward(H, Lq, Lk, d, causal):
+    """The optional table of work units: every query tile of a head exactly once, the list row with the
+    most rounds paired with the one with the fewest; and the forward under it."""
+    from paper_2012_02030_b200 import binding as ap
+
+    mask = _masks("mixed", H, Lq, Lk, causal)
+    tiles = ap.Tiles(H, Lq, Lk, paired=True)
+    ap.ap_mask_to_tiles(mask.cuda(), tiles)
+    n_qt, n_half = tiles.n_qt, (tiles.n_qt + 1) // 2
+    units = tiles.unit_qt.cpu().numpy()
+    rounds = np.diff(tiles.round_ptr.cpu().numpy()).reshape(H, n_qt)
+    for h in range(H):
+        order = sorted(range(n_qt), key=lambda qq: (-rounds[h, qq], qq))
+        want = [[order[j], order[n_qt - 1 - j] if j != n_qt - 1 - j else -1] for j in range(n_half)]
+        assert units[h].tolist() == want
+    gen = torch.Generator().manual_seed(5)
+    B = 2
+    q = torch.randn((B, H, Lq, d), generator=gen).to(torch.bfloat16)
+    k, v = (torch.randn((B, H, Lk, d), generator=gen).to(torch.bfloat16) for _ in range(2))
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), mask.numpy())
+    out = torch.full_like(q, float("nan")).cuda()
+    ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), tiles, out)
+    assert ap.ap_device_status() == ap.AP_OK
+    assert_close_attention(out, ref, "bf16", "balanced units")
+    dense = ap.Tiles(H, Lq, Lk, paired=True)
+    ap.ap_dense_tiles(dense, causal=causal)
+    full = np.ones((H, Lq, Lk), dtype=np.uint8)
+    if causal:
+        full = np.tril(full, Lk - Lq)
+    ref = orc.attention_fwd(inputs.widen(q), inputs.widen(k), inputs.widen(v), full)
+    out.fill_(float("nan"))
+    ap.ap_sparse_attention_fwd(q.cuda(), k.cuda(), v.cuda(), dense, out)
+    assert_close_attention(out, ref, "bf16", "balanced units, dense list")
