@@ -84,7 +84,7 @@ class ClockSampler:
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int, period_s: float = 0.004):
+    def __init__(self, gpu_index: int, period_s: float = 0.001):
         import threading
 
         vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
