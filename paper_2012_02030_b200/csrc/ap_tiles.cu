@@ -69,8 +69,18 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
   for (int base = 0; base < n_tiles; base += 1024 * kPer) {
     const int idx0 = base + (int)threadIdx.x * kPer;
     int cnt[kPer];
+    const bool vec = idx0 + kPer <= n_tiles && (reinterpret_cast<uintptr_t>(stage_count) & 15u) == 0 &&
+                     (reinterpret_cast<uintptr_t>(stage_pos) & 15u) == 0;
+    if (vec) {  // four 16-byte loads instead of sixteen strided 4-byte ones
 #pragma unroll
-    for (int e = 0; e < kPer; ++e) cnt[e] = idx0 + e < n_tiles ? stage_count[idx0 + e] : 0;
+      for (int q = 0; q < kPer / 4; ++q) {
+        const int4 c4 = reinterpret_cast<const int4 *>(stage_count + idx0)[q];
+        cnt[4 * q] = c4.x, cnt[4 * q + 1] = c4.y, cnt[4 * q + 2] = c4.z, cnt[4 * q + 3] = c4.w;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) cnt[e] = idx0 + e < n_tiles ? stage_count[idx0 + e] : 0;
+    }
     int mine = 0;
 #pragma unroll
     for (int e = 0; e < kPer; ++e) mine += cnt[e] > 0 ? 1 : 0;
@@ -95,12 +105,14 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
     const int carry = carry_s;
     int before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - mine;
     int row = idx0 / n_kt, kt = idx0 - row * n_kt;  // list row and key tile of the tile, stepped below
+    int pos[kPer];
 #pragma unroll
     for (int e = 0; e < kPer; ++e) {
       const int idx = idx0 + e;
       const int flag = cnt[e] > 0 ? 1 : 0;
+      pos[e] = flag ? before : -1;
       if (idx < n_tiles) {
-        stage_pos[idx] = flag ? before : -1;
+        if (!vec) stage_pos[idx] = pos[e];
         if (kt == n_kt - 1) row_ptr[row + 1] = min(before + flag, cap);
       }
       before += flag;
@@ -108,6 +120,11 @@ __global__ void __launch_bounds__(1024) scan_tiles_kernel(const int32_t *__restr
         kt = 0;
         ++row;
       }
+    }
+    if (vec) {
+#pragma unroll
+      for (int q = 0; q < kPer / 4; ++q)
+        reinterpret_cast<int4 *>(stage_pos + idx0)[q] = make_int4(pos[4 * q], pos[4 * q + 1], pos[4 * q + 2], pos[4 * q + 3]);
     }
     __syncthreads();
     if (threadIdx.x == 1023) carry_s = carry + warp_sums[31];
